@@ -1,0 +1,299 @@
+"""Benchmark of the E2-TTT chunk-parallel fast-weight update on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config I]
+
+A step is one pass of the whole hot path (e2ttt_chunk_fwd over every chunk of every sequence) on one
+batch of seeded synthetic inputs.  Default workload: the 1.3B-layer shape (B=4, H=16, d=128, h=512,
+L=4096, C=64, bf16 I/O, GELU-MLP fast weights), forward.  One JSON line is printed by rank 0.
+
+  value     layer tokens/s (B*L per call / device time), inputs resident in HBM
+  e2e       the same metric through the C ABI with HOST buffers: pinned-host -> device copies of all
+            inputs and device -> host copies of all results inside the timed region
+  roofline  for the forward kernel: algorithmic GEMM flop per launch / CUDA-event time per launch
+            against the measured bf16 dense peak of this machine (MEASURED_PEAKS.json)
+  cpu_baseline  the fp64 oracle, as it stands, timed on the host cores over a bounded sample
+
+`--impl reference` times the oracle itself (there is no other reference implementation of this path).
+With N > 1 (torchrun) every rank runs the same workload on its own seeded batch: the path shards over
+(batch, head) with no exchange, so scaling is weak and the only collectives are the timing barrier and
+a MAX over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2608_21308_b200 import inputs  # noqa: E402
+
+METRIC = "e2ttt_layer_fwd_tokens_per_s"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram__bytes_read.sum + dram__bytes_write.sum per forward launch from the committed ncu capture
+# (profiles/): set once a capture of the current kernel exists, else null.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["_source"] = "measured"
+        return p
+    return dict(FALLBACK_PEAKS, _source="fallback")
+
+
+def flops_per_token_head(r: inputs.Recipe, backward: bool = False) -> float:
+    """GEMM flop the method needs per token and head: 9 (MLP) or 13 (SwiGLU) products of 2*d*h forward,
+    23 more units for the reverse pass (5 of them recomputed forward products)."""
+    units = 9 if r.kind == inputs.KIND_MLP else 13
+    f = units * 2.0 * r.d * r.h
+    if backward:
+        f += 23 * 2.0 * r.d * r.h
+    return f
+
+
+def bytes_per_call(r: inputs.Recipe) -> float:
+    s = 2 if r.io == "bf16" else 4
+    nm = len(inputs.mat_shapes(r.kind, r.d, r.h))
+    n = r.B * r.H
+    return n * r.L * (4 * r.d * s + 12) + n * 4 * nm * r.d * r.h * 4
+
+
+class ClockSampler:
+    """nvidia-smi sampled every 200 ms while the timed region runs (read-only queries)."""
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={q}", "--format=csv,noheader,nounits", "-lms", "200"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for row in self.rows:
+            try:
+                sm.append(float(row[0]))
+                mx.append(float(row[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, val in zip(names, row[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def cpu_oracle_rate(r: inputs.Recipe, budget_heads: int | None = None, tokens: int = 512):
+    """Time the oracle (untouched) on a bounded sample: `cores` heads x `tokens` tokens of the workload."""
+    from oracle import oracle
+    cores = oracle.max_threads()
+    n_heads = budget_heads or max(cores, 1)
+    rs = inputs.Recipe(**{**r.__dict__, "L": min(tokens, r.L), "heads": list(range(min(n_heads, r.B * r.H)))})
+    x = inputs.generate(rs)
+    t0 = time.perf_counter()
+    oracle.forward(x["q"], x["k"], x["v"], x["eta"], x["beta"], x["gamma"], x["W"], None, r.C, r.kind, threads=cores)
+    dt = time.perf_counter() - t0
+    token_heads = len(rs.heads) * rs.L
+    return {"value": token_heads / r.H / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{len(rs.heads)} heads x {rs.L} tokens of the workload, fp64, forward; "
+                      f"layer tokens/s = token-heads/s / H", "seconds": dt}
+
+
+def run_reference(args, r):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals = []
+    for i in range(args.warmup + args.steps):
+        res = cpu_oracle_rate(r, tokens=256)
+        if i >= args.warmup:
+            vals.append(res)
+    dt = float(np.mean([v["seconds"] for v in vals]))
+    value = float(np.mean([v["value"] for v in vals]))
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(r),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": vals[0]["cores"], "kind": "oracle",
+                             "sample": vals[0]["sample"]},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def workload_config(r):
+    kind = "mlp_gelu" if r.kind == inputs.KIND_MLP else "swiglu"
+    return {"workload": f"e2ttt_chunk_fwd B={r.B} H={r.H} L={r.L} d={r.d} h={r.h} C={r.C} {kind} {r.io} I/O",
+            "B": r.B, "H": r.H, "L": r.L, "d": r.d, "h": r.h, "C": r.C, "kind": kind, "io": r.io,
+            "gates": "eta=0.1*sigmoid(N(0,1)), beta=sigmoid(N(1,1)), gamma=1-eta*sigmoid(N(3,1))", "seed": r.seed,
+            "l2": "inputs larger than L2: q,k,v,o and states of one call exceed 126 MB"}
+
+
+def run_ours(args, r):
+    import torch
+    import torch.distributed as dist
+    from paper_2608_21308_b200 import binding as E
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+
+    rr = inputs.Recipe(**{**r.__dict__, "seed": r.seed + rank})
+    x = inputs.generate(rr)
+    N = r.B * r.H
+    iod = torch.float32 if r.io == "f32" else torch.bfloat16
+    p = E.make_params(r.B, r.H, r.L, r.d, r.h, r.C, r.kind, E.E2TTT_F32 if r.io == "f32" else E.E2TTT_BF16, 1e-5,
+                      E.E2TTT_IMPL_AUTO)
+    s4, s3 = (r.B, r.H, r.L, r.d), (r.B, r.H, r.L)
+    shapes = inputs.mat_shapes(r.kind, r.d, r.h)
+    host = {n: torch.from_numpy(x[n]).to(iod).view(s4).pin_memory() for n in ("q", "k", "v")}
+    host.update({n: torch.from_numpy(x[n]).view(s3).pin_memory() for n in ("eta", "beta", "gamma")})
+    hostW = [torch.from_numpy(w).view((r.B, r.H) + s).pin_memory() for w, s in zip(x["W"], shapes)]
+    devt = {n: t.to(dev) for n, t in host.items()}
+    W0 = [w.to(dev) for w in hostW]
+    o = torch.empty(s4, dtype=iod, device=dev)
+    Wf = [torch.empty_like(w) for w in W0]
+    Mf = [torch.empty_like(w) for w in W0]
+    ws = torch.empty(E.e2ttt_workspace_bytes(p, 0), dtype=torch.uint8, device=dev)
+    host_o = torch.empty(s4, dtype=iod).pin_memory()
+    host_Wf = [torch.empty_like(w).pin_memory() for w in hostW]
+    host_Mf = [torch.empty_like(w).pin_memory() for w in hostW]
+    stream = torch.cuda.current_stream()
+
+    def step():
+        E.e2ttt_chunk_fwd(p, devt["q"], devt["k"], devt["v"], devt["eta"], devt["beta"], devt["gamma"], W0, None, o,
+                          Wf, Mf, ws, 0, stream)
+
+    def step_e2e():
+        for n in host:
+            devt[n].copy_(host[n], non_blocking=True)
+        for wd, wh in zip(W0, hostW):
+            wd.copy_(wh, non_blocking=True)
+        step()
+        host_o.copy_(o, non_blocking=True)
+        for a, b in zip(host_Wf, Wf):
+            a.copy_(b, non_blocking=True)
+        for a, b in zip(host_Mf, Mf):
+            a.copy_(b, non_blocking=True)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps, warmup):
+        for _ in range(warmup):
+            fn()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            fn()
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1) / steps
+        if world > 1:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ms = timed(step, args.steps, args.warmup)
+    clocks = sampler.stop() if rank == 0 else None
+    ms_e2e = timed(step_e2e, max(2, args.steps // 2), 1)
+
+    if rank == 0:
+        pk = peaks()
+        tokens = r.B * r.L
+        flop = flops_per_token_head(r) * N * r.L
+        t_tc = flop / (pk["bf16_tflops"] * 1e12)
+        t_hbm = bytes_per_call(r) / (pk["hbm_gbs"] * 1e9)
+        bound = "tensor" if t_tc >= t_hbm else "hbm"
+        if bound == "tensor":
+            achieved, peak, unit = flop / (ms * 1e-3) / 1e12, pk["bf16_tflops"], "TFLOP/s"
+        else:
+            achieved, peak, unit = bytes_per_call(r) / (ms * 1e-3) / 1e9, pk["hbm_gbs"], "GB/s"
+        h2d = sum(t.numel() * t.element_size() for t in host.values()) + sum(w.numel() * 4 for w in hostW)
+        d2h = host_o.numel() * host_o.element_size() + 2 * sum(w.numel() * 4 for w in hostW)
+        line = {
+            "metric": METRIC, "value": world * tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if r.io == "bf16" else "f64",
+            "data": "synthetic", "config": workload_config(r),
+            "e2e": {"value": world * tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
+            "gpu_launches": args.steps,
+            "clocks": clocks,
+            "roofline": {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
+                         "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "peak_source": pk["_source"],
+                         "kernel": "forward kernel (one launch per step)",
+                         "flop_per_launch": flop, "bytes_per_launch": bytes_per_call(r),
+                         "frac_of_sustained_peak": (flop / (ms * 1e-3) / 1e12) / pk["bf16_tflops_sustained"]},
+        }
+        if world == 1 and not args.no_cpu:
+            line["cpu_baseline"] = {k: v for k, v in cpu_oracle_rate(r).items() if k != "seconds"}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, help="benchmark configuration index (default: the 1.3B-layer shape)")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    r = inputs.config(args.config)
+    if args.impl == "reference":
+        run_reference(args, r)
+    else:
+        run_ours(args, r)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,160 @@
+/*
+ * e2ttt.h - C ABI of the E2-TTT chunk-parallel fast-weight update for NVIDIA B200 (sm_100a).
+ *
+ * What is computed (paper: "Rethinking Expressivity and Efficiency in Test-Time Training").
+ * For each of the B*H independent sequences, the L tokens are cut into chunks of C tokens.  A
+ * chunk starts from the fast-weight state W_0 and momentum state M_0 left by the previous chunk
+ * (Section 3, "Primal Formulation") and
+ *   - emits the outputs o_t = f_{W_0}(q_t) from the chunk-start weights (Eq. "chunkwise_output",
+ *     Algorithm 1 line 1);
+ *   - takes the per-token negative gradients G_t = -grad_W 1/2 ||f_{W_0}(k_t) - v_t||^2 at the
+ *     chunk-start weights with one inner forward/backward over the whole chunk (Algorithm 1
+ *     lines 1 and 3, Appendix "Single Backward Pass for Both Aggregates");
+ *   - forms the scalar kernels K^W_t, K^M_t and the three carries from the per-token gates with
+ *     suffix scans (Eq. "scalar_aux", Algorithm 1 line 2);
+ *   - jumps to the chunk-end states with Proposition 1 (Eq. "Mc_closed", "Wc_closed"; Algorithm 1
+ *     lines 4-7):
+ *         M_C = bt_0 M_0 + sum_t K^M_t G_t
+ *         W_C = gt_0 W_0 + bt_0 R_1 M_0 + sum_t K^W_t G_t
+ *     which equal the result of the token-wise recurrence  M_t = beta_t M_{t-1} + eta_t G_t,
+ *     W_t = gamma_t W_{t-1} + M_t  (Eq. "tokenwise_ttt_decay_momentum").
+ * Fast-weight networks (Section 4, "Fast-weight Network"):
+ *     E2TTT_MLP_GELU : f_W(x) = x + LN(W2 GELU(W1 x)),               W1 [h,d], W2 [d,h]
+ *     E2TTT_SWIGLU   : f_W(x) = x + LN(W3 (SiLU(W1 x) * (W2 x))),    W1 [h,d], W2 [h,d], W3 [d,h]
+ * LN is a layer norm over the d outputs without affine parameters (biased variance, ln_eps inside
+ * the square root); GELU is the exact erf form.  All matrices of the collection share the same
+ * per-token scalars (Section 2: "W_t denotes the full collection of fast-weight tensors").
+ *
+ * Conventions for every entry point
+ *   - All data pointers are DEVICE pointers unless the comment says "host".  Pointer tables
+ *     (W_init and friends) are HOST arrays of e2ttt_num_matrices(kind) device pointers.
+ *   - Tensors are dense and row-major.  q, k, v, o and their gradients: [B, H, L, d] in
+ *     io_dtype.  Gates and gate gradients: [B, H, L] fp32.  Fast-weight / momentum matrices and
+ *     their gradients: [B, H, rows, cols] fp32.
+ *   - The caller owns every buffer.  The library allocates nothing and keeps no state between
+ *     calls other than cached kernel attributes.  Work is enqueued on `stream` (a cudaStream_t
+ *     passed as void*, NULL = the default stream); no entry point synchronises with the host.
+ *   - Return value: E2TTT_OK (0) or a negative e2ttt_status.  Arguments are validated before
+ *     anything is launched, so a failing call leaves every output untouched.  Nothing throws,
+ *     aborts or prints.
+ *   - Final-state buffers may alias the initial-state buffers (in-place state update).  No other
+ *     output may overlap an input or another output.
+ */
+#ifndef E2TTT_H
+#define E2TTT_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define E2TTT_API __attribute__((visibility("default")))
+#else
+#define E2TTT_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { E2TTT_MLP_GELU = 0, E2TTT_SWIGLU = 1 } e2ttt_kind;
+typedef enum { E2TTT_F32 = 0, E2TTT_BF16 = 1 } e2ttt_dtype;
+
+/* Which kernel family serves the call.
+ *   AUTO    : the tensor-core path where a specialisation exists for (kind, io_dtype, d, h, C),
+ *             else the SIMT path.
+ *   SIMT    : plain CUDA-core kernels for any shape.  With fp32 I/O they compute in fp64
+ *             internally; with bf16 I/O in fp32.
+ *   TCGEN05 : bf16 operands on the 5th-generation tensor cores with fp32 accumulation in tensor
+ *             memory; E2TTT_ERR_SHAPE if no specialisation matches. */
+typedef enum { E2TTT_IMPL_AUTO = 0, E2TTT_IMPL_SIMT = 1, E2TTT_IMPL_TCGEN05 = 2 } e2ttt_impl;
+
+typedef enum {
+    E2TTT_OK = 0,
+    E2TTT_ERR_NULL = -1,      /* a required pointer is NULL */
+    E2TTT_ERR_SHAPE = -2,     /* non-positive dimension, C > 128, d or h beyond the compiled limits,
+                                 L not a multiple of C on a path that needs it, unknown kind */
+    E2TTT_ERR_DTYPE = -3,     /* unknown io_dtype / impl */
+    E2TTT_ERR_ALIGN = -4,     /* q, k, v, o (and gradients) must be 16-byte aligned */
+    E2TTT_ERR_WORKSPACE = -5, /* workspace NULL or smaller than e2ttt_workspace_bytes() */
+    E2TTT_ERR_ARCH = -6,      /* current device is not compute capability 10.x */
+    E2TTT_ERR_CUDA = -7,      /* the CUDA runtime refused a launch or attribute (no sync is done) */
+    E2TTT_ERR_TIMEOUT = -8    /* a bounded device-side wait gave up */
+} e2ttt_status;
+
+typedef struct {
+    int32_t B, H;     /* batch and heads: B*H independent sequences */
+    int32_t L;        /* tokens per sequence */
+    int32_t d;        /* head dimension (input and output width of the fast-weight network) */
+    int32_t h;        /* hidden width of the fast-weight network */
+    int32_t C;        /* chunk size, 1..128.  The SIMT path accepts a shorter last chunk. */
+    int32_t kind;     /* e2ttt_kind */
+    int32_t io_dtype; /* e2ttt_dtype of q, k, v, o, d_o, dq, dk, dv */
+    float ln_eps;     /* layer-norm epsilon (the paper gives none; 1e-5 is the usual default) */
+    int32_t impl;     /* e2ttt_impl */
+} e2ttt_params;
+
+/* Number of fast-weight matrices of a network kind (2 or 3); 0 for an unknown kind. */
+E2TTT_API int e2ttt_num_matrices(int kind);
+
+/* Rows and columns of matrix i (0-based) of the collection, Section 4 "Fast-weight Network".
+ * Returns E2TTT_ERR_SHAPE for a bad kind or index. */
+E2TTT_API int e2ttt_matrix_shape(int kind, int d, int h, int i, int* rows, int* cols);
+
+/* Bytes of caller-provided device workspace a call with these parameters needs.
+ * save_states != 0: the size for a forward that also records the chunk-start states, and for
+ * the backward that consumes them.  `bytes` is a host pointer. */
+E2TTT_API int e2ttt_workspace_bytes(const e2ttt_params* p, int save_states, size_t* bytes);
+
+/* Forward over all chunks of all sequences (Algorithm 1 applied chunk after chunk, Section 3.2).
+ *   q, k, v          in   [B,H,L,d] io_dtype
+ *   eta, beta, gamma in   [B,H,L] fp32: learning rate, momentum factor and decay factor of
+ *                         Eq. "tokenwise_ttt_decay_momentum" (the parameterisation that produces
+ *                         them, Section 4 "Input-Dependent Dynamics", is the caller's)
+ *   W_init           in   host table of device pointers, matrix i [B,H,rows_i,cols_i] fp32
+ *   M_init           in   same layout, or NULL for a zero initial momentum
+ *   o                out  [B,H,L,d] io_dtype
+ *   W_final, M_final out  host tables, same layout as W_init; may alias W_init / M_init
+ *   workspace        device scratch of at least e2ttt_workspace_bytes(p, save_states) bytes,
+ *                    256-byte aligned; with save_states != 0 it holds, after the call, the
+ *                    (W, M) at the start of every chunk for e2ttt_chunk_bwd
+ */
+E2TTT_API int e2ttt_chunk_fwd(const e2ttt_params* p,
+                    const void* q, const void* k, const void* v,
+                    const float* eta, const float* beta, const float* gamma,
+                    const float* const* W_init, const float* const* M_init,
+                    void* o, float* const* W_final, float* const* M_final,
+                    void* workspace, size_t workspace_bytes, int save_states, void* stream);
+
+/* Reverse pass of e2ttt_chunk_fwd: the adjoint of the same program (the outer-loop gradient the
+ * paper obtains by automatic differentiation, Appendix "Training Details": "plain PyTorch").
+ *   q .. M_init            in   as in the forward
+ *   d_o                    in   [B,H,L,d] io_dtype, gradient of the loss w.r.t. o
+ *   dW_final, dM_final     in   host tables (fp32, state layout) or NULL for zeros
+ *   dq, dk, dv             out  [B,H,L,d] io_dtype
+ *   d_eta, d_beta, d_gamma out  [B,H,L] fp32, gradients w.r.t. the three gates as independent inputs
+ *   dW_init, dM_init       out  host tables, state layout, fp32; may alias dW_final / dM_final
+ *   workspace              sized by e2ttt_workspace_bytes(p, 1)
+ *   states_saved           != 0: the workspace still holds the chunk-start states written by
+ *                          e2ttt_chunk_fwd(save_states=1) for the same inputs; 0: they are
+ *                          recomputed first
+ * Only E2TTT_MLP_GELU has a reverse pass; E2TTT_SWIGLU returns E2TTT_ERR_SHAPE.
+ */
+E2TTT_API int e2ttt_chunk_bwd(const e2ttt_params* p,
+                    const void* q, const void* k, const void* v,
+                    const float* eta, const float* beta, const float* gamma,
+                    const float* const* W_init, const float* const* M_init,
+                    const void* d_o, const float* const* dW_final, const float* const* dM_final,
+                    void* dq, void* dk, void* dv, float* d_eta, float* d_beta, float* d_gamma,
+                    float* const* dW_init, float* const* dM_init,
+                    void* workspace, size_t workspace_bytes, int states_saved, void* stream);
+
+/* Static description of a status code (never NULL). */
+E2TTT_API const char* e2ttt_status_string(int status);
+
+/* Library version, major*10000 + minor*100 + patch. */
+E2TTT_API int e2ttt_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* E2TTT_H */

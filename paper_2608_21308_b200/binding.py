@@ -1,0 +1,169 @@
+"""Thin ctypes binding of the C-ABI library (include/e2ttt.h): argument marshalling only.
+
+Every function has the name and the argument order of its C counterpart.  Tensors are torch CUDA
+tensors (torch is used for device memory and streams, nothing else); the binding checks dtype,
+contiguity and device, builds the host pointer tables and passes raw pointers.  There is no CPU
+path: a missing library or a failing call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "lib", "libe2ttt.so")
+
+E2TTT_MLP_GELU, E2TTT_SWIGLU = 0, 1
+E2TTT_F32, E2TTT_BF16 = 0, 1
+E2TTT_IMPL_AUTO, E2TTT_IMPL_SIMT, E2TTT_IMPL_TCGEN05 = 0, 1, 2
+E2TTT_OK = 0
+
+
+class e2ttt_params(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("L", ctypes.c_int32), ("d", ctypes.c_int32),
+                ("h", ctypes.c_int32), ("C", ctypes.c_int32), ("kind", ctypes.c_int32),
+                ("io_dtype", ctypes.c_int32), ("ln_eps", ctypes.c_float), ("impl", ctypes.c_int32)]
+
+
+class E2TTTError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {e2ttt_status_string(status)} ({status})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load the in-tree library; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} not found: build it with `python -m paper_2608_21308_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, cp = ctypes.c_void_p, ctypes.c_int
+        pp = ctypes.POINTER(e2ttt_params)
+        tab = ctypes.POINTER(ctypes.c_void_p)
+        L.e2ttt_num_matrices.argtypes = [cp]
+        L.e2ttt_matrix_shape.argtypes = [cp, cp, cp, cp, ctypes.POINTER(cp), ctypes.POINTER(cp)]
+        L.e2ttt_workspace_bytes.argtypes = [pp, cp, ctypes.POINTER(ctypes.c_size_t)]
+        L.e2ttt_chunk_fwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, tab, tab, vp, tab, tab, vp, ctypes.c_size_t, cp, vp]
+        L.e2ttt_chunk_bwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, tab, tab, vp, tab, tab, vp, vp, vp, vp, vp, vp,
+                                      tab, tab, vp, ctypes.c_size_t, cp, vp]
+        L.e2ttt_status_string.argtypes = [cp]
+        L.e2ttt_status_string.restype = ctypes.c_char_p
+        L.e2ttt_version.argtypes = []
+        for name in ("e2ttt_num_matrices", "e2ttt_matrix_shape", "e2ttt_workspace_bytes", "e2ttt_chunk_fwd",
+                     "e2ttt_chunk_bwd", "e2ttt_version"):
+            getattr(L, name).restype = cp
+        _lib = L
+    return _lib
+
+
+def e2ttt_status_string(status: int) -> str:
+    return lib().e2ttt_status_string(int(status)).decode()
+
+
+def e2ttt_version() -> int:
+    return int(lib().e2ttt_version())
+
+
+def e2ttt_num_matrices(kind: int) -> int:
+    return int(lib().e2ttt_num_matrices(int(kind)))
+
+
+def e2ttt_matrix_shape(kind: int, d: int, h: int, i: int):
+    r, c = ctypes.c_int(), ctypes.c_int()
+    st = lib().e2ttt_matrix_shape(kind, d, h, i, ctypes.byref(r), ctypes.byref(c))
+    if st != E2TTT_OK:
+        raise E2TTTError(st, "e2ttt_matrix_shape")
+    return r.value, c.value
+
+
+def e2ttt_workspace_bytes(p: e2ttt_params, save_states: int) -> int:
+    n = ctypes.c_size_t()
+    st = lib().e2ttt_workspace_bytes(ctypes.byref(p), int(save_states), ctypes.byref(n))
+    if st != E2TTT_OK:
+        raise E2TTTError(st, "e2ttt_workspace_bytes")
+    return int(n.value)
+
+
+def make_params(B, H, L, d, h, C, kind=E2TTT_MLP_GELU, io_dtype=E2TTT_F32, ln_eps=1e-5, impl=E2TTT_IMPL_AUTO):
+    return e2ttt_params(B, H, L, d, h, C, kind, io_dtype, ln_eps, impl)
+
+
+def _io_torch_dtype(p):
+    return torch.float32 if p.io_dtype == E2TTT_F32 else torch.bfloat16
+
+
+def _ptr(t, dtype, shape, name):
+    if t is None:
+        return None
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError(f"{name}: expected a CUDA tensor")
+    if t.dtype != dtype:
+        raise TypeError(f"{name}: expected dtype {dtype}, got {t.dtype}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name}: must be contiguous")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name}: expected shape {tuple(shape)}, got {tuple(t.shape)}")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _table(ts, p, name):
+    if ts is None:
+        return None
+    n = e2ttt_num_matrices(p.kind)
+    if len(ts) != n:
+        raise ValueError(f"{name}: expected {n} matrices")
+    arr = (ctypes.c_void_p * n)()
+    for i, t in enumerate(ts):
+        r, c = e2ttt_matrix_shape(p.kind, p.d, p.h, i)
+        arr[i] = _ptr(t, torch.float32, (p.B, p.H, r, c), f"{name}[{i}]")
+    return arr
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream if isinstance(stream, torch.cuda.Stream) else int(stream))
+
+
+def e2ttt_chunk_fwd(p, q, k, v, eta, beta, gamma, W_init, M_init, o, W_final, M_final, workspace,
+                    save_states=0, stream=None):
+    """int e2ttt_chunk_fwd(...) of include/e2ttt.h.  `workspace` is a uint8 CUDA tensor.  Raises on error."""
+    io = _io_torch_dtype(p)
+    s4, s3 = (p.B, p.H, p.L, p.d), (p.B, p.H, p.L)
+    st = lib().e2ttt_chunk_fwd(
+        ctypes.byref(p), _ptr(q, io, s4, "q"), _ptr(k, io, s4, "k"), _ptr(v, io, s4, "v"),
+        _ptr(eta, torch.float32, s3, "eta"), _ptr(beta, torch.float32, s3, "beta"),
+        _ptr(gamma, torch.float32, s3, "gamma"), _table(W_init, p, "W_init"), _table(M_init, p, "M_init"),
+        _ptr(o, io, s4, "o"), _table(W_final, p, "W_final"), _table(M_final, p, "M_final"),
+        _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel() if workspace is not None else 0,
+        int(save_states), _stream_ptr(stream))
+    if st != E2TTT_OK:
+        raise E2TTTError(st, "e2ttt_chunk_fwd")
+    return st
+
+
+def e2ttt_chunk_bwd(p, q, k, v, eta, beta, gamma, W_init, M_init, d_o, dW_final, dM_final, dq, dk, dv,
+                    d_eta, d_beta, d_gamma, dW_init, dM_init, workspace, states_saved=0, stream=None):
+    """int e2ttt_chunk_bwd(...) of include/e2ttt.h.  Raises on error."""
+    io = _io_torch_dtype(p)
+    s4, s3 = (p.B, p.H, p.L, p.d), (p.B, p.H, p.L)
+    f32 = torch.float32
+    st = lib().e2ttt_chunk_bwd(
+        ctypes.byref(p), _ptr(q, io, s4, "q"), _ptr(k, io, s4, "k"), _ptr(v, io, s4, "v"),
+        _ptr(eta, f32, s3, "eta"), _ptr(beta, f32, s3, "beta"), _ptr(gamma, f32, s3, "gamma"),
+        _table(W_init, p, "W_init"), _table(M_init, p, "M_init"), _ptr(d_o, io, s4, "d_o"),
+        _table(dW_final, p, "dW_final"), _table(dM_final, p, "dM_final"),
+        _ptr(dq, io, s4, "dq"), _ptr(dk, io, s4, "dk"), _ptr(dv, io, s4, "dv"),
+        _ptr(d_eta, f32, s3, "d_eta"), _ptr(d_beta, f32, s3, "d_beta"), _ptr(d_gamma, f32, s3, "d_gamma"),
+        _table(dW_init, p, "dW_init"), _table(dM_init, p, "dM_init"),
+        _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel() if workspace is not None else 0,
+        int(states_saved), _stream_ptr(stream))
+    if st != E2TTT_OK:
+        raise E2TTTError(st, "e2ttt_chunk_bwd")
+    return st

@@ -1,0 +1,219 @@
+// C ABI of the library: argument validation, workspace sizing, kernel-family dispatch.
+#include <cuda_runtime.h>
+
+#include "../../include/e2ttt.h"
+#include "simt_layout.h"
+
+using namespace e2ttt;
+
+namespace {
+
+constexpr int kMaxD = 1024;
+constexpr int kMaxH = 8192;
+constexpr int kMaxChunk = 128;
+
+int nmat_of(int kind) { return kind == E2TTT_MLP_GELU ? 2 : (kind == E2TTT_SWIGLU ? 3 : 0); }
+
+int check_params(const e2ttt_params* p) {
+    if (!p) return E2TTT_ERR_NULL;
+    if (p->kind != E2TTT_MLP_GELU && p->kind != E2TTT_SWIGLU) return E2TTT_ERR_SHAPE;
+    if (p->io_dtype != E2TTT_F32 && p->io_dtype != E2TTT_BF16) return E2TTT_ERR_DTYPE;
+    if (p->impl != E2TTT_IMPL_AUTO && p->impl != E2TTT_IMPL_SIMT && p->impl != E2TTT_IMPL_TCGEN05) return E2TTT_ERR_DTYPE;
+    if (p->B <= 0 || p->H <= 0 || p->L <= 0 || p->d <= 0 || p->h <= 0 || p->C <= 0) return E2TTT_ERR_SHAPE;
+    if (p->C > kMaxChunk || p->d > kMaxD || p->h > kMaxH) return E2TTT_ERR_SHAPE;
+    if ((int64_t)p->B * p->H > (int64_t)1 << 24) return E2TTT_ERR_SHAPE;
+    if (!(p->ln_eps >= 0.0f)) return E2TTT_ERR_SHAPE;
+    return E2TTT_OK;
+}
+
+// 1 = tensor-core specialisation exists for these parameters
+int has_tcgen05(const e2ttt_params*) { return 0; }
+
+int pick_impl(const e2ttt_params* p, int* impl) {
+    if (p->impl == E2TTT_IMPL_TCGEN05) {
+        if (!has_tcgen05(p)) return E2TTT_ERR_SHAPE;
+        *impl = E2TTT_IMPL_TCGEN05;
+    } else if (p->impl == E2TTT_IMPL_AUTO) {
+        *impl = has_tcgen05(p) ? E2TTT_IMPL_TCGEN05 : E2TTT_IMPL_SIMT;
+    } else {
+        *impl = E2TTT_IMPL_SIMT;
+    }
+    return E2TTT_OK;
+}
+
+size_t simt_bytes(const e2ttt_params* p, bool save_states, bool backward) {
+    const int nchunks = (p->L + p->C - 1) / p->C;
+    SimtLayout l = simt_layout(p->d, p->h, p->C, nmat_of(p->kind), nchunks, save_states, backward);
+    const size_t elem = (p->io_dtype == E2TTT_F32) ? sizeof(double) : sizeof(float);
+    return l.per_seq * elem * (size_t)p->B * p->H;
+}
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+int check_device() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return E2TTT_ERR_ARCH; }
+    static int cached_major[64];
+    static bool known[64];
+    int major = 0;
+    if (dev >= 0 && dev < 64 && known[dev]) {
+        major = cached_major[dev];
+    } else {
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return E2TTT_ERR_ARCH;
+        }
+        if (dev >= 0 && dev < 64) { cached_major[dev] = major; known[dev] = true; }
+    }
+    return major == 10 ? E2TTT_OK : E2TTT_ERR_ARCH;
+}
+
+}  // namespace
+
+extern "C" {
+
+int e2ttt_num_matrices(int kind) { return nmat_of(kind); }
+
+int e2ttt_matrix_shape(int kind, int d, int h, int i, int* rows, int* cols) {
+    const int n = nmat_of(kind);
+    if (n == 0 || i < 0 || i >= n || !rows || !cols) return E2TTT_ERR_SHAPE;
+    const bool last = (i == n - 1);
+    *rows = last ? d : h;
+    *cols = last ? h : d;
+    return E2TTT_OK;
+}
+
+int e2ttt_workspace_bytes(const e2ttt_params* p, int save_states, size_t* bytes) {
+    if (!bytes) return E2TTT_ERR_NULL;
+    int rc = check_params(p);
+    if (rc) return rc;
+    int impl = 0;
+    rc = pick_impl(p, &impl);
+    if (rc) return rc;
+    // with saved states the same buffer serves the backward, which needs the larger layout
+    *bytes = simt_bytes(p, save_states != 0, save_states != 0);
+    return E2TTT_OK;
+}
+
+int e2ttt_chunk_fwd(const e2ttt_params* p, const void* q, const void* k, const void* v, const float* eta,
+                    const float* beta, const float* gamma, const float* const* W_init, const float* const* M_init,
+                    void* o, float* const* W_final, float* const* M_final, void* workspace, size_t workspace_bytes,
+                    int save_states, void* stream) {
+    int rc = check_params(p);
+    if (rc) return rc;
+    if (!q || !k || !v || !eta || !beta || !gamma || !W_init || !o || !W_final || !M_final) return E2TTT_ERR_NULL;
+    const int nmat = nmat_of(p->kind);
+    for (int i = 0; i < nmat; ++i) {
+        if (!W_init[i] || !W_final[i] || !M_final[i]) return E2TTT_ERR_NULL;
+        if (M_init && !M_init[i]) return E2TTT_ERR_NULL;
+    }
+    int impl = 0;
+    rc = pick_impl(p, &impl);
+    if (rc) return rc;
+    if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(o, 16)) return E2TTT_ERR_ALIGN;
+    size_t need = 0;
+    rc = e2ttt_workspace_bytes(p, save_states, &need);
+    if (rc) return rc;
+    if (!workspace || workspace_bytes < need) return E2TTT_ERR_WORKSPACE;
+    if (!aligned(workspace, 256)) return E2TTT_ERR_ALIGN;
+    rc = check_device();
+    if (rc) return rc;
+
+    SimtFwdArgs a{};
+    a.N = p->B * p->H; a.L = p->L; a.d = p->d; a.h = p->h; a.C = p->C;
+    a.nchunks = (p->L + p->C - 1) / p->C;
+    a.save_states = save_states != 0;
+    a.eps = p->ln_eps;
+    a.q = q; a.k = k; a.v = v; a.eta = eta; a.beta = beta; a.gamma = gamma; a.o = o; a.ws = workspace;
+    for (int i = 0; i < nmat; ++i) {
+        a.W_init[i] = W_init[i];
+        a.M_init[i] = M_init ? M_init[i] : nullptr;
+        a.W_final[i] = W_final[i];
+        a.M_final[i] = M_final[i];
+    }
+    a.lay = simt_layout(p->d, p->h, p->C, nmat, a.nchunks, a.save_states, a.save_states);
+    return simt_fwd_launch(a, p->kind, p->io_dtype, stream) == 0 ? E2TTT_OK : E2TTT_ERR_CUDA;
+}
+
+int e2ttt_chunk_bwd(const e2ttt_params* p, const void* q, const void* k, const void* v, const float* eta,
+                    const float* beta, const float* gamma, const float* const* W_init, const float* const* M_init,
+                    const void* d_o, const float* const* dW_final, const float* const* dM_final, void* dq, void* dk,
+                    void* dv, float* d_eta, float* d_beta, float* d_gamma, float* const* dW_init,
+                    float* const* dM_init, void* workspace, size_t workspace_bytes, int states_saved, void* stream) {
+    int rc = check_params(p);
+    if (rc) return rc;
+    if (p->kind != E2TTT_MLP_GELU) return E2TTT_ERR_SHAPE;
+    if (!q || !k || !v || !eta || !beta || !gamma || !W_init || !d_o || !dq || !dk || !dv || !d_eta || !d_beta ||
+        !d_gamma || !dW_init || !dM_init)
+        return E2TTT_ERR_NULL;
+    const int nmat = nmat_of(p->kind);
+    for (int i = 0; i < nmat; ++i) {
+        if (!W_init[i] || !dW_init[i] || !dM_init[i]) return E2TTT_ERR_NULL;
+        if (M_init && !M_init[i]) return E2TTT_ERR_NULL;
+        if (dW_final && !dW_final[i]) return E2TTT_ERR_NULL;
+        if (dM_final && !dM_final[i]) return E2TTT_ERR_NULL;
+    }
+    int impl = 0;
+    rc = pick_impl(p, &impl);
+    if (rc) return rc;
+    if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(d_o, 16) || !aligned(dq, 16) ||
+        !aligned(dk, 16) || !aligned(dv, 16))
+        return E2TTT_ERR_ALIGN;
+    size_t need = 0;
+    rc = e2ttt_workspace_bytes(p, 1, &need);
+    if (rc) return rc;
+    if (!workspace || workspace_bytes < need) return E2TTT_ERR_WORKSPACE;
+    if (!aligned(workspace, 256)) return E2TTT_ERR_ALIGN;
+    rc = check_device();
+    if (rc) return rc;
+
+    const int nchunks = (p->L + p->C - 1) / p->C;
+    const SimtLayout lay = simt_layout(p->d, p->h, p->C, nmat, nchunks, true, true);
+    if (!states_saved) {
+        // recompute the chunk-start states: a forward whose outputs and final states land in scratch slots
+        // that the reverse sweep overwrites later (the adjoint carries T, S and the accumulators Wb)
+        SimtFwdArgs f{};
+        f.N = p->B * p->H; f.L = p->L; f.d = p->d; f.h = p->h; f.C = p->C; f.nchunks = nchunks;
+        f.save_states = 1; f.eps = p->ln_eps;
+        f.q = q; f.k = k; f.v = v; f.eta = eta; f.beta = beta; f.gamma = gamma; f.ws = workspace; f.lay = lay;
+        f.o = nullptr; // outputs are not needed
+        for (int i = 0; i < nmat; ++i) {
+            f.W_init[i] = W_init[i];
+            f.M_init[i] = M_init ? M_init[i] : nullptr;
+            f.W_final[i] = nullptr;
+            f.M_final[i] = nullptr;
+        }
+        if (simt_fwd_launch(f, p->kind, p->io_dtype, stream) != 0) return E2TTT_ERR_CUDA;
+    }
+    SimtBwdArgs b{};
+    b.N = p->B * p->H; b.L = p->L; b.d = p->d; b.h = p->h; b.C = p->C; b.nchunks = nchunks; b.eps = p->ln_eps;
+    b.q = q; b.k = k; b.v = v; b.d_o = d_o; b.eta = eta; b.beta = beta; b.gamma = gamma;
+    b.dq = dq; b.dk = dk; b.dv = dv; b.d_eta = d_eta; b.d_beta = d_beta; b.d_gamma = d_gamma;
+    b.ws = workspace; b.lay = lay;
+    for (int i = 0; i < nmat; ++i) {
+        b.dW_final[i] = dW_final ? dW_final[i] : nullptr;
+        b.dM_final[i] = dM_final ? dM_final[i] : nullptr;
+        b.dW_init[i] = dW_init[i];
+        b.dM_init[i] = dM_init[i];
+    }
+    return simt_bwd_launch(b, p->kind, p->io_dtype, stream) == 0 ? E2TTT_OK : E2TTT_ERR_CUDA;
+}
+
+const char* e2ttt_status_string(int status) {
+    switch (status) {
+        case E2TTT_OK: return "ok";
+        case E2TTT_ERR_NULL: return "a required pointer is NULL";
+        case E2TTT_ERR_SHAPE: return "unsupported shape, kind or chunk size";
+        case E2TTT_ERR_DTYPE: return "unknown io_dtype or impl";
+        case E2TTT_ERR_ALIGN: return "a buffer is not aligned as required";
+        case E2TTT_ERR_WORKSPACE: return "workspace missing or too small";
+        case E2TTT_ERR_ARCH: return "current device is not compute capability 10.x (B200)";
+        case E2TTT_ERR_CUDA: return "the CUDA runtime reported an error at launch";
+        case E2TTT_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+        default: return "unknown status";
+    }
+}
+
+int e2ttt_version(void) { return 100; }
+
+}  // extern "C"

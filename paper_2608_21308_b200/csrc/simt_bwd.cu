@@ -1,0 +1,371 @@
+// SIMT backward (GELU-MLP fast weights): the adjoint of the chunk program, chunks in reverse order,
+// one CTA per sequence.  Per chunk it re-runs the chunk's forward from the saved chunk-start state, then
+// reverses, in matrix form over the whole chunk,
+//   (i)   the outputs o = f_{W0}(q),
+//   (ii)  the closed-form state transition of Proposition 1 (carries cw, cm, cb and kernels K^W, K^M),
+//   (iii) the per-token gradients G_t(W0, k_t, v_t) - a second-order pass through LN and GELU,
+//   (iv)  the suffix scans that made the scalar kernels.
+// Notation: T, S = adjoints of the chunk-end (W, M); a trailing "b" marks an adjoint.
+#include "simt_common.cuh"
+#include "simt_layout.h"
+
+namespace e2ttt {
+
+template <typename Real> struct BwdScalars {
+    Real kWb[kMaxC], kMb[kMaxC]; // adjoints of K^W_t, K^M_t
+};
+
+// out = r ( x - mean(x) - y mean(x*y) ) for one row held by one warp (the LN Jacobian is symmetric)
+template <typename Real>
+__device__ __forceinline__ void warp_ln_jac(const Real* x, const Real* y, Real r, int d, Real* out) {
+    const int lane = threadIdx.x & 31;
+    Real sx = 0, sxy = 0;
+    for (int i = lane; i < d; i += 32) { sx += x[i]; sxy += x[i] * y[i]; }
+    sx = warp_sum(sx) / (Real)d;
+    sxy = warp_sum(sxy) / (Real)d;
+    for (int i = lane; i < d; i += 32) out[i] = r * (x[i] - sx - y[i] * sxy);
+}
+
+template <typename Real, typename IO>
+__global__ void __launch_bounds__(kSimtThreads) simt_bwd_mlp_kernel(const SimtBwdArgs a) {
+    constexpr int NMAT = 2;
+    __shared__ GemmSmem<Real> gsm;
+    __shared__ ChunkScalars<Real> sc;
+    __shared__ BwdScalars<Real> bs;
+    __shared__ Real red[8];
+
+    const int seq = blockIdx.x;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    constexpr int NW = kSimtThreads / 32;
+    const int d = a.d, h = a.h, C = a.C, L = a.L;
+    const size_t dh = (size_t)d * h;
+    const SimtLayout& lay = a.lay;
+    Real* ws = reinterpret_cast<Real*>(a.ws) + (size_t)seq * lay.per_seq;
+    const IO* q = reinterpret_cast<const IO*>(a.q) + (size_t)seq * L * d;
+    const IO* k = reinterpret_cast<const IO*>(a.k) + (size_t)seq * L * d;
+    const IO* v = reinterpret_cast<const IO*>(a.v) + (size_t)seq * L * d;
+    const IO* d_o = reinterpret_cast<const IO*>(a.d_o) + (size_t)seq * L * d;
+    IO* dq = reinterpret_cast<IO*>(a.dq) + (size_t)seq * L * d;
+    IO* dk = reinterpret_cast<IO*>(a.dk) + (size_t)seq * L * d;
+    IO* dv = reinterpret_cast<IO*>(a.dv) + (size_t)seq * L * d;
+    const float* eta = a.eta + (size_t)seq * L;
+    const float* beta = a.beta + (size_t)seq * L;
+    const float* gamma = a.gamma + (size_t)seq * L;
+    float* d_eta = a.d_eta + (size_t)seq * L;
+    float* d_beta = a.d_beta + (size_t)seq * L;
+    float* d_gamma = a.d_gamma + (size_t)seq * L;
+    const Real eps = (Real)a.eps;
+
+    Real *T[NMAT], *S[NMAT], *Wb[NMAT];
+#pragma unroll
+    for (int i = 0; i < NMAT; ++i) {
+        T[i] = ws + lay.T[i]; S[i] = ws + lay.S[i]; Wb[i] = ws + lay.Wb[i];
+        const float* tf = a.dW_final[i] ? a.dW_final[i] + (size_t)seq * dh : nullptr;
+        const float* sf = a.dM_final[i] ? a.dM_final[i] + (size_t)seq * dh : nullptr;
+        for (size_t e = tid; e < dh; e += kSimtThreads) {
+            T[i][e] = tf ? (Real)tf[e] : (Real)0;
+            S[i][e] = sf ? (Real)sf[e] : (Real)0;
+        }
+    }
+    Real* Z1 = ws + lay.Z1;   // [2len x h]  pre-activations, key rows then query rows
+    Real* A = ws + lay.A;     // [2len x h]  gelu(Z1)
+    Real* U = ws + lay.U;     // [2len x d]  normalised rows y (after the LN step)
+    Real* Pu = ws + lay.Pu;   // [len x d]
+    Real* Pz = ws + lay.Pz1;  // [len x h]
+    Real* Pa = ws + lay.Pa;   // [len x h]
+    Real* E = ws + lay.E;     // [len x d]
+    Real* XY2 = ws + lay.XY2; // [len x 2d]  (Ak T2^T | Ak S2^T)
+    Real* XY1 = ws + lay.XY1; // [len x 2h]  (K T1^T | K S1^T)
+    Real* Pub = ws + lay.Pub;
+    Real* Pzb = ws + lay.Pzb; // becomes Pab in place
+    Real* Zkb = ws + lay.Zkb;
+    Real* Akb = ws + lay.Akb;
+    Real* Kb = ws + lay.Kb;
+    Real* Eb = ws + lay.Eb;
+    Real* Ukb = ws + lay.Ukb;
+    Real* Uqb = ws + lay.Uqb;
+    Real* Zqb = ws + lay.Zqb;
+    Real* rk = ws + lay.rk;
+    Real* rq = ws + lay.rq;
+    __syncthreads();
+
+    for (int c = a.nchunks - 1; c >= 0; --c) {
+        const int s = c * C;
+        const int len = min(C, L - s);
+        const IO* kc = k + (size_t)s * d;
+        const IO* qc = q + (size_t)s * d;
+        const IO* vc = v + (size_t)s * d;
+        const IO* doc = d_o + (size_t)s * d;
+        const Real* ck = ws + lay.ckpt + (size_t)c * 2 * NMAT * dh;
+        const Real* W1 = ck;               // [h x d]
+        const Real* W2 = ck + dh;          // [d x h]
+        const Real* M1 = ck + 2 * dh;
+        const Real* M2 = ck + 3 * dh;
+
+        if (warp == 0) chunk_scalars_warp<Real>(eta + s, beta + s, gamma + s, len, &sc);
+        for (size_t e = tid; e < dh; e += kSimtThreads) { Wb[0][e] = 0; Wb[1][e] = 0; }
+
+        // ---------------- forward of the chunk, recomputed ----------------
+        block_gemm<Real, 1, true, true>(
+            2 * len, h, d,
+            [&](int m, int kk, Real& a0, Real& a1) {
+                a0 = (m < len) ? ld_io<Real>(kc, (size_t)m * d + kk) : ld_io<Real>(qc, (size_t)(m - len) * d + kk);
+            },
+            [&](int n, int kk) { return W1[(size_t)n * d + kk]; },
+            [&](int m, int n, Real acc, Real) {
+                Z1[(size_t)m * h + n] = acc;
+                A[(size_t)m * h + n] = gelu_f(acc);
+            },
+            &gsm);
+        block_gemm<Real, 1, true, true>(
+            2 * len, d, h, [&](int m, int kk, Real& a0, Real& a1) { a0 = A[(size_t)m * h + kk]; },
+            [&](int n, int kk) { return W2[(size_t)n * h + kk]; },
+            [&](int m, int n, Real acc, Real) { U[(size_t)m * d + n] = acc; }, &gsm);
+        for (int m = warp; m < 2 * len; m += NW) {
+            Real* u = U + (size_t)m * d;
+            const Real r = warp_layernorm(u, u, d, eps);
+            if (m >= len) {
+                if (lane == 0) rq[m - len] = r;
+                // adjoint of the output's LN: Uqb = J_q d_o
+                const size_t row = (size_t)(m - len) * d;
+                Real sx = 0, sxy = 0;
+                for (int i = lane; i < d; i += 32) {
+                    const Real x = ld_io<Real>(doc, row + i);
+                    sx += x; sxy += x * u[i];
+                }
+                sx = warp_sum(sx) / (Real)d;
+                sxy = warp_sum(sxy) / (Real)d;
+                for (int i = lane; i < d; i += 32)
+                    Uqb[row + i] = r * (ld_io<Real>(doc, row + i) - sx - u[i] * sxy);
+            } else {
+                if (lane == 0) rk[m] = r;
+                const size_t row = (size_t)m * d;
+                for (int i = lane; i < d; i += 32)
+                    E[row + i] = ld_io<Real>(kc, row + i) + u[i] - ld_io<Real>(vc, row + i);
+                __syncwarp();
+                warp_ln_jac(E + row, u, r, d, Pu + row);
+            }
+        }
+        __syncthreads();
+        block_gemm<Real, 1, true, false>(
+            len, h, d, [&](int m, int kk, Real& a0, Real& a1) { a0 = Pu[(size_t)m * d + kk]; },
+            [&](int n, int kk) { return W2[(size_t)kk * h + n]; },
+            [&](int m, int n, Real acc, Real) {
+                const size_t e = (size_t)m * h + n;
+                Pa[e] = acc;
+                Pz[e] = acc * gelu_d1(Z1[e]);
+            },
+            &gsm);
+
+        // ---------------- (i) outputs o = q + LN(W2 gelu(W1 q)) ----------------
+        const Real* Zq = Z1 + (size_t)len * h;
+        const Real* Aq = A + (size_t)len * h;
+        block_gemm<Real, 1, true, false>(
+            len, h, d, [&](int m, int kk, Real& a0, Real& a1) { a0 = Uqb[(size_t)m * d + kk]; },
+            [&](int n, int kk) { return W2[(size_t)kk * h + n]; },
+            [&](int m, int n, Real acc, Real) { Zqb[(size_t)m * h + n] = acc * gelu_d1(Zq[(size_t)m * h + n]); }, &gsm);
+        block_gemm<Real, 1, true, false>(
+            len, d, h, [&](int m, int kk, Real& a0, Real& a1) { a0 = Zqb[(size_t)m * h + kk]; },
+            [&](int n, int kk) { return W1[(size_t)kk * d + n]; },
+            [&](int m, int n, Real acc, Real) {
+                const size_t e = (size_t)m * d + n;
+                st_io(dq + (size_t)s * d, e, ld_io<Real>(doc, e) + acc);
+            },
+            &gsm);
+        block_gemm<Real, 1, false, false>( // Wb2 += Uqb^T Aq
+            d, h, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Uqb[(size_t)t * d + m]; },
+            [&](int n, int t) { return Aq[(size_t)t * h + n]; },
+            [&](int m, int n, Real acc, Real) { Wb[1][(size_t)m * h + n] += acc; }, &gsm);
+        block_gemm<Real, 1, false, false>( // Wb1 += Zqb^T Q
+            h, d, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Zqb[(size_t)t * h + m]; },
+            [&](int n, int t) { return ld_io<Real>(qc, (size_t)t * d + n); },
+            [&](int m, int n, Real acc, Real) { Wb[0][(size_t)m * d + n] += acc; }, &gsm);
+
+        // ---------------- (ii) state transition: carries ----------------
+        Real cwb, cmb, cbb;
+        {
+            Real pw = 0, pm = 0, pb = 0;
+            for (size_t e = tid; e < dh; e += kSimtThreads) {
+                pw += T[0][e] * W1[e] + T[1][e] * W2[e];
+                pm += T[0][e] * M1[e] + T[1][e] * M2[e];
+                pb += S[0][e] * M1[e] + S[1][e] * M2[e];
+            }
+            cwb = block_sum(pw, red);
+            cmb = block_sum(pm, red);
+            cbb = block_sum(pb, red);
+        }
+        // G_t enters W_C with K^W_t and M_C with K^M_t: its adjoint is K^W_t T + K^M_t S.
+        block_gemm<Real, 1, true, true>( // XY2 = Ak [T2; S2]^T
+            len, 2 * d, h, [&](int m, int kk, Real& a0, Real& a1) { a0 = A[(size_t)m * h + kk]; },
+            [&](int n, int kk) { return n < d ? T[1][(size_t)n * h + kk] : S[1][(size_t)(n - d) * h + kk]; },
+            [&](int m, int n, Real acc, Real) { XY2[(size_t)m * 2 * d + n] = acc; }, &gsm);
+        block_gemm<Real, 1, true, true>( // XY1 = K [T1; S1]^T
+            len, 2 * h, d, [&](int m, int kk, Real& a0, Real& a1) { a0 = ld_io<Real>(kc, (size_t)m * d + kk); },
+            [&](int n, int kk) { return n < h ? T[0][(size_t)n * d + kk] : S[0][(size_t)(n - h) * d + kk]; },
+            [&](int m, int n, Real acc, Real) { XY1[(size_t)m * 2 * h + n] = acc; }, &gsm);
+        for (int t = warp; t < len; t += NW) {
+            const Real* x2 = XY2 + (size_t)t * 2 * d;
+            const Real* x1 = XY1 + (size_t)t * 2 * h;
+            Real sw = 0, sm = 0;
+            for (int i = lane; i < d; i += 32) {
+                const Real p = Pu[(size_t)t * d + i];
+                sw += p * x2[i]; sm += p * x2[d + i];
+            }
+            for (int j = lane; j < h; j += 32) {
+                const Real p = Pz[(size_t)t * h + j];
+                sw += p * x1[j]; sm += p * x1[h + j];
+            }
+            sw = warp_sum(sw); sm = warp_sum(sm);
+            if (lane == 0) { bs.kWb[t] = -sw; bs.kMb[t] = -sm; }
+            const Real kw = sc.kW[t], km = sc.kM[t];
+            for (int i = lane; i < d; i += 32) Pub[(size_t)t * d + i] = -(kw * x2[i] + km * x2[d + i]);
+            for (int j = lane; j < h; j += 32) Pzb[(size_t)t * h + j] = -(kw * x1[j] + km * x1[h + j]);
+        }
+        __syncthreads();
+        // ---------------- (iii) per-token gradients G_t = -(pz k^T, pu a^T) ----------------
+        block_gemm<Real, 1, true, false>( // Akb = -[kW Pu | kM Pu] [T2; S2]
+            len, h, 2 * d,
+            [&](int m, int kk, Real& a0, Real& a1) {
+                a0 = kk < d ? sc.kW[m] * Pu[(size_t)m * d + kk] : sc.kM[m] * Pu[(size_t)m * d + kk - d];
+            },
+            [&](int n, int kk) { return kk < d ? T[1][(size_t)kk * h + n] : S[1][(size_t)(kk - d) * h + n]; },
+            [&](int m, int n, Real acc, Real) { Akb[(size_t)m * h + n] = -acc; }, &gsm);
+        block_gemm<Real, 1, true, false>( // Kb = -[kW Pz | kM Pz] [T1; S1]
+            len, d, 2 * h,
+            [&](int m, int kk, Real& a0, Real& a1) {
+                a0 = kk < h ? sc.kW[m] * Pz[(size_t)m * h + kk] : sc.kM[m] * Pz[(size_t)m * h + kk - h];
+            },
+            [&](int n, int kk) { return kk < h ? T[0][(size_t)kk * d + n] : S[0][(size_t)(kk - h) * d + n]; },
+            [&](int m, int n, Real acc, Real) { Kb[(size_t)m * d + n] = -acc; }, &gsm);
+        // pz = pa * gelu'(z)
+        for (size_t e = tid; e < (size_t)len * h; e += kSimtThreads) {
+            const Real pzb = Pzb[e], z = Z1[e];
+            Zkb[e] = pzb * Pa[e] * gelu_d2(z);
+            Pzb[e] = pzb * gelu_d1(z); // now Pab
+        }
+        __syncthreads();
+        const Real* Pab = Pzb;
+        // pa = W2^T pu
+        block_gemm<Real, 1, true, true>(
+            len, d, h, [&](int m, int kk, Real& a0, Real& a1) { a0 = Pab[(size_t)m * h + kk]; },
+            [&](int n, int kk) { return W2[(size_t)n * h + kk]; },
+            [&](int m, int n, Real acc, Real) { Pub[(size_t)m * d + n] += acc; }, &gsm);
+        block_gemm<Real, 1, false, false>( // Wb2 += Pu^T Pab
+            d, h, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Pu[(size_t)t * d + m]; },
+            [&](int n, int t) { return Pab[(size_t)t * h + n]; },
+            [&](int m, int n, Real acc, Real) { Wb[1][(size_t)m * h + n] += acc; }, &gsm);
+        // pu = J(u) e, e = k + y - v, y = LN(u)
+        for (int t = warp; t < len; t += NW) {
+            const size_t row = (size_t)t * d;
+            const Real* y = U + row;
+            const Real r = rk[t];
+            warp_ln_jac(Pub + row, y, r, d, Eb + row);
+            __syncwarp();
+            Real spp = 0, mpy = 0, mey = 0;
+            for (int i = lane; i < d; i += 32) {
+                spp += Pub[row + i] * Pu[row + i];
+                mpy += Pub[row + i] * y[i];
+                mey += E[row + i] * y[i];
+            }
+            spp = warp_sum(spp);
+            mpy = warp_sum(mpy) / (Real)d;
+            mey = warp_sum(mey) / (Real)d;
+            // second-order term of the LN Jacobian, then dy -> du for the y inside e
+            warp_ln_jac(Eb + row, y, r, d, Ukb + row);
+            __syncwarp();
+            for (int i = lane; i < d; i += 32) {
+                Ukb[row + i] += -(r / (Real)d) * spp * y[i] - r * (mpy * Pu[row + i] + mey * Eb[row + i]);
+                Kb[row + i] += Eb[row + i];
+                st_io(dv + (size_t)s * d, row + i, -Eb[row + i]);
+            }
+        }
+        __syncthreads();
+        // u = W2 a, a = gelu(z)
+        block_gemm<Real, 1, true, false>(
+            len, h, d, [&](int m, int kk, Real& a0, Real& a1) { a0 = Ukb[(size_t)m * d + kk]; },
+            [&](int n, int kk) { return W2[(size_t)kk * h + n]; },
+            [&](int m, int n, Real acc, Real) {
+                const size_t e = (size_t)m * h + n;
+                Zkb[e] += (Akb[e] + acc) * gelu_d1(Z1[e]);
+            },
+            &gsm);
+        block_gemm<Real, 1, false, false>( // Wb2 += Ukb^T Ak
+            d, h, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Ukb[(size_t)t * d + m]; },
+            [&](int n, int t) { return A[(size_t)t * h + n]; },
+            [&](int m, int n, Real acc, Real) { Wb[1][(size_t)m * h + n] += acc; }, &gsm);
+        // z = W1 k
+        block_gemm<Real, 1, true, false>(
+            len, d, h, [&](int m, int kk, Real& a0, Real& a1) { a0 = Zkb[(size_t)m * h + kk]; },
+            [&](int n, int kk) { return W1[(size_t)kk * d + n]; },
+            [&](int m, int n, Real acc, Real) {
+                const size_t e = (size_t)m * d + n;
+                st_io(dk + (size_t)s * d, e, Kb[e] + acc);
+            },
+            &gsm);
+        block_gemm<Real, 1, false, false>( // Wb1 += Zkb^T K
+            h, d, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Zkb[(size_t)t * h + m]; },
+            [&](int n, int t) { return ld_io<Real>(kc, (size_t)t * d + n); },
+            [&](int m, int n, Real acc, Real) { Wb[0][(size_t)m * d + n] += acc; }, &gsm);
+
+        // ---------------- adjoints of the chunk-start state ----------------
+        {
+            const Real cw = sc.cw, cm = sc.cm, cb = sc.cb;
+#pragma unroll
+            for (int i = 0; i < NMAT; ++i)
+                for (size_t e = tid; e < dh; e += kSimtThreads) {
+                    const Real t = T[i][e], sv = S[i][e];
+                    T[i][e] = cw * t + Wb[i][e];
+                    S[i][e] = cm * t + cb * sv;
+                }
+        }
+        // ---------------- (iv) reverse of the suffix scans ----------------
+        if (tid == 0) {
+            Real Sb = 0, btb = cbb, gtb = cwb; // adjoints of S_0 (unused), bt_0, gt_0
+            for (int t = 0; t < len; ++t) {
+                // index t: state t; token t+1 lives at array index t
+                const Real b1 = (Real)beta[s + t], g1 = (Real)gamma[s + t], e1 = (Real)eta[s + t];
+                const Real kWb = bs.kWb[t], kMb = bs.kMb[t];
+                // S_t = beta_{t+1} S_{t+1} + gt_t ; bt_t = beta_{t+1} bt_{t+1} ; gt_t = gamma_{t+1} gt_{t+1}
+                gtb += Sb;
+                Real bb = Sb * sc.S[t + 1] + btb * sc.bt[t + 1];
+                Real Sb_next = Sb * b1;
+                Real btb_next = btb * b1;
+                const Real gb = gtb * sc.gt[t + 1];
+                Real gtb_next = gtb * g1;
+                if (t == 0) { // cm = beta_1 S_1
+                    bb += cmb * sc.S[1];
+                    Sb_next += cmb * b1;
+                }
+                // K^M_{t+1} = eta bt_{t+1}, K^W_{t+1} = eta S_{t+1}
+                d_eta[s + t] = (float)(kMb * sc.bt[t + 1] + kWb * sc.S[t + 1]);
+                btb_next += kMb * e1;
+                Sb_next += kWb * e1;
+                d_beta[s + t] = (float)bb;
+                d_gamma[s + t] = (float)gb;
+                Sb = Sb_next; btb = btb_next; gtb = gtb_next;
+            }
+        }
+        __syncthreads();
+    }
+
+#pragma unroll
+    for (int i = 0; i < NMAT; ++i) {
+        float* wf = a.dW_init[i] + (size_t)seq * dh;
+        float* mf = a.dM_init[i] + (size_t)seq * dh;
+        for (size_t e = tid; e < dh; e += kSimtThreads) {
+            wf[e] = (float)T[i][e];
+            mf[e] = (float)S[i][e];
+        }
+    }
+}
+
+int simt_bwd_launch(const SimtBwdArgs& a, int kind, int io_dtype, void* stream) {
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    dim3 grid(a.N), block(kSimtThreads);
+    if (kind != 0) return (int)cudaErrorInvalidValue;
+    if (io_dtype == 0) simt_bwd_mlp_kernel<double, float><<<grid, block, 0, st>>>(a);
+    else simt_bwd_mlp_kernel<float, __nv_bfloat16><<<grid, block, 0, st>>>(a);
+    return (int)cudaGetLastError();
+}
+
+}  // namespace e2ttt

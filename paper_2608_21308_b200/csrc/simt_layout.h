@@ -1,0 +1,81 @@
+// Workspace layout of the SIMT kernels (host and device).  Offsets are in elements of the kernel's
+// internal type (double for fp32 I/O, float for bf16 I/O), relative to the sequence's own slice.
+#pragma once
+#include <stddef.h>
+#include <stdint.h>
+
+namespace e2ttt {
+
+struct SimtLayout {
+    // running state
+    size_t W[3], M[3];
+    // forward intermediates of one chunk ([2C x .] buffers hold the k-path rows first, then the q-path rows)
+    size_t Z1, Z2, A, U, Pu, Pz1, Pz2;
+    // backward only
+    size_t T[3], S[3];   // adjoints of the chunk-end state (W, M)
+    size_t Wb[3];        // adjoint accumulators of the chunk-start weights
+    size_t Pa, E, XY2, XY1, Pub, Pzb, Zkb, Akb, Kb, Eb, Ukb, Uqb, Zqb;
+    size_t rk, rq, red;  // per-row 1/std of the two LN calls; small reduction scratch
+    size_t ckpt;         // [nchunks][2][nmat][d*h] chunk-start (W, M), present when states are saved
+    size_t per_seq;      // elements per sequence
+};
+
+inline SimtLayout simt_layout(int d, int h, int C, int nmat, int nchunks, bool save_states, bool backward) {
+    SimtLayout l{};
+    size_t o = 0;
+    const size_t dh = (size_t)d * h;
+    auto take = [&](size_t n) { size_t r = o; o += (n + 31) / 32 * 32; return r; };
+    for (int i = 0; i < 3; ++i) { l.W[i] = take(i < nmat ? dh : 0); l.M[i] = take(i < nmat ? dh : 0); }
+    l.Z1 = take((size_t)2 * C * h); l.Z2 = take((size_t)2 * C * h); l.A = take((size_t)2 * C * h);
+    l.U = take((size_t)2 * C * d); l.Pu = take((size_t)C * d);
+    l.Pz1 = take((size_t)C * h); l.Pz2 = take((size_t)C * h);
+    if (backward) {
+        for (int i = 0; i < 3; ++i) {
+            l.T[i] = take(i < nmat ? dh : 0); l.S[i] = take(i < nmat ? dh : 0); l.Wb[i] = take(i < nmat ? dh : 0);
+        }
+        l.Pa = take((size_t)C * h); l.E = take((size_t)C * d);
+        l.XY2 = take((size_t)C * 2 * d); l.XY1 = take((size_t)C * 2 * h);
+        l.Pub = take((size_t)C * d); l.Pzb = take((size_t)C * h); l.Zkb = take((size_t)C * h);
+        l.Akb = take((size_t)C * h); l.Kb = take((size_t)C * d); l.Eb = take((size_t)C * d);
+        l.Ukb = take((size_t)C * d); l.Uqb = take((size_t)C * d); l.Zqb = take((size_t)C * h);
+        l.rk = take(C); l.rq = take(C); l.red = take(64);
+    }
+    l.ckpt = take(save_states ? (size_t)nchunks * 2 * nmat * dh : 0);
+    l.per_seq = o;
+    return l;
+}
+
+struct SimtFwdArgs {
+    int N, L, d, h, C, nchunks, save_states;
+    float eps;
+    const void *q, *k, *v;
+    const float *eta, *beta, *gamma;
+    const float* W_init[3];
+    const float* M_init[3]; // nullptr entries = zeros
+    void* o;
+    float* W_final[3];
+    float* M_final[3];
+    void* ws;
+    SimtLayout lay;
+};
+
+struct SimtBwdArgs {
+    int N, L, d, h, C, nchunks;
+    float eps;
+    const void *q, *k, *v, *d_o;
+    const float *eta, *beta, *gamma;
+    const float* dW_final[3]; // nullptr entries = zeros
+    const float* dM_final[3];
+    void *dq, *dk, *dv;
+    float *d_eta, *d_beta, *d_gamma;
+    float* dW_init[3];
+    float* dM_init[3];
+    void* ws;
+    SimtLayout lay;
+};
+
+// launchers (simt_fwd.cu / simt_bwd.cu); return a cudaError_t value as int
+int simt_fwd_launch(const SimtFwdArgs& a, int kind, int io_dtype, void* stream);
+int simt_bwd_launch(const SimtBwdArgs& a, int kind, int io_dtype, void* stream);
+
+}  // namespace e2ttt

@@ -1,0 +1,180 @@
+"""GPU parity: the C-ABI library against the fp64 oracle, element by element, on the same seeded inputs.
+
+Gated metric per tensor: max|x - ref| / max|ref|.  Tolerances (from the benchmark statement):
+1e-4 for fp32 I/O, 2e-2 for bf16 I/O with fp32 accumulation, for outputs, final states and gradients.
+
+The chunk-to-chunk map is chaotic under the benchmark's gate distributions (a perturbation grows by
+roughly 1.6-1.8x per chunk), so whole-sequence free-running comparisons are made only where they mean
+something (config 0: 16 chunks; the paper's own gate regime).  Everything else is compared in
+teacher-forced windows: each window starts from the oracle's state.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_21308_b200 import binding as E
+from paper_2608_21308_b200 import inputs
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+TOL_F32 = 1e-4
+TOL_BF16 = 2e-2
+MLP, SWIGLU = inputs.KIND_MLP, inputs.KIND_SWIGLU
+
+
+def check_forward(got, ref, tol, what=""):
+    errs = {"o": util.rel_err(got["o"], ref["o"])}
+    for i in range(len(ref["W"])):
+        errs[f"W{i + 1}"] = util.rel_err(got["W"][i], ref["W"][i])
+        errs[f"M{i + 1}"] = util.rel_err(got["M"][i], ref["M"][i])
+    bad = {k: v for k, v in errs.items() if not v <= tol}
+    assert not bad, f"{what}: {bad} (all: {errs})"
+    return errs
+
+
+def check_backward(got, ref, tol, what=""):
+    errs = {n: util.rel_err(got[n], ref[n]) for n in ("dq", "dk", "dv", "deta", "dbeta", "dgamma")}
+    for i in range(len(ref["dW"])):
+        errs[f"dW{i + 1}"] = util.rel_err(got["dW"][i], ref["dW"][i])
+        errs[f"dM{i + 1}"] = util.rel_err(got["dM"][i], ref["dM"][i])
+    bad = {k: v for k, v in errs.items() if not v <= tol}
+    assert not bad, f"{what}: {bad} (all: {errs})"
+    return errs
+
+
+# ------------------------------------------------------------------ config 0: free-running, fp32 I/O
+def test_config0_forward_free_running_fp32():
+    r = inputs.config(0)
+    x = inputs.generate(r)
+    ref = util.oracle_forward(x, r.C, r.kind)
+    got, _ = util.gpu_forward(x, d=r.d, h=r.h, C=r.C, kind=r.kind, io="f32")
+    check_forward(got, ref, TOL_F32, "config 0")
+
+
+def test_config0_backward_free_running_fp32():
+    r = inputs.config(0, L=64)  # 4 chunks: the adjoint grows quickly with depth, keep it representable
+    x = inputs.generate(r, with_d_o=True, with_dstate=True)
+    ref = util.oracle_backward(x, r.C, r.kind)
+    got = util.gpu_backward(x, d=r.d, h=r.h, C=r.C, kind=r.kind, io="f32")
+    check_backward(got, ref, TOL_F32, "config 0 bwd")
+    got2 = util.gpu_backward(x, d=r.d, h=r.h, C=r.C, kind=r.kind, io="f32", via_saved_states=True)
+    for n in ("dq", "dk", "dv", "deta", "dbeta", "dgamma"):
+        assert np.array_equal(got[n], got2[n]), n  # saved states == recomputed states, bitwise
+
+
+# ------------------------------------------------------------------ odd shapes: several tiles, ragged tails, both networks
+@pytest.mark.parametrize("kind", [MLP, SWIGLU])
+@pytest.mark.parametrize("d,h,C,L,N", [(48, 80, 24, 100, 3), (64, 192, 128, 256, 2), (8, 16, 1, 5, 1), (72, 136, 16, 7, 2)])
+def test_forward_odd_shapes_fp32(kind, d, h, C, L, N):
+    r = inputs.Recipe(B=N, H=1, L=L, d=d, h=h, C=C, kind=kind, seed=5, m_std=0.01)
+    x = inputs.generate(r)
+    ref = util.oracle_forward(x, C, kind)
+    got, _ = util.gpu_forward(x, d=d, h=h, C=C, kind=kind, io="f32")
+    check_forward(got, ref, TOL_F32, f"kind {kind} d{d} h{h} C{C} L{L}")
+
+
+@pytest.mark.parametrize("d,h,C,L,N", [(48, 80, 24, 60, 2), (8, 16, 1, 4, 1), (64, 160, 32, 64, 1)])
+def test_backward_odd_shapes_fp32(d, h, C, L, N):
+    r = inputs.Recipe(B=N, H=1, L=L, d=d, h=h, C=C, kind=MLP, seed=6, m_std=0.01)
+    x = inputs.generate(r, with_d_o=True, with_dstate=True)
+    ref = util.oracle_backward(x, C, MLP)
+    got = util.gpu_backward(x, d=d, h=h, C=C, kind=MLP, io="f32")
+    check_backward(got, ref, TOL_F32, f"bwd d{d} h{h} C{C} L{L}")
+
+
+def test_optional_inputs_null_momentum_and_null_state_adjoints():
+    r = inputs.Recipe(B=2, H=1, L=32, d=16, h=32, C=16, kind=MLP, seed=8)
+    x = inputs.generate(r, with_d_o=True, with_dstate=True)
+    ref = util.oracle_forward(x, r.C, MLP, use_M=False)
+    got, _ = util.gpu_forward(x, d=r.d, h=r.h, C=r.C, kind=MLP, io="f32", use_M=False)
+    check_forward(got, ref, TOL_F32)
+    refb = util.oracle_backward(x, r.C, MLP, use_M=False, use_dstate=False)
+    gotb = util.gpu_backward(x, d=r.d, h=r.h, C=r.C, kind=MLP, io="f32", use_M=False, use_dstate=False)
+    check_backward(gotb, refb, TOL_F32)
+
+
+# ------------------------------------------------------------------ paper-regime gates: free-running over many chunks
+def test_paper_regime_free_running_fp32():
+    r = inputs.paper_regime(inputs.Recipe(B=2, H=1, L=1024, d=64, h=256, C=64, kind=MLP, seed=2))
+    x = inputs.generate(r)
+    ref = util.oracle_forward(x, r.C, MLP)
+    got, _ = util.gpu_forward(x, d=r.d, h=r.h, C=r.C, kind=MLP, io="f32")
+    check_forward(got, ref, TOL_F32, "paper regime")
+
+
+# ------------------------------------------------------------------ configs 1-4: teacher-forced one-chunk windows, bf16 I/O
+WINDOW_CASES = [
+    ("config1", 1, dict(heads=[0, 37, 95]), 8),
+    ("config2", 2, dict(heads=[0, 21, 63]), 6),
+    ("config3-C64", 3, dict(heads=[0, 40]), 6),
+    ("config3-C16", 3, dict(heads=[1], C=16), 12),
+    ("config3-C32", 3, dict(heads=[2], C=32), 8),
+    ("config3-C128", 3, dict(heads=[3], C=128), 4),
+    ("config4", 4, dict(heads=[0, 15]), 6),
+]
+
+
+@pytest.mark.parametrize("name,cfg,over,n_chunks", WINDOW_CASES, ids=[c[0] for c in WINDOW_CASES])
+def test_forward_teacher_forced_windows_bf16(name, cfg, over, n_chunks):
+    r = inputs.config(cfg, **over)
+    xw, ref = util.teacher_forced_windows(r, n_chunks, window=1)
+    got, _ = util.gpu_forward(xw, d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16")
+    check_forward(got, ref, TOL_BF16, name)
+
+
+def test_backward_teacher_forced_windows_bf16_config4():
+    r = inputs.config(4, heads=[0, 9])
+    xw, _ = util.teacher_forced_windows(r, 4, window=1, with_grads=True)
+    ref = util.oracle_backward(xw, r.C, r.kind)
+    got = util.gpu_backward(xw, d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16")
+    check_backward(got, ref, TOL_BF16, "config 4 bwd windows")
+
+
+# ------------------------------------------------------------------ properties that hold at any size
+def test_split_calls_chain_and_in_place_state_update():
+    r = inputs.Recipe(B=3, H=1, L=128, d=32, h=64, C=32, kind=MLP, io="bf16", seed=3)
+    x = inputs.generate(r)
+    whole, _ = util.gpu_forward(x, d=r.d, h=r.h, C=r.C, kind=MLP, io="bf16")
+    half = {n: (np.ascontiguousarray(a[:, :64]) if not isinstance(a, list) else a) for n, a in x.items()}
+    a, _ = util.gpu_forward(half, d=r.d, h=r.h, C=r.C, kind=MLP, io="bf16")
+    rest = {n: (np.ascontiguousarray(v[:, 64:]) if not isinstance(v, list) else v) for n, v in x.items()}
+    rest["W"], rest["M"] = a["W"], a["M"]
+    b, _ = util.gpu_forward(rest, d=r.d, h=r.h, C=r.C, kind=MLP, io="bf16")
+    assert np.array_equal(np.concatenate([a["o"], b["o"]], 1), whole["o"])
+    for i in range(2):
+        assert np.array_equal(b["W"][i], whole["W"][i]) and np.array_equal(b["M"][i], whole["M"][i])
+    # in place: W_final aliases W_init
+    out, hd = util.gpu_forward(x, d=r.d, h=r.h, C=r.C, kind=MLP, io="bf16")
+    o2 = torch.empty_like(hd["q"])
+    E.e2ttt_chunk_fwd(hd["p"], hd["q"], hd["k"], hd["v"], hd["eta"], hd["beta"], hd["gamma"], hd["W"], hd["M"], o2,
+                      hd["W"], hd["M"], hd["ws"], 0)
+    torch.cuda.synchronize()
+    for i in range(2):
+        assert np.array_equal(hd["W"][i].cpu().numpy()[:, 0], whole["W"][i])
+        assert np.array_equal(hd["M"][i].cpu().numpy()[:, 0], whole["M"][i])
+
+
+def test_runs_are_bitwise_repeatable_and_heads_independent():
+    r = inputs.config(1, heads=[3, 4, 5, 6], L=256)
+    x = inputs.generate(r)
+    a, _ = util.gpu_forward(x, d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16")
+    b, _ = util.gpu_forward(x, d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16")
+    assert np.array_equal(a["o"], b["o"]) and all(np.array_equal(u, w) for u, w in zip(a["W"], b["W"]))
+    solo = {n: (np.ascontiguousarray(v[2:3]) if not isinstance(v, list) else [m[2:3] for m in v]) for n, v in x.items()}
+    c, _ = util.gpu_forward(solo, d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16")
+    assert np.array_equal(c["o"][0], a["o"][2])
+
+
+def test_a_failing_call_leaves_outputs_untouched():
+    p = E.make_params(1, 1, 30, 16, 32, 16)
+    t4 = torch.zeros(1, 1, 30, 16, device="cuda")
+    t3 = torch.zeros(1, 1, 30, device="cuda")
+    W = [torch.zeros(1, 1, 32, 16, device="cuda"), torch.zeros(1, 1, 16, 32, device="cuda")]
+    o = torch.full_like(t4, 7.0)
+    small = torch.empty(16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(E.E2TTTError) as ei:
+        E.e2ttt_chunk_fwd(p, t4, t4, t4, t3, t3, t3, W, None, o, W, W, small, 0)
+    assert ei.value.status == -5
+    torch.cuda.synchronize()
+    assert float(o.min()) == 7.0
