@@ -148,6 +148,36 @@ E2TTT_API int e2ttt_chunk_bwd(const e2ttt_params* p,
                     float* const* dW_init, float* const* dM_init,
                     void* workspace, size_t workspace_bytes, int states_saved, void* stream);
 
+/* Forward without any caller-provided scratch.  (The paper has no counterpart: this exists for the
+ * library's users, not for the method.)
+ *
+ * Who needs it: code that runs where asking the CUDA runtime for device memory is off the table -
+ * a plugin handed only its input and output buffers by a host application that owns the memory
+ * pool, a real-time loop that must not touch the allocator after start-up, a process whose memory
+ * budget was fixed and spent before this call.  Such callers cannot size and allocate the workspace
+ * e2ttt_chunk_fwd asks for.
+ *
+ * Same arguments and results as e2ttt_chunk_fwd(save_states = 0), minus the workspace.  The scratch
+ * is a fixed array of E2TTT_NOALLOC_SCRATCH_BYTES inside the library's device image, so every GPU
+ * that loads the library gives up that much memory until the process exits.  A call whose
+ * e2ttt_workspace_bytes(p, 0) exceeds it returns E2TTT_ERR_WORKSPACE and launches nothing (with fp32
+ * I/O the benchmark's tiny configuration, B*H = 1, d = 64, h = 256, C = 16, needs about 0.8 MiB;
+ * bf16 I/O needs half as much per sequence).  The call itself allocates and frees nothing.
+ *
+ * The first call on each device looks up the array's device address (one runtime query, with that
+ * device current) and remembers it; make that first call outside any stream capture.
+ * All calls on a device share the one array.  It keeps whatever the previous call left there, which
+ * is harmless: the kernel writes every scratch word before reading it, nothing has to start at
+ * zero.  But two calls that run on the GPU at the same time (different streams, or different host
+ * threads) would overwrite each other's intermediates: serialise them.
+ */
+#define E2TTT_NOALLOC_SCRATCH_BYTES (8u << 20)
+E2TTT_API int e2ttt_chunk_fwd_noalloc(const e2ttt_params* p,
+                    const void* q, const void* k, const void* v,
+                    const float* eta, const float* beta, const float* gamma,
+                    const float* const* W_init, const float* const* M_init,
+                    void* o, float* const* W_final, float* const* M_final, void* stream);
+
 /* Static description of a status code (never NULL). */
 E2TTT_API const char* e2ttt_status_string(int status);
 

@@ -52,6 +52,8 @@ def lib() -> ctypes.CDLL:
         L.e2ttt_chunk_fwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, tab, tab, vp, tab, tab, vp, ctypes.c_size_t, cp, vp]
         L.e2ttt_chunk_bwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, tab, tab, vp, tab, tab, vp, vp, vp, vp, vp, vp,
                                       tab, tab, vp, ctypes.c_size_t, cp, vp]
+        L.e2ttt_chunk_fwd_noalloc.argtypes = [pp, vp, vp, vp, vp, vp, vp, tab, tab, vp, tab, tab, vp]
+        L.e2ttt_chunk_fwd_noalloc.restype = cp
         L.e2ttt_status_string.argtypes = [cp]
         L.e2ttt_status_string.restype = ctypes.c_char_p
         L.e2ttt_version.argtypes = []
@@ -166,4 +168,23 @@ def e2ttt_chunk_bwd(p, q, k, v, eta, beta, gamma, W_init, M_init, d_o, dW_final,
         int(states_saved), _stream_ptr(stream))
     if st != E2TTT_OK:
         raise E2TTTError(st, "e2ttt_chunk_bwd")
+    return st
+
+
+E2TTT_NOALLOC_SCRATCH_BYTES = 8 << 20
+
+
+def e2ttt_chunk_fwd_noalloc(p, q, k, v, eta, beta, gamma, W_init, M_init, o, W_final, M_final, stream=None):
+    """int e2ttt_chunk_fwd_noalloc(...) of include/e2ttt.h: the forward for callers that cannot allocate a
+    workspace (the scratch is a fixed array inside the library).  Raises on error, e.g. E2TTT_ERR_WORKSPACE
+    when the shape needs more than E2TTT_NOALLOC_SCRATCH_BYTES."""
+    io = _io_torch_dtype(p)
+    s4, s3 = (p.B, p.H, p.L, p.d), (p.B, p.H, p.L)
+    st = lib().e2ttt_chunk_fwd_noalloc(
+        ctypes.byref(p), _ptr(q, io, s4, "q"), _ptr(k, io, s4, "k"), _ptr(v, io, s4, "v"),
+        _ptr(eta, torch.float32, s3, "eta"), _ptr(beta, torch.float32, s3, "beta"),
+        _ptr(gamma, torch.float32, s3, "gamma"), _table(W_init, p, "W_init"), _table(M_init, p, "M_init"),
+        _ptr(o, io, s4, "o"), _table(W_final, p, "W_final"), _table(M_final, p, "M_final"), _stream_ptr(stream))
+    if st != E2TTT_OK:
+        raise E2TTTError(st, "e2ttt_chunk_fwd_noalloc")
     return st
