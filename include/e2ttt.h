@@ -116,7 +116,8 @@ E2TTT_API int e2ttt_workspace_bytes(const e2ttt_params* p, int save_states, size
  *   W_final, M_final out  host tables, same layout as W_init; may alias W_init / M_init
  *   workspace        device scratch of at least e2ttt_workspace_bytes(p, save_states) bytes,
  *                    256-byte aligned; with save_states != 0 it holds, after the call, the
- *                    (W, M) at the start of every chunk for e2ttt_chunk_bwd
+ *                    (W, M) at the start of every chunk for e2ttt_chunk_bwd (a forward that
+ *                    saves states always runs on the SIMT path)
  */
 E2TTT_API int e2ttt_chunk_fwd(const e2ttt_params* p,
                     const void* q, const void* k, const void* v,
@@ -147,6 +148,14 @@ E2TTT_API int e2ttt_chunk_bwd(const e2ttt_params* p,
                     void* dq, void* dk, void* dv, float* d_eta, float* d_beta, float* d_gamma,
                     float* const* dW_init, float* const* dM_init,
                     void* workspace, size_t workspace_bytes, int states_saved, void* stream);
+
+/* Reads back the device status word of the last launch that used `workspace` (the first word of every
+ * workspace).  This is the one entry point that synchronises: it waits for `stream`.
+ *   status  out (host)  0 after a clean run; otherwise the code of the first bounded device-side wait
+ *                       that gave up (the tensor-core kernels never spin without a limit)
+ * Returns E2TTT_OK, E2TTT_ERR_TIMEOUT when the word is non-zero, or E2TTT_ERR_NULL / E2TTT_ERR_CUDA.
+ * (No counterpart in the paper: an operational guard of this implementation.) */
+E2TTT_API int e2ttt_device_status(const void* workspace, void* stream, int* status);
 
 /* Forward without any caller-provided scratch.  (The paper has no counterpart: this exists for the
  * library's users, not for the method.)

@@ -54,6 +54,8 @@ def lib() -> ctypes.CDLL:
                                       tab, tab, vp, ctypes.c_size_t, cp, vp]
         L.e2ttt_chunk_fwd_noalloc.argtypes = [pp, vp, vp, vp, vp, vp, vp, tab, tab, vp, tab, tab, vp]
         L.e2ttt_chunk_fwd_noalloc.restype = cp
+        L.e2ttt_device_status.argtypes = [vp, vp, ctypes.POINTER(cp)]
+        L.e2ttt_device_status.restype = cp
         L.e2ttt_status_string.argtypes = [cp]
         L.e2ttt_status_string.restype = ctypes.c_char_p
         L.e2ttt_version.argtypes = []
@@ -169,6 +171,15 @@ def e2ttt_chunk_bwd(p, q, k, v, eta, beta, gamma, W_init, M_init, d_o, dW_final,
     if st != E2TTT_OK:
         raise E2TTTError(st, "e2ttt_chunk_bwd")
     return st
+
+
+def e2ttt_device_status(workspace, stream=None) -> int:
+    """int e2ttt_device_status(...): waits for the stream and returns the device status word (0 = clean)."""
+    word = ctypes.c_int(-1)
+    st = lib().e2ttt_device_status(_ptr(workspace, torch.uint8, None, "workspace"), _stream_ptr(stream), ctypes.byref(word))
+    if st not in (E2TTT_OK, -8):
+        raise E2TTTError(st, "e2ttt_device_status")
+    return int(word.value)
 
 
 E2TTT_NOALLOC_SCRATCH_BYTES = 8 << 20

@@ -3,6 +3,7 @@
 
 #include "../../include/e2ttt.h"
 #include "simt_layout.h"
+#include "tc_fwd.h"
 
 using namespace e2ttt;
 
@@ -26,15 +27,21 @@ int check_params(const e2ttt_params* p) {
     return E2TTT_OK;
 }
 
-// 1 = tensor-core specialisation exists for these parameters
-int has_tcgen05(const e2ttt_params*) { return 0; }
+// Every workspace starts with a status block: word 0 is the device status of the last launch that used it.
+constexpr size_t kStatusBytes = 256;
 
-int pick_impl(const e2ttt_params* p, int* impl) {
+// 1 = a tensor-core specialisation exists for these parameters (forward without saved chunk states)
+int has_tcgen05(const e2ttt_params* p, bool save_states) {
+    return !save_states && p->kind == E2TTT_MLP_GELU && p->io_dtype == E2TTT_BF16 && p->d == 128 && p->h == 512 &&
+           p->C == 64 && p->L % 64 == 0;
+}
+
+int pick_impl(const e2ttt_params* p, bool save_states, int* impl) {
     if (p->impl == E2TTT_IMPL_TCGEN05) {
-        if (!has_tcgen05(p)) return E2TTT_ERR_SHAPE;
+        if (!has_tcgen05(p, save_states)) return E2TTT_ERR_SHAPE;
         *impl = E2TTT_IMPL_TCGEN05;
     } else if (p->impl == E2TTT_IMPL_AUTO) {
-        *impl = has_tcgen05(p) ? E2TTT_IMPL_TCGEN05 : E2TTT_IMPL_SIMT;
+        *impl = has_tcgen05(p, save_states) ? E2TTT_IMPL_TCGEN05 : E2TTT_IMPL_SIMT;
     } else {
         *impl = E2TTT_IMPL_SIMT;
     }
@@ -45,7 +52,7 @@ size_t simt_bytes(const e2ttt_params* p, bool save_states, bool backward) {
     const int nchunks = (p->L + p->C - 1) / p->C;
     SimtLayout l = simt_layout(p->d, p->h, p->C, nmat_of(p->kind), nchunks, save_states, backward);
     const size_t elem = (p->io_dtype == E2TTT_F32) ? sizeof(double) : sizeof(float);
-    return l.per_seq * elem * (size_t)p->B * p->H;
+    return kStatusBytes + l.per_seq * elem * (size_t)p->B * p->H;
 }
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
@@ -88,10 +95,11 @@ int e2ttt_workspace_bytes(const e2ttt_params* p, int save_states, size_t* bytes)
     int rc = check_params(p);
     if (rc) return rc;
     int impl = 0;
-    rc = pick_impl(p, &impl);
+    rc = pick_impl(p, save_states != 0, &impl);
     if (rc) return rc;
-    // with saved states the same buffer serves the backward, which needs the larger layout
-    *bytes = simt_bytes(p, save_states != 0, save_states != 0);
+    // tensor-core path: all state lives on chip, only the status block is needed.
+    // SIMT path: with saved states the same buffer serves the backward, which needs the larger layout.
+    *bytes = (impl == E2TTT_IMPL_TCGEN05) ? kStatusBytes : simt_bytes(p, save_states != 0, save_states != 0);
     return E2TTT_OK;
 }
 
@@ -108,7 +116,7 @@ int e2ttt_chunk_fwd(const e2ttt_params* p, const void* q, const void* k, const v
         if (M_init && !M_init[i]) return E2TTT_ERR_NULL;
     }
     int impl = 0;
-    rc = pick_impl(p, &impl);
+    rc = pick_impl(p, save_states != 0, &impl);
     if (rc) return rc;
     if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(o, 16)) return E2TTT_ERR_ALIGN;
     size_t need = 0;
@@ -119,12 +127,30 @@ int e2ttt_chunk_fwd(const e2ttt_params* p, const void* q, const void* k, const v
     rc = check_device();
     if (rc) return rc;
 
+    if (impl == E2TTT_IMPL_TCGEN05) {
+        TcFwdArgs t{};
+        t.N = p->B * p->H; t.L = p->L; t.eps = p->ln_eps;
+        t.q = static_cast<const __nv_bfloat16*>(q); t.k = static_cast<const __nv_bfloat16*>(k);
+        t.v = static_cast<const __nv_bfloat16*>(v); t.o = static_cast<__nv_bfloat16*>(o);
+        t.eta = eta; t.beta = beta; t.gamma = gamma;
+        t.W1_init = W_init[0]; t.W2_init = W_init[1];
+        t.M1_init = M_init ? M_init[0] : nullptr; t.M2_init = M_init ? M_init[1] : nullptr;
+        t.W1_final = W_final[0]; t.W2_final = W_final[1]; t.M1_final = M_final[0]; t.M2_final = M_final[1];
+        t.status = static_cast<int*>(workspace);
+        return tc_fwd_launch(t, stream) == 0 ? E2TTT_OK : E2TTT_ERR_CUDA;
+    }
+    if (cudaMemsetAsync(workspace, 0, sizeof(int), reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return E2TTT_ERR_CUDA;
+    }
+
     SimtFwdArgs a{};
     a.N = p->B * p->H; a.L = p->L; a.d = p->d; a.h = p->h; a.C = p->C;
     a.nchunks = (p->L + p->C - 1) / p->C;
     a.save_states = save_states != 0;
     a.eps = p->ln_eps;
-    a.q = q; a.k = k; a.v = v; a.eta = eta; a.beta = beta; a.gamma = gamma; a.o = o; a.ws = workspace;
+    a.q = q; a.k = k; a.v = v; a.eta = eta; a.beta = beta; a.gamma = gamma; a.o = o;
+    a.ws = static_cast<char*>(workspace) + kStatusBytes;
     for (int i = 0; i < nmat; ++i) {
         a.W_init[i] = W_init[i];
         a.M_init[i] = M_init ? M_init[i] : nullptr;
@@ -154,7 +180,7 @@ int e2ttt_chunk_bwd(const e2ttt_params* p, const void* q, const void* k, const v
         if (dM_final && !dM_final[i]) return E2TTT_ERR_NULL;
     }
     int impl = 0;
-    rc = pick_impl(p, &impl);
+    rc = pick_impl(p, true, &impl);
     if (rc) return rc;
     if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(d_o, 16) || !aligned(dq, 16) ||
         !aligned(dk, 16) || !aligned(dv, 16))
@@ -169,13 +195,18 @@ int e2ttt_chunk_bwd(const e2ttt_params* p, const void* q, const void* k, const v
 
     const int nchunks = (p->L + p->C - 1) / p->C;
     const SimtLayout lay = simt_layout(p->d, p->h, p->C, nmat, nchunks, true, true);
+    void* ws_data = static_cast<char*>(workspace) + kStatusBytes;
+    if (cudaMemsetAsync(workspace, 0, sizeof(int), reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return E2TTT_ERR_CUDA;
+    }
     if (!states_saved) {
         // recompute the chunk-start states: a forward whose outputs and final states land in scratch slots
         // that the reverse sweep overwrites later (the adjoint carries T, S and the accumulators Wb)
         SimtFwdArgs f{};
         f.N = p->B * p->H; f.L = p->L; f.d = p->d; f.h = p->h; f.C = p->C; f.nchunks = nchunks;
         f.save_states = 1; f.eps = p->ln_eps;
-        f.q = q; f.k = k; f.v = v; f.eta = eta; f.beta = beta; f.gamma = gamma; f.ws = workspace; f.lay = lay;
+        f.q = q; f.k = k; f.v = v; f.eta = eta; f.beta = beta; f.gamma = gamma; f.ws = ws_data; f.lay = lay;
         f.o = nullptr; // outputs are not needed
         for (int i = 0; i < nmat; ++i) {
             f.W_init[i] = W_init[i];
@@ -189,7 +220,7 @@ int e2ttt_chunk_bwd(const e2ttt_params* p, const void* q, const void* k, const v
     b.N = p->B * p->H; b.L = p->L; b.d = p->d; b.h = p->h; b.C = p->C; b.nchunks = nchunks; b.eps = p->ln_eps;
     b.q = q; b.k = k; b.v = v; b.d_o = d_o; b.eta = eta; b.beta = beta; b.gamma = gamma;
     b.dq = dq; b.dk = dk; b.dv = dv; b.d_eta = d_eta; b.d_beta = d_beta; b.d_gamma = d_gamma;
-    b.ws = workspace; b.lay = lay;
+    b.ws = ws_data; b.lay = lay;
     for (int i = 0; i < nmat; ++i) {
         b.dW_final[i] = dW_final ? dW_final[i] : nullptr;
         b.dM_final[i] = dM_final ? dM_final[i] : nullptr;
@@ -197,6 +228,19 @@ int e2ttt_chunk_bwd(const e2ttt_params* p, const void* q, const void* k, const v
         b.dM_init[i] = dM_init[i];
     }
     return simt_bwd_launch(b, p->kind, p->io_dtype, stream) == 0 ? E2TTT_OK : E2TTT_ERR_CUDA;
+}
+
+int e2ttt_device_status(const void* workspace, void* stream, int* status) {
+    if (!workspace || !status) return E2TTT_ERR_NULL;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    int word = 0;
+    if (cudaMemcpyAsync(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return E2TTT_ERR_CUDA;
+    }
+    *status = word;
+    return word == 0 ? E2TTT_OK : E2TTT_ERR_TIMEOUT;
 }
 
 const char* e2ttt_status_string(int status) {

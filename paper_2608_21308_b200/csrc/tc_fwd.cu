@@ -1,0 +1,653 @@
+// Tensor-core forward for GELU-MLP fast weights, d = 128, h = 512, C = 64, bf16 I/O (sm_100a).
+//
+// One cluster of 4 CTAs per sequence; CTA c owns hidden units [128c, 128c+128): rows of W1, columns of W2.
+// Everything that carries over from chunk to chunk stays on chip for the whole sequence:
+//   - fp32 master copy of the CTA's W1/W2 slices: tensor memory columns [0,256).  The aggregation MMAs
+//     accumulate -sum_t K^W_t grad_t straight into it (it is pre-scaled by the decay carry cw beforehand).
+//   - fp32 master copy of the momentum slices: registers (each thread keeps the 2 x 128/NG elements it owns).
+//   - bf16 operand copy of W1/W2: shared memory, refreshed once per chunk from the fp32 master.
+// Per chunk (Algorithm 1), rows = tokens (64 keys then 64 queries), all GEMMs on tcgen05 with TMEM accumulators:
+//   G1  Z = [K;Q] W1c^T          G2  Upart = gelu(Z) W2c^T      -> cross-CTA sum of Upart through DSMEM (each CTA
+//   owns 32 token rows: LN, output rows o = q + LN(u), or e = k + LN(u) - v and pu = dL/du), pu rows broadcast
+//   G3  Pa = Pu W2c, Pz = Pa * gelu'(Z)
+//   aggregations (contraction over the 64 tokens, MN-major operands):
+//       W1c -= (kW*Pz)^T K    M1acc = -(kM*Pz)^T K    W2c -= Pu^T (kW*Ak)    M2acc = -Pu^T (kM*Ak)
+//   state pass: W = Wacc + cm M0;  M = cb M0 + Macc;  bf16(W) -> shared;  cw_next W -> TMEM.
+// Every wait on an mbarrier is bounded (sm100.cuh); a wait that gives up is reported through the status word.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "simt_common.cuh"
+#include "sm100.cuh"
+#include "tc_fwd.h"
+
+namespace e2ttt {
+using namespace sm100;
+
+namespace {
+
+constexpr int D = 128, HC = 128, C = 64, NC = 4;
+constexpr int NG = TC_NG;                // column groups per TMEM lane quadrant
+constexpr int NTHREADS = 128 * NG;
+constexpr int CW = 128 / NG;             // accumulator columns a thread owns in a 128-column region
+constexpr int NB = CW / 16;              // 16-column batches per thread
+
+// TMEM columns
+constexpr uint32_t T_W1 = 0, T_W2 = 128, T_R0 = 256, T_R1 = 384;
+
+struct Scalars {
+    float kW[C], kM[C];
+    float cw, cm, cb, pad;
+};
+
+struct __align__(1024) Smem {
+    uint8_t W1[2][16384];  // bf16 W1c  [128 j][64 i] per slab (i = 64 s ..)         K-major B of G1
+    uint8_t W2[2][16384];  // bf16 W2c  [128 i][64 j] per slab (j = 64 s ..)         K-major B of G2, MN-major B of G3
+    uint8_t X[2][16384];   // [128 tokens][64 i] per slab; rows 0..63 keys, 64..127 queries (TMA)
+    uint8_t A[2][16384];   // bf16 gelu(Z) [128 tokens][64 j] per slab               K-major A of G2
+    uint8_t AkW[2][8192];  // kW_t gelu(Zk) [64 t][64 j] per slab                    MN-major B of the W2 aggregation
+    uint8_t AkM[2][8192];  // kM_t gelu(Zk)
+    uint8_t Pu[2][8192];   // bf16 pu [64 t][64 i] per slab                          K-major A of G3, MN-major A of the W2 aggregations
+    uint8_t PzW[2][8192];  // kW_t pz [64 t][64 j] per slab                          MN-major A of the W1 aggregation; staging slot 0
+    uint8_t PzM[2][8192];  // kM_t pz                                                 staging slot 1
+    uint8_t Stage2[16384]; // staging slot 2
+    Scalars sc[2];
+    float red[3][NG][32];
+    uint64_t bar_x, bar_g1, bar_g2, bar_g3, bar_agg, bar_part, bar_pu, bar_credit;
+    uint32_t tmem_base;
+    int dead;
+};
+
+__device__ __forceinline__ uint64_t desc_k(uint32_t base, uint32_t slab_stride, int k) {
+    return make_smem_desc(base + (uint32_t)(k >> 2) * slab_stride + (uint32_t)(k & 3) * 32u, 16, 1024);
+}
+__device__ __forceinline__ uint64_t desc_mn(uint32_t base, uint32_t slab_stride, int k) {
+    return make_smem_desc(base + (uint32_t)k * 2048u, slab_stride, 1024);
+}
+
+// Suffix scans of one 64-token chunk by one warp (two tokens per lane), same recurrences as the SIMT path:
+// a step is the map (bt, gt, S) -> (beta bt, gamma gt, beta S + gamma gt); suffix composites by warp shuffles.
+__device__ void tc_chunk_scalars(const float* eta, const float* beta, const float* gamma, Scalars* out) {
+    const int lane = threadIdx.x & 31;
+    ScanMap<float> e0, e1, id;
+    id.B = 1.0f; id.G = 1.0f; id.X = 0.0f;
+    e0.B = beta[2 * lane]; e0.G = gamma[2 * lane]; e0.X = e0.G;
+    e1.B = beta[2 * lane + 1]; e1.G = gamma[2 * lane + 1]; e1.X = e1.G;
+    const ScanMap<float> loc1 = e1;                 // tokens 2l+1 .. of this lane
+    const ScanMap<float> loc0 = compose(e0, loc1);  // tokens 2l ..   of this lane
+    ScanMap<float> incl = loc0;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        ScanMap<float> o;
+        o.B = __shfl_down_sync(0xffffffffu, incl.B, off);
+        o.G = __shfl_down_sync(0xffffffffu, incl.G, off);
+        o.X = __shfl_down_sync(0xffffffffu, incl.X, off);
+        if (lane + off < 32) incl = compose(incl, o);
+    }
+    ScanMap<float> excl;
+    excl.B = __shfl_down_sync(0xffffffffu, incl.B, 1);
+    excl.G = __shfl_down_sync(0xffffffffu, incl.G, 1);
+    excl.X = __shfl_down_sync(0xffffffffu, incl.X, 1);
+    if (lane == 31) excl = id;
+    // token index 2l sees the state after tokens 2l+1.., token 2l+1 the state after the later lanes' tokens
+    const ScanMap<float> f1 = compose(loc1, excl);
+    const float et0 = eta[2 * lane], et1 = eta[2 * lane + 1];
+    out->kW[2 * lane] = et0 * (f1.B + f1.X);
+    out->kM[2 * lane] = et0 * f1.B;
+    out->kW[2 * lane + 1] = et1 * (excl.B + excl.X);
+    out->kM[2 * lane + 1] = et1 * excl.B;
+    if (lane == 0) {
+        const ScanMap<float> f0 = compose(loc0, excl);
+        out->cw = f0.G;
+        out->cb = f0.B;
+        out->cm = e0.B * (f1.B + f1.X);  // beta_1 S_1
+    }
+}
+
+__device__ __forceinline__ float gelu_fast(float z, float& dgelu) {
+    // exact-erf GELU and its derivative (fp32 library erf/exp)
+    const float cdf = 0.5f * (1.0f + erff(z * 0.70710678118654752440f));
+    const float pdf = 0.39894228040143267794f * __expf(-0.5f * z * z);
+    dgelu = cdf + z * pdf;
+    return z * cdf;
+}
+
+// 16 bf16 (32 bytes) = two 16-byte chunks into a swizzled slab row
+__device__ __forceinline__ void st_slab16(uint8_t* slab, int row, int col0, const float (&v)[16]) {
+    const int c = col0 >> 3;
+    uint4 a, b;
+    a.x = pack_bf16(v[0], v[1]); a.y = pack_bf16(v[2], v[3]); a.z = pack_bf16(v[4], v[5]); a.w = pack_bf16(v[6], v[7]);
+    b.x = pack_bf16(v[8], v[9]); b.y = pack_bf16(v[10], v[11]); b.z = pack_bf16(v[12], v[13]); b.w = pack_bf16(v[14], v[15]);
+    *reinterpret_cast<uint4*>(slab + row * 128 + (((c) ^ (row & 7)) << 4)) = a;
+    *reinterpret_cast<uint4*>(slab + row * 128 + (((c + 1) ^ (row & 7)) << 4)) = b;
+}
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ, const TcFwdArgs a) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    Smem& s = *reinterpret_cast<Smem*>(smem_raw);
+    if ((smem_u32(smem_raw) & 1023u) != 0u) {  // the swizzled tiles need a 1024-byte aligned base: refuse to run otherwise
+        if (threadIdx.x == 0) atomicCAS(a.status, 0, 99);
+        return;
+    }
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int q = warp & 3;          // TMEM lane quadrant
+    const int g = warp >> 2;         // column group
+    const int row = 32 * q + lane;   // TMEM lane this thread reads
+    const int c0 = CW * g;           // first of its columns inside a 128-column region
+    const uint32_t me = cluster_ctarank();
+    const int seq = blockIdx.x / NC;
+    const int issuer_warp = (int)((me + 1) & 3);  // a warp that never owns layer-norm rows of this CTA
+    const bool is_issuer = (warp == issuer_warp) && (lane == 0);
+    const bool ln_owner = (q == (int)me);
+    const int L = a.L, nchunks = L / C;
+    WaitCtx wc{&s.dead, a.status};
+
+    const __nv_bfloat16* gk = a.k + (size_t)seq * L * D;
+    const __nv_bfloat16* gv = a.v + (size_t)seq * L * D;
+    const __nv_bfloat16* gq = a.q + (size_t)seq * L * D;
+    __nv_bfloat16* go = a.o + (size_t)seq * L * D;
+    const float* eta = a.eta + (size_t)seq * L;
+    const float* beta = a.beta + (size_t)seq * L;
+    const float* gamma = a.gamma + (size_t)seq * L;
+
+    if (tid == 0) {
+        s.dead = 0;
+        mbar_init(&s.bar_x, 1);
+        mbar_init(&s.bar_g1, 1);
+        mbar_init(&s.bar_g2, 1);
+        mbar_init(&s.bar_g3, 1);
+        mbar_init(&s.bar_agg, 1);
+        mbar_init(&s.bar_part, 3 * NG);
+        mbar_init(&s.bar_pu, 2 * NG);
+        mbar_init(&s.bar_credit, 3);
+        fence_mbar_init();
+        tma_prefetch_desc(&tmK);
+        tma_prefetch_desc(&tmQ);
+    }
+    if (warp == 0) { tmem_alloc(&s.tmem_base, 512); tmem_relinquish(); }
+    if (warp == 1) tc_chunk_scalars(eta, beta, gamma, &s.sc[0]);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tb = s.tmem_base;
+    const uint32_t lane_addr = tb + ((uint32_t)(32 * q) << 16);
+
+    // ---- load the state: fp32 master of W -> TMEM (pre-scaled by the first decay carry) and bf16 -> shared; M -> registers
+    float M1[CW], M2[CW];
+    {
+        const float cw0 = s.sc[0].cw;
+        const size_t head = (size_t)seq * (size_t)(D * 4 * HC);
+        // W1c[j][i]: global W1 [h][d], row 128 me + j
+        const float* w1 = a.W1_init + head + ((size_t)(HC * me) + row) * D + c0;
+        const float* m1 = a.M1_init ? a.M1_init + head + ((size_t)(HC * me) + row) * D + c0 : nullptr;
+        // W2c[i][j]: global W2 [d][h], row i, column 128 me + j
+        const float* w2 = a.W2_init + head + (size_t)row * (4 * HC) + HC * me + c0;
+        const float* m2 = a.M2_init ? a.M2_init + head + (size_t)row * (4 * HC) + HC * me + c0 : nullptr;
+#pragma unroll
+        for (int b = 0; b < NB; ++b) {
+            float w[16];
+            uint32_t st[16];
+#pragma unroll
+            for (int j = 0; j < 16; j += 4) {
+                const float4 x = *reinterpret_cast<const float4*>(w1 + 16 * b + j);
+                w[j] = x.x; w[j + 1] = x.y; w[j + 2] = x.z; w[j + 3] = x.w;
+            }
+#pragma unroll
+            for (int j = 0; j < 16; ++j) { st[j] = __float_as_uint(cw0 * w[j]); M1[16 * b + j] = m1 ? m1[16 * b + j] : 0.0f; }
+            tmem_st16(lane_addr + T_W1 + c0 + 16 * b, st);
+            st_slab16(s.W1[(c0 + 16 * b) >> 6], row, (c0 + 16 * b) & 63, w);
+#pragma unroll
+            for (int j = 0; j < 16; j += 4) {
+                const float4 x = *reinterpret_cast<const float4*>(w2 + 16 * b + j);
+                w[j] = x.x; w[j + 1] = x.y; w[j + 2] = x.z; w[j + 3] = x.w;
+            }
+#pragma unroll
+            for (int j = 0; j < 16; ++j) { st[j] = __float_as_uint(cw0 * w[j]); M2[16 * b + j] = m2 ? m2[16 * b + j] : 0.0f; }
+            tmem_st16(lane_addr + T_W2 + c0 + 16 * b, st);
+            st_slab16(s.W2[(c0 + 16 * b) >> 6], row, (c0 + 16 * b) & 63, w);
+        }
+        tmem_wait_st();
+    }
+    if (is_issuer) {
+        mbar_expect_tx(&s.bar_x, 32768);
+        const int y = seq * L;
+        tma_load_2d(s.X[0], &tmK, 0, y, &s.bar_x);
+        tma_load_2d(s.X[1], &tmK, 64, y, &s.bar_x);
+        tma_load_2d(s.X[0] + 8192, &tmQ, 0, y, &s.bar_x);
+        tma_load_2d(s.X[1] + 8192, &tmQ, 64, y, &s.bar_x);
+    }
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+    // every CTA's barriers are initialised before any peer may arrive on them
+    cluster_sync();
+    tc_fence_after_sync();
+
+    const uint32_t id_kk = make_idesc(128, 128, false, false);
+    const uint32_t id_kmn = make_idesc(128, 128, false, true);
+    const uint32_t id_agg = make_idesc(128, 128, true, true) | (1u << 13);  // negate A: G_t is minus the gradient
+
+    for (int r = 0; r < nchunks; ++r) {
+        const uint32_t ph = (uint32_t)(r & 1);
+        const Scalars& sc = s.sc[r & 1];
+        const int tok0 = r * C;
+
+        // scalars of the next chunk (suffix scans over its gates), by a warp that is not the issuer
+        if (warp == ((issuer_warp + 2) & 3) + 4 * (NG - 1) && r + 1 < nchunks) {
+            tc_chunk_scalars(eta + tok0 + C, beta + tok0 + C, gamma + tok0 + C, &s.sc[(r + 1) & 1]);
+        }
+
+        // ---------------- G1: Z = X W1c^T -> R0
+        if (is_issuer) {
+            mbar_wait(&s.bar_x, ph, wc, 100 + 1);
+            tc_fence_after_sync();
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                umma_bf16(tb + T_R0, desc_k(smem_u32(s.X[0]), 16384, k), desc_k(smem_u32(s.W1[0]), 16384, k), id_kk, k > 0);
+            umma_commit(&s.bar_g1);
+        }
+        mbar_wait(&s.bar_g1, ph, wc, 100 + 2);
+        __syncwarp();
+        tc_fence_after_sync();
+        // epilogue: a = gelu(z) -> A (bf16); for key rows also kW a, kM a and gelu'(z) (kept in TMEM over z)
+        {
+            const bool key_row = row < C;
+            const float kw = key_row ? sc.kW[row] : 0.0f, km = key_row ? sc.kM[row] : 0.0f;
+#pragma unroll
+            for (int b = 0; b < NB; ++b) {
+                uint32_t z[16];
+                tmem_ld16(lane_addr + T_R0 + c0 + 16 * b, z);
+                tmem_wait_ld();
+                float av[16], aw[16], am[16];
+                uint32_t dg[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    float d1;
+                    av[j] = gelu_fast(__uint_as_float(z[j]), d1);
+                    dg[j] = __float_as_uint(d1);
+                    aw[j] = kw * av[j];
+                    am[j] = km * av[j];
+                }
+                const int col = c0 + 16 * b;
+                st_slab16(s.A[col >> 6], row, col & 63, av);
+                if (key_row) {
+                    st_slab16(s.AkW[col >> 6], row, col & 63, aw);
+                    st_slab16(s.AkM[col >> 6], row, col & 63, am);
+                    tmem_st16(lane_addr + T_R0 + col, dg);
+                }
+            }
+            tmem_wait_st();
+        }
+        fence_proxy_async_smem();
+        tc_fence_before_sync();
+        __syncthreads();
+
+        // ---------------- G2: Upart = A W2c^T -> R1
+        if (is_issuer) {
+            tc_fence_after_sync();
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                umma_bf16(tb + T_R1, desc_k(smem_u32(s.A[0]), 16384, k), desc_k(smem_u32(s.W2[0]), 16384, k), id_kk, k > 0);
+            umma_commit(&s.bar_g2);
+        }
+        mbar_wait(&s.bar_g2, ph, wc, 100 + 3);
+        __syncwarp();
+        tc_fence_after_sync();
+
+        // ---------------- cross-CTA sum of Upart: rows of quadrant x go to CTA x
+        float own[CW];
+        if (r > 0) mbar_wait(&s.bar_credit, (uint32_t)((r - 1) & 1), wc, 100 + 4);
+        __syncwarp();
+        {
+            const uint32_t slot = (me - (uint32_t)q - 1u) & 3u;  // where CTA q keeps what comes from me
+            uint32_t dst_base = 0;
+            if (!ln_owner) {
+                const uint8_t* p = (slot == 0) ? s.PzW[0] : (slot == 1) ? s.PzM[0] : s.Stage2;
+                dst_base = map_to_cta(smem_u32(p), (uint32_t)q);
+            }
+#pragma unroll
+            for (int b = 0; b < NB; ++b) {
+                uint32_t u[16];
+                tmem_ld16(lane_addr + T_R1 + c0 + 16 * b, u);
+                tmem_wait_ld();
+                if (ln_owner) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) own[16 * b + j] = __uint_as_float(u[j]);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 16; j += 4) {
+                        const int c4 = (c0 + 16 * b + j) >> 2;
+                        st_cluster_v4_b32(dst_base + (uint32_t)(c4 * 32 + lane) * 16u, u[j], u[j + 1], u[j + 2], u[j + 3]);
+                    }
+                }
+            }
+            if (!ln_owner) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive_remote(map_to_cta(smem_u32(&s.bar_part), (uint32_t)q));
+            }
+        }
+        tc_fence_before_sync();
+        __syncthreads();  // R1 has been read by everyone: G3 may overwrite it
+
+        // ---------------- layer norm on the 32 rows this CTA owns (the warps of quadrant `me`)
+        if (ln_owner) {
+            mbar_wait(&s.bar_part, ph, wc, 100 + 5);
+            __syncwarp();
+            float u[CW];
+#pragma unroll
+            for (int j = 0; j < CW; ++j) u[j] = 0.0f;
+#pragma unroll
+            for (int src = 0; src < NC; ++src) {  // fixed order: the sum does not depend on arrival order
+                if (src == (int)me) {
+#pragma unroll
+                    for (int j = 0; j < CW; ++j) u[j] += own[j];
+                } else {
+                    const uint32_t slot = ((uint32_t)src - me - 1u) & 3u;
+                    const uint8_t* p = (slot == 0) ? s.PzW[0] : (slot == 1) ? s.PzM[0] : s.Stage2;
+#pragma unroll
+                    for (int j = 0; j < CW; j += 4) {
+                        const float4 x = *reinterpret_cast<const float4*>(p + (size_t)(((c0 + j) >> 2) * 32 + lane) * 16);
+                        u[j] += x.x; u[j + 1] += x.y; u[j + 2] += x.z; u[j + 3] += x.w;
+                    }
+                }
+            }
+            // row statistics: each of the NG warps holds CW columns of every row
+            auto row_sum = [&](float v, int round) -> float {
+                s.red[round][g][lane] = v;
+                asm volatile("bar.sync 1, %0;" ::"r"(32 * NG) : "memory");
+                float t = 0.0f;
+#pragma unroll
+                for (int gg = 0; gg < NG; ++gg) t += s.red[round][gg][lane];
+                return t;
+            };
+            float sum = 0.0f;
+#pragma unroll
+            for (int j = 0; j < CW; ++j) sum += u[j];
+            const float mu = row_sum(sum, 0) * (1.0f / D);
+            float vs = 0.0f;
+#pragma unroll
+            for (int j = 0; j < CW; ++j) { u[j] -= mu; vs += u[j] * u[j]; }
+            const float rstd = rsqrtf(row_sum(vs, 1) * (1.0f / D) + a.eps);
+#pragma unroll
+            for (int j = 0; j < CW; ++j) u[j] *= rstd;  // y
+            if (me < 2) {
+                // key rows: e = k + y - v, pu = rstd (e - mean(e) - y mean(e y))
+                const int t = 32 * (int)me + lane;
+                const size_t off = (size_t)(tok0 + t) * D + c0;
+                float e[CW];
+                float se = 0.0f, sey = 0.0f;
+#pragma unroll
+                for (int j = 0; j < CW; j += 8) {
+                    const uint4 kk = *reinterpret_cast<const uint4*>(gk + off + j);
+                    const uint4 vv = *reinterpret_cast<const uint4*>(gv + off + j);
+                    const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&kk);
+                    const __nv_bfloat162* v2 = reinterpret_cast<const __nv_bfloat162*>(&vv);
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) {
+                        const float2 kf = __bfloat1622float2(k2[x]), vf = __bfloat1622float2(v2[x]);
+                        e[j + 2 * x] = kf.x + u[j + 2 * x] - vf.x;
+                        e[j + 2 * x + 1] = kf.y + u[j + 2 * x + 1] - vf.y;
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < CW; ++j) { se += e[j]; sey += e[j] * u[j]; }
+                const float me_ = row_sum(se, 2) * (1.0f / D);
+                const float mey = row_sum(sey, 0) * (1.0f / D);  // plane 0 was last read two barriers ago
+                // broadcast the bf16 pu row piece to every CTA of the cluster
+                uint32_t pk[CW / 2];
+#pragma unroll
+                for (int j = 0; j < CW; j += 2)
+                    pk[j / 2] = pack_bf16(rstd * (e[j] - me_ - u[j] * mey), rstd * (e[j + 1] - me_ - u[j + 1] * mey));
+                const uint32_t pu_local = smem_u32(s.Pu[c0 >> 6]);
+#pragma unroll
+                for (uint32_t dst = 0; dst < NC; ++dst) {
+                    const uint32_t base = map_to_cta(pu_local, dst) + (uint32_t)t * 128u;
+#pragma unroll
+                    for (int ch = 0; ch < CW / 8; ++ch) {
+                        const uint32_t c = (uint32_t)(((c0 & 63) >> 3) + ch);
+                        st_cluster_v4_b32(base + ((c ^ ((uint32_t)t & 7u)) << 4), pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2],
+                                          pk[4 * ch + 3]);
+                    }
+                }
+                asm volatile("fence.proxy.async;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) {
+#pragma unroll
+                    for (uint32_t dst = 0; dst < NC; ++dst) mbar_arrive_remote(map_to_cta(smem_u32(&s.bar_pu), dst));
+                }
+            } else {
+                // query rows: o = q + y
+                const int t = 32 * ((int)me - 2) + lane;
+                const size_t off = (size_t)(tok0 + t) * D + c0;
+#pragma unroll
+                for (int j = 0; j < CW; j += 8) {
+                    const uint4 qq = *reinterpret_cast<const uint4*>(gq + off + j);
+                    const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&qq);
+                    uint4 ov;
+                    uint32_t* o32 = reinterpret_cast<uint32_t*>(&ov);
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) {
+                        const float2 qf = __bfloat1622float2(q2[x]);
+                        o32[x] = pack_bf16(qf.x + u[j + 2 * x], qf.y + u[j + 2 * x + 1]);
+                    }
+                    *reinterpret_cast<uint4*>(go + off + j) = ov;
+                }
+            }
+        }
+
+        // ---------------- G3: Pa = Pu W2c -> R1 ; then the W2 aggregation that needs nothing else
+        if (is_issuer) {
+            mbar_wait(&s.bar_pu, ph, wc, 100 + 6);
+            asm volatile("fence.proxy.async;" ::: "memory");
+            tc_fence_after_sync();
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                umma_bf16(tb + T_R1, desc_k(smem_u32(s.Pu[0]), 8192, k), desc_mn(smem_u32(s.W2[0]), 16384, k), id_kmn, k > 0);
+            umma_commit(&s.bar_g3);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                umma_bf16(tb + T_W2, desc_mn(smem_u32(s.Pu[0]), 8192, k), desc_mn(smem_u32(s.AkW[0]), 8192, k), id_agg, true);
+        }
+        mbar_wait(&s.bar_g3, ph, wc, 100 + 7);
+        __syncwarp();
+        tc_fence_after_sync();
+        if (row < C) {
+            const float kw = sc.kW[row], km = sc.kM[row];
+#pragma unroll
+            for (int b = 0; b < NB; ++b) {
+                uint32_t pa[16], dg[16];
+                tmem_ld16(lane_addr + T_R1 + c0 + 16 * b, pa);
+                tmem_ld16(lane_addr + T_R0 + c0 + 16 * b, dg);
+                tmem_wait_ld();
+                float pw[16], pm[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const float pz = __uint_as_float(pa[j]) * __uint_as_float(dg[j]);
+                    pw[j] = kw * pz;
+                    pm[j] = km * pz;
+                }
+                const int col = c0 + 16 * b;
+                st_slab16(s.PzW[col >> 6], row, col & 63, pw);
+                st_slab16(s.PzM[col >> 6], row, col & 63, pm);
+            }
+        }
+        fence_proxy_async_smem();
+        tc_fence_before_sync();
+        __syncthreads();
+
+        // ---------------- remaining aggregations
+        if (is_issuer) {
+            tc_fence_after_sync();
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                umma_bf16(tb + T_W1, desc_mn(smem_u32(s.PzW[0]), 8192, k), desc_mn(smem_u32(s.X[0]), 16384, k), id_agg, true);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                umma_bf16(tb + T_R0, desc_mn(smem_u32(s.PzM[0]), 8192, k), desc_mn(smem_u32(s.X[0]), 16384, k), id_agg, k > 0);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                umma_bf16(tb + T_R1, desc_mn(smem_u32(s.Pu[0]), 8192, k), desc_mn(smem_u32(s.AkM[0]), 8192, k), id_agg, k > 0);
+            umma_commit(&s.bar_agg);
+        }
+        mbar_wait(&s.bar_agg, ph, wc, 100 + 8);
+        __syncwarp();
+        tc_fence_after_sync();
+        if (is_issuer) {
+            // peers may now overwrite this CTA's staging / Pu buffers; the next chunk's tokens may land in X
+#pragma unroll
+            for (uint32_t dst = 0; dst < NC; ++dst)
+                if (dst != me) mbar_arrive_remote(map_to_cta(smem_u32(&s.bar_credit), dst));
+            if (r + 1 < nchunks) {
+                mbar_expect_tx(&s.bar_x, 32768);
+                const int y = seq * L + tok0 + C;
+                tma_load_2d(s.X[0], &tmK, 0, y, &s.bar_x);
+                tma_load_2d(s.X[1], &tmK, 64, y, &s.bar_x);
+                tma_load_2d(s.X[0] + 8192, &tmQ, 0, y, &s.bar_x);
+                tma_load_2d(s.X[1] + 8192, &tmQ, 64, y, &s.bar_x);
+            }
+        }
+        __syncwarp();
+
+        // ---------------- state pass (Algorithm 1 lines 6-7)
+        {
+            const bool last = (r + 1 == nchunks);
+            const float cm = sc.cm, cb = sc.cb;
+            const float cwn = last ? 1.0f : s.sc[(r + 1) & 1].cw;
+            const size_t head = (size_t)seq * (size_t)(D * 4 * HC);
+#pragma unroll
+            for (int b = 0; b < NB; ++b) {
+                const int col = c0 + 16 * b;
+                uint32_t wa[16], ma[16], st[16];
+                float wn[16];
+                tmem_ld16(lane_addr + T_W1 + col, wa);
+                tmem_ld16(lane_addr + T_R0 + col, ma);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const float m0 = M1[16 * b + j];
+                    wn[j] = __uint_as_float(wa[j]) + cm * m0;
+                    M1[16 * b + j] = cb * m0 + __uint_as_float(ma[j]);
+                    st[j] = __float_as_uint(cwn * wn[j]);
+                }
+                tmem_st16(lane_addr + T_W1 + col, st);
+                st_slab16(s.W1[col >> 6], row, col & 63, wn);
+                if (last) {
+                    float* wf = a.W1_final + head + ((size_t)(HC * me) + row) * D + col;
+                    float* mf = a.M1_final + head + ((size_t)(HC * me) + row) * D + col;
+#pragma unroll
+                    for (int j = 0; j < 16; j += 4) {
+                        *reinterpret_cast<float4*>(wf + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
+                        *reinterpret_cast<float4*>(mf + j) =
+                            make_float4(M1[16 * b + j], M1[16 * b + j + 1], M1[16 * b + j + 2], M1[16 * b + j + 3]);
+                    }
+                }
+                tmem_ld16(lane_addr + T_W2 + col, wa);
+                tmem_ld16(lane_addr + T_R1 + col, ma);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const float m0 = M2[16 * b + j];
+                    wn[j] = __uint_as_float(wa[j]) + cm * m0;
+                    M2[16 * b + j] = cb * m0 + __uint_as_float(ma[j]);
+                    st[j] = __float_as_uint(cwn * wn[j]);
+                }
+                tmem_st16(lane_addr + T_W2 + col, st);
+                st_slab16(s.W2[col >> 6], row, col & 63, wn);
+                if (last) {
+                    float* wf = a.W2_final + head + (size_t)row * (4 * HC) + HC * me + col;
+                    float* mf = a.M2_final + head + (size_t)row * (4 * HC) + HC * me + col;
+#pragma unroll
+                    for (int j = 0; j < 16; j += 4) {
+                        *reinterpret_cast<float4*>(wf + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
+                        *reinterpret_cast<float4*>(mf + j) =
+                            make_float4(M2[16 * b + j], M2[16 * b + j + 1], M2[16 * b + j + 2], M2[16 * b + j + 3]);
+                    }
+                }
+            }
+            tmem_wait_st();
+        }
+        fence_proxy_async_smem();
+        tc_fence_before_sync();
+        __syncthreads();
+        tc_fence_after_sync();
+    }
+
+    // no CTA leaves while a peer may still write into its shared memory or arrive on its barriers
+    tc_fence_before_sync();
+    cluster_sync();
+    if (warp == 0) tmem_dealloc(tb, 512);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) != cudaSuccess ||
+            qr != cudaDriverEntryPointSuccess) {
+            (void)cudaGetLastError();
+            return nullptr;
+        }
+        fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// [rows][128] bf16 row-major, tiles of 64 rows x 64 columns, 128-byte swizzle
+bool make_token_map(CUtensorMap* tm, const void* base, size_t rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)D * 2};
+    cuuint32_t box[2] = {64, 64};
+    cuuint32_t es[2] = {1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+size_t tc_fwd_smem_bytes() { return sizeof(Smem); }
+
+int tc_fwd_launch(const TcFwdArgs& a, void* stream) {
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    CUtensorMap tmK, tmQ;
+    const size_t rows = (size_t)a.N * a.L;
+    if (!make_token_map(&tmK, a.k, rows) || !make_token_map(&tmQ, a.q, rows)) return (int)cudaErrorInvalidValue;
+    static bool attr_done[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return (int)cudaGetLastError();
+    const int smem = (int)tc_fwd_smem_bytes();
+    if (dev < 0 || dev >= 64 || !attr_done[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return (int)e;
+        if (dev >= 0 && dev < 64) attr_done[dev] = true;
+    }
+    cudaError_t e = cudaMemsetAsync(a.status, 0, sizeof(int), st);
+    if (e != cudaSuccess) return (int)e;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)(a.N * NC));
+    cfg.blockDim = dim3(NTHREADS);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = NC;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, tc_fwd_kernel, tmK, tmQ, a);
+    if (e != cudaSuccess) return (int)e;
+    return (int)cudaGetLastError();
+}
+
+}  // namespace e2ttt

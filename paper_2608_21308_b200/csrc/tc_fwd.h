@@ -1,0 +1,27 @@
+// Host interface of the tensor-core forward (tc_fwd.cu).
+#pragma once
+#include <cuda_bf16.h>
+#include <stddef.h>
+
+#ifndef TC_NG
+#define TC_NG 4  // column groups per tensor-memory lane quadrant: the kernel runs 128 * TC_NG threads
+#endif
+
+namespace e2ttt {
+
+struct TcFwdArgs {
+    int N, L;  // sequences, tokens per sequence (L a multiple of 64)
+    float eps;
+    const __nv_bfloat16 *q, *k, *v;
+    const float *eta, *beta, *gamma;
+    const float *W1_init, *W2_init, *M1_init, *M2_init;  // M*_init may be nullptr (zeros)
+    __nv_bfloat16* o;
+    float *W1_final, *W2_final, *M1_final, *M2_final;
+    int* status;  // device word, 0 after a clean run
+};
+
+size_t tc_fwd_smem_bytes();
+// returns a cudaError_t value as int (0 = launched)
+int tc_fwd_launch(const TcFwdArgs& a, void* stream);
+
+}  // namespace e2ttt

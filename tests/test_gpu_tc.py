@@ -1,0 +1,62 @@
+"""Tensor-core forward (tcgen05 path) against the fp64 oracle and against the SIMT path."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_21308_b200 import binding as E
+from paper_2608_21308_b200 import inputs
+from tests import util
+from tests.test_gpu_parity import TOL_BF16, check_forward
+
+pytestmark = pytest.mark.gpu
+MLP = inputs.KIND_MLP
+SHAPE = dict(d=128, h=512, C=64, kind=MLP, io="bf16")
+
+
+def test_tc_is_selected_and_reports_clean_status():
+    r = inputs.config(2, heads=[5], L=128)
+    x = inputs.generate(r)
+    got, hd = util.gpu_forward(x, impl=E.E2TTT_IMPL_TCGEN05, **SHAPE)
+    assert hd["ws"].numel() == 256                      # tensor-core path: status block only
+    assert E.e2ttt_device_status(hd["ws"]) == 0
+    assert np.isfinite(got["o"]).all()
+
+
+@pytest.mark.parametrize("window", [1, 2])
+def test_tc_windows_match_oracle_and_simt(window):
+    r = inputs.config(2, heads=[3, 30], m_std=0.002)
+    xw, ref = util.teacher_forced_windows(r, 4, window=window)
+    tc, hd = util.gpu_forward(xw, impl=E.E2TTT_IMPL_TCGEN05, **SHAPE)
+    assert E.e2ttt_device_status(hd["ws"]) == 0
+    simt, _ = util.gpu_forward(xw, impl=E.E2TTT_IMPL_SIMT, **SHAPE)
+    tol = TOL_BF16 if window == 1 else 3 * TOL_BF16   # two chunks: the map's own amplification of bf16 rounding
+    errs = check_forward(tc, ref, tol, f"tc window {window}")
+    check_forward(simt, ref, tol, f"simt window {window}")
+    print("tc", errs)
+
+
+def test_tc_free_running_paper_regime():
+    r = inputs.paper_regime(inputs.Recipe(B=3, H=1, L=1024, d=128, h=512, C=64, kind=MLP, io="bf16", seed=4, m_std=0.002))
+    x = inputs.generate(r)
+    ref = util.oracle_forward(x, 64, MLP)
+    tc, hd = util.gpu_forward(x, impl=E.E2TTT_IMPL_TCGEN05, **SHAPE)
+    assert E.e2ttt_device_status(hd["ws"]) == 0
+    check_forward(tc, ref, TOL_BF16, "tc paper regime, 16 chunks free-running")
+
+
+def test_tc_null_momentum_determinism_and_many_sequences():
+    r = inputs.config(2, heads=list(range(40)), L=256)       # 40 clusters: more than one wave of clusters is not needed, just many
+    x = inputs.generate(r)
+    a, hd = util.gpu_forward(x, impl=E.E2TTT_IMPL_TCGEN05, use_M=False, **SHAPE)
+    b, _ = util.gpu_forward(x, impl=E.E2TTT_IMPL_TCGEN05, use_M=False, **SHAPE)
+    assert E.e2ttt_device_status(hd["ws"]) == 0
+    assert np.array_equal(a["o"], b["o"])
+    for i in range(2):
+        assert np.array_equal(a["W"][i], b["W"][i]) and np.array_equal(a["M"][i], b["M"][i])
+    solo = {n: (np.ascontiguousarray(v[7:8]) if not isinstance(v, list) else [m[7:8] for m in v]) for n, v in x.items()}
+    c, _ = util.gpu_forward(solo, impl=E.E2TTT_IMPL_TCGEN05, use_M=False, **SHAPE)
+    assert np.array_equal(c["o"][0], a["o"][7])
+    # first chunk of every sequence against the oracle (no amplification yet)
+    first = {n: (np.ascontiguousarray(v[:, :64]) if not isinstance(v, list) else v) for n, v in x.items()}
+    ref = util.oracle_forward(first, 64, MLP, use_M=False)
+    assert util.rel_err(a["o"][:, :64], ref["o"]) <= TOL_BF16

@@ -52,7 +52,7 @@ def test_noalloc_forward_matches_the_ordinary_entry_point_twice_in_a_row():
 
 
 def test_noalloc_refuses_shapes_beyond_its_fixed_scratch():
-    p = E.make_params(4, 16, 64, 128, 512, 64, io_dtype=E.E2TTT_BF16)
+    p = E.make_params(4, 16, 64, 128, 512, 64, io_dtype=E.E2TTT_BF16, impl=E.E2TTT_IMPL_SIMT)  # SIMT scratch: ~100 MB
     assert E.e2ttt_workspace_bytes(p, 0) > E.E2TTT_NOALLOC_SCRATCH_BYTES
     t4 = torch.zeros(4, 16, 64, 128, device="cuda", dtype=torch.bfloat16)
     t3 = torch.zeros(4, 16, 64, device="cuda")
