@@ -26,15 +26,33 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// the same without ordering of its own: pair it with one fence_cluster() before a group of arrives
+__device__ __forceinline__ void mbar_arrive_remote_relaxed(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void fence_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
+// Probe of a barrier phase.  CLUSTER = true gives the acquire cluster scope (needed only when the data guarded by the
+// barrier was written by another CTA of the cluster; it is several hundred cycles dearer than the CTA-scope form).
+template <bool CLUSTER>
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
+    if (CLUSTER) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(smem_u32(bar)), "r"(parity)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(smem_u32(bar)), "r"(parity)
+            : "memory");
+    }
     return ok != 0;
 }
 
@@ -47,13 +65,15 @@ struct WaitCtx {
 };
 constexpr long long kWaitCycles = 2000000000LL;  // ~1 s at B200 clocks
 
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const WaitCtx& w, int where) {
+// Single-thread wait (the caller is one elected lane).
+template <bool CLUSTER = false>
+__device__ __forceinline__ bool mbar_wait_one(uint64_t* bar, uint32_t parity, const WaitCtx& w, int where) {
     if (*w.dead) return false;
-    if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait<CLUSTER>(bar, parity)) return true;
     const long long t0 = clock64();
     int spins = 0;
-    while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 255) == 0) {
+    while (!mbar_try_wait<CLUSTER>(bar, parity)) {
+        if ((++spins & 63) == 0) {
             if (*w.dead) return false;
             if (clock64() - t0 > kWaitCycles) {
                 *w.dead = 1;
@@ -63,6 +83,13 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const 
         }
     }
     return true;
+}
+// Warp-collective wait (all 32 lanes call it together): lane 0 waits, the others park at the warp barrier, which
+// also orders their later reads after lane 0's acquire.
+template <bool CLUSTER = false>
+__device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, const WaitCtx& w, int where) {
+    if ((threadIdx.x & 31) == 0) mbar_wait_one<CLUSTER>(bar, parity, w, where);
+    __syncwarp();
 }
 
 // ------------------------------------------------------------------ proxies and fences
@@ -199,6 +226,14 @@ __device__ __forceinline__ void st_cluster_v4(uint32_t cluster_addr, float a, fl
 }
 __device__ __forceinline__ void st_cluster_v4_b32(uint32_t cluster_addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+// Asynchronous 16-byte store into the shared memory of a CTA of the cluster; the destination's mbarrier (same CTA
+// as the data) gets 16 bytes of its expected transaction count when the data has landed.  No fence, no arrive.
+__device__ __forceinline__ void st_async_v4(uint32_t cluster_addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d,
+                                            uint32_t cluster_mbar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
+                 ::"r"(cluster_addr), "r"(a), "r"(b), "r"(c), "r"(d), "r"(cluster_mbar)
+                 : "memory");
 }
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }

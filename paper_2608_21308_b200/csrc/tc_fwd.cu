@@ -25,6 +25,17 @@
 namespace e2ttt {
 using namespace sm100;
 
+#ifdef TC_PROFILE
+// Debug build only: cycle stamps of thread 0 of CTA 0 at the phase boundaries of the first 64 chunks.
+__device__ long long g_tc_prof[64 * 16];
+#define PROF(i)                                                                      \
+    do {                                                                             \
+        if (blockIdx.x == 0 && threadIdx.x == 0 && r < 64) g_tc_prof[r * 16 + (i)] = clock64(); \
+    } while (0)
+#else
+#define PROF(i)
+#endif
+
 namespace {
 
 constexpr int D = 128, HC = 128, C = 64, NC = 4;
@@ -53,7 +64,6 @@ struct __align__(1024) Smem {
     uint8_t PzM[2][8192];  // kM_t pz                                                 staging slot 1
     uint8_t Stage2[16384]; // staging slot 2
     Scalars sc[2];
-    float red[3][NG][32];
     uint64_t bar_x, bar_g1, bar_g2, bar_g3, bar_agg, bar_part, bar_pu, bar_credit;
     uint32_t tmem_base;
     int dead;
@@ -105,11 +115,32 @@ __device__ void tc_chunk_scalars(const float* eta, const float* beta, const floa
     }
 }
 
+// GELU z Phi(z) and its derivative Phi(z) + z phi(z).  Phi through the five-term rational form of erfc
+// (Abramowitz & Stegun 7.1.26, absolute error 1.5e-7): one reciprocal, one exponential, a handful of FMAs.
+// The exponential exp(-z^2/2) is shared with the density phi.
+__device__ __forceinline__ float fast_rcp(float x) {
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float fast_ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 __device__ __forceinline__ float gelu_fast(float z, float& dgelu) {
-    // exact-erf GELU and its derivative (fp32 library erf/exp)
-    const float cdf = 0.5f * (1.0f + erff(z * 0.70710678118654752440f));
-    const float pdf = 0.39894228040143267794f * __expf(-0.5f * z * z);
-    dgelu = cdf + z * pdf;
+    const float x = fabsf(z) * 0.70710678118654752440f;
+    const float t = fast_rcp(fmaf(0.3275911f, x, 1.0f));
+    // 0.5 * (a1 t + ... + a5 t^5)
+    float p = fmaf(t, 0.5307027145f, -0.7265760135f);
+    p = fmaf(t, p, 0.7107068705f);
+    p = fmaf(t, p, -0.142248368f);
+    p = fmaf(t, p, 0.127414796f);
+    p *= t;
+    const float e = fast_ex2(x * x * -1.44269504088896341f);  // exp(-z^2/2)
+    const float half_erfc = p * e;                             // Phi(-|z|)
+    const float cdf = z >= 0.0f ? 1.0f - half_erfc : half_erfc;
+    dgelu = fmaf(z * 0.39894228040143267794f, e, cdf);
     return z * cdf;
 }
 
@@ -141,7 +172,6 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     const int seq = blockIdx.x / NC;
     const int issuer_warp = (int)((me + 1) & 3);  // a warp that never owns layer-norm rows of this CTA
     const bool is_issuer = (warp == issuer_warp) && (lane == 0);
-    const bool ln_owner = (q == (int)me);
     const int L = a.L, nchunks = L / C;
     WaitCtx wc{&s.dead, a.status};
 
@@ -160,8 +190,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         mbar_init(&s.bar_g2, 1);
         mbar_init(&s.bar_g3, 1);
         mbar_init(&s.bar_agg, 1);
-        mbar_init(&s.bar_part, 3 * NG);
-        mbar_init(&s.bar_pu, 2 * NG);
+        mbar_init(&s.bar_part, 1);  // + 3 x 16 KB of peer partial sums per chunk
+        mbar_init(&s.bar_pu, 1);    // + 16 KB of pu rows per chunk
         mbar_init(&s.bar_credit, 3);
         fence_mbar_init();
         tma_prefetch_desc(&tmK);
@@ -240,9 +270,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             tc_chunk_scalars(eta + tok0 + C, beta + tok0 + C, gamma + tok0 + C, &s.sc[(r + 1) & 1]);
         }
 
+        PROF(0);
         // ---------------- G1: Z = X W1c^T -> R0
         if (is_issuer) {
-            mbar_wait(&s.bar_x, ph, wc, 100 + 1);
+            mbar_expect_tx(&s.bar_part, 3 * 16384);  // this chunk's incoming partial sums and pu rows
+            mbar_expect_tx(&s.bar_pu, 16384);
+            mbar_wait_one(&s.bar_x, ph, wc, 100 + 1);
             tc_fence_after_sync();
 #pragma unroll
             for (int k = 0; k < 8; ++k)
@@ -252,6 +285,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         mbar_wait(&s.bar_g1, ph, wc, 100 + 2);
         __syncwarp();
         tc_fence_after_sync();
+        PROF(1);
         // epilogue: a = gelu(z) -> A (bf16); for key rows also kW a, kM a and gelu'(z) (kept in TMEM over z)
         {
             const bool key_row = row < C;
@@ -285,6 +319,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         tc_fence_before_sync();
         __syncthreads();
 
+        PROF(2);
         // ---------------- G2: Upart = A W2c^T -> R1
         if (is_issuer) {
             tc_fence_after_sync();
@@ -297,150 +332,148 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         __syncwarp();
         tc_fence_after_sync();
 
+        PROF(3);
         // ---------------- cross-CTA sum of Upart: rows of quadrant x go to CTA x
-        float own[CW];
-        if (r > 0) mbar_wait(&s.bar_credit, (uint32_t)((r - 1) & 1), wc, 100 + 4);
-        __syncwarp();
+        // staging slot = 32 rows x 512 B, the 16-byte piece c4 of row r kept at piece position c4 ^ (r & 7)
+        if (r > 0) mbar_wait<true>(&s.bar_credit, (uint32_t)((r - 1) & 1), wc, 100 + 4);
+        // Row ownership: CTA c normalises key tokens 16c..16c+15 and query tokens 16c..16c+15, so every CTA carries
+        // the same mix of work.  TMEM lane 32q+l holds key token 32q+l (q < 2) or query token 32(q-2)+l.
         {
-            const uint32_t slot = (me - (uint32_t)q - 1u) & 3u;  // where CTA q keeps what comes from me
-            uint32_t dst_base = 0;
-            if (!ln_owner) {
+            const uint32_t owner = 2u * ((uint32_t)q & 1u) + ((uint32_t)lane >> 4);
+            const uint32_t srow = ((q < 2) ? 0u : 16u) + ((uint32_t)lane & 15u);  // row inside the owner's staging slot
+            const bool mine = owner == me;
+            uint32_t dst_base, dst_bar = 0;
+            if (mine) {
+                dst_base = smem_u32(s.A[1]);  // own rows: the gelu tile is dead once G2 has completed
+            } else {
+                const uint32_t slot = (me - owner - 1u) & 3u;  // where the owner keeps what comes from me
                 const uint8_t* p = (slot == 0) ? s.PzW[0] : (slot == 1) ? s.PzM[0] : s.Stage2;
-                dst_base = map_to_cta(smem_u32(p), (uint32_t)q);
+                dst_base = map_to_cta(smem_u32(p), owner);
+                dst_bar = map_to_cta(smem_u32(&s.bar_part), owner);
             }
+            dst_base += srow * 512u;
 #pragma unroll
             for (int b = 0; b < NB; ++b) {
                 uint32_t u[16];
                 tmem_ld16(lane_addr + T_R1 + c0 + 16 * b, u);
                 tmem_wait_ld();
-                if (ln_owner) {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) own[16 * b + j] = __uint_as_float(u[j]);
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 16; j += 4) {
-                        const int c4 = (c0 + 16 * b + j) >> 2;
-                        st_cluster_v4_b32(dst_base + (uint32_t)(c4 * 32 + lane) * 16u, u[j], u[j + 1], u[j + 2], u[j + 3]);
-                    }
+                for (int j = 0; j < 16; j += 4) {
+                    const uint32_t c4 = (uint32_t)((c0 + 16 * b + j) >> 2);
+                    const uint32_t dst = dst_base + ((c4 ^ (srow & 7u)) << 4);
+                    if (mine) st_cluster_v4_b32(dst, u[j], u[j + 1], u[j + 2], u[j + 3]);
+                    else st_async_v4(dst, u[j], u[j + 1], u[j + 2], u[j + 3], dst_bar);
                 }
-            }
-            if (!ln_owner) {
-                __syncwarp();
-                if (lane == 0) mbar_arrive_remote(map_to_cta(smem_u32(&s.bar_part), (uint32_t)q));
             }
         }
         tc_fence_before_sync();
-        __syncthreads();  // R1 has been read by everyone: G3 may overwrite it
+        __syncthreads();  // R1 has been read by everyone (G3 may overwrite it); own rows are staged
+        PROF(4);
 
-        // ---------------- layer norm on the 32 rows this CTA owns (the warps of quadrant `me`)
-        if (ln_owner) {
-            mbar_wait(&s.bar_part, ph, wc, 100 + 5);
-            __syncwarp();
-            float u[CW];
+        // ---------------- layer norm on the 16 key and 16 query rows this CTA owns, all threads: TPR threads per row
+        {
+            constexpr int TPR = NTHREADS / 32, CPT = 128 / TPR;  // threads per row, columns per thread
+            const int lrow = tid / TPR, cg = tid % TPR;  // staging rows 0..15: key tokens, 16..31: query tokens
+            const bool key_rows = lrow < 16;             // warp-uniform: a warp covers 32 / TPR whole rows
+            const int t = 16 * (int)me + (lrow & 15);    // token inside the chunk
+            const int xrow = key_rows ? t : 64 + t;      // its row in the X tile
+            const int col0 = CPT * cg;
+            const size_t off = (size_t)(tok0 + t) * D + col0;
+            uint4 vraw[CPT / 8], xraw[CPT / 8];
 #pragma unroll
-            for (int j = 0; j < CW; ++j) u[j] = 0.0f;
+            for (int ch = 0; ch < CPT / 8; ++ch) {
+                if (key_rows) vraw[ch] = *reinterpret_cast<const uint4*>(gv + off + 8 * ch);
+                const int c = ((col0 & 63) >> 3) + ch;
+                xraw[ch] = *reinterpret_cast<const uint4*>(s.X[col0 >> 6] + xrow * 128 + ((c ^ (xrow & 7)) << 4));
+            }
+            mbar_wait<true>(&s.bar_part, ph, wc, 100 + 5);
+            float u[CPT];
+#pragma unroll
+            for (int j = 0; j < CPT; ++j) u[j] = 0.0f;
 #pragma unroll
             for (int src = 0; src < NC; ++src) {  // fixed order: the sum does not depend on arrival order
-                if (src == (int)me) {
+                const uint32_t slot = ((uint32_t)src - me - 1u) & 3u;
+                const uint8_t* p = (src == (int)me) ? s.A[1] : (slot == 0) ? s.PzW[0] : (slot == 1) ? s.PzM[0] : s.Stage2;
 #pragma unroll
-                    for (int j = 0; j < CW; ++j) u[j] += own[j];
-                } else {
-                    const uint32_t slot = ((uint32_t)src - me - 1u) & 3u;
-                    const uint8_t* p = (slot == 0) ? s.PzW[0] : (slot == 1) ? s.PzM[0] : s.Stage2;
-#pragma unroll
-                    for (int j = 0; j < CW; j += 4) {
-                        const float4 x = *reinterpret_cast<const float4*>(p + (size_t)(((c0 + j) >> 2) * 32 + lane) * 16);
-                        u[j] += x.x; u[j + 1] += x.y; u[j + 2] += x.z; u[j + 3] += x.w;
-                    }
+                for (int j = 0; j < CPT; j += 4) {
+                    const int c4 = (col0 + j) >> 2;
+                    const float4 x = *reinterpret_cast<const float4*>(p + lrow * 512 + ((c4 ^ (lrow & 7)) << 4));
+                    u[j] += x.x; u[j + 1] += x.y; u[j + 2] += x.z; u[j + 3] += x.w;
                 }
             }
-            // row statistics: each of the NG warps holds CW columns of every row
-            auto row_sum = [&](float v, int round) -> float {
-                s.red[round][g][lane] = v;
-                asm volatile("bar.sync 1, %0;" ::"r"(32 * NG) : "memory");
-                float t = 0.0f;
+            PROF(5);
+            auto row_sum = [&](float v) -> float {  // over the TPR lanes that share a row
 #pragma unroll
-                for (int gg = 0; gg < NG; ++gg) t += s.red[round][gg][lane];
-                return t;
+                for (int o = TPR / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                return v;
             };
             float sum = 0.0f;
 #pragma unroll
-            for (int j = 0; j < CW; ++j) sum += u[j];
-            const float mu = row_sum(sum, 0) * (1.0f / D);
-            float vs = 0.0f;
+            for (int j = 0; j < CPT; ++j) sum += u[j];
+            const float mu = row_sum(sum) * (1.0f / D);
+            float sq = 0.0f;
 #pragma unroll
-            for (int j = 0; j < CW; ++j) { u[j] -= mu; vs += u[j] * u[j]; }
-            const float rstd = rsqrtf(row_sum(vs, 1) * (1.0f / D) + a.eps);
+            for (int j = 0; j < CPT; ++j) { u[j] -= mu; sq = fmaf(u[j], u[j], sq); }
+            const float rstd = rsqrtf(row_sum(sq) * (1.0f / D) + a.eps);
 #pragma unroll
-            for (int j = 0; j < CW; ++j) u[j] *= rstd;  // y
-            if (me < 2) {
+            for (int j = 0; j < CPT; ++j) u[j] *= rstd;  // y
+            if (key_rows) {
                 // key rows: e = k + y - v, pu = rstd (e - mean(e) - y mean(e y))
-                const int t = 32 * (int)me + lane;
-                const size_t off = (size_t)(tok0 + t) * D + c0;
-                float e[CW];
+                float e[CPT];
                 float se = 0.0f, sey = 0.0f;
 #pragma unroll
-                for (int j = 0; j < CW; j += 8) {
-                    const uint4 kk = *reinterpret_cast<const uint4*>(gk + off + j);
-                    const uint4 vv = *reinterpret_cast<const uint4*>(gv + off + j);
-                    const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&kk);
-                    const __nv_bfloat162* v2 = reinterpret_cast<const __nv_bfloat162*>(&vv);
+                for (int ch = 0; ch < CPT / 8; ++ch) {
+                    const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&xraw[ch]);
+                    const __nv_bfloat162* v2 = reinterpret_cast<const __nv_bfloat162*>(&vraw[ch]);
 #pragma unroll
                     for (int x = 0; x < 4; ++x) {
                         const float2 kf = __bfloat1622float2(k2[x]), vf = __bfloat1622float2(v2[x]);
-                        e[j + 2 * x] = kf.x + u[j + 2 * x] - vf.x;
-                        e[j + 2 * x + 1] = kf.y + u[j + 2 * x + 1] - vf.y;
+                        const int j = 8 * ch + 2 * x;
+                        e[j] = kf.x + u[j] - vf.x;
+                        e[j + 1] = kf.y + u[j + 1] - vf.y;
                     }
                 }
 #pragma unroll
-                for (int j = 0; j < CW; ++j) { se += e[j]; sey += e[j] * u[j]; }
-                const float me_ = row_sum(se, 2) * (1.0f / D);
-                const float mey = row_sum(sey, 0) * (1.0f / D);  // plane 0 was last read two barriers ago
-                // broadcast the bf16 pu row piece to every CTA of the cluster
-                uint32_t pk[CW / 2];
+                for (int j = 0; j < CPT; ++j) { se += e[j]; sey = fmaf(e[j], u[j], sey); }
+                const float me_ = row_sum(se) * (1.0f / D), mey = row_sum(sey) * (1.0f / D);
+                    // broadcast the bf16 pu row piece to every CTA of the cluster
+                uint32_t pk[CPT / 2];
 #pragma unroll
-                for (int j = 0; j < CW; j += 2)
+                for (int j = 0; j < CPT; j += 2)
                     pk[j / 2] = pack_bf16(rstd * (e[j] - me_ - u[j] * mey), rstd * (e[j + 1] - me_ - u[j + 1] * mey));
-                const uint32_t pu_local = smem_u32(s.Pu[c0 >> 6]);
+                const uint32_t pu_local = smem_u32(s.Pu[col0 >> 6]);
 #pragma unroll
                 for (uint32_t dst = 0; dst < NC; ++dst) {
                     const uint32_t base = map_to_cta(pu_local, dst) + (uint32_t)t * 128u;
+                    const uint32_t bar = map_to_cta(smem_u32(&s.bar_pu), dst);
 #pragma unroll
-                    for (int ch = 0; ch < CW / 8; ++ch) {
-                        const uint32_t c = (uint32_t)(((c0 & 63) >> 3) + ch);
-                        st_cluster_v4_b32(base + ((c ^ ((uint32_t)t & 7u)) << 4), pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2],
-                                          pk[4 * ch + 3]);
+                    for (int ch = 0; ch < CPT / 8; ++ch) {
+                        const uint32_t c = (uint32_t)(((col0 & 63) >> 3) + ch);
+                        st_async_v4(base + ((c ^ ((uint32_t)t & 7u)) << 4), pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2],
+                                    pk[4 * ch + 3], bar);
                     }
-                }
-                asm volatile("fence.proxy.async;" ::: "memory");
-                __syncwarp();
-                if (lane == 0) {
-#pragma unroll
-                    for (uint32_t dst = 0; dst < NC; ++dst) mbar_arrive_remote(map_to_cta(smem_u32(&s.bar_pu), dst));
                 }
             } else {
                 // query rows: o = q + y
-                const int t = 32 * ((int)me - 2) + lane;
-                const size_t off = (size_t)(tok0 + t) * D + c0;
 #pragma unroll
-                for (int j = 0; j < CW; j += 8) {
-                    const uint4 qq = *reinterpret_cast<const uint4*>(gq + off + j);
-                    const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&qq);
+                for (int ch = 0; ch < CPT / 8; ++ch) {
+                    const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&xraw[ch]);
                     uint4 ov;
                     uint32_t* o32 = reinterpret_cast<uint32_t*>(&ov);
 #pragma unroll
                     for (int x = 0; x < 4; ++x) {
                         const float2 qf = __bfloat1622float2(q2[x]);
-                        o32[x] = pack_bf16(qf.x + u[j + 2 * x], qf.y + u[j + 2 * x + 1]);
+                        o32[x] = pack_bf16(qf.x + u[8 * ch + 2 * x], qf.y + u[8 * ch + 2 * x + 1]);
                     }
-                    *reinterpret_cast<uint4*>(go + off + j) = ov;
+                    *reinterpret_cast<uint4*>(go + off + 8 * ch) = ov;
                 }
             }
         }
 
+        PROF(6);
         // ---------------- G3: Pa = Pu W2c -> R1 ; then the W2 aggregation that needs nothing else
         if (is_issuer) {
-            mbar_wait(&s.bar_pu, ph, wc, 100 + 6);
+            mbar_wait_one<true>(&s.bar_pu, ph, wc, 100 + 6);
             asm volatile("fence.proxy.async;" ::: "memory");
             tc_fence_after_sync();
 #pragma unroll
@@ -453,6 +486,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         }
         mbar_wait(&s.bar_g3, ph, wc, 100 + 7);
         __syncwarp();
+        PROF(7);
         tc_fence_after_sync();
         if (row < C) {
             const float kw = sc.kW[row], km = sc.kM[row];
@@ -478,6 +512,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         tc_fence_before_sync();
         __syncthreads();
 
+        PROF(8);
         // ---------------- remaining aggregations
         if (is_issuer) {
             tc_fence_after_sync();
@@ -494,6 +529,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         }
         mbar_wait(&s.bar_agg, ph, wc, 100 + 8);
         __syncwarp();
+        PROF(9);
         tc_fence_after_sync();
         if (is_issuer) {
             // peers may now overwrite this CTA's staging / Pu buffers; the next chunk's tokens may land in X
@@ -511,6 +547,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         }
         __syncwarp();
 
+        PROF(10);
         // ---------------- state pass (Algorithm 1 lines 6-7)
         {
             const bool last = (r + 1 == nchunks);
@@ -573,6 +610,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         tc_fence_before_sync();
         __syncthreads();
         tc_fence_after_sync();
+        PROF(11);
     }
 
     // no CTA leaves while a peer may still write into its shared memory or arrive on its barriers
@@ -616,6 +654,12 @@ bool make_token_map(CUtensorMap* tm, const void* base, size_t rows) {
 }  // namespace
 
 size_t tc_fwd_smem_bytes() { return sizeof(Smem); }
+
+#ifdef TC_PROFILE
+extern "C" __attribute__((visibility("default"))) int e2ttt_debug_read_profile(long long* host, int n) {
+    return (int)cudaMemcpyFromSymbol(host, g_tc_prof, sizeof(long long) * (size_t)n);
+}
+#endif
 
 int tc_fwd_launch(const TcFwdArgs& a, void* stream) {
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
