@@ -13,7 +13,7 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "lib", "libe2ttt.so")
+LIB_PATH = os.environ.get("E2TTT_LIB") or os.path.join(_HERE, "lib", "libe2ttt.so")  # E2TTT_LIB: use another build
 
 E2TTT_MLP_GELU, E2TTT_SWIGLU = 0, 1
 E2TTT_F32, E2TTT_BF16 = 0, 1

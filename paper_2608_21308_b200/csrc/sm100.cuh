@@ -73,6 +73,9 @@ __device__ __forceinline__ bool mbar_wait_one(uint64_t* bar, uint32_t parity, co
     const long long t0 = clock64();
     int spins = 0;
     while (!mbar_try_wait<CLUSTER>(bar, parity)) {
+#if defined(E2TTT_POLL_SLEEP)
+        __nanosleep(E2TTT_POLL_SLEEP);
+#endif
         if ((++spins & 63) == 0) {
             if (*w.dead) return false;
             if (clock64() - t0 > kWaitCycles) {

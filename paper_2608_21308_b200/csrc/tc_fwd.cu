@@ -144,6 +144,14 @@ __device__ __forceinline__ float gelu_fast(float z, float& dgelu) {
     return z * cdf;
 }
 
+// Staging slot for partial sums: 32 rows x 128 fp32, kept as 16-byte pieces.  Piece c4 (4 columns) of row r sits at
+// piece index c4 * 32 + (r ^ ((c4 >> 1) & 15)): the 16 lanes that send one piece of 16 neighbouring rows write 256
+// contiguous bytes (DSMEM moves whole segments; scattered 16-byte stores cost several times the bandwidth), and the
+// layer-norm readers (16 threads per row, pieces 2cg and 2cg+1) spread over all banks.
+__device__ __forceinline__ uint32_t stage_offset(uint32_t c4, uint32_t r) {
+    return (c4 * 32u + (r ^ ((c4 >> 1) & 15u))) << 4;
+}
+
 // 16 bf16 (32 bytes) = two 16-byte chunks into a swizzled slab row
 __device__ __forceinline__ void st_slab16(uint8_t* slab, int row, int col0, const float (&v)[16]) {
     const int c = col0 >> 3;
@@ -334,7 +342,6 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 
         PROF(3);
         // ---------------- cross-CTA sum of Upart: rows of quadrant x go to CTA x
-        // staging slot = 32 rows x 512 B, the 16-byte piece c4 of row r kept at piece position c4 ^ (r & 7)
         if (r > 0) mbar_wait<true>(&s.bar_credit, (uint32_t)((r - 1) & 1), wc, 100 + 4);
         // Row ownership: CTA c normalises key tokens 16c..16c+15 and query tokens 16c..16c+15, so every CTA carries
         // the same mix of work.  TMEM lane 32q+l holds key token 32q+l (q < 2) or query token 32(q-2)+l.
@@ -351,7 +358,6 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 dst_base = map_to_cta(smem_u32(p), owner);
                 dst_bar = map_to_cta(smem_u32(&s.bar_part), owner);
             }
-            dst_base += srow * 512u;
 #pragma unroll
             for (int b = 0; b < NB; ++b) {
                 uint32_t u[16];
@@ -360,7 +366,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 #pragma unroll
                 for (int j = 0; j < 16; j += 4) {
                     const uint32_t c4 = (uint32_t)((c0 + 16 * b + j) >> 2);
-                    const uint32_t dst = dst_base + ((c4 ^ (srow & 7u)) << 4);
+                    const uint32_t dst = dst_base + stage_offset(c4, srow);
                     if (mine) st_cluster_v4_b32(dst, u[j], u[j + 1], u[j + 2], u[j + 3]);
                     else st_async_v4(dst, u[j], u[j + 1], u[j + 2], u[j + 3], dst_bar);
                 }
@@ -397,7 +403,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 #pragma unroll
                 for (int j = 0; j < CPT; j += 4) {
                     const int c4 = (col0 + j) >> 2;
-                    const float4 x = *reinterpret_cast<const float4*>(p + lrow * 512 + ((c4 ^ (lrow & 7)) << 4));
+                    const float4 x = *reinterpret_cast<const float4*>(p + stage_offset((uint32_t)c4, (uint32_t)lrow));
                     u[j] += x.x; u[j + 1] += x.y; u[j + 2] += x.z; u[j + 3] += x.w;
                 }
             }
