@@ -40,7 +40,7 @@ UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per forward launch from the committed ncu capture
 # (profiles/): set once a capture of the current kernel exists, else null.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 331.3e6  # profiles/tc_fwd_kernel_config2.md: 239.5 MB read + 91.9 MB written
 
 
 def peaks():
@@ -266,7 +266,8 @@ def run_ours(args, r):
             "gpu_launches": args.steps,
             "clocks": clocks,
             "roofline": {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
-                         "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "peak_source": pk["_source"],
+                         "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if args.config == 2 else None,
+                         "peak_source": pk["_source"],
                          "kernel": "forward kernel (one launch per step)",
                          "flop_per_launch": flop, "bytes_per_launch": bytes_per_call(r),
                          "frac_of_sustained_peak": (flop / (ms * 1e-3) / 1e12) / pk["bf16_tflops_sustained"]},
