@@ -64,7 +64,7 @@ struct __align__(1024) Smem {
     uint8_t PzM[2][8192];  // kM_t pz                                                 staging slot 1
     uint8_t Stage2[16384]; // staging slot 2
     Scalars sc[2];
-    uint64_t bar_x, bar_g1, bar_g2, bar_g3, bar_agg, bar_part, bar_pu, bar_credit;
+    uint64_t bar_x, bar_g1, bar_g2, bar_g3, bar_agg, bar_agg2, bar_part, bar_pu, bar_credit;
     uint32_t tmem_base;
     int dead;
 };
@@ -198,6 +198,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         mbar_init(&s.bar_g2, 1);
         mbar_init(&s.bar_g3, 1);
         mbar_init(&s.bar_agg, 1);
+        mbar_init(&s.bar_agg2, 1);
         mbar_init(&s.bar_part, 1);  // + 3 x 16 KB of peer partial sums per chunk
         mbar_init(&s.bar_pu, 1);    // + 16 KB of pu rows per chunk
         mbar_init(&s.bar_credit, 3);
@@ -268,6 +269,18 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     const uint32_t id_kmn = make_idesc(128, 128, false, true);
     const uint32_t id_agg = make_idesc(128, 128, true, true) | (1u << 13);  // negate A: G_t is minus the gradient
 
+    // G1 of chunk `chunk` (issuer thread only): needs that chunk's tokens in X and the refreshed bf16 W1
+    auto issue_g1 = [&](int chunk) {
+        mbar_wait_one(&s.bar_x, (uint32_t)(chunk & 1), wc, 100 + 1);
+        tc_fence_after_sync();
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+            umma_bf16(tb + T_R0, desc_k(smem_u32(s.X[0]), 16384, k), desc_k(smem_u32(s.W1[0]), 16384, k), id_kk, k > 0);
+        umma_commit(&s.bar_g1);
+    };
+    if (is_issuer) issue_g1(0);
+    __syncwarp();
+
     for (int r = 0; r < nchunks; ++r) {
         const uint32_t ph = (uint32_t)(r & 1);
         const Scalars& sc = s.sc[r & 1];
@@ -279,16 +292,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         }
 
         PROF(0);
-        // ---------------- G1: Z = X W1c^T -> R0
+        // ---------------- G1: Z = X W1c^T -> R0 (issued at the end of the previous iteration / before the loop)
         if (is_issuer) {
             mbar_expect_tx(&s.bar_part, 3 * 16384);  // this chunk's incoming partial sums and pu rows
             mbar_expect_tx(&s.bar_pu, 16384);
-            mbar_wait_one(&s.bar_x, ph, wc, 100 + 1);
-            tc_fence_after_sync();
-#pragma unroll
-            for (int k = 0; k < 8; ++k)
-                umma_bf16(tb + T_R0, desc_k(smem_u32(s.X[0]), 16384, k), desc_k(smem_u32(s.W1[0]), 16384, k), id_kk, k > 0);
-            umma_commit(&s.bar_g1);
         }
         mbar_wait(&s.bar_g1, ph, wc, 100 + 2);
         __syncwarp();
@@ -519,7 +526,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         __syncthreads();
 
         PROF(8);
-        // ---------------- remaining aggregations
+        // ---------------- remaining aggregations, in two groups so that the state pass can start on W1 early
         if (is_issuer) {
             tc_fence_after_sync();
 #pragma unroll
@@ -528,90 +535,106 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 #pragma unroll
             for (int k = 0; k < 4; ++k)
                 umma_bf16(tb + T_R0, desc_mn(smem_u32(s.PzM[0]), 8192, k), desc_mn(smem_u32(s.X[0]), 16384, k), id_agg, k > 0);
+            umma_commit(&s.bar_agg);
 #pragma unroll
             for (int k = 0; k < 4; ++k)
                 umma_bf16(tb + T_R1, desc_mn(smem_u32(s.Pu[0]), 8192, k), desc_mn(smem_u32(s.AkM[0]), 8192, k), id_agg, k > 0);
-            umma_commit(&s.bar_agg);
+            umma_commit(&s.bar_agg2);
         }
+        const bool last = (r + 1 == nchunks);
+        const float cm = sc.cm, cb = sc.cb;
+        const float cwn = last ? 1.0f : s.sc[(r + 1) & 1].cw;
+        const size_t head = (size_t)seq * (size_t)(D * 4 * HC);
+
         mbar_wait(&s.bar_agg, ph, wc, 100 + 8);
-        __syncwarp();
         PROF(9);
         tc_fence_after_sync();
+        if (is_issuer && !last) {
+            // the W1 aggregations were the last readers of the key tile: the next chunk's tokens may land in X
+            mbar_expect_tx(&s.bar_x, 32768);
+            const int y = seq * L + tok0 + C;
+            tma_load_2d(s.X[0], &tmK, 0, y, &s.bar_x);
+            tma_load_2d(s.X[1], &tmK, 64, y, &s.bar_x);
+            tma_load_2d(s.X[0] + 8192, &tmQ, 0, y, &s.bar_x);
+            tma_load_2d(s.X[1] + 8192, &tmQ, 64, y, &s.bar_x);
+        }
+        __syncwarp();
+        PROF(10);
+        // ---------------- state pass, W1 half (Algorithm 1 lines 6-7), while the M2 aggregation still runs
+#pragma unroll
+        for (int b = 0; b < NB; ++b) {
+            const int col = c0 + 16 * b;
+            uint32_t wa[16], ma[16], st[16];
+            float wn[16];
+            tmem_ld16(lane_addr + T_W1 + col, wa);
+            tmem_ld16(lane_addr + T_R0 + col, ma);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const float m0 = M1[16 * b + j];
+                wn[j] = __uint_as_float(wa[j]) + cm * m0;
+                M1[16 * b + j] = cb * m0 + __uint_as_float(ma[j]);
+                st[j] = __float_as_uint(cwn * wn[j]);
+            }
+            tmem_st16(lane_addr + T_W1 + col, st);
+            st_slab16(s.W1[col >> 6], row, col & 63, wn);
+            if (last) {
+                float* wf = a.W1_final + head + ((size_t)(HC * me) + row) * D + col;
+                float* mf = a.M1_final + head + ((size_t)(HC * me) + row) * D + col;
+#pragma unroll
+                for (int j = 0; j < 16; j += 4) {
+                    *reinterpret_cast<float4*>(wf + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
+                    *reinterpret_cast<float4*>(mf + j) =
+                        make_float4(M1[16 * b + j], M1[16 * b + j + 1], M1[16 * b + j + 2], M1[16 * b + j + 3]);
+                }
+            }
+        }
+        tmem_wait_st();
+        fence_proxy_async_smem();
+        tc_fence_before_sync();
+        __syncthreads();  // bf16 W1 is complete and R0 is free: the next chunk's G1 may run under the W2 half
+        if (is_issuer && !last) issue_g1(r + 1);
+        __syncwarp();
+
+        mbar_wait(&s.bar_agg2, ph, wc, 100 + 9);
+        tc_fence_after_sync();
         if (is_issuer) {
-            // peers may now overwrite this CTA's staging / Pu buffers; the next chunk's tokens may land in X
+            // every reader of this chunk's staging / pu / scaled-activation buffers is done: peers may overwrite them
 #pragma unroll
             for (uint32_t dst = 0; dst < NC; ++dst)
                 if (dst != me) mbar_arrive_remote(map_to_cta(smem_u32(&s.bar_credit), dst));
-            if (r + 1 < nchunks) {
-                mbar_expect_tx(&s.bar_x, 32768);
-                const int y = seq * L + tok0 + C;
-                tma_load_2d(s.X[0], &tmK, 0, y, &s.bar_x);
-                tma_load_2d(s.X[1], &tmK, 64, y, &s.bar_x);
-                tma_load_2d(s.X[0] + 8192, &tmQ, 0, y, &s.bar_x);
-                tma_load_2d(s.X[1] + 8192, &tmQ, 64, y, &s.bar_x);
-            }
         }
         __syncwarp();
-
-        PROF(10);
-        // ---------------- state pass (Algorithm 1 lines 6-7)
-        {
-            const bool last = (r + 1 == nchunks);
-            const float cm = sc.cm, cb = sc.cb;
-            const float cwn = last ? 1.0f : s.sc[(r + 1) & 1].cw;
-            const size_t head = (size_t)seq * (size_t)(D * 4 * HC);
+        // ---------------- state pass, W2 half
 #pragma unroll
-            for (int b = 0; b < NB; ++b) {
-                const int col = c0 + 16 * b;
-                uint32_t wa[16], ma[16], st[16];
-                float wn[16];
-                tmem_ld16(lane_addr + T_W1 + col, wa);
-                tmem_ld16(lane_addr + T_R0 + col, ma);
-                tmem_wait_ld();
+        for (int b = 0; b < NB; ++b) {
+            const int col = c0 + 16 * b;
+            uint32_t wa[16], ma[16], st[16];
+            float wn[16];
+            tmem_ld16(lane_addr + T_W2 + col, wa);
+            tmem_ld16(lane_addr + T_R1 + col, ma);
+            tmem_wait_ld();
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const float m0 = M1[16 * b + j];
-                    wn[j] = __uint_as_float(wa[j]) + cm * m0;
-                    M1[16 * b + j] = cb * m0 + __uint_as_float(ma[j]);
-                    st[j] = __float_as_uint(cwn * wn[j]);
-                }
-                tmem_st16(lane_addr + T_W1 + col, st);
-                st_slab16(s.W1[col >> 6], row, col & 63, wn);
-                if (last) {
-                    float* wf = a.W1_final + head + ((size_t)(HC * me) + row) * D + col;
-                    float* mf = a.M1_final + head + ((size_t)(HC * me) + row) * D + col;
+            for (int j = 0; j < 16; ++j) {
+                const float m0 = M2[16 * b + j];
+                wn[j] = __uint_as_float(wa[j]) + cm * m0;
+                M2[16 * b + j] = cb * m0 + __uint_as_float(ma[j]);
+                st[j] = __float_as_uint(cwn * wn[j]);
+            }
+            tmem_st16(lane_addr + T_W2 + col, st);
+            st_slab16(s.W2[col >> 6], row, col & 63, wn);
+            if (last) {
+                float* wf = a.W2_final + head + (size_t)row * (4 * HC) + HC * me + col;
+                float* mf = a.M2_final + head + (size_t)row * (4 * HC) + HC * me + col;
 #pragma unroll
-                    for (int j = 0; j < 16; j += 4) {
-                        *reinterpret_cast<float4*>(wf + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
-                        *reinterpret_cast<float4*>(mf + j) =
-                            make_float4(M1[16 * b + j], M1[16 * b + j + 1], M1[16 * b + j + 2], M1[16 * b + j + 3]);
-                    }
-                }
-                tmem_ld16(lane_addr + T_W2 + col, wa);
-                tmem_ld16(lane_addr + T_R1 + col, ma);
-                tmem_wait_ld();
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const float m0 = M2[16 * b + j];
-                    wn[j] = __uint_as_float(wa[j]) + cm * m0;
-                    M2[16 * b + j] = cb * m0 + __uint_as_float(ma[j]);
-                    st[j] = __float_as_uint(cwn * wn[j]);
-                }
-                tmem_st16(lane_addr + T_W2 + col, st);
-                st_slab16(s.W2[col >> 6], row, col & 63, wn);
-                if (last) {
-                    float* wf = a.W2_final + head + (size_t)row * (4 * HC) + HC * me + col;
-                    float* mf = a.M2_final + head + (size_t)row * (4 * HC) + HC * me + col;
-#pragma unroll
-                    for (int j = 0; j < 16; j += 4) {
-                        *reinterpret_cast<float4*>(wf + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
-                        *reinterpret_cast<float4*>(mf + j) =
-                            make_float4(M2[16 * b + j], M2[16 * b + j + 1], M2[16 * b + j + 2], M2[16 * b + j + 3]);
-                    }
+                for (int j = 0; j < 16; j += 4) {
+                    *reinterpret_cast<float4*>(wf + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
+                    *reinterpret_cast<float4*>(mf + j) =
+                        make_float4(M2[16 * b + j], M2[16 * b + j + 1], M2[16 * b + j + 2], M2[16 * b + j + 3]);
                 }
             }
-            tmem_wait_st();
         }
+        tmem_wait_st();
         fence_proxy_async_smem();
         tc_fence_before_sync();
         __syncthreads();
