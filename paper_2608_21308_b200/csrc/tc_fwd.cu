@@ -64,7 +64,7 @@ struct __align__(1024) Smem {
     uint8_t PzM[2][8192];  // kM_t pz                                                 staging slot 1
     uint8_t Stage2[16384]; // staging slot 2
     Scalars sc[2];
-    uint64_t bar_x, bar_g1, bar_g2, bar_g3, bar_agg, bar_agg2, bar_part, bar_pu, bar_credit;
+    uint64_t bar_x, bar_g1, bar_g2, bar_g3, bar_agg, bar_agg2, bar_ak, bar_part, bar_pu, bar_credit;
     uint32_t tmem_base;
     int dead;
 };
@@ -128,6 +128,17 @@ __device__ __forceinline__ float fast_ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+__device__ __forceinline__ float gelu_only(float z) {
+    const float x = fabsf(z) * 0.70710678118654752440f;
+    const float t = fast_rcp(fmaf(0.3275911f, x, 1.0f));
+    float p = fmaf(t, 0.5307027145f, -0.7265760135f);
+    p = fmaf(t, p, 0.7107068705f);
+    p = fmaf(t, p, -0.142248368f);
+    p = fmaf(t, p, 0.127414796f);
+    p *= t;
+    const float half_erfc = p * fast_ex2(x * x * -1.44269504088896341f);
+    return z * (z >= 0.0f ? 1.0f - half_erfc : half_erfc);
+}
 __device__ __forceinline__ float gelu_fast(float z, float& dgelu) {
     const float x = fabsf(z) * 0.70710678118654752440f;
     const float t = fast_rcp(fmaf(0.3275911f, x, 1.0f));
@@ -178,7 +189,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     const int c0 = CW * g;           // first of its columns inside a 128-column region
     const uint32_t me = cluster_ctarank();
     const int seq = blockIdx.x / NC;
-    const int issuer_warp = (int)((me + 1) & 3);  // a warp that never owns layer-norm rows of this CTA
+    const int issuer_warp = 2;  // a warp of quadrant 2: free while quadrants 0/1 produce the backward-only operands
     const bool is_issuer = (warp == issuer_warp) && (lane == 0);
     const int L = a.L, nchunks = L / C;
     WaitCtx wc{&s.dead, a.status};
@@ -199,6 +210,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         mbar_init(&s.bar_g3, 1);
         mbar_init(&s.bar_agg, 1);
         mbar_init(&s.bar_agg2, 1);
+        mbar_init(&s.bar_ak, 2 * NG);
         mbar_init(&s.bar_part, 1);  // + 3 x 16 KB of peer partial sums per chunk
         mbar_init(&s.bar_pu, 1);    // + 16 KB of pu rows per chunk
         mbar_init(&s.bar_credit, 3);
@@ -287,7 +299,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         const int tok0 = r * C;
 
         // scalars of the next chunk (suffix scans over its gates), by a warp that is not the issuer
-        if (warp == ((issuer_warp + 2) & 3) + 4 * (NG - 1) && r + 1 < nchunks) {
+        if (warp == 3 + 4 * (NG - 1) && r + 1 < nchunks) {
             tc_chunk_scalars(eta + tok0 + C, beta + tok0 + C, gamma + tok0 + C, &s.sc[(r + 1) & 1]);
         }
 
@@ -302,33 +314,17 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         tc_fence_after_sync();
         PROF(1);
         // epilogue: a = gelu(z) -> A (bf16); for key rows also kW a, kM a and gelu'(z) (kept in TMEM over z)
-        {
-            const bool key_row = row < C;
-            const float kw = key_row ? sc.kW[row] : 0.0f, km = key_row ? sc.kM[row] : 0.0f;
+        // a = gelu(z) -> A (bf16) for all 128 rows: all that G2 needs
 #pragma unroll
-            for (int b = 0; b < NB; ++b) {
-                uint32_t z[16];
-                tmem_ld16(lane_addr + T_R0 + c0 + 16 * b, z);
-                tmem_wait_ld();
-                float av[16], aw[16], am[16];
-                uint32_t dg[16];
+        for (int b = 0; b < NB; ++b) {
+            uint32_t z[16];
+            tmem_ld16(lane_addr + T_R0 + c0 + 16 * b, z);
+            tmem_wait_ld();
+            float av[16];
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    float d1;
-                    av[j] = gelu_fast(__uint_as_float(z[j]), d1);
-                    dg[j] = __float_as_uint(d1);
-                    aw[j] = kw * av[j];
-                    am[j] = km * av[j];
-                }
-                const int col = c0 + 16 * b;
-                st_slab16(s.A[col >> 6], row, col & 63, av);
-                if (key_row) {
-                    st_slab16(s.AkW[col >> 6], row, col & 63, aw);
-                    st_slab16(s.AkM[col >> 6], row, col & 63, am);
-                    tmem_st16(lane_addr + T_R0 + col, dg);
-                }
-            }
-            tmem_wait_st();
+            for (int j = 0; j < 16; ++j) av[j] = gelu_only(__uint_as_float(z[j]));
+            const int col = c0 + 16 * b;
+            st_slab16(s.A[col >> 6], row, col & 63, av);
         }
         fence_proxy_async_smem();
         tc_fence_before_sync();
@@ -343,6 +339,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 umma_bf16(tb + T_R1, desc_k(smem_u32(s.A[0]), 16384, k), desc_k(smem_u32(s.W2[0]), 16384, k), id_kk, k > 0);
             umma_commit(&s.bar_g2);
         }
+        __syncwarp();
         mbar_wait(&s.bar_g2, ph, wc, 100 + 3);
         __syncwarp();
         tc_fence_after_sync();
@@ -383,11 +380,46 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         __syncthreads();  // R1 has been read by everyone (G3 may overwrite it); own rows are staged
         PROF(4);
 
+        // While the partial sums travel: what only the inner backward needs, for the key rows (the warps of TMEM
+        // quadrants 0 and 1): kW a, kM a (operands of the W2 aggregations) and gelu'(z), which replaces z in TMEM.
+        if (row < C) {
+            const float kw = sc.kW[row], km = sc.kM[row];
+#pragma unroll
+            for (int b = 0; b < NB; ++b) {
+                uint32_t z[16];
+                tmem_ld16(lane_addr + T_R0 + c0 + 16 * b, z);
+                tmem_wait_ld();
+                float aw[16], am[16];
+                uint32_t dg[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    float d1;
+                    const float av = gelu_fast(__uint_as_float(z[j]), d1);
+                    dg[j] = __float_as_uint(d1);
+                    aw[j] = kw * av;
+                    am[j] = km * av;
+                }
+                const int col = c0 + 16 * b;
+                st_slab16(s.AkW[col >> 6], row, col & 63, aw);
+                st_slab16(s.AkM[col >> 6], row, col & 63, am);
+                tmem_st16(lane_addr + T_R0 + col, dg);
+            }
+            tmem_wait_st();
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&s.bar_ak);
+        }
+
         // ---------------- layer norm on the 16 key and 16 query rows this CTA owns, all threads: TPR threads per row
         {
             constexpr int TPR = NTHREADS / 32, CPT = 128 / TPR;  // threads per row, columns per thread
-            const int lrow = tid / TPR, cg = tid % TPR;  // staging rows 0..15: key tokens, 16..31: query tokens
-            const bool key_rows = lrow < 16;             // warp-uniform: a warp covers 32 / TPR whole rows
+            static_assert(TPR == 16, "row mapping below assumes two rows per warp");
+            // staging rows 0..15: key tokens, 16..31: query tokens.  The key rows (which the whole cluster waits for)
+            // go to the warps of quadrants 2 and 3, which are free; the warps of quadrants 0 and 1 arrive later
+            // (they have just produced the backward-only operands) and take the query rows.
+            const bool key_rows = q >= 2;
+            const int lrow = (key_rows ? 0 : 16) + 2 * ((q & 1) + 2 * g) + (lane >> 4);
+            const int cg = lane & 15;
             const int t = 16 * (int)me + (lrow & 15);    // token inside the chunk
             const int xrow = key_rows ? t : 64 + t;      // its row in the X tile
             const int col0 = CPT * cg;
@@ -493,6 +525,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             for (int k = 0; k < 8; ++k)
                 umma_bf16(tb + T_R1, desc_k(smem_u32(s.Pu[0]), 8192, k), desc_mn(smem_u32(s.W2[0]), 16384, k), id_kmn, k > 0);
             umma_commit(&s.bar_g3);
+            mbar_wait_one(&s.bar_ak, ph, wc, 100 + 10);  // kW a / kM a written by the quadrant-0/1 warps
+            tc_fence_after_sync();
 #pragma unroll
             for (int k = 0; k < 4; ++k)
                 umma_bf16(tb + T_W2, desc_mn(smem_u32(s.Pu[0]), 8192, k), desc_mn(smem_u32(s.AkW[0]), 8192, k), id_agg, true);
@@ -502,6 +536,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         PROF(7);
         tc_fence_after_sync();
         if (row < C) {
+            // these warps also read the staging slots (query rows) that the Pz tiles overlay: all of them are past that
+            asm volatile("bar.sync 2, %0;" ::"r"(64 * NG) : "memory");
             const float kw = sc.kW[row], km = sc.kM[row];
 #pragma unroll
             for (int b = 0; b < NB; ++b) {
