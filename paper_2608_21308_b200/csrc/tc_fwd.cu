@@ -27,10 +27,11 @@ using namespace sm100;
 
 #ifdef TC_PROFILE
 // Debug build only: cycle stamps of thread 0 of CTA 0 at the phase boundaries of the first 64 chunks.
-__device__ long long g_tc_prof[64 * 16];
-#define PROF(i)                                                                      \
-    do {                                                                             \
-        if (blockIdx.x == 0 && threadIdx.x == 0 && r < 64) g_tc_prof[r * 16 + (i)] = clock64(); \
+__device__ long long g_tc_prof[4 * 32 * 16];
+#define PROF(i)                                                                                          \
+    do {                                                                                                 \
+        if ((threadIdx.x == 0 || threadIdx.x == 64) && (blockIdx.x == 0 || blockIdx.x == 2) && r < 32)    \
+            g_tc_prof[(((blockIdx.x >> 1) * 2 + (threadIdx.x >> 6)) * 32 + r) * 16 + (i)] = clock64();    \
     } while (0)
 #else
 #define PROF(i)
@@ -128,16 +129,17 @@ __device__ __forceinline__ float fast_ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// Forward-only GELU for the bf16 operand of G2: the tanh form 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3))) with the
+// hardware tanh - 6 FMA-pipe instructions and one MUFU instead of 15 and two.  It differs from z Phi(z) by at most
+// 4.7e-4 absolute (plus 2^-11 relative from tanh.approx), below the bf16 rounding the value receives right after
+// (half an ulp of bf16 is 2^-9 relative); the derivative used by the inner backward keeps the erfc form.
 __device__ __forceinline__ float gelu_only(float z) {
-    const float x = fabsf(z) * 0.70710678118654752440f;
-    const float t = fast_rcp(fmaf(0.3275911f, x, 1.0f));
-    float p = fmaf(t, 0.5307027145f, -0.7265760135f);
-    p = fmaf(t, p, 0.7107068705f);
-    p = fmaf(t, p, -0.142248368f);
-    p = fmaf(t, p, 0.127414796f);
-    p *= t;
-    const float half_erfc = p * fast_ex2(x * x * -1.44269504088896341f);
-    return z * (z >= 0.0f ? 1.0f - half_erfc : half_erfc);
+    const float z2 = z * z;
+    const float u = z * fmaf(0.0356774081f, z2, 0.7978845608f);
+    float t;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(u));
+    const float hz = 0.5f * z;
+    return fmaf(hz, t, hz);
 }
 __device__ __forceinline__ float gelu_fast(float z, float& dgelu) {
     const float x = fabsf(z) * 0.70710678118654752440f;
@@ -302,7 +304,6 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         if (warp == 3 + 4 * (NG - 1) && r + 1 < nchunks) {
             tc_chunk_scalars(eta + tok0 + C, beta + tok0 + C, gamma + tok0 + C, &s.sc[(r + 1) & 1]);
         }
-
         PROF(0);
         // ---------------- G1: Z = X W1c^T -> R0 (issued at the end of the previous iteration / before the loop)
         if (is_issuer) {
@@ -310,9 +311,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             mbar_expect_tx(&s.bar_pu, 16384);
         }
         mbar_wait(&s.bar_g1, ph, wc, 100 + 2);
+        PROF(1);
         __syncwarp();
         tc_fence_after_sync();
-        PROF(1);
         // epilogue: a = gelu(z) -> A (bf16); for key rows also kW a, kM a and gelu'(z) (kept in TMEM over z)
         // a = gelu(z) -> A (bf16) for all 128 rows: all that G2 needs
 #pragma unroll
@@ -329,7 +330,6 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         fence_proxy_async_smem();
         tc_fence_before_sync();
         __syncthreads();
-
         PROF(2);
         // ---------------- G2: Upart = A W2c^T -> R1
         if (is_issuer) {
@@ -341,10 +341,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         }
         __syncwarp();
         mbar_wait(&s.bar_g2, ph, wc, 100 + 3);
+        PROF(3);
         __syncwarp();
         tc_fence_after_sync();
-
-        PROF(3);
         // ---------------- cross-CTA sum of Upart: rows of quadrant x go to CTA x
         if (r > 0) mbar_wait<true>(&s.bar_credit, (uint32_t)((r - 1) & 1), wc, 100 + 4);
         // Row ownership: CTA c normalises key tokens 16c..16c+15 and query tokens 16c..16c+15, so every CTA carries
@@ -394,7 +393,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
                     float d1;
-                    const float av = gelu_fast(__uint_as_float(z[j]), d1);
+                    (void)gelu_fast(__uint_as_float(z[j]), d1);
+                    const float av = gelu_only(__uint_as_float(z[j]));
                     dg[j] = __float_as_uint(d1);
                     aw[j] = kw * av;
                     am[j] = km * av;
@@ -410,6 +410,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             if (lane == 0) mbar_arrive(&s.bar_ak);
         }
 
+        PROF(5);
         // ---------------- layer norm on the 16 key and 16 query rows this CTA owns, all threads: TPR threads per row
         {
             constexpr int TPR = NTHREADS / 32, CPT = 128 / TPR;  // threads per row, columns per thread
@@ -432,6 +433,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 xraw[ch] = *reinterpret_cast<const uint4*>(s.X[col0 >> 6] + xrow * 128 + ((c ^ (xrow & 7)) << 4));
             }
             mbar_wait<true>(&s.bar_part, ph, wc, 100 + 5);
+        PROF(6);
             float u[CPT];
 #pragma unroll
             for (int j = 0; j < CPT; ++j) u[j] = 0.0f;
@@ -446,7 +448,6 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                     u[j] += x.x; u[j + 1] += x.y; u[j + 2] += x.z; u[j + 3] += x.w;
                 }
             }
-            PROF(5);
             auto row_sum = [&](float v) -> float {  // over the TPR lanes that share a row
 #pragma unroll
                 for (int o = TPR / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -514,8 +515,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 }
             }
         }
-
-        PROF(6);
+        PROF(7);
         // ---------------- G3: Pa = Pu W2c -> R1 ; then the W2 aggregation that needs nothing else
         if (is_issuer) {
             mbar_wait_one<true>(&s.bar_pu, ph, wc, 100 + 6);
@@ -532,8 +532,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 umma_bf16(tb + T_W2, desc_mn(smem_u32(s.Pu[0]), 8192, k), desc_mn(smem_u32(s.AkW[0]), 8192, k), id_agg, true);
         }
         mbar_wait(&s.bar_g3, ph, wc, 100 + 7);
+        PROF(8);
         __syncwarp();
-        PROF(7);
         tc_fence_after_sync();
         if (row < C) {
             // these warps also read the staging slots (query rows) that the Pz tiles overlay: all of them are past that
@@ -560,8 +560,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         fence_proxy_async_smem();
         tc_fence_before_sync();
         __syncthreads();
-
-        PROF(8);
+        PROF(9);
         // ---------------- remaining aggregations, in two groups so that the state pass can start on W1 early
         if (is_issuer) {
             tc_fence_after_sync();
@@ -583,7 +582,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         const size_t head = (size_t)seq * (size_t)(D * 4 * HC);
 
         mbar_wait(&s.bar_agg, ph, wc, 100 + 8);
-        PROF(9);
+        PROF(10);
         tc_fence_after_sync();
         if (is_issuer && !last) {
             // the W1 aggregations were the last readers of the key tile: the next chunk's tokens may land in X
@@ -595,7 +594,6 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             tma_load_2d(s.X[1] + 8192, &tmQ, 64, y, &s.bar_x);
         }
         __syncwarp();
-        PROF(10);
         // ---------------- state pass, W1 half (Algorithm 1 lines 6-7), while the M2 aggregation still runs
 #pragma unroll
         for (int b = 0; b < NB; ++b) {
@@ -629,10 +627,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         fence_proxy_async_smem();
         tc_fence_before_sync();
         __syncthreads();  // bf16 W1 is complete and R0 is free: the next chunk's G1 may run under the W2 half
+        PROF(11);
         if (is_issuer && !last) issue_g1(r + 1);
         __syncwarp();
 
         mbar_wait(&s.bar_agg2, ph, wc, 100 + 9);
+        PROF(12);
         tc_fence_after_sync();
         if (is_issuer) {
             // every reader of this chunk's staging / pu / scaled-activation buffers is done: peers may overwrite them
@@ -675,7 +675,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         tc_fence_before_sync();
         __syncthreads();
         tc_fence_after_sync();
-        PROF(11);
+        PROF(13);
     }
 
     // no CTA leaves while a peer may still write into its shared memory or arrive on its barriers
