@@ -65,7 +65,7 @@ struct __align__(1024) Smem {
     uint8_t PzM[2][8192];  // kM_t pz                                                 staging slot 1
     uint8_t Stage2[16384]; // staging slot 2
     Scalars sc[2];
-    uint64_t bar_x, bar_g1, bar_g2, bar_g3, bar_agg, bar_agg2, bar_ak, bar_part, bar_pu, bar_credit;
+    uint64_t bar_x, bar_g1, bar_g2, bar_g3, bar_agg, bar_agg2, bar_ak, bar_v, bar_part, bar_pu, bar_credit;
     uint32_t tmem_base;
     int dead;
 };
@@ -116,45 +116,29 @@ __device__ void tc_chunk_scalars(const float* eta, const float* beta, const floa
     }
 }
 
-// GELU z Phi(z) and its derivative Phi(z) + z phi(z).  Phi through the five-term rational form of erfc
-// (Abramowitz & Stegun 7.1.26, absolute error 1.5e-7): one reciprocal, one exponential, a handful of FMAs.
-// The exponential exp(-z^2/2) is shared with the density phi.
-__device__ __forceinline__ float fast_rcp(float x) {
-    float y;
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
+// GELU on the bf16 path: the tanh form g(z) = 0.5 z (1 + tanh(u)), u = sqrt(2/pi) (z + 0.044715 z^3), with the
+// hardware tanh (6 FMA-pipe instructions and one MUFU), and its exact derivative
+// g'(z) = 0.5 (1 + T) + 0.5 z (1 - T^2) u'(z).  g differs from z Phi(z) by at most 4.7e-4 absolute and g' from
+// Phi(z) + z phi(z) by at most 8.7e-4 (plus 2^-11 relative from tanh.approx); both values are rounded to bf16 right
+// after (half an ulp = 2^-9 relative).  The fp32/fp64 SIMT path keeps the exact erf form.
+__device__ __forceinline__ float fast_tanh(float x) {
+    float t;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(x));
+    return t;
 }
-__device__ __forceinline__ float fast_ex2(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-// Forward-only GELU for the bf16 operand of G2: the tanh form 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3))) with the
-// hardware tanh - 6 FMA-pipe instructions and one MUFU instead of 15 and two.  It differs from z Phi(z) by at most
-// 4.7e-4 absolute (plus 2^-11 relative from tanh.approx), below the bf16 rounding the value receives right after
-// (half an ulp of bf16 is 2^-9 relative); the derivative used by the inner backward keeps the erfc form.
 __device__ __forceinline__ float gelu_only(float z) {
     const float z2 = z * z;
-    const float u = z * fmaf(0.0356774081f, z2, 0.7978845608f);
-    float t;
-    asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(u));
+    const float t = fast_tanh(z * fmaf(0.0356774081f, z2, 0.7978845608f));
     const float hz = 0.5f * z;
     return fmaf(hz, t, hz);
 }
 __device__ __forceinline__ float gelu_fast(float z, float& dgelu) {
-    const float x = fabsf(z) * 0.70710678118654752440f;
-    const float t = fast_rcp(fmaf(0.3275911f, x, 1.0f));
-    // 0.5 * (a1 t + ... + a5 t^5)
-    float p = fmaf(t, 0.5307027145f, -0.7265760135f);
-    p = fmaf(t, p, 0.7107068705f);
-    p = fmaf(t, p, -0.142248368f);
-    p = fmaf(t, p, 0.127414796f);
-    p *= t;
-    const float e = fast_ex2(x * x * -1.44269504088896341f);  // exp(-z^2/2)
-    const float half_erfc = p * e;                             // Phi(-|z|)
-    const float cdf = z >= 0.0f ? 1.0f - half_erfc : half_erfc;
-    dgelu = fmaf(z * 0.39894228040143267794f, e, cdf);
-    return z * cdf;
+    const float z2 = z * z;
+    const float t = fast_tanh(z * fmaf(0.0356774081f, z2, 0.7978845608f));
+    const float hz = 0.5f * z;
+    const float du = fmaf(0.1070322243f, z2, 0.7978845608f);  // u'(z)
+    dgelu = fmaf(hz * fmaf(-t, t, 1.0f), du, fmaf(0.5f, t, 0.5f));
+    return fmaf(hz, t, hz);
 }
 
 // Staging slot for partial sums: 32 rows x 128 fp32, kept as 16-byte pieces.  Piece c4 (4 columns) of row r sits at
@@ -176,7 +160,8 @@ __device__ __forceinline__ void st_slab16(uint8_t* slab, int row, int col0, cons
 }
 
 __global__ void __launch_bounds__(NTHREADS, 1)
-tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ, const TcFwdArgs a) {
+tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
+              const __grid_constant__ CUtensorMap tmV, const TcFwdArgs a) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     Smem& s = *reinterpret_cast<Smem*>(smem_raw);
     if ((smem_u32(smem_raw) & 1023u) != 0u) {  // the swizzled tiles need a 1024-byte aligned base: refuse to run otherwise
@@ -197,7 +182,6 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     WaitCtx wc{&s.dead, a.status};
 
     const __nv_bfloat16* gk = a.k + (size_t)seq * L * D;
-    const __nv_bfloat16* gv = a.v + (size_t)seq * L * D;
     const __nv_bfloat16* gq = a.q + (size_t)seq * L * D;
     __nv_bfloat16* go = a.o + (size_t)seq * L * D;
     const float* eta = a.eta + (size_t)seq * L;
@@ -213,12 +197,14 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         mbar_init(&s.bar_agg, 1);
         mbar_init(&s.bar_agg2, 1);
         mbar_init(&s.bar_ak, 2 * NG);
+        mbar_init(&s.bar_v, 1);
         mbar_init(&s.bar_part, 1);  // + 3 x 16 KB of peer partial sums per chunk
         mbar_init(&s.bar_pu, 1);    // + 16 KB of pu rows per chunk
         mbar_init(&s.bar_credit, 3);
         fence_mbar_init();
         tma_prefetch_desc(&tmK);
         tma_prefetch_desc(&tmQ);
+        tma_prefetch_desc(&tmV);
     }
     if (warp == 0) { tmem_alloc(&s.tmem_base, 512); tmem_relinquish(); }
     if (warp == 1) tc_chunk_scalars(eta, beta, gamma, &s.sc[0]);
@@ -341,6 +327,14 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         }
         __syncwarp();
         mbar_wait(&s.bar_g2, ph, wc, 100 + 3);
+        if (is_issuer) {
+            // the 16 value rows this CTA needs for its key rows: into the gelu tile's first slab, dead once G2 is done
+            mbar_expect_tx(&s.bar_v, 4096);
+            const int y = seq * L + tok0 + 16 * (int)me;
+            tma_load_2d(s.A[0], &tmV, 0, y, &s.bar_v);
+            tma_load_2d(s.A[0] + 2048, &tmV, 64, y, &s.bar_v);
+        }
+        __syncwarp();
         PROF(3);
         __syncwarp();
         tc_fence_after_sync();
@@ -393,8 +387,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
                     float d1;
-                    (void)gelu_fast(__uint_as_float(z[j]), d1);
-                    const float av = gelu_only(__uint_as_float(z[j]));
+                    const float av = gelu_fast(__uint_as_float(z[j]), d1);
                     dg[j] = __float_as_uint(d1);
                     aw[j] = kw * av;
                     am[j] = km * av;
@@ -428,11 +421,19 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             uint4 vraw[CPT / 8], xraw[CPT / 8];
 #pragma unroll
             for (int ch = 0; ch < CPT / 8; ++ch) {
-                if (key_rows) vraw[ch] = *reinterpret_cast<const uint4*>(gv + off + 8 * ch);
                 const int c = ((col0 & 63) >> 3) + ch;
                 xraw[ch] = *reinterpret_cast<const uint4*>(s.X[col0 >> 6] + xrow * 128 + ((c ^ (xrow & 7)) << 4));
             }
             mbar_wait<true>(&s.bar_part, ph, wc, 100 + 5);
+            if (key_rows) {
+                mbar_wait(&s.bar_v, ph, wc, 100 + 11);
+                const int lr = lrow & 15;
+#pragma unroll
+                for (int ch = 0; ch < CPT / 8; ++ch) {
+                    const int c = ((col0 & 63) >> 3) + ch;
+                    vraw[ch] = *reinterpret_cast<const uint4*>(s.A[0] + (col0 >> 6) * 2048 + lr * 128 + ((c ^ (lr & 7)) << 4));
+                }
+            }
         PROF(6);
             float u[CPT];
 #pragma unroll
@@ -703,13 +704,13 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// [rows][128] bf16 row-major, tiles of 64 rows x 64 columns, 128-byte swizzle
-bool make_token_map(CUtensorMap* tm, const void* base, size_t rows) {
+// [rows][128] bf16 row-major, tiles of box_rows rows x 64 columns, 128-byte swizzle
+bool make_token_map(CUtensorMap* tm, const void* base, size_t rows, unsigned box_rows) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)D * 2};
-    cuuint32_t box[2] = {64, 64};
+    cuuint32_t box[2] = {64, box_rows};
     cuuint32_t es[2] = {1, 1};
     return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -728,9 +729,10 @@ extern "C" __attribute__((visibility("default"))) int e2ttt_debug_read_profile(l
 
 int tc_fwd_launch(const TcFwdArgs& a, void* stream) {
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    CUtensorMap tmK, tmQ;
+    CUtensorMap tmK, tmQ, tmV;
     const size_t rows = (size_t)a.N * a.L;
-    if (!make_token_map(&tmK, a.k, rows) || !make_token_map(&tmQ, a.q, rows)) return (int)cudaErrorInvalidValue;
+    if (!make_token_map(&tmK, a.k, rows, 64) || !make_token_map(&tmQ, a.q, rows, 64) || !make_token_map(&tmV, a.v, rows, 16))
+        return (int)cudaErrorInvalidValue;
     static bool attr_done[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return (int)cudaGetLastError();
@@ -754,7 +756,7 @@ int tc_fwd_launch(const TcFwdArgs& a, void* stream) {
     at[0].val.clusterDim.z = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    e = cudaLaunchKernelEx(&cfg, tc_fwd_kernel, tmK, tmQ, a);
+    e = cudaLaunchKernelEx(&cfg, tc_fwd_kernel, tmK, tmQ, tmV, a);
     if (e != cudaSuccess) return (int)e;
     return (int)cudaGetLastError();
 }
