@@ -65,7 +65,7 @@ struct __align__(1024) Smem {
     uint8_t PzM[2][8192];  // kM_t pz                                                 staging slot 1
     uint8_t Stage2[16384]; // staging slot 2
     Scalars sc[2];
-    uint64_t bar_x, bar_g1, bar_g2, bar_g3, bar_agg, bar_agg2, bar_ak, bar_v, bar_part, bar_pu, bar_credit;
+    uint64_t bar_x, bar_g1, bar_g2, bar_g3, bar_agg, bar_agg2, bar_ak, bar_v, bar_ksent, bar_partK, bar_partQ, bar_pu, bar_credit;
     uint32_t tmem_base;
     int dead;
 };
@@ -198,7 +198,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         mbar_init(&s.bar_agg2, 1);
         mbar_init(&s.bar_ak, 2 * NG);
         mbar_init(&s.bar_v, 1);
-        mbar_init(&s.bar_part, 1);  // + 3 x 16 KB of peer partial sums per chunk
+        mbar_init(&s.bar_partK, 1);  // + 3 x 8 KB of peer partial sums (key rows) per chunk
+        mbar_init(&s.bar_partQ, 1);  // + 3 x 8 KB (query rows)
+        mbar_init(&s.bar_ksent, 2 * NG);
         mbar_init(&s.bar_pu, 1);    // + 16 KB of pu rows per chunk
         mbar_init(&s.bar_credit, 3);
         fence_mbar_init();
@@ -293,7 +295,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         PROF(0);
         // ---------------- G1: Z = X W1c^T -> R0 (issued at the end of the previous iteration / before the loop)
         if (is_issuer) {
-            mbar_expect_tx(&s.bar_part, 3 * 16384);  // this chunk's incoming partial sums and pu rows
+            mbar_expect_tx(&s.bar_partK, 3 * 8192);  // this chunk's incoming partial sums and pu rows
+            mbar_expect_tx(&s.bar_partQ, 3 * 8192);
             mbar_expect_tx(&s.bar_pu, 16384);
         }
         mbar_wait(&s.bar_g1, ph, wc, 100 + 2);
@@ -338,11 +341,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         PROF(3);
         __syncwarp();
         tc_fence_after_sync();
-        // ---------------- cross-CTA sum of Upart: rows of quadrant x go to CTA x
-        if (r > 0) mbar_wait<true>(&s.bar_credit, (uint32_t)((r - 1) & 1), wc, 100 + 4);
         // Row ownership: CTA c normalises key tokens 16c..16c+15 and query tokens 16c..16c+15, so every CTA carries
         // the same mix of work.  TMEM lane 32q+l holds key token 32q+l (q < 2) or query token 32(q-2)+l.
-        {
+        auto send_rows = [&](uint64_t* bar_local) {
             const uint32_t owner = 2u * ((uint32_t)q & 1u) + ((uint32_t)lane >> 4);
             const uint32_t srow = ((q < 2) ? 0u : 16u) + ((uint32_t)lane & 15u);  // row inside the owner's staging slot
             const bool mine = owner == me;
@@ -353,7 +354,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 const uint32_t slot = (me - owner - 1u) & 3u;  // where the owner keeps what comes from me
                 const uint8_t* p = (slot == 0) ? s.PzW[0] : (slot == 1) ? s.PzM[0] : s.Stage2;
                 dst_base = map_to_cta(smem_u32(p), owner);
-                dst_bar = map_to_cta(smem_u32(&s.bar_part), owner);
+                dst_bar = map_to_cta(smem_u32(bar_local), owner);
             }
 #pragma unroll
             for (int b = 0; b < NB; ++b) {
@@ -368,14 +369,11 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                     else st_async_v4(dst, u[j], u[j + 1], u[j + 2], u[j + 3], dst_bar);
                 }
             }
-        }
-        tc_fence_before_sync();
-        __syncthreads();  // R1 has been read by everyone (G3 may overwrite it); own rows are staged
-        PROF(4);
+        };
 
-        // While the partial sums travel: what only the inner backward needs, for the key rows (the warps of TMEM
-        // quadrants 0 and 1): kW a, kM a (operands of the W2 aggregations) and gelu'(z), which replaces z in TMEM.
-        if (row < C) {
+        // What only the inner backward needs, for the key rows (the warps of TMEM quadrants 0 and 1): kW a, kM a
+        // (operands of the W2 aggregations) and gelu'(z), which replaces z in TMEM.  Runs while pu travels.
+        auto backward_extras = [&]() {
             const float kw = sc.kW[row], km = sc.kM[row];
 #pragma unroll
             for (int b = 0; b < NB; ++b) {
@@ -401,17 +399,14 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) mbar_arrive(&s.bar_ak);
-        }
+        };
 
-        PROF(5);
-        // ---------------- layer norm on the 16 key and 16 query rows this CTA owns, all threads: TPR threads per row
-        {
+        // Layer norm on the 16 key rows (warps of quadrants 0/1) or the 16 query rows (quadrants 2/3) this CTA owns:
+        // 16 threads per row, 8 columns each.
+        auto layer_norm = [&](const bool key_rows) {
             constexpr int TPR = NTHREADS / 32, CPT = 128 / TPR;  // threads per row, columns per thread
             static_assert(TPR == 16, "row mapping below assumes two rows per warp");
-            // staging rows 0..15: key tokens, 16..31: query tokens.  The key rows (which the whole cluster waits for)
-            // go to the warps of quadrants 2 and 3, which are free; the warps of quadrants 0 and 1 arrive later
-            // (they have just produced the backward-only operands) and take the query rows.
-            const bool key_rows = q >= 2;
+            // staging rows 0..15: key tokens, 16..31: query tokens
             const int lrow = (key_rows ? 0 : 16) + 2 * ((q & 1) + 2 * g) + (lane >> 4);
             const int cg = lane & 15;
             const int t = 16 * (int)me + (lrow & 15);    // token inside the chunk
@@ -424,7 +419,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 const int c = ((col0 & 63) >> 3) + ch;
                 xraw[ch] = *reinterpret_cast<const uint4*>(s.X[col0 >> 6] + xrow * 128 + ((c ^ (xrow & 7)) << 4));
             }
-            mbar_wait<true>(&s.bar_part, ph, wc, 100 + 5);
+            mbar_wait<true>(key_rows ? &s.bar_partK : &s.bar_partQ, ph, wc, 100 + 5);
             if (key_rows) {
                 mbar_wait(&s.bar_v, ph, wc, 100 + 11);
                 const int lr = lrow & 15;
@@ -434,7 +429,6 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                     vraw[ch] = *reinterpret_cast<const uint4*>(s.A[0] + (col0 >> 6) * 2048 + lr * 128 + ((c ^ (lr & 7)) << 4));
                 }
             }
-        PROF(6);
             float u[CPT];
 #pragma unroll
             for (int j = 0; j < CPT; ++j) u[j] = 0.0f;
@@ -515,6 +509,35 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                     *reinterpret_cast<uint4*>(go + off + 8 * ch) = ov;
                 }
             }
+        };
+
+        // ---------------- cross-CTA sum of Upart, layer norm, pu broadcast
+        // The key rows are on the critical path of the whole cluster, the query rows are not.  So the warps holding
+        // key rows (quadrants 0/1) hand them to the network first, normalise this CTA's key rows as soon as the
+        // peers' pieces are in, broadcast pu, and only then produce the backward-only operands; the warps holding
+        // query rows (quadrants 2/3) send after the key rows have gone out, normalise the query rows, write o.
+        if (r > 0) mbar_wait<true>(&s.bar_credit, (uint32_t)((r - 1) & 1), wc, 100 + 4);
+        if (q < 2) {
+            send_rows(&s.bar_partK);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&s.bar_ksent);
+            asm volatile("bar.sync 4, %0;" ::"r"(64 * NG) : "memory");  // this CTA's own key rows are staged
+            PROF(4);
+            layer_norm(true);
+            PROF(5);
+            backward_extras();
+            PROF(6);
+            // the Pz tiles (G3 epilogue, below) overlay staging slots: wait until the query-row readers are done too
+            asm volatile("bar.sync 3, %0;" ::"r"(128 * NG) : "memory");
+        } else {
+            mbar_wait(&s.bar_ksent, ph, wc, 100 + 12);
+            send_rows(&s.bar_partQ);
+            asm volatile("bar.sync 5, %0;" ::"r"(64 * NG) : "memory");  // own query rows staged; R1 fully read
+            PROF(4);
+            layer_norm(false);
+            PROF(5);
+            asm volatile("bar.arrive 3, %0;" ::"r"(128 * NG) : "memory");
+            PROF(6);
         }
         PROF(7);
         // ---------------- G3: Pa = Pu W2c -> R1 ; then the W2 aggregation that needs nothing else
@@ -537,8 +560,6 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         __syncwarp();
         tc_fence_after_sync();
         if (row < C) {
-            // these warps also read the staging slots (query rows) that the Pz tiles overlay: all of them are past that
-            asm volatile("bar.sync 2, %0;" ::"r"(64 * NG) : "memory");
             const float kw = sc.kW[row], km = sc.kM[row];
 #pragma unroll
             for (int b = 0; b < NB; ++b) {
