@@ -295,6 +295,13 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         PROF(0);
         // ---------------- G1: Z = X W1c^T -> R0 (issued at the end of the previous iteration / before the loop)
         if (is_issuer) {
+            if (r + 1 < nchunks) {
+                // the next chunk's tokens: into L2 now, so that the loads issued at the end of this chunk are short
+                const int y = seq * L + tok0 + C;
+                tma_prefetch_l2_2d(&tmK, 0, y); tma_prefetch_l2_2d(&tmK, 64, y);
+                tma_prefetch_l2_2d(&tmQ, 0, y); tma_prefetch_l2_2d(&tmQ, 64, y);
+                tma_prefetch_l2_2d(&tmV, 0, y + 16 * (int)me); tma_prefetch_l2_2d(&tmV, 64, y + 16 * (int)me);
+            }
             mbar_expect_tx(&s.bar_partK, 3 * 8192);  // this chunk's incoming partial sums and pu rows
             mbar_expect_tx(&s.bar_partQ, 3 * 8192);
             mbar_expect_tx(&s.bar_pu, 16384);
