@@ -279,6 +279,85 @@ def run_ours(args, r):
         dist.destroy_process_group()
 
 
+def run_fwd_bwd(args, r):
+    """Optional second workload (--backward): one step = e2ttt_chunk_fwd(save_states=1) + e2ttt_chunk_bwd on the same
+    batch (GELU-MLP only).  Both run on the SIMT path today; the line says so."""
+    import torch
+    from paper_2608_21308_b200 import binding as E
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    x = inputs.generate(r, with_d_o=True)
+    N = r.B * r.H
+    iod = torch.float32 if r.io == "f32" else torch.bfloat16
+    p = E.make_params(r.B, r.H, r.L, r.d, r.h, r.C, r.kind, E.E2TTT_F32 if r.io == "f32" else E.E2TTT_BF16, 1e-5,
+                      E.E2TTT_IMPL_AUTO)
+    s4, s3 = (r.B, r.H, r.L, r.d), (r.B, r.H, r.L)
+    shapes = inputs.mat_shapes(r.kind, r.d, r.h)
+    host = {n: torch.from_numpy(x[n]).to(iod).view(s4).pin_memory() for n in ("q", "k", "v", "d_o")}
+    host.update({n: torch.from_numpy(x[n]).view(s3).pin_memory() for n in ("eta", "beta", "gamma")})
+    hostW = [torch.from_numpy(w).view((r.B, r.H) + s).pin_memory() for w, s in zip(x["W"], shapes)]
+    t = {n: v.to(dev) for n, v in host.items()}
+    W0 = [w.to(dev) for w in hostW]
+    o = torch.empty(s4, dtype=iod, device=dev)
+    Wf = [torch.empty_like(w) for w in W0]
+    Mf = [torch.empty_like(w) for w in W0]
+    dq, dk, dv = (torch.empty(s4, dtype=iod, device=dev) for _ in range(3))
+    de, db, dg = (torch.empty(s3, dtype=torch.float32, device=dev) for _ in range(3))
+    dW = [torch.empty_like(w) for w in W0]
+    dM = [torch.empty_like(w) for w in W0]
+    ws = torch.empty(E.e2ttt_workspace_bytes(p, 1), dtype=torch.uint8, device=dev)
+    hout = [torch.empty(s4, dtype=iod).pin_memory() for _ in range(4)]
+    stream = torch.cuda.current_stream()
+
+    def step():
+        E.e2ttt_chunk_fwd(p, t["q"], t["k"], t["v"], t["eta"], t["beta"], t["gamma"], W0, None, o, Wf, Mf, ws, 1, stream)
+        E.e2ttt_chunk_bwd(p, t["q"], t["k"], t["v"], t["eta"], t["beta"], t["gamma"], W0, None, t["d_o"], None, None,
+                          dq, dk, dv, de, db, dg, dW, dM, ws, 1, stream)
+
+    def step_e2e():
+        for n in host:
+            t[n].copy_(host[n], non_blocking=True)
+        step()
+        for a, b in zip(hout, (o, dq, dk, dv)):
+            a.copy_(b, non_blocking=True)
+
+    def timed(fn, steps, warmup):
+        for _ in range(warmup):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+
+    sampler = ClockSampler(0)
+    sampler.start()
+    ms = timed(step, args.steps, args.warmup)
+    clocks = sampler.stop()
+    ms_e2e = timed(step_e2e, max(1, args.steps // 2), 1)
+    pk = peaks()
+    tokens = r.B * r.L
+    flop = flops_per_token_head(r, backward=True) * N * r.L
+    cfg = workload_config(r)
+    cfg["workload"] = cfg["workload"].replace("e2ttt_chunk_fwd", "e2ttt_chunk_fwd(save_states) + e2ttt_chunk_bwd")
+    cfg["path"] = "SIMT kernels (the tensor-core path covers the forward without saved states only)"
+    line = {"metric": "e2ttt_layer_fwd_bwd_tokens_per_s", "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if r.io == "bf16" else "f64", "data": "synthetic", "config": cfg,
+            "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": sum(v.numel() * v.element_size() for v in host.values()),
+                    "d2h_bytes_per_step": sum(v.numel() * v.element_size() for v in hout), "ms_per_step": ms_e2e},
+            "gpu_launches": 2 * args.steps, "clocks": clocks,
+            "roofline": {"bound": "tensor", "achieved": flop / (ms * 1e-3) / 1e12, "peak": pk["bf16_tflops"],
+                         "unit": "TFLOP/s", "frac": flop / (ms * 1e-3) / 1e12 / pk["bf16_tflops"], "traffic": None,
+                         "peak_source": pk["_source"], "flop_per_step": flop}}
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -287,10 +366,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, help="benchmark configuration index (default: the 1.3B-layer shape)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--backward", action="store_true", help="time forward + backward instead (1 GPU, GELU-MLP configs)")
+    ap.add_argument("--chunk", type=int, default=0, help="override the chunk size C of the configuration")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    r = inputs.config(args.config)
-    if args.impl == "reference":
+    r = inputs.config(args.config, **({"C": args.chunk} if args.chunk else {}))
+    if args.backward and args.impl == "ours":
+        run_fwd_bwd(args, r)
+    elif args.impl == "reference":
         run_reference(args, r)
     else:
         run_ours(args, r)
