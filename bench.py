@@ -155,6 +155,23 @@ def run_reference(args, r):
     print(json.dumps(line))
 
 
+def shard_recipe(r, rank: int):
+    """Rank `rank`'s share of an N-GPU run: the same shapes, its own seeded batch (weak scaling, no exchange)."""
+    return inputs.Recipe(**{**r.__dict__, "seed": r.seed + rank})
+
+
+def whole_job_value(world: int, tokens_per_rank: int, ms_max_over_ranks: float) -> float:
+    """Whole-job throughput: the tokens all ranks processed / the slowest rank's device time."""
+    return world * tokens_per_rank / (ms_max_over_ranks * 1e-3)
+
+
+def max_over_ranks(ms: float, dist, device) -> float:
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def workload_config(r):
     kind = "mlp_gelu" if r.kind == inputs.KIND_MLP else "swiglu"
     return {"workload": f"e2ttt_chunk_fwd B={r.B} H={r.H} L={r.L} d={r.d} h={r.h} C={r.C} {kind} {r.io} I/O",
@@ -176,8 +193,7 @@ def run_ours(args, r):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     dev = torch.device("cuda", local)
 
-    rr = inputs.Recipe(**{**r.__dict__, "seed": r.seed + rank})
-    x = inputs.generate(rr)
+    x = inputs.generate(shard_recipe(r, rank))
     N = r.B * r.H
     iod = torch.float32 if r.io == "f32" else torch.bfloat16
     p = E.make_params(r.B, r.H, r.L, r.d, r.h, r.C, r.kind, E.E2TTT_F32 if r.io == "f32" else E.E2TTT_BF16, 1e-5,
@@ -231,9 +247,7 @@ def run_ours(args, r):
         barrier()
         ms = e0.elapsed_time(e1) / steps
         if world > 1:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+            ms = max_over_ranks(ms, dist, dev)
         return ms
 
     sampler = ClockSampler(local)
@@ -257,11 +271,11 @@ def run_ours(args, r):
         h2d = sum(t.numel() * t.element_size() for t in host.values()) + sum(w.numel() * 4 for w in hostW)
         d2h = host_o.numel() * host_o.element_size() + 2 * sum(w.numel() * 4 for w in hostW)
         line = {
-            "metric": METRIC, "value": world * tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "metric": METRIC, "value": whole_job_value(world, tokens, ms), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if r.io == "bf16" else "f64",
             "data": "synthetic", "config": workload_config(r),
-            "e2e": {"value": world * tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "e2e": {"value": whole_job_value(world, tokens, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
             "gpu_launches": args.steps,
             "clocks": clocks,
