@@ -71,7 +71,7 @@ typedef enum { E2TTT_IMPL_AUTO = 0, E2TTT_IMPL_SIMT = 1, E2TTT_IMPL_TCGEN05 = 2 
 typedef enum {
     E2TTT_OK = 0,
     E2TTT_ERR_NULL = -1,      /* a required pointer is NULL */
-    E2TTT_ERR_SHAPE = -2,     /* non-positive dimension, C > 128, d or h beyond the compiled limits,
+    E2TTT_ERR_SHAPE = -2,     /* non-positive dimension, C > 512, d or h beyond the compiled limits,
                                  L not a multiple of C on a path that needs it, unknown kind */
     E2TTT_ERR_DTYPE = -3,     /* unknown io_dtype / impl */
     E2TTT_ERR_ALIGN = -4,     /* q, k, v, o (and gradients) must be 16-byte aligned */
@@ -86,7 +86,8 @@ typedef struct {
     int32_t L;        /* tokens per sequence */
     int32_t d;        /* head dimension (input and output width of the fast-weight network) */
     int32_t h;        /* hidden width of the fast-weight network */
-    int32_t C;        /* chunk size, 1..128.  The SIMT path accepts a shorter last chunk. */
+    int32_t C;        /* chunk size, 1..512 (the paper trains with 512); the tensor-core path serves C = 64.
+                         The SIMT path accepts a shorter last chunk. */
     int32_t kind;     /* e2ttt_kind */
     int32_t io_dtype; /* e2ttt_dtype of q, k, v, o, d_o, dq, dk, dv */
     float ln_eps;     /* layer-norm epsilon (the paper gives none; 1e-5 is the usual default) */

@@ -11,7 +11,7 @@ namespace {
 
 constexpr int kMaxD = 1024;
 constexpr int kMaxH = 8192;
-constexpr int kMaxChunk = 128;
+constexpr int kMaxChunk = 512;
 
 int nmat_of(int kind) { return kind == E2TTT_MLP_GELU ? 2 : (kind == E2TTT_SWIGLU ? 3 : 0); }
 

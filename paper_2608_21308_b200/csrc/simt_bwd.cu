@@ -29,10 +29,13 @@ __device__ __forceinline__ void warp_ln_jac(const Real* x, const Real* y, Real r
 template <typename Real, typename IO>
 __global__ void __launch_bounds__(kSimtThreads) simt_bwd_mlp_kernel(const SimtBwdArgs a) {
     constexpr int NMAT = 2;
-    __shared__ GemmSmem<Real> gsm;
-    __shared__ ChunkScalars<Real> sc;
-    __shared__ BwdScalars<Real> bs;
-    __shared__ Real red[8];
+    extern __shared__ __align__(16) unsigned char simt_smem_raw[];
+    GemmSmem<Real>& gsm = *reinterpret_cast<GemmSmem<Real>*>(simt_smem_raw);
+    ChunkScalars<Real>& sc = *reinterpret_cast<ChunkScalars<Real>*>(simt_smem_raw + sizeof(GemmSmem<Real>));
+    BwdScalars<Real>& bs =
+        *reinterpret_cast<BwdScalars<Real>*>(simt_smem_raw + sizeof(GemmSmem<Real>) + sizeof(ChunkScalars<Real>));
+    Real* red = reinterpret_cast<Real*>(simt_smem_raw + sizeof(GemmSmem<Real>) + sizeof(ChunkScalars<Real>) +
+                                        sizeof(BwdScalars<Real>));
 
     const int seq = blockIdx.x;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -359,13 +362,26 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_mlp_kernel(const SimtBw
     }
 }
 
+template <typename Real, typename IO>
+static int launch_bwd(const SimtBwdArgs& a, cudaStream_t st) {
+    constexpr size_t smem =
+        sizeof(GemmSmem<Real>) + sizeof(ChunkScalars<Real>) + sizeof(BwdScalars<Real>) + 8 * sizeof(Real);
+    static bool attr_done[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return (int)cudaGetLastError();
+    if (dev < 0 || dev >= 64 || !attr_done[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(simt_bwd_mlp_kernel<Real, IO>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return (int)e;
+        if (dev >= 0 && dev < 64) attr_done[dev] = true;
+    }
+    simt_bwd_mlp_kernel<Real, IO><<<dim3(a.N), dim3(kSimtThreads), smem, st>>>(a);
+    return (int)cudaGetLastError();
+}
+
 int simt_bwd_launch(const SimtBwdArgs& a, int kind, int io_dtype, void* stream) {
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    dim3 grid(a.N), block(kSimtThreads);
     if (kind != 0) return (int)cudaErrorInvalidValue;
-    if (io_dtype == 0) simt_bwd_mlp_kernel<double, float><<<grid, block, 0, st>>>(a);
-    else simt_bwd_mlp_kernel<float, __nv_bfloat16><<<grid, block, 0, st>>>(a);
-    return (int)cudaGetLastError();
+    return io_dtype == 0 ? launch_bwd<double, float>(a, st) : launch_bwd<float, __nv_bfloat16>(a, st);
 }
 
 }  // namespace e2ttt

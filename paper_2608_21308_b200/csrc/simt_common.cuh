@@ -8,7 +8,7 @@
 namespace e2ttt {
 
 constexpr int kSimtThreads = 256;
-constexpr int kMaxC = 128;
+constexpr int kMaxC = 512;  // the paper trains with chunks of 512 tokens
 constexpr int kMaxMat = 3;
 constexpr int kBM = 64, kBN = 64, kBK = 16;
 

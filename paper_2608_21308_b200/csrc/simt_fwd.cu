@@ -9,8 +9,9 @@ template <typename Real, typename IO, int KIND>
 __global__ void __launch_bounds__(kSimtThreads) simt_fwd_kernel(const SimtFwdArgs a) {
     constexpr int NMAT = (KIND == 0) ? 2 : 3;
     constexpr int LAST = NMAT - 1;
-    __shared__ GemmSmem<Real> gsm;
-    __shared__ ChunkScalars<Real> sc;
+    extern __shared__ __align__(16) unsigned char simt_smem_raw[];
+    GemmSmem<Real>& gsm = *reinterpret_cast<GemmSmem<Real>*>(simt_smem_raw);
+    ChunkScalars<Real>& sc = *reinterpret_cast<ChunkScalars<Real>*>(simt_smem_raw + sizeof(GemmSmem<Real>));
 
     const int seq = blockIdx.x;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -167,17 +168,25 @@ __global__ void __launch_bounds__(kSimtThreads) simt_fwd_kernel(const SimtFwdArg
     }
 }
 
+template <typename Real, typename IO, int KIND>
+static int launch_fwd(const SimtFwdArgs& a, cudaStream_t st) {
+    constexpr size_t smem = sizeof(GemmSmem<Real>) + sizeof(ChunkScalars<Real>);
+    static bool attr_done[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return (int)cudaGetLastError();
+    if (dev < 0 || dev >= 64 || !attr_done[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(simt_fwd_kernel<Real, IO, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return (int)e;
+        if (dev >= 0 && dev < 64) attr_done[dev] = true;
+    }
+    simt_fwd_kernel<Real, IO, KIND><<<dim3(a.N), dim3(kSimtThreads), smem, st>>>(a);
+    return (int)cudaGetLastError();
+}
+
 int simt_fwd_launch(const SimtFwdArgs& a, int kind, int io_dtype, void* stream) {
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    dim3 grid(a.N), block(kSimtThreads);
-    if (io_dtype == 0) {
-        if (kind == 0) simt_fwd_kernel<double, float, 0><<<grid, block, 0, st>>>(a);
-        else simt_fwd_kernel<double, float, 1><<<grid, block, 0, st>>>(a);
-    } else {
-        if (kind == 0) simt_fwd_kernel<float, __nv_bfloat16, 0><<<grid, block, 0, st>>>(a);
-        else simt_fwd_kernel<float, __nv_bfloat16, 1><<<grid, block, 0, st>>>(a);
-    }
-    return (int)cudaGetLastError();
+    if (io_dtype == 0) return kind == 0 ? launch_fwd<double, float, 0>(a, st) : launch_fwd<double, float, 1>(a, st);
+    return kind == 0 ? launch_fwd<float, __nv_bfloat16, 0>(a, st) : launch_fwd<float, __nv_bfloat16, 1>(a, st);
 }
 
 }  // namespace e2ttt

@@ -75,7 +75,7 @@ def test_workspace_sizes(L):
 
 
 @pytest.mark.parametrize("field,value,status", [
-    ("B", 0, -2), ("L", -1, -2), ("C", 0, -2), ("C", 129, -2), ("d", 0, -2), ("h", 100000, -2),
+    ("B", 0, -2), ("L", -1, -2), ("C", 0, -2), ("C", 513, -2), ("d", 0, -2), ("h", 100000, -2),
     ("kind", 2, -2), ("io_dtype", 5, -3), ("impl", 9, -3), ("impl", 2, -2),
 ])
 def test_bad_parameters_are_rejected(L, field, value, status):

@@ -103,6 +103,25 @@ def test_paper_regime_free_running_fp32():
     check_forward(got, ref, TOL_F32, "paper regime")
 
 
+def test_paper_chunk_size_512_forward_and_backward_fp32():
+    """The paper's own setting: chunks of 512 tokens, eta_base 0.01, tau 32, alpha_base 0.1 (free-running)."""
+    r = inputs.paper_regime(inputs.Recipe(B=2, H=1, L=1024 + 100, d=64, h=256, C=512, kind=MLP, seed=12, m_std=0.002))
+    x = inputs.generate(r, with_d_o=True, with_dstate=True)
+    ref = util.oracle_forward(x, r.C, MLP)
+    got, _ = util.gpu_forward(x, d=r.d, h=r.h, C=r.C, kind=MLP, io="f32")
+    check_forward(got, ref, TOL_F32, "C=512 forward")
+    rs = inputs.paper_regime(inputs.Recipe(B=1, H=1, L=768, d=32, h=64, C=512, kind=MLP, seed=13, m_std=0.002))
+    xs = inputs.generate(rs, with_d_o=True, with_dstate=True)
+    refb = util.oracle_backward(xs, rs.C, MLP)
+    gotb = util.gpu_backward(xs, d=rs.d, h=rs.h, C=rs.C, kind=MLP, io="f32")
+    check_backward(gotb, refb, TOL_F32, "C=512 backward")
+    rw = inputs.paper_regime(inputs.Recipe(B=2, H=1, L=512, d=64, h=192, C=256, kind=SWIGLU, io="bf16", seed=14))
+    xw = inputs.generate(rw)
+    refw = util.oracle_forward(xw, rw.C, SWIGLU)
+    gotw, _ = util.gpu_forward(xw, d=rw.d, h=rw.h, C=rw.C, kind=SWIGLU, io="bf16")
+    check_forward(gotw, refw, TOL_BF16, "C=256 SwiGLU bf16 forward")
+
+
 # ------------------------------------------------------------------ configs 1-4: teacher-forced one-chunk windows, bf16 I/O
 WINDOW_CASES = [
     ("config1", 1, dict(heads=[0, 37, 95]), 8),
