@@ -139,7 +139,7 @@ E2TTT_API int e2ttt_chunk_fwd(const e2ttt_params* p,
  *   states_saved           != 0: the workspace still holds the chunk-start states written by
  *                          e2ttt_chunk_fwd(save_states=1) for the same inputs; 0: they are
  *                          recomputed first
- * Only E2TTT_MLP_GELU has a reverse pass; E2TTT_SWIGLU returns E2TTT_ERR_SHAPE.
+ * Both network kinds are supported (SIMT path).
  */
 E2TTT_API int e2ttt_chunk_bwd(const e2ttt_params* p,
                     const void* q, const void* k, const void* v,

@@ -168,7 +168,6 @@ int e2ttt_chunk_bwd(const e2ttt_params* p, const void* q, const void* k, const v
                     float* const* dM_init, void* workspace, size_t workspace_bytes, int states_saved, void* stream) {
     int rc = check_params(p);
     if (rc) return rc;
-    if (p->kind != E2TTT_MLP_GELU) return E2TTT_ERR_SHAPE;
     if (!q || !k || !v || !eta || !beta || !gamma || !W_init || !d_o || !dq || !dk || !dv || !d_eta || !d_beta ||
         !d_gamma || !dW_init || !dM_init)
         return E2TTT_ERR_NULL;

@@ -1,11 +1,14 @@
-// SIMT backward (GELU-MLP fast weights): the adjoint of the chunk program, chunks in reverse order,
-// one CTA per sequence.  Per chunk it re-runs the chunk's forward from the saved chunk-start state, then
-// reverses, in matrix form over the whole chunk,
+// SIMT backward: the adjoint of the chunk program, chunks in reverse order, one CTA per sequence, for both
+// fast-weight networks.  Per chunk it re-runs the chunk's forward from the saved chunk-start state, then reverses,
+// in matrix form over the whole chunk,
 //   (i)   the outputs o = f_{W0}(q),
 //   (ii)  the closed-form state transition of Proposition 1 (carries cw, cm, cb and kernels K^W, K^M),
-//   (iii) the per-token gradients G_t(W0, k_t, v_t) - a second-order pass through LN and GELU,
+//   (iii) the per-token gradients G_t(W0, k_t, v_t) - a second-order pass through LN and the activation,
 //   (iv)  the suffix scans that made the scalar kernels.
-// Notation: T, S = adjoints of the chunk-end (W, M); a trailing "b" marks an adjoint.
+// Notation: T, S = adjoints of the chunk-end (W, M); a trailing "b" marks an adjoint.  "Wl" is the last matrix
+// [d x h] (W2 of the GELU MLP, W3 of SwiGLU); the first matrices are [h x d].
+//   GELU MLP : hidden a = gelu(z1)                 pz1 = ph gelu'(z1)
+//   SwiGLU   : hidden a = silu(z1) z2              pz1 = ph z2 silu'(z1),  pz2 = ph silu(z1)
 #include "simt_common.cuh"
 #include "simt_layout.h"
 
@@ -14,6 +17,11 @@ namespace e2ttt {
 template <typename Real> struct BwdScalars {
     Real kWb[kMaxC], kMb[kMaxC]; // adjoints of K^W_t, K^M_t
 };
+
+template <typename Real> __device__ __forceinline__ Real silu_d2(Real z) {
+    const Real s = sigmoid_f(z);
+    return s * ((Real)1 - s) * ((Real)2 + z * ((Real)1 - (Real)2 * s));
+}
 
 // out = r ( x - mean(x) - y mean(x*y) ) for one row held by one warp (the LN Jacobian is symmetric)
 template <typename Real>
@@ -26,9 +34,11 @@ __device__ __forceinline__ void warp_ln_jac(const Real* x, const Real* y, Real r
     for (int i = lane; i < d; i += 32) out[i] = r * (x[i] - sx - y[i] * sxy);
 }
 
-template <typename Real, typename IO>
-__global__ void __launch_bounds__(kSimtThreads) simt_bwd_mlp_kernel(const SimtBwdArgs a) {
-    constexpr int NMAT = 2;
+template <typename Real, typename IO, int KIND>
+__global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArgs a) {
+    constexpr int NMAT = (KIND == 0) ? 2 : 3;
+    constexpr int LAST = NMAT - 1;
+    constexpr bool SW = (KIND == 1);
     extern __shared__ __align__(16) unsigned char simt_smem_raw[];
     GemmSmem<Real>& gsm = *reinterpret_cast<GemmSmem<Real>*>(simt_smem_raw);
     ChunkScalars<Real>& sc = *reinterpret_cast<ChunkScalars<Real>*>(simt_smem_raw + sizeof(GemmSmem<Real>));
@@ -70,24 +80,30 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_mlp_kernel(const SimtBw
             S[i][e] = sf ? (Real)sf[e] : (Real)0;
         }
     }
-    Real* Z1 = ws + lay.Z1;   // [2len x h]  pre-activations, key rows then query rows
-    Real* A = ws + lay.A;     // [2len x h]  gelu(Z1)
-    Real* U = ws + lay.U;     // [2len x d]  normalised rows y (after the LN step)
-    Real* Pu = ws + lay.Pu;   // [len x d]
-    Real* Pz = ws + lay.Pz1;  // [len x h]
-    Real* Pa = ws + lay.Pa;   // [len x h]
-    Real* E = ws + lay.E;     // [len x d]
-    Real* XY2 = ws + lay.XY2; // [len x 2d]  (Ak T2^T | Ak S2^T)
-    Real* XY1 = ws + lay.XY1; // [len x 2h]  (K T1^T | K S1^T)
+    Real* Z1 = ws + lay.Z1;    // [2len x h]  pre-activations of matrix 1, key rows then query rows
+    Real* Z2 = ws + lay.Z2;    // [2len x h]  SwiGLU: pre-activations of matrix 2
+    Real* A = ws + lay.A;      // [2len x h]  hidden activation fed to the last matrix
+    Real* U = ws + lay.U;      // [2len x d]  normalised rows y (after the LN step)
+    Real* Pu = ws + lay.Pu;    // [len x d]
+    Real* Pz1 = ws + lay.Pz1;  // [len x h]
+    Real* Pz2 = ws + lay.Pz2;  // [len x h]   SwiGLU
+    Real* Pa = ws + lay.Pa;    // [len x h]   ph = dL/d(hidden activation)
+    Real* E = ws + lay.E;      // [len x d]
+    Real* XY2 = ws + lay.XY2;  // [len x 2d]  (Ak Tl^T | Ak Sl^T)
+    Real* XY1 = ws + lay.XY1;  // [len x 2h]  (K T1^T | K S1^T)
+    Real* XY1b = ws + lay.XY1b;// [len x 2h]  SwiGLU: (K T2^T | K S2^T)
     Real* Pub = ws + lay.Pub;
-    Real* Pzb = ws + lay.Pzb; // becomes Pab in place
-    Real* Zkb = ws + lay.Zkb;
-    Real* Akb = ws + lay.Akb;
+    Real* Pzb = ws + lay.Pzb;  // adjoint of pz1; MLP: becomes the adjoint of ph in place
+    Real* Pzb2 = ws + lay.Pzb2;
+    Real* Zkb = ws + lay.Zkb;  // adjoint of z1 (key rows)
+    Real* Zkb2 = ws + lay.Zkb2;
+    Real* Akb = ws + lay.Akb;  // adjoint of the hidden activation (key rows)
     Real* Kb = ws + lay.Kb;
     Real* Eb = ws + lay.Eb;
     Real* Ukb = ws + lay.Ukb;
     Real* Uqb = ws + lay.Uqb;
     Real* Zqb = ws + lay.Zqb;
+    Real* Zqb2 = ws + lay.Zqb2;
     Real* rk = ws + lay.rk;
     Real* rq = ws + lay.rq;
     __syncthreads();
@@ -100,29 +116,44 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_mlp_kernel(const SimtBw
         const IO* vc = v + (size_t)s * d;
         const IO* doc = d_o + (size_t)s * d;
         const Real* ck = ws + lay.ckpt + (size_t)c * 2 * NMAT * dh;
-        const Real* W1 = ck;               // [h x d]
-        const Real* W2 = ck + dh;          // [d x h]
-        const Real* M1 = ck + 2 * dh;
-        const Real* M2 = ck + 3 * dh;
+        const Real* W1 = ck;                        // [h x d]
+        const Real* W2 = ck + dh;                   // SwiGLU: [h x d]
+        const Real* Wl = ck + (size_t)LAST * dh;    // [d x h]
+        const Real* M0[NMAT];
+#pragma unroll
+        for (int i = 0; i < NMAT; ++i) M0[i] = ck + (size_t)(NMAT + i) * dh;
 
         if (warp == 0) chunk_scalars_warp<Real>(eta + s, beta + s, gamma + s, len, &sc);
-        for (size_t e = tid; e < dh; e += kSimtThreads) { Wb[0][e] = 0; Wb[1][e] = 0; }
+#pragma unroll
+        for (int i = 0; i < NMAT; ++i)
+            for (size_t e = tid; e < dh; e += kSimtThreads) Wb[i][e] = 0;
+
+        auto load_x = [&](int m, int kk, Real& a0, Real& a1) {
+            a0 = (m < len) ? ld_io<Real>(kc, (size_t)m * d + kk) : ld_io<Real>(qc, (size_t)(m - len) * d + kk);
+        };
+        auto load_k = [&](int m, int kk, Real& a0, Real& a1) { a0 = ld_io<Real>(kc, (size_t)m * d + kk); };
 
         // ---------------- forward of the chunk, recomputed ----------------
         block_gemm<Real, 1, true, true>(
-            2 * len, h, d,
-            [&](int m, int kk, Real& a0, Real& a1) {
-                a0 = (m < len) ? ld_io<Real>(kc, (size_t)m * d + kk) : ld_io<Real>(qc, (size_t)(m - len) * d + kk);
-            },
-            [&](int n, int kk) { return W1[(size_t)n * d + kk]; },
+            2 * len, h, d, load_x, [&](int n, int kk) { return W1[(size_t)n * d + kk]; },
             [&](int m, int n, Real acc, Real) {
                 Z1[(size_t)m * h + n] = acc;
-                A[(size_t)m * h + n] = gelu_f(acc);
+                if (!SW) A[(size_t)m * h + n] = gelu_f(acc);
             },
             &gsm);
+        if (SW) {
+            block_gemm<Real, 1, true, true>(
+                2 * len, h, d, load_x, [&](int n, int kk) { return W2[(size_t)n * d + kk]; },
+                [&](int m, int n, Real acc, Real) {
+                    const size_t e = (size_t)m * h + n;
+                    Z2[e] = acc;
+                    A[e] = silu_f(Z1[e]) * acc;
+                },
+                &gsm);
+        }
         block_gemm<Real, 1, true, true>(
             2 * len, d, h, [&](int m, int kk, Real& a0, Real& a1) { a0 = A[(size_t)m * h + kk]; },
-            [&](int n, int kk) { return W2[(size_t)n * h + kk]; },
+            [&](int n, int kk) { return Wl[(size_t)n * h + kk]; },
             [&](int m, int n, Real acc, Real) { U[(size_t)m * d + n] = acc; }, &gsm);
         for (int m = warp; m < 2 * len; m += NW) {
             Real* u = U + (size_t)m * d;
@@ -152,111 +183,167 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_mlp_kernel(const SimtBw
         __syncthreads();
         block_gemm<Real, 1, true, false>(
             len, h, d, [&](int m, int kk, Real& a0, Real& a1) { a0 = Pu[(size_t)m * d + kk]; },
-            [&](int n, int kk) { return W2[(size_t)kk * h + n]; },
+            [&](int n, int kk) { return Wl[(size_t)kk * h + n]; },
             [&](int m, int n, Real acc, Real) {
                 const size_t e = (size_t)m * h + n;
                 Pa[e] = acc;
-                Pz[e] = acc * gelu_d1(Z1[e]);
+                if (!SW) {
+                    Pz1[e] = acc * gelu_d1(Z1[e]);
+                } else {
+                    Pz1[e] = acc * Z2[e] * silu_d1(Z1[e]);
+                    Pz2[e] = acc * silu_f(Z1[e]);
+                }
             },
             &gsm);
 
-        // ---------------- (i) outputs o = q + LN(W2 gelu(W1 q)) ----------------
-        const Real* Zq = Z1 + (size_t)len * h;
+        // ---------------- (i) outputs o = q + LN(Wl a(q)) ----------------
+        const Real* Z1q = Z1 + (size_t)len * h;
+        const Real* Z2q = Z2 + (size_t)len * h;
         const Real* Aq = A + (size_t)len * h;
         block_gemm<Real, 1, true, false>(
             len, h, d, [&](int m, int kk, Real& a0, Real& a1) { a0 = Uqb[(size_t)m * d + kk]; },
-            [&](int n, int kk) { return W2[(size_t)kk * h + n]; },
-            [&](int m, int n, Real acc, Real) { Zqb[(size_t)m * h + n] = acc * gelu_d1(Zq[(size_t)m * h + n]); }, &gsm);
+            [&](int n, int kk) { return Wl[(size_t)kk * h + n]; },
+            [&](int m, int n, Real acc, Real) {
+                const size_t e = (size_t)m * h + n;
+                if (!SW) {
+                    Zqb[e] = acc * gelu_d1(Z1q[e]);
+                } else {
+                    Zqb[e] = acc * Z2q[e] * silu_d1(Z1q[e]);
+                    Zqb2[e] = acc * silu_f(Z1q[e]);
+                }
+            },
+            &gsm);
         block_gemm<Real, 1, true, false>(
-            len, d, h, [&](int m, int kk, Real& a0, Real& a1) { a0 = Zqb[(size_t)m * h + kk]; },
-            [&](int n, int kk) { return W1[(size_t)kk * d + n]; },
+            len, d, SW ? 2 * h : h,
+            [&](int m, int kk, Real& a0, Real& a1) {
+                a0 = kk < h ? Zqb[(size_t)m * h + kk] : Zqb2[(size_t)m * h + kk - h];
+            },
+            [&](int n, int kk) { return kk < h ? W1[(size_t)kk * d + n] : W2[(size_t)(kk - h) * d + n]; },
             [&](int m, int n, Real acc, Real) {
                 const size_t e = (size_t)m * d + n;
                 st_io(dq + (size_t)s * d, e, ld_io<Real>(doc, e) + acc);
             },
             &gsm);
-        block_gemm<Real, 1, false, false>( // Wb2 += Uqb^T Aq
+        block_gemm<Real, 1, false, false>( // Wbl += Uqb^T Aq
             d, h, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Uqb[(size_t)t * d + m]; },
             [&](int n, int t) { return Aq[(size_t)t * h + n]; },
-            [&](int m, int n, Real acc, Real) { Wb[1][(size_t)m * h + n] += acc; }, &gsm);
+            [&](int m, int n, Real acc, Real) { Wb[LAST][(size_t)m * h + n] += acc; }, &gsm);
         block_gemm<Real, 1, false, false>( // Wb1 += Zqb^T Q
             h, d, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Zqb[(size_t)t * h + m]; },
             [&](int n, int t) { return ld_io<Real>(qc, (size_t)t * d + n); },
             [&](int m, int n, Real acc, Real) { Wb[0][(size_t)m * d + n] += acc; }, &gsm);
+        if (SW)
+            block_gemm<Real, 1, false, false>( // Wb2 += Zqb2^T Q
+                h, d, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Zqb2[(size_t)t * h + m]; },
+                [&](int n, int t) { return ld_io<Real>(qc, (size_t)t * d + n); },
+                [&](int m, int n, Real acc, Real) { Wb[1][(size_t)m * d + n] += acc; }, &gsm);
 
         // ---------------- (ii) state transition: carries ----------------
         Real cwb, cmb, cbb;
         {
             Real pw = 0, pm = 0, pb = 0;
-            for (size_t e = tid; e < dh; e += kSimtThreads) {
-                pw += T[0][e] * W1[e] + T[1][e] * W2[e];
-                pm += T[0][e] * M1[e] + T[1][e] * M2[e];
-                pb += S[0][e] * M1[e] + S[1][e] * M2[e];
+#pragma unroll
+            for (int i = 0; i < NMAT; ++i) {
+                const Real* Wi = ck + (size_t)i * dh;
+                for (size_t e = tid; e < dh; e += kSimtThreads) {
+                    pw += T[i][e] * Wi[e];
+                    pm += T[i][e] * M0[i][e];
+                    pb += S[i][e] * M0[i][e];
+                }
             }
             cwb = block_sum(pw, red);
             cmb = block_sum(pm, red);
             cbb = block_sum(pb, red);
         }
         // G_t enters W_C with K^W_t and M_C with K^M_t: its adjoint is K^W_t T + K^M_t S.
-        block_gemm<Real, 1, true, true>( // XY2 = Ak [T2; S2]^T
+        block_gemm<Real, 1, true, true>( // XY2 = Ak [Tl; Sl]^T
             len, 2 * d, h, [&](int m, int kk, Real& a0, Real& a1) { a0 = A[(size_t)m * h + kk]; },
-            [&](int n, int kk) { return n < d ? T[1][(size_t)n * h + kk] : S[1][(size_t)(n - d) * h + kk]; },
+            [&](int n, int kk) { return n < d ? T[LAST][(size_t)n * h + kk] : S[LAST][(size_t)(n - d) * h + kk]; },
             [&](int m, int n, Real acc, Real) { XY2[(size_t)m * 2 * d + n] = acc; }, &gsm);
         block_gemm<Real, 1, true, true>( // XY1 = K [T1; S1]^T
-            len, 2 * h, d, [&](int m, int kk, Real& a0, Real& a1) { a0 = ld_io<Real>(kc, (size_t)m * d + kk); },
+            len, 2 * h, d, load_k,
             [&](int n, int kk) { return n < h ? T[0][(size_t)n * d + kk] : S[0][(size_t)(n - h) * d + kk]; },
             [&](int m, int n, Real acc, Real) { XY1[(size_t)m * 2 * h + n] = acc; }, &gsm);
+        if (SW)
+            block_gemm<Real, 1, true, true>( // XY1b = K [T2; S2]^T
+                len, 2 * h, d, load_k,
+                [&](int n, int kk) { return n < h ? T[1][(size_t)n * d + kk] : S[1][(size_t)(n - h) * d + kk]; },
+                [&](int m, int n, Real acc, Real) { XY1b[(size_t)m * 2 * h + n] = acc; }, &gsm);
         for (int t = warp; t < len; t += NW) {
             const Real* x2 = XY2 + (size_t)t * 2 * d;
             const Real* x1 = XY1 + (size_t)t * 2 * h;
+            const Real* x1b = XY1b + (size_t)t * 2 * h;
             Real sw = 0, sm = 0;
             for (int i = lane; i < d; i += 32) {
                 const Real p = Pu[(size_t)t * d + i];
                 sw += p * x2[i]; sm += p * x2[d + i];
             }
             for (int j = lane; j < h; j += 32) {
-                const Real p = Pz[(size_t)t * h + j];
+                const Real p = Pz1[(size_t)t * h + j];
                 sw += p * x1[j]; sm += p * x1[h + j];
+                if (SW) {
+                    const Real p2 = Pz2[(size_t)t * h + j];
+                    sw += p2 * x1b[j]; sm += p2 * x1b[h + j];
+                }
             }
             sw = warp_sum(sw); sm = warp_sum(sm);
             if (lane == 0) { bs.kWb[t] = -sw; bs.kMb[t] = -sm; }
             const Real kw = sc.kW[t], km = sc.kM[t];
             for (int i = lane; i < d; i += 32) Pub[(size_t)t * d + i] = -(kw * x2[i] + km * x2[d + i]);
-            for (int j = lane; j < h; j += 32) Pzb[(size_t)t * h + j] = -(kw * x1[j] + km * x1[h + j]);
+            for (int j = lane; j < h; j += 32) {
+                Pzb[(size_t)t * h + j] = -(kw * x1[j] + km * x1[h + j]);
+                if (SW) Pzb2[(size_t)t * h + j] = -(kw * x1b[j] + km * x1b[h + j]);
+            }
         }
         __syncthreads();
-        // ---------------- (iii) per-token gradients G_t = -(pz k^T, pu a^T) ----------------
-        block_gemm<Real, 1, true, false>( // Akb = -[kW Pu | kM Pu] [T2; S2]
+        // ---------------- (iii) per-token gradients G_t = -(pz1 k^T, [pz2 k^T,] pu a^T) ----------------
+        block_gemm<Real, 1, true, false>( // Akb = -[kW Pu | kM Pu] [Tl; Sl]
             len, h, 2 * d,
             [&](int m, int kk, Real& a0, Real& a1) {
                 a0 = kk < d ? sc.kW[m] * Pu[(size_t)m * d + kk] : sc.kM[m] * Pu[(size_t)m * d + kk - d];
             },
-            [&](int n, int kk) { return kk < d ? T[1][(size_t)kk * h + n] : S[1][(size_t)(kk - d) * h + n]; },
+            [&](int n, int kk) { return kk < d ? T[LAST][(size_t)kk * h + n] : S[LAST][(size_t)(kk - d) * h + n]; },
             [&](int m, int n, Real acc, Real) { Akb[(size_t)m * h + n] = -acc; }, &gsm);
-        block_gemm<Real, 1, true, false>( // Kb = -[kW Pz | kM Pz] [T1; S1]
+        block_gemm<Real, 1, true, false>( // Kb = -[kW Pz1 | kM Pz1] [T1; S1]
             len, d, 2 * h,
             [&](int m, int kk, Real& a0, Real& a1) {
-                a0 = kk < h ? sc.kW[m] * Pz[(size_t)m * h + kk] : sc.kM[m] * Pz[(size_t)m * h + kk - h];
+                a0 = kk < h ? sc.kW[m] * Pz1[(size_t)m * h + kk] : sc.kM[m] * Pz1[(size_t)m * h + kk - h];
             },
             [&](int n, int kk) { return kk < h ? T[0][(size_t)kk * d + n] : S[0][(size_t)(kk - h) * d + n]; },
             [&](int m, int n, Real acc, Real) { Kb[(size_t)m * d + n] = -acc; }, &gsm);
-        // pz = pa * gelu'(z)
+        if (SW)
+            block_gemm<Real, 1, true, false>( // Kb -= [kW Pz2 | kM Pz2] [T2; S2]
+                len, d, 2 * h,
+                [&](int m, int kk, Real& a0, Real& a1) {
+                    a0 = kk < h ? sc.kW[m] * Pz2[(size_t)m * h + kk] : sc.kM[m] * Pz2[(size_t)m * h + kk - h];
+                },
+                [&](int n, int kk) { return kk < h ? T[1][(size_t)kk * d + n] : S[1][(size_t)(kk - h) * d + n]; },
+                [&](int m, int n, Real acc, Real) { Kb[(size_t)m * d + n] -= acc; }, &gsm);
+        // back through pz: Pzb becomes the adjoint of ph; Zkb (Zkb2) start with the second-order terms
         for (size_t e = tid; e < (size_t)len * h; e += kSimtThreads) {
-            const Real pzb = Pzb[e], z = Z1[e];
-            Zkb[e] = pzb * Pa[e] * gelu_d2(z);
-            Pzb[e] = pzb * gelu_d1(z); // now Pab
+            const Real z1 = Z1[e], ph = Pa[e];
+            if (!SW) {
+                const Real pzb = Pzb[e];
+                Zkb[e] = pzb * ph * gelu_d2(z1);
+                Pzb[e] = pzb * gelu_d1(z1);
+            } else {
+                const Real b1 = Pzb[e], b2 = Pzb2[e], z2 = Z2[e], g1 = silu_d1(z1);
+                Pzb[e] = b1 * z2 * g1 + b2 * silu_f(z1);
+                Zkb2[e] = b1 * ph * g1;
+                Zkb[e] = b1 * ph * z2 * silu_d2(z1) + b2 * ph * g1;
+            }
         }
         __syncthreads();
-        const Real* Pab = Pzb;
-        // pa = W2^T pu
+        const Real* Phb = Pzb;
+        // ph = Wl^T pu
         block_gemm<Real, 1, true, true>(
-            len, d, h, [&](int m, int kk, Real& a0, Real& a1) { a0 = Pab[(size_t)m * h + kk]; },
-            [&](int n, int kk) { return W2[(size_t)n * h + kk]; },
+            len, d, h, [&](int m, int kk, Real& a0, Real& a1) { a0 = Phb[(size_t)m * h + kk]; },
+            [&](int n, int kk) { return Wl[(size_t)n * h + kk]; },
             [&](int m, int n, Real acc, Real) { Pub[(size_t)m * d + n] += acc; }, &gsm);
-        block_gemm<Real, 1, false, false>( // Wb2 += Pu^T Pab
+        block_gemm<Real, 1, false, false>( // Wbl += Pu^T Phb
             d, h, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Pu[(size_t)t * d + m]; },
-            [&](int n, int t) { return Pab[(size_t)t * h + n]; },
-            [&](int m, int n, Real acc, Real) { Wb[1][(size_t)m * h + n] += acc; }, &gsm);
+            [&](int n, int t) { return Phb[(size_t)t * h + n]; },
+            [&](int m, int n, Real acc, Real) { Wb[LAST][(size_t)m * h + n] += acc; }, &gsm);
         // pu = J(u) e, e = k + y - v, y = LN(u)
         for (int t = warp; t < len; t += NW) {
             const size_t row = (size_t)t * d;
@@ -283,23 +370,32 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_mlp_kernel(const SimtBw
             }
         }
         __syncthreads();
-        // u = W2 a, a = gelu(z)
+        // u = Wl a ; a = gelu(z1)  or  silu(z1) z2
         block_gemm<Real, 1, true, false>(
             len, h, d, [&](int m, int kk, Real& a0, Real& a1) { a0 = Ukb[(size_t)m * d + kk]; },
-            [&](int n, int kk) { return W2[(size_t)kk * h + n]; },
+            [&](int n, int kk) { return Wl[(size_t)kk * h + n]; },
             [&](int m, int n, Real acc, Real) {
                 const size_t e = (size_t)m * h + n;
-                Zkb[e] += (Akb[e] + acc) * gelu_d1(Z1[e]);
+                const Real ab = Akb[e] + acc;
+                if (!SW) {
+                    Zkb[e] += ab * gelu_d1(Z1[e]);
+                } else {
+                    Zkb[e] += ab * Z2[e] * silu_d1(Z1[e]);
+                    Zkb2[e] += ab * silu_f(Z1[e]);
+                }
             },
             &gsm);
-        block_gemm<Real, 1, false, false>( // Wb2 += Ukb^T Ak
+        block_gemm<Real, 1, false, false>( // Wbl += Ukb^T Ak
             d, h, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Ukb[(size_t)t * d + m]; },
             [&](int n, int t) { return A[(size_t)t * h + n]; },
-            [&](int m, int n, Real acc, Real) { Wb[1][(size_t)m * h + n] += acc; }, &gsm);
-        // z = W1 k
+            [&](int m, int n, Real acc, Real) { Wb[LAST][(size_t)m * h + n] += acc; }, &gsm);
+        // z1 = W1 k (, z2 = W2 k)
         block_gemm<Real, 1, true, false>(
-            len, d, h, [&](int m, int kk, Real& a0, Real& a1) { a0 = Zkb[(size_t)m * h + kk]; },
-            [&](int n, int kk) { return W1[(size_t)kk * d + n]; },
+            len, d, SW ? 2 * h : h,
+            [&](int m, int kk, Real& a0, Real& a1) {
+                a0 = kk < h ? Zkb[(size_t)m * h + kk] : Zkb2[(size_t)m * h + kk - h];
+            },
+            [&](int n, int kk) { return kk < h ? W1[(size_t)kk * d + n] : W2[(size_t)(kk - h) * d + n]; },
             [&](int m, int n, Real acc, Real) {
                 const size_t e = (size_t)m * d + n;
                 st_io(dk + (size_t)s * d, e, Kb[e] + acc);
@@ -309,6 +405,11 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_mlp_kernel(const SimtBw
             h, d, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Zkb[(size_t)t * h + m]; },
             [&](int n, int t) { return ld_io<Real>(kc, (size_t)t * d + n); },
             [&](int m, int n, Real acc, Real) { Wb[0][(size_t)m * d + n] += acc; }, &gsm);
+        if (SW)
+            block_gemm<Real, 1, false, false>( // Wb2 += Zkb2^T K
+                h, d, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Zkb2[(size_t)t * h + m]; },
+                [&](int n, int t) { return ld_io<Real>(kc, (size_t)t * d + n); },
+                [&](int m, int n, Real acc, Real) { Wb[1][(size_t)m * d + n] += acc; }, &gsm);
 
         // ---------------- adjoints of the chunk-start state ----------------
         {
@@ -362,7 +463,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_mlp_kernel(const SimtBw
     }
 }
 
-template <typename Real, typename IO>
+template <typename Real, typename IO, int KIND>
 static int launch_bwd(const SimtBwdArgs& a, cudaStream_t st) {
     constexpr size_t smem =
         sizeof(GemmSmem<Real>) + sizeof(ChunkScalars<Real>) + sizeof(BwdScalars<Real>) + 8 * sizeof(Real);
@@ -370,18 +471,20 @@ static int launch_bwd(const SimtBwdArgs& a, cudaStream_t st) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return (int)cudaGetLastError();
     if (dev < 0 || dev >= 64 || !attr_done[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(simt_bwd_mlp_kernel<Real, IO>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e =
+            cudaFuncSetAttribute(simt_bwd_kernel<Real, IO, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return (int)e;
         if (dev >= 0 && dev < 64) attr_done[dev] = true;
     }
-    simt_bwd_mlp_kernel<Real, IO><<<dim3(a.N), dim3(kSimtThreads), smem, st>>>(a);
+    simt_bwd_kernel<Real, IO, KIND><<<dim3(a.N), dim3(kSimtThreads), smem, st>>>(a);
     return (int)cudaGetLastError();
 }
 
 int simt_bwd_launch(const SimtBwdArgs& a, int kind, int io_dtype, void* stream) {
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    if (kind != 0) return (int)cudaErrorInvalidValue;
-    return io_dtype == 0 ? launch_bwd<double, float>(a, st) : launch_bwd<float, __nv_bfloat16>(a, st);
+    if (io_dtype == 0)
+        return kind == 0 ? launch_bwd<double, float, 0>(a, st) : launch_bwd<double, float, 1>(a, st);
+    return kind == 0 ? launch_bwd<float, __nv_bfloat16, 0>(a, st) : launch_bwd<float, __nv_bfloat16, 1>(a, st);
 }
 
 }  // namespace e2ttt

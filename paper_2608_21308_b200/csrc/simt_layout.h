@@ -15,6 +15,7 @@ struct SimtLayout {
     size_t T[3], S[3];   // adjoints of the chunk-end state (W, M)
     size_t Wb[3];        // adjoint accumulators of the chunk-start weights
     size_t Pa, E, XY2, XY1, Pub, Pzb, Zkb, Akb, Kb, Eb, Ukb, Uqb, Zqb;
+    size_t XY1b, Pzb2, Zkb2, Zqb2;  // SwiGLU only: the second [h x d] matrix
     size_t rk, rq, red;  // per-row 1/std of the two LN calls; small reduction scratch
     size_t ckpt;         // [nchunks][2][nmat][d*h] chunk-start (W, M), present when states are saved
     size_t per_seq;      // elements per sequence
@@ -38,6 +39,8 @@ inline SimtLayout simt_layout(int d, int h, int C, int nmat, int nchunks, bool s
         l.Pub = take((size_t)C * d); l.Pzb = take((size_t)C * h); l.Zkb = take((size_t)C * h);
         l.Akb = take((size_t)C * h); l.Kb = take((size_t)C * d); l.Eb = take((size_t)C * d);
         l.Ukb = take((size_t)C * d); l.Uqb = take((size_t)C * d); l.Zqb = take((size_t)C * h);
+        const size_t sw = (nmat == 3) ? 1 : 0;
+        l.XY1b = take(sw * C * 2 * h); l.Pzb2 = take(sw * C * h); l.Zkb2 = take(sw * C * h); l.Zqb2 = take(sw * C * h);
         l.rk = take(C); l.rq = take(C); l.red = take(64);
     }
     l.ckpt = take(save_states ? (size_t)nchunks * 2 * nmat * dh : 0);

@@ -74,13 +74,22 @@ def test_forward_odd_shapes_fp32(kind, d, h, C, L, N):
     check_forward(got, ref, TOL_F32, f"kind {kind} d{d} h{h} C{C} L{L}")
 
 
+@pytest.mark.parametrize("kind", [MLP, SWIGLU])
 @pytest.mark.parametrize("d,h,C,L,N", [(48, 80, 24, 60, 2), (8, 16, 1, 4, 1), (64, 160, 32, 64, 1)])
-def test_backward_odd_shapes_fp32(d, h, C, L, N):
-    r = inputs.Recipe(B=N, H=1, L=L, d=d, h=h, C=C, kind=MLP, seed=6, m_std=0.01)
+def test_backward_odd_shapes_fp32(kind, d, h, C, L, N):
+    r = inputs.Recipe(B=N, H=1, L=L, d=d, h=h, C=C, kind=kind, seed=6, m_std=0.01)
     x = inputs.generate(r, with_d_o=True, with_dstate=True)
-    ref = util.oracle_backward(x, C, MLP)
-    got = util.gpu_backward(x, d=d, h=h, C=C, kind=MLP, io="f32")
-    check_backward(got, ref, TOL_F32, f"bwd d{d} h{h} C{C} L{L}")
+    ref = util.oracle_backward(x, C, kind)
+    got = util.gpu_backward(x, d=d, h=h, C=C, kind=kind, io="f32")
+    check_backward(got, ref, TOL_F32, f"bwd kind {kind} d{d} h{h} C{C} L{L}")
+
+
+def test_backward_swiglu_config3_windows_bf16():
+    r = inputs.config(3, heads=[5])
+    xw, _ = util.teacher_forced_windows(r, 3, window=1, with_grads=True)
+    ref = util.oracle_backward(xw, r.C, r.kind)
+    got = util.gpu_backward(xw, d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16")
+    check_backward(got, ref, TOL_BF16, "config 3 (SwiGLU) bwd windows")
 
 
 def test_optional_inputs_null_momentum_and_null_state_adjoints():
