@@ -600,10 +600,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             for (int k = 0; k < 4; ++k)
                 umma_bf16(tb + T_R0, desc_mn(smem_u32(s.PzM[0]), 8192, k), desc_mn(smem_u32(s.X[0]), 16384, k), id_agg, k > 0);
             umma_commit(&s.bar_agg);
+            PROF(14);
 #pragma unroll
             for (int k = 0; k < 4; ++k)
                 umma_bf16(tb + T_R1, desc_mn(smem_u32(s.Pu[0]), 8192, k), desc_mn(smem_u32(s.AkM[0]), 8192, k), id_agg, k > 0);
             umma_commit(&s.bar_agg2);
+            PROF(15);
         }
         const bool last = (r + 1 == nchunks);
         const float cm = sc.cm, cb = sc.cb;

@@ -60,3 +60,27 @@ def test_tc_null_momentum_determinism_and_many_sequences():
     first = {n: (np.ascontiguousarray(v[:, :64]) if not isinstance(v, list) else v) for n, v in x.items()}
     ref = util.oracle_forward(first, 64, MLP, use_M=False)
     assert util.rel_err(a["o"][:, :64], ref["o"]) <= TOL_BF16
+
+
+def test_tc_full_benchmark_size_properties_and_sampled_outputs():
+    """The launch configuration bench.py times (B=4, H=16, L=4096): device status, split invariance (bitwise),
+    and the first chunk of sampled sequences against the oracle (later chunks are covered by the windows)."""
+    r = inputs.config(2)
+    x = inputs.generate(r)
+    whole, hd = util.gpu_forward(x, impl=E.E2TTT_IMPL_TCGEN05, use_M=False, **SHAPE)
+    assert E.e2ttt_device_status(hd["ws"]) == 0
+    assert np.isfinite(whole["o"]).all() and all(np.isfinite(w).all() for w in whole["W"] + whole["M"])
+    half = r.L // 2
+    first = {n: (np.ascontiguousarray(v[:, :half]) if not isinstance(v, list) else v) for n, v in x.items()}
+    a, _ = util.gpu_forward(first, impl=E.E2TTT_IMPL_TCGEN05, use_M=False, **SHAPE)
+    rest = {n: (np.ascontiguousarray(v[:, half:]) if not isinstance(v, list) else v) for n, v in x.items()}
+    rest["W"], rest["M"] = a["W"], a["M"]
+    b, _ = util.gpu_forward(rest, impl=E.E2TTT_IMPL_TCGEN05, **SHAPE)
+    assert np.array_equal(np.concatenate([a["o"], b["o"]], 1), whole["o"])
+    for i in range(2):
+        assert np.array_equal(b["W"][i], whole["W"][i]) and np.array_equal(b["M"][i], whole["M"][i])
+    heads = [0, 17, 42, 63]
+    sample = {n: (np.ascontiguousarray(v[heads, :64]) if not isinstance(v, list) else [m[heads] for m in v])
+              for n, v in x.items()}
+    ref = util.oracle_forward(sample, 64, MLP, use_M=False)
+    assert util.rel_err(whole["o"][heads, :64], ref["o"]) <= TOL_BF16
