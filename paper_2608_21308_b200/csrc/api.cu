@@ -147,6 +147,7 @@ int e2ttt_chunk_fwd(const e2ttt_params* p, const void* q, const void* k, const v
     SimtFwdArgs a{};
     a.N = p->B * p->H; a.L = p->L; a.d = p->d; a.h = p->h; a.C = p->C;
     a.nchunks = (p->L + p->C - 1) / p->C;
+    a.cl = simt_cluster_size(a.N);
     a.save_states = save_states != 0;
     a.eps = p->ln_eps;
     a.q = q; a.k = k; a.v = v; a.eta = eta; a.beta = beta; a.gamma = gamma; a.o = o;
@@ -204,7 +205,7 @@ int e2ttt_chunk_bwd(const e2ttt_params* p, const void* q, const void* k, const v
         // that the reverse sweep overwrites later (the adjoint carries T, S and the accumulators Wb)
         SimtFwdArgs f{};
         f.N = p->B * p->H; f.L = p->L; f.d = p->d; f.h = p->h; f.C = p->C; f.nchunks = nchunks;
-        f.save_states = 1; f.eps = p->ln_eps;
+        f.save_states = 1; f.eps = p->ln_eps; f.cl = simt_cluster_size(f.N);
         f.q = q; f.k = k; f.v = v; f.eta = eta; f.beta = beta; f.gamma = gamma; f.ws = ws_data; f.lay = lay;
         f.o = nullptr; // outputs are not needed
         for (int i = 0; i < nmat; ++i) {
@@ -217,6 +218,7 @@ int e2ttt_chunk_bwd(const e2ttt_params* p, const void* q, const void* k, const v
     }
     SimtBwdArgs b{};
     b.N = p->B * p->H; b.L = p->L; b.d = p->d; b.h = p->h; b.C = p->C; b.nchunks = nchunks; b.eps = p->ln_eps;
+    b.cl = simt_cluster_size(b.N);
     b.q = q; b.k = k; b.v = v; b.d_o = d_o; b.eta = eta; b.beta = beta; b.gamma = gamma;
     b.dq = dq; b.dk = dk; b.dv = dv; b.d_eta = d_eta; b.d_beta = d_beta; b.d_gamma = d_gamma;
     b.ws = ws_data; b.lay = lay;

@@ -14,10 +14,6 @@
 
 namespace e2ttt {
 
-template <typename Real> struct BwdScalars {
-    Real kWb[kMaxC], kMb[kMaxC]; // adjoints of K^W_t, K^M_t
-};
-
 template <typename Real> __device__ __forceinline__ Real silu_d2(Real z) {
     const Real s = sigmoid_f(z);
     return s * ((Real)1 - s) * ((Real)2 + z * ((Real)1 - (Real)2 * s));
@@ -42,12 +38,10 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
     extern __shared__ __align__(16) unsigned char simt_smem_raw[];
     GemmSmem<Real>& gsm = *reinterpret_cast<GemmSmem<Real>*>(simt_smem_raw);
     ChunkScalars<Real>& sc = *reinterpret_cast<ChunkScalars<Real>*>(simt_smem_raw + sizeof(GemmSmem<Real>));
-    BwdScalars<Real>& bs =
-        *reinterpret_cast<BwdScalars<Real>*>(simt_smem_raw + sizeof(GemmSmem<Real>) + sizeof(ChunkScalars<Real>));
-    Real* red = reinterpret_cast<Real*>(simt_smem_raw + sizeof(GemmSmem<Real>) + sizeof(ChunkScalars<Real>) +
-                                        sizeof(BwdScalars<Real>));
+    Real* red = reinterpret_cast<Real*>(simt_smem_raw + sizeof(GemmSmem<Real>) + sizeof(ChunkScalars<Real>));
 
-    const int seq = blockIdx.x;
+    const int CL = a.cl;                 // CTAs working on this sequence (one cluster)
+    const int seq = blockIdx.x / CL, rank = blockIdx.x % CL;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     constexpr int NW = kSimtThreads / 32;
     const int d = a.d, h = a.h, C = a.C, L = a.L;
@@ -75,7 +69,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
         T[i] = ws + lay.T[i]; S[i] = ws + lay.S[i]; Wb[i] = ws + lay.Wb[i];
         const float* tf = a.dW_final[i] ? a.dW_final[i] + (size_t)seq * dh : nullptr;
         const float* sf = a.dM_final[i] ? a.dM_final[i] + (size_t)seq * dh : nullptr;
-        for (size_t e = tid; e < dh; e += kSimtThreads) {
+        for (size_t e = tid + (size_t)rank * kSimtThreads; e < dh; e += (size_t)kSimtThreads * CL) {
             T[i][e] = tf ? (Real)tf[e] : (Real)0;
             S[i][e] = sf ? (Real)sf[e] : (Real)0;
         }
@@ -106,7 +100,9 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
     Real* Zqb2 = ws + lay.Zqb2;
     Real* rk = ws + lay.rk;
     Real* rq = ws + lay.rq;
-    __syncthreads();
+    Real* kWb_g = ws + lay.kWb;  // adjoints of K^W_t, K^M_t (rows are produced by different CTAs)
+    Real* kMb_g = ws + lay.kMb;
+    phase_sync(CL);
 
     for (int c = a.nchunks - 1; c >= 0; --c) {
         const int s = c * C;
@@ -126,7 +122,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
         if (warp == 0) chunk_scalars_warp<Real>(eta + s, beta + s, gamma + s, len, &sc);
 #pragma unroll
         for (int i = 0; i < NMAT; ++i)
-            for (size_t e = tid; e < dh; e += kSimtThreads) Wb[i][e] = 0;
+            for (size_t e = tid + (size_t)rank * kSimtThreads; e < dh; e += (size_t)kSimtThreads * CL) Wb[i][e] = 0;
 
         auto load_x = [&](int m, int kk, Real& a0, Real& a1) {
             a0 = (m < len) ? ld_io<Real>(kc, (size_t)m * d + kk) : ld_io<Real>(qc, (size_t)(m - len) * d + kk);
@@ -140,7 +136,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
                 Z1[(size_t)m * h + n] = acc;
                 if (!SW) A[(size_t)m * h + n] = gelu_f(acc);
             },
-            &gsm);
+            &gsm, rank, CL);
         if (SW) {
             block_gemm<Real, 1, true, true>(
                 2 * len, h, d, load_x, [&](int n, int kk) { return W2[(size_t)n * d + kk]; },
@@ -149,13 +145,13 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
                     Z2[e] = acc;
                     A[e] = silu_f(Z1[e]) * acc;
                 },
-                &gsm);
+                &gsm, rank, CL);
         }
         block_gemm<Real, 1, true, true>(
             2 * len, d, h, [&](int m, int kk, Real& a0, Real& a1) { a0 = A[(size_t)m * h + kk]; },
             [&](int n, int kk) { return Wl[(size_t)n * h + kk]; },
-            [&](int m, int n, Real acc, Real) { U[(size_t)m * d + n] = acc; }, &gsm);
-        for (int m = warp; m < 2 * len; m += NW) {
+            [&](int m, int n, Real acc, Real) { U[(size_t)m * d + n] = acc; }, &gsm, rank, CL);
+        for (int m = warp + rank * (kSimtThreads / 32); m < 2 * len; m += (kSimtThreads / 32) * CL) {
             Real* u = U + (size_t)m * d;
             const Real r = warp_layernorm(u, u, d, eps);
             if (m >= len) {
@@ -180,7 +176,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
                 warp_ln_jac(E + row, u, r, d, Pu + row);
             }
         }
-        __syncthreads();
+        phase_sync(CL);
         block_gemm<Real, 1, true, false>(
             len, h, d, [&](int m, int kk, Real& a0, Real& a1) { a0 = Pu[(size_t)m * d + kk]; },
             [&](int n, int kk) { return Wl[(size_t)kk * h + n]; },
@@ -194,7 +190,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
                     Pz2[e] = acc * silu_f(Z1[e]);
                 }
             },
-            &gsm);
+            &gsm, rank, CL);
 
         // ---------------- (i) outputs o = q + LN(Wl a(q)) ----------------
         const Real* Z1q = Z1 + (size_t)len * h;
@@ -212,7 +208,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
                     Zqb2[e] = acc * silu_f(Z1q[e]);
                 }
             },
-            &gsm);
+            &gsm, rank, CL);
         block_gemm<Real, 1, true, false>(
             len, d, SW ? 2 * h : h,
             [&](int m, int kk, Real& a0, Real& a1) {
@@ -223,20 +219,20 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
                 const size_t e = (size_t)m * d + n;
                 st_io(dq + (size_t)s * d, e, ld_io<Real>(doc, e) + acc);
             },
-            &gsm);
+            &gsm, rank, CL);
         block_gemm<Real, 1, false, false>( // Wbl += Uqb^T Aq
             d, h, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Uqb[(size_t)t * d + m]; },
             [&](int n, int t) { return Aq[(size_t)t * h + n]; },
-            [&](int m, int n, Real acc, Real) { Wb[LAST][(size_t)m * h + n] += acc; }, &gsm);
+            [&](int m, int n, Real acc, Real) { Wb[LAST][(size_t)m * h + n] += acc; }, &gsm, rank, CL);
         block_gemm<Real, 1, false, false>( // Wb1 += Zqb^T Q
             h, d, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Zqb[(size_t)t * h + m]; },
             [&](int n, int t) { return ld_io<Real>(qc, (size_t)t * d + n); },
-            [&](int m, int n, Real acc, Real) { Wb[0][(size_t)m * d + n] += acc; }, &gsm);
+            [&](int m, int n, Real acc, Real) { Wb[0][(size_t)m * d + n] += acc; }, &gsm, rank, CL);
         if (SW)
             block_gemm<Real, 1, false, false>( // Wb2 += Zqb2^T Q
                 h, d, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Zqb2[(size_t)t * h + m]; },
                 [&](int n, int t) { return ld_io<Real>(qc, (size_t)t * d + n); },
-                [&](int m, int n, Real acc, Real) { Wb[1][(size_t)m * d + n] += acc; }, &gsm);
+                [&](int m, int n, Real acc, Real) { Wb[1][(size_t)m * d + n] += acc; }, &gsm, rank, CL);
 
         // ---------------- (ii) state transition: carries ----------------
         Real cwb, cmb, cbb;
@@ -245,7 +241,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
 #pragma unroll
             for (int i = 0; i < NMAT; ++i) {
                 const Real* Wi = ck + (size_t)i * dh;
-                for (size_t e = tid; e < dh; e += kSimtThreads) {
+                for (size_t e = tid; e < dh; e += kSimtThreads) {  // every CTA sums everything: same value everywhere
                     pw += T[i][e] * Wi[e];
                     pm += T[i][e] * M0[i][e];
                     pb += S[i][e] * M0[i][e];
@@ -259,17 +255,17 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
         block_gemm<Real, 1, true, true>( // XY2 = Ak [Tl; Sl]^T
             len, 2 * d, h, [&](int m, int kk, Real& a0, Real& a1) { a0 = A[(size_t)m * h + kk]; },
             [&](int n, int kk) { return n < d ? T[LAST][(size_t)n * h + kk] : S[LAST][(size_t)(n - d) * h + kk]; },
-            [&](int m, int n, Real acc, Real) { XY2[(size_t)m * 2 * d + n] = acc; }, &gsm);
+            [&](int m, int n, Real acc, Real) { XY2[(size_t)m * 2 * d + n] = acc; }, &gsm, rank, CL);
         block_gemm<Real, 1, true, true>( // XY1 = K [T1; S1]^T
             len, 2 * h, d, load_k,
             [&](int n, int kk) { return n < h ? T[0][(size_t)n * d + kk] : S[0][(size_t)(n - h) * d + kk]; },
-            [&](int m, int n, Real acc, Real) { XY1[(size_t)m * 2 * h + n] = acc; }, &gsm);
+            [&](int m, int n, Real acc, Real) { XY1[(size_t)m * 2 * h + n] = acc; }, &gsm, rank, CL);
         if (SW)
             block_gemm<Real, 1, true, true>( // XY1b = K [T2; S2]^T
                 len, 2 * h, d, load_k,
                 [&](int n, int kk) { return n < h ? T[1][(size_t)n * d + kk] : S[1][(size_t)(n - h) * d + kk]; },
-                [&](int m, int n, Real acc, Real) { XY1b[(size_t)m * 2 * h + n] = acc; }, &gsm);
-        for (int t = warp; t < len; t += NW) {
+                [&](int m, int n, Real acc, Real) { XY1b[(size_t)m * 2 * h + n] = acc; }, &gsm, rank, CL);
+        for (int t = warp + rank * (kSimtThreads / 32); t < len; t += (kSimtThreads / 32) * CL) {
             const Real* x2 = XY2 + (size_t)t * 2 * d;
             const Real* x1 = XY1 + (size_t)t * 2 * h;
             const Real* x1b = XY1b + (size_t)t * 2 * h;
@@ -287,7 +283,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
                 }
             }
             sw = warp_sum(sw); sm = warp_sum(sm);
-            if (lane == 0) { bs.kWb[t] = -sw; bs.kMb[t] = -sm; }
+            if (lane == 0) { kWb_g[t] = -sw; kMb_g[t] = -sm; }
             const Real kw = sc.kW[t], km = sc.kM[t];
             for (int i = lane; i < d; i += 32) Pub[(size_t)t * d + i] = -(kw * x2[i] + km * x2[d + i]);
             for (int j = lane; j < h; j += 32) {
@@ -295,7 +291,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
                 if (SW) Pzb2[(size_t)t * h + j] = -(kw * x1b[j] + km * x1b[h + j]);
             }
         }
-        __syncthreads();
+        phase_sync(CL);
         // ---------------- (iii) per-token gradients G_t = -(pz1 k^T, [pz2 k^T,] pu a^T) ----------------
         block_gemm<Real, 1, true, false>( // Akb = -[kW Pu | kM Pu] [Tl; Sl]
             len, h, 2 * d,
@@ -303,14 +299,14 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
                 a0 = kk < d ? sc.kW[m] * Pu[(size_t)m * d + kk] : sc.kM[m] * Pu[(size_t)m * d + kk - d];
             },
             [&](int n, int kk) { return kk < d ? T[LAST][(size_t)kk * h + n] : S[LAST][(size_t)(kk - d) * h + n]; },
-            [&](int m, int n, Real acc, Real) { Akb[(size_t)m * h + n] = -acc; }, &gsm);
+            [&](int m, int n, Real acc, Real) { Akb[(size_t)m * h + n] = -acc; }, &gsm, rank, CL);
         block_gemm<Real, 1, true, false>( // Kb = -[kW Pz1 | kM Pz1] [T1; S1]
             len, d, 2 * h,
             [&](int m, int kk, Real& a0, Real& a1) {
                 a0 = kk < h ? sc.kW[m] * Pz1[(size_t)m * h + kk] : sc.kM[m] * Pz1[(size_t)m * h + kk - h];
             },
             [&](int n, int kk) { return kk < h ? T[0][(size_t)kk * d + n] : S[0][(size_t)(kk - h) * d + n]; },
-            [&](int m, int n, Real acc, Real) { Kb[(size_t)m * d + n] = -acc; }, &gsm);
+            [&](int m, int n, Real acc, Real) { Kb[(size_t)m * d + n] = -acc; }, &gsm, rank, CL);
         if (SW)
             block_gemm<Real, 1, true, false>( // Kb -= [kW Pz2 | kM Pz2] [T2; S2]
                 len, d, 2 * h,
@@ -318,9 +314,9 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
                     a0 = kk < h ? sc.kW[m] * Pz2[(size_t)m * h + kk] : sc.kM[m] * Pz2[(size_t)m * h + kk - h];
                 },
                 [&](int n, int kk) { return kk < h ? T[1][(size_t)kk * d + n] : S[1][(size_t)(kk - h) * d + n]; },
-                [&](int m, int n, Real acc, Real) { Kb[(size_t)m * d + n] -= acc; }, &gsm);
+                [&](int m, int n, Real acc, Real) { Kb[(size_t)m * d + n] -= acc; }, &gsm, rank, CL);
         // back through pz: Pzb becomes the adjoint of ph; Zkb (Zkb2) start with the second-order terms
-        for (size_t e = tid; e < (size_t)len * h; e += kSimtThreads) {
+        for (size_t e = tid + (size_t)rank * kSimtThreads; e < (size_t)len * h; e += (size_t)kSimtThreads * CL) {
             const Real z1 = Z1[e], ph = Pa[e];
             if (!SW) {
                 const Real pzb = Pzb[e];
@@ -333,19 +329,19 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
                 Zkb[e] = b1 * ph * z2 * silu_d2(z1) + b2 * ph * g1;
             }
         }
-        __syncthreads();
+        phase_sync(CL);
         const Real* Phb = Pzb;
         // ph = Wl^T pu
         block_gemm<Real, 1, true, true>(
             len, d, h, [&](int m, int kk, Real& a0, Real& a1) { a0 = Phb[(size_t)m * h + kk]; },
             [&](int n, int kk) { return Wl[(size_t)n * h + kk]; },
-            [&](int m, int n, Real acc, Real) { Pub[(size_t)m * d + n] += acc; }, &gsm);
+            [&](int m, int n, Real acc, Real) { Pub[(size_t)m * d + n] += acc; }, &gsm, rank, CL);
         block_gemm<Real, 1, false, false>( // Wbl += Pu^T Phb
             d, h, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Pu[(size_t)t * d + m]; },
             [&](int n, int t) { return Phb[(size_t)t * h + n]; },
-            [&](int m, int n, Real acc, Real) { Wb[LAST][(size_t)m * h + n] += acc; }, &gsm);
+            [&](int m, int n, Real acc, Real) { Wb[LAST][(size_t)m * h + n] += acc; }, &gsm, rank, CL);
         // pu = J(u) e, e = k + y - v, y = LN(u)
-        for (int t = warp; t < len; t += NW) {
+        for (int t = warp + rank * (kSimtThreads / 32); t < len; t += (kSimtThreads / 32) * CL) {
             const size_t row = (size_t)t * d;
             const Real* y = U + row;
             const Real r = rk[t];
@@ -369,7 +365,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
                 st_io(dv + (size_t)s * d, row + i, -Eb[row + i]);
             }
         }
-        __syncthreads();
+        phase_sync(CL);
         // u = Wl a ; a = gelu(z1)  or  silu(z1) z2
         block_gemm<Real, 1, true, false>(
             len, h, d, [&](int m, int kk, Real& a0, Real& a1) { a0 = Ukb[(size_t)m * d + kk]; },
@@ -384,11 +380,11 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
                     Zkb2[e] += ab * silu_f(Z1[e]);
                 }
             },
-            &gsm);
+            &gsm, rank, CL);
         block_gemm<Real, 1, false, false>( // Wbl += Ukb^T Ak
             d, h, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Ukb[(size_t)t * d + m]; },
             [&](int n, int t) { return A[(size_t)t * h + n]; },
-            [&](int m, int n, Real acc, Real) { Wb[LAST][(size_t)m * h + n] += acc; }, &gsm);
+            [&](int m, int n, Real acc, Real) { Wb[LAST][(size_t)m * h + n] += acc; }, &gsm, rank, CL);
         // z1 = W1 k (, z2 = W2 k)
         block_gemm<Real, 1, true, false>(
             len, d, SW ? 2 * h : h,
@@ -400,35 +396,35 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
                 const size_t e = (size_t)m * d + n;
                 st_io(dk + (size_t)s * d, e, Kb[e] + acc);
             },
-            &gsm);
+            &gsm, rank, CL);
         block_gemm<Real, 1, false, false>( // Wb1 += Zkb^T K
             h, d, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Zkb[(size_t)t * h + m]; },
             [&](int n, int t) { return ld_io<Real>(kc, (size_t)t * d + n); },
-            [&](int m, int n, Real acc, Real) { Wb[0][(size_t)m * d + n] += acc; }, &gsm);
+            [&](int m, int n, Real acc, Real) { Wb[0][(size_t)m * d + n] += acc; }, &gsm, rank, CL);
         if (SW)
             block_gemm<Real, 1, false, false>( // Wb2 += Zkb2^T K
                 h, d, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Zkb2[(size_t)t * h + m]; },
                 [&](int n, int t) { return ld_io<Real>(kc, (size_t)t * d + n); },
-                [&](int m, int n, Real acc, Real) { Wb[1][(size_t)m * d + n] += acc; }, &gsm);
+                [&](int m, int n, Real acc, Real) { Wb[1][(size_t)m * d + n] += acc; }, &gsm, rank, CL);
 
         // ---------------- adjoints of the chunk-start state ----------------
         {
             const Real cw = sc.cw, cm = sc.cm, cb = sc.cb;
 #pragma unroll
             for (int i = 0; i < NMAT; ++i)
-                for (size_t e = tid; e < dh; e += kSimtThreads) {
+                for (size_t e = tid + (size_t)rank * kSimtThreads; e < dh; e += (size_t)kSimtThreads * CL) {
                     const Real t = T[i][e], sv = S[i][e];
                     T[i][e] = cw * t + Wb[i][e];
                     S[i][e] = cm * t + cb * sv;
                 }
         }
         // ---------------- (iv) reverse of the suffix scans ----------------
-        if (tid == 0) {
+        if (tid == 0 && rank == 0) {
             Real Sb = 0, btb = cbb, gtb = cwb; // adjoints of S_0 (unused), bt_0, gt_0
             for (int t = 0; t < len; ++t) {
                 // index t: state t; token t+1 lives at array index t
                 const Real b1 = (Real)beta[s + t], g1 = (Real)gamma[s + t], e1 = (Real)eta[s + t];
-                const Real kWb = bs.kWb[t], kMb = bs.kMb[t];
+                const Real kWb = kWb_g[t], kMb = kMb_g[t];
                 // S_t = beta_{t+1} S_{t+1} + gt_t ; bt_t = beta_{t+1} bt_{t+1} ; gt_t = gamma_{t+1} gt_{t+1}
                 gtb += Sb;
                 Real bb = Sb * sc.S[t + 1] + btb * sc.bt[t + 1];
@@ -449,14 +445,14 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
                 Sb = Sb_next; btb = btb_next; gtb = gtb_next;
             }
         }
-        __syncthreads();
+        phase_sync(CL);
     }
 
 #pragma unroll
     for (int i = 0; i < NMAT; ++i) {
         float* wf = a.dW_init[i] + (size_t)seq * dh;
         float* mf = a.dM_init[i] + (size_t)seq * dh;
-        for (size_t e = tid; e < dh; e += kSimtThreads) {
+        for (size_t e = tid + (size_t)rank * kSimtThreads; e < dh; e += (size_t)kSimtThreads * CL) {
             wf[e] = (float)T[i][e];
             mf[e] = (float)S[i][e];
         }
@@ -466,7 +462,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
 template <typename Real, typename IO, int KIND>
 static int launch_bwd(const SimtBwdArgs& a, cudaStream_t st) {
     constexpr size_t smem =
-        sizeof(GemmSmem<Real>) + sizeof(ChunkScalars<Real>) + sizeof(BwdScalars<Real>) + 8 * sizeof(Real);
+        sizeof(GemmSmem<Real>) + sizeof(ChunkScalars<Real>) + 8 * sizeof(Real);
     static bool attr_done[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return (int)cudaGetLastError();
@@ -476,7 +472,20 @@ static int launch_bwd(const SimtBwdArgs& a, cudaStream_t st) {
         if (e != cudaSuccess) return (int)e;
         if (dev >= 0 && dev < 64) attr_done[dev] = true;
     }
-    simt_bwd_kernel<Real, IO, KIND><<<dim3(a.N), dim3(kSimtThreads), smem, st>>>(a);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)(a.N * a.cl));
+    cfg.blockDim = dim3(kSimtThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = (unsigned)a.cl;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, simt_bwd_kernel<Real, IO, KIND>, a);
+    if (e != cudaSuccess) return (int)e;
     return (int)cudaGetLastError();
 }
 

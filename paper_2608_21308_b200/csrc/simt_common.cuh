@@ -149,22 +149,38 @@ __device__ void chunk_scalars_warp(const float* eta, const float* beta, const fl
     }
 }
 
+// ---- phase barrier ---------------------------------------------------------------------------------
+// A sequence may be worked on by a cluster of `nranks` CTAs that split every phase (GEMM tiles, rows, elements)
+// and share all intermediates through global memory.  The hardware cluster barrier (release / acquire at cluster
+// scope) orders one phase's global writes before the next phase's reads; with one CTA it is the CTA barrier.
+__device__ __forceinline__ void phase_sync(int nranks) {
+    if (nranks == 1) {
+        __syncthreads();
+    } else {
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    }
+}
+
 // ---- generic CTA GEMM --------------------------------------------------------------------------
 // out(m, n) = sum_k a(m, k) * b(n, k), m < M, n < N, k < K, for NACC (1 or 2) A operands sharing one B.
 //   fa(m, k, a0, a1) writes the A value(s); fb(n, k) returns the B value; epi(m, n, acc0, acc1) consumes a result.
 // A_KFAST / B_KFAST say which index is contiguous in memory, so that neighbouring threads read neighbouring words.
-// 64x64 output tiles, 16-deep k slices through shared memory, 4x4 results per thread.  Ends with __syncthreads().
+// 64x64 output tiles (dealt round-robin to the `nranks` CTAs of the sequence's cluster), 16-deep k slices through
+// shared memory, 4x4 results per thread.  Ends with phase_sync().
 template <typename Real> struct GemmSmem {
     Real A[2][kBK][kBM + 4];
     Real B[kBK][kBN + 4];
 };
 
 template <typename Real, int NACC, bool A_KFAST, bool B_KFAST, typename FA, typename FB, typename FE>
-__device__ void block_gemm(int M, int N, int K, FA fa, FB fb, FE epi, GemmSmem<Real>* sm) {
+__device__ void block_gemm(int M, int N, int K, FA fa, FB fb, FE epi, GemmSmem<Real>* sm, int rank, int nranks) {
     const int tid = threadIdx.x;
     const int tx = tid & 15, ty = tid >> 4;
+    int tile = 0;
     for (int m0 = 0; m0 < M; m0 += kBM) {
-        for (int n0 = 0; n0 < N; n0 += kBN) {
+        for (int n0 = 0; n0 < N; n0 += kBN, ++tile) {
+            if (tile % nranks != rank) continue;
             Real acc[NACC][4][4];
 #pragma unroll
             for (int a = 0; a < NACC; ++a)
@@ -219,7 +235,7 @@ __device__ void block_gemm(int M, int N, int K, FA fa, FB fb, FE epi, GemmSmem<R
                 }
         }
     }
-    __syncthreads();
+    phase_sync(nranks);
 }
 
 // ---- layer norm of one row by one warp -----------------------------------------------------------

@@ -13,7 +13,8 @@ __global__ void __launch_bounds__(kSimtThreads) simt_fwd_kernel(const SimtFwdArg
     GemmSmem<Real>& gsm = *reinterpret_cast<GemmSmem<Real>*>(simt_smem_raw);
     ChunkScalars<Real>& sc = *reinterpret_cast<ChunkScalars<Real>*>(simt_smem_raw + sizeof(GemmSmem<Real>));
 
-    const int seq = blockIdx.x;
+    const int CL = a.cl;                 // CTAs working on this sequence (one cluster)
+    const int seq = blockIdx.x / CL, rank = blockIdx.x % CL;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int d = a.d, h = a.h, C = a.C, L = a.L;
     const size_t dh = (size_t)d * h;
@@ -36,7 +37,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_fwd_kernel(const SimtFwdArg
         M[i] = ws + lay.M[i];
         const float* wi = a.W_init[i] + (size_t)seq * dh;
         const float* mi = a.M_init[i] ? a.M_init[i] + (size_t)seq * dh : nullptr;
-        for (size_t e = tid; e < dh; e += kSimtThreads) {
+        for (size_t e = tid + (size_t)rank * kSimtThreads; e < dh; e += (size_t)kSimtThreads * CL) {
             W[i][e] = (Real)wi[e];
             M[i][e] = mi ? (Real)mi[e] : (Real)0;
         }
@@ -48,7 +49,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_fwd_kernel(const SimtFwdArg
     Real* Pu = ws + lay.Pu;
     Real* Pz1 = ws + lay.Pz1;
     Real* Pz2 = ws + lay.Pz2;
-    __syncthreads();
+    phase_sync(CL);
 
     for (int c = 0; c < a.nchunks; ++c) {
         const int s = c * C;
@@ -63,7 +64,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_fwd_kernel(const SimtFwdArg
             Real* ck = ws + lay.ckpt + (size_t)c * 2 * NMAT * dh;
 #pragma unroll
             for (int i = 0; i < NMAT; ++i)
-                for (size_t e = tid; e < dh; e += kSimtThreads) {
+                for (size_t e = tid + (size_t)rank * kSimtThreads; e < dh; e += (size_t)kSimtThreads * CL) {
                     ck[(size_t)i * dh + e] = W[i][e];
                     ck[(size_t)(NMAT + i) * dh + e] = M[i][e];
                 }
@@ -75,21 +76,21 @@ __global__ void __launch_bounds__(kSimtThreads) simt_fwd_kernel(const SimtFwdArg
         };
         block_gemm<Real, 1, true, true>(
             2 * len, h, d, load_x, [&](int n, int kk) { return W[0][(size_t)n * d + kk]; },
-            [&](int m, int n, Real acc, Real) { Z1[(size_t)m * h + n] = acc; }, &gsm);
+            [&](int m, int n, Real acc, Real) { Z1[(size_t)m * h + n] = acc; }, &gsm, rank, CL);
         if (KIND == 1)
             block_gemm<Real, 1, true, true>(
                 2 * len, h, d, load_x, [&](int n, int kk) { return W[1][(size_t)n * d + kk]; },
-                [&](int m, int n, Real acc, Real) { Z2[(size_t)m * h + n] = acc; }, &gsm);
-        for (size_t e = tid; e < (size_t)2 * len * h; e += kSimtThreads)
+                [&](int m, int n, Real acc, Real) { Z2[(size_t)m * h + n] = acc; }, &gsm, rank, CL);
+        for (size_t e = tid + (size_t)rank * kSimtThreads; e < (size_t)2 * len * h; e += (size_t)kSimtThreads * CL)
             A[e] = (KIND == 0) ? gelu_f(Z1[e]) : silu_f(Z1[e]) * Z2[e];
-        __syncthreads();
+        phase_sync(CL);
         block_gemm<Real, 1, true, true>(
             2 * len, d, h, [&](int m, int kk, Real& a0, Real& a1) { a0 = A[(size_t)m * h + kk]; },
             [&](int n, int kk) { return W[LAST][(size_t)n * h + kk]; },
-            [&](int m, int n, Real acc, Real) { U[(size_t)m * d + n] = acc; }, &gsm);
+            [&](int m, int n, Real acc, Real) { U[(size_t)m * d + n] = acc; }, &gsm, rank, CL);
 
         // layer norm; outputs for the query rows; e = f(k) - v and pu = dL/du for the key rows (Algorithm 1 line 3)
-        for (int m = warp; m < 2 * len; m += kSimtThreads / 32) {
+        for (int m = warp + rank * (kSimtThreads / 32); m < 2 * len; m += (kSimtThreads / 32) * CL) {
             Real* u = U + (size_t)m * d;
             const Real r = warp_layernorm(u, u, d, eps);
             if (m >= len) {
@@ -113,7 +114,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_fwd_kernel(const SimtFwdArg
                 }
             }
         }
-        __syncthreads();
+        phase_sync(CL);
 
         // back through the last matrix and the activation
         block_gemm<Real, 1, true, false>(
@@ -128,7 +129,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_fwd_kernel(const SimtFwdArg
                     Pz2[e] = acc * silu_f(Z1[e]);
                 }
             },
-            &gsm);
+            &gsm, rank, CL);
 
         // Algorithm 1 lines 4-7: both weighted aggregations of every matrix, fused with the state transition
         const Real cw = sc.cw, cm = sc.cm, cb = sc.cb;
@@ -147,7 +148,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_fwd_kernel(const SimtFwdArg
                     Wm[e] = cw * w + cm * mm - aW; // G_t = -grad: the aggregations enter with a minus sign
                     Mm[e] = cb * mm - aM;
                 },
-                &gsm);
+                &gsm, rank, CL);
         };
         auto key_col = [&](int n, int t) { return ld_io<Real>(kc, (size_t)t * d + n); };
         auto act_col = [&](int n, int t) { return A[(size_t)t * h + n]; };
@@ -161,7 +162,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_fwd_kernel(const SimtFwdArg
         if (!a.W_final[i]) continue; // state-recompute run of the backward: only the saved chunk states matter
         float* wf = a.W_final[i] + (size_t)seq * dh;
         float* mf = a.M_final[i] + (size_t)seq * dh;
-        for (size_t e = tid; e < dh; e += kSimtThreads) {
+        for (size_t e = tid + (size_t)rank * kSimtThreads; e < dh; e += (size_t)kSimtThreads * CL) {
             wf[e] = (float)W[i][e];
             mf[e] = (float)M[i][e];
         }
@@ -179,7 +180,20 @@ static int launch_fwd(const SimtFwdArgs& a, cudaStream_t st) {
         if (e != cudaSuccess) return (int)e;
         if (dev >= 0 && dev < 64) attr_done[dev] = true;
     }
-    simt_fwd_kernel<Real, IO, KIND><<<dim3(a.N), dim3(kSimtThreads), smem, st>>>(a);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)(a.N * a.cl));
+    cfg.blockDim = dim3(kSimtThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = (unsigned)a.cl;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, simt_fwd_kernel<Real, IO, KIND>, a);
+    if (e != cudaSuccess) return (int)e;
     return (int)cudaGetLastError();
 }
 

@@ -17,6 +17,7 @@ struct SimtLayout {
     size_t Pa, E, XY2, XY1, Pub, Pzb, Zkb, Akb, Kb, Eb, Ukb, Uqb, Zqb;
     size_t XY1b, Pzb2, Zkb2, Zqb2;  // SwiGLU only: the second [h x d] matrix
     size_t rk, rq, red;  // per-row 1/std of the two LN calls; small reduction scratch
+    size_t kWb, kMb;     // adjoints of the scalar kernels, one per token of the chunk
     size_t ckpt;         // [nchunks][2][nmat][d*h] chunk-start (W, M), present when states are saved
     size_t per_seq;      // elements per sequence
 };
@@ -42,6 +43,7 @@ inline SimtLayout simt_layout(int d, int h, int C, int nmat, int nchunks, bool s
         const size_t sw = (nmat == 3) ? 1 : 0;
         l.XY1b = take(sw * C * 2 * h); l.Pzb2 = take(sw * C * h); l.Zkb2 = take(sw * C * h); l.Zqb2 = take(sw * C * h);
         l.rk = take(C); l.rq = take(C); l.red = take(64);
+        l.kWb = take(C); l.kMb = take(C);
     }
     l.ckpt = take(save_states ? (size_t)nchunks * 2 * nmat * dh : 0);
     l.per_seq = o;
@@ -50,6 +52,7 @@ inline SimtLayout simt_layout(int d, int h, int C, int nmat, int nchunks, bool s
 
 struct SimtFwdArgs {
     int N, L, d, h, C, nchunks, save_states;
+    int cl;  // CTAs per sequence (cluster size), chosen by the launcher
     float eps;
     const void *q, *k, *v;
     const float *eta, *beta, *gamma;
@@ -64,6 +67,7 @@ struct SimtFwdArgs {
 
 struct SimtBwdArgs {
     int N, L, d, h, C, nchunks;
+    int cl;  // CTAs per sequence (cluster size), chosen by the launcher
     float eps;
     const void *q, *k, *v, *d_o;
     const float *eta, *beta, *gamma;
@@ -76,6 +80,13 @@ struct SimtBwdArgs {
     void* ws;
     SimtLayout lay;
 };
+
+// CTAs per sequence: the largest power of two <= 8 that keeps N * cl within one wave of the GPU's SMs
+inline int simt_cluster_size(int N) {
+    int cl = 1;
+    while (cl < 8 && (long long)N * (cl * 2) <= 148) cl *= 2;
+    return cl;
+}
 
 // launchers (simt_fwd.cu / simt_bwd.cu); return a cudaError_t value as int
 int simt_fwd_launch(const SimtFwdArgs& a, int kind, int io_dtype, void* stream);
