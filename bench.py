@@ -358,7 +358,7 @@ def run_fwd_bwd(args, r):
     flop = flops_per_token_head(r, backward=True) * N * r.L
     cfg = workload_config(r)
     cfg["workload"] = cfg["workload"].replace("e2ttt_chunk_fwd", "e2ttt_chunk_fwd(save_states) + e2ttt_chunk_bwd")
-    cfg["path"] = "SIMT kernels (the tensor-core path covers the forward without saved states only)"
+    cfg["path"] = "tensor-core forward writing chunk-start states where a specialisation exists, SIMT backward"
     line = {"metric": "e2ttt_layer_fwd_bwd_tokens_per_s", "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if r.io == "bf16" else "f64", "data": "synthetic", "config": cfg,

@@ -117,8 +117,7 @@ E2TTT_API int e2ttt_workspace_bytes(const e2ttt_params* p, int save_states, size
  *   W_final, M_final out  host tables, same layout as W_init; may alias W_init / M_init
  *   workspace        device scratch of at least e2ttt_workspace_bytes(p, save_states) bytes,
  *                    256-byte aligned; with save_states != 0 it holds, after the call, the
- *                    (W, M) at the start of every chunk for e2ttt_chunk_bwd (a forward that
- *                    saves states always runs on the SIMT path)
+ *                    (W, M) at the start of every chunk for e2ttt_chunk_bwd
  */
 E2TTT_API int e2ttt_chunk_fwd(const e2ttt_params* p,
                     const void* q, const void* k, const void* v,

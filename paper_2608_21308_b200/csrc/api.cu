@@ -30,9 +30,10 @@ int check_params(const e2ttt_params* p) {
 // Every workspace starts with a status block: word 0 is the device status of the last launch that used it.
 constexpr size_t kStatusBytes = 256;
 
-// 1 = a tensor-core specialisation exists for these parameters (forward without saved chunk states)
-int has_tcgen05(const e2ttt_params* p, bool save_states) {
-    return !save_states && p->kind == E2TTT_MLP_GELU && p->io_dtype == E2TTT_BF16 && p->d == 128 && p->h == 512 &&
+// 1 = a tensor-core specialisation exists for these parameters (the forward; with save_states it also writes the
+// chunk-start states in the layout the SIMT backward reads)
+int has_tcgen05(const e2ttt_params* p, bool /*save_states*/) {
+    return p->kind == E2TTT_MLP_GELU && p->io_dtype == E2TTT_BF16 && p->d == 128 && p->h == 512 &&
            p->C == 64 && p->L % 64 == 0;
 }
 
@@ -99,7 +100,7 @@ int e2ttt_workspace_bytes(const e2ttt_params* p, int save_states, size_t* bytes)
     if (rc) return rc;
     // tensor-core path: all state lives on chip, only the status block is needed.
     // SIMT path: with saved states the same buffer serves the backward, which needs the larger layout.
-    *bytes = (impl == E2TTT_IMPL_TCGEN05) ? kStatusBytes : simt_bytes(p, save_states != 0, save_states != 0);
+    *bytes = (impl == E2TTT_IMPL_TCGEN05 && !save_states) ? kStatusBytes : simt_bytes(p, save_states != 0, save_states != 0);
     return E2TTT_OK;
 }
 
@@ -137,6 +138,11 @@ int e2ttt_chunk_fwd(const e2ttt_params* p, const void* q, const void* k, const v
         t.M1_init = M_init ? M_init[0] : nullptr; t.M2_init = M_init ? M_init[1] : nullptr;
         t.W1_final = W_final[0]; t.W2_final = W_final[1]; t.M1_final = M_final[0]; t.M2_final = M_final[1];
         t.status = static_cast<int*>(workspace);
+        if (save_states) {
+            const SimtLayout lay = simt_layout(p->d, p->h, p->C, nmat, p->L / p->C, true, true);
+            t.ckpt = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBytes) + lay.ckpt;
+            t.ckpt_seq_stride = lay.per_seq;
+        }
         return tc_fwd_launch(t, stream) == 0 ? E2TTT_OK : E2TTT_ERR_CUDA;
     }
     if (cudaMemsetAsync(workspace, 0, sizeof(int), reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) {

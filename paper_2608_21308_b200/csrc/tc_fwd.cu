@@ -249,6 +249,22 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             for (int j = 0; j < 16; ++j) { st[j] = __float_as_uint(cw0 * w[j]); M2[16 * b + j] = m2 ? m2[16 * b + j] : 0.0f; }
             tmem_st16(lane_addr + T_W2 + c0 + 16 * b, st);
             st_slab16(s.W2[(c0 + 16 * b) >> 6], row, (c0 + 16 * b) & 63, w);
+            if (a.ckpt) {  // chunk-start state of chunk 0 (w currently holds the W2 piece)
+                float* ck = a.ckpt + (size_t)seq * a.ckpt_seq_stride;
+                float* d2 = ck + (size_t)(D * 4 * HC) + (size_t)row * (4 * HC) + HC * me + c0 + 16 * b;
+                float* dm1 = ck + 2 * (size_t)(D * 4 * HC) + ((size_t)(HC * me) + row) * D + c0 + 16 * b;
+                float* dm2 = ck + 3 * (size_t)(D * 4 * HC) + (size_t)row * (4 * HC) + HC * me + c0 + 16 * b;
+                float* d1 = ck + ((size_t)(HC * me) + row) * D + c0 + 16 * b;
+#pragma unroll
+                for (int j = 0; j < 16; j += 4) {
+                    *reinterpret_cast<float4*>(d2 + j) = make_float4(w[j], w[j + 1], w[j + 2], w[j + 3]);
+                    *reinterpret_cast<float4*>(d1 + j) = *reinterpret_cast<const float4*>(w1 + 16 * b + j);
+                    *reinterpret_cast<float4*>(dm1 + j) =
+                        make_float4(M1[16 * b + j], M1[16 * b + j + 1], M1[16 * b + j + 2], M1[16 * b + j + 3]);
+                    *reinterpret_cast<float4*>(dm2 + j) =
+                        make_float4(M2[16 * b + j], M2[16 * b + j + 1], M2[16 * b + j + 2], M2[16 * b + j + 3]);
+                }
+            }
         }
         tmem_wait_st();
     }
@@ -643,9 +659,11 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             }
             tmem_st16(lane_addr + T_W1 + col, st);
             st_slab16(s.W1[col >> 6], row, col & 63, wn);
-            if (last) {
-                float* wf = a.W1_final + head + ((size_t)(HC * me) + row) * D + col;
-                float* mf = a.M1_final + head + ((size_t)(HC * me) + row) * D + col;
+            if (last || a.ckpt) {  // final state, or the next chunk's start state for the backward
+                const size_t off = ((size_t)(HC * me) + row) * D + col;
+                float* ck = last ? nullptr : a.ckpt + (size_t)seq * a.ckpt_seq_stride + (size_t)(r + 1) * 4 * (size_t)(D * 4 * HC);
+                float* wf = last ? a.W1_final + head + off : ck + off;
+                float* mf = last ? a.M1_final + head + off : ck + 2 * (size_t)(D * 4 * HC) + off;
 #pragma unroll
                 for (int j = 0; j < 16; j += 4) {
                     *reinterpret_cast<float4*>(wf + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
@@ -690,9 +708,11 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             }
             tmem_st16(lane_addr + T_W2 + col, st);
             st_slab16(s.W2[col >> 6], row, col & 63, wn);
-            if (last) {
-                float* wf = a.W2_final + head + (size_t)row * (4 * HC) + HC * me + col;
-                float* mf = a.M2_final + head + (size_t)row * (4 * HC) + HC * me + col;
+            if (last || a.ckpt) {
+                const size_t off = (size_t)row * (4 * HC) + HC * me + col;
+                float* ck = last ? nullptr : a.ckpt + (size_t)seq * a.ckpt_seq_stride + (size_t)(r + 1) * 4 * (size_t)(D * 4 * HC);
+                float* wf = last ? a.W2_final + head + off : ck + (size_t)(D * 4 * HC) + off;
+                float* mf = last ? a.M2_final + head + off : ck + 3 * (size_t)(D * 4 * HC) + off;
 #pragma unroll
                 for (int j = 0; j < 16; j += 4) {
                     *reinterpret_cast<float4*>(wf + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);

@@ -18,6 +18,9 @@ struct TcFwdArgs {
     __nv_bfloat16* o;
     float *W1_final, *W2_final, *M1_final, *M2_final;
     int* status;  // device word, 0 after a clean run
+    // optional: chunk-start states for the backward, fp32, [N][nchunks][W1 | W2 | M1 | M2] (nullptr = do not save)
+    float* ckpt;
+    size_t ckpt_seq_stride;  // floats between two sequences
 };
 
 size_t tc_fwd_smem_bytes();

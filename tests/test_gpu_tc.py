@@ -84,3 +84,19 @@ def test_tc_full_benchmark_size_properties_and_sampled_outputs():
               for n, v in x.items()}
     ref = util.oracle_forward(sample, 64, MLP, use_M=False)
     assert util.rel_err(whole["o"][heads, :64], ref["o"]) <= TOL_BF16
+
+
+def test_tc_forward_saves_states_for_the_backward():
+    """Training flow on config 4's shape: tensor-core forward writes the chunk-start states, the reverse pass reads them."""
+    from tests.test_gpu_parity import check_backward
+    r = inputs.config(4, heads=[2, 11])
+    xw, _ = util.teacher_forced_windows(r, 3, window=1, with_grads=True)
+    ref = util.oracle_backward(xw, r.C, r.kind)
+    got = util.gpu_backward(xw, d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16", via_saved_states=True)
+    check_backward(got, ref, TOL_BF16, "bwd from tensor-core saved states")
+    # two chunks per call: the second chunk's start state comes from the tensor-core state pass
+    x2, _ = util.teacher_forced_windows(r, 4, window=2, with_grads=True)
+    a = util.gpu_backward(x2, d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16", via_saved_states=True)
+    b = util.gpu_backward(x2, d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16", via_saved_states=False)
+    for n in ("dq", "dk", "dv", "deta", "dbeta", "dgamma"):
+        assert util.rel_err(a[n], b[n]) <= 3 * TOL_BF16, n   # saved (tensor-core) vs recomputed (SIMT) forward states
