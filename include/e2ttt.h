@@ -60,8 +60,9 @@ typedef enum { E2TTT_MLP_GELU = 0, E2TTT_SWIGLU = 1 } e2ttt_kind;
 typedef enum { E2TTT_F32 = 0, E2TTT_BF16 = 1 } e2ttt_dtype;
 
 /* Which kernel family serves the call.
- *   AUTO    : the tensor-core path where a specialisation exists for (kind, io_dtype, d, h, C),
- *             else the SIMT path.
+ *   AUTO    : the tensor-core path where it serves (kind, io_dtype, d, h, C), else the SIMT path.
+ *             Served today: GELU-MLP, bf16 I/O, C = 64, L a multiple of 64, d in {64, 128},
+ *             h in {128, 256, 384, 512} (shapes below 128 x 512 run zero-padded in the same tiles).
  *   SIMT    : plain CUDA-core kernels for any shape.  With fp32 I/O they compute in fp64
  *             internally; with bf16 I/O in fp32.
  *   TCGEN05 : bf16 operands on the 5th-generation tensor cores with fp32 accumulation in tensor

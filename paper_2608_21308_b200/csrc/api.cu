@@ -33,8 +33,8 @@ constexpr size_t kStatusBytes = 256;
 // 1 = a tensor-core specialisation exists for these parameters (the forward; with save_states it also writes the
 // chunk-start states in the layout the SIMT backward reads)
 int has_tcgen05(const e2ttt_params* p, bool /*save_states*/) {
-    return p->kind == E2TTT_MLP_GELU && p->io_dtype == E2TTT_BF16 && p->d == 128 && p->h == 512 &&
-           p->C == 64 && p->L % 64 == 0;
+    return p->kind == E2TTT_MLP_GELU && p->io_dtype == E2TTT_BF16 && (p->d == 128 || p->d == 64) && p->h % 128 == 0 &&
+           p->h <= 512 && p->C == 64 && p->L % 64 == 0;
 }
 
 int pick_impl(const e2ttt_params* p, bool save_states, int* impl) {
@@ -130,7 +130,7 @@ int e2ttt_chunk_fwd(const e2ttt_params* p, const void* q, const void* k, const v
 
     if (impl == E2TTT_IMPL_TCGEN05) {
         TcFwdArgs t{};
-        t.N = p->B * p->H; t.L = p->L; t.eps = p->ln_eps;
+        t.N = p->B * p->H; t.L = p->L; t.d = p->d; t.h = p->h; t.eps = p->ln_eps;
         t.q = static_cast<const __nv_bfloat16*>(q); t.k = static_cast<const __nv_bfloat16*>(k);
         t.v = static_cast<const __nv_bfloat16*>(v); t.o = static_cast<__nv_bfloat16*>(o);
         t.eta = eta; t.beta = beta; t.gamma = gamma;

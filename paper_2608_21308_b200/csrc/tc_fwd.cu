@@ -159,6 +159,8 @@ __device__ __forceinline__ void st_slab16(uint8_t* slab, int row, int col0, cons
     *reinterpret_cast<uint4*>(slab + row * 128 + (((c + 1) ^ (row & 7)) << 4)) = b;
 }
 
+// PAD = false: the native 128 x 512 shape, every mask folds away.  PAD = true: d and h come from the arguments.
+template <bool PAD>
 __global__ void __launch_bounds__(NTHREADS, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
               const __grid_constant__ CUtensorMap tmV, const TcFwdArgs a) {
@@ -181,9 +183,13 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     const int L = a.L, nchunks = L / C;
     WaitCtx wc{&s.dead, a.status};
 
-    const __nv_bfloat16* gk = a.k + (size_t)seq * L * D;
-    const __nv_bfloat16* gq = a.q + (size_t)seq * L * D;
-    __nv_bfloat16* go = a.o + (size_t)seq * L * D;
+    // Real shape: de x he.  Columns >= de of every token tile and hidden units >= he are zero padding: they stay
+    // exactly zero through every product, so only the layer norm (divisor, masks) and the global I/O know about them.
+    const int de = PAD ? a.d : D, he = PAD ? a.h : NC * HC;
+    const size_t dh = (size_t)de * he;
+    const bool cta_real = HC * (int)me < he;  // this CTA's 128 hidden units exist
+    const float inv_d = 1.0f / (float)de;
+    __nv_bfloat16* go = a.o + (size_t)seq * L * de;
     const float* eta = a.eta + (size_t)seq * L;
     const float* beta = a.beta + (size_t)seq * L;
     const float* gamma = a.gamma + (size_t)seq * L;
@@ -220,62 +226,72 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     float M1[CW], M2[CW];
     {
         const float cw0 = s.sc[0].cw;
-        const size_t head = (size_t)seq * (size_t)(D * 4 * HC);
+        const size_t head = (size_t)seq * dh;
         // W1c[j][i]: global W1 [h][d], row 128 me + j
-        const float* w1 = a.W1_init + head + ((size_t)(HC * me) + row) * D + c0;
-        const float* m1 = a.M1_init ? a.M1_init + head + ((size_t)(HC * me) + row) * D + c0 : nullptr;
+        const float* w1 = a.W1_init + head + ((size_t)(HC * me) + row) * de + c0;
+        const float* m1 = a.M1_init ? a.M1_init + head + ((size_t)(HC * me) + row) * de + c0 : nullptr;
         // W2c[i][j]: global W2 [d][h], row i, column 128 me + j
-        const float* w2 = a.W2_init + head + (size_t)row * (4 * HC) + HC * me + c0;
-        const float* m2 = a.M2_init ? a.M2_init + head + (size_t)row * (4 * HC) + HC * me + c0 : nullptr;
+        const float* w2 = a.W2_init + head + (size_t)row * he + HC * me + c0;
+        const float* m2 = a.M2_init ? a.M2_init + head + (size_t)row * he + HC * me + c0 : nullptr;
+        const bool real2 = cta_real && row < de;  // this thread's W2 row exists
 #pragma unroll
         for (int b = 0; b < NB; ++b) {
             float w[16];
             uint32_t st[16];
+            const bool real1 = cta_real && c0 + 16 * b < de;  // these 16 columns of W1 exist
 #pragma unroll
             for (int j = 0; j < 16; j += 4) {
-                const float4 x = *reinterpret_cast<const float4*>(w1 + 16 * b + j);
+                const float4 x = real1 ? *reinterpret_cast<const float4*>(w1 + 16 * b + j) : make_float4(0.f, 0.f, 0.f, 0.f);
                 w[j] = x.x; w[j + 1] = x.y; w[j + 2] = x.z; w[j + 3] = x.w;
             }
 #pragma unroll
-            for (int j = 0; j < 16; ++j) { st[j] = __float_as_uint(cw0 * w[j]); M1[16 * b + j] = m1 ? m1[16 * b + j] : 0.0f; }
+            for (int j = 0; j < 16; ++j) { st[j] = __float_as_uint(cw0 * w[j]); M1[16 * b + j] = (m1 && real1) ? m1[16 * b + j] : 0.0f; }
             tmem_st16(lane_addr + T_W1 + c0 + 16 * b, st);
             st_slab16(s.W1[(c0 + 16 * b) >> 6], row, (c0 + 16 * b) & 63, w);
+            float* ck = a.ckpt ? a.ckpt + (size_t)seq * a.ckpt_seq_stride : nullptr;  // chunk-start state of chunk 0
+            if (ck && real1) {
+                const size_t o1 = ((size_t)(HC * me) + row) * de + c0 + 16 * b;
+#pragma unroll
+                for (int j = 0; j < 16; j += 4) {
+                    *reinterpret_cast<float4*>(ck + o1 + j) = make_float4(w[j], w[j + 1], w[j + 2], w[j + 3]);
+                    *reinterpret_cast<float4*>(ck + 2 * dh + o1 + j) =
+                        make_float4(M1[16 * b + j], M1[16 * b + j + 1], M1[16 * b + j + 2], M1[16 * b + j + 3]);
+                }
+            }
 #pragma unroll
             for (int j = 0; j < 16; j += 4) {
-                const float4 x = *reinterpret_cast<const float4*>(w2 + 16 * b + j);
+                const float4 x = real2 ? *reinterpret_cast<const float4*>(w2 + 16 * b + j) : make_float4(0.f, 0.f, 0.f, 0.f);
                 w[j] = x.x; w[j + 1] = x.y; w[j + 2] = x.z; w[j + 3] = x.w;
             }
 #pragma unroll
-            for (int j = 0; j < 16; ++j) { st[j] = __float_as_uint(cw0 * w[j]); M2[16 * b + j] = m2 ? m2[16 * b + j] : 0.0f; }
+            for (int j = 0; j < 16; ++j) { st[j] = __float_as_uint(cw0 * w[j]); M2[16 * b + j] = (m2 && real2) ? m2[16 * b + j] : 0.0f; }
             tmem_st16(lane_addr + T_W2 + c0 + 16 * b, st);
             st_slab16(s.W2[(c0 + 16 * b) >> 6], row, (c0 + 16 * b) & 63, w);
-            if (a.ckpt) {  // chunk-start state of chunk 0 (w currently holds the W2 piece)
-                float* ck = a.ckpt + (size_t)seq * a.ckpt_seq_stride;
-                float* d2 = ck + (size_t)(D * 4 * HC) + (size_t)row * (4 * HC) + HC * me + c0 + 16 * b;
-                float* dm1 = ck + 2 * (size_t)(D * 4 * HC) + ((size_t)(HC * me) + row) * D + c0 + 16 * b;
-                float* dm2 = ck + 3 * (size_t)(D * 4 * HC) + (size_t)row * (4 * HC) + HC * me + c0 + 16 * b;
-                float* d1 = ck + ((size_t)(HC * me) + row) * D + c0 + 16 * b;
+            if (ck && real2) {
+                const size_t o2 = (size_t)row * he + HC * me + c0 + 16 * b;
 #pragma unroll
                 for (int j = 0; j < 16; j += 4) {
-                    *reinterpret_cast<float4*>(d2 + j) = make_float4(w[j], w[j + 1], w[j + 2], w[j + 3]);
-                    *reinterpret_cast<float4*>(d1 + j) = *reinterpret_cast<const float4*>(w1 + 16 * b + j);
-                    *reinterpret_cast<float4*>(dm1 + j) =
-                        make_float4(M1[16 * b + j], M1[16 * b + j + 1], M1[16 * b + j + 2], M1[16 * b + j + 3]);
-                    *reinterpret_cast<float4*>(dm2 + j) =
+                    *reinterpret_cast<float4*>(ck + dh + o2 + j) = make_float4(w[j], w[j + 1], w[j + 2], w[j + 3]);
+                    *reinterpret_cast<float4*>(ck + 3 * dh + o2 + j) =
                         make_float4(M2[16 * b + j], M2[16 * b + j + 1], M2[16 * b + j + 2], M2[16 * b + j + 3]);
                 }
             }
         }
         tmem_wait_st();
     }
-    if (is_issuer) {
-        mbar_expect_tx(&s.bar_x, 32768);
-        const int y = seq * L;
+    // token tile of the chunk that starts at global row y: keys into rows 0..63, queries into rows 64..127
+    auto load_tokens = [&](int y) {
+        mbar_expect_tx(&s.bar_x, de == 128 ? 32768u : 16384u);
         tma_load_2d(s.X[0], &tmK, 0, y, &s.bar_x);
-        tma_load_2d(s.X[1], &tmK, 64, y, &s.bar_x);
         tma_load_2d(s.X[0] + 8192, &tmQ, 0, y, &s.bar_x);
-        tma_load_2d(s.X[1] + 8192, &tmQ, 64, y, &s.bar_x);
-    }
+        if (de == 128) {
+            tma_load_2d(s.X[1], &tmK, 64, y, &s.bar_x);
+            tma_load_2d(s.X[1] + 8192, &tmQ, 64, y, &s.bar_x);
+        }
+    };
+    if (de < 128)  // the padded half of the token tile is never loaded: zero it once
+        for (int i = tid; i < 16384 / 16; i += NTHREADS) reinterpret_cast<uint4*>(s.X[1])[i] = make_uint4(0u, 0u, 0u, 0u);
+    if (is_issuer) load_tokens(seq * L);
     fence_proxy_async_smem();
     tc_fence_before_sync();
     __syncthreads();
@@ -314,9 +330,14 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             if (r + 1 < nchunks) {
                 // the next chunk's tokens: into L2 now, so that the loads issued at the end of this chunk are short
                 const int y = seq * L + tok0 + C;
-                tma_prefetch_l2_2d(&tmK, 0, y); tma_prefetch_l2_2d(&tmK, 64, y);
-                tma_prefetch_l2_2d(&tmQ, 0, y); tma_prefetch_l2_2d(&tmQ, 64, y);
-                tma_prefetch_l2_2d(&tmV, 0, y + 16 * (int)me); tma_prefetch_l2_2d(&tmV, 64, y + 16 * (int)me);
+                tma_prefetch_l2_2d(&tmK, 0, y);
+                tma_prefetch_l2_2d(&tmQ, 0, y);
+                tma_prefetch_l2_2d(&tmV, 0, y + 16 * (int)me);
+                if (de == 128) {
+                    tma_prefetch_l2_2d(&tmK, 64, y);
+                    tma_prefetch_l2_2d(&tmQ, 64, y);
+                    tma_prefetch_l2_2d(&tmV, 64, y + 16 * (int)me);
+                }
             }
             mbar_expect_tx(&s.bar_partK, 3 * 8192);  // this chunk's incoming partial sums and pu rows
             mbar_expect_tx(&s.bar_partQ, 3 * 8192);
@@ -355,10 +376,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         mbar_wait(&s.bar_g2, ph, wc, 100 + 3);
         if (is_issuer) {
             // the 16 value rows this CTA needs for its key rows: into the gelu tile's first slab, dead once G2 is done
-            mbar_expect_tx(&s.bar_v, 4096);
+            mbar_expect_tx(&s.bar_v, de == 128 ? 4096u : 2048u);
             const int y = seq * L + tok0 + 16 * (int)me;
             tma_load_2d(s.A[0], &tmV, 0, y, &s.bar_v);
-            tma_load_2d(s.A[0] + 2048, &tmV, 64, y, &s.bar_v);
+            if (de == 128) tma_load_2d(s.A[0] + 2048, &tmV, 64, y, &s.bar_v);
         }
         __syncwarp();
         PROF(3);
@@ -435,7 +456,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             const int t = 16 * (int)me + (lrow & 15);    // token inside the chunk
             const int xrow = key_rows ? t : 64 + t;      // its row in the X tile
             const int col0 = CPT * cg;
-            const size_t off = (size_t)(tok0 + t) * D + col0;
+            const size_t off = (size_t)(tok0 + t) * de + col0;
+            const bool real = col0 < de;  // this thread's 8 columns exist (padding columns carry exact zeros)
             uint4 vraw[CPT / 8], xraw[CPT / 8];
 #pragma unroll
             for (int ch = 0; ch < CPT / 8; ++ch) {
@@ -449,7 +471,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 #pragma unroll
                 for (int ch = 0; ch < CPT / 8; ++ch) {
                     const int c = ((col0 & 63) >> 3) + ch;
-                    vraw[ch] = *reinterpret_cast<const uint4*>(s.A[0] + (col0 >> 6) * 2048 + lr * 128 + ((c ^ (lr & 7)) << 4));
+                    vraw[ch] = real ? *reinterpret_cast<const uint4*>(s.A[0] + (col0 >> 6) * 2048 + lr * 128 + ((c ^ (lr & 7)) << 4))
+                                    : make_uint4(0u, 0u, 0u, 0u);
                 }
             }
             float u[CPT];
@@ -474,13 +497,13 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             float sum = 0.0f;
 #pragma unroll
             for (int j = 0; j < CPT; ++j) sum += u[j];
-            const float mu = row_sum(sum) * (1.0f / D);
+            const float mu = row_sum(sum) * inv_d;
             float sq = 0.0f;
 #pragma unroll
-            for (int j = 0; j < CPT; ++j) { u[j] -= mu; sq = fmaf(u[j], u[j], sq); }
-            const float rstd = rsqrtf(row_sum(sq) * (1.0f / D) + a.eps);
+            for (int j = 0; j < CPT; ++j) { u[j] = real ? u[j] - mu : 0.0f; sq = fmaf(u[j], u[j], sq); }
+            const float rstd = rsqrtf(row_sum(sq) * inv_d + a.eps);
 #pragma unroll
-            for (int j = 0; j < CPT; ++j) u[j] *= rstd;  // y
+            for (int j = 0; j < CPT; ++j) u[j] *= rstd;  // y (zero in the padding)
             if (key_rows) {
                 // key rows: e = k + y - v, pu = rstd (e - mean(e) - y mean(e y))
                 float e[CPT];
@@ -499,12 +522,13 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 }
 #pragma unroll
                 for (int j = 0; j < CPT; ++j) { se += e[j]; sey = fmaf(e[j], u[j], sey); }
-                const float me_ = row_sum(se) * (1.0f / D), mey = row_sum(sey) * (1.0f / D);
+                const float me_ = real ? row_sum(se) * inv_d : (row_sum(se), 0.0f);
+                const float mey = row_sum(sey) * inv_d;
                     // broadcast the bf16 pu row piece to every CTA of the cluster
                 uint32_t pk[CPT / 2];
 #pragma unroll
                 for (int j = 0; j < CPT; j += 2)
-                    pk[j / 2] = pack_bf16(rstd * (e[j] - me_ - u[j] * mey), rstd * (e[j + 1] - me_ - u[j + 1] * mey));
+                    pk[j / 2] = pack_bf16(rstd * (e[j] - me_ - u[j] * mey), rstd * (e[j + 1] - me_ - u[j + 1] * mey));  // 0 in the padding
                 const uint32_t pu_local = smem_u32(s.Pu[col0 >> 6]);
 #pragma unroll
                 for (uint32_t dst = 0; dst < NC; ++dst) {
@@ -529,7 +553,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                         const float2 qf = __bfloat1622float2(q2[x]);
                         o32[x] = pack_bf16(qf.x + u[8 * ch + 2 * x], qf.y + u[8 * ch + 2 * x + 1]);
                     }
-                    *reinterpret_cast<uint4*>(go + off + 8 * ch) = ov;
+                    if (real) *reinterpret_cast<uint4*>(go + off + 8 * ch) = ov;
                 }
             }
         };
@@ -626,19 +650,14 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         const bool last = (r + 1 == nchunks);
         const float cm = sc.cm, cb = sc.cb;
         const float cwn = last ? 1.0f : s.sc[(r + 1) & 1].cw;
-        const size_t head = (size_t)seq * (size_t)(D * 4 * HC);
+        const size_t head = (size_t)seq * dh;
 
         mbar_wait(&s.bar_agg, ph, wc, 100 + 8);
         PROF(10);
         tc_fence_after_sync();
         if (is_issuer && !last) {
             // the W1 aggregations were the last readers of the key tile: the next chunk's tokens may land in X
-            mbar_expect_tx(&s.bar_x, 32768);
-            const int y = seq * L + tok0 + C;
-            tma_load_2d(s.X[0], &tmK, 0, y, &s.bar_x);
-            tma_load_2d(s.X[1], &tmK, 64, y, &s.bar_x);
-            tma_load_2d(s.X[0] + 8192, &tmQ, 0, y, &s.bar_x);
-            tma_load_2d(s.X[1] + 8192, &tmQ, 64, y, &s.bar_x);
+            load_tokens(seq * L + tok0 + C);
         }
         __syncwarp();
         // ---------------- state pass, W1 half (Algorithm 1 lines 6-7), while the M2 aggregation still runs
@@ -659,11 +678,11 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             }
             tmem_st16(lane_addr + T_W1 + col, st);
             st_slab16(s.W1[col >> 6], row, col & 63, wn);
-            if (last || a.ckpt) {  // final state, or the next chunk's start state for the backward
-                const size_t off = ((size_t)(HC * me) + row) * D + col;
-                float* ck = last ? nullptr : a.ckpt + (size_t)seq * a.ckpt_seq_stride + (size_t)(r + 1) * 4 * (size_t)(D * 4 * HC);
+            if ((last || a.ckpt) && cta_real && col < de) {  // final state, or the next chunk's start state for the backward
+                const size_t off = ((size_t)(HC * me) + row) * de + col;
+                float* ck = last ? nullptr : a.ckpt + (size_t)seq * a.ckpt_seq_stride + (size_t)(r + 1) * 4 * dh;
                 float* wf = last ? a.W1_final + head + off : ck + off;
-                float* mf = last ? a.M1_final + head + off : ck + 2 * (size_t)(D * 4 * HC) + off;
+                float* mf = last ? a.M1_final + head + off : ck + 2 * dh + off;
 #pragma unroll
                 for (int j = 0; j < 16; j += 4) {
                     *reinterpret_cast<float4*>(wf + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
@@ -708,11 +727,11 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             }
             tmem_st16(lane_addr + T_W2 + col, st);
             st_slab16(s.W2[col >> 6], row, col & 63, wn);
-            if (last || a.ckpt) {
-                const size_t off = (size_t)row * (4 * HC) + HC * me + col;
-                float* ck = last ? nullptr : a.ckpt + (size_t)seq * a.ckpt_seq_stride + (size_t)(r + 1) * 4 * (size_t)(D * 4 * HC);
-                float* wf = last ? a.W2_final + head + off : ck + (size_t)(D * 4 * HC) + off;
-                float* mf = last ? a.M2_final + head + off : ck + 3 * (size_t)(D * 4 * HC) + off;
+            if ((last || a.ckpt) && cta_real && row < de) {
+                const size_t off = (size_t)row * he + HC * me + col;
+                float* ck = last ? nullptr : a.ckpt + (size_t)seq * a.ckpt_seq_stride + (size_t)(r + 1) * 4 * dh;
+                float* wf = last ? a.W2_final + head + off : ck + dh + off;
+                float* mf = last ? a.M2_final + head + off : ck + 3 * dh + off;
 #pragma unroll
                 for (int j = 0; j < 16; j += 4) {
                     *reinterpret_cast<float4*>(wf + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
@@ -754,12 +773,12 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// [rows][128] bf16 row-major, tiles of box_rows rows x 64 columns, 128-byte swizzle
-bool make_token_map(CUtensorMap* tm, const void* base, size_t rows, unsigned box_rows) {
+// [rows][d] bf16 row-major, tiles of box_rows rows x 64 columns, 128-byte swizzle
+bool make_token_map(CUtensorMap* tm, const void* base, size_t rows, unsigned box_rows, int d) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)D * 2};
+    cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)d * 2};
     cuuint32_t box[2] = {64, box_rows};
     cuuint32_t es[2] = {1, 1};
     return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
@@ -781,14 +800,16 @@ int tc_fwd_launch(const TcFwdArgs& a, void* stream) {
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     CUtensorMap tmK, tmQ, tmV;
     const size_t rows = (size_t)a.N * a.L;
-    if (!make_token_map(&tmK, a.k, rows, 64) || !make_token_map(&tmQ, a.q, rows, 64) || !make_token_map(&tmV, a.v, rows, 16))
+    if (!make_token_map(&tmK, a.k, rows, 64, a.d) || !make_token_map(&tmQ, a.q, rows, 64, a.d) ||
+        !make_token_map(&tmV, a.v, rows, 16, a.d))
         return (int)cudaErrorInvalidValue;
     static bool attr_done[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return (int)cudaGetLastError();
     const int smem = (int)tc_fwd_smem_bytes();
     if (dev < 0 || dev >= 64 || !attr_done[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        cudaError_t e = cudaFuncSetAttribute(tc_fwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_fwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return (int)e;
         if (dev >= 0 && dev < 64) attr_done[dev] = true;
     }
@@ -806,7 +827,9 @@ int tc_fwd_launch(const TcFwdArgs& a, void* stream) {
     at[0].val.clusterDim.z = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    e = cudaLaunchKernelEx(&cfg, tc_fwd_kernel, tmK, tmQ, tmV, a);
+    const bool native = a.d == D && a.h == NC * HC;
+    e = native ? cudaLaunchKernelEx(&cfg, tc_fwd_kernel<false>, tmK, tmQ, tmV, a)
+               : cudaLaunchKernelEx(&cfg, tc_fwd_kernel<true>, tmK, tmQ, tmV, a);
     if (e != cudaSuccess) return (int)e;
     return (int)cudaGetLastError();
 }

@@ -11,6 +11,8 @@ namespace e2ttt {
 
 struct TcFwdArgs {
     int N, L;  // sequences, tokens per sequence (L a multiple of 64)
+    int d, h;  // head dimension (64 or 128) and hidden width (a multiple of 128, at most 512): smaller shapes run
+               // zero-padded inside the 128 x 512 tiles the kernel is built for
     float eps;
     const __nv_bfloat16 *q, *k, *v;
     const float *eta, *beta, *gamma;

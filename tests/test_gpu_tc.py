@@ -100,3 +100,42 @@ def test_tc_forward_saves_states_for_the_backward():
     b = util.gpu_backward(x2, d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16", via_saved_states=False)
     for n in ("dq", "dk", "dv", "deta", "dbeta", "dgamma"):
         assert util.rel_err(a[n], b[n]) <= 3 * TOL_BF16, n   # saved (tensor-core) vs recomputed (SIMT) forward states
+
+
+# ---- smaller shapes run zero-padded inside the same 128 x 512 tiles (d = 64, h a multiple of 128)
+
+@pytest.mark.parametrize("d,h", [(64, 256), (64, 128), (128, 384), (64, 512)])
+def test_tc_padded_shapes_windows(d, h):
+    r = inputs.config(1, heads=[1, 50], m_std=0.002, d=d, h=h)
+    shape = dict(d=d, h=h, C=64, kind=MLP, io="bf16")
+    xw, ref = util.teacher_forced_windows(r, 4, window=1)
+    tc, hd = util.gpu_forward(xw, impl=E.E2TTT_IMPL_TCGEN05, **shape)
+    assert hd["ws"].numel() == 256
+    assert E.e2ttt_device_status(hd["ws"]) == 0
+    errs = check_forward(tc, ref, TOL_BF16, f"tc padded d={d} h={h}")
+    print(d, h, errs)
+
+
+def test_tc_padded_free_running_paper_regime_and_auto_selection():
+    r = inputs.paper_regime(inputs.Recipe(B=3, H=1, L=1024, d=64, h=256, C=64, kind=MLP, io="bf16", seed=6, m_std=0.002))
+    x = inputs.generate(r)
+    ref = util.oracle_forward(x, 64, MLP)
+    shape = dict(d=64, h=256, C=64, kind=MLP, io="bf16")
+    tc, hd = util.gpu_forward(x, **shape)               # impl left to the library: it must pick the tensor-core path
+    assert hd["ws"].numel() == 256
+    assert E.e2ttt_device_status(hd["ws"]) == 0
+    check_forward(tc, ref, TOL_BF16, "tc padded paper regime, 16 chunks free-running")
+
+
+def test_tc_padded_saved_states_feed_the_backward():
+    from tests.test_gpu_parity import check_backward
+    r = inputs.config(1, heads=[4, 77])
+    xw, _ = util.teacher_forced_windows(r, 3, window=2, with_grads=True)
+    ref_free = util.gpu_backward(xw, d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16", via_saved_states=False)
+    got = util.gpu_backward(xw, d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16", via_saved_states=True)
+    for n in ("dq", "dk", "dv", "deta", "dbeta", "dgamma"):
+        assert util.rel_err(got[n], ref_free[n]) <= 3 * TOL_BF16, n
+    x1, _ = util.teacher_forced_windows(r, 3, window=1, with_grads=True)
+    ref = util.oracle_backward(x1, r.C, r.kind)
+    got1 = util.gpu_backward(x1, d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16", via_saved_states=True)
+    check_backward(got1, ref, TOL_BF16, "padded bwd from tensor-core saved states")
