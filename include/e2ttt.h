@@ -60,14 +60,19 @@ typedef enum { E2TTT_MLP_GELU = 0, E2TTT_SWIGLU = 1 } e2ttt_kind;
 typedef enum { E2TTT_F32 = 0, E2TTT_BF16 = 1 } e2ttt_dtype;
 
 /* Which kernel family serves the call.
- *   AUTO    : the tensor-core path where it serves (kind, io_dtype, d, h, C), else the SIMT path.
- *             Served today: GELU-MLP, bf16 I/O, C = 64, L a multiple of 64, d in {64, 128},
+ *   AUTO    : TCGEN05 where it serves (kind, io_dtype, d, h, C); else TILED for bf16 I/O and SIMT for
+ *             fp32 I/O.  The backward has no fused kernel: AUTO and TCGEN05 mean TILED there.
+ *             TCGEN05 serves today: GELU-MLP, bf16 I/O, C = 64, L a multiple of 64, d in {64, 128},
  *             h in {128, 256, 384, 512} (shapes below 128 x 512 run zero-padded in the same tiles).
  *   SIMT    : plain CUDA-core kernels for any shape.  With fp32 I/O they compute in fp64
  *             internally; with bf16 I/O in fp32.
- *   TCGEN05 : bf16 operands on the 5th-generation tensor cores with fp32 accumulation in tensor
- *             memory; E2TTT_ERR_SHAPE if no specialisation matches. */
-typedef enum { E2TTT_IMPL_AUTO = 0, E2TTT_IMPL_SIMT = 1, E2TTT_IMPL_TCGEN05 = 2 } e2ttt_impl;
+ *   TCGEN05 : the fused kernel: bf16 operands on the 5th-generation tensor cores, fp32 accumulation
+ *             and the fp32 state in tensor memory for the whole sequence; E2TTT_ERR_SHAPE if it
+ *             does not serve the shape.
+ *   TILED   : the any-shape kernels of SIMT with every matrix product on the 5th-generation tensor
+ *             cores (operands rounded to bf16, fp32 accumulation); intermediates and state stay
+ *             fp32 in the workspace.  bf16 I/O only (E2TTT_ERR_SHAPE otherwise). */
+typedef enum { E2TTT_IMPL_AUTO = 0, E2TTT_IMPL_SIMT = 1, E2TTT_IMPL_TCGEN05 = 2, E2TTT_IMPL_TILED = 3 } e2ttt_impl;
 
 typedef enum {
     E2TTT_OK = 0,

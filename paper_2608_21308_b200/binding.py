@@ -17,7 +17,7 @@ LIB_PATH = os.environ.get("E2TTT_LIB") or os.path.join(_HERE, "lib", "libe2ttt.s
 
 E2TTT_MLP_GELU, E2TTT_SWIGLU = 0, 1
 E2TTT_F32, E2TTT_BF16 = 0, 1
-E2TTT_IMPL_AUTO, E2TTT_IMPL_SIMT, E2TTT_IMPL_TCGEN05 = 0, 1, 2
+E2TTT_IMPL_AUTO, E2TTT_IMPL_SIMT, E2TTT_IMPL_TCGEN05, E2TTT_IMPL_TILED = 0, 1, 2, 3
 E2TTT_OK = 0
 
 

@@ -19,7 +19,9 @@ int check_params(const e2ttt_params* p) {
     if (!p) return E2TTT_ERR_NULL;
     if (p->kind != E2TTT_MLP_GELU && p->kind != E2TTT_SWIGLU) return E2TTT_ERR_SHAPE;
     if (p->io_dtype != E2TTT_F32 && p->io_dtype != E2TTT_BF16) return E2TTT_ERR_DTYPE;
-    if (p->impl != E2TTT_IMPL_AUTO && p->impl != E2TTT_IMPL_SIMT && p->impl != E2TTT_IMPL_TCGEN05) return E2TTT_ERR_DTYPE;
+    if (p->impl != E2TTT_IMPL_AUTO && p->impl != E2TTT_IMPL_SIMT && p->impl != E2TTT_IMPL_TCGEN05 &&
+        p->impl != E2TTT_IMPL_TILED)
+        return E2TTT_ERR_DTYPE;
     if (p->B <= 0 || p->H <= 0 || p->L <= 0 || p->d <= 0 || p->h <= 0 || p->C <= 0) return E2TTT_ERR_SHAPE;
     if (p->C > kMaxChunk || p->d > kMaxD || p->h > kMaxH) return E2TTT_ERR_SHAPE;
     if ((int64_t)p->B * p->H > (int64_t)1 << 24) return E2TTT_ERR_SHAPE;
@@ -41,8 +43,12 @@ int pick_impl(const e2ttt_params* p, bool save_states, int* impl) {
     if (p->impl == E2TTT_IMPL_TCGEN05) {
         if (!has_tcgen05(p, save_states)) return E2TTT_ERR_SHAPE;
         *impl = E2TTT_IMPL_TCGEN05;
+    } else if (p->impl == E2TTT_IMPL_TILED) {
+        if (p->io_dtype != E2TTT_BF16) return E2TTT_ERR_SHAPE;
+        *impl = E2TTT_IMPL_TILED;
     } else if (p->impl == E2TTT_IMPL_AUTO) {
-        *impl = has_tcgen05(p, save_states) ? E2TTT_IMPL_TCGEN05 : E2TTT_IMPL_SIMT;
+        *impl = has_tcgen05(p, save_states) ? E2TTT_IMPL_TCGEN05
+                                            : (p->io_dtype == E2TTT_BF16 ? E2TTT_IMPL_TILED : E2TTT_IMPL_SIMT);
     } else {
         *impl = E2TTT_IMPL_SIMT;
     }
@@ -98,8 +104,8 @@ int e2ttt_workspace_bytes(const e2ttt_params* p, int save_states, size_t* bytes)
     int impl = 0;
     rc = pick_impl(p, save_states != 0, &impl);
     if (rc) return rc;
-    // tensor-core path: all state lives on chip, only the status block is needed.
-    // SIMT path: with saved states the same buffer serves the backward, which needs the larger layout.
+    // fused tensor-core path: all state lives on chip, only the status block is needed.
+    // any-shape kernels: with saved states the same buffer serves the backward, which needs the larger layout.
     *bytes = (impl == E2TTT_IMPL_TCGEN05 && !save_states) ? kStatusBytes : simt_bytes(p, save_states != 0, save_states != 0);
     return E2TTT_OK;
 }
@@ -154,6 +160,8 @@ int e2ttt_chunk_fwd(const e2ttt_params* p, const void* q, const void* k, const v
     a.N = p->B * p->H; a.L = p->L; a.d = p->d; a.h = p->h; a.C = p->C;
     a.nchunks = (p->L + p->C - 1) / p->C;
     a.cl = simt_cluster_size(a.N);
+    a.tc = impl == E2TTT_IMPL_TILED;
+    a.status = static_cast<int*>(workspace);
     a.save_states = save_states != 0;
     a.eps = p->ln_eps;
     a.q = q; a.k = k; a.v = v; a.eta = eta; a.beta = beta; a.gamma = gamma; a.o = o;
@@ -212,6 +220,7 @@ int e2ttt_chunk_bwd(const e2ttt_params* p, const void* q, const void* k, const v
         SimtFwdArgs f{};
         f.N = p->B * p->H; f.L = p->L; f.d = p->d; f.h = p->h; f.C = p->C; f.nchunks = nchunks;
         f.save_states = 1; f.eps = p->ln_eps; f.cl = simt_cluster_size(f.N);
+        f.tc = impl != E2TTT_IMPL_SIMT; f.status = static_cast<int*>(workspace);
         f.q = q; f.k = k; f.v = v; f.eta = eta; f.beta = beta; f.gamma = gamma; f.ws = ws_data; f.lay = lay;
         f.o = nullptr; // outputs are not needed
         for (int i = 0; i < nmat; ++i) {
@@ -225,6 +234,7 @@ int e2ttt_chunk_bwd(const e2ttt_params* p, const void* q, const void* k, const v
     SimtBwdArgs b{};
     b.N = p->B * p->H; b.L = p->L; b.d = p->d; b.h = p->h; b.C = p->C; b.nchunks = nchunks; b.eps = p->ln_eps;
     b.cl = simt_cluster_size(b.N);
+    b.tc = impl != E2TTT_IMPL_SIMT; b.status = static_cast<int*>(workspace);
     b.q = q; b.k = k; b.v = v; b.d_o = d_o; b.eta = eta; b.beta = beta; b.gamma = gamma;
     b.dq = dq; b.dk = dk; b.dv = dv; b.d_eta = d_eta; b.d_beta = d_beta; b.d_gamma = d_gamma;
     b.ws = ws_data; b.lay = lay;

@@ -9,8 +9,11 @@
 // [d x h] (W2 of the GELU MLP, W3 of SwiGLU); the first matrices are [h x d].
 //   GELU MLP : hidden a = gelu(z1)                 pz1 = ph gelu'(z1)
 //   SwiGLU   : hidden a = silu(z1) z2              pz1 = ph z2 silu'(z1),  pz2 = ph silu(z1)
+#include <type_traits>
+
 #include "simt_common.cuh"
 #include "simt_layout.h"
+#include "tc_gemm.cuh"
 
 namespace e2ttt {
 
@@ -30,20 +33,25 @@ __device__ __forceinline__ void warp_ln_jac(const Real* x, const Real* y, Real r
     for (int i = lane; i < d; i += 32) out[i] = r * (x[i] - sx - y[i] * sxy);
 }
 
-template <typename Real, typename IO, int KIND>
-__global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArgs a) {
+// TC = true (bf16 I/O only): every GEMM runs on the tensor cores with bf16 operands; everything else is unchanged.
+template <typename Real, typename IO, int KIND, bool TC>
+__global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_kernel(const SimtBwdArgs a) {
     constexpr int NMAT = (KIND == 0) ? 2 : 3;
     constexpr int LAST = NMAT - 1;
     constexpr bool SW = (KIND == 1);
+    using Engine = typename std::conditional<TC, TcGemm, FmaGemm<Real>>::type;
+    constexpr int NT = Engine::kThreads;  // threads per CTA
     extern __shared__ __align__(16) unsigned char simt_smem_raw[];
-    GemmSmem<Real>& gsm = *reinterpret_cast<GemmSmem<Real>*>(simt_smem_raw);
-    ChunkScalars<Real>& sc = *reinterpret_cast<ChunkScalars<Real>*>(simt_smem_raw + sizeof(GemmSmem<Real>));
-    Real* red = reinterpret_cast<Real*>(simt_smem_raw + sizeof(GemmSmem<Real>) + sizeof(ChunkScalars<Real>));
+    unsigned char* smem_base = Engine::align(simt_smem_raw);
+    ChunkScalars<Real>& sc = *reinterpret_cast<ChunkScalars<Real>*>(smem_base + Engine::kBytes);
+    Real* red = reinterpret_cast<Real*>(smem_base + Engine::kBytes + sizeof(ChunkScalars<Real>));
 
     const int CL = a.cl;                 // CTAs working on this sequence (one cluster)
     const int seq = blockIdx.x / CL, rank = blockIdx.x % CL;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    constexpr int NW = kSimtThreads / 32;
+    constexpr int NW = NT / 32;
+    Engine G;
+    G.setup(smem_base, a.status, rank, CL);
     const int d = a.d, h = a.h, C = a.C, L = a.L;
     const size_t dh = (size_t)d * h;
     const SimtLayout& lay = a.lay;
@@ -69,7 +77,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
         T[i] = ws + lay.T[i]; S[i] = ws + lay.S[i]; Wb[i] = ws + lay.Wb[i];
         const float* tf = a.dW_final[i] ? a.dW_final[i] + (size_t)seq * dh : nullptr;
         const float* sf = a.dM_final[i] ? a.dM_final[i] + (size_t)seq * dh : nullptr;
-        for (size_t e = tid + (size_t)rank * kSimtThreads; e < dh; e += (size_t)kSimtThreads * CL) {
+        for (size_t e = tid + (size_t)rank * NT; e < dh; e += (size_t)NT * CL) {
             T[i][e] = tf ? (Real)tf[e] : (Real)0;
             S[i][e] = sf ? (Real)sf[e] : (Real)0;
         }
@@ -122,7 +130,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
         if (warp == 0) chunk_scalars_warp<Real>(eta + s, beta + s, gamma + s, len, &sc);
 #pragma unroll
         for (int i = 0; i < NMAT; ++i)
-            for (size_t e = tid + (size_t)rank * kSimtThreads; e < dh; e += (size_t)kSimtThreads * CL) Wb[i][e] = 0;
+            for (size_t e = tid + (size_t)rank * NT; e < dh; e += (size_t)NT * CL) Wb[i][e] = 0;
 
         auto load_x = [&](int m, int kk, Real& a0, Real& a1) {
             a0 = (m < len) ? ld_io<Real>(kc, (size_t)m * d + kk) : ld_io<Real>(qc, (size_t)(m - len) * d + kk);
@@ -130,28 +138,26 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
         auto load_k = [&](int m, int kk, Real& a0, Real& a1) { a0 = ld_io<Real>(kc, (size_t)m * d + kk); };
 
         // ---------------- forward of the chunk, recomputed ----------------
-        block_gemm<Real, 1, true, true>(
+        G.template run<1, true, true>(
             2 * len, h, d, load_x, [&](int n, int kk) { return W1[(size_t)n * d + kk]; },
             [&](int m, int n, Real acc, Real) {
                 Z1[(size_t)m * h + n] = acc;
                 if (!SW) A[(size_t)m * h + n] = gelu_f(acc);
-            },
-            &gsm, rank, CL);
+            });
         if (SW) {
-            block_gemm<Real, 1, true, true>(
+            G.template run<1, true, true>(
                 2 * len, h, d, load_x, [&](int n, int kk) { return W2[(size_t)n * d + kk]; },
                 [&](int m, int n, Real acc, Real) {
                     const size_t e = (size_t)m * h + n;
                     Z2[e] = acc;
                     A[e] = silu_f(Z1[e]) * acc;
-                },
-                &gsm, rank, CL);
+                });
         }
-        block_gemm<Real, 1, true, true>(
+        G.template run<1, true, true>(
             2 * len, d, h, [&](int m, int kk, Real& a0, Real& a1) { a0 = A[(size_t)m * h + kk]; },
             [&](int n, int kk) { return Wl[(size_t)n * h + kk]; },
-            [&](int m, int n, Real acc, Real) { U[(size_t)m * d + n] = acc; }, &gsm, rank, CL);
-        for (int m = warp + rank * (kSimtThreads / 32); m < 2 * len; m += (kSimtThreads / 32) * CL) {
+            [&](int m, int n, Real acc, Real) { U[(size_t)m * d + n] = acc; });
+        for (int m = warp + rank * (NT / 32); m < 2 * len; m += (NT / 32) * CL) {
             Real* u = U + (size_t)m * d;
             const Real r = warp_layernorm(u, u, d, eps);
             if (m >= len) {
@@ -177,7 +183,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
             }
         }
         phase_sync(CL);
-        block_gemm<Real, 1, true, false>(
+        G.template run<1, true, false>(
             len, h, d, [&](int m, int kk, Real& a0, Real& a1) { a0 = Pu[(size_t)m * d + kk]; },
             [&](int n, int kk) { return Wl[(size_t)kk * h + n]; },
             [&](int m, int n, Real acc, Real) {
@@ -189,14 +195,13 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
                     Pz1[e] = acc * Z2[e] * silu_d1(Z1[e]);
                     Pz2[e] = acc * silu_f(Z1[e]);
                 }
-            },
-            &gsm, rank, CL);
+            });
 
         // ---------------- (i) outputs o = q + LN(Wl a(q)) ----------------
         const Real* Z1q = Z1 + (size_t)len * h;
         const Real* Z2q = Z2 + (size_t)len * h;
         const Real* Aq = A + (size_t)len * h;
-        block_gemm<Real, 1, true, false>(
+        G.template run<1, true, false>(
             len, h, d, [&](int m, int kk, Real& a0, Real& a1) { a0 = Uqb[(size_t)m * d + kk]; },
             [&](int n, int kk) { return Wl[(size_t)kk * h + n]; },
             [&](int m, int n, Real acc, Real) {
@@ -207,9 +212,8 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
                     Zqb[e] = acc * Z2q[e] * silu_d1(Z1q[e]);
                     Zqb2[e] = acc * silu_f(Z1q[e]);
                 }
-            },
-            &gsm, rank, CL);
-        block_gemm<Real, 1, true, false>(
+            });
+        G.template run<1, true, false>(
             len, d, SW ? 2 * h : h,
             [&](int m, int kk, Real& a0, Real& a1) {
                 a0 = kk < h ? Zqb[(size_t)m * h + kk] : Zqb2[(size_t)m * h + kk - h];
@@ -218,21 +222,20 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
             [&](int m, int n, Real acc, Real) {
                 const size_t e = (size_t)m * d + n;
                 st_io(dq + (size_t)s * d, e, ld_io<Real>(doc, e) + acc);
-            },
-            &gsm, rank, CL);
-        block_gemm<Real, 1, false, false>( // Wbl += Uqb^T Aq
+            });
+        G.template run<1, false, false>( // Wbl += Uqb^T Aq
             d, h, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Uqb[(size_t)t * d + m]; },
             [&](int n, int t) { return Aq[(size_t)t * h + n]; },
-            [&](int m, int n, Real acc, Real) { Wb[LAST][(size_t)m * h + n] += acc; }, &gsm, rank, CL);
-        block_gemm<Real, 1, false, false>( // Wb1 += Zqb^T Q
+            [&](int m, int n, Real acc, Real) { Wb[LAST][(size_t)m * h + n] += acc; });
+        G.template run<1, false, false>( // Wb1 += Zqb^T Q
             h, d, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Zqb[(size_t)t * h + m]; },
             [&](int n, int t) { return ld_io<Real>(qc, (size_t)t * d + n); },
-            [&](int m, int n, Real acc, Real) { Wb[0][(size_t)m * d + n] += acc; }, &gsm, rank, CL);
+            [&](int m, int n, Real acc, Real) { Wb[0][(size_t)m * d + n] += acc; });
         if (SW)
-            block_gemm<Real, 1, false, false>( // Wb2 += Zqb2^T Q
+            G.template run<1, false, false>( // Wb2 += Zqb2^T Q
                 h, d, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Zqb2[(size_t)t * h + m]; },
                 [&](int n, int t) { return ld_io<Real>(qc, (size_t)t * d + n); },
-                [&](int m, int n, Real acc, Real) { Wb[1][(size_t)m * d + n] += acc; }, &gsm, rank, CL);
+                [&](int m, int n, Real acc, Real) { Wb[1][(size_t)m * d + n] += acc; });
 
         // ---------------- (ii) state transition: carries ----------------
         Real cwb, cmb, cbb;
@@ -241,7 +244,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
 #pragma unroll
             for (int i = 0; i < NMAT; ++i) {
                 const Real* Wi = ck + (size_t)i * dh;
-                for (size_t e = tid; e < dh; e += kSimtThreads) {  // every CTA sums everything: same value everywhere
+                for (size_t e = tid; e < dh; e += NT) {  // every CTA sums everything: same value everywhere
                     pw += T[i][e] * Wi[e];
                     pm += T[i][e] * M0[i][e];
                     pb += S[i][e] * M0[i][e];
@@ -252,20 +255,20 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
             cbb = block_sum(pb, red);
         }
         // G_t enters W_C with K^W_t and M_C with K^M_t: its adjoint is K^W_t T + K^M_t S.
-        block_gemm<Real, 1, true, true>( // XY2 = Ak [Tl; Sl]^T
+        G.template run<1, true, true>( // XY2 = Ak [Tl; Sl]^T
             len, 2 * d, h, [&](int m, int kk, Real& a0, Real& a1) { a0 = A[(size_t)m * h + kk]; },
             [&](int n, int kk) { return n < d ? T[LAST][(size_t)n * h + kk] : S[LAST][(size_t)(n - d) * h + kk]; },
-            [&](int m, int n, Real acc, Real) { XY2[(size_t)m * 2 * d + n] = acc; }, &gsm, rank, CL);
-        block_gemm<Real, 1, true, true>( // XY1 = K [T1; S1]^T
+            [&](int m, int n, Real acc, Real) { XY2[(size_t)m * 2 * d + n] = acc; });
+        G.template run<1, true, true>( // XY1 = K [T1; S1]^T
             len, 2 * h, d, load_k,
             [&](int n, int kk) { return n < h ? T[0][(size_t)n * d + kk] : S[0][(size_t)(n - h) * d + kk]; },
-            [&](int m, int n, Real acc, Real) { XY1[(size_t)m * 2 * h + n] = acc; }, &gsm, rank, CL);
+            [&](int m, int n, Real acc, Real) { XY1[(size_t)m * 2 * h + n] = acc; });
         if (SW)
-            block_gemm<Real, 1, true, true>( // XY1b = K [T2; S2]^T
+            G.template run<1, true, true>( // XY1b = K [T2; S2]^T
                 len, 2 * h, d, load_k,
                 [&](int n, int kk) { return n < h ? T[1][(size_t)n * d + kk] : S[1][(size_t)(n - h) * d + kk]; },
-                [&](int m, int n, Real acc, Real) { XY1b[(size_t)m * 2 * h + n] = acc; }, &gsm, rank, CL);
-        for (int t = warp + rank * (kSimtThreads / 32); t < len; t += (kSimtThreads / 32) * CL) {
+                [&](int m, int n, Real acc, Real) { XY1b[(size_t)m * 2 * h + n] = acc; });
+        for (int t = warp + rank * (NT / 32); t < len; t += (NT / 32) * CL) {
             const Real* x2 = XY2 + (size_t)t * 2 * d;
             const Real* x1 = XY1 + (size_t)t * 2 * h;
             const Real* x1b = XY1b + (size_t)t * 2 * h;
@@ -293,30 +296,30 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
         }
         phase_sync(CL);
         // ---------------- (iii) per-token gradients G_t = -(pz1 k^T, [pz2 k^T,] pu a^T) ----------------
-        block_gemm<Real, 1, true, false>( // Akb = -[kW Pu | kM Pu] [Tl; Sl]
+        G.template run<1, true, false>( // Akb = -[kW Pu | kM Pu] [Tl; Sl]
             len, h, 2 * d,
             [&](int m, int kk, Real& a0, Real& a1) {
                 a0 = kk < d ? sc.kW[m] * Pu[(size_t)m * d + kk] : sc.kM[m] * Pu[(size_t)m * d + kk - d];
             },
             [&](int n, int kk) { return kk < d ? T[LAST][(size_t)kk * h + n] : S[LAST][(size_t)(kk - d) * h + n]; },
-            [&](int m, int n, Real acc, Real) { Akb[(size_t)m * h + n] = -acc; }, &gsm, rank, CL);
-        block_gemm<Real, 1, true, false>( // Kb = -[kW Pz1 | kM Pz1] [T1; S1]
+            [&](int m, int n, Real acc, Real) { Akb[(size_t)m * h + n] = -acc; });
+        G.template run<1, true, false>( // Kb = -[kW Pz1 | kM Pz1] [T1; S1]
             len, d, 2 * h,
             [&](int m, int kk, Real& a0, Real& a1) {
                 a0 = kk < h ? sc.kW[m] * Pz1[(size_t)m * h + kk] : sc.kM[m] * Pz1[(size_t)m * h + kk - h];
             },
             [&](int n, int kk) { return kk < h ? T[0][(size_t)kk * d + n] : S[0][(size_t)(kk - h) * d + n]; },
-            [&](int m, int n, Real acc, Real) { Kb[(size_t)m * d + n] = -acc; }, &gsm, rank, CL);
+            [&](int m, int n, Real acc, Real) { Kb[(size_t)m * d + n] = -acc; });
         if (SW)
-            block_gemm<Real, 1, true, false>( // Kb -= [kW Pz2 | kM Pz2] [T2; S2]
+            G.template run<1, true, false>( // Kb -= [kW Pz2 | kM Pz2] [T2; S2]
                 len, d, 2 * h,
                 [&](int m, int kk, Real& a0, Real& a1) {
                     a0 = kk < h ? sc.kW[m] * Pz2[(size_t)m * h + kk] : sc.kM[m] * Pz2[(size_t)m * h + kk - h];
                 },
                 [&](int n, int kk) { return kk < h ? T[1][(size_t)kk * d + n] : S[1][(size_t)(kk - h) * d + n]; },
-                [&](int m, int n, Real acc, Real) { Kb[(size_t)m * d + n] -= acc; }, &gsm, rank, CL);
+                [&](int m, int n, Real acc, Real) { Kb[(size_t)m * d + n] -= acc; });
         // back through pz: Pzb becomes the adjoint of ph; Zkb (Zkb2) start with the second-order terms
-        for (size_t e = tid + (size_t)rank * kSimtThreads; e < (size_t)len * h; e += (size_t)kSimtThreads * CL) {
+        for (size_t e = tid + (size_t)rank * NT; e < (size_t)len * h; e += (size_t)NT * CL) {
             const Real z1 = Z1[e], ph = Pa[e];
             if (!SW) {
                 const Real pzb = Pzb[e];
@@ -332,16 +335,16 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
         phase_sync(CL);
         const Real* Phb = Pzb;
         // ph = Wl^T pu
-        block_gemm<Real, 1, true, true>(
+        G.template run<1, true, true>(
             len, d, h, [&](int m, int kk, Real& a0, Real& a1) { a0 = Phb[(size_t)m * h + kk]; },
             [&](int n, int kk) { return Wl[(size_t)n * h + kk]; },
-            [&](int m, int n, Real acc, Real) { Pub[(size_t)m * d + n] += acc; }, &gsm, rank, CL);
-        block_gemm<Real, 1, false, false>( // Wbl += Pu^T Phb
+            [&](int m, int n, Real acc, Real) { Pub[(size_t)m * d + n] += acc; });
+        G.template run<1, false, false>( // Wbl += Pu^T Phb
             d, h, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Pu[(size_t)t * d + m]; },
             [&](int n, int t) { return Phb[(size_t)t * h + n]; },
-            [&](int m, int n, Real acc, Real) { Wb[LAST][(size_t)m * h + n] += acc; }, &gsm, rank, CL);
+            [&](int m, int n, Real acc, Real) { Wb[LAST][(size_t)m * h + n] += acc; });
         // pu = J(u) e, e = k + y - v, y = LN(u)
-        for (int t = warp + rank * (kSimtThreads / 32); t < len; t += (kSimtThreads / 32) * CL) {
+        for (int t = warp + rank * (NT / 32); t < len; t += (NT / 32) * CL) {
             const size_t row = (size_t)t * d;
             const Real* y = U + row;
             const Real r = rk[t];
@@ -367,7 +370,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
         }
         phase_sync(CL);
         // u = Wl a ; a = gelu(z1)  or  silu(z1) z2
-        block_gemm<Real, 1, true, false>(
+        G.template run<1, true, false>(
             len, h, d, [&](int m, int kk, Real& a0, Real& a1) { a0 = Ukb[(size_t)m * d + kk]; },
             [&](int n, int kk) { return Wl[(size_t)kk * h + n]; },
             [&](int m, int n, Real acc, Real) {
@@ -379,14 +382,13 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
                     Zkb[e] += ab * Z2[e] * silu_d1(Z1[e]);
                     Zkb2[e] += ab * silu_f(Z1[e]);
                 }
-            },
-            &gsm, rank, CL);
-        block_gemm<Real, 1, false, false>( // Wbl += Ukb^T Ak
+            });
+        G.template run<1, false, false>( // Wbl += Ukb^T Ak
             d, h, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Ukb[(size_t)t * d + m]; },
             [&](int n, int t) { return A[(size_t)t * h + n]; },
-            [&](int m, int n, Real acc, Real) { Wb[LAST][(size_t)m * h + n] += acc; }, &gsm, rank, CL);
+            [&](int m, int n, Real acc, Real) { Wb[LAST][(size_t)m * h + n] += acc; });
         // z1 = W1 k (, z2 = W2 k)
-        block_gemm<Real, 1, true, false>(
+        G.template run<1, true, false>(
             len, d, SW ? 2 * h : h,
             [&](int m, int kk, Real& a0, Real& a1) {
                 a0 = kk < h ? Zkb[(size_t)m * h + kk] : Zkb2[(size_t)m * h + kk - h];
@@ -395,24 +397,23 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
             [&](int m, int n, Real acc, Real) {
                 const size_t e = (size_t)m * d + n;
                 st_io(dk + (size_t)s * d, e, Kb[e] + acc);
-            },
-            &gsm, rank, CL);
-        block_gemm<Real, 1, false, false>( // Wb1 += Zkb^T K
+            });
+        G.template run<1, false, false>( // Wb1 += Zkb^T K
             h, d, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Zkb[(size_t)t * h + m]; },
             [&](int n, int t) { return ld_io<Real>(kc, (size_t)t * d + n); },
-            [&](int m, int n, Real acc, Real) { Wb[0][(size_t)m * d + n] += acc; }, &gsm, rank, CL);
+            [&](int m, int n, Real acc, Real) { Wb[0][(size_t)m * d + n] += acc; });
         if (SW)
-            block_gemm<Real, 1, false, false>( // Wb2 += Zkb2^T K
+            G.template run<1, false, false>( // Wb2 += Zkb2^T K
                 h, d, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Zkb2[(size_t)t * h + m]; },
                 [&](int n, int t) { return ld_io<Real>(kc, (size_t)t * d + n); },
-                [&](int m, int n, Real acc, Real) { Wb[1][(size_t)m * d + n] += acc; }, &gsm, rank, CL);
+                [&](int m, int n, Real acc, Real) { Wb[1][(size_t)m * d + n] += acc; });
 
         // ---------------- adjoints of the chunk-start state ----------------
         {
             const Real cw = sc.cw, cm = sc.cm, cb = sc.cb;
 #pragma unroll
             for (int i = 0; i < NMAT; ++i)
-                for (size_t e = tid + (size_t)rank * kSimtThreads; e < dh; e += (size_t)kSimtThreads * CL) {
+                for (size_t e = tid + (size_t)rank * NT; e < dh; e += (size_t)NT * CL) {
                     const Real t = T[i][e], sv = S[i][e];
                     T[i][e] = cw * t + Wb[i][e];
                     S[i][e] = cm * t + cb * sv;
@@ -452,29 +453,30 @@ __global__ void __launch_bounds__(kSimtThreads) simt_bwd_kernel(const SimtBwdArg
     for (int i = 0; i < NMAT; ++i) {
         float* wf = a.dW_init[i] + (size_t)seq * dh;
         float* mf = a.dM_init[i] + (size_t)seq * dh;
-        for (size_t e = tid + (size_t)rank * kSimtThreads; e < dh; e += (size_t)kSimtThreads * CL) {
+        for (size_t e = tid + (size_t)rank * NT; e < dh; e += (size_t)NT * CL) {
             wf[e] = (float)T[i][e];
             mf[e] = (float)S[i][e];
         }
     }
+    G.teardown();
 }
 
-template <typename Real, typename IO, int KIND>
+template <typename Real, typename IO, int KIND, bool TC>
 static int launch_bwd(const SimtBwdArgs& a, cudaStream_t st) {
-    constexpr size_t smem =
-        sizeof(GemmSmem<Real>) + sizeof(ChunkScalars<Real>) + 8 * sizeof(Real);
+    using Engine = typename std::conditional<TC, TcGemm, FmaGemm<Real>>::type;
+    constexpr size_t smem = Engine::kBytes + sizeof(ChunkScalars<Real>) + 16 * sizeof(Real) + (TC ? 1024 : 0);
     static bool attr_done[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return (int)cudaGetLastError();
     if (dev < 0 || dev >= 64 || !attr_done[dev]) {
         cudaError_t e =
-            cudaFuncSetAttribute(simt_bwd_kernel<Real, IO, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            cudaFuncSetAttribute(simt_bwd_kernel<Real, IO, KIND, TC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return (int)e;
         if (dev >= 0 && dev < 64) attr_done[dev] = true;
     }
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)(a.N * a.cl));
-    cfg.blockDim = dim3(kSimtThreads);
+    cfg.blockDim = dim3(Engine::kThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute at[1];
@@ -484,7 +486,7 @@ static int launch_bwd(const SimtBwdArgs& a, cudaStream_t st) {
     at[0].val.clusterDim.z = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, simt_bwd_kernel<Real, IO, KIND>, a);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, simt_bwd_kernel<Real, IO, KIND, TC>, a);
     if (e != cudaSuccess) return (int)e;
     return (int)cudaGetLastError();
 }
@@ -492,8 +494,10 @@ static int launch_bwd(const SimtBwdArgs& a, cudaStream_t st) {
 int simt_bwd_launch(const SimtBwdArgs& a, int kind, int io_dtype, void* stream) {
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     if (io_dtype == 0)
-        return kind == 0 ? launch_bwd<double, float, 0>(a, st) : launch_bwd<double, float, 1>(a, st);
-    return kind == 0 ? launch_bwd<float, __nv_bfloat16, 0>(a, st) : launch_bwd<float, __nv_bfloat16, 1>(a, st);
+        return kind == 0 ? launch_bwd<double, float, 0, false>(a, st) : launch_bwd<double, float, 1, false>(a, st);
+    if (a.tc)
+        return kind == 0 ? launch_bwd<float, __nv_bfloat16, 0, true>(a, st) : launch_bwd<float, __nv_bfloat16, 1, true>(a, st);
+    return kind == 0 ? launch_bwd<float, __nv_bfloat16, 0, false>(a, st) : launch_bwd<float, __nv_bfloat16, 1, false>(a, st);
 }
 
 }  // namespace e2ttt

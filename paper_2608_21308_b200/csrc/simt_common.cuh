@@ -57,7 +57,7 @@ template <typename Real> __device__ __forceinline__ Real warp_sum(Real v) {
     return v;
 }
 
-// Deterministic CTA-wide sum (fixed tree); every thread gets the result. red: >= 8 Reals of shared memory.
+// Deterministic CTA-wide sum (fixed tree); every thread gets the result. red: >= 16 Reals of shared memory.
 template <typename Real> __device__ Real block_sum(Real v, Real* red) {
     v = warp_sum(v);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -65,8 +65,8 @@ template <typename Real> __device__ Real block_sum(Real v, Real* red) {
     if (lane == 0) red[warp] = v;
     __syncthreads();
     Real s = 0;
-#pragma unroll
-    for (int w = 0; w < kSimtThreads / 32; ++w) s += red[w];
+    const int nw = (int)blockDim.x >> 5;
+    for (int w = 0; w < nw; ++w) s += red[w];
     return s;
 }
 
@@ -149,6 +149,29 @@ __device__ void chunk_scalars_warp(const float* eta, const float* beta, const fl
     }
 }
 
+// ---- elementwise pass with batched loads ---------------------------------------------------------
+// for e = begin, begin + stride, ... < end:  store(e, load(e)).  `load` returns everything element e needs from
+// memory (a value or a small struct), `store` computes and writes.  U loads are issued before the U stores that
+// follow them; written as one loop body, every load would wait for the previous element's store (the compiler must
+// assume they alias) and the pass would take one memory round trip per element.
+template <int U, typename FL, typename FS>
+__device__ __forceinline__ void batched_for(size_t begin, size_t end, size_t stride, FL load, FS store) {
+    using P = decltype(load((size_t)0));
+    for (size_t e0 = begin; e0 < end; e0 += stride * U) {
+        P p[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t e = e0 + (size_t)u * stride;
+            if (e < end) p[u] = load(e);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t e = e0 + (size_t)u * stride;
+            if (e < end) store(e, p[u]);
+        }
+    }
+}
+
 // ---- phase barrier ---------------------------------------------------------------------------------
 // A sequence may be worked on by a cluster of `nranks` CTAs that split every phase (GEMM tiles, rows, elements)
 // and share all intermediates through global memory.  The hardware cluster barrier (release / acquire at cluster
@@ -164,7 +187,8 @@ __device__ __forceinline__ void phase_sync(int nranks) {
 
 // ---- generic CTA GEMM --------------------------------------------------------------------------
 // out(m, n) = sum_k a(m, k) * b(n, k), m < M, n < N, k < K, for NACC (1 or 2) A operands sharing one B.
-//   fa(m, k, a0, a1) writes the A value(s); fb(n, k) returns the B value; epi(m, n, acc0, acc1) consumes a result.
+//   fa(m, k, a0, a1) writes the A value(s); fb(n, k) returns the B value; pre(m, n) loads what a result combines
+//   with; epi(m, n, acc0, acc1, loaded) consumes a result.
 // A_KFAST / B_KFAST say which index is contiguous in memory, so that neighbouring threads read neighbouring words.
 // 64x64 output tiles (dealt round-robin to the `nranks` CTAs of the sequence's cluster), 16-deep k slices through
 // shared memory, 4x4 results per thread.  Ends with phase_sync().
@@ -173,8 +197,8 @@ template <typename Real> struct GemmSmem {
     Real B[kBK][kBN + 4];
 };
 
-template <typename Real, int NACC, bool A_KFAST, bool B_KFAST, typename FA, typename FB, typename FE>
-__device__ void block_gemm(int M, int N, int K, FA fa, FB fb, FE epi, GemmSmem<Real>* sm, int rank, int nranks) {
+template <typename Real, int NACC, bool A_KFAST, bool B_KFAST, typename FA, typename FB, typename FP, typename FE>
+__device__ void block_gemm(int M, int N, int K, FA fa, FB fb, FP pre, FE epi, GemmSmem<Real>* sm, int rank, int nranks) {
     const int tid = threadIdx.x;
     const int tx = tid & 15, ty = tid >> 4;
     int tile = 0;
@@ -226,12 +250,22 @@ __device__ void block_gemm(int M, int N, int K, FA fa, FB fb, FE epi, GemmSmem<R
                     }
                 }
             }
+            // what the results combine with is loaded for the whole 4x4 block first (loads in flight together)
+            using P = decltype(pre(0, 0));
+            P p[4][4];
 #pragma unroll
             for (int i = 0; i < 4; ++i)
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const int m = m0 + ty * 4 + i, n = n0 + tx * 4 + j;
-                    if (m < M && n < N) epi(m, n, acc[0][i][j], NACC == 2 ? acc[NACC - 1][i][j] : (Real)0);
+                    if (m < M && n < N) p[i][j] = pre(m, n);
+                }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int m = m0 + ty * 4 + i, n = n0 + tx * 4 + j;
+                    if (m < M && n < N) epi(m, n, acc[0][i][j], NACC == 2 ? acc[NACC - 1][i][j] : (Real)0, p[i][j]);
                 }
         }
     }

@@ -1,21 +1,43 @@
 // SIMT forward: Algorithm 1 applied chunk after chunk, one CTA per sequence, for any shape.
 // The fp32-I/O instantiation computes in fp64 and is the GPU-side reference for the tensor-core path.
+#include <type_traits>
+
 #include "simt_common.cuh"
 #include "simt_layout.h"
+#include "tc_gemm.cuh"
 
 namespace e2ttt {
 
-template <typename Real, typename IO, int KIND>
-__global__ void __launch_bounds__(kSimtThreads) simt_fwd_kernel(const SimtFwdArgs a) {
+#ifdef SIMT_PROFILE
+// Debug build only: cycle stamps of thread 0 of CTA 0 at the phase boundaries of the first 32 chunks.
+__device__ long long g_simt_fwd_prof[32 * 16];
+#define SPROF(i)                                                                                      \
+    do {                                                                                              \
+        if (threadIdx.x == 0 && blockIdx.x == 0 && c < 32) g_simt_fwd_prof[c * 16 + (i)] = clock64(); \
+    } while (0)
+extern "C" __attribute__((visibility("default"))) int e2ttt_debug_read_simt_fwd_profile(long long* host, int n) {
+    return (int)cudaMemcpyFromSymbol(host, g_simt_fwd_prof, sizeof(long long) * (size_t)n);
+}
+#else
+#define SPROF(i)
+#endif
+
+// TC = true (bf16 I/O only): every GEMM runs on the tensor cores with bf16 operands; everything else is unchanged.
+template <typename Real, typename IO, int KIND, bool TC>
+__global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_fwd_kernel(const SimtFwdArgs a) {
     constexpr int NMAT = (KIND == 0) ? 2 : 3;
     constexpr int LAST = NMAT - 1;
+    using Engine = typename std::conditional<TC, TcGemm, FmaGemm<Real>>::type;
+    constexpr int NT = Engine::kThreads;  // threads per CTA
     extern __shared__ __align__(16) unsigned char simt_smem_raw[];
-    GemmSmem<Real>& gsm = *reinterpret_cast<GemmSmem<Real>*>(simt_smem_raw);
-    ChunkScalars<Real>& sc = *reinterpret_cast<ChunkScalars<Real>*>(simt_smem_raw + sizeof(GemmSmem<Real>));
+    unsigned char* smem_base = Engine::align(simt_smem_raw);
+    ChunkScalars<Real>& sc = *reinterpret_cast<ChunkScalars<Real>*>(smem_base + Engine::kBytes);
 
     const int CL = a.cl;                 // CTAs working on this sequence (one cluster)
     const int seq = blockIdx.x / CL, rank = blockIdx.x % CL;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    Engine G;
+    G.setup(smem_base, a.status, rank, CL);
     const int d = a.d, h = a.h, C = a.C, L = a.L;
     const size_t dh = (size_t)d * h;
     const SimtLayout& lay = a.lay;
@@ -37,10 +59,10 @@ __global__ void __launch_bounds__(kSimtThreads) simt_fwd_kernel(const SimtFwdArg
         M[i] = ws + lay.M[i];
         const float* wi = a.W_init[i] + (size_t)seq * dh;
         const float* mi = a.M_init[i] ? a.M_init[i] + (size_t)seq * dh : nullptr;
-        for (size_t e = tid + (size_t)rank * kSimtThreads; e < dh; e += (size_t)kSimtThreads * CL) {
-            W[i][e] = (Real)wi[e];
-            M[i][e] = mi ? (Real)mi[e] : (Real)0;
-        }
+        struct WM { Real w, m; };
+        batched_for<8>(tid + (size_t)rank * NT, dh, (size_t)NT * CL,
+                       [&](size_t e) { return WM{(Real)wi[e], mi ? (Real)mi[e] : (Real)0}; },
+                       [&](size_t e, const WM& x) { W[i][e] = x.w; M[i][e] = x.m; });
     }
     Real* Z1 = ws + lay.Z1;
     Real* Z2 = ws + lay.Z2;
@@ -58,39 +80,51 @@ __global__ void __launch_bounds__(kSimtThreads) simt_fwd_kernel(const SimtFwdArg
         const IO* qc = q + (size_t)s * d;
         const IO* vc = v + (size_t)s * d;
 
+        SPROF(0);
         // Algorithm 1 line 2: scalar kernels and carries
         if (warp == 0) chunk_scalars_warp<Real>(eta + s, beta + s, gamma + s, len, &sc);
         if (a.save_states) {
             Real* ck = ws + lay.ckpt + (size_t)c * 2 * NMAT * dh;
 #pragma unroll
-            for (int i = 0; i < NMAT; ++i)
-                for (size_t e = tid + (size_t)rank * kSimtThreads; e < dh; e += (size_t)kSimtThreads * CL) {
-                    ck[(size_t)i * dh + e] = W[i][e];
-                    ck[(size_t)(NMAT + i) * dh + e] = M[i][e];
-                }
+            for (int i = 0; i < NMAT; ++i) {
+                struct WM { Real w, m; };
+                batched_for<8>(tid + (size_t)rank * NT, dh, (size_t)NT * CL,
+                               [&](size_t e) { return WM{W[i][e], M[i][e]}; },
+                               [&](size_t e, const WM& x) {
+                                   ck[(size_t)i * dh + e] = x.w;
+                                   ck[(size_t)(NMAT + i) * dh + e] = x.m;
+                               });
+            }
         }
 
+        SPROF(1);
         // Algorithm 1 line 1: the network on the chunk's keys (rows 0..len-1) and queries (rows len..2len-1)
         auto load_x = [&](int m, int kk, Real& a0, Real& a1) {
             a0 = (m < len) ? ld_io<Real>(kc, (size_t)m * d + kk) : ld_io<Real>(qc, (size_t)(m - len) * d + kk);
         };
-        block_gemm<Real, 1, true, true>(
+        G.template run<1, true, true>(
             2 * len, h, d, load_x, [&](int n, int kk) { return W[0][(size_t)n * d + kk]; },
-            [&](int m, int n, Real acc, Real) { Z1[(size_t)m * h + n] = acc; }, &gsm, rank, CL);
+            [&](int m, int n, Real acc, Real) { Z1[(size_t)m * h + n] = acc; });
+        SPROF(2);
         if (KIND == 1)
-            block_gemm<Real, 1, true, true>(
+            G.template run<1, true, true>(
                 2 * len, h, d, load_x, [&](int n, int kk) { return W[1][(size_t)n * d + kk]; },
-                [&](int m, int n, Real acc, Real) { Z2[(size_t)m * h + n] = acc; }, &gsm, rank, CL);
-        for (size_t e = tid + (size_t)rank * kSimtThreads; e < (size_t)2 * len * h; e += (size_t)kSimtThreads * CL)
-            A[e] = (KIND == 0) ? gelu_f(Z1[e]) : silu_f(Z1[e]) * Z2[e];
+                [&](int m, int n, Real acc, Real) { Z2[(size_t)m * h + n] = acc; });
+        SPROF(3);
+        struct ZZ { Real z1, z2; };
+        batched_for<8>(tid + (size_t)rank * NT, (size_t)2 * len * h, (size_t)NT * CL,
+                       [&](size_t e) { return ZZ{Z1[e], KIND == 0 ? (Real)0 : Z2[e]}; },
+                       [&](size_t e, const ZZ& z) { A[e] = (KIND == 0) ? gelu_f(z.z1) : silu_f(z.z1) * z.z2; });
         phase_sync(CL);
-        block_gemm<Real, 1, true, true>(
+        SPROF(4);
+        G.template run<1, true, true>(
             2 * len, d, h, [&](int m, int kk, Real& a0, Real& a1) { a0 = A[(size_t)m * h + kk]; },
             [&](int n, int kk) { return W[LAST][(size_t)n * h + kk]; },
-            [&](int m, int n, Real acc, Real) { U[(size_t)m * d + n] = acc; }, &gsm, rank, CL);
+            [&](int m, int n, Real acc, Real) { U[(size_t)m * d + n] = acc; });
 
+        SPROF(5);
         // layer norm; outputs for the query rows; e = f(k) - v and pu = dL/du for the key rows (Algorithm 1 line 3)
-        for (int m = warp + rank * (kSimtThreads / 32); m < 2 * len; m += (kSimtThreads / 32) * CL) {
+        for (int m = warp + rank * (NT / 32); m < 2 * len; m += (NT / 32) * CL) {
             Real* u = U + (size_t)m * d;
             const Real r = warp_layernorm(u, u, d, eps);
             if (m >= len) {
@@ -116,25 +150,30 @@ __global__ void __launch_bounds__(kSimtThreads) simt_fwd_kernel(const SimtFwdArg
         }
         phase_sync(CL);
 
+        SPROF(6);
         // back through the last matrix and the activation
-        block_gemm<Real, 1, true, false>(
+        G.template run_rmw<1, true, false>(
             len, h, d, [&](int m, int kk, Real& a0, Real& a1) { a0 = Pu[(size_t)m * d + kk]; },
             [&](int n, int kk) { return W[LAST][(size_t)kk * h + n]; },
-            [&](int m, int n, Real acc, Real) {
+            [&](int m, int n) {
+                const size_t e = (size_t)m * h + n;
+                return ZZ{Z1[e], KIND == 0 ? (Real)0 : Z2[e]};
+            },
+            [&](int m, int n, Real acc, Real, const ZZ& z) {
                 const size_t e = (size_t)m * h + n;
                 if (KIND == 0) {
-                    Pz1[e] = acc * gelu_d1(Z1[e]);
+                    Pz1[e] = acc * gelu_d1(z.z1);
                 } else {
-                    Pz1[e] = acc * Z2[e] * silu_d1(Z1[e]);
-                    Pz2[e] = acc * silu_f(Z1[e]);
+                    Pz1[e] = acc * z.z2 * silu_d1(z.z1);
+                    Pz2[e] = acc * silu_f(z.z1);
                 }
-            },
-            &gsm, rank, CL);
+            });
 
+        SPROF(7);
         // Algorithm 1 lines 4-7: both weighted aggregations of every matrix, fused with the state transition
         const Real cw = sc.cw, cm = sc.cm, cb = sc.cb;
         auto update = [&](Real* Wm, Real* Mm, int rows, int cols, const Real* P, auto load_xcol) {
-            block_gemm<Real, 2, false, false>(
+            G.template run_rmw<2, false, false>(
                 rows, cols, len,
                 [&](int m, int t, Real& a0, Real& a1) {
                     const Real p = P[(size_t)t * rows + m];
@@ -142,19 +181,24 @@ __global__ void __launch_bounds__(kSimtThreads) simt_fwd_kernel(const SimtFwdArg
                     a1 = sc.kM[t] * p;
                 },
                 load_xcol,
-                [&](int m, int n, Real aW, Real aM) {
+                [&](int m, int n) {
                     const size_t e = (size_t)m * cols + n;
-                    const Real w = Wm[e], mm = Mm[e];
-                    Wm[e] = cw * w + cm * mm - aW; // G_t = -grad: the aggregations enter with a minus sign
-                    Mm[e] = cb * mm - aM;
+                    return ZZ{Wm[e], Mm[e]};
                 },
-                &gsm, rank, CL);
+                [&](int m, int n, Real aW, Real aM, const ZZ& wm) {
+                    const size_t e = (size_t)m * cols + n;
+                    Wm[e] = cw * wm.z1 + cm * wm.z2 - aW; // G_t = -grad: the aggregations enter with a minus sign
+                    Mm[e] = cb * wm.z2 - aM;
+                });
         };
         auto key_col = [&](int n, int t) { return ld_io<Real>(kc, (size_t)t * d + n); };
         auto act_col = [&](int n, int t) { return A[(size_t)t * h + n]; };
         update(W[0], M[0], h, d, Pz1, key_col);
+        SPROF(8);
         if (KIND == 1) update(W[1], M[1], h, d, Pz2, key_col);
+        SPROF(9);
         update(W[LAST], M[LAST], d, h, Pu, act_col);
+        SPROF(10);
     }
 
 #pragma unroll
@@ -162,27 +206,29 @@ __global__ void __launch_bounds__(kSimtThreads) simt_fwd_kernel(const SimtFwdArg
         if (!a.W_final[i]) continue; // state-recompute run of the backward: only the saved chunk states matter
         float* wf = a.W_final[i] + (size_t)seq * dh;
         float* mf = a.M_final[i] + (size_t)seq * dh;
-        for (size_t e = tid + (size_t)rank * kSimtThreads; e < dh; e += (size_t)kSimtThreads * CL) {
-            wf[e] = (float)W[i][e];
-            mf[e] = (float)M[i][e];
-        }
+        struct WM { Real w, m; };
+        batched_for<8>(tid + (size_t)rank * NT, dh, (size_t)NT * CL,
+                       [&](size_t e) { return WM{W[i][e], M[i][e]}; },
+                       [&](size_t e, const WM& x) { wf[e] = (float)x.w; mf[e] = (float)x.m; });
     }
+    G.teardown();
 }
 
-template <typename Real, typename IO, int KIND>
+template <typename Real, typename IO, int KIND, bool TC>
 static int launch_fwd(const SimtFwdArgs& a, cudaStream_t st) {
-    constexpr size_t smem = sizeof(GemmSmem<Real>) + sizeof(ChunkScalars<Real>);
+    using Engine = typename std::conditional<TC, TcGemm, FmaGemm<Real>>::type;
+    constexpr size_t smem = Engine::kBytes + sizeof(ChunkScalars<Real>) + (TC ? 1024 : 0);
     static bool attr_done[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return (int)cudaGetLastError();
     if (dev < 0 || dev >= 64 || !attr_done[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(simt_fwd_kernel<Real, IO, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(simt_fwd_kernel<Real, IO, KIND, TC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return (int)e;
         if (dev >= 0 && dev < 64) attr_done[dev] = true;
     }
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)(a.N * a.cl));
-    cfg.blockDim = dim3(kSimtThreads);
+    cfg.blockDim = dim3(Engine::kThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute at[1];
@@ -192,15 +238,18 @@ static int launch_fwd(const SimtFwdArgs& a, cudaStream_t st) {
     at[0].val.clusterDim.z = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, simt_fwd_kernel<Real, IO, KIND>, a);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, simt_fwd_kernel<Real, IO, KIND, TC>, a);
     if (e != cudaSuccess) return (int)e;
     return (int)cudaGetLastError();
 }
 
 int simt_fwd_launch(const SimtFwdArgs& a, int kind, int io_dtype, void* stream) {
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    if (io_dtype == 0) return kind == 0 ? launch_fwd<double, float, 0>(a, st) : launch_fwd<double, float, 1>(a, st);
-    return kind == 0 ? launch_fwd<float, __nv_bfloat16, 0>(a, st) : launch_fwd<float, __nv_bfloat16, 1>(a, st);
+    if (io_dtype == 0)
+        return kind == 0 ? launch_fwd<double, float, 0, false>(a, st) : launch_fwd<double, float, 1, false>(a, st);
+    if (a.tc)
+        return kind == 0 ? launch_fwd<float, __nv_bfloat16, 0, true>(a, st) : launch_fwd<float, __nv_bfloat16, 1, true>(a, st);
+    return kind == 0 ? launch_fwd<float, __nv_bfloat16, 0, false>(a, st) : launch_fwd<float, __nv_bfloat16, 1, false>(a, st);
 }
 
 }  // namespace e2ttt

@@ -53,6 +53,8 @@ inline SimtLayout simt_layout(int d, int h, int C, int nmat, int nchunks, bool s
 struct SimtFwdArgs {
     int N, L, d, h, C, nchunks, save_states;
     int cl;  // CTAs per sequence (cluster size), chosen by the launcher
+    int tc;  // GEMMs on the tensor cores with bf16 operands (bf16 I/O only) instead of fp32 FMAs
+    int* status;  // device status word of the call (bounded waits report here)
     float eps;
     const void *q, *k, *v;
     const float *eta, *beta, *gamma;
@@ -68,6 +70,8 @@ struct SimtFwdArgs {
 struct SimtBwdArgs {
     int N, L, d, h, C, nchunks;
     int cl;  // CTAs per sequence (cluster size), chosen by the launcher
+    int tc;  // GEMMs on the tensor cores with bf16 operands (bf16 I/O only) instead of fp32 FMAs
+    int* status;  // device status word of the call (bounded waits report here)
     float eps;
     const void *q, *k, *v, *d_o;
     const float *eta, *beta, *gamma;
