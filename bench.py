@@ -295,7 +295,7 @@ def run_ours(args, r):
 
 def run_fwd_bwd(args, r):
     """Optional second workload (--backward): one step = e2ttt_chunk_fwd(save_states=1) + e2ttt_chunk_bwd on the same
-    batch (GELU-MLP only).  Both run on the SIMT path today; the line says so."""
+    batch (both networks).  The line names the kernels that ran."""
     import torch
     from paper_2608_21308_b200 import binding as E
 
@@ -358,7 +358,7 @@ def run_fwd_bwd(args, r):
     flop = flops_per_token_head(r, backward=True) * N * r.L
     cfg = workload_config(r)
     cfg["workload"] = cfg["workload"].replace("e2ttt_chunk_fwd", "e2ttt_chunk_fwd(save_states) + e2ttt_chunk_bwd")
-    cfg["path"] = "tensor-core forward writing chunk-start states where a specialisation exists, SIMT backward"
+    cfg["path"] = "fused tensor-core forward writing chunk-start states where it serves the shape, any-shape backward with tcgen05 GEMMs"
     line = {"metric": "e2ttt_layer_fwd_bwd_tokens_per_s", "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if r.io == "bf16" else "f64", "data": "synthetic", "config": cfg,
@@ -372,6 +372,106 @@ def run_fwd_bwd(args, r):
     print(json.dumps(line))
 
 
+def run_decode(args, r):
+    """Optional third workload (--decode): one step = e2ttt_apply for ONE new token of every sequence (the decode path
+    between chunk boundaries).  HBM-bound: the step reads every sequence's fast weights once.  The weights of one
+    step fit in L2, so the steps rotate over enough independent state copies to exceed it, as the layers of a model do."""
+    import torch
+    from paper_2608_21308_b200 import binding as E
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    rr = inputs.Recipe(**{**r.__dict__, "L": 1})
+    x = inputs.generate(rr)
+    N = r.B * r.H
+    iod = torch.float32 if r.io == "f32" else torch.bfloat16
+    p = E.make_params(r.B, r.H, 1, r.d, r.h, 1, r.kind, E.E2TTT_F32 if r.io == "f32" else E.E2TTT_BF16, 1e-5,
+                      E.E2TTT_IMPL_AUTO)
+    shapes = inputs.mat_shapes(r.kind, r.d, r.h)
+    s4 = (r.B, r.H, 1, r.d)
+    host_q = torch.from_numpy(x["q"]).to(iod).view(s4).pin_memory()
+    host_o = torch.empty(s4, dtype=iod).pin_memory()
+    q = host_q.to(dev)
+    o = torch.empty_like(q)
+    state_bytes = sum(4 * N * a * b for a, b in shapes)
+    copies = max(2, int(3 * 126e6 // state_bytes) + 1)
+    Ws = []
+    for c in range(copies):
+        Ws.append([torch.from_numpy(w).view((r.B, r.H) + s).to(dev) * (1.0 + 0.01 * c) for w, s in zip(x["W"], shapes)])
+    stream = torch.cuda.current_stream()
+    it = [0]
+
+    def step(st=None):
+        E.e2ttt_apply(p, q, Ws[it[0] % copies], o, st if st is not None else stream)
+        it[0] += 1
+
+    def step_e2e():
+        q.copy_(host_q, non_blocking=True)
+        step()
+        host_o.copy_(o, non_blocking=True)
+
+    # A step is a ~10 us kernel: launched one by one from Python the host, not the GPU, sets the pace.  So one pass
+    # over the state copies is captured in a CUDA graph (the library call only enqueues a kernel) and replayed.
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for _ in range(copies):
+            step(torch.cuda.current_stream())
+    replays = max(1, -(-max(args.steps, 50) // copies))
+    steps = replays * copies
+
+    def timed_graph():
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(replays):
+            graph.replay()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+
+    def timed(fn, n, warmup):
+        for _ in range(warmup):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(n):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    sampler = ClockSampler(0)
+    sampler.start()
+    ms = timed_graph()
+    clocks = sampler.stop()
+    ms_eager = timed(step, steps, 3)
+    ms_e2e = timed(step_e2e, steps, 3)
+    pk = peaks()
+    io_bytes = 2 * N * r.d * (2 if r.io == "bf16" else 4)
+    nbytes = state_bytes + io_bytes
+    kind = "mlp_gelu" if r.kind == inputs.KIND_MLP else "swiglu"
+    line = {"metric": "e2ttt_decode_tokens_per_s", "value": r.B / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": steps,
+            "warmup": max(args.warmup, copies), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"e2ttt_apply, one token per sequence, B={r.B} H={r.H} d={r.d} h={r.h} {kind} {r.io} I/O",
+                       "B": r.B, "H": r.H, "d": r.d, "h": r.h, "kind": kind, "io": r.io, "seed": r.seed,
+                       "l2": f"steps rotate over {copies} independent state copies ({copies * state_bytes / 1e6:.0f} MB > 126 MB L2)"},
+            "e2e": {"value": r.B / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": host_q.numel() * host_q.element_size(),
+                    "d2h_bytes_per_step": host_o.numel() * host_o.element_size(), "ms_per_step": ms_e2e},
+            "gpu_launches": steps, "clocks": clocks,
+            "roofline": {"bound": "hbm", "achieved": nbytes / (ms * 1e-3) / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                         "frac": nbytes / (ms * 1e-3) / 1e9 / pk["hbm_gbs"], "traffic": None, "peak_source": pk["_source"],
+                         "kernel": "apply kernel (one launch per step, steps replayed from a CUDA graph)",
+                         "bytes_per_launch": nbytes, "ms_per_step_launched_from_python": ms_eager}}
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -381,11 +481,14 @@ def main():
     ap.add_argument("--config", type=int, default=2, help="benchmark configuration index (default: the 1.3B-layer shape)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--backward", action="store_true", help="time forward + backward instead (1 GPU, GELU-MLP configs)")
+    ap.add_argument("--decode", action="store_true", help="time the decode step instead: e2ttt_apply on one token per sequence (1 GPU)")
     ap.add_argument("--chunk", type=int, default=0, help="override the chunk size C of the configuration")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     r = inputs.config(args.config, **({"C": args.chunk} if args.chunk else {}))
-    if args.backward and args.impl == "ours":
+    if args.decode and args.impl == "ours":
+        run_decode(args, r)
+    elif args.backward and args.impl == "ours":
         run_fwd_bwd(args, r)
     elif args.impl == "reference":
         run_reference(args, r)

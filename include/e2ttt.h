@@ -155,6 +155,23 @@ E2TTT_API int e2ttt_chunk_bwd(const e2ttt_params* p,
                     float* const* dW_init, float* const* dM_init,
                     void* workspace, size_t workspace_bytes, int states_saved, void* stream);
 
+/* Outputs of fixed fast weights, no update: o[b,h,t,:] = f_W(q[b,h,t,:]) for t < p->L  (Algorithm 1 line 1
+ * with the weights held fixed; the streaming / decode use of the method).  Between two chunk boundaries every
+ * token is answered from the chunk-start weights W_0, and the state changes only when a whole chunk of keys,
+ * values and gates has accumulated: that step is e2ttt_chunk_fwd over those C tokens (its `o` equals what this
+ * call returned for the same tokens).  So a decoder calls e2ttt_apply per incoming token (p->L = 1) and
+ * e2ttt_chunk_fwd once every C tokens.
+ *   p        in  (host)    B, H, d, h, kind, io_dtype, ln_eps as above; L = tokens per sequence in this call;
+ *                          C and impl are ignored
+ *   q        in  (device)  [B,H,L,d] io_dtype, 16-byte aligned
+ *   W        in  (host array of device pointers)  the nmat fast-weight matrices, fp32, shapes as above
+ *   o        out (device)  [B,H,L,d] io_dtype, 16-byte aligned
+ * Needs no workspace; the work is enqueued on `stream`; nothing is allocated and the host is not synchronised.
+ * Arithmetic: fp32 throughout (weights are read as fp32, never rounded).  For a few tokens the call is bound
+ * by reading W once: 4 * nmat * d * h bytes per (b, h).
+ * Returns E2TTT_OK or E2TTT_ERR_NULL / _SHAPE / _DTYPE / _ALIGN / _ARCH / _CUDA. */
+E2TTT_API int e2ttt_apply(const e2ttt_params* p, const void* q, const float* const* W, void* o, void* stream);
+
 /* Reads back the device status word of the last launch that used `workspace` (the first word of every
  * workspace).  This is the one entry point that synchronises: it waits for `stream`.
  *   status  out (host)  0 after a clean run; otherwise the code of the first bounded device-side wait

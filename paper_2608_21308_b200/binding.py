@@ -54,6 +54,8 @@ def lib() -> ctypes.CDLL:
                                       tab, tab, vp, ctypes.c_size_t, cp, vp]
         L.e2ttt_chunk_fwd_noalloc.argtypes = [pp, vp, vp, vp, vp, vp, vp, tab, tab, vp, tab, tab, vp]
         L.e2ttt_chunk_fwd_noalloc.restype = cp
+        L.e2ttt_apply.argtypes = [pp, vp, tab, vp, vp]
+        L.e2ttt_apply.restype = cp
         L.e2ttt_device_status.argtypes = [vp, vp, ctypes.POINTER(cp)]
         L.e2ttt_device_status.restype = cp
         L.e2ttt_status_string.argtypes = [cp]
@@ -149,6 +151,17 @@ def e2ttt_chunk_fwd(p, q, k, v, eta, beta, gamma, W_init, M_init, o, W_final, M_
         int(save_states), _stream_ptr(stream))
     if st != E2TTT_OK:
         raise E2TTTError(st, "e2ttt_chunk_fwd")
+    return st
+
+
+def e2ttt_apply(p, q, W, o, stream=None):
+    """int e2ttt_apply(...) of include/e2ttt.h: o = f_W(q) for p.L tokens per sequence, no update.  Raises on error."""
+    io = _io_torch_dtype(p)
+    s4 = (p.B, p.H, p.L, p.d)
+    st = lib().e2ttt_apply(ctypes.byref(p), _ptr(q, io, s4, "q"), _table(W, p, "W"), _ptr(o, io, s4, "o"),
+                           _stream_ptr(stream))
+    if st != E2TTT_OK:
+        raise E2TTTError(st, "e2ttt_apply")
     return st
 
 

@@ -2,6 +2,7 @@
 #include <cuda_runtime.h>
 
 #include "../../include/e2ttt.h"
+#include "apply.h"
 #include "simt_layout.h"
 #include "tc_fwd.h"
 
@@ -245,6 +246,28 @@ int e2ttt_chunk_bwd(const e2ttt_params* p, const void* q, const void* k, const v
         b.dM_init[i] = dM_init[i];
     }
     return simt_bwd_launch(b, p->kind, p->io_dtype, stream) == 0 ? E2TTT_OK : E2TTT_ERR_CUDA;
+}
+
+int e2ttt_apply(const e2ttt_params* p, const void* q, const float* const* W, void* o, void* stream) {
+    int rc = check_params(p);
+    if (rc) return rc;
+    if (!q || !W || !o) return E2TTT_ERR_NULL;
+    const int nmat = nmat_of(p->kind);
+    for (int i = 0; i < nmat; ++i)
+        if (!W[i]) return E2TTT_ERR_NULL;
+    if (!aligned(q, 16) || !aligned(o, 16)) return E2TTT_ERR_ALIGN;
+    rc = check_device();
+    if (rc) return rc;
+    ApplyArgs a{};
+    a.N = p->B * p->H; a.T = p->L; a.d = p->d; a.h = p->h; a.eps = p->ln_eps;
+    a.cl = apply_cluster_size(a.N);
+    a.tb = apply_token_block(a.T);
+    while (a.cl > 1 && apply_smem_bytes(a.d, a.cl, a.tb) > 40 * 1024) a.cl /= 2;  // room for two CTAs per SM
+    if (apply_smem_bytes(a.d, a.cl, a.tb) > 200 * 1024) return E2TTT_ERR_SHAPE;
+    a.stage = apply_smem_bytes(a.d, a.cl, a.tb) <= 40 * 1024 && apply_can_stage(a.d, a.h, a.cl);
+    a.q = q; a.o = o;
+    for (int i = 0; i < nmat; ++i) a.W[i] = W[i];
+    return apply_launch(a, p->kind, p->io_dtype, stream) == 0 ? E2TTT_OK : E2TTT_ERR_CUDA;
 }
 
 int e2ttt_device_status(const void* workspace, void* stream, int* status) {

@@ -18,6 +18,14 @@ __device__ long long g_simt_fwd_prof[32 * 16];
 extern "C" __attribute__((visibility("default"))) int e2ttt_debug_read_simt_fwd_profile(long long* host, int n) {
     return (int)cudaMemcpyFromSymbol(host, g_simt_fwd_prof, sizeof(long long) * (size_t)n);
 }
+extern "C" __attribute__((visibility("default"))) int e2ttt_debug_read_gemm_profile(long long* host, int reset) {
+    const cudaError_t e = cudaMemcpyFromSymbol(host, g_tg_prof, sizeof(long long) * 16);
+    if (reset) {
+        long long z[16] = {0};
+        cudaMemcpyToSymbol(g_tg_prof, z, sizeof(z));
+    }
+    return (int)e;
+}
 #else
 #define SPROF(i)
 #endif

@@ -121,6 +121,23 @@ __device__ __forceinline__ void tg_fill(uint8_t* hi0, uint8_t* lo0, uint8_t* hi1
     }
 }
 
+#ifdef SIMT_PROFILE
+// Debug build only: cycles thread 0 of CTA 0 spends in each section of TcGemm::run_rmw, summed over the launch.
+__device__ long long g_tg_prof[16];
+#define TGPROF(i)                                                          \
+    do {                                                                   \
+        if (threadIdx.x == 0 && blockIdx.x == 0) {                         \
+            const long long now_ = clock64();                              \
+            g_tg_prof[i] += now_ - tgp_;                                   \
+            tgp_ = now_;                                                   \
+        }                                                                  \
+    } while (0)
+#define TGPROF_START() long long tgp_ = clock64()
+#else
+#define TGPROF(i)
+#define TGPROF_START()
+#endif
+
 struct TcGemm {
     static constexpr int kThreads = kTgThreads;
     static constexpr size_t kBytes = sizeof(TcGemmSmem);
@@ -174,6 +191,7 @@ struct TcGemm {
         const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
         const uint32_t idesc = make_idesc(kTgBN, kTgBM, false, false);
         int tile = 0;
+        TGPROF_START();
         for (int n0 = 0; n0 < N; n0 += kTgBN) {
             for (int m0 = 0; m0 < M; m0 += kTgBM, ++tile) {
                 if (tile % nranks != rank) continue;
@@ -182,11 +200,13 @@ struct TcGemm {
                     const uint32_t s = it & 1u;
                     // the MMAs of the slice that used this stage two slices ago have read it
                     if (it >= 2) mbar_wait(&sm->bar[s], ((it >> 1) - 1u) & 1u, wc, 200 + 1);
+                    TGPROF(0);
                     const int kc16 = (min(kTgBK, K - k0) + 15) >> 4;  // MMAs (16 k each) in this slice
                     tg_fill<kTgBN, B_KFAST, 1>(sm->R[s][0], sm->R[s][1], nullptr, nullptr, 2 * kc16,
                                                [&](int r, int kk, float& v0, float&) {
                                                    if (n0 + r < N && k0 + kk < K) v0 = (float)fb(n0 + r, k0 + kk);
                                                });
+                    TGPROF(1);
                     tg_fill<kTgBM, A_KFAST, NACC>(sm->Cc[s][0][0], sm->Cc[s][0][1], sm->Cc[s][1][0], sm->Cc[s][1][1], 2 * kc16,
                                                   [&](int r, int kk, float& v0, float& v1) {
                                                       if (m0 + r < M && k0 + kk < K) {
@@ -196,8 +216,10 @@ struct TcGemm {
                                                           v1 = a1;
                                                       }
                                                   });
+                    TGPROF(2);
                     fence_proxy_async_smem();
                     __syncthreads();
+                    TGPROF(3);
                     if (tid == 0) {
                         tc_fence_after_sync();
                         for (int k = 0; k < kc16; ++k) {
@@ -217,10 +239,12 @@ struct TcGemm {
                     }
                     last_it = it;
                     ++it;
+                    TGPROF(4);
                 }
                 // all MMAs of the tile are done when the last slice's are (they complete in order)
                 mbar_wait(&sm->bar[last_it & 1u], (last_it >> 1) & 1u, wc, 200 + 2);
                 tc_fence_after_sync();
+                TGPROF(5);
                 {
                     const int qd = warp & 3, grp = warp >> 2;  // lane quadrant of this warp; which 16 of the 64 columns
                     const uint32_t taddr = tmem + ((uint32_t)(32 * qd) << 16) + (uint32_t)(16 * grp);
@@ -250,12 +274,15 @@ struct TcGemm {
                         }
                     }
                 }
+                TGPROF(6);
                 tc_fence_before_sync();
                 __syncthreads();  // the accumulators may be overwritten by the next tile
                 tc_fence_after_sync();
+                TGPROF(7);
             }
         }
         phase_sync(nranks);
+        TGPROF(8);
     }
 };
 
