@@ -18,6 +18,12 @@
  *     affine parameters; GELU = x Phi(x) with the exact erf (both readings: the paper does
  *     not say).
  *
+ *   - optional post-chunk normalisation (Appendix "Implementation details": L2 normalisation of the
+ *     fast-weight matrices at each chunk boundary; the paper gives neither axis nor target - a
+ *     reading): after the last token of a chunk every row w of every W_i (one output unit's
+ *     weights; the momentum is left alone) becomes  n w / (||w||_2 + eps_n), n the row's target norm,
+ *     an input.  The next chunk starts from, and the final state is, the normalised W.
+ *
  * The closed form of Proposition 1 is NOT used here: this file is the definition the closed
  * form must reproduce.  The reverse pass is the adjoint of exactly this program, swept token
  * by token.
@@ -26,7 +32,8 @@
  * chunk-end states vs Proposition 1 and vs the division-free unrolled Eq. "unroll_recurrence";
  * neutral gates reduce to one plain chunk-wise step; C = 1 reduces to the token-wise update;
  * the hand-expanded C = 2 case; the reverse pass vs finite differences and vs an independent
- * automatic-differentiation run.  The paper prints no output or state VALUES, so absolute
+ * automatic-differentiation run; the normalisation vs an independent chunk-by-chunk restatement and
+ * its reverse pass vs finite differences.  The paper prints no output or state VALUES, so absolute
  * values are fixed only by those pins and by the readings above.
  *
  * Layouts (row-major, dense, double): q, k, v, o [N, L, d]; eta, beta, gamma [N, L];
@@ -308,11 +315,45 @@ static void neg_grad_vjp(const net_t* n, const double* const* W, const double* k
     }
 }
 
+/* ---------- post-chunk normalisation of one matrix: rows w -> n w / (||w|| + eps_n) ---------- */
+static int mat_rows(const net_t* n, int i) { return (i == n->nmat - 1) ? n->d : n->h; }
+
+static void rows_normalise(const net_t* n, int i, double* W, const double* target, double eps_n) {
+    const int rows = mat_rows(n, i);
+    const size_t cols = n->n / (size_t)rows;
+    for (int r = 0; r < rows; ++r) {
+        double* w = W + (size_t)r * cols;
+        const double s = sqrt(dot(cols, w, w));
+        const double f = target[r] / (s + eps_n);
+        for (size_t c = 0; c < cols; ++c) w[c] *= f;
+    }
+}
+
+/* adjoint of rows_normalise: Wt = the rows BEFORE normalisation; Yb (in) = adjoint of the normalised rows, (out) =
+ * adjoint of Wt; nb, if not NULL, accumulates the adjoint of the targets.
+ *   y = n w / (s + e),  s = ||w||:   wb = n/(s+e) (yb - w <yb, w> / (s (s+e))),   nb = <yb, w> / (s+e)          */
+static void rows_normalise_vjp(const net_t* n, int i, const double* Wt, const double* target, double eps_n,
+                               double* Yb, double* nb) {
+    const int rows = mat_rows(n, i);
+    const size_t cols = n->n / (size_t)rows;
+    for (int r = 0; r < rows; ++r) {
+        const double* w = Wt + (size_t)r * cols;
+        double* yb = Yb + (size_t)r * cols;
+        const double s = sqrt(dot(cols, w, w));
+        const double yw = dot(cols, yb, w);
+        if (nb) nb[r] += yw / (s + eps_n);
+        const double f = target[r] / (s + eps_n);
+        const double g = (s > 0.0) ? yw / (s * (s + eps_n)) : 0.0;
+        for (size_t c = 0; c < cols; ++c) yb[c] = f * (yb[c] - w[c] * g);
+    }
+}
+
 /* ---------- one sequence, forward ---------- */
 static int seq_forward(const net_t* n, int L, int C, const double* q, const double* k, const double* v,
                        const double* eta, const double* beta, const double* gamma,
                        double* const* W, double* const* M, /* in: initial state, out: final state */
-                       double* o /* may be NULL */, double* chunk_states /* may be NULL: [nchunks][2][nmat][n] */) {
+                       double* o /* may be NULL */, double* chunk_states /* may be NULL: [nchunks][2][nmat][n] */,
+                       const double* const* row_norm /* NULL: no post-chunk normalisation */, double eps_n) {
     const int d = n->d;
     tok_t t;
     if (tok_alloc(&t, n->d, n->h)) return -1;
@@ -348,6 +389,8 @@ static int seq_forward(const net_t* n, int L, int C, const double* q, const doub
                 }
             }
         }
+        if (row_norm)
+            for (int i = 0; i < n->nmat; ++i) rows_normalise(n, i, W[i], row_norm[i], eps_n);
     }
     for (int i = 0; i < n->nmat; ++i) { free(W0[i]); free(G[i]); }
     tok_free(&t);
@@ -359,7 +402,9 @@ static int seq_backward(const net_t* n, int L, int C, const double* q, const dou
                         const double* eta, const double* beta, const double* gamma,
                         const double* const* W_init, const double* const* M_init, /* M_init[i] never NULL here */
                         const double* d_o, double* const* Wb, double* const* Mb, /* in: adjoints of the final state; out: of the initial state */
-                        double* dq, double* dk, double* dv, double* deta, double* dbeta, double* dgamma) {
+                        double* dq, double* dk, double* dv, double* deta, double* dbeta, double* dgamma,
+                        const double* const* row_norm /* NULL: no post-chunk normalisation */, double eps_n,
+                        double* const* row_norm_b /* NULL or out: adjoints of the targets (accumulated) */) {
     const int d = n->d, nm = n->nmat;
     const size_t ne = n->n;
     const int nchunks = (L + C - 1) / C;
@@ -380,7 +425,7 @@ static int seq_backward(const net_t* n, int L, int C, const double* q, const dou
         memcpy(W[i], W_init[i], ne * sizeof(double));
         memcpy(M[i], M_init[i], ne * sizeof(double));
     }
-    if (seq_forward(n, L, C, q, k, v, eta, beta, gamma, W, M, NULL, cs)) return -1;
+    if (seq_forward(n, L, C, q, k, v, eta, beta, gamma, W, M, NULL, cs, row_norm, eps_n)) return -1;
 
     for (int c = nchunks - 1; c >= 0; --c) {
         const int s = c * C;
@@ -407,6 +452,10 @@ static int seq_backward(const net_t* n, int L, int C, const double* q, const dou
                     W[i][e] = gamma[tt] * W[i][e] + M[i][e];
                 }
         }
+        /* W now holds the chunk-end weights before normalisation: pull the adjoint back through it */
+        if (row_norm)
+            for (int i = 0; i < nm; ++i)
+                rows_normalise_vjp(n, i, W[i], row_norm[i], eps_n, Wb[i], row_norm_b ? row_norm_b[i] : NULL);
         /* reverse the token-wise recurrence */
         for (int j = len - 1; j >= 0; --j) {
             const int tt = s + j;
@@ -456,12 +505,13 @@ int e2ttt_oracle_max_threads(void) {
 /* Forward over N sequences.  W_final/M_final receive the final states; M_init may be NULL (zeros).
  * chunk_states, if not NULL, receives [N][nchunks][2][nmat][d*h]: the (W, M) at every chunk start.
  * Returns 0, or -1 on allocation failure / bad arguments.  threads <= 0: all cores. */
-int e2ttt_oracle_fwd(int N, int L, int d, int h, int C, int kind, double eps,
-                     const double* q, const double* k, const double* v,
-                     const double* eta, const double* beta, const double* gamma,
-                     const double* const* W_init, const double* const* M_init,
-                     double* o, double* const* W_final, double* const* M_final,
-                     double* chunk_states, int threads) {
+int e2ttt_oracle_fwd_norm(int N, int L, int d, int h, int C, int kind, double eps,
+                          const double* q, const double* k, const double* v,
+                          const double* eta, const double* beta, const double* gamma,
+                          const double* const* W_init, const double* const* M_init,
+                          double* o, double* const* W_final, double* const* M_final,
+                          double* chunk_states, int threads,
+                          const double* const* row_norm /* NULL or nmat x [N, rows_i] */, double eps_n) {
     if (N <= 0 || L <= 0 || d <= 0 || h <= 0 || C <= 0 || (kind != KIND_MLP && kind != KIND_SWIGLU)) return -1;
     net_t n = make_net(d, h, kind, eps);
     const int nchunks = (L + C - 1) / C;
@@ -480,9 +530,12 @@ int e2ttt_oracle_fwd(int N, int L, int d, int h, int C, int kind, double eps,
             else memset(M[i], 0, n.n * sizeof(double));
         }
         const size_t off = (size_t)s * L;
+        const double* rn[MAXMAT];
+        for (int i = 0; i < n.nmat; ++i) rn[i] = row_norm ? row_norm[i] + (size_t)s * mat_rows(&n, i) : NULL;
         int rc = seq_forward(&n, L, C, q + off * d, k + off * d, v + off * d, eta + off, beta + off, gamma + off,
                              W, M, o ? o + off * d : NULL,
-                             chunk_states ? chunk_states + (size_t)s * nchunks * 2 * n.nmat * n.n : NULL);
+                             chunk_states ? chunk_states + (size_t)s * nchunks * 2 * n.nmat * n.n : NULL,
+                             row_norm ? rn : NULL, eps_n);
         if (rc) {
 #ifdef _OPENMP
 #pragma omp atomic write
@@ -493,15 +546,27 @@ int e2ttt_oracle_fwd(int N, int L, int d, int h, int C, int kind, double eps,
     return fail ? -1 : 0;
 }
 
-/* Reverse pass over N sequences: adjoints of everything e2ttt_oracle_fwd reads, given d_o and the
- * adjoints of the final state (dW_final / dM_final, NULL = zeros). */
-int e2ttt_oracle_bwd(int N, int L, int d, int h, int C, int kind, double eps,
+int e2ttt_oracle_fwd(int N, int L, int d, int h, int C, int kind, double eps,
                      const double* q, const double* k, const double* v,
                      const double* eta, const double* beta, const double* gamma,
                      const double* const* W_init, const double* const* M_init,
-                     const double* d_o, const double* const* dW_final, const double* const* dM_final,
-                     double* dq, double* dk, double* dv, double* deta, double* dbeta, double* dgamma,
-                     double* const* dW_init, double* const* dM_init, int threads) {
+                     double* o, double* const* W_final, double* const* M_final,
+                     double* chunk_states, int threads) {
+    return e2ttt_oracle_fwd_norm(N, L, d, h, C, kind, eps, q, k, v, eta, beta, gamma, W_init, M_init, o, W_final,
+                                 M_final, chunk_states, threads, NULL, 0.0);
+}
+
+/* Reverse pass over N sequences: adjoints of everything the forward reads, given d_o and the
+ * adjoints of the final state (dW_final / dM_final, NULL = zeros).  With row_norm (post-chunk normalisation)
+ * d_row_norm (NULL or nmat x [N, rows_i]) receives the adjoints of the targets. */
+int e2ttt_oracle_bwd_norm(int N, int L, int d, int h, int C, int kind, double eps,
+                          const double* q, const double* k, const double* v,
+                          const double* eta, const double* beta, const double* gamma,
+                          const double* const* W_init, const double* const* M_init,
+                          const double* d_o, const double* const* dW_final, const double* const* dM_final,
+                          double* dq, double* dk, double* dv, double* deta, double* dbeta, double* dgamma,
+                          double* const* dW_init, double* const* dM_init, int threads,
+                          const double* const* row_norm, double eps_n, double* const* d_row_norm) {
     if (N <= 0 || L <= 0 || d <= 0 || h <= 0 || C <= 0 || (kind != KIND_MLP && kind != KIND_SWIGLU)) return -1;
     net_t n = make_net(d, h, kind, eps);
     int fail = 0;
@@ -525,10 +590,18 @@ int e2ttt_oracle_bwd(int N, int L, int d, int h, int C, int kind, double eps,
             else memset(Mb[i], 0, n.n * sizeof(double));
         }
         const size_t off = (size_t)s * L;
+        const double* rn[MAXMAT];
+        double* rnb[MAXMAT];
+        for (int i = 0; i < n.nmat; ++i) {
+            rn[i] = row_norm ? row_norm[i] + (size_t)s * mat_rows(&n, i) : NULL;
+            rnb[i] = (row_norm && d_row_norm) ? d_row_norm[i] + (size_t)s * mat_rows(&n, i) : NULL;
+            if (rnb[i]) memset(rnb[i], 0, (size_t)mat_rows(&n, i) * sizeof(double));
+        }
         int rc = (!M_init && !zeros) ? -1 :
                  seq_backward(&n, L, C, q + off * d, k + off * d, v + off * d, eta + off, beta + off, gamma + off,
                               Wi, Mi, d_o + off * d, Wb, Mb, dq + off * d, dk + off * d, dv + off * d,
-                              deta + off, dbeta + off, dgamma + off);
+                              deta + off, dbeta + off, dgamma + off, row_norm ? rn : NULL, eps_n,
+                              (row_norm && d_row_norm) ? rnb : NULL);
         free(zeros);
         if (rc) {
 #ifdef _OPENMP
@@ -538,6 +611,17 @@ int e2ttt_oracle_bwd(int N, int L, int d, int h, int C, int kind, double eps,
         }
     }
     return fail ? -1 : 0;
+}
+
+int e2ttt_oracle_bwd(int N, int L, int d, int h, int C, int kind, double eps,
+                     const double* q, const double* k, const double* v,
+                     const double* eta, const double* beta, const double* gamma,
+                     const double* const* W_init, const double* const* M_init,
+                     const double* d_o, const double* const* dW_final, const double* const* dM_final,
+                     double* dq, double* dk, double* dv, double* deta, double* dbeta, double* dgamma,
+                     double* const* dW_init, double* const* dM_init, int threads) {
+    return e2ttt_oracle_bwd_norm(N, L, d, h, C, kind, eps, q, k, v, eta, beta, gamma, W_init, M_init, d_o, dW_final,
+                                 dM_final, dq, dk, dv, deta, dbeta, dgamma, dW_init, dM_init, threads, NULL, 0.0, NULL);
 }
 
 /* One token at fixed weights: the inner loss and G_i = -dL/dW_i (for the finite-difference pin and

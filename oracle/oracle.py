@@ -73,9 +73,12 @@ def _f64l(lst):
     return None if lst is None else [_f64(a) for a in lst]
 
 
-def forward(q, k, v, eta, beta, gamma, W_init, M_init, C, kind, eps=1e-5, threads=0, want_states=False):
+def forward(q, k, v, eta, beta, gamma, W_init, M_init, C, kind, eps=1e-5, threads=0, want_states=False,
+            row_norm=None, norm_eps=1e-5):
     """q, k, v [N, L, d]; gates [N, L]; W_init list of [N, rows, cols]; M_init same or None.
 
+    row_norm: None, or a list of [N, rows_i] target norms: every row of every W_i is rescaled to its target after
+    each chunk (post-chunk normalisation).
     Returns dict(o, W, M[, states]) in fp64; states [N, nchunks, 2, nmat, d*h] holds (W, M) at chunk starts.
     """
     q, k, v, eta, beta, gamma = map(_f64, (q, k, v, eta, beta, gamma))
@@ -89,9 +92,11 @@ def forward(q, k, v, eta, beta, gamma, W_init, M_init, C, kind, eps=1e-5, thread
     Mf = [np.empty((N,) + s) for s in shapes]
     nchunks = (L + C - 1) // C
     states = np.empty((N, nchunks, 2, len(shapes), d * h)) if want_states else None
-    rc = lib().e2ttt_oracle_fwd(
+    row_norm = _f64l(row_norm)
+    rc = lib().e2ttt_oracle_fwd_norm(
         N, L, d, h, C, kind, ctypes.c_double(eps), _p(q), _p(k), _p(v), _p(eta), _p(beta), _p(gamma),
-        _pp(W_init), _pp(M_init), _p(o), _pp(Wf), _pp(Mf), _p(states), threads)
+        _pp(W_init), _pp(M_init), _p(o), _pp(Wf), _pp(Mf), _p(states), threads, _pp(row_norm),
+        ctypes.c_double(norm_eps))
     if rc != 0:
         raise RuntimeError("oracle forward failed")
     out = {"o": o, "W": Wf, "M": Mf}
@@ -100,8 +105,10 @@ def forward(q, k, v, eta, beta, gamma, W_init, M_init, C, kind, eps=1e-5, thread
     return out
 
 
-def backward(q, k, v, eta, beta, gamma, W_init, M_init, d_o, dW_final, dM_final, C, kind, eps=1e-5, threads=0):
-    """Adjoints of every input of forward(), given d_o and (optional) adjoints of the final state."""
+def backward(q, k, v, eta, beta, gamma, W_init, M_init, d_o, dW_final, dM_final, C, kind, eps=1e-5, threads=0,
+             row_norm=None, norm_eps=1e-5):
+    """Adjoints of every input of forward(), given d_o and (optional) adjoints of the final state.
+    With row_norm the result also holds "drow_norm", the adjoints of the target norms."""
     q, k, v, eta, beta, gamma, d_o = map(_f64, (q, k, v, eta, beta, gamma, d_o))
     W_init, M_init, dW_final, dM_final = map(_f64l, (W_init, M_init, dW_final, dM_final))
     N, L, d = q.shape
@@ -111,13 +118,19 @@ def backward(q, k, v, eta, beta, gamma, W_init, M_init, d_o, dW_final, dM_final,
     de, db, dg = np.empty((N, L)), np.empty((N, L)), np.empty((N, L))
     dW = [np.empty((N,) + s) for s in shapes]
     dM = [np.empty((N,) + s) for s in shapes]
-    rc = lib().e2ttt_oracle_bwd(
+    row_norm = _f64l(row_norm)
+    drn = [np.zeros((N, s[0])) for s in shapes] if row_norm is not None else None
+    rc = lib().e2ttt_oracle_bwd_norm(
         N, L, d, h, C, kind, ctypes.c_double(eps), _p(q), _p(k), _p(v), _p(eta), _p(beta), _p(gamma),
         _pp(W_init), _pp(M_init), _p(d_o), _pp(dW_final), _pp(dM_final),
-        _p(dq), _p(dk), _p(dv), _p(de), _p(db), _p(dg), _pp(dW), _pp(dM), threads)
+        _p(dq), _p(dk), _p(dv), _p(de), _p(db), _p(dg), _pp(dW), _pp(dM), threads, _pp(row_norm),
+        ctypes.c_double(norm_eps), _pp(drn))
     if rc != 0:
         raise RuntimeError("oracle backward failed")
-    return {"dq": dq, "dk": dk, "dv": dv, "deta": de, "dbeta": db, "dgamma": dg, "dW": dW, "dM": dM}
+    out = {"dq": dq, "dk": dk, "dv": dv, "deta": de, "dbeta": db, "dgamma": dg, "dW": dW, "dM": dM}
+    if drn is not None:
+        out["drow_norm"] = drn
+    return out
 
 
 def inner(W, k, v, kind, eps=1e-5, want_grad=True):

@@ -360,6 +360,111 @@ def test_reverse_pass_matches_finite_differences_of_own_forward(kind):
                 assert abs(fd - bw[gname][i][idx]) <= 2e-6 * max(1.0, abs(fd)), (name, i, idx, fd, bw[gname][i][idx])
 
 
+
+# ---------------------------------------------------------------- post-chunk normalisation (a reading: rows, to a target)
+def _targets(x, scale=1.0):
+    """Target norms as a model would set them: the row norms of the initial fast weights (times a factor)."""
+    return [scale * np.sqrt((w.astype(np.float64) ** 2).sum(-1)) for w in x["W"]]
+
+
+def _normalise_rows(W, target, eps_n):
+    """Independent restatement in numpy: every row w -> n w / (||w|| + eps_n)."""
+    s = np.sqrt((W ** 2).sum(-1, keepdims=True))
+    return W * (target[..., None] / (s + eps_n))
+
+
+@pytest.mark.parametrize("kind", KINDS)
+def test_post_chunk_normalisation_equals_chunk_by_chunk_restatement(kind):
+    """Normalised run == for every chunk: the (already pinned) un-normalised update of that chunk alone, followed by a
+    row normalisation written here in numpy.  Also: the final rows have norm n s/(s + eps_n), the momentum is untouched
+    by the normalisation itself, and the outputs of chunk c come from the normalised state of chunk c - 1."""
+    C, eps_n = 4, 1e-5
+    r, x = tiny(kind, d=4, h=8, L=3 * C + 2, C=C, seed=31, N=2)
+    tgt = _targets(x, 1.3)
+    got = oracle.forward(x["q"], x["k"], x["v"], x["eta"], x["beta"], x["gamma"], x["W"], x["M"], C, kind,
+                         row_norm=tgt, norm_eps=eps_n)
+    W = [w.astype(np.float64) for w in x["W"]]
+    M = [m.astype(np.float64) for m in x["M"]]
+    outs = []
+    for s0 in range(0, r.L, C):
+        sl = slice(s0, min(s0 + C, r.L))
+        one = oracle.forward(x["q"][:, sl], x["k"][:, sl], x["v"][:, sl], x["eta"][:, sl], x["beta"][:, sl],
+                             x["gamma"][:, sl], W, M, C, kind)
+        outs.append(one["o"])
+        pre = one["W"]
+        W = [_normalise_rows(w, t, eps_n) for w, t in zip(pre, tgt)]
+        M = one["M"]
+    assert rel(got["o"], np.concatenate(outs, 1)) <= 1e-13
+    for i in range(len(W)):
+        assert rel(got["W"][i], W[i]) <= 1e-13 and rel(got["M"][i], M[i]) <= 1e-13
+        s_pre = np.sqrt((pre[i] ** 2).sum(-1))
+        assert np.allclose(np.sqrt((got["W"][i] ** 2).sum(-1)), tgt[i] * s_pre / (s_pre + eps_n), rtol=1e-12)
+    plain = oracle.forward(x["q"], x["k"], x["v"], x["eta"], x["beta"], x["gamma"], x["W"], x["M"], C, kind)
+    assert rel(got["o"][:, :C], plain["o"][:, :C]) == 0.0           # the first chunk reads the un-normalised initial state
+    assert rel(got["o"][:, C:], plain["o"][:, C:]) > 1e-3           # later chunks do see the normalisation
+
+
+def test_post_chunk_normalisation_is_invariant_to_the_scale_of_the_update():
+    """Rows that are rescaled to a fixed norm forget their length: with targets t, a run started from c * W_init
+    (eta = 0, gamma = 1, so the update leaves the direction alone) ends at rows of norm t in the direction of W_init."""
+    C, eps_n = 4, 0.0
+    r, x = tiny(inputs.KIND_MLP, d=4, h=8, L=2 * C, C=C, seed=33, m_std=0.0)
+    x["eta"][:] = 0.0
+    x["gamma"][:] = 1.0
+    tgt = [np.full(w.shape[:2], 2.0) for w in x["W"]]
+    got = oracle.forward(x["q"], x["k"], x["v"], x["eta"], x["beta"], x["gamma"], [5.0 * w.astype(np.float64) for w in x["W"]], x["M"], C, inputs.KIND_MLP,
+                         row_norm=tgt, norm_eps=eps_n)
+    for i, w in enumerate(x["W"]):
+        w = w.astype(np.float64)
+        unit = w / np.sqrt((w ** 2).sum(-1, keepdims=True))
+        assert rel(got["W"][i], 2.0 * unit) <= 1e-13
+
+
+@pytest.mark.parametrize("kind", KINDS)
+def test_reverse_pass_through_the_normalisation_matches_finite_differences(kind):
+    C, eps_n = 3, 1e-3
+    r, x = tiny(kind, d=4, h=6, L=2 * C + 1, C=C, seed=37)
+    x64 = {n: (([a.astype(np.float64) for a in val]) if isinstance(val, list) else val.astype(np.float64))
+           for n, val in x.items()}
+    x64["row_norm"] = _targets(x, 0.8)
+    bw = oracle.backward(x64["q"], x64["k"], x64["v"], x64["eta"], x64["beta"], x64["gamma"], x64["W"], x64["M"],
+                         x64["d_o"], x64["dW"], x64["dM"], C, kind, row_norm=x64["row_norm"], norm_eps=eps_n)
+
+    def objective(xx):
+        fw = oracle.forward(xx["q"], xx["k"], xx["v"], xx["eta"], xx["beta"], xx["gamma"], xx["W"], xx["M"], C, kind,
+                            row_norm=xx["row_norm"], norm_eps=eps_n)
+        s = float(np.sum(fw["o"] * xx["d_o"]))
+        for i in range(len(xx["W"])):
+            s += float(np.sum(fw["W"][i] * xx["dW"][i]) + np.sum(fw["M"][i] * xx["dM"][i]))
+        return s
+
+    rng = np.random.default_rng(1)
+    step = 1e-6
+
+    def probe(arr, grad, what):
+        idx = tuple(rng.integers(0, s) for s in arr.shape)
+        keep = arr[idx]
+        arr[idx] = keep + step
+        up = objective(x64)
+        arr[idx] = keep - step
+        dn = objective(x64)
+        arr[idx] = keep
+        fd = (up - dn) / (2 * step)
+        assert abs(fd - grad[idx]) <= 5e-6 * max(1.0, abs(fd)), (what, idx, fd, grad[idx])
+
+    for name, gname in [("q", "dq"), ("k", "dk"), ("v", "dv"), ("eta", "deta"), ("beta", "dbeta"), ("gamma", "dgamma")]:
+        for _ in range(4):
+            probe(x64[name], bw[gname], name)
+    for name, gname in (("W", "dW"), ("M", "dM"), ("row_norm", "drow_norm")):
+        for i in range(len(x64[name])):
+            for _ in range(3):
+                probe(x64[name][i], bw[gname][i], (name, i))
+    # without normalisation the new entry points are the old ones
+    a = oracle.backward(x64["q"], x64["k"], x64["v"], x64["eta"], x64["beta"], x64["gamma"], x64["W"], x64["M"],
+                        x64["d_o"], x64["dW"], x64["dM"], C, kind)
+    assert "drow_norm" not in a
+
+
 # ---------------------------------------------------------------- input generator sanity (data only)
 def test_generator_follows_the_stated_distributions():
     r = inputs.config(0)
