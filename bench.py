@@ -208,15 +208,22 @@ def run_ours(args, r):
     o = torch.empty(s4, dtype=iod, device=dev)
     Wf = [torch.empty_like(w) for w in W0]
     Mf = [torch.empty_like(w) for w in W0]
-    ws = torch.empty(E.e2ttt_workspace_bytes(p, 0), dtype=torch.uint8, device=dev)
+    ws = torch.empty((E.e2ttt_workspace_bytes_normed if args.post_norm else E.e2ttt_workspace_bytes)(p, 0),
+                     dtype=torch.uint8, device=dev)
+    # --post-norm: targets = the row norms of the initial fast weights, as a model would set them
+    row_norm = [w.float().pow(2).sum(-1).sqrt().contiguous() for w in W0] if args.post_norm else None
     host_o = torch.empty(s4, dtype=iod).pin_memory()
     host_Wf = [torch.empty_like(w).pin_memory() for w in hostW]
     host_Mf = [torch.empty_like(w).pin_memory() for w in hostW]
     stream = torch.cuda.current_stream()
 
     def step():
-        E.e2ttt_chunk_fwd(p, devt["q"], devt["k"], devt["v"], devt["eta"], devt["beta"], devt["gamma"], W0, None, o,
-                          Wf, Mf, ws, 0, stream)
+        if args.post_norm:
+            E.e2ttt_chunk_fwd_normed(p, devt["q"], devt["k"], devt["v"], devt["eta"], devt["beta"], devt["gamma"], W0, None,
+                                     row_norm, 1e-5, o, Wf, Mf, ws, 0, stream)
+        else:
+            E.e2ttt_chunk_fwd(p, devt["q"], devt["k"], devt["v"], devt["eta"], devt["beta"], devt["gamma"], W0, None, o,
+                              Wf, Mf, ws, 0, stream)
 
     def step_e2e():
         for n in host:
@@ -274,7 +281,8 @@ def run_ours(args, r):
             "metric": METRIC, "value": whole_job_value(world, tokens, ms), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if r.io == "bf16" else "f64",
-            "data": "synthetic", "config": workload_config(r),
+            "data": "synthetic",
+            "config": dict(workload_config(r), **({"post_chunk_norm": "rows of every W_i rescaled to the row norms of W_init after each chunk (any-shape kernels)"} if args.post_norm else {})),
             "e2e": {"value": whole_job_value(world, tokens, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
             "gpu_launches": args.steps,
@@ -482,6 +490,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--backward", action="store_true", help="time forward + backward instead (1 GPU, GELU-MLP configs)")
     ap.add_argument("--decode", action="store_true", help="time the decode step instead: e2ttt_apply on one token per sequence (1 GPU)")
+    ap.add_argument("--post-norm", action="store_true", help="forward with post-chunk normalisation of the fast weights (e2ttt_chunk_fwd_normed)")
     ap.add_argument("--chunk", type=int, default=0, help="override the chunk size C of the configuration")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

@@ -155,6 +155,36 @@ E2TTT_API int e2ttt_chunk_bwd(const e2ttt_params* p,
                     float* const* dW_init, float* const* dM_init,
                     void* workspace, size_t workspace_bytes, int states_saved, void* stream);
 
+/* The same two calls with post-chunk normalisation of the fast weights (Appendix "Implementation details":
+ * L2 normalisation of the fast-weight matrices at each chunk boundary, as a stabiliser).  The paper gives neither
+ * the axis nor the target; the reading taken here: after the state transition of every chunk, each row w of each
+ * W_i (the weights of one output unit; the momentum is left alone) becomes  n w / (||w||_2 + norm_eps), where n
+ * is that row's target norm.  The next chunk starts from, and W_final is, the normalised state, so calls chain.
+ *   row_norm    in  (host array of nmat device pointers)  [B,H,rows_i] fp32 targets (rows_i as in
+ *                                                          e2ttt_matrix_shape); a model passes the row norms
+ *                                                          of its learned initial fast weights
+ *   norm_eps    in                                         >= 0
+ *   d_row_norm  out (host array of nmat device pointers, or NULL)  adjoints of the targets, [B,H,rows_i] fp32
+ * Everything else as in e2ttt_chunk_fwd / e2ttt_chunk_bwd.  Served by the any-shape kernels (impl SIMT or TILED;
+ * AUTO picks between them; TCGEN05 gives E2TTT_ERR_SHAPE), whose workspace e2ttt_workspace_bytes_normed sizes
+ * (the backward always needs the save_states = 1 size).  A backward with states_saved = 1 needs the states of
+ * e2ttt_chunk_fwd_normed(save_states = 1) with the same targets. */
+E2TTT_API int e2ttt_workspace_bytes_normed(const e2ttt_params* p, int save_states, size_t* bytes);
+E2TTT_API int e2ttt_chunk_fwd_normed(const e2ttt_params* p, const void* q, const void* k, const void* v,
+                                     const float* eta, const float* beta, const float* gamma,
+                                     const float* const* W_init, const float* const* M_init,
+                                     const float* const* row_norm, float norm_eps,
+                                     void* o, float* const* W_final, float* const* M_final,
+                                     void* workspace, size_t workspace_bytes, int save_states, void* stream);
+E2TTT_API int e2ttt_chunk_bwd_normed(const e2ttt_params* p, const void* q, const void* k, const void* v,
+                                     const float* eta, const float* beta, const float* gamma,
+                                     const float* const* W_init, const float* const* M_init,
+                                     const float* const* row_norm, float norm_eps,
+                                     const void* d_o, const float* const* dW_final, const float* const* dM_final,
+                                     void* dq, void* dk, void* dv, float* d_eta, float* d_beta, float* d_gamma,
+                                     float* const* dW_init, float* const* dM_init, float* const* d_row_norm,
+                                     void* workspace, size_t workspace_bytes, int states_saved, void* stream);
+
 /* Outputs of fixed fast weights, no update: o[b,h,t,:] = f_W(q[b,h,t,:]) for t < p->L  (Algorithm 1 line 1
  * with the weights held fixed; the streaming / decode use of the method).  Between two chunk boundaries every
  * token is answered from the chunk-start weights W_0, and the state changes only when a whole chunk of keys,

@@ -49,11 +49,19 @@ def lib() -> ctypes.CDLL:
         L.e2ttt_num_matrices.argtypes = [cp]
         L.e2ttt_matrix_shape.argtypes = [cp, cp, cp, cp, ctypes.POINTER(cp), ctypes.POINTER(cp)]
         L.e2ttt_workspace_bytes.argtypes = [pp, cp, ctypes.POINTER(ctypes.c_size_t)]
+        L.e2ttt_workspace_bytes_normed.argtypes = [pp, cp, ctypes.POINTER(ctypes.c_size_t)]
+        L.e2ttt_workspace_bytes_normed.restype = cp
         L.e2ttt_chunk_fwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, tab, tab, vp, tab, tab, vp, ctypes.c_size_t, cp, vp]
         L.e2ttt_chunk_bwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, tab, tab, vp, tab, tab, vp, vp, vp, vp, vp, vp,
                                       tab, tab, vp, ctypes.c_size_t, cp, vp]
         L.e2ttt_chunk_fwd_noalloc.argtypes = [pp, vp, vp, vp, vp, vp, vp, tab, tab, vp, tab, tab, vp]
         L.e2ttt_chunk_fwd_noalloc.restype = cp
+        L.e2ttt_chunk_fwd_normed.argtypes = [pp, vp, vp, vp, vp, vp, vp, tab, tab, tab, ctypes.c_float, vp, tab, tab, vp,
+                                             ctypes.c_size_t, cp, vp]
+        L.e2ttt_chunk_fwd_normed.restype = cp
+        L.e2ttt_chunk_bwd_normed.argtypes = [pp, vp, vp, vp, vp, vp, vp, tab, tab, tab, ctypes.c_float, vp, tab, tab, vp, vp,
+                                             vp, vp, vp, vp, tab, tab, tab, vp, ctypes.c_size_t, cp, vp]
+        L.e2ttt_chunk_bwd_normed.restype = cp
         L.e2ttt_apply.argtypes = [pp, vp, tab, vp, vp]
         L.e2ttt_apply.restype = cp
         L.e2ttt_device_status.argtypes = [vp, vp, ctypes.POINTER(cp)]
@@ -93,6 +101,14 @@ def e2ttt_workspace_bytes(p: e2ttt_params, save_states: int) -> int:
     st = lib().e2ttt_workspace_bytes(ctypes.byref(p), int(save_states), ctypes.byref(n))
     if st != E2TTT_OK:
         raise E2TTTError(st, "e2ttt_workspace_bytes")
+    return int(n.value)
+
+
+def e2ttt_workspace_bytes_normed(p: e2ttt_params, save_states: int) -> int:
+    n = ctypes.c_size_t()
+    st = lib().e2ttt_workspace_bytes_normed(ctypes.byref(p), int(save_states), ctypes.byref(n))
+    if st != E2TTT_OK:
+        raise E2TTTError(st, "e2ttt_workspace_bytes_normed")
     return int(n.value)
 
 
@@ -151,6 +167,60 @@ def e2ttt_chunk_fwd(p, q, k, v, eta, beta, gamma, W_init, M_init, o, W_final, M_
         int(save_states), _stream_ptr(stream))
     if st != E2TTT_OK:
         raise E2TTTError(st, "e2ttt_chunk_fwd")
+    return st
+
+
+def _row_table(ts, p, name):
+    """nmat pointers to [B, H, rows_i] fp32 tensors (row targets of the post-chunk normalisation, or their adjoints)."""
+    if ts is None:
+        return None
+    n = e2ttt_num_matrices(p.kind)
+    if len(ts) != n:
+        raise ValueError(f"{name}: expected {n} tensors")
+    arr = (ctypes.c_void_p * n)()
+    for i, t in enumerate(ts):
+        r, _ = e2ttt_matrix_shape(p.kind, p.d, p.h, i)
+        arr[i] = _ptr(t, torch.float32, (p.B, p.H, r), f"{name}[{i}]")
+    return arr
+
+
+def e2ttt_chunk_fwd_normed(p, q, k, v, eta, beta, gamma, W_init, M_init, row_norm, norm_eps, o, W_final, M_final,
+                           workspace, save_states=0, stream=None):
+    """int e2ttt_chunk_fwd_normed(...) of include/e2ttt.h.  Raises on error."""
+    io = _io_torch_dtype(p)
+    s4, s3 = (p.B, p.H, p.L, p.d), (p.B, p.H, p.L)
+    st = lib().e2ttt_chunk_fwd_normed(
+        ctypes.byref(p), _ptr(q, io, s4, "q"), _ptr(k, io, s4, "k"), _ptr(v, io, s4, "v"),
+        _ptr(eta, torch.float32, s3, "eta"), _ptr(beta, torch.float32, s3, "beta"),
+        _ptr(gamma, torch.float32, s3, "gamma"), _table(W_init, p, "W_init"), _table(M_init, p, "M_init"),
+        _row_table(row_norm, p, "row_norm"), float(norm_eps),
+        _ptr(o, io, s4, "o"), _table(W_final, p, "W_final"), _table(M_final, p, "M_final"),
+        _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel() if workspace is not None else 0,
+        int(save_states), _stream_ptr(stream))
+    if st != E2TTT_OK:
+        raise E2TTTError(st, "e2ttt_chunk_fwd_normed")
+    return st
+
+
+def e2ttt_chunk_bwd_normed(p, q, k, v, eta, beta, gamma, W_init, M_init, row_norm, norm_eps, d_o, dW_final, dM_final,
+                           dq, dk, dv, d_eta, d_beta, d_gamma, dW_init, dM_init, d_row_norm, workspace,
+                           states_saved=0, stream=None):
+    """int e2ttt_chunk_bwd_normed(...) of include/e2ttt.h.  Raises on error."""
+    io = _io_torch_dtype(p)
+    s4, s3 = (p.B, p.H, p.L, p.d), (p.B, p.H, p.L)
+    f32 = torch.float32
+    st = lib().e2ttt_chunk_bwd_normed(
+        ctypes.byref(p), _ptr(q, io, s4, "q"), _ptr(k, io, s4, "k"), _ptr(v, io, s4, "v"),
+        _ptr(eta, f32, s3, "eta"), _ptr(beta, f32, s3, "beta"), _ptr(gamma, f32, s3, "gamma"),
+        _table(W_init, p, "W_init"), _table(M_init, p, "M_init"), _row_table(row_norm, p, "row_norm"), float(norm_eps),
+        _ptr(d_o, io, s4, "d_o"), _table(dW_final, p, "dW_final"), _table(dM_final, p, "dM_final"),
+        _ptr(dq, io, s4, "dq"), _ptr(dk, io, s4, "dk"), _ptr(dv, io, s4, "dv"),
+        _ptr(d_eta, f32, s3, "d_eta"), _ptr(d_beta, f32, s3, "d_beta"), _ptr(d_gamma, f32, s3, "d_gamma"),
+        _table(dW_init, p, "dW_init"), _table(dM_init, p, "dM_init"), _row_table(d_row_norm, p, "d_row_norm"),
+        _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel() if workspace is not None else 0,
+        int(states_saved), _stream_ptr(stream))
+    if st != E2TTT_OK:
+        raise E2TTTError(st, "e2ttt_chunk_bwd_normed")
     return st
 
 

@@ -111,10 +111,20 @@ int e2ttt_workspace_bytes(const e2ttt_params* p, int save_states, size_t* bytes)
     return E2TTT_OK;
 }
 
-int e2ttt_chunk_fwd(const e2ttt_params* p, const void* q, const void* k, const void* v, const float* eta,
-                    const float* beta, const float* gamma, const float* const* W_init, const float* const* M_init,
-                    void* o, float* const* W_final, float* const* M_final, void* workspace, size_t workspace_bytes,
-                    int save_states, void* stream) {
+int e2ttt_workspace_bytes_normed(const e2ttt_params* p, int save_states, size_t* bytes) {
+    if (!bytes) return E2TTT_ERR_NULL;
+    int rc = check_params(p);
+    if (rc) return rc;
+    if (p->impl == E2TTT_IMPL_TCGEN05) return E2TTT_ERR_SHAPE;
+    *bytes = simt_bytes(p, save_states != 0, save_states != 0);
+    return E2TTT_OK;
+}
+
+static int fwd_common(const e2ttt_params* p, const void* q, const void* k, const void* v, const float* eta,
+                      const float* beta, const float* gamma, const float* const* W_init, const float* const* M_init,
+                      const float* const* row_norm, float norm_eps,
+                      void* o, float* const* W_final, float* const* M_final, void* workspace, size_t workspace_bytes,
+                      int save_states, void* stream) {
     int rc = check_params(p);
     if (rc) return rc;
     if (!q || !k || !v || !eta || !beta || !gamma || !W_init || !o || !W_final || !M_final) return E2TTT_ERR_NULL;
@@ -128,8 +138,17 @@ int e2ttt_chunk_fwd(const e2ttt_params* p, const void* q, const void* k, const v
     if (rc) return rc;
     if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(o, 16)) return E2TTT_ERR_ALIGN;
     size_t need = 0;
-    rc = e2ttt_workspace_bytes(p, save_states, &need);
-    if (rc) return rc;
+    if (row_norm) {
+        // the fused kernel has no normalisation step: the any-shape kernels serve the call
+        if (p->impl == E2TTT_IMPL_TCGEN05 || !(norm_eps >= 0.0f)) return E2TTT_ERR_SHAPE;
+        for (int i = 0; i < nmat; ++i)
+            if (!row_norm[i]) return E2TTT_ERR_NULL;
+        if (impl == E2TTT_IMPL_TCGEN05) impl = E2TTT_IMPL_TILED;
+        need = simt_bytes(p, save_states != 0, save_states != 0);
+    } else {
+        rc = e2ttt_workspace_bytes(p, save_states, &need);
+        if (rc) return rc;
+    }
     if (!workspace || workspace_bytes < need) return E2TTT_ERR_WORKSPACE;
     if (!aligned(workspace, 256)) return E2TTT_ERR_ALIGN;
     rc = check_device();
@@ -172,16 +191,38 @@ int e2ttt_chunk_fwd(const e2ttt_params* p, const void* q, const void* k, const v
         a.M_init[i] = M_init ? M_init[i] : nullptr;
         a.W_final[i] = W_final[i];
         a.M_final[i] = M_final[i];
+        a.row_norm[i] = row_norm ? row_norm[i] : nullptr;
     }
+    a.norm_eps = norm_eps;
     a.lay = simt_layout(p->d, p->h, p->C, nmat, a.nchunks, a.save_states, a.save_states);
     return simt_fwd_launch(a, p->kind, p->io_dtype, stream) == 0 ? E2TTT_OK : E2TTT_ERR_CUDA;
 }
 
-int e2ttt_chunk_bwd(const e2ttt_params* p, const void* q, const void* k, const void* v, const float* eta,
+int e2ttt_chunk_fwd(const e2ttt_params* p, const void* q, const void* k, const void* v, const float* eta,
                     const float* beta, const float* gamma, const float* const* W_init, const float* const* M_init,
-                    const void* d_o, const float* const* dW_final, const float* const* dM_final, void* dq, void* dk,
-                    void* dv, float* d_eta, float* d_beta, float* d_gamma, float* const* dW_init,
-                    float* const* dM_init, void* workspace, size_t workspace_bytes, int states_saved, void* stream) {
+                    void* o, float* const* W_final, float* const* M_final, void* workspace, size_t workspace_bytes,
+                    int save_states, void* stream) {
+    return fwd_common(p, q, k, v, eta, beta, gamma, W_init, M_init, nullptr, 0.0f, o, W_final, M_final, workspace,
+                      workspace_bytes, save_states, stream);
+}
+
+int e2ttt_chunk_fwd_normed(const e2ttt_params* p, const void* q, const void* k, const void* v, const float* eta,
+                           const float* beta, const float* gamma, const float* const* W_init,
+                           const float* const* M_init, const float* const* row_norm, float norm_eps, void* o,
+                           float* const* W_final, float* const* M_final, void* workspace, size_t workspace_bytes,
+                           int save_states, void* stream) {
+    if (!row_norm) return E2TTT_ERR_NULL;
+    return fwd_common(p, q, k, v, eta, beta, gamma, W_init, M_init, row_norm, norm_eps, o, W_final, M_final, workspace,
+                      workspace_bytes, save_states, stream);
+}
+
+static int bwd_common(const e2ttt_params* p, const void* q, const void* k, const void* v, const float* eta,
+                      const float* beta, const float* gamma, const float* const* W_init, const float* const* M_init,
+                      const float* const* row_norm, float norm_eps,
+                      const void* d_o, const float* const* dW_final, const float* const* dM_final, void* dq, void* dk,
+                      void* dv, float* d_eta, float* d_beta, float* d_gamma, float* const* dW_init,
+                      float* const* dM_init, float* const* d_row_norm, void* workspace, size_t workspace_bytes,
+                      int states_saved, void* stream) {
     int rc = check_params(p);
     if (rc) return rc;
     if (!q || !k || !v || !eta || !beta || !gamma || !W_init || !d_o || !dq || !dk || !dv || !d_eta || !d_beta ||
@@ -197,6 +238,11 @@ int e2ttt_chunk_bwd(const e2ttt_params* p, const void* q, const void* k, const v
     int impl = 0;
     rc = pick_impl(p, true, &impl);
     if (rc) return rc;
+    if (row_norm) {
+        if (p->impl == E2TTT_IMPL_TCGEN05 || !(norm_eps >= 0.0f)) return E2TTT_ERR_SHAPE;
+        for (int i = 0; i < nmat; ++i)
+            if (!row_norm[i]) return E2TTT_ERR_NULL;
+    }
     if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(d_o, 16) || !aligned(dq, 16) ||
         !aligned(dk, 16) || !aligned(dv, 16))
         return E2TTT_ERR_ALIGN;
@@ -229,7 +275,9 @@ int e2ttt_chunk_bwd(const e2ttt_params* p, const void* q, const void* k, const v
             f.M_init[i] = M_init ? M_init[i] : nullptr;
             f.W_final[i] = nullptr;
             f.M_final[i] = nullptr;
+            f.row_norm[i] = row_norm ? row_norm[i] : nullptr;
         }
+        f.norm_eps = norm_eps;
         if (simt_fwd_launch(f, p->kind, p->io_dtype, stream) != 0) return E2TTT_ERR_CUDA;
     }
     SimtBwdArgs b{};
@@ -244,8 +292,33 @@ int e2ttt_chunk_bwd(const e2ttt_params* p, const void* q, const void* k, const v
         b.dM_final[i] = dM_final ? dM_final[i] : nullptr;
         b.dW_init[i] = dW_init[i];
         b.dM_init[i] = dM_init[i];
+        b.row_norm[i] = row_norm ? row_norm[i] : nullptr;
+        b.d_row_norm[i] = (row_norm && d_row_norm) ? d_row_norm[i] : nullptr;
     }
+    b.norm_eps = norm_eps;
     return simt_bwd_launch(b, p->kind, p->io_dtype, stream) == 0 ? E2TTT_OK : E2TTT_ERR_CUDA;
+}
+
+int e2ttt_chunk_bwd(const e2ttt_params* p, const void* q, const void* k, const void* v, const float* eta,
+                    const float* beta, const float* gamma, const float* const* W_init, const float* const* M_init,
+                    const void* d_o, const float* const* dW_final, const float* const* dM_final, void* dq, void* dk,
+                    void* dv, float* d_eta, float* d_beta, float* d_gamma, float* const* dW_init,
+                    float* const* dM_init, void* workspace, size_t workspace_bytes, int states_saved, void* stream) {
+    return bwd_common(p, q, k, v, eta, beta, gamma, W_init, M_init, nullptr, 0.0f, d_o, dW_final, dM_final, dq, dk, dv,
+                      d_eta, d_beta, d_gamma, dW_init, dM_init, nullptr, workspace, workspace_bytes, states_saved, stream);
+}
+
+int e2ttt_chunk_bwd_normed(const e2ttt_params* p, const void* q, const void* k, const void* v, const float* eta,
+                           const float* beta, const float* gamma, const float* const* W_init,
+                           const float* const* M_init, const float* const* row_norm, float norm_eps, const void* d_o,
+                           const float* const* dW_final, const float* const* dM_final, void* dq, void* dk, void* dv,
+                           float* d_eta, float* d_beta, float* d_gamma, float* const* dW_init, float* const* dM_init,
+                           float* const* d_row_norm, void* workspace, size_t workspace_bytes, int states_saved,
+                           void* stream) {
+    if (!row_norm) return E2TTT_ERR_NULL;
+    return bwd_common(p, q, k, v, eta, beta, gamma, W_init, M_init, row_norm, norm_eps, d_o, dW_final, dM_final, dq, dk,
+                      dv, d_eta, d_beta, d_gamma, dW_init, dM_init, d_row_norm, workspace, workspace_bytes, states_saved,
+                      stream);
 }
 
 int e2ttt_apply(const e2ttt_params* p, const void* q, const float* const* W, void* o, void* stream) {

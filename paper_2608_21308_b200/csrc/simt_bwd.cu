@@ -132,6 +132,36 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_ke
         for (int i = 0; i < NMAT; ++i)
             for (size_t e = tid + (size_t)rank * NT; e < dh; e += (size_t)NT * CL) Wb[i][e] = 0;
 
+        // post-chunk normalisation (optional): T arrives as the adjoint of the normalised chunk-end weights
+        // y = n w / (s + eps_n), s = ||w||.  With y itself (the next chunk's saved start state) and the saved s:
+        //   w_bar = n/(s + eps_n) y_bar - y <y_bar, y> / (n s),      n_bar = <y_bar, y> / n
+        if (a.row_norm[0]) {
+            const int maxdim = d > h ? d : h;
+            const Real* nxt = ck + (size_t)2 * NMAT * dh;  // state after this chunk: W part
+#pragma unroll
+            for (int i = 0; i < NMAT; ++i) {
+                const int rows = (i == LAST) ? d : h, cols = (i == LAST) ? h : d;
+                const float* target = a.row_norm[i] + (size_t)seq * rows;
+                float* tb = a.d_row_norm[i] ? a.d_row_norm[i] + (size_t)seq * rows : nullptr;
+                for (int r = warp + rank * (NT / 32); r < rows; r += (NT / 32) * CL) {
+                    Real* t = T[i] + (size_t)r * cols;
+                    const Real* y = nxt + (size_t)i * dh + (size_t)r * cols;
+                    Real ty = 0;
+                    for (int j = lane; j < cols; j += 32) ty += t[j] * y[j];
+                    ty = warp_sum(ty);
+                    const Real n = (Real)target[r], nrm = ws[lay.rown + ((size_t)c * 3 + i) * maxdim + r];
+                    const Real f = n / (nrm + (Real)a.norm_eps);
+                    const Real g = (n != (Real)0 && nrm > (Real)0) ? ty / (n * nrm) : (Real)0;
+                    for (int j = lane; j < cols; j += 32) t[j] = f * t[j] - y[j] * g;
+                    if (tb && lane == 0) {
+                        const Real nb = (n != (Real)0) ? ty / n : (Real)0;
+                        tb[r] = (c == a.nchunks - 1) ? (float)nb : tb[r] + (float)nb;
+                    }
+                }
+            }
+            phase_sync(CL);
+        }
+
         auto load_x = [&](int m, int kk, Real& a0, Real& a1) {
             a0 = (m < len) ? ld_io<Real>(kc, (size_t)m * d + kk) : ld_io<Real>(qc, (size_t)(m - len) * d + kk);
         };

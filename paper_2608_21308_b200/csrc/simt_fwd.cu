@@ -207,6 +207,39 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_fwd_ke
         SPROF(9);
         update(W[LAST], M[LAST], d, h, Pu, act_col);
         SPROF(10);
+
+        // post-chunk normalisation (optional): every row w of every W_i becomes n w / (||w|| + eps_n); one warp per row
+        if (a.row_norm[0]) {
+            const int maxdim = d > h ? d : h;
+#pragma unroll
+            for (int i = 0; i < NMAT; ++i) {
+                const int rows = (i == LAST) ? d : h, cols = (i == LAST) ? h : d;
+                const float* target = a.row_norm[i] + (size_t)seq * rows;
+                for (int r = warp + rank * (NT / 32); r < rows; r += (NT / 32) * CL) {
+                    Real* w = W[i] + (size_t)r * cols;
+                    Real ss = 0;
+                    for (int j = lane; j < cols; j += 32) ss += w[j] * w[j];
+                    const Real nrm = sqrt(warp_sum(ss));
+                    const Real f = (Real)target[r] / (nrm + (Real)a.norm_eps);
+                    for (int j = lane; j < cols; j += 32) w[j] *= f;
+                    if (a.save_states && lane == 0) ws[lay.rown + ((size_t)c * 3 + i) * maxdim + r] = nrm;
+                }
+            }
+            phase_sync(CL);
+        }
+    }
+    if (a.save_states && a.row_norm[0]) {  // the reverse pass needs the normalised end state of the last chunk too
+        Real* ck = ws + lay.ckpt + (size_t)a.nchunks * 2 * NMAT * dh;
+#pragma unroll
+        for (int i = 0; i < NMAT; ++i) {
+            struct WM { Real w, m; };
+            batched_for<8>(tid + (size_t)rank * NT, dh, (size_t)NT * CL,
+                           [&](size_t e) { return WM{W[i][e], M[i][e]}; },
+                           [&](size_t e, const WM& x) {
+                               ck[(size_t)i * dh + e] = x.w;
+                               ck[(size_t)(NMAT + i) * dh + e] = x.m;
+                           });
+        }
     }
 
 #pragma unroll

@@ -18,7 +18,8 @@ struct SimtLayout {
     size_t XY1b, Pzb2, Zkb2, Zqb2;  // SwiGLU only: the second [h x d] matrix
     size_t rk, rq, red;  // per-row 1/std of the two LN calls; small reduction scratch
     size_t kWb, kMb;     // adjoints of the scalar kernels, one per token of the chunk
-    size_t ckpt;         // [nchunks][2][nmat][d*h] chunk-start (W, M), present when states are saved
+    size_t rown;         // [nchunks][3][max(d,h)] row norms of the chunk-end weights before their normalisation
+    size_t ckpt;         // [nchunks + 1][2][nmat][d*h] chunk-start (W, M) and, last, the final state; when states are saved
     size_t per_seq;      // elements per sequence
 };
 
@@ -45,7 +46,8 @@ inline SimtLayout simt_layout(int d, int h, int C, int nmat, int nchunks, bool s
         l.rk = take(C); l.rq = take(C); l.red = take(64);
         l.kWb = take(C); l.kMb = take(C);
     }
-    l.ckpt = take(save_states ? (size_t)nchunks * 2 * nmat * dh : 0);
+    l.rown = take(save_states ? (size_t)nchunks * 3 * (size_t)(d > h ? d : h) : 0);
+    l.ckpt = take(save_states ? (size_t)(nchunks + 1) * 2 * nmat * dh : 0);
     l.per_seq = o;
     return l;
 }
@@ -63,6 +65,8 @@ struct SimtFwdArgs {
     void* o;
     float* W_final[3];
     float* M_final[3];
+    const float* row_norm[3];  // post-chunk normalisation targets [N, rows_i]; row_norm[0] == nullptr: none
+    float norm_eps;
     void* ws;
     SimtLayout lay;
 };
@@ -81,6 +85,9 @@ struct SimtBwdArgs {
     float *d_eta, *d_beta, *d_gamma;
     float* dW_init[3];
     float* dM_init[3];
+    const float* row_norm[3];  // post-chunk normalisation targets [N, rows_i]; row_norm[0] == nullptr: none
+    float* d_row_norm[3];      // adjoints of the targets (nullptr entries: not wanted)
+    float norm_eps;
     void* ws;
     SimtLayout lay;
 };
