@@ -17,6 +17,29 @@
 
 namespace e2ttt {
 
+#ifdef SIMT_PROFILE
+// Debug build only: cycles thread 0 of CTA 0 spends between consecutive stamps, summed over the chunks of a launch.
+__device__ long long g_simt_bwd_prof[32];
+#define BPROF(i)                                            \
+    do {                                                    \
+        if (threadIdx.x == 0 && blockIdx.x == 0) {          \
+            const long long now_ = clock64();               \
+            g_simt_bwd_prof[i] += now_ - bp_;               \
+            bp_ = now_;                                     \
+        }                                                   \
+    } while (0)
+extern "C" __attribute__((visibility("default"))) int e2ttt_debug_read_simt_bwd_profile(long long* host, int reset) {
+    const cudaError_t e = cudaMemcpyFromSymbol(host, g_simt_bwd_prof, sizeof(long long) * 32);
+    if (reset) {
+        long long z[32] = {0};
+        cudaMemcpyToSymbol(g_simt_bwd_prof, z, sizeof(z));
+    }
+    return (int)e;
+}
+#else
+#define BPROF(i)
+#endif
+
 template <typename Real> __device__ __forceinline__ Real silu_d2(Real z) {
     const Real s = sigmoid_f(z);
     return s * ((Real)1 - s) * ((Real)2 + z * ((Real)1 - (Real)2 * s));
@@ -39,12 +62,13 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_ke
     constexpr int NMAT = (KIND == 0) ? 2 : 3;
     constexpr int LAST = NMAT - 1;
     constexpr bool SW = (KIND == 1);
-    using Engine = typename std::conditional<TC, TcGemm, FmaGemm<Real>>::type;
+    using Engine = typename std::conditional<TC, TcGemmT<true>, FmaGemm<Real>>::type;
     constexpr int NT = Engine::kThreads;  // threads per CTA
     extern __shared__ __align__(16) unsigned char simt_smem_raw[];
     unsigned char* smem_base = Engine::align(simt_smem_raw);
     ChunkScalars<Real>& sc = *reinterpret_cast<ChunkScalars<Real>*>(smem_base + Engine::kBytes);
     Real* red = reinterpret_cast<Real*>(smem_base + Engine::kBytes + sizeof(ChunkScalars<Real>));
+    Real* rev = red + 16;  // [8][kMaxC] operands and results of the reverse scan
 
     const int CL = a.cl;                 // CTAs working on this sequence (one cluster)
     const int seq = blockIdx.x / CL, rank = blockIdx.x % CL;
@@ -56,6 +80,7 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_ke
     const size_t dh = (size_t)d * h;
     const SimtLayout& lay = a.lay;
     Real* ws = reinterpret_cast<Real*>(a.ws) + (size_t)seq * lay.per_seq;
+    G.set_scratch(ws + lay.splitk);
     const IO* q = reinterpret_cast<const IO*>(a.q) + (size_t)seq * L * d;
     const IO* k = reinterpret_cast<const IO*>(a.k) + (size_t)seq * L * d;
     const IO* v = reinterpret_cast<const IO*>(a.v) + (size_t)seq * L * d;
@@ -113,6 +138,9 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_ke
     phase_sync(CL);
 
     for (int c = a.nchunks - 1; c >= 0; --c) {
+#ifdef SIMT_PROFILE
+        long long bp_ = clock64();
+#endif
         const int s = c * C;
         const int len = min(C, L - s);
         const IO* kc = k + (size_t)s * d;
@@ -167,7 +195,9 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_ke
         };
         auto load_k = [&](int m, int kk, Real& a0, Real& a1) { a0 = ld_io<Real>(kc, (size_t)m * d + kk); };
 
+        BPROF(0);
         // ---------------- forward of the chunk, recomputed ----------------
+        BPROF(1);
         G.template run<1, true, true>(
             2 * len, h, d, load_x, [&](int n, int kk) { return W1[(size_t)n * d + kk]; },
             [&](int m, int n, Real acc, Real) {
@@ -183,10 +213,12 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_ke
                     A[e] = silu_f(Z1[e]) * acc;
                 });
         }
+        BPROF(2);
         G.template run<1, true, true>(
             2 * len, d, h, [&](int m, int kk, Real& a0, Real& a1) { a0 = A[(size_t)m * h + kk]; },
             [&](int n, int kk) { return Wl[(size_t)n * h + kk]; },
             [&](int m, int n, Real acc, Real) { U[(size_t)m * d + n] = acc; });
+        BPROF(3);
         for (int m = warp + rank * (NT / 32); m < 2 * len; m += (NT / 32) * CL) {
             Real* u = U + (size_t)m * d;
             const Real r = warp_layernorm(u, u, d, eps);
@@ -213,6 +245,7 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_ke
             }
         }
         phase_sync(CL);
+        BPROF(4);
         G.template run<1, true, false>(
             len, h, d, [&](int m, int kk, Real& a0, Real& a1) { a0 = Pu[(size_t)m * d + kk]; },
             [&](int n, int kk) { return Wl[(size_t)kk * h + n]; },
@@ -227,10 +260,12 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_ke
                 }
             });
 
+        BPROF(5);
         // ---------------- (i) outputs o = q + LN(Wl a(q)) ----------------
         const Real* Z1q = Z1 + (size_t)len * h;
         const Real* Z2q = Z2 + (size_t)len * h;
         const Real* Aq = A + (size_t)len * h;
+        BPROF(6);
         G.template run<1, true, false>(
             len, h, d, [&](int m, int kk, Real& a0, Real& a1) { a0 = Uqb[(size_t)m * d + kk]; },
             [&](int n, int kk) { return Wl[(size_t)kk * h + n]; },
@@ -243,6 +278,7 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_ke
                     Zqb2[e] = acc * silu_f(Z1q[e]);
                 }
             });
+        BPROF(7);
         G.template run<1, true, false>(
             len, d, SW ? 2 * h : h,
             [&](int m, int kk, Real& a0, Real& a1) {
@@ -253,20 +289,24 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_ke
                 const size_t e = (size_t)m * d + n;
                 st_io(dq + (size_t)s * d, e, ld_io<Real>(doc, e) + acc);
             });
+        BPROF(8);
         G.template run<1, false, false>( // Wbl += Uqb^T Aq
             d, h, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Uqb[(size_t)t * d + m]; },
             [&](int n, int t) { return Aq[(size_t)t * h + n]; },
             [&](int m, int n, Real acc, Real) { Wb[LAST][(size_t)m * h + n] += acc; });
+        BPROF(9);
         G.template run<1, false, false>( // Wb1 += Zqb^T Q
             h, d, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Zqb[(size_t)t * h + m]; },
             [&](int n, int t) { return ld_io<Real>(qc, (size_t)t * d + n); },
             [&](int m, int n, Real acc, Real) { Wb[0][(size_t)m * d + n] += acc; });
+        BPROF(10);
         if (SW)
             G.template run<1, false, false>( // Wb2 += Zqb2^T Q
                 h, d, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Zqb2[(size_t)t * h + m]; },
                 [&](int n, int t) { return ld_io<Real>(qc, (size_t)t * d + n); },
                 [&](int m, int n, Real acc, Real) { Wb[1][(size_t)m * d + n] += acc; });
 
+        BPROF(11);
         // ---------------- (ii) state transition: carries ----------------
         Real cwb, cmb, cbb;
         {
@@ -274,30 +314,40 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_ke
 #pragma unroll
             for (int i = 0; i < NMAT; ++i) {
                 const Real* Wi = ck + (size_t)i * dh;
-                for (size_t e = tid; e < dh; e += NT) {  // every CTA sums everything: same value everywhere
+                for (size_t e = tid + (size_t)rank * NT; e < dh; e += (size_t)NT * CL) {  // this CTA's share
                     pw += T[i][e] * Wi[e];
                     pm += T[i][e] * M0[i][e];
                     pb += S[i][e] * M0[i][e];
                 }
             }
-            cwb = block_sum(pw, red);
-            cmb = block_sum(pm, red);
-            cbb = block_sum(pb, red);
+            pw = block_sum(pw, red);
+            pm = block_sum(pm, red);
+            pb = block_sum(pb, red);
+            // the shares meet in the workspace; every CTA adds them in rank order: same value everywhere
+            Real* shares = ws + lay.red;
+            if (tid == 0) { shares[3 * rank] = pw; shares[3 * rank + 1] = pm; shares[3 * rank + 2] = pb; }
+            phase_sync(CL);
+            cwb = 0; cmb = 0; cbb = 0;
+            for (int r = 0; r < CL; ++r) { cwb += shares[3 * r]; cmb += shares[3 * r + 1]; cbb += shares[3 * r + 2]; }
         }
         // G_t enters W_C with K^W_t and M_C with K^M_t: its adjoint is K^W_t T + K^M_t S.
+        BPROF(12);
         G.template run<1, true, true>( // XY2 = Ak [Tl; Sl]^T
             len, 2 * d, h, [&](int m, int kk, Real& a0, Real& a1) { a0 = A[(size_t)m * h + kk]; },
             [&](int n, int kk) { return n < d ? T[LAST][(size_t)n * h + kk] : S[LAST][(size_t)(n - d) * h + kk]; },
             [&](int m, int n, Real acc, Real) { XY2[(size_t)m * 2 * d + n] = acc; });
+        BPROF(13);
         G.template run<1, true, true>( // XY1 = K [T1; S1]^T
             len, 2 * h, d, load_k,
             [&](int n, int kk) { return n < h ? T[0][(size_t)n * d + kk] : S[0][(size_t)(n - h) * d + kk]; },
             [&](int m, int n, Real acc, Real) { XY1[(size_t)m * 2 * h + n] = acc; });
+        BPROF(14);
         if (SW)
             G.template run<1, true, true>( // XY1b = K [T2; S2]^T
                 len, 2 * h, d, load_k,
                 [&](int n, int kk) { return n < h ? T[1][(size_t)n * d + kk] : S[1][(size_t)(n - h) * d + kk]; },
                 [&](int m, int n, Real acc, Real) { XY1b[(size_t)m * 2 * h + n] = acc; });
+        BPROF(15);
         for (int t = warp + rank * (NT / 32); t < len; t += (NT / 32) * CL) {
             const Real* x2 = XY2 + (size_t)t * 2 * d;
             const Real* x1 = XY1 + (size_t)t * 2 * h;
@@ -325,7 +375,9 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_ke
             }
         }
         phase_sync(CL);
+        BPROF(16);
         // ---------------- (iii) per-token gradients G_t = -(pz1 k^T, [pz2 k^T,] pu a^T) ----------------
+        BPROF(17);
         G.template run<1, true, false>( // Akb = -[kW Pu | kM Pu] [Tl; Sl]
             len, h, 2 * d,
             [&](int m, int kk, Real& a0, Real& a1) {
@@ -333,6 +385,7 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_ke
             },
             [&](int n, int kk) { return kk < d ? T[LAST][(size_t)kk * h + n] : S[LAST][(size_t)(kk - d) * h + n]; },
             [&](int m, int n, Real acc, Real) { Akb[(size_t)m * h + n] = -acc; });
+        BPROF(18);
         G.template run<1, true, false>( // Kb = -[kW Pz1 | kM Pz1] [T1; S1]
             len, d, 2 * h,
             [&](int m, int kk, Real& a0, Real& a1) {
@@ -340,6 +393,7 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_ke
             },
             [&](int n, int kk) { return kk < h ? T[0][(size_t)kk * d + n] : S[0][(size_t)(kk - h) * d + n]; },
             [&](int m, int n, Real acc, Real) { Kb[(size_t)m * d + n] = -acc; });
+        BPROF(19);
         if (SW)
             G.template run<1, true, false>( // Kb -= [kW Pz2 | kM Pz2] [T2; S2]
                 len, d, 2 * h,
@@ -349,6 +403,7 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_ke
                 [&](int n, int kk) { return kk < h ? T[1][(size_t)kk * d + n] : S[1][(size_t)(kk - h) * d + n]; },
                 [&](int m, int n, Real acc, Real) { Kb[(size_t)m * d + n] -= acc; });
         // back through pz: Pzb becomes the adjoint of ph; Zkb (Zkb2) start with the second-order terms
+        BPROF(20);
         for (size_t e = tid + (size_t)rank * NT; e < (size_t)len * h; e += (size_t)NT * CL) {
             const Real z1 = Z1[e], ph = Pa[e];
             if (!SW) {
@@ -365,15 +420,18 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_ke
         phase_sync(CL);
         const Real* Phb = Pzb;
         // ph = Wl^T pu
+        BPROF(21);
         G.template run<1, true, true>(
             len, d, h, [&](int m, int kk, Real& a0, Real& a1) { a0 = Phb[(size_t)m * h + kk]; },
             [&](int n, int kk) { return Wl[(size_t)n * h + kk]; },
             [&](int m, int n, Real acc, Real) { Pub[(size_t)m * d + n] += acc; });
+        BPROF(22);
         G.template run<1, false, false>( // Wbl += Pu^T Phb
             d, h, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Pu[(size_t)t * d + m]; },
             [&](int n, int t) { return Phb[(size_t)t * h + n]; },
             [&](int m, int n, Real acc, Real) { Wb[LAST][(size_t)m * h + n] += acc; });
         // pu = J(u) e, e = k + y - v, y = LN(u)
+        BPROF(23);
         for (int t = warp + rank * (NT / 32); t < len; t += (NT / 32) * CL) {
             const size_t row = (size_t)t * d;
             const Real* y = U + row;
@@ -400,6 +458,7 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_ke
         }
         phase_sync(CL);
         // u = Wl a ; a = gelu(z1)  or  silu(z1) z2
+        BPROF(24);
         G.template run<1, true, false>(
             len, h, d, [&](int m, int kk, Real& a0, Real& a1) { a0 = Ukb[(size_t)m * d + kk]; },
             [&](int n, int kk) { return Wl[(size_t)kk * h + n]; },
@@ -413,11 +472,13 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_ke
                     Zkb2[e] += ab * silu_f(Z1[e]);
                 }
             });
+        BPROF(25);
         G.template run<1, false, false>( // Wbl += Ukb^T Ak
             d, h, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Ukb[(size_t)t * d + m]; },
             [&](int n, int t) { return A[(size_t)t * h + n]; },
             [&](int m, int n, Real acc, Real) { Wb[LAST][(size_t)m * h + n] += acc; });
         // z1 = W1 k (, z2 = W2 k)
+        BPROF(26);
         G.template run<1, true, false>(
             len, d, SW ? 2 * h : h,
             [&](int m, int kk, Real& a0, Real& a1) {
@@ -428,16 +489,19 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_ke
                 const size_t e = (size_t)m * d + n;
                 st_io(dk + (size_t)s * d, e, Kb[e] + acc);
             });
+        BPROF(27);
         G.template run<1, false, false>( // Wb1 += Zkb^T K
             h, d, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Zkb[(size_t)t * h + m]; },
             [&](int n, int t) { return ld_io<Real>(kc, (size_t)t * d + n); },
             [&](int m, int n, Real acc, Real) { Wb[0][(size_t)m * d + n] += acc; });
+        BPROF(28);
         if (SW)
             G.template run<1, false, false>( // Wb2 += Zkb2^T K
                 h, d, len, [&](int m, int t, Real& a0, Real& a1) { a0 = Zkb2[(size_t)t * h + m]; },
                 [&](int n, int t) { return ld_io<Real>(kc, (size_t)t * d + n); },
                 [&](int m, int n, Real acc, Real) { Wb[1][(size_t)m * d + n] += acc; });
 
+        BPROF(29);
         // ---------------- adjoints of the chunk-start state ----------------
         {
             const Real cw = sc.cw, cm = sc.cm, cb = sc.cb;
@@ -449,31 +513,53 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_ke
                     S[i][e] = cm * t + cb * sv;
                 }
         }
+        BPROF(30);
         // ---------------- (iv) reverse of the suffix scans ----------------
-        if (tid == 0 && rank == 0) {
-            Real Sb = 0, btb = cbb, gtb = cwb; // adjoints of S_0 (unused), bt_0, gt_0
-            for (int t = 0; t < len; ++t) {
-                // index t: state t; token t+1 lives at array index t
-                const Real b1 = (Real)beta[s + t], g1 = (Real)gamma[s + t], e1 = (Real)eta[s + t];
-                const Real kWb = kWb_g[t], kMb = kMb_g[t];
-                // S_t = beta_{t+1} S_{t+1} + gt_t ; bt_t = beta_{t+1} bt_{t+1} ; gt_t = gamma_{t+1} gt_{t+1}
-                gtb += Sb;
-                Real bb = Sb * sc.S[t + 1] + btb * sc.bt[t + 1];
-                Real Sb_next = Sb * b1;
-                Real btb_next = btb * b1;
-                const Real gb = gtb * sc.gt[t + 1];
-                Real gtb_next = gtb * g1;
-                if (t == 0) { // cm = beta_1 S_1
-                    bb += cmb * sc.S[1];
-                    Sb_next += cmb * b1;
+        // One thread walks the chunk (a 3-term linear recurrence, ~10 flop per token); its operands are brought into
+        // shared memory by the whole CTA first and its results leave the same way, so the walk itself never waits
+        // for global memory.
+        if (rank == 0) {
+            Real* r_beta = rev, *r_gamma = rev + kMaxC, *r_eta = rev + 2 * kMaxC, *r_kWb = rev + 3 * kMaxC,
+                 *r_kMb = rev + 4 * kMaxC, *r_de = rev + 5 * kMaxC, *r_db = rev + 6 * kMaxC, *r_dg = rev + 7 * kMaxC;
+            for (int t = tid; t < len; t += NT) {
+                r_beta[t] = (Real)beta[s + t];
+                r_gamma[t] = (Real)gamma[s + t];
+                r_eta[t] = (Real)eta[s + t];
+                r_kWb[t] = kWb_g[t];
+                r_kMb[t] = kMb_g[t];
+            }
+            __syncthreads();
+            if (tid == 0) {
+                Real Sb = 0, btb = cbb, gtb = cwb; // adjoints of S_0 (unused), bt_0, gt_0
+                for (int t = 0; t < len; ++t) {
+                    // index t: state t; token t+1 lives at array index t
+                    const Real b1 = r_beta[t], g1 = r_gamma[t], e1 = r_eta[t];
+                    const Real kWb = r_kWb[t], kMb = r_kMb[t];
+                    // S_t = beta_{t+1} S_{t+1} + gt_t ; bt_t = beta_{t+1} bt_{t+1} ; gt_t = gamma_{t+1} gt_{t+1}
+                    gtb += Sb;
+                    Real bb = Sb * sc.S[t + 1] + btb * sc.bt[t + 1];
+                    Real Sb_next = Sb * b1;
+                    Real btb_next = btb * b1;
+                    const Real gb = gtb * sc.gt[t + 1];
+                    Real gtb_next = gtb * g1;
+                    if (t == 0) { // cm = beta_1 S_1
+                        bb += cmb * sc.S[1];
+                        Sb_next += cmb * b1;
+                    }
+                    // K^M_{t+1} = eta bt_{t+1}, K^W_{t+1} = eta S_{t+1}
+                    r_de[t] = kMb * sc.bt[t + 1] + kWb * sc.S[t + 1];
+                    btb_next += kMb * e1;
+                    Sb_next += kWb * e1;
+                    r_db[t] = bb;
+                    r_dg[t] = gb;
+                    Sb = Sb_next; btb = btb_next; gtb = gtb_next;
                 }
-                // K^M_{t+1} = eta bt_{t+1}, K^W_{t+1} = eta S_{t+1}
-                d_eta[s + t] = (float)(kMb * sc.bt[t + 1] + kWb * sc.S[t + 1]);
-                btb_next += kMb * e1;
-                Sb_next += kWb * e1;
-                d_beta[s + t] = (float)bb;
-                d_gamma[s + t] = (float)gb;
-                Sb = Sb_next; btb = btb_next; gtb = gtb_next;
+            }
+            __syncthreads();
+            for (int t = tid; t < len; t += NT) {
+                d_eta[s + t] = (float)r_de[t];
+                d_beta[s + t] = (float)r_db[t];
+                d_gamma[s + t] = (float)r_dg[t];
             }
         }
         phase_sync(CL);
@@ -493,8 +579,8 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_ke
 
 template <typename Real, typename IO, int KIND, bool TC>
 static int launch_bwd(const SimtBwdArgs& a, cudaStream_t st) {
-    using Engine = typename std::conditional<TC, TcGemm, FmaGemm<Real>>::type;
-    constexpr size_t smem = Engine::kBytes + sizeof(ChunkScalars<Real>) + 16 * sizeof(Real) + (TC ? 1024 : 0);
+    using Engine = typename std::conditional<TC, TcGemmT<true>, FmaGemm<Real>>::type;
+    constexpr size_t smem = Engine::kBytes + sizeof(ChunkScalars<Real>) + (16 + 8 * kMaxC) * sizeof(Real) + (TC ? 1024 : 0);
     static bool attr_done[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return (int)cudaGetLastError();

@@ -35,7 +35,7 @@ template <typename Real, typename IO, int KIND, bool TC>
 __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_fwd_kernel(const SimtFwdArgs a) {
     constexpr int NMAT = (KIND == 0) ? 2 : 3;
     constexpr int LAST = NMAT - 1;
-    using Engine = typename std::conditional<TC, TcGemm, FmaGemm<Real>>::type;
+    using Engine = typename std::conditional<TC, TcGemmT<false>, FmaGemm<Real>>::type;
     constexpr int NT = Engine::kThreads;  // threads per CTA
     extern __shared__ __align__(16) unsigned char simt_smem_raw[];
     unsigned char* smem_base = Engine::align(simt_smem_raw);
@@ -50,6 +50,7 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_fwd_ke
     const size_t dh = (size_t)d * h;
     const SimtLayout& lay = a.lay;
     Real* ws = reinterpret_cast<Real*>(a.ws) + (size_t)seq * lay.per_seq;
+    G.set_scratch(ws + lay.splitk);
     const IO* q = reinterpret_cast<const IO*>(a.q) + (size_t)seq * L * d;
     const IO* k = reinterpret_cast<const IO*>(a.k) + (size_t)seq * L * d;
     const IO* v = reinterpret_cast<const IO*>(a.v) + (size_t)seq * L * d;
@@ -257,7 +258,7 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_fwd_ke
 
 template <typename Real, typename IO, int KIND, bool TC>
 static int launch_fwd(const SimtFwdArgs& a, cudaStream_t st) {
-    using Engine = typename std::conditional<TC, TcGemm, FmaGemm<Real>>::type;
+    using Engine = typename std::conditional<TC, TcGemmT<false>, FmaGemm<Real>>::type;
     constexpr size_t smem = Engine::kBytes + sizeof(ChunkScalars<Real>) + (TC ? 1024 : 0);
     static bool attr_done[64];
     int dev = 0;

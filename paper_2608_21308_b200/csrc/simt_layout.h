@@ -18,6 +18,7 @@ struct SimtLayout {
     size_t XY1b, Pzb2, Zkb2, Zqb2;  // SwiGLU only: the second [h x d] matrix
     size_t rk, rq, red;  // per-row 1/std of the two LN calls; small reduction scratch
     size_t kWb, kMb;     // adjoints of the scalar kernels, one per token of the chunk
+    size_t splitk;       // split-K partial sums of the tensor-core GEMM engine (2 * 8 * 128 * 64 elements)
     size_t rown;         // [nchunks][3][max(d,h)] row norms of the chunk-end weights before their normalisation
     size_t ckpt;         // [nchunks + 1][2][nmat][d*h] chunk-start (W, M) and, last, the final state; when states are saved
     size_t per_seq;      // elements per sequence
@@ -46,6 +47,7 @@ inline SimtLayout simt_layout(int d, int h, int C, int nmat, int nchunks, bool s
         l.rk = take(C); l.rq = take(C); l.red = take(64);
         l.kWb = take(C); l.kMb = take(C);
     }
+    l.splitk = take((size_t)2 * 8 * 128 * 64);
     l.rown = take(save_states ? (size_t)nchunks * 3 * (size_t)(d > h ? d : h) : 0);
     l.ckpt = take(save_states ? (size_t)(nchunks + 1) * 2 * nmat * dh : 0);
     l.per_seq = o;

@@ -35,6 +35,7 @@ template <typename Real> struct FmaGemm {
         nranks = nranks_;
     }
     __device__ void teardown() {}
+    __device__ void set_scratch(Real*) {}
     template <int NACC, bool A_KFAST, bool B_KFAST, typename FA, typename FB, typename FP, typename FE>
     __device__ void run_rmw(int M, int N, int K, FA fa, FB fb, FP pre, FE epi) {
         block_gemm<Real, NACC, A_KFAST, B_KFAST>(M, N, K, fa, fb, pre, epi, sm, rank, nranks);
@@ -54,12 +55,18 @@ template <typename Real> struct FmaGemm {
 // The contraction runs in slices of 64 k.  A slice of an operand is one "slab": rows of 128 bytes (64 bf16),
 // 16-byte chunk c of row r stored at chunk position c ^ (r & 7) (the 128-byte swizzle of the MMA descriptors).
 // Two stages: while the tensor core works on one slice, all threads stage the next.
+// Split-K: a product with fewer output tiles than CTAs in the cluster (a [tokens x d] result with a long contraction)
+// is cut along k into as many parts as there are idle CTAs; every part writes its raw accumulators to a scratch area
+// of the workspace, and after a phase barrier all CTAs sum the parts in a fixed order (so the result does not depend
+// on timing) and run the epilogue elementwise.
 constexpr int kTgStages = 2;
 constexpr int kTgBN = 128;
 constexpr int kTgBM = 64;
 constexpr int kTgBK = 64;
 constexpr uint32_t kTgTmemCols = 128;  // two accumulators of 64 columns
 constexpr int kTgThreads = 512;        // 16 warps: four per tensor-memory lane quadrant, 16 accumulator columns each
+constexpr int kTgMaxParts = 8;         // split-K: parts x tiles <= 8 (the largest cluster)
+constexpr size_t kTgScratchElems = (size_t)2 * kTgMaxParts * kTgBN * kTgBM;  // floats per sequence
 
 struct __align__(1024) TcGemmSmem {
     uint8_t R[kTgStages][2][kTgBN * 128];      // fb operand, row = n; [hi, lo]
@@ -138,7 +145,8 @@ __device__ long long g_tg_prof[16];
 #define TGPROF_START()
 #endif
 
-struct TcGemm {
+// SPLITK = false compiles the split-K path out (the forward kernel: its clusters are small and its code size matters).
+template <bool SPLITK> struct TcGemmT {
     static constexpr int kThreads = kTgThreads;
     static constexpr size_t kBytes = sizeof(TcGemmSmem);
     TcGemmSmem* sm;
@@ -146,6 +154,9 @@ struct TcGemm {
     uint32_t it;  // slices issued so far by this CTA: slice `it` uses stage it & 1 and is that stage's (it >> 1)-th use
     sm100::WaitCtx wc;
     int rank, nranks;
+    float* scratch;  // split-K partial sums of this sequence (kTgScratchElems floats), or nullptr: no split-K
+
+    __device__ void set_scratch(float* p) { scratch = p; }
 
     // the slabs need 1024-byte alignment; the dynamic shared memory carries 1024 bytes of slack for it
     __device__ static unsigned char* align(unsigned char* raw) {
@@ -157,6 +168,7 @@ struct TcGemm {
         rank = rank_;
         nranks = nranks_;
         it = 0;
+        scratch = nullptr;
         if (threadIdx.x == 0) {
             for (int s = 0; s < kTgStages; ++s) sm100::mbar_init(&sm->bar[s], 1);
             sm->dead = 0;
@@ -190,13 +202,27 @@ struct TcGemm {
         using namespace sm100;
         const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
         const uint32_t idesc = make_idesc(kTgBN, kTgBM, false, false);
-        int tile = 0;
+        const int tiles_m = (M + kTgBM - 1) / kTgBM, tiles = ((N + kTgBN - 1) / kTgBN) * tiles_m;
+        const int nslab = (K + kTgBK - 1) / kTgBK;
+        int parts = 1;
+        if (SPLITK && scratch && tiles < nranks && nslab >= 2) parts = min(min(nranks / tiles, nslab), kTgMaxParts / tiles);
+        if (parts < 1) parts = 1;
+        const int slabs_per_part = (nslab + parts - 1) / parts;
         TGPROF_START();
-        for (int n0 = 0; n0 < N; n0 += kTgBN) {
-            for (int m0 = 0; m0 < M; m0 += kTgBM, ++tile) {
-                if (tile % nranks != rank) continue;
+        for (int w = rank; w < tiles * parts; w += nranks) {  // work item = (tile, k part)
+            const int tile = w / parts, part = w - tile * parts;
+            const int n0 = (tile / tiles_m) * kTgBN, m0 = (tile % tiles_m) * kTgBM;
+            const int kbeg = part * slabs_per_part * kTgBK, kend = min(K, kbeg + slabs_per_part * kTgBK);
+            if (SPLITK && kbeg >= kend) {  // an empty part (more parts than slices): its partial sum is zero
+                for (int e = tid; e < NACC * kTgBM * kTgBN; e += kTgThreads) {
+                    const int acc = e / (kTgBM * kTgBN), r = e - acc * (kTgBM * kTgBN);
+                    scratch[((size_t)(acc * kTgMaxParts + part * tiles + tile)) * (kTgBM * kTgBN) + r] = 0.0f;
+                }
+                continue;
+            }
+            {
                 uint32_t last_it = 0;
-                for (int k0 = 0; k0 < K; k0 += kTgBK) {
+                for (int k0 = kbeg; k0 < kend; k0 += kTgBK) {
                     const uint32_t s = it & 1u;
                     // the MMAs of the slice that used this stage two slices ago have read it
                     if (it >= 2) mbar_wait(&sm->bar[s], ((it >> 1) - 1u) & 1u, wc, 200 + 1);
@@ -230,7 +256,7 @@ struct TcGemm {
                                 const uint64_t db_hi = make_smem_desc(smem_u32(sm->Cc[s][acc][0]) + 32u * k, 16, 1024);
                                 const uint64_t db_lo = make_smem_desc(smem_u32(sm->Cc[s][acc][1]) + 32u * k, 16, 1024);
                                 const uint32_t dst = tmem + (uint32_t)(acc * kTgBM);
-                                umma_bf16(dst, da_lo, db_hi, idesc, k0 > 0 || k > 0);  // small terms first
+                                umma_bf16(dst, da_lo, db_hi, idesc, k0 > kbeg || k > 0);  // small terms first
                                 umma_bf16(dst, da_hi, db_lo, idesc, true);
                                 umma_bf16(dst, da_hi, db_hi, idesc, true);
                             }
@@ -252,8 +278,17 @@ struct TcGemm {
                     tmem_ld16(taddr, acc0);
                     if (NACC == 2) tmem_ld16(taddr + kTgBM, acc1);
                     tmem_wait_ld();
-                    const int n = n0 + 32 * qd + lane;
-                    if (n < N) {
+                    const int nl = 32 * qd + lane;
+                    const int n = n0 + nl;
+                    if (SPLITK && parts > 1) {
+                        // raw partial sums: [accumulator][part x tile][m (64)][n (128)], coalesced over the lanes
+                        float* dst = scratch + ((size_t)(part * tiles + tile)) * (kTgBM * kTgBN) + (size_t)(16 * grp) * kTgBN + nl;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            dst[(size_t)j * kTgBN] = __uint_as_float(acc0[j]);
+                            if (NACC == 2) dst[(size_t)kTgMaxParts * (kTgBM * kTgBN) + (size_t)j * kTgBN] = __uint_as_float(acc1[j]);
+                        }
+                    } else if (n < N) {
                         using P = decltype(pre(0, 0));
                         constexpr int kBatch = 8;
 #pragma unroll
@@ -279,6 +314,45 @@ struct TcGemm {
                 __syncthreads();  // the accumulators may be overwritten by the next tile
                 tc_fence_after_sync();
                 TGPROF(7);
+            }
+        }
+        if (SPLITK && parts > 1) {
+            // every part is in the scratch area: sum them in part order and run the epilogue, elementwise over all CTAs
+            phase_sync(nranks);
+            using P = decltype(pre(0, 0));
+            constexpr int kBatch = 4;
+            const int total = tiles * kTgBM * kTgBN;
+            const int stride = kTgThreads * nranks;
+            for (int e0 = tid + rank * kTgThreads; e0 < total; e0 += stride * kBatch) {
+                P p[kBatch];
+                float s0[kBatch], s1[kBatch];
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u) {
+                    const int e = e0 + u * stride;
+                    s0[u] = 0.0f;
+                    s1[u] = 0.0f;
+                    if (e < total) {
+                        const int tile = e / (kTgBM * kTgBN), r = e - tile * (kTgBM * kTgBN);
+                        const int m = (tile % tiles_m) * kTgBM + r / kTgBN, n = (tile / tiles_m) * kTgBN + r % kTgBN;
+                        if (m < M && n < N) {
+                            for (int part = 0; part < parts; ++part) {
+                                const float* src = scratch + ((size_t)(part * tiles + tile)) * (kTgBM * kTgBN) + r;
+                                s0[u] += src[0];
+                                if (NACC == 2) s1[u] += src[(size_t)kTgMaxParts * (kTgBM * kTgBN)];
+                            }
+                            p[u] = pre(m, n);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u) {
+                    const int e = e0 + u * stride;
+                    if (e < total) {
+                        const int tile = e / (kTgBM * kTgBN), r = e - tile * (kTgBM * kTgBN);
+                        const int m = (tile % tiles_m) * kTgBM + r / kTgBN, n = (tile / tiles_m) * kTgBN + r % kTgBN;
+                        if (m < M && n < N) epi(m, n, s0[u], s1[u], p[u]);
+                    }
+                }
             }
         }
         phase_sync(nranks);
