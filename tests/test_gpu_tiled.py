@@ -74,3 +74,15 @@ def test_tiled_is_the_default_for_bf16_shapes_without_a_fused_kernel_and_is_repe
         assert np.array_equal(a["W"][i], b["W"][i]) and np.array_equal(a["M"][i], b["M"][i])
     with pytest.raises(Exception):
         util.gpu_forward(x, impl=E.E2TTT_IMPL_TILED, d=r.d, h=r.h, C=r.C, kind=r.kind, io="f32")
+
+
+@pytest.mark.parametrize("kind,h", [(SWIGLU, 384), (MLP, 512)])
+def test_tiled_free_running_paper_regime_at_benchmark_shapes(kind, h):
+    """16 chunks free-running under the paper's gate regime (where the recurrence is well conditioned), d = 128."""
+    r = inputs.paper_regime(inputs.Recipe(B=3, H=1, L=1024, d=128, h=h, C=64, kind=kind, io="bf16", seed=4, m_std=0.002))
+    x = inputs.generate(r)
+    ref = util.oracle_forward(x, 64, kind)
+    got, hd = util.gpu_forward(x, impl=E.E2TTT_IMPL_TILED, **_shape(r))
+    assert E.e2ttt_device_status(hd["ws"]) == 0
+    errs = check_forward(got, ref, TOL_BF16, "tiled paper regime, 16 chunks free-running")
+    print(kind, errs)
