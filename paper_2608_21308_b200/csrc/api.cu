@@ -115,7 +115,7 @@ int e2ttt_workspace_bytes_normed(const e2ttt_params* p, int save_states, size_t*
     if (!bytes) return E2TTT_ERR_NULL;
     int rc = check_params(p);
     if (rc) return rc;
-    if (p->impl == E2TTT_IMPL_TCGEN05) return E2TTT_ERR_SHAPE;
+    if (p->impl == E2TTT_IMPL_TCGEN05 && (save_states || !has_tcgen05(p, false))) return E2TTT_ERR_SHAPE;
     *bytes = simt_bytes(p, save_states != 0, save_states != 0);
     return E2TTT_OK;
 }
@@ -139,12 +139,15 @@ static int fwd_common(const e2ttt_params* p, const void* q, const void* k, const
     if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(o, 16)) return E2TTT_ERR_ALIGN;
     size_t need = 0;
     if (row_norm) {
-        // the fused kernel has no normalisation step: the any-shape kernels serve the call
-        if (p->impl == E2TTT_IMPL_TCGEN05 || !(norm_eps >= 0.0f)) return E2TTT_ERR_SHAPE;
+        // the fused kernel normalises, but does not write the saved-state layout of the normalised reverse pass
+        if (!(norm_eps >= 0.0f)) return E2TTT_ERR_SHAPE;
         for (int i = 0; i < nmat; ++i)
             if (!row_norm[i]) return E2TTT_ERR_NULL;
-        if (impl == E2TTT_IMPL_TCGEN05) impl = E2TTT_IMPL_TILED;
-        need = simt_bytes(p, save_states != 0, save_states != 0);
+        if (impl == E2TTT_IMPL_TCGEN05 && save_states) {
+            if (p->impl == E2TTT_IMPL_TCGEN05) return E2TTT_ERR_SHAPE;
+            impl = E2TTT_IMPL_TILED;
+        }
+        need = simt_bytes(p, save_states != 0, save_states != 0);  // the size e2ttt_workspace_bytes_normed reports
     } else {
         rc = e2ttt_workspace_bytes(p, save_states, &need);
         if (rc) return rc;
@@ -164,6 +167,7 @@ static int fwd_common(const e2ttt_params* p, const void* q, const void* k, const
         t.M1_init = M_init ? M_init[0] : nullptr; t.M2_init = M_init ? M_init[1] : nullptr;
         t.W1_final = W_final[0]; t.W2_final = W_final[1]; t.M1_final = M_final[0]; t.M2_final = M_final[1];
         t.status = static_cast<int*>(workspace);
+        if (row_norm) { t.norm1 = row_norm[0]; t.norm2 = row_norm[1]; t.norm_eps = norm_eps; }
         if (save_states) {
             const SimtLayout lay = simt_layout(p->d, p->h, p->C, nmat, p->L / p->C, true, true);
             t.ckpt = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBytes) + lay.ckpt;

@@ -65,7 +65,7 @@ struct __align__(1024) Smem {
     uint8_t PzM[2][8192];  // kM_t pz                                                 staging slot 1
     uint8_t Stage2[16384]; // staging slot 2
     Scalars sc[2];
-    uint64_t bar_x, bar_g1, bar_g2, bar_g3, bar_agg, bar_agg2, bar_ak, bar_v, bar_ksent, bar_partK, bar_partQ, bar_pu, bar_credit;
+    uint64_t bar_x, bar_g1, bar_g2, bar_g3, bar_agg, bar_agg2, bar_ak, bar_v, bar_ksent, bar_partK, bar_partQ, bar_pu, bar_credit, bar_rs;
     uint32_t tmem_base;
     int dead;
 };
@@ -160,7 +160,10 @@ __device__ __forceinline__ void st_slab16(uint8_t* slab, int row, int col0, cons
 }
 
 // PAD = false: the native 128 x 512 shape, every mask folds away.  PAD = true: d and h come from the arguments.
-template <bool PAD>
+// NORM = true: post-chunk normalisation - after the state transition every row of W1 and of W2 is rescaled to its
+// target norm.  A row of W1c lives in one CTA (its 128 columns spread over the 4 column-group warps); a row of W2
+// spans the 4 CTAs, so its sum of squares crosses the cluster once per chunk.
+template <bool PAD, bool NORM>
 __global__ void __launch_bounds__(NTHREADS, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
               const __grid_constant__ CUtensorMap tmV, const TcFwdArgs a) {
@@ -189,6 +192,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     const size_t dh = (size_t)de * he;
     const bool cta_real = HC * (int)me < he;  // this CTA's 128 hidden units exist
     const float inv_d = 1.0f / (float)de;
+    // normalisation targets of this thread's rows: hidden unit 128 me + row of W1, output row `row` of W2
+    const float tgt1 = (NORM && cta_real) ? a.norm1[(size_t)seq * he + HC * me + row] : 0.0f;
+    const float tgt2 = (NORM && row < de) ? a.norm2[(size_t)seq * de + row] : 0.0f;
     __nv_bfloat16* go = a.o + (size_t)seq * L * de;
     const float* eta = a.eta + (size_t)seq * L;
     const float* beta = a.beta + (size_t)seq * L;
@@ -209,6 +215,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         mbar_init(&s.bar_ksent, 2 * NG);
         mbar_init(&s.bar_pu, 1);    // + 16 KB of pu rows per chunk
         mbar_init(&s.bar_credit, 3);
+        mbar_init(&s.bar_rs, 1);    // + 3 x 512 B of peer row sums per chunk (normalisation only)
         fence_mbar_init();
         tma_prefetch_desc(&tmK);
         tma_prefetch_desc(&tmQ);
@@ -342,6 +349,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             mbar_expect_tx(&s.bar_partK, 3 * 8192);  // this chunk's incoming partial sums and pu rows
             mbar_expect_tx(&s.bar_partQ, 3 * 8192);
             mbar_expect_tx(&s.bar_pu, 16384);
+            if (NORM) mbar_expect_tx(&s.bar_rs, 3 * 512);
         }
         mbar_wait(&s.bar_g1, ph, wc, 100 + 2);
         PROF(1);
@@ -661,6 +669,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         }
         __syncwarp();
         // ---------------- state pass, W1 half (Algorithm 1 lines 6-7), while the M2 aggregation still runs
+        float ss1 = 0.0f;
 #pragma unroll
         for (int b = 0; b < NB; ++b) {
             const int col = c0 + 16 * b;
@@ -674,20 +683,60 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 const float m0 = M1[16 * b + j];
                 wn[j] = __uint_as_float(wa[j]) + cm * m0;
                 M1[16 * b + j] = cb * m0 + __uint_as_float(ma[j]);
-                st[j] = __float_as_uint(cwn * wn[j]);
+                st[j] = __float_as_uint(NORM ? wn[j] : cwn * wn[j]);
+                if (NORM) ss1 = fmaf(wn[j], wn[j], ss1);
             }
             tmem_st16(lane_addr + T_W1 + col, st);
-            st_slab16(s.W1[col >> 6], row, col & 63, wn);
-            if ((last || a.ckpt) && cta_real && col < de) {  // final state, or the next chunk's start state for the backward
-                const size_t off = ((size_t)(HC * me) + row) * de + col;
-                float* ck = last ? nullptr : a.ckpt + (size_t)seq * a.ckpt_seq_stride + (size_t)(r + 1) * 4 * dh;
-                float* wf = last ? a.W1_final + head + off : ck + off;
-                float* mf = last ? a.M1_final + head + off : ck + 2 * dh + off;
+            if (!NORM) {
+                st_slab16(s.W1[col >> 6], row, col & 63, wn);
+                if ((last || a.ckpt) && cta_real && col < de) {  // final state, or the next chunk's start state for the backward
+                    const size_t off = ((size_t)(HC * me) + row) * de + col;
+                    float* ck = last ? nullptr : a.ckpt + (size_t)seq * a.ckpt_seq_stride + (size_t)(r + 1) * 4 * dh;
+                    float* wf = last ? a.W1_final + head + off : ck + off;
+                    float* mf = last ? a.M1_final + head + off : ck + 2 * dh + off;
 #pragma unroll
-                for (int j = 0; j < 16; j += 4) {
-                    *reinterpret_cast<float4*>(wf + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
-                    *reinterpret_cast<float4*>(mf + j) =
-                        make_float4(M1[16 * b + j], M1[16 * b + j + 1], M1[16 * b + j + 2], M1[16 * b + j + 3]);
+                    for (int j = 0; j < 16; j += 4) {
+                        *reinterpret_cast<float4*>(wf + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
+                        *reinterpret_cast<float4*>(mf + j) =
+                            make_float4(M1[16 * b + j], M1[16 * b + j + 1], M1[16 * b + j + 2], M1[16 * b + j + 3]);
+                    }
+                }
+            }
+        }
+        if (NORM) {
+            // row sums of squares: the four column-group warps of a row meet in shared memory (the Pz tile is dead)
+            float* rs = reinterpret_cast<float*>(s.PzW[0]);  // [NG][128]
+            rs[g * 128 + row] = ss1;
+            tmem_wait_st();
+            tc_fence_before_sync();
+            __syncthreads();
+            tc_fence_after_sync();
+            float tot = 0.0f;
+#pragma unroll
+            for (int gg = 0; gg < NG; ++gg) tot += rs[gg * 128 + row];
+            const float f = tgt1 / (sqrtf(tot) + a.norm_eps);
+#pragma unroll
+            for (int b = 0; b < NB; ++b) {
+                const int col = c0 + 16 * b;
+                uint32_t wa[16], st[16];
+                float wn[16];
+                tmem_ld16(lane_addr + T_W1 + col, wa);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    wn[j] = __uint_as_float(wa[j]) * f;
+                    st[j] = __float_as_uint(cwn * wn[j]);
+                }
+                tmem_st16(lane_addr + T_W1 + col, st);
+                st_slab16(s.W1[col >> 6], row, col & 63, wn);
+                if (last && cta_real && col < de) {
+                    const size_t off = ((size_t)(HC * me) + row) * de + col;
+#pragma unroll
+                    for (int j = 0; j < 16; j += 4) {
+                        *reinterpret_cast<float4*>(a.W1_final + head + off + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
+                        *reinterpret_cast<float4*>(a.M1_final + head + off + j) =
+                            make_float4(M1[16 * b + j], M1[16 * b + j + 1], M1[16 * b + j + 2], M1[16 * b + j + 3]);
+                    }
                 }
             }
         }
@@ -710,6 +759,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         }
         __syncwarp();
         // ---------------- state pass, W2 half
+        float ss2 = 0.0f;
 #pragma unroll
         for (int b = 0; b < NB; ++b) {
             const int col = c0 + 16 * b;
@@ -723,20 +773,85 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 const float m0 = M2[16 * b + j];
                 wn[j] = __uint_as_float(wa[j]) + cm * m0;
                 M2[16 * b + j] = cb * m0 + __uint_as_float(ma[j]);
-                st[j] = __float_as_uint(cwn * wn[j]);
+                st[j] = __float_as_uint(NORM ? wn[j] : cwn * wn[j]);
+                if (NORM) ss2 = fmaf(wn[j], wn[j], ss2);
             }
             tmem_st16(lane_addr + T_W2 + col, st);
-            st_slab16(s.W2[col >> 6], row, col & 63, wn);
-            if ((last || a.ckpt) && cta_real && row < de) {
-                const size_t off = (size_t)row * he + HC * me + col;
-                float* ck = last ? nullptr : a.ckpt + (size_t)seq * a.ckpt_seq_stride + (size_t)(r + 1) * 4 * dh;
-                float* wf = last ? a.W2_final + head + off : ck + dh + off;
-                float* mf = last ? a.M2_final + head + off : ck + 3 * dh + off;
+            if (!NORM) {
+                st_slab16(s.W2[col >> 6], row, col & 63, wn);
+                if ((last || a.ckpt) && cta_real && row < de) {
+                    const size_t off = (size_t)row * he + HC * me + col;
+                    float* ck = last ? nullptr : a.ckpt + (size_t)seq * a.ckpt_seq_stride + (size_t)(r + 1) * 4 * dh;
+                    float* wf = last ? a.W2_final + head + off : ck + dh + off;
+                    float* mf = last ? a.M2_final + head + off : ck + 3 * dh + off;
 #pragma unroll
-                for (int j = 0; j < 16; j += 4) {
-                    *reinterpret_cast<float4*>(wf + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
-                    *reinterpret_cast<float4*>(mf + j) =
-                        make_float4(M2[16 * b + j], M2[16 * b + j + 1], M2[16 * b + j + 2], M2[16 * b + j + 3]);
+                    for (int j = 0; j < 16; j += 4) {
+                        *reinterpret_cast<float4*>(wf + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
+                        *reinterpret_cast<float4*>(mf + j) =
+                            make_float4(M2[16 * b + j], M2[16 * b + j + 1], M2[16 * b + j + 2], M2[16 * b + j + 3]);
+                    }
+                }
+            }
+        }
+        if (NORM) {
+            // A row of W2 spans the cluster: the CTA's own sum of squares (over its four column-group warps) goes to
+            // every CTA, each adds the four pieces in CTA order (the same number everywhere).  The kW a tile is dead.
+            float* rs = reinterpret_cast<float*>(s.AkW[0]);          // [NG][128] this CTA's pieces
+            float* got = reinterpret_cast<float*>(s.AkW[0]) + 1024;  // [NC][128] one row-sum vector per CTA
+            rs[g * 128 + row] = ss2;
+            tmem_wait_st();
+            tc_fence_before_sync();
+            __syncthreads();
+            tc_fence_after_sync();
+            if (warp == 0) {  // 32 lanes x 4 rows
+                // a peer's receive area overlays an operand tile of its W2 aggregations: it is free once that peer
+                // has seen them finish, which is what its credit of this chunk says
+                mbar_wait<true>(&s.bar_credit, ph, wc, 100 + 14);
+                float4 v;
+                float* pv = reinterpret_cast<float*>(&v);
+#pragma unroll
+                for (int x = 0; x < 4; ++x) {
+                    float t = 0.0f;
+#pragma unroll
+                    for (int gg = 0; gg < NG; ++gg) t += rs[gg * 128 + 4 * lane + x];
+                    pv[x] = t;
+                }
+                const uint32_t local = smem_u32(got + me * 128 + 4 * lane);
+                *reinterpret_cast<float4*>(got + me * 128 + 4 * lane) = v;
+#pragma unroll
+                for (uint32_t dst = 0; dst < NC; ++dst)
+                    if (dst != me)
+                        st_async_v4(map_to_cta(local, dst), __float_as_uint(v.x), __float_as_uint(v.y), __float_as_uint(v.z),
+                                    __float_as_uint(v.w), map_to_cta(smem_u32(&s.bar_rs), dst));
+            }
+            __syncthreads();  // the CTA's own vector is in place
+            mbar_wait<true>(&s.bar_rs, ph, wc, 100 + 13);
+            float tot = 0.0f;
+#pragma unroll
+            for (uint32_t c = 0; c < NC; ++c) tot += got[c * 128 + row];
+            const float f = tgt2 / (sqrtf(tot) + a.norm_eps);
+#pragma unroll
+            for (int b = 0; b < NB; ++b) {
+                const int col = c0 + 16 * b;
+                uint32_t wa[16], st[16];
+                float wn[16];
+                tmem_ld16(lane_addr + T_W2 + col, wa);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    wn[j] = __uint_as_float(wa[j]) * f;
+                    st[j] = __float_as_uint(cwn * wn[j]);
+                }
+                tmem_st16(lane_addr + T_W2 + col, st);
+                st_slab16(s.W2[col >> 6], row, col & 63, wn);
+                if (last && cta_real && row < de) {
+                    const size_t off = (size_t)row * he + HC * me + col;
+#pragma unroll
+                    for (int j = 0; j < 16; j += 4) {
+                        *reinterpret_cast<float4*>(a.W2_final + head + off + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
+                        *reinterpret_cast<float4*>(a.M2_final + head + off + j) =
+                            make_float4(M2[16 * b + j], M2[16 * b + j + 1], M2[16 * b + j + 2], M2[16 * b + j + 3]);
+                    }
                 }
             }
         }
@@ -808,8 +923,10 @@ int tc_fwd_launch(const TcFwdArgs& a, void* stream) {
     if (cudaGetDevice(&dev) != cudaSuccess) return (int)cudaGetLastError();
     const int smem = (int)tc_fwd_smem_bytes();
     if (dev < 0 || dev >= 64 || !attr_done[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(tc_fwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_fwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        cudaError_t e = cudaFuncSetAttribute(tc_fwd_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_fwd_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_fwd_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_fwd_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return (int)e;
         if (dev >= 0 && dev < 64) attr_done[dev] = true;
     }
@@ -828,8 +945,14 @@ int tc_fwd_launch(const TcFwdArgs& a, void* stream) {
     cfg.attrs = at;
     cfg.numAttrs = 1;
     const bool native = a.d == D && a.h == NC * HC;
-    e = native ? cudaLaunchKernelEx(&cfg, tc_fwd_kernel<false>, tmK, tmQ, tmV, a)
-               : cudaLaunchKernelEx(&cfg, tc_fwd_kernel<true>, tmK, tmQ, tmV, a);
+    if (a.norm1 && a.norm2) {
+        if (a.ckpt) return (int)cudaErrorInvalidValue;  // the saved-state layout of the normalised reverse pass is not written here
+        e = native ? cudaLaunchKernelEx(&cfg, tc_fwd_kernel<false, true>, tmK, tmQ, tmV, a)
+                   : cudaLaunchKernelEx(&cfg, tc_fwd_kernel<true, true>, tmK, tmQ, tmV, a);
+    } else {
+        e = native ? cudaLaunchKernelEx(&cfg, tc_fwd_kernel<false, false>, tmK, tmQ, tmV, a)
+                   : cudaLaunchKernelEx(&cfg, tc_fwd_kernel<true, false>, tmK, tmQ, tmV, a);
+    }
     if (e != cudaSuccess) return (int)e;
     return (int)cudaGetLastError();
 }

@@ -137,11 +137,51 @@ def test_normed_backward_windows_bf16(cfg):
         assert util.rel_err(got["drow_norm"][i], ref["drow_norm"][i]) <= TOL_BF16, i
 
 
-def test_normed_calls_reject_the_fused_kernel_and_missing_targets():
+def test_normed_calls_reject_missing_targets_and_the_fused_kernel_with_saved_states():
     r = inputs.config(2, heads=[0], L=64)
     x = inputs.generate(r)
     tgt = targets(x)
-    with pytest.raises(Exception):
-        gpu_forward_normed(x, tgt, d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16", impl=E.E2TTT_IMPL_TCGEN05)
+    with pytest.raises(Exception):   # the fused kernel does not write the states the normalised reverse pass reads
+        gpu_forward_normed(x, tgt, d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16", impl=E.E2TTT_IMPL_TCGEN05, save_states=True)
     with pytest.raises(Exception):
         gpu_forward_normed(x, tgt[:1], d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16", impl=E.E2TTT_IMPL_TILED)
+
+
+# ---- the fused tensor-core forward with the normalisation in its state pass
+
+@pytest.mark.parametrize("cfg,over", [(2, {}), (1, {}), (2, dict(h=384))], ids=["128x512", "64x256-padded", "128x384-padded"])
+def test_fused_normed_forward_windows(cfg, over):
+    r = inputs.config(cfg, heads=[3, 30], m_std=0.002, **over)
+    xw, _ = util.teacher_forced_windows(r, 4, window=1)
+    tgt = targets(xw, 0.9)
+    ref = oracle_fwd(xw, tgt, r.C, r.kind)
+    got = gpu_forward_normed(xw, tgt, d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16", impl=E.E2TTT_IMPL_TCGEN05)
+    errs = check_forward(got, ref, TOL_BF16, f"fused normed fwd config {cfg} {over}")
+    for i, t in enumerate(tgt):
+        assert np.allclose(np.sqrt((got["W"][i].astype(np.float64) ** 2).sum(-1)), t, rtol=1e-3)
+    print(errs)
+
+
+def test_fused_normed_forward_free_running_and_auto_selection():
+    """16 chunks free-running under the paper's gate regime; AUTO must take the fused kernel (same bits as TCGEN05);
+    two calls of half the length chain to the same result (the final state is the normalised one)."""
+    r = inputs.paper_regime(inputs.Recipe(B=3, H=1, L=1024, d=128, h=512, C=64, kind=MLP, io="bf16", seed=4, m_std=0.002))
+    x = inputs.generate(r)
+    tgt = targets(x, 1.1)
+    ref = oracle_fwd(x, tgt, 64, MLP)
+    shape = dict(d=128, h=512, C=64, kind=MLP, io="bf16")
+    got = gpu_forward_normed(x, tgt, impl=E.E2TTT_IMPL_TCGEN05, **shape)
+    check_forward(got, ref, TOL_BF16, "fused normed, 16 chunks free-running")
+    auto = gpu_forward_normed(x, tgt, impl=E.E2TTT_IMPL_AUTO, **shape)
+    assert np.array_equal(auto["o"], got["o"]) and all(np.array_equal(a, b) for a, b in zip(auto["W"], got["W"]))
+    tiled = gpu_forward_normed(x, tgt, impl=E.E2TTT_IMPL_TILED, **shape)
+    check_forward(tiled, ref, TOL_BF16, "tiled normed")
+    half = r.L // 2
+    first = {n: (np.ascontiguousarray(v[:, :half]) if not isinstance(v, list) else v) for n, v in x.items()}
+    a = gpu_forward_normed(first, tgt, impl=E.E2TTT_IMPL_TCGEN05, **shape)
+    rest = {n: (np.ascontiguousarray(v[:, half:]) if not isinstance(v, list) else v) for n, v in x.items()}
+    rest["W"], rest["M"] = a["W"], a["M"]
+    b = gpu_forward_normed(rest, tgt, impl=E.E2TTT_IMPL_TCGEN05, **shape)
+    assert np.array_equal(np.concatenate([a["o"], b["o"]], 1), got["o"])
+    for i in range(2):
+        assert np.array_equal(b["W"][i], got["W"][i]) and np.array_equal(b["M"][i], got["M"][i])
