@@ -206,3 +206,24 @@ def test_a_failing_call_leaves_outputs_untouched():
     assert ei.value.status == -5
     torch.cuda.synchronize()
     assert float(o.min()) == 7.0
+
+
+@pytest.mark.parametrize("cfg", [1, 3, 4])
+def test_full_benchmark_sizes_status_repeatability_and_sampled_first_chunk(cfg):
+    """Configs 1, 3 and 4 at their full sizes, in the launch configuration bench.py times (impl AUTO): clean device
+    status, finite results, bitwise repeatable, and the first chunk of sampled sequences against the oracle (later
+    chunks of the benchmark gates are covered by the teacher-forced windows)."""
+    r = inputs.config(cfg)
+    x = inputs.generate(r)
+    shape = dict(d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16")
+    a, hd = util.gpu_forward(x, use_M=False, **shape)
+    assert E.e2ttt_device_status(hd["ws"]) == 0
+    assert np.isfinite(a["o"]).all() and all(np.isfinite(w).all() for w in a["W"] + a["M"])
+    b, _ = util.gpu_forward(x, use_M=False, **shape)
+    assert np.array_equal(a["o"], b["o"]) and all(np.array_equal(u, v) for u, v in zip(a["W"] + a["M"], b["W"] + b["M"]))
+    N = x["q"].shape[0]
+    heads = sorted({0, N // 3, N - 1})
+    sample = {n: (np.ascontiguousarray(v[heads, :r.C]) if not isinstance(v, list) else [m[heads] for m in v])
+              for n, v in x.items()}
+    ref = util.oracle_forward(sample, r.C, r.kind, use_M=False)
+    assert util.rel_err(a["o"][heads, :r.C], ref["o"]) <= TOL_BF16
