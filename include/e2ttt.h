@@ -165,11 +165,11 @@ E2TTT_API int e2ttt_chunk_bwd(const e2ttt_params* p,
  *                                                          of its learned initial fast weights
  *   norm_eps    in                                         >= 0
  *   d_row_norm  out (host array of nmat device pointers, or NULL)  adjoints of the targets, [B,H,rows_i] fp32
- * Everything else as in e2ttt_chunk_fwd / e2ttt_chunk_bwd.  The forward without saved states runs on the fused
- * tensor-core kernel where that serves the shape (AUTO, TCGEN05); a forward that saves states and the backward run
- * on the any-shape kernels (SIMT or TILED; TCGEN05 gives E2TTT_ERR_SHAPE there).  e2ttt_workspace_bytes_normed
- * sizes the workspace for either (the backward always needs the save_states = 1 size).  A backward with
- * states_saved = 1 needs the states of e2ttt_chunk_fwd_normed(save_states = 1) with the same targets. */
+ * Everything else as in e2ttt_chunk_fwd / e2ttt_chunk_bwd.  The forward runs on the fused tensor-core kernel
+ * where that serves the shape (AUTO, TCGEN05), the backward on the any-shape kernels (TCGEN05 means TILED
+ * there).  e2ttt_workspace_bytes_normed sizes the workspace for either (the backward always needs the
+ * save_states = 1 size).  A backward with states_saved = 1 needs the states of
+ * e2ttt_chunk_fwd_normed(save_states = 1) with the same targets. */
 E2TTT_API int e2ttt_workspace_bytes_normed(const e2ttt_params* p, int save_states, size_t* bytes);
 E2TTT_API int e2ttt_chunk_fwd_normed(const e2ttt_params* p, const void* q, const void* k, const void* v,
                                      const float* eta, const float* beta, const float* gamma,

@@ -115,7 +115,7 @@ int e2ttt_workspace_bytes_normed(const e2ttt_params* p, int save_states, size_t*
     if (!bytes) return E2TTT_ERR_NULL;
     int rc = check_params(p);
     if (rc) return rc;
-    if (p->impl == E2TTT_IMPL_TCGEN05 && (save_states || !has_tcgen05(p, false))) return E2TTT_ERR_SHAPE;
+    if (p->impl == E2TTT_IMPL_TCGEN05 && !has_tcgen05(p, false)) return E2TTT_ERR_SHAPE;
     *bytes = simt_bytes(p, save_states != 0, save_states != 0);
     return E2TTT_OK;
 }
@@ -139,14 +139,9 @@ static int fwd_common(const e2ttt_params* p, const void* q, const void* k, const
     if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(o, 16)) return E2TTT_ERR_ALIGN;
     size_t need = 0;
     if (row_norm) {
-        // the fused kernel normalises, but does not write the saved-state layout of the normalised reverse pass
         if (!(norm_eps >= 0.0f)) return E2TTT_ERR_SHAPE;
         for (int i = 0; i < nmat; ++i)
             if (!row_norm[i]) return E2TTT_ERR_NULL;
-        if (impl == E2TTT_IMPL_TCGEN05 && save_states) {
-            if (p->impl == E2TTT_IMPL_TCGEN05) return E2TTT_ERR_SHAPE;
-            impl = E2TTT_IMPL_TILED;
-        }
         need = simt_bytes(p, save_states != 0, save_states != 0);  // the size e2ttt_workspace_bytes_normed reports
     } else {
         rc = e2ttt_workspace_bytes(p, save_states, &need);
@@ -172,6 +167,7 @@ static int fwd_common(const e2ttt_params* p, const void* q, const void* k, const
             const SimtLayout lay = simt_layout(p->d, p->h, p->C, nmat, p->L / p->C, true, true);
             t.ckpt = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBytes) + lay.ckpt;
             t.ckpt_seq_stride = lay.per_seq;
+            t.rown = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBytes) + lay.rown;
         }
         return tc_fwd_launch(t, stream) == 0 ? E2TTT_OK : E2TTT_ERR_CUDA;
     }
@@ -243,7 +239,7 @@ static int bwd_common(const e2ttt_params* p, const void* q, const void* k, const
     rc = pick_impl(p, true, &impl);
     if (rc) return rc;
     if (row_norm) {
-        if (p->impl == E2TTT_IMPL_TCGEN05 || !(norm_eps >= 0.0f)) return E2TTT_ERR_SHAPE;
+        if (!(norm_eps >= 0.0f)) return E2TTT_ERR_SHAPE;
         for (int i = 0; i < nmat; ++i)
             if (!row_norm[i]) return E2TTT_ERR_NULL;
     }

@@ -729,16 +729,29 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 }
                 tmem_st16(lane_addr + T_W1 + col, st);
                 st_slab16(s.W1[col >> 6], row, col & 63, wn);
-                if (last && cta_real && col < de) {
+                if (cta_real && col < de) {
                     const size_t off = ((size_t)(HC * me) + row) * de + col;
+                    if (last) {
 #pragma unroll
-                    for (int j = 0; j < 16; j += 4) {
-                        *reinterpret_cast<float4*>(a.W1_final + head + off + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
-                        *reinterpret_cast<float4*>(a.M1_final + head + off + j) =
-                            make_float4(M1[16 * b + j], M1[16 * b + j + 1], M1[16 * b + j + 2], M1[16 * b + j + 3]);
+                        for (int j = 0; j < 16; j += 4) {
+                            *reinterpret_cast<float4*>(a.W1_final + head + off + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
+                            *reinterpret_cast<float4*>(a.M1_final + head + off + j) =
+                                make_float4(M1[16 * b + j], M1[16 * b + j + 1], M1[16 * b + j + 2], M1[16 * b + j + 3]);
+                        }
+                    }
+                    if (a.ckpt) {  // the state after this chunk: slot r + 1 (the last slot is the final state)
+                        float* ck = a.ckpt + (size_t)seq * a.ckpt_seq_stride + (size_t)(r + 1) * 4 * dh;
+#pragma unroll
+                        for (int j = 0; j < 16; j += 4) {
+                            *reinterpret_cast<float4*>(ck + off + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
+                            *reinterpret_cast<float4*>(ck + 2 * dh + off + j) =
+                                make_float4(M1[16 * b + j], M1[16 * b + j + 1], M1[16 * b + j + 2], M1[16 * b + j + 3]);
+                        }
                     }
                 }
             }
+            if (a.ckpt && g == 0 && cta_real)  // row norm before the normalisation, for the reverse pass
+                a.rown[(size_t)seq * a.ckpt_seq_stride + ((size_t)r * 3 + 0) * (size_t)max(de, he) + HC * me + row] = sqrtf(tot);
         }
         tmem_wait_st();
         fence_proxy_async_smem();
@@ -844,16 +857,29 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 }
                 tmem_st16(lane_addr + T_W2 + col, st);
                 st_slab16(s.W2[col >> 6], row, col & 63, wn);
-                if (last && cta_real && row < de) {
+                if (cta_real && row < de) {
                     const size_t off = (size_t)row * he + HC * me + col;
+                    if (last) {
 #pragma unroll
-                    for (int j = 0; j < 16; j += 4) {
-                        *reinterpret_cast<float4*>(a.W2_final + head + off + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
-                        *reinterpret_cast<float4*>(a.M2_final + head + off + j) =
-                            make_float4(M2[16 * b + j], M2[16 * b + j + 1], M2[16 * b + j + 2], M2[16 * b + j + 3]);
+                        for (int j = 0; j < 16; j += 4) {
+                            *reinterpret_cast<float4*>(a.W2_final + head + off + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
+                            *reinterpret_cast<float4*>(a.M2_final + head + off + j) =
+                                make_float4(M2[16 * b + j], M2[16 * b + j + 1], M2[16 * b + j + 2], M2[16 * b + j + 3]);
+                        }
+                    }
+                    if (a.ckpt) {
+                        float* ck = a.ckpt + (size_t)seq * a.ckpt_seq_stride + (size_t)(r + 1) * 4 * dh;
+#pragma unroll
+                        for (int j = 0; j < 16; j += 4) {
+                            *reinterpret_cast<float4*>(ck + dh + off + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
+                            *reinterpret_cast<float4*>(ck + 3 * dh + off + j) =
+                                make_float4(M2[16 * b + j], M2[16 * b + j + 1], M2[16 * b + j + 2], M2[16 * b + j + 3]);
+                        }
                     }
                 }
             }
+            if (a.ckpt && g == 0 && me == 0 && row < de)
+                a.rown[(size_t)seq * a.ckpt_seq_stride + ((size_t)r * 3 + 1) * (size_t)max(de, he) + row] = sqrtf(tot);
         }
         tmem_wait_st();
         fence_proxy_async_smem();
@@ -946,7 +972,7 @@ int tc_fwd_launch(const TcFwdArgs& a, void* stream) {
     cfg.numAttrs = 1;
     const bool native = a.d == D && a.h == NC * HC;
     if (a.norm1 && a.norm2) {
-        if (a.ckpt) return (int)cudaErrorInvalidValue;  // the saved-state layout of the normalised reverse pass is not written here
+        if (a.ckpt && !a.rown) return (int)cudaErrorInvalidValue;
         e = native ? cudaLaunchKernelEx(&cfg, tc_fwd_kernel<false, true>, tmK, tmQ, tmV, a)
                    : cudaLaunchKernelEx(&cfg, tc_fwd_kernel<true, true>, tmK, tmQ, tmV, a);
     } else {

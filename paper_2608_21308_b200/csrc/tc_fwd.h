@@ -23,10 +23,12 @@ struct TcFwdArgs {
     // optional: chunk-start states for the backward, fp32, [N][nchunks][W1 | W2 | M1 | M2] (nullptr = do not save)
     float* ckpt;
     size_t ckpt_seq_stride;  // floats between two sequences
-    // optional post-chunk normalisation: per-row target norms of W1 [N, h] and W2 [N, d] (nullptr = none); not
-    // together with ckpt
+    // optional post-chunk normalisation: per-row target norms of W1 [N, h] and W2 [N, d] (nullptr = none).  With ckpt
+    // the kernel also writes what the normalised reverse pass reads: the final state as one more ckpt slot and the
+    // row norms before normalisation, rown[N (stride ckpt_seq_stride)][nchunks][3][max(d, h)]
     const float *norm1, *norm2;
     float norm_eps;
+    float* rown;
 };
 
 size_t tc_fwd_smem_bytes();

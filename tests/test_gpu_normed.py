@@ -137,12 +137,10 @@ def test_normed_backward_windows_bf16(cfg):
         assert util.rel_err(got["drow_norm"][i], ref["drow_norm"][i]) <= TOL_BF16, i
 
 
-def test_normed_calls_reject_missing_targets_and_the_fused_kernel_with_saved_states():
+def test_normed_calls_reject_missing_targets():
     r = inputs.config(2, heads=[0], L=64)
     x = inputs.generate(r)
     tgt = targets(x)
-    with pytest.raises(Exception):   # the fused kernel does not write the states the normalised reverse pass reads
-        gpu_forward_normed(x, tgt, d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16", impl=E.E2TTT_IMPL_TCGEN05, save_states=True)
     with pytest.raises(Exception):
         gpu_forward_normed(x, tgt[:1], d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16", impl=E.E2TTT_IMPL_TILED)
 
@@ -185,3 +183,26 @@ def test_fused_normed_forward_free_running_and_auto_selection():
     assert np.array_equal(np.concatenate([a["o"], b["o"]], 1), got["o"])
     for i in range(2):
         assert np.array_equal(b["W"][i], got["W"][i]) and np.array_equal(b["M"][i], got["M"][i])
+
+
+def test_fused_normed_forward_saves_what_the_normalised_reverse_pass_reads():
+    """Training flow: the fused forward (two chunks per call) writes start states, row norms and the final slot; the
+    reverse pass from them agrees with the reverse pass that recomputes everything on the any-shape kernels, and a
+    one-chunk window agrees with the oracle."""
+    r = inputs.config(4, heads=[2, 11])
+    x2, _ = util.teacher_forced_windows(r, 4, window=2, with_grads=True)
+    tgt = targets(x2, 1.0)
+    shape = dict(d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16")
+    a = gpu_backward_normed(x2, tgt, impl=E.E2TTT_IMPL_TCGEN05, via_saved_states=True, **shape)
+    b = gpu_backward_normed(x2, tgt, impl=E.E2TTT_IMPL_TILED, via_saved_states=False, **shape)
+    for n in ("dq", "dk", "dv", "deta", "dbeta", "dgamma"):
+        assert util.rel_err(a[n], b[n]) <= 3 * TOL_BF16, n
+    for i in range(2):
+        assert util.rel_err(a["drow_norm"][i], b["drow_norm"][i]) <= 3 * TOL_BF16, i
+    x1, _ = util.teacher_forced_windows(r, 3, window=1, with_grads=True)
+    tgt1 = targets(x1, 1.0)
+    ref = oracle_bwd(x1, tgt1, r.C, r.kind)
+    got = gpu_backward_normed(x1, tgt1, impl=E.E2TTT_IMPL_TCGEN05, via_saved_states=True, **shape)
+    check_backward(got, ref, TOL_BF16, "normed bwd from the fused forward's saved states")
+    for i in range(2):
+        assert util.rel_err(got["drow_norm"][i], ref["drow_norm"][i]) <= TOL_BF16, i
