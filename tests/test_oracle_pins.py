@@ -481,3 +481,34 @@ def test_generator_follows_the_stated_distributions():
     assert np.array_equal(inputs.from_bf16_bits(bits), a["q"])     # bf16 I/O values are exactly representable
     t = torch.tensor(inputs.generate(inputs.config(1, heads=[5], io="f32"))["q"])
     assert np.array_equal(t.to(torch.bfloat16).float().numpy(), a["q"])  # same rounding as the hardware convert
+
+
+# ---------------------------------------------------------------- token preparation (SiLU + L2 norm, gate parameterisation)
+def test_prepare_oracle_matches_library_ops_and_autograd():
+    from oracle import prepare
+    rng = np.random.default_rng(3)
+    x = rng.standard_normal((5, 7, 16))
+    yb = rng.standard_normal((5, 7, 16))
+    xt = torch.tensor(x, dtype=torch.float64, requires_grad=True)
+    yt = torch.nn.functional.normalize(torch.nn.functional.silu(xt), dim=-1, eps=1e-12)
+    assert rel(prepare.silu_l2norm(x), yt.detach().numpy()) <= 1e-14
+    (yt * torch.tensor(yb)).sum().backward()
+    assert rel(prepare.silu_l2norm_vjp(x, yb), xt.grad.numpy()) <= 1e-12
+    assert np.allclose(np.sqrt((prepare.silu_l2norm(x) ** 2).sum(-1)), 1.0, atol=1e-14)       # unit rows
+    assert np.array_equal(prepare.silu_l2norm(np.zeros((2, 4))), np.zeros((2, 4)))            # zero vector stays zero
+    a, b, c = (rng.standard_normal((5, 7)) * 2 for _ in range(3))
+    de, db, dg = (rng.standard_normal((5, 7)) for _ in range(3))
+    eb, tau, ab = 0.01, 32.0, 0.1
+    at, bt, ct = (torch.tensor(t, dtype=torch.float64, requires_grad=True) for t in (a, b, c))
+    eta_t = eb * torch.sigmoid(at)
+    beta_t = torch.sigmoid(bt) ** (1.0 / tau)
+    gamma_t = 1.0 - eta_t * (ab * torch.sigmoid(ct))
+    eta, beta, gamma = prepare.gates(a, b, c, eb, tau, ab)
+    assert rel(eta, eta_t.detach().numpy()) <= 1e-14 and rel(beta, beta_t.detach().numpy()) <= 1e-14
+    assert rel(gamma, gamma_t.detach().numpy()) <= 1e-14
+    (eta_t * torch.tensor(de) + beta_t * torch.tensor(db) + gamma_t * torch.tensor(dg)).sum().backward()
+    da, dbb, dc = prepare.gates_vjp(a, b, c, eb, tau, ab, de, db, dg)
+    assert rel(da, at.grad.numpy()) <= 1e-12 and rel(dbb, bt.grad.numpy()) <= 1e-12 and rel(dc, ct.grad.numpy()) <= 1e-12
+    # ranges the method relies on: 0 < eta < eta_base, 0 < beta < 1, 1 - eta_base alpha_base < gamma < 1
+    assert (eta > 0).all() and (eta < eb).all() and (beta > 0).all() and (beta < 1).all()
+    assert (gamma < 1).all() and (gamma > 1 - eb * ab).all()
