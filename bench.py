@@ -527,6 +527,77 @@ def run_decode(args, r):
     print(json.dumps(line))
 
 
+def run_prepare(args, r):
+    """Optional workload (--prepare): one step = e2ttt_prepare_fwd over all token-heads of the configuration (SiLU + L2
+    normalisation of q and k, gate parameterisation).  Streaming, HBM-bound: every byte read once, written once."""
+    import torch
+    from paper_2608_21308_b200 import binding as E
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    iod = torch.float32 if r.io == "f32" else torch.bfloat16
+    s4, s3 = (r.B, r.H, r.L, r.d), (r.B, r.H, r.L)
+    gen = torch.Generator(device="cpu").manual_seed(r.seed)
+    host = {n: torch.randn(s4, generator=gen).to(iod).pin_memory() for n in ("q_raw", "k_raw")}
+    host.update({n: (2.0 * torch.randn(s3, generator=gen)).pin_memory() for n in ("a_eta", "a_beta", "a_alpha")})
+    t = {n: v.to(dev) for n, v in host.items()}
+    q, k = torch.empty_like(t["q_raw"]), torch.empty_like(t["k_raw"])
+    eta, beta, gamma = (torch.empty(s3, dtype=torch.float32, device=dev) for _ in range(3))
+    hout = [torch.empty_like(host["q_raw"]).pin_memory(), torch.empty_like(host["k_raw"]).pin_memory()] + \
+           [torch.empty(s3).pin_memory() for _ in range(3)]
+    p = E.make_params(r.B, r.H, r.L, r.d, r.h, r.C, r.kind, E.E2TTT_F32 if r.io == "f32" else E.E2TTT_BF16, 1e-5,
+                      E.E2TTT_IMPL_AUTO)
+    gp = E.e2ttt_gate_params(0.01, 32.0, 0.1, 1e-12)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        E.e2ttt_prepare_fwd(p, gp, t["q_raw"], t["k_raw"], t["a_eta"], t["a_beta"], t["a_alpha"], q, k, eta, beta, gamma, stream)
+
+    def step_e2e():
+        for n in host:
+            t[n].copy_(host[n], non_blocking=True)
+        step()
+        for a, b in zip(hout, (q, k, eta, beta, gamma)):
+            a.copy_(b, non_blocking=True)
+
+    def timed(fn, n, warmup):
+        for _ in range(warmup):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(n):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    steps = max(args.steps, 20)
+    sampler = ClockSampler(0)
+    sampler.start()
+    ms = timed(step, steps, args.warmup)
+    clocks = sampler.stop()
+    ms_e2e = timed(step_e2e, max(2, steps // 4), 1)
+    pk = peaks()
+    rows = r.B * r.H * r.L
+    es = 2 if r.io == "bf16" else 4
+    nbytes = rows * (4 * r.d * es + 24)
+    line = {"metric": "e2ttt_prepare_tokens_per_s", "value": r.B * r.L / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"e2ttt_prepare_fwd B={r.B} H={r.H} L={r.L} d={r.d} {r.io} I/O", "B": r.B, "H": r.H, "L": r.L,
+                       "d": r.d, "io": r.io, "seed": r.seed,
+                       "l2": f"inputs larger than L2: one step reads and writes {nbytes / 1e6:.0f} MB"},
+            "e2e": {"value": r.B * r.L / (ms_e2e * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": sum(v.numel() * v.element_size() for v in host.values()),
+                    "d2h_bytes_per_step": sum(v.numel() * v.element_size() for v in hout), "ms_per_step": ms_e2e},
+            "gpu_launches": steps, "clocks": clocks,
+            "roofline": {"bound": "hbm", "achieved": nbytes / (ms * 1e-3) / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                         "frac": nbytes / (ms * 1e-3) / 1e9 / pk["hbm_gbs"], "traffic": None, "peak_source": pk["_source"],
+                         "kernel": "prepare_fwd_kernel (one launch per step)", "bytes_per_launch": nbytes}}
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -537,12 +608,15 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--backward", action="store_true", help="time forward + backward instead (1 GPU, GELU-MLP configs)")
     ap.add_argument("--decode", action="store_true", help="time the decode step instead: e2ttt_apply on one token per sequence (1 GPU)")
+    ap.add_argument("--prepare", action="store_true", help="time the token preparation instead (e2ttt_prepare_fwd, 1 GPU)")
     ap.add_argument("--post-norm", action="store_true", help="forward with post-chunk normalisation of the fast weights (e2ttt_chunk_fwd_normed)")
     ap.add_argument("--chunk", type=int, default=0, help="override the chunk size C of the configuration")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     r = inputs.config(args.config, **({"C": args.chunk} if args.chunk else {}))
-    if args.decode and args.impl == "ours":
+    if args.prepare and args.impl == "ours":
+        run_prepare(args, r)
+    elif args.decode and args.impl == "ours":
         run_decode(args, r)
     elif args.backward and args.impl == "ours":
         run_fwd_bwd(args, r)

@@ -203,6 +203,35 @@ E2TTT_API int e2ttt_chunk_bwd_normed(const e2ttt_params* p, const void* q, const
  * Returns E2TTT_OK or E2TTT_ERR_NULL / _SHAPE / _DTYPE / _ALIGN / _ARCH / _CUDA. */
 E2TTT_API int e2ttt_apply(const e2ttt_params* p, const void* q, const float* const* W, void* o, void* stream);
 
+/* Token preparation, the step of the model right before the chunk update (Section 4, "Overall Architecture",
+ * Eqs. "eta_parameterization", "beta_parameterization", "decay_derivation"):
+ *   q = silu(q_raw) / max(||silu(q_raw)||_2, norm_eps)  per token and head, k likewise from k_raw;
+ *   eta = eta_base sigmoid(a_eta),  beta = sigmoid(a_beta)^(1/tau),
+ *   gamma = 1 - eta * alpha_base sigmoid(a_alpha).
+ * The logits a_* are the outputs of the model's small linear heads, which stay with the caller.  (The paper does
+ * not say how a zero vector is normalised: the max(., norm_eps) of the common library routine is a reading.)
+ *   p        in  (host)    B, H, L, d, io_dtype; the other fields are ignored
+ *   g        in  (host)    eta_base > 0, tau > 0, alpha_base >= 0, norm_eps >= 0
+ *   q_raw, k_raw      in  (device)  [B,H,L,d] io_dtype
+ *   a_eta, a_beta, a_alpha  in (device)  [B,H,L] fp32
+ *   q, k     out (device)  [B,H,L,d] io_dtype (may alias q_raw, k_raw)
+ *   eta, beta, gamma  out (device)  [B,H,L] fp32: what e2ttt_chunk_fwd takes
+ * e2ttt_prepare_bwd gives the adjoints of q_raw, k_raw and the three logits from those of q, k, eta, beta,
+ * gamma (what e2ttt_chunk_bwd returns); it re-reads the forward's inputs and needs none of its outputs.
+ * Arithmetic in fp32; no workspace; enqueued on `stream`; HBM-bound (every byte read once, written once).
+ * Returns E2TTT_OK or E2TTT_ERR_NULL / _SHAPE / _DTYPE / _ARCH / _CUDA. */
+typedef struct {
+    float eta_base, tau, alpha_base, norm_eps;
+} e2ttt_gate_params;
+E2TTT_API int e2ttt_prepare_fwd(const e2ttt_params* p, const e2ttt_gate_params* g, const void* q_raw,
+                                const void* k_raw, const float* a_eta, const float* a_beta, const float* a_alpha,
+                                void* q, void* k, float* eta, float* beta, float* gamma, void* stream);
+E2TTT_API int e2ttt_prepare_bwd(const e2ttt_params* p, const e2ttt_gate_params* g, const void* q_raw,
+                                const void* k_raw, const float* a_eta, const float* a_beta, const float* a_alpha,
+                                const void* dq, const void* dk, const float* d_eta, const float* d_beta,
+                                const float* d_gamma, void* dq_raw, void* dk_raw, float* da_eta, float* da_beta,
+                                float* da_alpha, void* stream);
+
 /* Reads back the device status word of the last launch that used `workspace` (the first word of every
  * workspace).  This is the one entry point that synchronises: it waits for `stream`.
  *   status  out (host)  0 after a clean run; otherwise the code of the first bounded device-side wait

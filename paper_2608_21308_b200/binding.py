@@ -21,6 +21,11 @@ E2TTT_IMPL_AUTO, E2TTT_IMPL_SIMT, E2TTT_IMPL_TCGEN05, E2TTT_IMPL_TILED = 0, 1, 2
 E2TTT_OK = 0
 
 
+class e2ttt_gate_params(ctypes.Structure):
+    _fields_ = [("eta_base", ctypes.c_float), ("tau", ctypes.c_float), ("alpha_base", ctypes.c_float),
+                ("norm_eps", ctypes.c_float)]
+
+
 class e2ttt_params(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("L", ctypes.c_int32), ("d", ctypes.c_int32),
                 ("h", ctypes.c_int32), ("C", ctypes.c_int32), ("kind", ctypes.c_int32),
@@ -62,6 +67,11 @@ def lib() -> ctypes.CDLL:
         L.e2ttt_chunk_bwd_normed.argtypes = [pp, vp, vp, vp, vp, vp, vp, tab, tab, tab, ctypes.c_float, vp, tab, tab, vp, vp,
                                              vp, vp, vp, vp, tab, tab, tab, vp, ctypes.c_size_t, cp, vp]
         L.e2ttt_chunk_bwd_normed.restype = cp
+        gp = ctypes.POINTER(e2ttt_gate_params)
+        L.e2ttt_prepare_fwd.argtypes = [pp, gp] + [vp] * 11
+        L.e2ttt_prepare_fwd.restype = cp
+        L.e2ttt_prepare_bwd.argtypes = [pp, gp] + [vp] * 16
+        L.e2ttt_prepare_bwd.restype = cp
         L.e2ttt_apply.argtypes = [pp, vp, tab, vp, vp]
         L.e2ttt_apply.restype = cp
         L.e2ttt_device_status.argtypes = [vp, vp, ctypes.POINTER(cp)]
@@ -221,6 +231,39 @@ def e2ttt_chunk_bwd_normed(p, q, k, v, eta, beta, gamma, W_init, M_init, row_nor
         int(states_saved), _stream_ptr(stream))
     if st != E2TTT_OK:
         raise E2TTTError(st, "e2ttt_chunk_bwd_normed")
+    return st
+
+
+def e2ttt_prepare_fwd(p, g, q_raw, k_raw, a_eta, a_beta, a_alpha, q, k, eta, beta, gamma, stream=None):
+    """int e2ttt_prepare_fwd(...) of include/e2ttt.h.  Raises on error."""
+    io = _io_torch_dtype(p)
+    s4, s3 = (p.B, p.H, p.L, p.d), (p.B, p.H, p.L)
+    f32 = torch.float32
+    st = lib().e2ttt_prepare_fwd(
+        ctypes.byref(p), ctypes.byref(g), _ptr(q_raw, io, s4, "q_raw"), _ptr(k_raw, io, s4, "k_raw"),
+        _ptr(a_eta, f32, s3, "a_eta"), _ptr(a_beta, f32, s3, "a_beta"), _ptr(a_alpha, f32, s3, "a_alpha"),
+        _ptr(q, io, s4, "q"), _ptr(k, io, s4, "k"), _ptr(eta, f32, s3, "eta"), _ptr(beta, f32, s3, "beta"),
+        _ptr(gamma, f32, s3, "gamma"), _stream_ptr(stream))
+    if st != E2TTT_OK:
+        raise E2TTTError(st, "e2ttt_prepare_fwd")
+    return st
+
+
+def e2ttt_prepare_bwd(p, g, q_raw, k_raw, a_eta, a_beta, a_alpha, dq, dk, d_eta, d_beta, d_gamma, dq_raw, dk_raw,
+                      da_eta, da_beta, da_alpha, stream=None):
+    """int e2ttt_prepare_bwd(...) of include/e2ttt.h.  Raises on error."""
+    io = _io_torch_dtype(p)
+    s4, s3 = (p.B, p.H, p.L, p.d), (p.B, p.H, p.L)
+    f32 = torch.float32
+    st = lib().e2ttt_prepare_bwd(
+        ctypes.byref(p), ctypes.byref(g), _ptr(q_raw, io, s4, "q_raw"), _ptr(k_raw, io, s4, "k_raw"),
+        _ptr(a_eta, f32, s3, "a_eta"), _ptr(a_beta, f32, s3, "a_beta"), _ptr(a_alpha, f32, s3, "a_alpha"),
+        _ptr(dq, io, s4, "dq"), _ptr(dk, io, s4, "dk"), _ptr(d_eta, f32, s3, "d_eta"), _ptr(d_beta, f32, s3, "d_beta"),
+        _ptr(d_gamma, f32, s3, "d_gamma"), _ptr(dq_raw, io, s4, "dq_raw"), _ptr(dk_raw, io, s4, "dk_raw"),
+        _ptr(da_eta, f32, s3, "da_eta"), _ptr(da_beta, f32, s3, "da_beta"), _ptr(da_alpha, f32, s3, "da_alpha"),
+        _stream_ptr(stream))
+    if st != E2TTT_OK:
+        raise E2TTTError(st, "e2ttt_prepare_bwd")
     return st
 
 

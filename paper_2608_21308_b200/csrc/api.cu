@@ -3,6 +3,7 @@
 
 #include "../../include/e2ttt.h"
 #include "apply.h"
+#include "prepare.h"
 #include "simt_layout.h"
 #include "tc_fwd.h"
 
@@ -341,6 +342,52 @@ int e2ttt_apply(const e2ttt_params* p, const void* q, const float* const* W, voi
     a.q = q; a.o = o;
     for (int i = 0; i < nmat; ++i) a.W[i] = W[i];
     return apply_launch(a, p->kind, p->io_dtype, stream) == 0 ? E2TTT_OK : E2TTT_ERR_CUDA;
+}
+
+static int check_gates(const e2ttt_gate_params* g) {
+    if (!g) return E2TTT_ERR_NULL;
+    if (!(g->eta_base > 0.0f) || !(g->tau > 0.0f) || !(g->alpha_base >= 0.0f) || !(g->norm_eps >= 0.0f)) return E2TTT_ERR_SHAPE;
+    return E2TTT_OK;
+}
+
+int e2ttt_prepare_fwd(const e2ttt_params* p, const e2ttt_gate_params* g, const void* q_raw, const void* k_raw,
+                      const float* a_eta, const float* a_beta, const float* a_alpha, void* q, void* k, float* eta,
+                      float* beta, float* gamma, void* stream) {
+    int rc = check_params(p);
+    if (rc) return rc;
+    rc = check_gates(g);
+    if (rc) return rc;
+    if (!q_raw || !k_raw || !a_eta || !a_beta || !a_alpha || !q || !k || !eta || !beta || !gamma) return E2TTT_ERR_NULL;
+    rc = check_device();
+    if (rc) return rc;
+    PrepareArgs a{};
+    a.rows = (long long)p->B * p->H * p->L; a.d = p->d;
+    a.eta_base = g->eta_base; a.tau = g->tau; a.alpha_base = g->alpha_base; a.norm_eps = g->norm_eps;
+    a.q_raw = q_raw; a.k_raw = k_raw; a.a_eta = a_eta; a.a_beta = a_beta; a.a_alpha = a_alpha;
+    a.q = q; a.k = k; a.eta = eta; a.beta = beta; a.gamma = gamma;
+    return prepare_fwd_launch(a, p->io_dtype, stream) == 0 ? E2TTT_OK : E2TTT_ERR_CUDA;
+}
+
+int e2ttt_prepare_bwd(const e2ttt_params* p, const e2ttt_gate_params* g, const void* q_raw, const void* k_raw,
+                      const float* a_eta, const float* a_beta, const float* a_alpha, const void* dq, const void* dk,
+                      const float* d_eta, const float* d_beta, const float* d_gamma, void* dq_raw, void* dk_raw,
+                      float* da_eta, float* da_beta, float* da_alpha, void* stream) {
+    int rc = check_params(p);
+    if (rc) return rc;
+    rc = check_gates(g);
+    if (rc) return rc;
+    if (!q_raw || !k_raw || !a_eta || !a_beta || !a_alpha || !dq || !dk || !d_eta || !d_beta || !d_gamma || !dq_raw ||
+        !dk_raw || !da_eta || !da_beta || !da_alpha)
+        return E2TTT_ERR_NULL;
+    rc = check_device();
+    if (rc) return rc;
+    PrepareBwdArgs b{};
+    b.f.rows = (long long)p->B * p->H * p->L; b.f.d = p->d;
+    b.f.eta_base = g->eta_base; b.f.tau = g->tau; b.f.alpha_base = g->alpha_base; b.f.norm_eps = g->norm_eps;
+    b.f.q_raw = q_raw; b.f.k_raw = k_raw; b.f.a_eta = a_eta; b.f.a_beta = a_beta; b.f.a_alpha = a_alpha;
+    b.dq = dq; b.dk = dk; b.d_eta = d_eta; b.d_beta = d_beta; b.d_gamma = d_gamma;
+    b.dq_raw = dq_raw; b.dk_raw = dk_raw; b.da_eta = da_eta; b.da_beta = da_beta; b.da_alpha = da_alpha;
+    return prepare_bwd_launch(b, p->io_dtype, stream) == 0 ? E2TTT_OK : E2TTT_ERR_CUDA;
 }
 
 int e2ttt_device_status(const void* workspace, void* stream, int* status) {

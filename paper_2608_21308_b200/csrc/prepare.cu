@@ -1,0 +1,235 @@
+// Token preparation upstream of the chunk update (Section 4, "Overall Architecture" and the gate parameterisation):
+//   q, k <- silu(x) / max(||silu(x)||_2, eps) per token and head;
+//   eta = eta_base sigmoid(a),  beta = sigmoid(b)^(1/tau),  gamma = 1 - eta alpha_base sigmoid(c)
+// and the reverse pass.  Pure streaming work: every byte is read once and written once, so the kernels are bound by
+// HBM.  One warp owns a token-head row of d elements: lane l holds the V-element pieces (p * 32 + l) of the row in
+// registers between the norm reduction and the scaled store (V and the piece count are compile-time, so nothing
+// spills to local memory), and works on the query and the key rows of two tokens at once so that four rows' loads
+// are in flight per lane.  Grid: one wave of 8-warp CTAs with a grid-stride loop over the token-heads.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <type_traits>
+
+#include "prepare.h"
+#include "simt_common.cuh"
+
+namespace e2ttt {
+namespace {
+
+constexpr int kPrThreads = 256;
+constexpr int kPrTokens = 2;  // tokens a warp works on at once
+
+// sigmoid with the hardware exp2 and reciprocal: the IEEE division alone costs more instructions than the rest of
+// an element's work, and the kernels are meant to be bound by memory, not by issue slots
+__device__ __forceinline__ float pr_sigmoid(float z) { return __fdividef(1.0f, 1.0f + __expf(-z)); }
+
+// V consecutive elements <-> registers, one memory access of V * sizeof(IO) bytes (V = 1, 2 or 4)
+template <typename IO, int V> __device__ __forceinline__ void ld_piece(const IO* p, float* v) {
+    if (sizeof(IO) == 4) {
+        if (V == 4) { const float4 x = *reinterpret_cast<const float4*>(p); v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w; }
+        else if (V == 2) { const float2 x = *reinterpret_cast<const float2*>(p); v[0] = x.x; v[1] = x.y; }
+        else v[0] = ld_io<float>(p, (size_t)0);
+    } else {
+        if (V == 4) {
+            const uint2 raw = *reinterpret_cast<const uint2*>(p);
+            const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
+            const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
+            v[0] = a.x; v[1] = a.y; v[2] = b.x; v[3] = b.y;
+        } else if (V == 2) {
+            const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(p));
+            v[0] = a.x; v[1] = a.y;
+        } else v[0] = ld_io<float>(p, (size_t)0);
+    }
+}
+template <typename IO, int V> __device__ __forceinline__ void st_piece(IO* p, const float* v) {
+    if (sizeof(IO) == 4) {
+        if (V == 4) *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+        else if (V == 2) *reinterpret_cast<float2*>(p) = make_float2(v[0], v[1]);
+        else st_io(p, (size_t)0, v[0]);
+    } else {
+        if (V == 4) {
+            uint2 raw;
+            *reinterpret_cast<__nv_bfloat162*>(&raw.x) = __floats2bfloat162_rn(v[0], v[1]);
+            *reinterpret_cast<__nv_bfloat162*>(&raw.y) = __floats2bfloat162_rn(v[2], v[3]);
+            *reinterpret_cast<uint2*>(p) = raw;
+        } else if (V == 2) {
+            *reinterpret_cast<__nv_bfloat162*>(p) = __floats2bfloat162_rn(v[0], v[1]);
+        } else st_io(p, (size_t)0, v[0]);
+    }
+}
+
+// a row in registers: NP pieces of V elements per lane
+template <typename IO, int V, int NP> __device__ __forceinline__ void ld_row(const IO* p, int d, float (&v)[NP * V]) {
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int pc = 0; pc < NP; ++pc) {
+        const int c = (pc * 32 + lane) * V;
+        if (c < d) ld_piece<IO, V>(p + c, &v[pc * V]);
+        else
+#pragma unroll
+            for (int j = 0; j < V; ++j) v[pc * V + j] = 0.0f;
+    }
+}
+template <typename IO, int V, int NP> __device__ __forceinline__ void st_row(IO* p, int d, const float (&v)[NP * V]) {
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int pc = 0; pc < NP; ++pc) {
+        const int c = (pc * 32 + lane) * V;
+        if (c < d) st_piece<IO, V>(p + c, &v[pc * V]);
+    }
+}
+
+template <typename IO, int V, int NP>
+__global__ void __launch_bounds__(kPrThreads) prepare_fwd_kernel(const PrepareArgs a) {
+    const long long warp = (long long)((blockIdx.x * (size_t)kPrThreads + threadIdx.x) >> 5);
+    const long long nwarps = (long long)((gridDim.x * (size_t)kPrThreads) >> 5);
+    const int lane = threadIdx.x & 31;
+    const int d = a.d;
+    const IO* q_raw = reinterpret_cast<const IO*>(a.q_raw);
+    const IO* k_raw = reinterpret_cast<const IO*>(a.k_raw);
+    IO* q = reinterpret_cast<IO*>(a.q);
+    IO* k = reinterpret_cast<IO*>(a.k);
+    for (long long t0 = warp * kPrTokens; t0 < a.rows; t0 += nwarps * kPrTokens) {
+        float x[2 * kPrTokens][NP * V];  // query and key rows of the warp's tokens
+#pragma unroll
+        for (int u = 0; u < kPrTokens; ++u) {
+            const long long t = t0 + u;
+            if (t < a.rows) {
+                ld_row<IO, V, NP>(q_raw + (size_t)t * d, d, x[2 * u]);
+                ld_row<IO, V, NP>(k_raw + (size_t)t * d, d, x[2 * u + 1]);
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < 2 * kPrTokens; ++r) {
+            const long long t = t0 + (r >> 1);
+            if (t >= a.rows) continue;
+            float ss = 0.0f;
+#pragma unroll
+            for (int j = 0; j < NP * V; ++j) {
+                x[r][j] = x[r][j] * pr_sigmoid(x[r][j]);
+                ss = fmaf(x[r][j], x[r][j], ss);
+            }
+            const float f = 1.0f / fmaxf(sqrtf(warp_sum(ss)), a.norm_eps);
+#pragma unroll
+            for (int j = 0; j < NP * V; ++j) x[r][j] *= f;
+            st_row<IO, V, NP>(((r & 1) ? k : q) + (size_t)t * d, d, x[r]);
+        }
+        if (lane < kPrTokens && t0 + lane < a.rows) {
+            const long long t = t0 + lane;
+            const float eta = a.eta_base * pr_sigmoid(a.a_eta[t]);
+            const float beta = __powf(pr_sigmoid(a.a_beta[t]), 1.0f / a.tau);
+            const float alpha = a.alpha_base * pr_sigmoid(a.a_alpha[t]);
+            a.eta[t] = eta;
+            a.beta[t] = beta;
+            a.gamma[t] = 1.0f - eta * alpha;
+        }
+    }
+}
+
+// reverse of a normalised row: y = s / m, m = max(||s||, eps), s = silu(x):  x_bar = silu'(x) (y_bar - y <y_bar, y>) / m
+template <typename IO, int V, int NP>
+__global__ void __launch_bounds__(kPrThreads) prepare_bwd_kernel(const PrepareBwdArgs a) {
+    const long long warp = (long long)((blockIdx.x * (size_t)kPrThreads + threadIdx.x) >> 5);
+    const long long nwarps = (long long)((gridDim.x * (size_t)kPrThreads) >> 5);
+    const int lane = threadIdx.x & 31;
+    const int d = a.f.d;
+    for (long long t = warp; t < a.f.rows; t += nwarps) {
+        const size_t off = (size_t)t * d;
+        float x[2][NP * V], g[2][NP * V];
+        ld_row<IO, V, NP>(reinterpret_cast<const IO*>(a.f.q_raw) + off, d, x[0]);
+        ld_row<IO, V, NP>(reinterpret_cast<const IO*>(a.f.k_raw) + off, d, x[1]);
+        ld_row<IO, V, NP>(reinterpret_cast<const IO*>(a.dq) + off, d, g[0]);
+        ld_row<IO, V, NP>(reinterpret_cast<const IO*>(a.dk) + off, d, g[1]);
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            float ss = 0.0f, sg = 0.0f;
+#pragma unroll
+            for (int j = 0; j < NP * V; ++j) {
+                const float sig = pr_sigmoid(x[r][j]);
+                const float s = x[r][j] * sig;
+                ss = fmaf(s, s, ss);
+                sg = fmaf(s, g[r][j], sg);
+                g[r][j] *= sig * (1.0f + x[r][j] * (1.0f - sig));  // y_bar silu'(x)
+                x[r][j] = s * sig * (1.0f + x[r][j] * (1.0f - sig));  // s silu'(x)
+            }
+            const float nrm = sqrtf(warp_sum(ss));
+            sg = warp_sum(sg);
+            const float m = fmaxf(nrm, a.f.norm_eps);
+            const float proj = (nrm > a.f.norm_eps) ? sg / (m * m) : 0.0f;  // <y_bar, y> / m
+            const float inv = 1.0f / m;
+#pragma unroll
+            for (int j = 0; j < NP * V; ++j) g[r][j] = (g[r][j] - x[r][j] * proj) * inv;
+            st_row<IO, V, NP>(reinterpret_cast<IO*>(r ? a.dk_raw : a.dq_raw) + off, d, g[r]);
+        }
+        if (lane == 0) {
+            const float sa = pr_sigmoid(a.f.a_eta[t]), sb = pr_sigmoid(a.f.a_beta[t]), sc = pr_sigmoid(a.f.a_alpha[t]);
+            const float eta = a.f.eta_base * sa, alpha = a.f.alpha_base * sc;
+            const float beta = __powf(sb, 1.0f / a.f.tau);
+            const float eta_bar = a.d_eta[t] - a.d_gamma[t] * alpha;
+            a.da_eta[t] = eta_bar * a.f.eta_base * sa * (1.0f - sa);
+            a.da_beta[t] = a.d_beta[t] * beta * (1.0f - sb) / a.f.tau;
+            a.da_alpha[t] = -a.d_gamma[t] * eta * a.f.alpha_base * sc * (1.0f - sc);
+        }
+    }
+}
+
+int grid_for(long long rows, int rows_per_warp) {
+    const long long warps = (rows + rows_per_warp - 1) / rows_per_warp;
+    const long long want = (warps + (kPrThreads / 32) - 1) / (kPrThreads / 32);
+    const long long cap = 148LL * 8;  // one wave at 8 CTAs of 256 threads per SM
+    return (int)(want < cap ? (want < 1 ? 1 : want) : cap);
+}
+
+// piece width and count: 4-element pieces when the rows allow aligned 8-/16-byte accesses, else scalar
+struct Shape { int v, np; };
+Shape pick_shape(int d, int io_bytes, const void* const* ptrs, int nptrs) {
+    bool al = true;
+    for (int i = 0; i < nptrs; ++i) al = al && (reinterpret_cast<uintptr_t>(ptrs[i]) % 16 == 0);
+    (void)io_bytes;
+    if (al && d % 4 == 0 && d >= 128) return {4, d <= 128 ? 1 : d <= 256 ? 2 : d <= 512 ? 4 : 8};
+    if (al && d % 2 == 0 && d <= 64) return {2, 1};
+    return {1, 32};
+}
+
+template <typename IO, typename Args, typename F> int dispatch(const Shape& s, F launch) {
+    if (s.v == 4 && s.np == 1) return launch(std::integral_constant<int, 4>(), std::integral_constant<int, 1>());
+    if (s.v == 4 && s.np == 2) return launch(std::integral_constant<int, 4>(), std::integral_constant<int, 2>());
+    if (s.v == 4 && s.np == 4) return launch(std::integral_constant<int, 4>(), std::integral_constant<int, 4>());
+    if (s.v == 4 && s.np == 8) return launch(std::integral_constant<int, 4>(), std::integral_constant<int, 8>());
+    if (s.v == 2) return launch(std::integral_constant<int, 2>(), std::integral_constant<int, 1>());
+    return launch(std::integral_constant<int, 1>(), std::integral_constant<int, 32>());
+}
+
+template <typename IO> int fwd_io(const PrepareArgs& a, cudaStream_t st) {
+    const void* ptrs[4] = {a.q_raw, a.k_raw, a.q, a.k};
+    const Shape s = pick_shape(a.d, (int)sizeof(IO), ptrs, 4);
+    const int grid = grid_for(a.rows, kPrTokens);
+    return dispatch<IO, PrepareArgs>(s, [&](auto v, auto np) {
+        prepare_fwd_kernel<IO, decltype(v)::value, decltype(np)::value><<<grid, kPrThreads, 0, st>>>(a);
+        return (int)cudaGetLastError();
+    });
+}
+template <typename IO> int bwd_io(const PrepareBwdArgs& a, cudaStream_t st) {
+    const void* ptrs[6] = {a.f.q_raw, a.f.k_raw, a.dq, a.dk, a.dq_raw, a.dk_raw};
+    const Shape s = pick_shape(a.f.d, (int)sizeof(IO), ptrs, 6);
+    const int grid = grid_for(a.f.rows, 1);
+    return dispatch<IO, PrepareBwdArgs>(s, [&](auto v, auto np) {
+        prepare_bwd_kernel<IO, decltype(v)::value, decltype(np)::value><<<grid, kPrThreads, 0, st>>>(a);
+        return (int)cudaGetLastError();
+    });
+}
+
+}  // namespace
+
+int prepare_fwd_launch(const PrepareArgs& a, int io_dtype, void* stream) {
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    return io_dtype == 0 ? fwd_io<float>(a, st) : fwd_io<__nv_bfloat16>(a, st);
+}
+
+int prepare_bwd_launch(const PrepareBwdArgs& a, int io_dtype, void* stream) {
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    return io_dtype == 0 ? bwd_io<float>(a, st) : bwd_io<__nv_bfloat16>(a, st);
+}
+
+}  // namespace e2ttt
