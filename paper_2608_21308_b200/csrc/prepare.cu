@@ -6,6 +6,10 @@
 // registers between the norm reduction and the scaled store (V and the piece count are compile-time, so nothing
 // spills to local memory), and works on the query and the key rows of two tokens at once so that four rows' loads
 // are in flight per lane.  Grid: one wave of 8-warp CTAs with a grid-stride loop over the token-heads.
+// The forward of rows that allow it (row bytes a multiple of 16, aligned bases, d <= 256) runs as a bulk-copy pipeline
+// instead: tiles of 32 tokens travel global -> shared memory -> global with `cp.async.bulk` (mbarrier transaction
+// counts on the way in, bulk groups on the way out), four tiles deep per CTA, so the bytes in flight do not depend
+// on registers or occupancy; the warps only touch shared memory.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -13,6 +17,7 @@
 
 #include "prepare.h"
 #include "simt_common.cuh"
+#include "sm100.cuh"
 
 namespace e2ttt {
 namespace {
@@ -23,6 +28,19 @@ constexpr int kPrTokens = 2;  // tokens a warp works on at once
 // sigmoid with the hardware exp2 and reciprocal: the IEEE division alone costs more instructions than the rest of
 // an element's work, and the kernels are meant to be bound by memory, not by issue slots
 __device__ __forceinline__ float pr_sigmoid(float z) { return __fdividef(1.0f, 1.0f + __expf(-z)); }
+
+// silu(x) = x sigmoid(x).  With bf16 I/O the result is rounded to 2^-9 relative right after, so the hardware tanh
+// serves: x sigmoid(x) = hx + hx tanh(hx), hx = x / 2 (one MUFU and two FMA-pipe instructions; tanh.approx is good to
+// about 2^-11).  fp32 I/O keeps the exp form.
+template <typename IO> __device__ __forceinline__ float pr_silu(float x) {
+    if (sizeof(IO) == 2) {
+        const float hx = 0.5f * x;
+        float t;
+        asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(hx));
+        return fmaf(hx, t, hx);
+    }
+    return x * pr_sigmoid(x);
+}
 
 // V consecutive elements <-> registers, one memory access of V * sizeof(IO) bytes (V = 1, 2 or 4)
 template <typename IO, int V> __device__ __forceinline__ void ld_piece(const IO* p, float* v) {
@@ -107,7 +125,7 @@ __global__ void __launch_bounds__(kPrThreads) prepare_fwd_kernel(const PrepareAr
             float ss = 0.0f;
 #pragma unroll
             for (int j = 0; j < NP * V; ++j) {
-                x[r][j] = x[r][j] * pr_sigmoid(x[r][j]);
+                x[r][j] = pr_silu<IO>(x[r][j]);
                 ss = fmaf(x[r][j], x[r][j], ss);
             }
             const float f = 1.0f / fmaxf(sqrtf(warp_sum(ss)), a.norm_eps);
@@ -174,6 +192,168 @@ __global__ void __launch_bounds__(kPrThreads) prepare_bwd_kernel(const PrepareBw
     }
 }
 
+// ---- forward as a bulk-copy pipeline ------------------------------------------------------------------------
+constexpr int kBkTok = 32;     // tokens per tile
+constexpr int kBkStages = 4;   // tiles in flight per CTA
+
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(sm100::smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(sm100::smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_store(void* gdst, const void* smem_src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 ::"l"(gdst), "r"(sm100::smem_u32(smem_src)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+template <int N> __device__ __forceinline__ void bulk_wait_all() {
+    asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
+}
+// bounded wait for a tile (about a second); on time-out the CTA stops waiting and finishes without meaning
+__device__ __forceinline__ bool bulk_wait_tile(uint64_t* bar, uint32_t parity, volatile int* dead) {
+    if ((threadIdx.x & 31) == 0 && !*dead) {
+        const long long t0 = clock64();
+        int spins = 0;
+        while (!sm100::mbar_try_wait<false>(bar, parity)) {
+            if ((++spins & 255) == 0 && clock64() - t0 > sm100::kWaitCycles) { *dead = 1; break; }
+        }
+    }
+    __syncwarp();
+    return !*dead;
+}
+
+// LPR = lanes per row: a row is LPR pieces of 16 bytes (d = LPR * 16 / sizeof(IO)), one piece per lane, so a warp works on
+// 32 / LPR rows at once and the norm reduction runs over LPR lanes only.
+template <typename IO, int LPR>
+__global__ void __launch_bounds__(kPrThreads) prepare_fwd_bulk_kernel(const PrepareArgs a) {
+    extern __shared__ __align__(128) unsigned char pr_smem[];
+    const int d = a.d;
+    const uint32_t row_bytes = (uint32_t)d * sizeof(IO);
+    const uint32_t tile_bytes = kBkTok * row_bytes;          // one of q / k
+    uint64_t* full = reinterpret_cast<uint64_t*>(pr_smem);   // [kBkStages]
+    volatile int* dead = reinterpret_cast<volatile int*>(pr_smem + 64);
+    unsigned char* tiles = pr_smem + 128;                    // [kBkStages][2][tile_bytes]
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const long long ntiles = (a.rows + kBkTok - 1) / kBkTok;
+    const IO* q_raw = reinterpret_cast<const IO*>(a.q_raw);
+    const IO* k_raw = reinterpret_cast<const IO*>(a.k_raw);
+    IO* q = reinterpret_cast<IO*>(a.q);
+    IO* k = reinterpret_cast<IO*>(a.k);
+
+    if (tid == 0) {
+        for (int s = 0; s < kBkStages; ++s) sm100::mbar_init(&full[s], 1);
+        *dead = 0;
+        sm100::fence_mbar_init();
+    }
+    __syncthreads();
+    auto tokens_of = [&](long long tile) { return (int)min((long long)kBkTok, a.rows - tile * kBkTok); };
+    auto issue = [&](long long tile, int s) {  // thread 0
+        const uint32_t bytes = (uint32_t)tokens_of(tile) * row_bytes;
+        sm100::mbar_expect_tx(&full[s], 2 * bytes);
+        bulk_load(tiles + (size_t)(2 * s) * tile_bytes, q_raw + (size_t)tile * kBkTok * d, bytes, &full[s]);
+        bulk_load(tiles + (size_t)(2 * s + 1) * tile_bytes, k_raw + (size_t)tile * kBkTok * d, bytes, &full[s]);
+    };
+    if (tid == 0)
+        for (int i = 0; i < kBkStages; ++i) {
+            const long long tile = blockIdx.x + (long long)i * gridDim.x;
+            if (tile < ntiles) issue(tile, i);
+        }
+
+    long long it = 0;
+    for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++it) {
+        const int s = (int)(it % kBkStages);
+        const uint32_t parity = (uint32_t)((it / kBkStages) & 1);
+        const int ntok = tokens_of(tile);
+        if (!bulk_wait_tile(&full[s], parity, dead)) break;
+        IO* tq = reinterpret_cast<IO*>(tiles + (size_t)(2 * s) * tile_bytes);
+        IO* tk = reinterpret_cast<IO*>(tiles + (size_t)(2 * s + 1) * tile_bytes);
+        // gates of the tile's tokens (plain coalesced accesses)
+        if (tid < ntok) {
+            const long long t = tile * kBkTok + tid;
+            const float eta = a.eta_base * pr_sigmoid(a.a_eta[t]);
+            const float beta = __powf(pr_sigmoid(a.a_beta[t]), 1.0f / a.tau);
+            const float alpha = a.alpha_base * pr_sigmoid(a.a_alpha[t]);
+            a.eta[t] = eta;
+            a.beta[t] = beta;
+            a.gamma[t] = 1.0f - eta * alpha;
+        }
+        // rows 0..31 of the tile pair are the query rows, 32..63 the key rows; a warp pass covers 32 / LPR of them, in place
+        {
+            constexpr int E = 16 / (int)sizeof(IO), RPP = 32 / LPR;
+            const int sub = lane / LPR, li = lane % LPR;
+            for (int base = warp * RPP; base < 2 * kBkTok; base += (kPrThreads / 32) * RPP) {
+                const int r = base + sub;
+                const int u = r & (kBkTok - 1);
+                const bool valid = u < ntok;
+                IO* piece = ((r >= kBkTok) ? tk : tq) + (size_t)u * d + li * E;
+                float x[E];
+                if (valid) {
+                    const uint4 raw = *reinterpret_cast<const uint4*>(piece);
+                    if (sizeof(IO) == 2) {
+                        const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+                        for (int j = 0; j < E / 2; ++j) {
+                            const float2 f2 = __bfloat1622float2(h2[j]);
+                            x[2 * j] = f2.x;
+                            x[2 * j + 1] = f2.y;
+                        }
+                    } else {
+                        const float* f4 = reinterpret_cast<const float*>(&raw);
+#pragma unroll
+                        for (int j = 0; j < E; ++j) x[j] = f4[j];
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < E; ++j) x[j] = 0.0f;
+                }
+                float ss = 0.0f;
+#pragma unroll
+                for (int j = 0; j < E; ++j) {
+                    x[j] = pr_silu<IO>(x[j]);
+                    ss = fmaf(x[j], x[j], ss);
+                }
+#pragma unroll
+                for (int off = LPR / 2; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+                // 1 / max(||s||, eps)
+                const float f = (ss > a.norm_eps * a.norm_eps) ? rsqrtf(ss) : __fdividef(1.0f, a.norm_eps);
+                if (valid) {
+                    uint4 raw;
+                    if (sizeof(IO) == 2) {
+                        __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&raw);
+#pragma unroll
+                        for (int j = 0; j < E / 2; ++j) h2[j] = __floats2bfloat162_rn(x[2 * j] * f, x[2 * j + 1] * f);
+                    } else {
+                        float* f4 = reinterpret_cast<float*>(&raw);
+#pragma unroll
+                        for (int j = 0; j < E; ++j) f4[j] = x[j] * f;
+                    }
+                    *reinterpret_cast<uint4*>(piece) = raw;
+                }
+            }
+        }
+        sm100::fence_proxy_async_smem();  // the normalised rows -> visible to the bulk store
+        __syncthreads();
+        if (tid == 0) {
+            const uint32_t bytes = (uint32_t)ntok * row_bytes;
+            bulk_store(q + (size_t)tile * kBkTok * d, tq, bytes);
+            bulk_store(k + (size_t)tile * kBkTok * d, tk, bytes);
+            bulk_commit();
+            // the stage used one tile ago is free once its store has read shared memory: refill it
+            if (it >= 1) {
+                bulk_wait_read<1>();
+                const long long next = tile + (long long)(kBkStages - 1) * gridDim.x;
+                if (next < ntiles) issue(next, (int)((it - 1) % kBkStages));
+            }
+        }
+    }
+    if (tid == 0) bulk_wait_all<0>();  // the CTA's shared memory must outlive its stores
+    __syncthreads();
+}
+
 int grid_for(long long rows, int rows_per_warp) {
     const long long warps = (rows + rows_per_warp - 1) / rows_per_warp;
     const long long want = (warps + (kPrThreads / 32) - 1) / (kPrThreads / 32);
@@ -201,9 +381,39 @@ template <typename IO, typename Args, typename F> int dispatch(const Shape& s, F
     return launch(std::integral_constant<int, 1>(), std::integral_constant<int, 32>());
 }
 
+size_t bulk_smem_bytes(int d, size_t io_bytes) { return 128 + (size_t)kBkStages * 2 * kBkTok * d * io_bytes; }
+
+template <typename IO, int LPR> int fwd_bulk(const PrepareArgs& a, cudaStream_t st) {
+    const size_t smem = bulk_smem_bytes(a.d, sizeof(IO));
+    static size_t attr_bytes[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return (int)cudaGetLastError();
+    if (dev < 0 || dev >= 64 || attr_bytes[dev] < smem) {
+        cudaError_t e = cudaFuncSetAttribute(prepare_fwd_bulk_kernel<IO, LPR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return (int)e;
+        if (dev >= 0 && dev < 64) attr_bytes[dev] = smem;
+    }
+    const long long ntiles = (a.rows + kBkTok - 1) / kBkTok;
+    const int per_sm = (int)(220 * 1024 / smem);
+    const long long cap = 148LL * (per_sm > 4 ? 4 : per_sm);
+    const int grid = (int)(ntiles < cap ? ntiles : cap);
+    prepare_fwd_bulk_kernel<IO, LPR><<<grid, kPrThreads, smem, st>>>(a);
+    return (int)cudaGetLastError();
+}
+
 template <typename IO> int fwd_io(const PrepareArgs& a, cudaStream_t st) {
     const void* ptrs[4] = {a.q_raw, a.k_raw, a.q, a.k};
     const Shape s = pick_shape(a.d, (int)sizeof(IO), ptrs, 4);
+    // the bulk-copy pipeline: rows of 8, 16 or 32 pieces of 16 bytes, aligned bases, enough rows to fill the stages
+    // (in-place use, q == q_raw, is fine: a tile is read before it is written)
+    bool al = true;
+    for (int i = 0; i < 4; ++i) al = al && (reinterpret_cast<uintptr_t>(ptrs[i]) % 16 == 0);
+    const int lpr = (int)(a.d * sizeof(IO) / 16);
+    if (al && (size_t)lpr * 16 == a.d * sizeof(IO) && (lpr == 8 || lpr == 16 || lpr == 32) && a.rows >= 4 * kBkTok) {
+        if (lpr == 8) return fwd_bulk<IO, 8>(a, st);
+        if (lpr == 16) return fwd_bulk<IO, 16>(a, st);
+        return fwd_bulk<IO, 32>(a, st);
+    }
     const int grid = grid_for(a.rows, kPrTokens);
     return dispatch<IO, PrepareArgs>(s, [&](auto v, auto np) {
         prepare_fwd_kernel<IO, decltype(v)::value, decltype(np)::value><<<grid, kPrThreads, 0, st>>>(a);

@@ -46,7 +46,9 @@ def _run(B, H, L, d, io, seed=0, backward=False):
     return x, s, g, {n: t.float().cpu().numpy() for n, t in out.items()}
 
 
-SHAPES = [(2, 3, 17, 128), (1, 2, 5, 64), (1, 1, 3, 48), (2, 1, 7, 256), (1, 1, 2, 1000), (1, 1, 1, 8), (1, 2, 33, 130)]
+SHAPES = [(2, 3, 17, 128), (1, 2, 5, 64), (1, 1, 3, 48), (2, 1, 7, 256), (1, 1, 2, 1000), (1, 1, 1, 8), (1, 2, 33, 130),
+          # the bulk-copy pipeline of the forward: several tiles per CTA, a ragged last tile
+          (4, 4, 5001, 128), (1, 3, 43, 128), (2, 2, 2500, 256), (2, 2, 300, 64), (1, 2, 200, 32)]
 
 
 @pytest.mark.parametrize("io", ["f32", "bf16"])
