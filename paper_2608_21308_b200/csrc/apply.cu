@@ -113,6 +113,27 @@ __global__ void __launch_bounds__(kApThreads, 2) apply_kernel(const ApplyArgs a)
     const int h0 = min(h, rank * per), h1 = min(h, h0 + per);
     float* slot0 = cluster.map_shared_rank(slots, 0);
 
+    // Programmatic dependent launch: this grid may start while the previous kernel of the stream is still running.
+    // Nothing it produces may be touched before griddepcontrol.wait - but the fast weights of this CTA can already be
+    // pulled from HBM into L2 (a prefetch has no effect on memory contents), so that the next layer's weights stream
+    // in under the tail of the previous kernel.  Without a programmatic predecessor the wait returns at once.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (h0 < h1) {
+        const int nrows = h1 - h0;
+        // rows [h0, h1) of the first matrices are contiguous; the last matrix contributes d row segments
+        const size_t bytes1 = (size_t)nrows * d * sizeof(float);
+        for (size_t off = (size_t)tid * 128; off < bytes1; off += (size_t)kApThreads * 128) {
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(W1 + (size_t)h0 * d) + off));
+            if (KIND == 1) asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(W2 + (size_t)h0 * d) + off));
+        }
+        const int seg = (nrows * (int)sizeof(float) + 127) / 128;  // 128-byte lines per row segment
+        for (int e = tid; e < d * seg; e += kApThreads) {
+            const int i = e / seg, c = e - i * seg;
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(Wl + (size_t)i * h + h0) + (size_t)c * 128));
+        }
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
     for (int t0 = 0; t0 < T; t0 += TB) {
         const int tb = min(TB, T - t0);
         for (int e = tid; e < TB * d; e += kApThreads) {
@@ -223,13 +244,15 @@ int launch_apply(const ApplyArgs& a, cudaStream_t st) {
     cfg.blockDim = dim3(kApThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute at[1];
+    cudaLaunchAttribute at[2];
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = (unsigned)a.cl;
     at[0].val.clusterDim.y = 1;
     at[0].val.clusterDim.z = 1;
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see griddepcontrol in the kernel
+    at[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     cudaError_t e = cudaLaunchKernelEx(&cfg, apply_kernel<IO, KIND, TB, VEC>, a);
     if (e != cudaSuccess) return (int)e;
     return (int)cudaGetLastError();
