@@ -139,3 +139,27 @@ def test_tc_padded_saved_states_feed_the_backward():
     ref = util.oracle_backward(x1, r.C, r.kind)
     got1 = util.gpu_backward(x1, d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16", via_saved_states=True)
     check_backward(got1, ref, TOL_BF16, "padded bwd from tensor-core saved states")
+
+
+def test_tc_boundary_gates():
+    """Gates on the boundary of their range (the division-free scans must not care): beta or gamma exactly 0 or 1,
+    eta exactly 0, mixed inside one chunk; one chunk per sequence against the oracle, all three kernel families."""
+    r = inputs.config(2, heads=[0, 1, 2, 3, 4, 5], L=64, m_std=0.002)
+    x = inputs.generate(r)
+    x["beta"][0, :] = 0.0
+    x["beta"][1, :] = 1.0
+    x["gamma"][2, :] = 1.0
+    x["gamma"][3, ::7] = 0.0
+    x["eta"][4, :] = 0.0
+    x["beta"][5, ::5] = 0.0
+    x["beta"][5, 1::5] = 1.0
+    x["gamma"][5, 2::5] = 1.0
+    x["eta"][5, 3::5] = 0.0
+    ref = util.oracle_forward(x, 64, MLP)
+    for impl in (E.E2TTT_IMPL_TCGEN05, E.E2TTT_IMPL_TILED, E.E2TTT_IMPL_SIMT):
+        got, hd = util.gpu_forward(x, impl=impl, **SHAPE)
+        assert E.e2ttt_device_status(hd["ws"]) == 0
+        assert np.isfinite(got["o"]).all() and all(np.isfinite(w).all() for w in got["W"] + got["M"])
+        check_forward(got, ref, TOL_BF16, f"boundary gates, impl {impl}")
+    # eta = 0 for a whole chunk: the gradients do not enter; W_C = cw W_0 + cm M_0, M_C = cb M_0 exactly in the oracle
+    assert util.rel_err(ref["M"][0][4], np.prod(x["beta"][4].astype(np.float64)) * x["M"][0][4]) <= 1e-12
