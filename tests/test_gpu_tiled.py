@@ -86,3 +86,17 @@ def test_tiled_free_running_paper_regime_at_benchmark_shapes(kind, h):
     assert E.e2ttt_device_status(hd["ws"]) == 0
     errs = check_forward(got, ref, TOL_BF16, "tiled paper regime, 16 chunks free-running")
     print(kind, errs)
+
+
+@pytest.mark.parametrize("io,impl", [("bf16", E.E2TTT_IMPL_TILED), ("f32", E.E2TTT_IMPL_SIMT)], ids=["tiled-bf16", "fma-fp32"])
+@pytest.mark.parametrize("kind", [MLP, SWIGLU])
+def test_wide_networks_forward_and_backward(kind, io, impl):
+    """d = 256, h = 1024 (several tiles in every direction, split-K parts with tails), one chunk of 48 tokens."""
+    r = inputs.paper_regime(inputs.Recipe(B=1, H=1, L=48, d=256, h=1024, C=48, kind=kind, io=io, seed=13, m_std=0.002))
+    x = inputs.generate(r, with_d_o=True, with_dstate=True)
+    shape = dict(d=r.d, h=r.h, C=r.C, kind=kind, io=io)
+    tol = TOL_BF16 if io == "bf16" else 1e-4
+    got, hd = util.gpu_forward(x, impl=impl, **shape)
+    assert E.e2ttt_device_status(hd["ws"]) == 0
+    check_forward(got, util.oracle_forward(x, r.C, kind), tol, "wide forward")
+    check_backward(util.gpu_backward(x, impl=impl, **shape), util.oracle_backward(x, r.C, kind), tol, "wide backward")
