@@ -1,5 +1,5 @@
-// SIMT backward: the adjoint of the chunk program, chunks in reverse order, one CTA per sequence, for both
-// fast-weight networks.  Per chunk it re-runs the chunk's forward from the saved chunk-start state, then reverses,
+// Any-shape backward: the adjoint of the chunk program, chunks in reverse order, a cluster of 1-8 CTAs per sequence,
+// for both fast-weight networks, on the same two GEMM engines as the forward (tc_gemm.cuh).  Per chunk it re-runs the chunk's forward from the saved chunk-start state, then reverses,
 // in matrix form over the whole chunk,
 //   (i)   the outputs o = f_{W0}(q),
 //   (ii)  the closed-form state transition of Proposition 1 (carries cw, cm, cb and kernels K^W, K^M),

@@ -1,4 +1,4 @@
-// Building blocks of the SIMT (CUDA-core) kernels: one CTA per sequence, 256 threads.
+// Building blocks of the any-shape kernels (scans, layer norm, reductions, phase barrier, the FMA GEMM).
 // Real = double for fp32 I/O, float for bf16 I/O.
 #pragma once
 #include <cuda_bf16.h>

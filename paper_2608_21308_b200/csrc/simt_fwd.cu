@@ -1,5 +1,7 @@
-// SIMT forward: Algorithm 1 applied chunk after chunk, one CTA per sequence, for any shape.
-// The fp32-I/O instantiation computes in fp64 and is the GPU-side reference for the tensor-core path.
+// Any-shape forward: Algorithm 1 applied chunk after chunk for any d, h, C and both networks.  A cluster of 1-8 CTAs
+// works on one sequence; the CTAs split every phase and share state and intermediates through the workspace, meeting
+// at the cluster barrier between phases.  The matrix products run on one of two engines (tc_gemm.cuh): CUDA-core FMAs
+// (fp64 for fp32 I/O - the GPU-side reference of the tensor-core paths - or fp32), or tcgen05 MMAs for bf16 I/O.
 #include <type_traits>
 
 #include "simt_common.cuh"
