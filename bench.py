@@ -507,6 +507,27 @@ def run_decode(args, r):
     clocks = sampler.stop()
     ms_eager = timed(step, steps, 3)
     ms_e2e = timed(step_e2e, steps, 3)
+
+    # the other half of decoding: once C tokens have accumulated, e2ttt_chunk_fwd over them moves the state on
+    C = r.C
+    rc = inputs.Recipe(**{**r.__dict__, "L": C})
+    xc = inputs.generate(rc)
+    pc = E.make_params(r.B, r.H, C, r.d, r.h, C, r.kind, E.E2TTT_F32 if r.io == "f32" else E.E2TTT_BF16, 1e-5,
+                       E.E2TTT_IMPL_AUTO)
+    sc4, sc3 = (r.B, r.H, C, r.d), (r.B, r.H, C)
+    cq, ck, cv = (torch.from_numpy(xc[n]).to(iod).view(sc4).to(dev) for n in ("q", "k", "v"))
+    ce, cb, cg = (torch.from_numpy(xc[n]).view(sc3).to(dev) for n in ("eta", "beta", "gamma"))
+    co = torch.empty_like(cq)
+    Wn = [torch.empty_like(w) for w in Ws[0]]
+    Mn = [torch.empty_like(w) for w in Ws[0]]
+    wsc = torch.empty(E.e2ttt_workspace_bytes(pc, 0), dtype=torch.uint8, device=dev)
+    iu = [0]
+
+    def update():
+        E.e2ttt_chunk_fwd(pc, cq, ck, cv, ce, cb, cg, Ws[iu[0] % copies], None, co, Wn, Mn, wsc, 0, stream)
+        iu[0] += 1
+
+    ms_update = timed(update, max(20, copies), 3)
     pk = peaks()
     io_bytes = 2 * N * r.d * (2 if r.io == "bf16" else 4)
     nbytes = state_bytes + io_bytes
@@ -523,7 +544,10 @@ def run_decode(args, r):
             "roofline": {"bound": "hbm", "achieved": nbytes / (ms * 1e-3) / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
                          "frac": nbytes / (ms * 1e-3) / 1e9 / pk["hbm_gbs"], "traffic": None, "peak_source": pk["_source"],
                          "kernel": "apply kernel (one launch per step, steps replayed from a CUDA graph)",
-                         "bytes_per_launch": nbytes, "ms_per_step_launched_from_python": ms_eager}}
+                         "bytes_per_launch": nbytes, "ms_per_step_launched_from_python": ms_eager},
+            "chunk_update": {"ms": ms_update, "every_tokens": C,
+                             "ms_per_token_amortised": ms + ms_update / C,
+                             "what": "e2ttt_chunk_fwd over the C accumulated tokens of every sequence (state in, state out)"}}
     print(json.dumps(line))
 
 
