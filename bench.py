@@ -602,10 +602,22 @@ def run_prepare(args, r):
     ms = timed(step, steps, args.warmup)
     clocks = sampler.stop()
     ms_e2e = timed(step_e2e, max(2, steps // 4), 1)
+    # the reverse pass of the same step (training): adjoints of q_raw, k_raw and the gate logits
+    dq, dk = torch.randn(s4, generator=gen).to(iod).to(dev), torch.randn(s4, generator=gen).to(iod).to(dev)
+    dg = [torch.randn(s3, generator=gen).to(dev) for _ in range(3)]
+    dqr, dkr = torch.empty_like(dq), torch.empty_like(dk)
+    dlog = [torch.empty(s3, dtype=torch.float32, device=dev) for _ in range(3)]
+
+    def step_bwd():
+        E.e2ttt_prepare_bwd(p, gp, t["q_raw"], t["k_raw"], t["a_eta"], t["a_beta"], t["a_alpha"], dq, dk, dg[0], dg[1], dg[2],
+                            dqr, dkr, dlog[0], dlog[1], dlog[2], stream)
+
+    ms_bwd = timed(step_bwd, steps, args.warmup)
     pk = peaks()
     rows = r.B * r.H * r.L
     es = 2 if r.io == "bf16" else 4
     nbytes = rows * (4 * r.d * es + 24)
+    nbytes_bwd = rows * (6 * r.d * es + 36)
     line = {"metric": "e2ttt_prepare_tokens_per_s", "value": r.B * r.L / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": steps,
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
@@ -618,7 +630,11 @@ def run_prepare(args, r):
             "gpu_launches": steps, "clocks": clocks,
             "roofline": {"bound": "hbm", "achieved": nbytes / (ms * 1e-3) / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
                          "frac": nbytes / (ms * 1e-3) / 1e9 / pk["hbm_gbs"], "traffic": None, "peak_source": pk["_source"],
-                         "kernel": "prepare_fwd_kernel (one launch per step)", "bytes_per_launch": nbytes}}
+                         "kernel": "prepare_fwd_bulk_kernel (one launch per step)", "bytes_per_launch": nbytes},
+            "reverse": {"ms_per_step": ms_bwd, "bytes_per_launch": nbytes_bwd,
+                        "achieved_gbs": nbytes_bwd / (ms_bwd * 1e-3) / 1e9,
+                        "frac_of_hbm_peak": nbytes_bwd / (ms_bwd * 1e-3) / 1e9 / pk["hbm_gbs"],
+                        "kernel": "prepare_bwd_bulk_kernel"}}
     print(json.dumps(line))
 
 

@@ -9,7 +9,8 @@
 // The forward of rows that allow it (row bytes a multiple of 16, aligned bases, d <= 256) runs as a bulk-copy pipeline
 // instead: tiles of 32 tokens travel global -> shared memory -> global with `cp.async.bulk` (mbarrier transaction
 // counts on the way in, bulk groups on the way out), four tiles deep per CTA, so the bytes in flight do not depend
-// on registers or occupancy; the warps only touch shared memory.
+// on registers or occupancy; the warps only touch shared memory.  The reverse pass has the same form (four tiles in,
+// two out, three deep).
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -381,6 +382,172 @@ template <typename IO, typename Args, typename F> int dispatch(const Shape& s, F
     return launch(std::integral_constant<int, 1>(), std::integral_constant<int, 32>());
 }
 
+// ---- reverse pass as the same kind of pipeline: four tiles in (x of q and k, y_bar of q and k), two out (in place) ----
+constexpr int kBkStagesBwd = 3;
+
+template <typename IO> __device__ __forceinline__ float pr_sig(float x) {
+    if (sizeof(IO) == 2) {  // bf16 I/O: hardware tanh, sigmoid(x) = 0.5 + 0.5 tanh(x / 2)
+        float t;
+        asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(0.5f * x));
+        return fmaf(0.5f, t, 0.5f);
+    }
+    return pr_sigmoid(x);
+}
+
+template <typename IO, int LPR>
+__global__ void __launch_bounds__(kPrThreads) prepare_bwd_bulk_kernel(const PrepareBwdArgs a) {
+    extern __shared__ __align__(128) unsigned char pr_smem[];
+    const int d = a.f.d;
+    const uint32_t row_bytes = (uint32_t)d * sizeof(IO);
+    const uint32_t tile_bytes = kBkTok * row_bytes;
+    uint64_t* full = reinterpret_cast<uint64_t*>(pr_smem);
+    volatile int* dead = reinterpret_cast<volatile int*>(pr_smem + 64);
+    unsigned char* tiles = pr_smem + 128;  // [stages][4][tile_bytes]: x_q, x_k, g_q, g_k
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const long long ntiles = (a.f.rows + kBkTok - 1) / kBkTok;
+    const IO* src[4] = {reinterpret_cast<const IO*>(a.f.q_raw), reinterpret_cast<const IO*>(a.f.k_raw),
+                        reinterpret_cast<const IO*>(a.dq), reinterpret_cast<const IO*>(a.dk)};
+    IO* dst[2] = {reinterpret_cast<IO*>(a.dq_raw), reinterpret_cast<IO*>(a.dk_raw)};
+
+    if (tid == 0) {
+        for (int s = 0; s < kBkStagesBwd; ++s) sm100::mbar_init(&full[s], 1);
+        *dead = 0;
+        sm100::fence_mbar_init();
+    }
+    __syncthreads();
+    auto tokens_of = [&](long long tile) { return (int)min((long long)kBkTok, a.f.rows - tile * kBkTok); };
+    auto issue = [&](long long tile, int s) {  // thread 0
+        const uint32_t bytes = (uint32_t)tokens_of(tile) * row_bytes;
+        sm100::mbar_expect_tx(&full[s], 4 * bytes);
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            bulk_load(tiles + (size_t)(4 * s + i) * tile_bytes, src[i] + (size_t)tile * kBkTok * d, bytes, &full[s]);
+    };
+    if (tid == 0)
+        for (int i = 0; i < kBkStagesBwd; ++i) {
+            const long long tile = blockIdx.x + (long long)i * gridDim.x;
+            if (tile < ntiles) issue(tile, i);
+        }
+
+    long long it = 0;
+    for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++it) {
+        const int s = (int)(it % kBkStagesBwd);
+        const uint32_t parity = (uint32_t)((it / kBkStagesBwd) & 1);
+        const int ntok = tokens_of(tile);
+        if (!bulk_wait_tile(&full[s], parity, dead)) break;
+        unsigned char* st = tiles + (size_t)(4 * s) * tile_bytes;
+        if (tid < ntok) {  // adjoints of the gate logits
+            const long long t = tile * kBkTok + tid;
+            const float sa = pr_sigmoid(a.f.a_eta[t]), sb = pr_sigmoid(a.f.a_beta[t]), sc = pr_sigmoid(a.f.a_alpha[t]);
+            const float eta = a.f.eta_base * sa, alpha = a.f.alpha_base * sc;
+            const float beta = __powf(sb, 1.0f / a.f.tau);
+            const float eta_bar = a.d_eta[t] - a.d_gamma[t] * alpha;
+            a.da_eta[t] = eta_bar * a.f.eta_base * sa * (1.0f - sa);
+            a.da_beta[t] = a.d_beta[t] * beta * (1.0f - sb) / a.f.tau;
+            a.da_alpha[t] = -a.d_gamma[t] * eta * a.f.alpha_base * sc * (1.0f - sc);
+        }
+        {
+            constexpr int E = 16 / (int)sizeof(IO), RPP = 32 / LPR;
+            const int sub = lane / LPR, li = lane % LPR;
+            for (int base = warp * RPP; base < 2 * kBkTok; base += (kPrThreads / 32) * RPP) {
+                const int r = base + sub;
+                const int u = r & (kBkTok - 1), which = r >= kBkTok ? 1 : 0;
+                const bool valid = u < ntok;
+                const IO* xp = reinterpret_cast<const IO*>(st + (size_t)which * tile_bytes) + (size_t)u * d + li * E;
+                IO* gp = reinterpret_cast<IO*>(st + (size_t)(2 + which) * tile_bytes) + (size_t)u * d + li * E;
+                float x[E], g[E];
+#pragma unroll
+                for (int j = 0; j < E; ++j) { x[j] = 0.0f; g[j] = 0.0f; }
+                if (valid) {
+                    const uint4 rx = *reinterpret_cast<const uint4*>(xp), rg = *reinterpret_cast<const uint4*>(gp);
+                    if (sizeof(IO) == 2) {
+                        const __nv_bfloat162* hx = reinterpret_cast<const __nv_bfloat162*>(&rx);
+                        const __nv_bfloat162* hg = reinterpret_cast<const __nv_bfloat162*>(&rg);
+#pragma unroll
+                        for (int j = 0; j < E / 2; ++j) {
+                            const float2 fx = __bfloat1622float2(hx[j]), fg = __bfloat1622float2(hg[j]);
+                            x[2 * j] = fx.x; x[2 * j + 1] = fx.y;
+                            g[2 * j] = fg.x; g[2 * j + 1] = fg.y;
+                        }
+                    } else {
+                        const float* fx = reinterpret_cast<const float*>(&rx);
+                        const float* fg = reinterpret_cast<const float*>(&rg);
+#pragma unroll
+                        for (int j = 0; j < E; ++j) { x[j] = fx[j]; g[j] = fg[j]; }
+                    }
+                }
+                float ss = 0.0f, sg = 0.0f;
+#pragma unroll
+                for (int j = 0; j < E; ++j) {
+                    const float sig = pr_sig<IO>(x[j]);
+                    const float sv = x[j] * sig;
+                    const float dsl = sig * (1.0f + x[j] * (1.0f - sig));  // silu'(x)
+                    ss = fmaf(sv, sv, ss);
+                    sg = fmaf(sv, g[j], sg);
+                    g[j] *= dsl;       // y_bar silu'(x)
+                    x[j] = sv * dsl;   // s silu'(x)
+                }
+#pragma unroll
+                for (int off = LPR / 2; off > 0; off >>= 1) {
+                    ss += __shfl_xor_sync(0xffffffffu, ss, off);
+                    sg += __shfl_xor_sync(0xffffffffu, sg, off);
+                }
+                const float eps = a.f.norm_eps;
+                const bool big = ss > eps * eps;
+                const float inv = big ? rsqrtf(ss) : __fdividef(1.0f, eps);   // 1 / max(||s||, eps)
+                const float proj = big ? sg * inv * inv : 0.0f;                // <y_bar, y> / m
+                if (valid) {
+                    uint4 raw;
+                    if (sizeof(IO) == 2) {
+                        __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&raw);
+#pragma unroll
+                        for (int j = 0; j < E / 2; ++j)
+                            h2[j] = __floats2bfloat162_rn((g[2 * j] - x[2 * j] * proj) * inv, (g[2 * j + 1] - x[2 * j + 1] * proj) * inv);
+                    } else {
+                        float* f4 = reinterpret_cast<float*>(&raw);
+#pragma unroll
+                        for (int j = 0; j < E; ++j) f4[j] = (g[j] - x[j] * proj) * inv;
+                    }
+                    *reinterpret_cast<uint4*>(gp) = raw;  // the adjoint replaces y_bar in its tile
+                }
+            }
+        }
+        sm100::fence_proxy_async_smem();
+        __syncthreads();
+        if (tid == 0) {
+            const uint32_t bytes = (uint32_t)ntok * row_bytes;
+            bulk_store(dst[0] + (size_t)tile * kBkTok * d, st + (size_t)2 * tile_bytes, bytes);
+            bulk_store(dst[1] + (size_t)tile * kBkTok * d, st + (size_t)3 * tile_bytes, bytes);
+            bulk_commit();
+            if (it >= 1) {
+                bulk_wait_read<1>();
+                const long long next = tile + (long long)(kBkStagesBwd - 1) * gridDim.x;
+                if (next < ntiles) issue(next, (int)((it - 1) % kBkStagesBwd));
+            }
+        }
+    }
+    if (tid == 0) bulk_wait_all<0>();
+    __syncthreads();
+}
+
+template <typename IO, int LPR> int bwd_bulk(const PrepareBwdArgs& a, cudaStream_t st) {
+    const size_t smem = 128 + (size_t)kBkStagesBwd * 4 * kBkTok * a.f.d * sizeof(IO);
+    static size_t attr_bytes[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return (int)cudaGetLastError();
+    if (dev < 0 || dev >= 64 || attr_bytes[dev] < smem) {
+        cudaError_t e = cudaFuncSetAttribute(prepare_bwd_bulk_kernel<IO, LPR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return (int)e;
+        if (dev >= 0 && dev < 64) attr_bytes[dev] = smem;
+    }
+    const long long ntiles = (a.f.rows + kBkTok - 1) / kBkTok;
+    const int per_sm = (int)(220 * 1024 / smem);
+    const long long cap = 148LL * (per_sm > 4 ? 4 : per_sm);
+    const int grid = (int)(ntiles < cap ? ntiles : cap);
+    prepare_bwd_bulk_kernel<IO, LPR><<<grid, kPrThreads, smem, st>>>(a);
+    return (int)cudaGetLastError();
+}
+
 size_t bulk_smem_bytes(int d, size_t io_bytes) { return 128 + (size_t)kBkStages * 2 * kBkTok * d * io_bytes; }
 
 template <typename IO, int LPR> int fwd_bulk(const PrepareArgs& a, cudaStream_t st) {
@@ -423,6 +590,14 @@ template <typename IO> int fwd_io(const PrepareArgs& a, cudaStream_t st) {
 template <typename IO> int bwd_io(const PrepareBwdArgs& a, cudaStream_t st) {
     const void* ptrs[6] = {a.f.q_raw, a.f.k_raw, a.dq, a.dk, a.dq_raw, a.dk_raw};
     const Shape s = pick_shape(a.f.d, (int)sizeof(IO), ptrs, 6);
+    bool al = true;
+    for (int i = 0; i < 6; ++i) al = al && (reinterpret_cast<uintptr_t>(ptrs[i]) % 16 == 0);
+    const int lpr = (int)(a.f.d * sizeof(IO) / 16);
+    if (al && (size_t)lpr * 16 == a.f.d * sizeof(IO) && (lpr == 8 || lpr == 16 || lpr == 32) && a.f.rows >= 4 * kBkTok) {
+        if (lpr == 8) return bwd_bulk<IO, 8>(a, st);
+        if (lpr == 16) return bwd_bulk<IO, 16>(a, st);
+        return bwd_bulk<IO, 32>(a, st);
+    }
     const int grid = grid_for(a.f.rows, 1);
     return dispatch<IO, PrepareBwdArgs>(s, [&](auto v, auto np) {
         prepare_bwd_kernel<IO, decltype(v)::value, decltype(np)::value><<<grid, kPrThreads, 0, st>>>(a);
