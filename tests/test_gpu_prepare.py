@@ -93,3 +93,23 @@ def test_prepare_feeds_the_chunk_update_in_the_papers_gate_regime():
     ref = util.oracle_forward(xin, 64, inputs.KIND_MLP)
     out, _ = util.gpu_forward(xin, d=d, h=512, C=64, kind=inputs.KIND_MLP, io="bf16")
     assert util.rel_err(out["o"], ref["o"]) <= 2e-2
+
+
+@pytest.mark.parametrize("L", [9, 4000])
+def test_prepare_forward_in_place(L):
+    """q and k may alias q_raw and k_raw (both code paths: the per-row kernel and the bulk-copy pipeline)."""
+    B, H, d = 2, 2, 128
+    rng = np.random.default_rng(7)
+    x = {n: _bf16(rng.standard_normal((B, H, L, d)).astype(np.float32)) for n in ("q_raw", "k_raw")}
+    s = {n: rng.standard_normal((B, H, L)).astype(np.float32) for n in ("a_eta", "a_beta", "a_alpha")}
+    p = E.make_params(B, H, L, d, 4 * d, 1, inputs.KIND_MLP, E.E2TTT_BF16, 1e-5, E.E2TTT_IMPL_AUTO)
+    gp = E.e2ttt_gate_params(GP["eta_base"], GP["tau"], GP["alpha_base"], GP["norm_eps"])
+    dev = lambda a, t=torch.float32: torch.tensor(a, dtype=torch.float32).to(t).cuda().contiguous()
+    qr, kr = dev(x["q_raw"], torch.bfloat16), dev(x["k_raw"], torch.bfloat16)
+    ae, ab, aa = dev(s["a_eta"]), dev(s["a_beta"]), dev(s["a_alpha"])
+    q, k = torch.empty_like(qr), torch.empty_like(kr)
+    eta, beta, gamma = torch.empty_like(ae), torch.empty_like(ae), torch.empty_like(ae)
+    E.e2ttt_prepare_fwd(p, gp, qr, kr, ae, ab, aa, q, k, eta, beta, gamma)
+    E.e2ttt_prepare_fwd(p, gp, qr, kr, ae, ab, aa, qr, kr, eta, beta, gamma)   # in place
+    torch.cuda.synchronize()
+    assert torch.equal(q, qr) and torch.equal(k, kr)
