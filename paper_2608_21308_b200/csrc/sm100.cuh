@@ -39,7 +39,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     if (CLUSTER) {
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
+#ifdef DBG_TESTWAIT
+            "mbarrier.test_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+#else
             "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+#endif
             "selp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(ok)
             : "r"(smem_u32(bar)), "r"(parity)
@@ -87,11 +91,28 @@ __device__ __forceinline__ bool mbar_wait_one(uint64_t* bar, uint32_t parity, co
     }
     return true;
 }
-// Warp-collective wait (all 32 lanes call it together): lane 0 waits, the others park at the warp barrier, which
-// also orders their later reads after lane 0's acquire.
+// Warp-collective wait (all 32 lanes call it together, converged).  Every lane polls: the warp stays converged while
+// it waits.  (One polling lane with the other 31 parked at a warp barrier makes the scheduler alternate between the
+// two divergent paths, and the polling lane then misses the completion by thousands of cycles.)
 template <bool CLUSTER = false>
 __device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, const WaitCtx& w, int where) {
-    if ((threadIdx.x & 31) == 0) mbar_wait_one<CLUSTER>(bar, parity, w, where);
+    if (!*w.dead && !mbar_try_wait<CLUSTER>(bar, parity)) {
+        const long long t0 = clock64();
+        int spins = 0;
+        while (!mbar_try_wait<CLUSTER>(bar, parity)) {
+#if defined(E2TTT_POLL_SLEEP)
+            __nanosleep(E2TTT_POLL_SLEEP);
+#endif
+            if ((++spins & 63) == 0) {
+                if (*w.dead) break;
+                if (clock64() - t0 > kWaitCycles) {
+                    *w.dead = 1;
+                    atomicCAS(w.status, 0, where);
+                    break;
+                }
+            }
+        }
+    }
     __syncwarp();
 }
 
@@ -178,6 +199,25 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate)
         : "memory");
+}
+// The same, called by all 32 converged lanes of a warp: the instruction is predicated on `issue` (true in one lane),
+// so the warp issues one MMA and stays converged (a one-lane branch would leave 31 lanes parked at a warp barrier).
+__device__ __forceinline__ void umma_bf16_elect(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool accumulate,
+                                                bool issue) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "setp.ne.b32 q, %5, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate), "r"((uint32_t)issue)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit_elect(uint64_t* bar, bool issue) {
+    asm volatile(
+        "{\n\t.reg .pred q;\n\t"
+        "setp.ne.b32 q, %1, 0;\n\t"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+        ::"r"(smem_u32(bar)), "r"((uint32_t)issue) : "memory");
 }
 // All MMAs issued so far by this thread arrive on `bar` when they have completed.
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {

@@ -4,7 +4,7 @@
 // Everything that carries over from chunk to chunk stays on chip for the whole sequence:
 //   - fp32 master copy of the CTA's W1/W2 slices: tensor memory columns [0,256).  The aggregation MMAs
 //     accumulate -sum_t K^W_t grad_t straight into it (it is pre-scaled by the decay carry cw beforehand).
-//   - fp32 master copy of the momentum slices: registers (each thread keeps the 2 x 128/NG elements it owns).
+//   - fp32 master copy of the momentum slices: registers (each epilogue thread keeps the 2 x 32 elements it owns).
 //   - bf16 operand copy of W1/W2: shared memory, refreshed once per chunk from the fp32 master.
 // Per chunk (Algorithm 1), rows = tokens (64 keys then 64 queries), all GEMMs on tcgen05 with TMEM accumulators:
 //   G1  Z = [K;Q] W1c^T          G2  Upart = gelu(Z) W2c^T      -> cross-CTA sum of Upart through DSMEM (each CTA
@@ -13,9 +13,16 @@
 //   aggregations (contraction over the 64 tokens, MN-major operands):
 //       W1c -= (kW*Pz)^T K    M1acc = -(kM*Pz)^T K    W2c -= Pu^T (kW*Ak)    M2acc = -Pu^T (kM*Ak)
 //   state pass: W = Wacc + cm M0;  M = cb M0 + Macc;  bf16(W) -> shared;  cw_next W -> TMEM.
+//
+// Warp roles (640 threads): warps 0-15 are epilogue warps (warp w reads TMEM lanes 32 (w & 3) .., columns
+// 32 (w >> 2) ..; quadrants 0/1 hold the key rows, 2/3 the query rows); warp 18 is the MMA issuer (one lane issues,
+// descriptors are compile-time offsets from one base); warp 19 loads tokens by TMA and runs the gate scans of the
+// next chunk.  Nothing is CTA-wide inside the chunk loop: producers and consumers meet on mbarriers (one per
+// buffer), the issuer never touches an epilogue.  setmaxnreg moves registers from the control warps to the epilogue warps.
 // Every wait on an mbarrier is bounded (sm100.cuh); a wait that gives up is reported through the status word.
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
 #include "simt_common.cuh"
@@ -26,24 +33,38 @@ namespace e2ttt {
 using namespace sm100;
 
 #ifdef TC_PROFILE
-// Debug build only: cycle stamps of thread 0 of CTA 0 at the phase boundaries of the first 64 chunks.
-__device__ long long g_tc_prof[4 * 32 * 16];
-#define PROF(i)                                                                                          \
-    do {                                                                                                 \
-        if ((threadIdx.x == 0 || threadIdx.x == 64) && (blockIdx.x == 0 || blockIdx.x == 2) && r < 32)    \
-            g_tc_prof[(((blockIdx.x >> 1) * 2 + (threadIdx.x >> 6)) * 32 + r) * 16 + (i)] = clock64();    \
+#ifndef TC_PROF_CTAS
+#define TC_PROF_CTAS 1
+#endif
+#ifndef TC_PROF_MASK
+#define TC_PROF_MASK 15
+#endif
+// Debug build only: cycle stamps at the phase boundaries of the first 32 chunks, CTA 0 of the grid, for one
+// key-row warp (thread 0), one query-row warp (thread 64), the issuer (thread 576) and the loader (thread 608).
+__device__ long long g_tc_prof[16 * 32 * 24];
+#define PROF(i)                                                                                      \
+    do {                                                                                             \
+        const int t_ = threadIdx.x;                                                                  \
+        if (blockIdx.x < TC_PROF_CTAS && r < 32 && (t_ == 0 || t_ == 64 || t_ == 576 || t_ == 608) && (blockIdx.x == 0 || ((TC_PROF_MASK >> ((t_ == 0) ? 0 : (t_ == 64) ? 1 : (t_ == 576) ? 2 : 3)) & 1)))            \
+            g_tc_prof[(((blockIdx.x * 4) + ((t_ == 0) ? 0 : (t_ == 64) ? 1 : (t_ == 576) ? 2 : 3)) * 32 + r) * 24 + (i)] = clock64(); \
     } while (0)
 #else
 #define PROF(i)
 #endif
 
+
 namespace {
 
 constexpr int D = 128, HC = 128, C = 64, NC = 4;
-constexpr int NG = TC_NG;                // column groups per TMEM lane quadrant
-constexpr int NTHREADS = 128 * NG;
+constexpr int NG = 4;                    // column groups per TMEM lane quadrant
+constexpr int NEPI = 128 * NG;           // epilogue threads
+constexpr int NTHREADS = NEPI + 128;     // + one control warpgroup (issuer warp, loader warp, two idle warps)
+constexpr int NEW = NEPI / 32;           // epilogue warps
 constexpr int CW = 128 / NG;             // accumulator columns a thread owns in a 128-column region
 constexpr int NB = CW / 16;              // 16-column batches per thread
+// The kernel starts with 96 registers per thread (640 threads).  The control warpgroup drops to 32 and its 64 x 128
+// registers go to the 512 epilogue threads (+16 each): a warp can only take what its own CTA released.
+constexpr int EPI_REGS = 112, CTRL_REGS = 32;
 
 // TMEM columns
 constexpr uint32_t T_W1 = 0, T_W2 = 128, T_R0 = 256, T_R1 = 384;
@@ -65,17 +86,34 @@ struct __align__(1024) Smem {
     uint8_t PzM[2][8192];  // kM_t pz                                                 staging slot 1
     uint8_t Stage2[16384]; // staging slot 2
     Scalars sc[2];
-    uint64_t bar_x, bar_g1, bar_g2, bar_g3, bar_agg, bar_agg2, bar_ak, bar_v, bar_ksent, bar_partK, bar_partQ, bar_pu, bar_credit, bar_rs;
+    // TMA / loader
+    uint64_t bar_x, bar_v, bar_sc;
+    // MMA completions (tcgen05.commit)
+    uint64_t bar_g1, bar_g2, bar_g3, bar_aw1, bar_am1, bar_am2;
+    // epilogue warps -> issuer: operand tiles written / accumulator regions read
+    uint64_t bar_a, bar_ak, bar_pz, bar_r1, bar_w1, bar_w2;
+    // cluster traffic
+    uint64_t bar_go, bar_ksent, bar_partK, bar_partQ, bar_pu, bar_credit, bar_rs;
     uint32_t tmem_base;
     int dead;
 };
 
-__device__ __forceinline__ uint64_t desc_k(uint32_t base, uint32_t slab_stride, int k) {
-    return make_smem_desc(base + (uint32_t)(k >> 2) * slab_stride + (uint32_t)(k & 3) * 32u, 16, 1024);
+// Shared-memory matrix descriptors as compile-time offsets from one run-time value: base16 = (address of the tile) >> 4.
+// High word: SBO = 1024 B, descriptor version 1, 128-byte swizzle.  Low word: start address >> 4 | LBO >> 4 << 16.
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+// K-major operand: k-step k covers columns 16k..16k+15 of slab (k >> 2); LBO is unused (16 B).
+__device__ __forceinline__ uint64_t dk(uint32_t base16, uint32_t slab_stride, int k) {
+    return ((uint64_t)kDescHi << 32) | (uint64_t)(base16 + (((uint32_t)(k >> 2) * slab_stride + (uint32_t)(k & 3) * 32u) >> 4) + (1u << 16));
 }
-__device__ __forceinline__ uint64_t desc_mn(uint32_t base, uint32_t slab_stride, int k) {
-    return make_smem_desc(base + (uint32_t)k * 2048u, slab_stride, 1024);
+// MN-major operand: k-step k covers rows 16k..16k+15; LBO = distance between the slabs of 64 M/N indices.
+__device__ __forceinline__ uint64_t dmn(uint32_t base16, uint32_t slab_stride, int k) {
+    return ((uint64_t)kDescHi << 32) | (uint64_t)(base16 + (((uint32_t)k * 2048u) >> 4) + ((slab_stride >> 4) << 16));
 }
+
+__device__ __forceinline__ void named_sync(int id, int nthreads) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory"); }
+__device__ __forceinline__ void named_arrive(int id, int nthreads) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(nthreads) : "memory"); }
+// barrier ids (0 is __syncthreads)
+constexpr int BAR_EPI = 1, BAR_STAGE = 3, BAR_KOWN = 4, BAR_QOWN = 5;
 
 // Suffix scans of one 64-token chunk by one warp (two tokens per lane), same recurrences as the SIMT path:
 // a step is the map (bt, gt, S) -> (beta bt, gamma gt, beta S + gamma gt); suffix composites by warp shuffles.
@@ -141,22 +179,56 @@ __device__ __forceinline__ float gelu_fast(float z, float& dgelu) {
     return fmaf(hz, t, hz);
 }
 
-// Staging slot for partial sums: 32 rows x 128 fp32, kept as 16-byte pieces.  Piece c4 (4 columns) of row r sits at
-// piece index c4 * 32 + (r ^ ((c4 >> 1) & 15)): the 16 lanes that send one piece of 16 neighbouring rows write 256
+// g'(z) alone
+__device__ __forceinline__ float gelu_d1_fast(float z) {
+    const float z2 = z * z;
+    const float t = fast_tanh(z * fmaf(0.0356774081f, z2, 0.7978845608f));
+    const float du = fmaf(0.1070322243f, z2, 0.7978845608f);
+    return fmaf((0.5f * z) * fmaf(-t, t, 1.0f), du, fmaf(0.5f, t, 0.5f));
+}
+
+// Staging slot for fp32 partial sums: 16 rows x 128 fp32 = 8 KB, kept as 16-byte pieces.  Piece c4 (4 columns) of row r
+// sits at piece index c4 * 16 + (r ^ ((c4 >> 1) & 15)): the 16 lanes that send one piece of 16 neighbouring rows write 256
 // contiguous bytes (DSMEM moves whole segments; scattered 16-byte stores cost several times the bandwidth), and the
 // layer-norm readers (16 threads per row, pieces 2cg and 2cg+1) spread over all banks.
 __device__ __forceinline__ uint32_t stage_offset(uint32_t c4, uint32_t r) {
-    return (c4 * 32u + (r ^ ((c4 >> 1) & 15u))) << 4;
+    return (c4 * 16u + (r ^ ((c4 >> 1) & 15u))) << 4;
+}
+// The same for bf16 partial sums: 16 rows x 128 bf16 = 4 KB, piece c8 (8 columns) of row r at c8 * 16 + (r ^ c8).
+__device__ __forceinline__ uint32_t stage_offset_q(uint32_t c8, uint32_t r) {
+    return (c8 * 16u + (r ^ c8)) << 4;
+}
+// Bulk copy of `bytes` (a multiple of 16) from this CTA's shared memory into a peer's; the peer's mbarrier gets the bytes.
+__device__ __forceinline__ void bulk_copy_to_cta(uint32_t dst_cluster_addr, uint32_t src_addr, uint32_t bytes, uint32_t dst_cluster_mbar) {
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_cluster_addr), "r"(src_addr), "r"(bytes), "r"(dst_cluster_mbar) : "memory");
 }
 
-// 16 bf16 (32 bytes) = two 16-byte chunks into a swizzled slab row
-__device__ __forceinline__ void st_slab16(uint8_t* slab, int row, int col0, const float (&v)[16]) {
+// 16 bf16 (32 bytes, already packed in pairs) = two 16-byte chunks into a swizzled slab row
+__device__ __forceinline__ void st_slab16p(uint8_t* slab, int row, int col0, const uint32_t (&p)[8]) {
     const int c = col0 >> 3;
-    uint4 a, b;
-    a.x = pack_bf16(v[0], v[1]); a.y = pack_bf16(v[2], v[3]); a.z = pack_bf16(v[4], v[5]); a.w = pack_bf16(v[6], v[7]);
-    b.x = pack_bf16(v[8], v[9]); b.y = pack_bf16(v[10], v[11]); b.z = pack_bf16(v[12], v[13]); b.w = pack_bf16(v[14], v[15]);
-    *reinterpret_cast<uint4*>(slab + row * 128 + (((c) ^ (row & 7)) << 4)) = a;
-    *reinterpret_cast<uint4*>(slab + row * 128 + (((c + 1) ^ (row & 7)) << 4)) = b;
+    *reinterpret_cast<uint4*>(slab + row * 128 + (((c) ^ (row & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
+    *reinterpret_cast<uint4*>(slab + row * 128 + (((c + 1) ^ (row & 7)) << 4)) = make_uint4(p[4], p[5], p[6], p[7]);
+}
+__device__ __forceinline__ void st_slab16(uint8_t* slab, int row, int col0, const float (&v)[16]) {
+    uint32_t p[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) p[i] = pack_bf16(v[2 * i], v[2 * i + 1]);
+    st_slab16p(slab, row, col0, p);
+}
+
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+    const __half2 v = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+// A warp has finished writing operand tiles in shared memory (generic proxy) and / or reading or writing tensor
+// memory: make that visible to the MMA issuer, then one lane arrives.
+__device__ __forceinline__ void warp_release(uint64_t* bar) {
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
 }
 
 // PAD = false: the native 128 x 512 shape, every mask folds away.  PAD = true: d and h come from the arguments.
@@ -175,27 +247,14 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     }
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int q = warp & 3;          // TMEM lane quadrant
-    const int g = warp >> 2;         // column group
-    const int row = 32 * q + lane;   // TMEM lane this thread reads
-    const int c0 = CW * g;           // first of its columns inside a 128-column region
     const uint32_t me = cluster_ctarank();
     const int seq = blockIdx.x / NC;
-    const int issuer_warp = 2;  // a warp of quadrant 2: free while quadrants 0/1 produce the backward-only operands
-    const bool is_issuer = (warp == issuer_warp) && (lane == 0);
     const int L = a.L, nchunks = L / C;
     WaitCtx wc{&s.dead, a.status};
 
     // Real shape: de x he.  Columns >= de of every token tile and hidden units >= he are zero padding: they stay
     // exactly zero through every product, so only the layer norm (divisor, masks) and the global I/O know about them.
     const int de = PAD ? a.d : D, he = PAD ? a.h : NC * HC;
-    const size_t dh = (size_t)de * he;
-    const bool cta_real = HC * (int)me < he;  // this CTA's 128 hidden units exist
-    const float inv_d = 1.0f / (float)de;
-    // normalisation targets of this thread's rows: hidden unit 128 me + row of W1, output row `row` of W2
-    const float tgt1 = (NORM && cta_real) ? a.norm1[(size_t)seq * he + HC * me + row] : 0.0f;
-    const float tgt2 = (NORM && row < de) ? a.norm2[(size_t)seq * de + row] : 0.0f;
-    __nv_bfloat16* go = a.o + (size_t)seq * L * de;
     const float* eta = a.eta + (size_t)seq * L;
     const float* beta = a.beta + (size_t)seq * L;
     const float* gamma = a.gamma + (size_t)seq * L;
@@ -203,19 +262,27 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     if (tid == 0) {
         s.dead = 0;
         mbar_init(&s.bar_x, 1);
+        mbar_init(&s.bar_v, 1);
+        mbar_init(&s.bar_sc, 1);
         mbar_init(&s.bar_g1, 1);
         mbar_init(&s.bar_g2, 1);
         mbar_init(&s.bar_g3, 1);
-        mbar_init(&s.bar_agg, 1);
-        mbar_init(&s.bar_agg2, 1);
-        mbar_init(&s.bar_ak, 2 * NG);
-        mbar_init(&s.bar_v, 1);
+        mbar_init(&s.bar_aw1, 1);
+        mbar_init(&s.bar_am1, 1);
+        mbar_init(&s.bar_am2, 1);
+        mbar_init(&s.bar_a, NEW);
+        mbar_init(&s.bar_ak, NEW / 2);
+        mbar_init(&s.bar_pz, NEW / 2);
+        mbar_init(&s.bar_r1, NEW);
+        mbar_init(&s.bar_w1, NEW);
+        mbar_init(&s.bar_w2, NEW);
+        mbar_init(&s.bar_ksent, NEW / 2);
+        mbar_init(&s.bar_go, 1);
         mbar_init(&s.bar_partK, 1);  // + 3 x 8 KB of peer partial sums (key rows) per chunk
-        mbar_init(&s.bar_partQ, 1);  // + 3 x 8 KB (query rows)
-        mbar_init(&s.bar_ksent, 2 * NG);
-        mbar_init(&s.bar_pu, 1);    // + 16 KB of pu rows per chunk
+        mbar_init(&s.bar_partQ, 1);  // + 3 x 4 KB (query rows, bf16)
+        mbar_init(&s.bar_pu, 2);     // + 12 KB of pu rows from the peers per chunk, one arrival for the own rows
         mbar_init(&s.bar_credit, 3);
-        mbar_init(&s.bar_rs, 1);    // + 3 x 512 B of peer row sums per chunk (normalisation only)
+        mbar_init(&s.bar_rs, 1);     // + 3 x 512 B of peer row sums per chunk (normalisation only)
         fence_mbar_init();
         tma_prefetch_desc(&tmK);
         tma_prefetch_desc(&tmQ);
@@ -223,674 +290,817 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     }
     if (warp == 0) { tmem_alloc(&s.tmem_base, 512); tmem_relinquish(); }
     if (warp == 1) tc_chunk_scalars(eta, beta, gamma, &s.sc[0]);
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-    const uint32_t tb = s.tmem_base;
-    const uint32_t lane_addr = tb + ((uint32_t)(32 * q) << 16);
-
-    // ---- load the state: fp32 master of W -> TMEM (pre-scaled by the first decay carry) and bf16 -> shared; M -> registers
-    float M1[CW], M2[CW];
-    {
-        const float cw0 = s.sc[0].cw;
-        const size_t head = (size_t)seq * dh;
-        // W1c[j][i]: global W1 [h][d], row 128 me + j
-        const float* w1 = a.W1_init + head + ((size_t)(HC * me) + row) * de + c0;
-        const float* m1 = a.M1_init ? a.M1_init + head + ((size_t)(HC * me) + row) * de + c0 : nullptr;
-        // W2c[i][j]: global W2 [d][h], row i, column 128 me + j
-        const float* w2 = a.W2_init + head + (size_t)row * he + HC * me + c0;
-        const float* m2 = a.M2_init ? a.M2_init + head + (size_t)row * he + HC * me + c0 : nullptr;
-        const bool real2 = cta_real && row < de;  // this thread's W2 row exists
-#pragma unroll
-        for (int b = 0; b < NB; ++b) {
-            float w[16];
-            uint32_t st[16];
-            const bool real1 = cta_real && c0 + 16 * b < de;  // these 16 columns of W1 exist
-#pragma unroll
-            for (int j = 0; j < 16; j += 4) {
-                const float4 x = real1 ? *reinterpret_cast<const float4*>(w1 + 16 * b + j) : make_float4(0.f, 0.f, 0.f, 0.f);
-                w[j] = x.x; w[j + 1] = x.y; w[j + 2] = x.z; w[j + 3] = x.w;
-            }
-#pragma unroll
-            for (int j = 0; j < 16; ++j) { st[j] = __float_as_uint(cw0 * w[j]); M1[16 * b + j] = (m1 && real1) ? m1[16 * b + j] : 0.0f; }
-            tmem_st16(lane_addr + T_W1 + c0 + 16 * b, st);
-            st_slab16(s.W1[(c0 + 16 * b) >> 6], row, (c0 + 16 * b) & 63, w);
-            float* ck = a.ckpt ? a.ckpt + (size_t)seq * a.ckpt_seq_stride : nullptr;  // chunk-start state of chunk 0
-            if (ck && real1) {
-                const size_t o1 = ((size_t)(HC * me) + row) * de + c0 + 16 * b;
-#pragma unroll
-                for (int j = 0; j < 16; j += 4) {
-                    *reinterpret_cast<float4*>(ck + o1 + j) = make_float4(w[j], w[j + 1], w[j + 2], w[j + 3]);
-                    *reinterpret_cast<float4*>(ck + 2 * dh + o1 + j) =
-                        make_float4(M1[16 * b + j], M1[16 * b + j + 1], M1[16 * b + j + 2], M1[16 * b + j + 3]);
-                }
-            }
-#pragma unroll
-            for (int j = 0; j < 16; j += 4) {
-                const float4 x = real2 ? *reinterpret_cast<const float4*>(w2 + 16 * b + j) : make_float4(0.f, 0.f, 0.f, 0.f);
-                w[j] = x.x; w[j + 1] = x.y; w[j + 2] = x.z; w[j + 3] = x.w;
-            }
-#pragma unroll
-            for (int j = 0; j < 16; ++j) { st[j] = __float_as_uint(cw0 * w[j]); M2[16 * b + j] = (m2 && real2) ? m2[16 * b + j] : 0.0f; }
-            tmem_st16(lane_addr + T_W2 + c0 + 16 * b, st);
-            st_slab16(s.W2[(c0 + 16 * b) >> 6], row, (c0 + 16 * b) & 63, w);
-            if (ck && real2) {
-                const size_t o2 = (size_t)row * he + HC * me + c0 + 16 * b;
-#pragma unroll
-                for (int j = 0; j < 16; j += 4) {
-                    *reinterpret_cast<float4*>(ck + dh + o2 + j) = make_float4(w[j], w[j + 1], w[j + 2], w[j + 3]);
-                    *reinterpret_cast<float4*>(ck + 3 * dh + o2 + j) =
-                        make_float4(M2[16 * b + j], M2[16 * b + j + 1], M2[16 * b + j + 2], M2[16 * b + j + 3]);
-                }
-            }
-        }
-        tmem_wait_st();
-    }
-    // token tile of the chunk that starts at global row y: keys into rows 0..63, queries into rows 64..127
-    auto load_tokens = [&](int y) {
-        mbar_expect_tx(&s.bar_x, de == 128 ? 32768u : 16384u);
-        tma_load_2d(s.X[0], &tmK, 0, y, &s.bar_x);
-        tma_load_2d(s.X[0] + 8192, &tmQ, 0, y, &s.bar_x);
-        if (de == 128) {
-            tma_load_2d(s.X[1], &tmK, 64, y, &s.bar_x);
-            tma_load_2d(s.X[1] + 8192, &tmQ, 64, y, &s.bar_x);
-        }
-    };
     if (de < 128)  // the padded half of the token tile is never loaded: zero it once
         for (int i = tid; i < 16384 / 16; i += NTHREADS) reinterpret_cast<uint4*>(s.X[1])[i] = make_uint4(0u, 0u, 0u, 0u);
-    if (is_issuer) load_tokens(seq * L);
     fence_proxy_async_smem();
     tc_fence_before_sync();
     __syncthreads();
     // every CTA's barriers are initialised before any peer may arrive on them
     cluster_sync();
     tc_fence_after_sync();
+    const uint32_t tb = s.tmem_base;
 
-    const uint32_t id_kk = make_idesc(128, 128, false, false);
-    const uint32_t id_kmn = make_idesc(128, 128, false, true);
-    const uint32_t id_agg = make_idesc(128, 128, true, true) | (1u << 13);  // negate A: G_t is minus the gradient
-
-    // G1 of chunk `chunk` (issuer thread only): needs that chunk's tokens in X and the refreshed bf16 W1
-    auto issue_g1 = [&](int chunk) {
-        mbar_wait_one(&s.bar_x, (uint32_t)(chunk & 1), wc, 100 + 1);
-        tc_fence_after_sync();
+    if (warp >= NEW) {
+        // =====================================================================================================
+        // control warpgroup
+        // =====================================================================================================
+#ifndef TC_NO_SETMAXNREG
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(CTRL_REGS));
+#endif
+        if (warp == NEW + 2) {
+            // the whole warp runs the loop converged (every lane polls the barriers); lane 0 issues
+            // ------------------------------------------------------------------------------------- MMA issuer
+            // the descriptor's address field has 14 bits; a shared::cta address of a CTA of a cluster carries more above them
+            const uint32_t sb = (smem_u32(smem_raw) >> 4) & 0x3FFFu;
+            constexpr uint32_t oW1 = offsetof(Smem, W1) >> 4, oW2 = offsetof(Smem, W2) >> 4, oX = offsetof(Smem, X) >> 4,
+                               oA = offsetof(Smem, A) >> 4, oAkW = offsetof(Smem, AkW) >> 4, oAkM = offsetof(Smem, AkM) >> 4,
+                               oPu = offsetof(Smem, Pu) >> 4, oPzW = offsetof(Smem, PzW) >> 4, oPzM = offsetof(Smem, PzM) >> 4;
+            const uint32_t id_kk = make_idesc(128, 128, false, false);
+            const uint32_t id_kmn = make_idesc(128, 128, false, true);
+            const uint32_t id_agg = make_idesc(128, 128, true, true) | (1u << 13);  // negate A: G_t is minus the gradient
+            const bool el = lane == 0;  // the lane whose MMA / commit instructions are not predicated off
+            for (int r = 0; r < nchunks; ++r) {
+                const uint32_t ph = (uint32_t)(r & 1);
+                // G1: Z = X W1c^T -> R0.  Needs the chunk's tokens, the refreshed bf16 W1 and R0 read out (M1 aggregate).
+                mbar_wait(&s.bar_x, ph, wc, 100 + 1);
+                mbar_wait(&s.bar_w1, ph, wc, 100 + 2);
+                tc_fence_after_sync();
+                PROF(0);
 #pragma unroll
-        for (int k = 0; k < 8; ++k)
-            umma_bf16(tb + T_R0, desc_k(smem_u32(s.X[0]), 16384, k), desc_k(smem_u32(s.W1[0]), 16384, k), id_kk, k > 0);
-        umma_commit(&s.bar_g1);
-    };
-    if (is_issuer) issue_g1(0);
-    __syncwarp();
-
-    for (int r = 0; r < nchunks; ++r) {
-        const uint32_t ph = (uint32_t)(r & 1);
-        const Scalars& sc = s.sc[r & 1];
-        const int tok0 = r * C;
-
-        // scalars of the next chunk (suffix scans over its gates), by a warp that is not the issuer
-        if (warp == 3 + 4 * (NG - 1) && r + 1 < nchunks) {
-            tc_chunk_scalars(eta + tok0 + C, beta + tok0 + C, gamma + tok0 + C, &s.sc[(r + 1) & 1]);
-        }
-        PROF(0);
-        // ---------------- G1: Z = X W1c^T -> R0 (issued at the end of the previous iteration / before the loop)
-        if (is_issuer) {
-            if (r + 1 < nchunks) {
-                // the next chunk's tokens: into L2 now, so that the loads issued at the end of this chunk are short
-                const int y = seq * L + tok0 + C;
-                tma_prefetch_l2_2d(&tmK, 0, y);
-                tma_prefetch_l2_2d(&tmQ, 0, y);
-                tma_prefetch_l2_2d(&tmV, 0, y + 16 * (int)me);
-                if (de == 128) {
-                    tma_prefetch_l2_2d(&tmK, 64, y);
-                    tma_prefetch_l2_2d(&tmQ, 64, y);
-                    tma_prefetch_l2_2d(&tmV, 64, y + 16 * (int)me);
+                for (int k = 0; k < 8; ++k) umma_bf16_elect(tb + T_R0, dk(sb + oX, 16384, k), dk(sb + oW1, 16384, k), id_kk, k > 0, el);
+                umma_commit_elect(&s.bar_g1, el);
+                PROF(1);
+                // G2: Upart = A W2c^T -> R1.  Needs gelu(Z) in A, the refreshed bf16 W2 and R1 read out (M2 aggregate).
+                mbar_wait(&s.bar_a, ph, wc, 100 + 3);
+                mbar_wait(&s.bar_w2, ph, wc, 100 + 4);
+                tc_fence_after_sync();
+                PROF(2);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) umma_bf16_elect(tb + T_R1, dk(sb + oA, 16384, k), dk(sb + oW2, 16384, k), id_kk, k > 0, el);
+                umma_commit_elect(&s.bar_g2, el);
+                PROF(3);
+                // G3: Pa = Pu W2c -> R1.  Needs every CTA's pu rows (bulk copies: async proxy, no proxy fence needed here) and
+                // the partial sums read out of R1 by all warps.
+                mbar_wait<true>(&s.bar_pu, ph, wc, 100 + 5);
+                PROF(13);
+                mbar_wait(&s.bar_r1, ph, wc, 100 + 6);
+                tc_fence_after_sync();
+                PROF(4);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) umma_bf16_elect(tb + T_R1, dk(sb + oPu, 8192, k), dmn(sb + oW2, 16384, k), id_kmn, k > 0, el);
+                umma_commit_elect(&s.bar_g3, el);
+                PROF(5);
+                // W2 aggregation on top of the master
+                mbar_wait(&s.bar_ak, ph, wc, 100 + 7);
+                tc_fence_after_sync();
+#pragma unroll
+                for (int k = 0; k < 4; ++k) umma_bf16_elect(tb + T_W2, dmn(sb + oPu, 8192, k), dmn(sb + oAkW, 8192, k), id_agg, true, el);
+                PROF(14);
+                // W1 aggregation first (the next chunk's G1 hangs on it), then the two momentum aggregates
+                mbar_wait(&s.bar_pz, ph, wc, 100 + 8);
+                tc_fence_after_sync();
+                PROF(6);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) umma_bf16_elect(tb + T_W1, dmn(sb + oPzW, 8192, k), dmn(sb + oX, 16384, k), id_agg, true, el);
+                umma_commit_elect(&s.bar_aw1, el);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) umma_bf16_elect(tb + T_R0, dmn(sb + oPzM, 8192, k), dmn(sb + oX, 16384, k), id_agg, k > 0, el);
+                umma_commit_elect(&s.bar_am1, el);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) umma_bf16_elect(tb + T_R1, dmn(sb + oPu, 8192, k), dmn(sb + oAkM, 8192, k), id_agg, k > 0, el);
+                umma_commit_elect(&s.bar_am2, el);
+                PROF(7);
+            }
+        } else if (warp == NEW + 3) {
+            // ------------------------------------------------------------------- token loads and gate scans
+            for (int r = 0; r < nchunks; ++r) {
+                const uint32_t ph = (uint32_t)(r & 1);
+                const int tok0 = r * C;
+                if (r == 0) {
+                    if (lane == 0) {
+                        mbar_expect_tx(&s.bar_x, de == 128 ? 32768u : 16384u);
+                        const int y = seq * L;
+                        tma_load_2d(s.X[0], &tmK, 0, y, &s.bar_x);
+                        tma_load_2d(s.X[0] + 8192, &tmQ, 0, y, &s.bar_x);
+                        if (de == 128) {
+                            tma_load_2d(s.X[1], &tmK, 64, y, &s.bar_x);
+                            tma_load_2d(s.X[1] + 8192, &tmQ, 64, y, &s.bar_x);
+                        }
+                    }
+                } else {
+                    // the previous chunk is over in this CTA: its scalars, barriers' phases and staging are history
+                    mbar_wait(&s.bar_w2, ph, wc, 100 + 20);
+                }
+                if (lane == 0) {
+                    mbar_expect_tx(&s.bar_partK, 3 * 8192);  // this chunk's incoming partial sums and pu rows
+                    mbar_expect_tx(&s.bar_partQ, 3 * 4096);
+                    mbar_expect_tx(&s.bar_pu, 12288);
+                    if (NORM) mbar_expect_tx(&s.bar_rs, 3 * 512);
+                    if (r + 1 < nchunks) {
+                        // the next chunk's tokens: into L2 now, so that the loads issued at the end of this chunk are short
+                        const int y = seq * L + tok0 + C;
+                        tma_prefetch_l2_2d(&tmK, 0, y);
+                        tma_prefetch_l2_2d(&tmQ, 0, y);
+                        tma_prefetch_l2_2d(&tmV, 0, y + 16 * (int)me);
+                        if (de == 128) {
+                            tma_prefetch_l2_2d(&tmK, 64, y);
+                            tma_prefetch_l2_2d(&tmQ, 64, y);
+                            tma_prefetch_l2_2d(&tmV, 64, y + 16 * (int)me);
+                        }
+                    }
+                }
+                __syncwarp();
+                if (r + 1 < nchunks) {
+                    // scalars of the next chunk (suffix scans over its gates)
+                    tc_chunk_scalars(eta + tok0 + C, beta + tok0 + C, gamma + tok0 + C, &s.sc[(r + 1) & 1]);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&s.bar_sc);
+                }
+                // the 16 value rows this CTA needs for its key rows: into the gelu tile's first slab, dead once G2 is done
+                mbar_wait(&s.bar_g2, ph, wc, 100 + 21);
+                if (lane == 0) {
+                    mbar_expect_tx(&s.bar_v, de == 128 ? 4096u : 2048u);
+                    const int y = seq * L + tok0 + 16 * (int)me;
+                    tma_load_2d(s.A[0], &tmV, 0, y, &s.bar_v);
+                    if (de == 128) tma_load_2d(s.A[0] + 2048, &tmV, 64, y, &s.bar_v);
+                }
+                if (r + 1 < nchunks) {
+                    // the W1 / M1 aggregations were the last readers of the key tile: the next chunk's tokens may land in X
+                    mbar_wait(&s.bar_am1, ph, wc, 100 + 22);
+                    if (lane == 0) {
+                        mbar_expect_tx(&s.bar_x, de == 128 ? 32768u : 16384u);
+                        const int y2 = seq * L + tok0 + C;
+                        tma_load_2d(s.X[0], &tmK, 0, y2, &s.bar_x);
+                        tma_load_2d(s.X[0] + 8192, &tmQ, 0, y2, &s.bar_x);
+                        if (de == 128) {
+                            tma_load_2d(s.X[1], &tmK, 64, y2, &s.bar_x);
+                            tma_load_2d(s.X[1] + 8192, &tmQ, 64, y2, &s.bar_x);
+                        }
+                    }
+                }
+                if (NORM || r + 1 < nchunks) {
+                    // Every reader of this chunk's staging / pu / scaled-activation buffers is done once the aggregations
+                    // have completed and every epilogue warp has left its layer norm (it has then released W1): tell the
+                    // peers they may overwrite them.  (With normalisation the last chunk's row sums still need it.)
+                    mbar_wait(&s.bar_am2, ph, wc, 100 + 23);
+                    mbar_wait(&s.bar_w1, ph ^ 1u, wc, 100 + 24);
+                    if (lane < NC && lane != (int)me) mbar_arrive_remote(map_to_cta(smem_u32(&s.bar_credit), (uint32_t)lane));
+                    __syncwarp();
+                }
+                if (r + 1 < nchunks) {
+                    // ... and pass the peers' credits on to the epilogue warps (a local barrier is cheaper to wait on)
+                    mbar_wait<true>(&s.bar_credit, ph, wc, 100 + 25);
+                    if (lane == 0) mbar_arrive(&s.bar_go);
+                    __syncwarp();
                 }
             }
-            mbar_expect_tx(&s.bar_partK, 3 * 8192);  // this chunk's incoming partial sums and pu rows
-            mbar_expect_tx(&s.bar_partQ, 3 * 8192);
-            mbar_expect_tx(&s.bar_pu, 16384);
-            if (NORM) mbar_expect_tx(&s.bar_rs, 3 * 512);
         }
-        mbar_wait(&s.bar_g1, ph, wc, 100 + 2);
-        PROF(1);
-        __syncwarp();
-        tc_fence_after_sync();
-        // epilogue: a = gelu(z) -> A (bf16); for key rows also kW a, kM a and gelu'(z) (kept in TMEM over z)
-        // a = gelu(z) -> A (bf16) for all 128 rows: all that G2 needs
-#pragma unroll
-        for (int b = 0; b < NB; ++b) {
-            uint32_t z[16];
-            tmem_ld16(lane_addr + T_R0 + c0 + 16 * b, z);
-            tmem_wait_ld();
-            float av[16];
-#pragma unroll
-            for (int j = 0; j < 16; ++j) av[j] = gelu_only(__uint_as_float(z[j]));
-            const int col = c0 + 16 * b;
-            st_slab16(s.A[col >> 6], row, col & 63, av);
-        }
-        fence_proxy_async_smem();
-        tc_fence_before_sync();
-        __syncthreads();
-        PROF(2);
-        // ---------------- G2: Upart = A W2c^T -> R1
-        if (is_issuer) {
-            tc_fence_after_sync();
-#pragma unroll
-            for (int k = 0; k < 8; ++k)
-                umma_bf16(tb + T_R1, desc_k(smem_u32(s.A[0]), 16384, k), desc_k(smem_u32(s.W2[0]), 16384, k), id_kk, k > 0);
-            umma_commit(&s.bar_g2);
-        }
-        __syncwarp();
-        mbar_wait(&s.bar_g2, ph, wc, 100 + 3);
-        if (is_issuer) {
-            // the 16 value rows this CTA needs for its key rows: into the gelu tile's first slab, dead once G2 is done
-            mbar_expect_tx(&s.bar_v, de == 128 ? 4096u : 2048u);
-            const int y = seq * L + tok0 + 16 * (int)me;
-            tma_load_2d(s.A[0], &tmV, 0, y, &s.bar_v);
-            if (de == 128) tma_load_2d(s.A[0] + 2048, &tmV, 64, y, &s.bar_v);
-        }
-        __syncwarp();
-        PROF(3);
-        __syncwarp();
-        tc_fence_after_sync();
-        // Row ownership: CTA c normalises key tokens 16c..16c+15 and query tokens 16c..16c+15, so every CTA carries
-        // the same mix of work.  TMEM lane 32q+l holds key token 32q+l (q < 2) or query token 32(q-2)+l.
-        auto send_rows = [&](uint64_t* bar_local) {
-            const uint32_t owner = 2u * ((uint32_t)q & 1u) + ((uint32_t)lane >> 4);
-            const uint32_t srow = ((q < 2) ? 0u : 16u) + ((uint32_t)lane & 15u);  // row inside the owner's staging slot
-            const bool mine = owner == me;
-            uint32_t dst_base, dst_bar = 0;
-            if (mine) {
-                dst_base = smem_u32(s.A[1]);  // own rows: the gelu tile is dead once G2 has completed
-            } else {
-                const uint32_t slot = (me - owner - 1u) & 3u;  // where the owner keeps what comes from me
-                const uint8_t* p = (slot == 0) ? s.PzW[0] : (slot == 1) ? s.PzM[0] : s.Stage2;
-                dst_base = map_to_cta(smem_u32(p), owner);
-                dst_bar = map_to_cta(smem_u32(bar_local), owner);
-            }
+    } else {
+        // =====================================================================================================
+        // epilogue warps
+        // =====================================================================================================
+#ifndef TC_NO_SETMAXNREG
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(EPI_REGS));
+#endif
+        const int q = warp & 3;          // TMEM lane quadrant
+        const int g = warp >> 2;         // column group
+        const int row = 32 * q + lane;   // TMEM lane this thread reads
+        const int c0 = CW * g;           // first of its columns inside a 128-column region
+        const uint32_t lane_addr = tb + ((uint32_t)(32 * q) << 16);
+        const size_t dh = (size_t)de * he;
+        const bool cta_real = HC * (int)me < he;  // this CTA's 128 hidden units exist
+        const float inv_d = 1.0f / (float)de;
+        // normalisation targets of this thread's rows: hidden unit 128 me + row of W1, output row `row` of W2
+        const float tgt1 = (NORM && cta_real) ? a.norm1[(size_t)seq * he + HC * me + row] : 0.0f;
+        const float tgt2 = (NORM && row < de) ? a.norm2[(size_t)seq * de + row] : 0.0f;
+        __nv_bfloat16* go = a.o + (size_t)seq * L * de;
+
+        // ---- load the state: fp32 master of W -> TMEM (pre-scaled by the first decay carry) and bf16 -> shared; M -> registers
+        float M1[CW], M2[CW];
+        {
+            const float cw0 = s.sc[0].cw;
+            const size_t head = (size_t)seq * dh;
+            // W1c[j][i]: global W1 [h][d], row 128 me + j
+            const float* w1 = a.W1_init + head + ((size_t)(HC * me) + row) * de + c0;
+            const float* m1 = a.M1_init ? a.M1_init + head + ((size_t)(HC * me) + row) * de + c0 : nullptr;
+            // W2c[i][j]: global W2 [d][h], row i, column 128 me + j
+            const float* w2 = a.W2_init + head + (size_t)row * he + HC * me + c0;
+            const float* m2 = a.M2_init ? a.M2_init + head + (size_t)row * he + HC * me + c0 : nullptr;
+            const bool real2 = cta_real && row < de;  // this thread's W2 row exists
 #pragma unroll
             for (int b = 0; b < NB; ++b) {
-                uint32_t u[16];
-                tmem_ld16(lane_addr + T_R1 + c0 + 16 * b, u);
-                tmem_wait_ld();
+                float w[16];
+                uint32_t st[16];
+                const bool real1 = cta_real && c0 + 16 * b < de;  // these 16 columns of W1 exist
 #pragma unroll
                 for (int j = 0; j < 16; j += 4) {
-                    const uint32_t c4 = (uint32_t)((c0 + 16 * b + j) >> 2);
-                    const uint32_t dst = dst_base + stage_offset(c4, srow);
-                    if (mine) st_cluster_v4_b32(dst, u[j], u[j + 1], u[j + 2], u[j + 3]);
-                    else st_async_v4(dst, u[j], u[j + 1], u[j + 2], u[j + 3], dst_bar);
+                    const float4 x = real1 ? *reinterpret_cast<const float4*>(w1 + 16 * b + j) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    w[j] = x.x; w[j + 1] = x.y; w[j + 2] = x.z; w[j + 3] = x.w;
                 }
-            }
-        };
-
-        // What only the inner backward needs, for the key rows (the warps of TMEM quadrants 0 and 1): kW a, kM a
-        // (operands of the W2 aggregations) and gelu'(z), which replaces z in TMEM.  Runs while pu travels.
-        auto backward_extras = [&]() {
-            const float kw = sc.kW[row], km = sc.kM[row];
 #pragma unroll
-            for (int b = 0; b < NB; ++b) {
-                uint32_t z[16];
-                tmem_ld16(lane_addr + T_R0 + c0 + 16 * b, z);
-                tmem_wait_ld();
-                float aw[16], am[16];
-                uint32_t dg[16];
+                for (int j = 0; j < 16; ++j) { st[j] = __float_as_uint(cw0 * w[j]); M1[16 * b + j] = (m1 && real1) ? m1[16 * b + j] : 0.0f; }
+                tmem_st16(lane_addr + T_W1 + c0 + 16 * b, st);
+                st_slab16(s.W1[(c0 + 16 * b) >> 6], row, (c0 + 16 * b) & 63, w);
+                float* ck = a.ckpt ? a.ckpt + (size_t)seq * a.ckpt_seq_stride : nullptr;  // chunk-start state of chunk 0
+                if (ck && real1) {
+                    const size_t o1 = ((size_t)(HC * me) + row) * de + c0 + 16 * b;
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    float d1;
-                    const float av = gelu_fast(__uint_as_float(z[j]), d1);
-                    dg[j] = __float_as_uint(d1);
-                    aw[j] = kw * av;
-                    am[j] = km * av;
+                    for (int j = 0; j < 16; j += 4) {
+                        *reinterpret_cast<float4*>(ck + o1 + j) = make_float4(w[j], w[j + 1], w[j + 2], w[j + 3]);
+                        *reinterpret_cast<float4*>(ck + 2 * dh + o1 + j) =
+                            make_float4(M1[16 * b + j], M1[16 * b + j + 1], M1[16 * b + j + 2], M1[16 * b + j + 3]);
+                    }
                 }
-                const int col = c0 + 16 * b;
-                st_slab16(s.AkW[col >> 6], row, col & 63, aw);
-                st_slab16(s.AkM[col >> 6], row, col & 63, am);
-                tmem_st16(lane_addr + T_R0 + col, dg);
+#pragma unroll
+                for (int j = 0; j < 16; j += 4) {
+                    const float4 x = real2 ? *reinterpret_cast<const float4*>(w2 + 16 * b + j) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    w[j] = x.x; w[j + 1] = x.y; w[j + 2] = x.z; w[j + 3] = x.w;
+                }
+#pragma unroll
+                for (int j = 0; j < 16; ++j) { st[j] = __float_as_uint(cw0 * w[j]); M2[16 * b + j] = (m2 && real2) ? m2[16 * b + j] : 0.0f; }
+                tmem_st16(lane_addr + T_W2 + c0 + 16 * b, st);
+                st_slab16(s.W2[(c0 + 16 * b) >> 6], row, (c0 + 16 * b) & 63, w);
+                if (ck && real2) {
+                    const size_t o2 = (size_t)row * he + HC * me + c0 + 16 * b;
+#pragma unroll
+                    for (int j = 0; j < 16; j += 4) {
+                        *reinterpret_cast<float4*>(ck + dh + o2 + j) = make_float4(w[j], w[j + 1], w[j + 2], w[j + 3]);
+                        *reinterpret_cast<float4*>(ck + 3 * dh + o2 + j) =
+                            make_float4(M2[16 * b + j], M2[16 * b + j + 1], M2[16 * b + j + 2], M2[16 * b + j + 3]);
+                    }
+                }
             }
             tmem_wait_st();
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&s.bar_ak);
-        };
+            warp_release(&s.bar_w1);
+            if (lane == 0) mbar_arrive(&s.bar_w2);
+        }
 
-        // Layer norm on the 16 key rows (warps of quadrants 0/1) or the 16 query rows (quadrants 2/3) this CTA owns:
-        // 16 threads per row, 8 columns each.
-        auto layer_norm = [&](const bool key_rows) {
-            constexpr int TPR = NTHREADS / 32, CPT = 128 / TPR;  // threads per row, columns per thread
-            static_assert(TPR == 16, "row mapping below assumes two rows per warp");
-            // staging rows 0..15: key tokens, 16..31: query tokens
-            const int lrow = (key_rows ? 0 : 16) + 2 * ((q & 1) + 2 * g) + (lane >> 4);
-            const int cg = lane & 15;
-            const int t = 16 * (int)me + (lrow & 15);    // token inside the chunk
-            const int xrow = key_rows ? t : 64 + t;      // its row in the X tile
-            const int col0 = CPT * cg;
-            const size_t off = (size_t)(tok0 + t) * de + col0;
-            const bool real = col0 < de;  // this thread's 8 columns exist (padding columns carry exact zeros)
-            uint4 vraw[CPT / 8], xraw[CPT / 8];
+        for (int r = 0; r < nchunks; ++r) {
+            const uint32_t ph = (uint32_t)(r & 1);
+            const Scalars& sc = s.sc[r & 1];
+            const int tok0 = r * C;
+            const bool last = (r + 1 == nchunks);
+            PROF(0);
+            // ---------------- G1 epilogue: a = gelu(z) -> A (bf16), all that G2 needs.  The key rows' a also goes, unscaled,
+            // (as fp16) into the kW a tile: the query-row warps turn it into bf16 kW a and kM a while G2 runs.
+            mbar_wait(&s.bar_g1, ph, wc, 100 + 30);
+            tc_fence_after_sync();
+            PROF(1);
+            {
+                {
+                    uint32_t z[NB][16];
 #pragma unroll
-            for (int ch = 0; ch < CPT / 8; ++ch) {
-                const int c = ((col0 & 63) >> 3) + ch;
-                xraw[ch] = *reinterpret_cast<const uint4*>(s.X[col0 >> 6] + xrow * 128 + ((c ^ (xrow & 7)) << 4));
-            }
-            mbar_wait<true>(key_rows ? &s.bar_partK : &s.bar_partQ, ph, wc, 100 + 5);
-            if (key_rows) {
-                mbar_wait(&s.bar_v, ph, wc, 100 + 11);
-                const int lr = lrow & 15;
+                    for (int b = 0; b < NB; ++b) tmem_ld16(lane_addr + T_R0 + c0 + 16 * b, z[b]);
+                    tmem_wait_ld();
 #pragma unroll
-                for (int ch = 0; ch < CPT / 8; ++ch) {
-                    const int c = ((col0 & 63) >> 3) + ch;
-                    vraw[ch] = real ? *reinterpret_cast<const uint4*>(s.A[0] + (col0 >> 6) * 2048 + lr * 128 + ((c ^ (lr & 7)) << 4))
-                                    : make_uint4(0u, 0u, 0u, 0u);
+                    for (int b = 0; b < NB; ++b) {
+                        uint32_t p[8], ph16[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const float a0 = gelu_only(__uint_as_float(z[b][2 * i])), a1 = gelu_only(__uint_as_float(z[b][2 * i + 1]));
+                            p[i] = pack_bf16(a0, a1);
+                            ph16[i] = pack_f16(a0, a1);  // fp16 keeps 3 more bits: no visible second rounding in kW a, kM a
+                        }
+                        const int col = c0 + 16 * b;
+                        st_slab16p(s.A[col >> 6], row, col & 63, p);
+                        if (q < 2) st_slab16p(s.AkW[col >> 6], row, col & 63, ph16);
+                    }
+                }
+                warp_release(&s.bar_a);
+                PROF(2);
+                if (q < 2) {
+                    // key rows: gelu'(z) replaces z in TMEM (the G3 epilogue multiplies by it), in the shadow of G2
+#pragma unroll
+                    for (int b = 0; b < NB; ++b) {
+                        uint32_t z[16];
+                        tmem_ld16(lane_addr + T_R0 + c0 + 16 * b, z);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) z[j] = __float_as_uint(gelu_d1_fast(__uint_as_float(z[j])));
+                        tmem_st16(lane_addr + T_R0 + c0 + 16 * b, z);
+                    }
+                    tmem_wait_st();
+                } else {
+                    // query-row warps: scale the key rows' a by kW and kM (operands of the W2 aggregations).  256 threads over
+                    // the [64 x 128] tile: 4 threads per row, 32 columns each; kW a overwrites a in place.
+                    mbar_wait(&s.bar_a, ph, wc, 100 + 38);
+                    const int tq = 32 * (2 * g + (q & 1)) + lane;
+                    const int ar = tq >> 2, ac = 32 * (tq & 3);
+                    const float kw = sc.kW[ar], km = sc.kM[ar];
+                    uint8_t* rw = s.AkW[ac >> 6] + ar * 128;
+                    uint8_t* rm = s.AkM[ac >> 6] + ar * 128;
+                    uint4 v[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) v[i] = *reinterpret_cast<const uint4*>(rw + (((((ac & 63) >> 3) + i) ^ (ar & 7)) << 4));
+                    auto scale2 = [](uint32_t x, float k) {  // two packed fp16 times k -> two packed bf16
+                        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&x));
+                        return pack_bf16(k * f.x, k * f.y);
+                    };
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int off = ((((ac & 63) >> 3) + i) ^ (ar & 7)) << 4;
+                        *reinterpret_cast<uint4*>(rw + off) = make_uint4(scale2(v[i].x, kw), scale2(v[i].y, kw), scale2(v[i].z, kw), scale2(v[i].w, kw));
+                        *reinterpret_cast<uint4*>(rm + off) = make_uint4(scale2(v[i].x, km), scale2(v[i].y, km), scale2(v[i].z, km), scale2(v[i].w, km));
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&s.bar_ak);
                 }
             }
-            float u[CPT];
-#pragma unroll
-            for (int j = 0; j < CPT; ++j) u[j] = 0.0f;
-#pragma unroll
-            for (int src = 0; src < NC; ++src) {  // fixed order: the sum does not depend on arrival order
-                const uint32_t slot = ((uint32_t)src - me - 1u) & 3u;
-                const uint8_t* p = (src == (int)me) ? s.A[1] : (slot == 0) ? s.PzW[0] : (slot == 1) ? s.PzM[0] : s.Stage2;
-#pragma unroll
-                for (int j = 0; j < CPT; j += 4) {
-                    const int c4 = (col0 + j) >> 2;
-                    const float4 x = *reinterpret_cast<const float4*>(p + stage_offset((uint32_t)c4, (uint32_t)lrow));
-                    u[j] += x.x; u[j + 1] += x.y; u[j + 2] += x.z; u[j + 3] += x.w;
+            PROF(3);
+
+            // Row ownership: CTA c normalises key tokens 16c..16c+15 and query tokens 16c..16c+15, so every CTA carries
+            // the same mix of work.  TMEM lane 32q+l holds key token 32q+l (q < 2) or query token 32(q-2)+l.
+            // Partial sums of the key rows travel as fp32 (they feed the state), those of the query rows as bf16 (they
+            // only feed o, which is rounded to bf16 anyway).  The sender's own rows stay fp32 in the dead gelu tile.
+            const uint32_t owner = 2u * ((uint32_t)q & 1u) + ((uint32_t)lane >> 4);
+            const uint32_t srow = (uint32_t)lane & 15u;                 // row inside the owner's slot
+            const uint32_t slot = (me - owner - 1u) & 3u;               // where the owner keeps what comes from this CTA
+            auto send_k = [&]() {
+                const bool mine = owner == me;
+                uint32_t dst_base, dst_bar = 0;
+                if (mine) {
+                    dst_base = smem_u32(s.A[1]);  // the gelu tile is dead once G2 has completed
+                } else {
+                    const uint8_t* p = (slot == 0) ? s.PzW[0] : (slot == 1) ? s.PzW[1] : s.PzM[0];
+                    dst_base = map_to_cta(smem_u32(p), owner);
+                    dst_bar = map_to_cta(smem_u32(&s.bar_partK), owner);
                 }
-            }
-            auto row_sum = [&](float v) -> float {  // over the TPR lanes that share a row
+                uint32_t u[NB][16];
 #pragma unroll
-                for (int o = TPR / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                return v;
+                for (int b = 0; b < NB; ++b) tmem_ld16(lane_addr + T_R1 + c0 + 16 * b, u[b]);
+                tmem_wait_ld();
+#pragma unroll
+                for (int b = 0; b < NB; ++b) {
+#pragma unroll
+                    for (int j = 0; j < 16; j += 4) {
+                        const uint32_t dst = dst_base + stage_offset((uint32_t)((c0 + 16 * b + j) >> 2), srow);
+                        if (mine) st_cluster_v4_b32(dst, u[b][j], u[b][j + 1], u[b][j + 2], u[b][j + 3]);
+                        else st_async_v4(dst, u[b][j], u[b][j + 1], u[b][j + 2], u[b][j + 3], dst_bar);
+                    }
+                }
+                // R1 may be overwritten by G3 once every warp has taken its rows
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) { mbar_arrive(&s.bar_r1); mbar_arrive(&s.bar_ksent); }
             };
-            float sum = 0.0f;
+            auto send_q = [&]() {
+                const bool mine = owner == me;
+                uint32_t u[NB][16];
 #pragma unroll
-            for (int j = 0; j < CPT; ++j) sum += u[j];
-            const float mu = row_sum(sum) * inv_d;
-            float sq = 0.0f;
+                for (int b = 0; b < NB; ++b) tmem_ld16(lane_addr + T_R1 + c0 + 16 * b, u[b]);
+                tmem_wait_ld();
+                if (mine) {
+                    const uint32_t dst_base = smem_u32(s.A[1]) + 8192u;
 #pragma unroll
-            for (int j = 0; j < CPT; ++j) { u[j] = real ? u[j] - mu : 0.0f; sq = fmaf(u[j], u[j], sq); }
-            const float rstd = rsqrtf(row_sum(sq) * inv_d + a.eps);
+                    for (int b = 0; b < NB; ++b)
 #pragma unroll
-            for (int j = 0; j < CPT; ++j) u[j] *= rstd;  // y (zero in the padding)
-            if (key_rows) {
-                // key rows: e = k + y - v, pu = rstd (e - mean(e) - y mean(e y))
-                float e[CPT];
-                float se = 0.0f, sey = 0.0f;
+                        for (int j = 0; j < 16; j += 4)
+                            st_cluster_v4_b32(dst_base + stage_offset((uint32_t)((c0 + 16 * b + j) >> 2), srow), u[b][j], u[b][j + 1],
+                                              u[b][j + 2], u[b][j + 3]);
+                } else {
+                    const uint32_t dst_base = map_to_cta(smem_u32(s.Stage2) + slot * 4096u, owner);
+                    const uint32_t dst_bar = map_to_cta(smem_u32(&s.bar_partQ), owner);
 #pragma unroll
-                for (int ch = 0; ch < CPT / 8; ++ch) {
-                    const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&xraw[ch]);
-                    const __nv_bfloat162* v2 = reinterpret_cast<const __nv_bfloat162*>(&vraw[ch]);
+                    for (int b = 0; b < NB; ++b)
+#pragma unroll
+                        for (int j = 0; j < 16; j += 8) {
+                            const uint32_t c8 = (uint32_t)((c0 + 16 * b + j) >> 3);
+                            st_async_v4(dst_base + stage_offset_q(c8, srow),
+                                        pack_bf16(__uint_as_float(u[b][j]), __uint_as_float(u[b][j + 1])),
+                                        pack_bf16(__uint_as_float(u[b][j + 2]), __uint_as_float(u[b][j + 3])),
+                                        pack_bf16(__uint_as_float(u[b][j + 4]), __uint_as_float(u[b][j + 5])),
+                                        pack_bf16(__uint_as_float(u[b][j + 6]), __uint_as_float(u[b][j + 7])), dst_bar);
+                        }
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&s.bar_r1);
+            };
+
+            // Layer norm on the 16 key rows (warps of quadrants 0/1) or the 16 query rows (quadrants 2/3) this CTA owns:
+            // 16 threads per row, 8 columns each.
+            auto layer_norm = [&](const bool key_rows) {
+                constexpr int TPR = NEPI / 32, CPT = 128 / TPR;  // threads per row, columns per thread
+                static_assert(TPR == 16 && CPT == 8, "row mapping below assumes two rows per warp, one 16-byte piece per thread");
+                const int lrow = 2 * ((q & 1) + 2 * g) + (lane >> 4);   // row of the slot (0..15)
+                const int cg = lane & 15;
+                const int t = 16 * (int)me + lrow;           // token inside the chunk
+                const int xrow = key_rows ? t : 64 + t;      // its row in the X tile
+                const int col0 = CPT * cg;
+                const size_t off = (size_t)(tok0 + t) * de + col0;
+                const bool real = col0 < de;  // this thread's 8 columns exist (padding columns carry exact zeros)
+                const int c = (col0 & 63) >> 3;
+                const uint4 xraw = *reinterpret_cast<const uint4*>(s.X[col0 >> 6] + xrow * 128 + ((c ^ (xrow & 7)) << 4));
+                float u[CPT];
+                {   // own rows, fp32
+                    const uint8_t* p = s.A[1] + (key_rows ? 0 : 8192);
+                    const float4 x0 = *reinterpret_cast<const float4*>(p + stage_offset((uint32_t)(2 * cg), (uint32_t)lrow));
+                    const float4 x1 = *reinterpret_cast<const float4*>(p + stage_offset((uint32_t)(2 * cg + 1), (uint32_t)lrow));
+                    u[0] = x0.x; u[1] = x0.y; u[2] = x0.z; u[3] = x0.w; u[4] = x1.x; u[5] = x1.y; u[6] = x1.z; u[7] = x1.w;
+                }
+                mbar_wait<true>(key_rows ? &s.bar_partK : &s.bar_partQ, ph, wc, 100 + 35);
+                PROF(15);
+                // the peers' pieces, added in a fixed order (slot 0, 1, 2 = the CTAs me+1, me+2, me+3): the sum does not
+                // depend on arrival order, and each CTA adds its four pieces in its own fixed order
+                if (key_rows) {
+#pragma unroll
+                    for (int sl = 0; sl < 3; ++sl) {
+                        const uint8_t* p = (sl == 0) ? s.PzW[0] : (sl == 1) ? s.PzW[1] : s.PzM[0];
+                        const float4 x0 = *reinterpret_cast<const float4*>(p + stage_offset((uint32_t)(2 * cg), (uint32_t)lrow));
+                        const float4 x1 = *reinterpret_cast<const float4*>(p + stage_offset((uint32_t)(2 * cg + 1), (uint32_t)lrow));
+                        u[0] += x0.x; u[1] += x0.y; u[2] += x0.z; u[3] += x0.w; u[4] += x1.x; u[5] += x1.y; u[6] += x1.z; u[7] += x1.w;
+                    }
+                } else {
+#pragma unroll
+                    for (int sl = 0; sl < 3; ++sl) {
+                        const uint4 x = *reinterpret_cast<const uint4*>(s.Stage2 + sl * 4096 + stage_offset_q((uint32_t)cg, (uint32_t)lrow));
+                        const __nv_bfloat162* x2 = reinterpret_cast<const __nv_bfloat162*>(&x);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const float2 f = __bfloat1622float2(x2[i]);
+                            u[2 * i] += f.x;
+                            u[2 * i + 1] += f.y;
+                        }
+                    }
+                }
+                auto row_sum = [&](float v) -> float {  // over the TPR lanes that share a row
+#pragma unroll
+                    for (int o = TPR / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                    return v;
+                };
+                float sum = 0.0f;
+#pragma unroll
+                for (int j = 0; j < CPT; ++j) sum += u[j];
+                const float mu = row_sum(sum) * inv_d;
+                float sq = 0.0f;
+#pragma unroll
+                for (int j = 0; j < CPT; ++j) { u[j] = real ? u[j] - mu : 0.0f; sq = fmaf(u[j], u[j], sq); }
+                const float rstd = rsqrtf(row_sum(sq) * inv_d + a.eps);
+#pragma unroll
+                for (int j = 0; j < CPT; ++j) u[j] *= rstd;  // y (zero in the padding)
+                if (key_rows) {
+                    // key rows: e = k + y - v, pu = rstd (e - mean(e) - y mean(e y))
+                    mbar_wait(&s.bar_v, ph, wc, 100 + 36);
+                    PROF(16);
+                    const uint4 vraw = real ? *reinterpret_cast<const uint4*>(s.A[0] + (col0 >> 6) * 2048 + lrow * 128 + ((c ^ (lrow & 7)) << 4))
+                                            : make_uint4(0u, 0u, 0u, 0u);
+                    float e[CPT];
+                    float se = 0.0f, sey = 0.0f;
+                    const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&xraw);
+                    const __nv_bfloat162* v2 = reinterpret_cast<const __nv_bfloat162*>(&vraw);
 #pragma unroll
                     for (int x = 0; x < 4; ++x) {
                         const float2 kf = __bfloat1622float2(k2[x]), vf = __bfloat1622float2(v2[x]);
-                        const int j = 8 * ch + 2 * x;
-                        e[j] = kf.x + u[j] - vf.x;
-                        e[j + 1] = kf.y + u[j + 1] - vf.y;
+                        e[2 * x] = kf.x + u[2 * x] - vf.x;
+                        e[2 * x + 1] = kf.y + u[2 * x + 1] - vf.y;
                     }
-                }
 #pragma unroll
-                for (int j = 0; j < CPT; ++j) { se += e[j]; sey = fmaf(e[j], u[j], sey); }
-                const float me_ = real ? row_sum(se) * inv_d : (row_sum(se), 0.0f);
-                const float mey = row_sum(sey) * inv_d;
-                    // broadcast the bf16 pu row piece to every CTA of the cluster
-                uint32_t pk[CPT / 2];
+                    for (int j = 0; j < CPT; ++j) { se += e[j]; sey = fmaf(e[j], u[j], sey); }
+                    const float me_ = real ? row_sum(se) * inv_d : (row_sum(se), 0.0f);
+                    const float mey = row_sum(sey) * inv_d;
+                    uint32_t pk[CPT / 2];
 #pragma unroll
-                for (int j = 0; j < CPT; j += 2)
-                    pk[j / 2] = pack_bf16(rstd * (e[j] - me_ - u[j] * mey), rstd * (e[j + 1] - me_ - u[j + 1] * mey));  // 0 in the padding
-                const uint32_t pu_local = smem_u32(s.Pu[col0 >> 6]);
-#pragma unroll
-                for (uint32_t dst = 0; dst < NC; ++dst) {
-                    const uint32_t base = map_to_cta(pu_local, dst) + (uint32_t)t * 128u;
-                    const uint32_t bar = map_to_cta(smem_u32(&s.bar_pu), dst);
-#pragma unroll
-                    for (int ch = 0; ch < CPT / 8; ++ch) {
-                        const uint32_t c = (uint32_t)(((col0 & 63) >> 3) + ch);
-                        st_async_v4(base + ((c ^ ((uint32_t)t & 7u)) << 4), pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2],
-                                    pk[4 * ch + 3], bar);
+                    for (int j = 0; j < CPT; j += 2)
+                        pk[j / 2] = pack_bf16(rstd * (e[j] - me_ - u[j] * mey), rstd * (e[j + 1] - me_ - u[j + 1] * mey));  // 0 in the padding
+                    // The bf16 pu rows go into this CTA's own pu tile; one bulk copy per peer and slab (2 KB: the 16 rows of a
+                    // slab are contiguous) then carries them to the peers' tiles.  Bulk copies write through the async proxy,
+                    // the one the MMAs read through, so the receivers need no proxy fence.
+                    *reinterpret_cast<uint4*>(s.Pu[col0 >> 6] + t * 128 + ((c ^ (t & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    fence_proxy_async_smem();
+                    named_sync(BAR_KOWN, NEPI / 2);
+                    if (warp == 0) {
+                        if (lane < 6) {
+                            const uint32_t dst = (me + 1u + (uint32_t)(lane >> 1)) & 3u;
+                            const uint32_t src = smem_u32(s.Pu[lane & 1]) + 2048u * me;
+                            bulk_copy_to_cta(map_to_cta(src, dst), src, 2048u, map_to_cta(smem_u32(&s.bar_pu), dst));
+                        }
+                        if (lane == 0) mbar_arrive(&s.bar_pu);  // the own rows are in place
                     }
-                }
-            } else {
-                // query rows: o = q + y
-#pragma unroll
-                for (int ch = 0; ch < CPT / 8; ++ch) {
-                    const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&xraw[ch]);
+                } else {
+                    // query rows: o = q + y
+                    const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&xraw);
                     uint4 ov;
                     uint32_t* o32 = reinterpret_cast<uint32_t*>(&ov);
 #pragma unroll
                     for (int x = 0; x < 4; ++x) {
                         const float2 qf = __bfloat1622float2(q2[x]);
-                        o32[x] = pack_bf16(qf.x + u[8 * ch + 2 * x], qf.y + u[8 * ch + 2 * x + 1]);
+                        o32[x] = pack_bf16(qf.x + u[2 * x], qf.y + u[2 * x + 1]);
                     }
-                    if (real) *reinterpret_cast<uint4*>(go + off + 8 * ch) = ov;
+                    if (real) *reinterpret_cast<uint4*>(go + off) = ov;
                 }
-            }
-        };
+            };
 
-        // ---------------- cross-CTA sum of Upart, layer norm, pu broadcast
-        // The key rows are on the critical path of the whole cluster, the query rows are not.  So the warps holding
-        // key rows (quadrants 0/1) hand them to the network first, normalise this CTA's key rows as soon as the
-        // peers' pieces are in, broadcast pu, and only then produce the backward-only operands; the warps holding
-        // query rows (quadrants 2/3) send after the key rows have gone out, normalise the query rows, write o.
-        if (r > 0) mbar_wait<true>(&s.bar_credit, (uint32_t)((r - 1) & 1), wc, 100 + 4);
-        if (q < 2) {
-            send_rows(&s.bar_partK);
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&s.bar_ksent);
-            asm volatile("bar.sync 4, %0;" ::"r"(64 * NG) : "memory");  // this CTA's own key rows are staged
+            // ---------------- cross-CTA sum of Upart, layer norm, pu broadcast
+            // The key rows are on the critical path of the whole cluster, the query rows are not.  So the warps holding
+            // key rows (quadrants 0/1) hand them to the network first, normalise this CTA's key rows as soon as the
+            // peers' pieces are in and broadcast pu; the warps holding query rows (quadrants 2/3) send after the key
+            // rows have gone out, normalise the query rows, write o.
+            mbar_wait(&s.bar_g2, ph, wc, 100 + 31);
+            tc_fence_after_sync();
             PROF(4);
-            layer_norm(true);
-            PROF(5);
-            backward_extras();
-            PROF(6);
-            // the Pz tiles (G3 epilogue, below) overlay staging slots: wait until the query-row readers are done too
-            asm volatile("bar.sync 3, %0;" ::"r"(128 * NG) : "memory");
-        } else {
-            mbar_wait(&s.bar_ksent, ph, wc, 100 + 12);
-            send_rows(&s.bar_partQ);
-            asm volatile("bar.sync 5, %0;" ::"r"(64 * NG) : "memory");  // own query rows staged; R1 fully read
-            PROF(4);
-            layer_norm(false);
-            PROF(5);
-            asm volatile("bar.arrive 3, %0;" ::"r"(128 * NG) : "memory");
-            PROF(6);
-        }
-        PROF(7);
-        // ---------------- G3: Pa = Pu W2c -> R1 ; then the W2 aggregation that needs nothing else
-        if (is_issuer) {
-            mbar_wait_one<true>(&s.bar_pu, ph, wc, 100 + 6);
-            asm volatile("fence.proxy.async;" ::: "memory");
-            tc_fence_after_sync();
+            // the peers' staging slots, pu tile and scaled-activation tiles are free again: every peer has finished the
+            // previous chunk (the loader warp collects the peers' credits)
+            if (r > 0) mbar_wait(&s.bar_go, (uint32_t)((r - 1) & 1), wc, 100 + 32);
+            PROF(13);
+            if (q < 2) {
+                send_k();
+                PROF(14);
+                named_sync(BAR_KOWN, NEPI / 2);  // this CTA's own key rows are staged
+                PROF(5);
+                layer_norm(true);
+                PROF(6);
+                PROF(17);
+                // ---------------- G3 epilogue: Pz = Pa * gelu'(Zk), scaled by kW and kM into two bf16 tiles
+                mbar_wait(&s.bar_g3, ph, wc, 100 + 33);
+                tc_fence_after_sync();
+                PROF(7);
+                {
+                    const float kw = sc.kW[row], km = sc.kM[row];
+                    uint32_t pa[NB][16], dg[NB][16];
 #pragma unroll
-            for (int k = 0; k < 8; ++k)
-                umma_bf16(tb + T_R1, desc_k(smem_u32(s.Pu[0]), 8192, k), desc_mn(smem_u32(s.W2[0]), 16384, k), id_kmn, k > 0);
-            umma_commit(&s.bar_g3);
-            mbar_wait_one(&s.bar_ak, ph, wc, 100 + 10);  // kW a / kM a written by the quadrant-0/1 warps
-            tc_fence_after_sync();
+                    for (int b = 0; b < NB; ++b) {
+                        tmem_ld16(lane_addr + T_R1 + c0 + 16 * b, pa[b]);
+                        tmem_ld16(lane_addr + T_R0 + c0 + 16 * b, dg[b]);
+                    }
+                    tmem_wait_ld();
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-                umma_bf16(tb + T_W2, desc_mn(smem_u32(s.Pu[0]), 8192, k), desc_mn(smem_u32(s.AkW[0]), 8192, k), id_agg, true);
-        }
-        mbar_wait(&s.bar_g3, ph, wc, 100 + 7);
-        PROF(8);
-        __syncwarp();
-        tc_fence_after_sync();
-        if (row < C) {
-            const float kw = sc.kW[row], km = sc.kM[row];
+                    for (int b = 0; b < NB; ++b) {
+                        float pw[16], pm[16];
 #pragma unroll
-            for (int b = 0; b < NB; ++b) {
-                uint32_t pa[16], dg[16];
-                tmem_ld16(lane_addr + T_R1 + c0 + 16 * b, pa);
-                tmem_ld16(lane_addr + T_R0 + c0 + 16 * b, dg);
-                tmem_wait_ld();
-                float pw[16], pm[16];
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const float pz = __uint_as_float(pa[j]) * __uint_as_float(dg[j]);
-                    pw[j] = kw * pz;
-                    pm[j] = km * pz;
+                        for (int j = 0; j < 16; ++j) {
+                            const float pz = __uint_as_float(pa[b][j]) * __uint_as_float(dg[b][j]);
+                            pw[j] = kw * pz;
+                            pm[j] = km * pz;
+                        }
+                        const int col = c0 + 16 * b;
+                        st_slab16(s.PzW[col >> 6], row, col & 63, pw);
+                        st_slab16(s.PzM[col >> 6], row, col & 63, pm);
+                    }
                 }
-                const int col = c0 + 16 * b;
-                st_slab16(s.PzW[col >> 6], row, col & 63, pw);
-                st_slab16(s.PzM[col >> 6], row, col & 63, pm);
+                warp_release(&s.bar_pz);
+                PROF(8);
+            } else {
+                mbar_wait(&s.bar_ksent, ph, wc, 100 + 34);
+                send_q();
+                PROF(14);
+                named_sync(BAR_QOWN, NEPI / 2);  // own query rows staged
+                PROF(5);
+                layer_norm(false);
+                PROF(6);
             }
-        }
-        fence_proxy_async_smem();
-        tc_fence_before_sync();
-        __syncthreads();
-        PROF(9);
-        // ---------------- remaining aggregations, in two groups so that the state pass can start on W1 early
-        if (is_issuer) {
-            tc_fence_after_sync();
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-                umma_bf16(tb + T_W1, desc_mn(smem_u32(s.PzW[0]), 8192, k), desc_mn(smem_u32(s.X[0]), 16384, k), id_agg, true);
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-                umma_bf16(tb + T_R0, desc_mn(smem_u32(s.PzM[0]), 8192, k), desc_mn(smem_u32(s.X[0]), 16384, k), id_agg, k > 0);
-            umma_commit(&s.bar_agg);
-            PROF(14);
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-                umma_bf16(tb + T_R1, desc_mn(smem_u32(s.Pu[0]), 8192, k), desc_mn(smem_u32(s.AkM[0]), 8192, k), id_agg, k > 0);
-            umma_commit(&s.bar_agg2);
-            PROF(15);
-        }
-        const bool last = (r + 1 == nchunks);
-        const float cm = sc.cm, cb = sc.cb;
-        const float cwn = last ? 1.0f : s.sc[(r + 1) & 1].cw;
-        const size_t head = (size_t)seq * dh;
 
-        mbar_wait(&s.bar_agg, ph, wc, 100 + 8);
-        PROF(10);
-        tc_fence_after_sync();
-        if (is_issuer && !last) {
-            // the W1 aggregations were the last readers of the key tile: the next chunk's tokens may land in X
-            load_tokens(seq * L + tok0 + C);
-        }
-        __syncwarp();
-        // ---------------- state pass, W1 half (Algorithm 1 lines 6-7), while the M2 aggregation still runs
-        float ss1 = 0.0f;
-#pragma unroll
-        for (int b = 0; b < NB; ++b) {
-            const int col = c0 + 16 * b;
-            uint32_t wa[16], ma[16], st[16];
-            float wn[16];
-            tmem_ld16(lane_addr + T_W1 + col, wa);
-            tmem_ld16(lane_addr + T_R0 + col, ma);
-            tmem_wait_ld();
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                const float m0 = M1[16 * b + j];
-                wn[j] = __uint_as_float(wa[j]) + cm * m0;
-                M1[16 * b + j] = cb * m0 + __uint_as_float(ma[j]);
-                st[j] = __float_as_uint(NORM ? wn[j] : cwn * wn[j]);
-                if (NORM) ss1 = fmaf(wn[j], wn[j], ss1);
-            }
-            tmem_st16(lane_addr + T_W1 + col, st);
-            if (!NORM) {
-                st_slab16(s.W1[col >> 6], row, col & 63, wn);
-                if ((last || a.ckpt) && cta_real && col < de) {  // final state, or the next chunk's start state for the backward
-                    const size_t off = ((size_t)(HC * me) + row) * de + col;
-                    float* ck = last ? nullptr : a.ckpt + (size_t)seq * a.ckpt_seq_stride + (size_t)(r + 1) * 4 * dh;
-                    float* wf = last ? a.W1_final + head + off : ck + off;
-                    float* mf = last ? a.M1_final + head + off : ck + 2 * dh + off;
-#pragma unroll
-                    for (int j = 0; j < 16; j += 4) {
-                        *reinterpret_cast<float4*>(wf + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
-                        *reinterpret_cast<float4*>(mf + j) =
-                            make_float4(M1[16 * b + j], M1[16 * b + j + 1], M1[16 * b + j + 2], M1[16 * b + j + 3]);
-                    }
-                }
-            }
-        }
-        if (NORM) {
-            // row sums of squares: the four column-group warps of a row meet in shared memory (the Pz tile is dead)
-            float* rs = reinterpret_cast<float*>(s.PzW[0]);  // [NG][128]
-            rs[g * 128 + row] = ss1;
-            tmem_wait_st();
-            tc_fence_before_sync();
-            __syncthreads();
-            tc_fence_after_sync();
-            float tot = 0.0f;
-#pragma unroll
-            for (int gg = 0; gg < NG; ++gg) tot += rs[gg * 128 + row];
-            const float f = tgt1 / (sqrtf(tot) + a.norm_eps);
-#pragma unroll
-            for (int b = 0; b < NB; ++b) {
-                const int col = c0 + 16 * b;
-                uint32_t wa[16], st[16];
-                float wn[16];
-                tmem_ld16(lane_addr + T_W1 + col, wa);
-                tmem_wait_ld();
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    wn[j] = __uint_as_float(wa[j]) * f;
-                    st[j] = __float_as_uint(cwn * wn[j]);
-                }
-                tmem_st16(lane_addr + T_W1 + col, st);
-                st_slab16(s.W1[col >> 6], row, col & 63, wn);
-                if (cta_real && col < de) {
-                    const size_t off = ((size_t)(HC * me) + row) * de + col;
-                    if (last) {
-#pragma unroll
-                        for (int j = 0; j < 16; j += 4) {
-                            *reinterpret_cast<float4*>(a.W1_final + head + off + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
-                            *reinterpret_cast<float4*>(a.M1_final + head + off + j) =
-                                make_float4(M1[16 * b + j], M1[16 * b + j + 1], M1[16 * b + j + 2], M1[16 * b + j + 3]);
-                        }
-                    }
-                    if (a.ckpt) {  // the state after this chunk: slot r + 1 (the last slot is the final state)
-                        float* ck = a.ckpt + (size_t)seq * a.ckpt_seq_stride + (size_t)(r + 1) * 4 * dh;
-#pragma unroll
-                        for (int j = 0; j < 16; j += 4) {
-                            *reinterpret_cast<float4*>(ck + off + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
-                            *reinterpret_cast<float4*>(ck + 2 * dh + off + j) =
-                                make_float4(M1[16 * b + j], M1[16 * b + j + 1], M1[16 * b + j + 2], M1[16 * b + j + 3]);
-                        }
-                    }
-                }
-            }
-            if (a.ckpt && g == 0 && cta_real)  // row norm before the normalisation, for the reverse pass
-                a.rown[(size_t)seq * a.ckpt_seq_stride + ((size_t)r * 3 + 0) * (size_t)max(de, he) + HC * me + row] = sqrtf(tot);
-        }
-        tmem_wait_st();
-        fence_proxy_async_smem();
-        tc_fence_before_sync();
-        __syncthreads();  // bf16 W1 is complete and R0 is free: the next chunk's G1 may run under the W2 half
-        PROF(11);
-        if (is_issuer && !last) issue_g1(r + 1);
-        __syncwarp();
+            // ---------------- state pass (Algorithm 1 lines 6-7)
+            if (!last) mbar_wait(&s.bar_sc, ph, wc, 100 + 37);  // the next chunk's scalars (its decay carry pre-scales the master)
+            PROF(18);
+            const float cm = sc.cm, cb = sc.cb;
+            const float cwn = last ? 1.0f : s.sc[(r + 1) & 1].cw;
+            const size_t head = (size_t)seq * dh;
+            // slot of the state after this chunk in the saved states (the slot after the last chunk is the final state)
+            float* ckn = a.ckpt ? a.ckpt + (size_t)seq * a.ckpt_seq_stride + (size_t)(r + 1) * 4 * dh : nullptr;
+            const bool save_ck = a.ckpt && (NORM || !last);
 
-        mbar_wait(&s.bar_agg2, ph, wc, 100 + 9);
-        PROF(12);
-        tc_fence_after_sync();
-        if (is_issuer) {
-            // every reader of this chunk's staging / pu / scaled-activation buffers is done: peers may overwrite them
-#pragma unroll
-            for (uint32_t dst = 0; dst < NC; ++dst)
-                if (dst != me) mbar_arrive_remote(map_to_cta(smem_u32(&s.bar_credit), dst));
-        }
-        __syncwarp();
-        // ---------------- state pass, W2 half
-        float ss2 = 0.0f;
-#pragma unroll
-        for (int b = 0; b < NB; ++b) {
-            const int col = c0 + 16 * b;
-            uint32_t wa[16], ma[16], st[16];
-            float wn[16];
-            tmem_ld16(lane_addr + T_W2 + col, wa);
-            tmem_ld16(lane_addr + T_R1 + col, ma);
-            tmem_wait_ld();
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                const float m0 = M2[16 * b + j];
-                wn[j] = __uint_as_float(wa[j]) + cm * m0;
-                M2[16 * b + j] = cb * m0 + __uint_as_float(ma[j]);
-                st[j] = __float_as_uint(NORM ? wn[j] : cwn * wn[j]);
-                if (NORM) ss2 = fmaf(wn[j], wn[j], ss2);
-            }
-            tmem_st16(lane_addr + T_W2 + col, st);
-            if (!NORM) {
-                st_slab16(s.W2[col >> 6], row, col & 63, wn);
-                if ((last || a.ckpt) && cta_real && row < de) {
-                    const size_t off = (size_t)row * he + HC * me + col;
-                    float* ck = last ? nullptr : a.ckpt + (size_t)seq * a.ckpt_seq_stride + (size_t)(r + 1) * 4 * dh;
-                    float* wf = last ? a.W2_final + head + off : ck + dh + off;
-                    float* mf = last ? a.M2_final + head + off : ck + 3 * dh + off;
-#pragma unroll
-                    for (int j = 0; j < 16; j += 4) {
-                        *reinterpret_cast<float4*>(wf + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
-                        *reinterpret_cast<float4*>(mf + j) =
-                            make_float4(M2[16 * b + j], M2[16 * b + j + 1], M2[16 * b + j + 2], M2[16 * b + j + 3]);
-                    }
-                }
-            }
-        }
-        if (NORM) {
-            // A row of W2 spans the cluster: the CTA's own sum of squares (over its four column-group warps) goes to
-            // every CTA, each adds the four pieces in CTA order (the same number everywhere).  The kW a tile is dead.
-            float* rs = reinterpret_cast<float*>(s.AkW[0]);          // [NG][128] this CTA's pieces
-            float* got = reinterpret_cast<float*>(s.AkW[0]) + 1024;  // [NC][128] one row-sum vector per CTA
-            rs[g * 128 + row] = ss2;
-            tmem_wait_st();
-            tc_fence_before_sync();
-            __syncthreads();
+            // W1 half, as soon as the W1 aggregation is in (the momentum aggregate follows right behind it)
+            mbar_wait(&s.bar_aw1, ph, wc, 100 + 38);
             tc_fence_after_sync();
-            if (warp == 0) {  // 32 lanes x 4 rows
-                // a peer's receive area overlays an operand tile of its W2 aggregations: it is free once that peer
-                // has seen them finish, which is what its credit of this chunk says
-                mbar_wait<true>(&s.bar_credit, ph, wc, 100 + 14);
-                float4 v;
-                float* pv = reinterpret_cast<float*>(&v);
+            PROF(9);
+            {
+                const bool real1 = cta_real;
+                const size_t off0 = ((size_t)(HC * me) + row) * de;
+                float ss1 = 0.0f;
 #pragma unroll
-                for (int x = 0; x < 4; ++x) {
-                    float t = 0.0f;
+                for (int b = 0; b < NB; ++b) {
+                    const int col = c0 + 16 * b;
+                    uint32_t wa[16], st[16];
+                    float wn[16];
+                    tmem_ld16(lane_addr + T_W1 + col, wa);
+                    tmem_wait_ld();
 #pragma unroll
-                    for (int gg = 0; gg < NG; ++gg) t += rs[gg * 128 + 4 * lane + x];
-                    pv[x] = t;
-                }
-                const uint32_t local = smem_u32(got + me * 128 + 4 * lane);
-                *reinterpret_cast<float4*>(got + me * 128 + 4 * lane) = v;
-#pragma unroll
-                for (uint32_t dst = 0; dst < NC; ++dst)
-                    if (dst != me)
-                        st_async_v4(map_to_cta(local, dst), __float_as_uint(v.x), __float_as_uint(v.y), __float_as_uint(v.z),
-                                    __float_as_uint(v.w), map_to_cta(smem_u32(&s.bar_rs), dst));
-            }
-            __syncthreads();  // the CTA's own vector is in place
-            mbar_wait<true>(&s.bar_rs, ph, wc, 100 + 13);
-            float tot = 0.0f;
-#pragma unroll
-            for (uint32_t c = 0; c < NC; ++c) tot += got[c * 128 + row];
-            const float f = tgt2 / (sqrtf(tot) + a.norm_eps);
-#pragma unroll
-            for (int b = 0; b < NB; ++b) {
-                const int col = c0 + 16 * b;
-                uint32_t wa[16], st[16];
-                float wn[16];
-                tmem_ld16(lane_addr + T_W2 + col, wa);
-                tmem_wait_ld();
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    wn[j] = __uint_as_float(wa[j]) * f;
-                    st[j] = __float_as_uint(cwn * wn[j]);
-                }
-                tmem_st16(lane_addr + T_W2 + col, st);
-                st_slab16(s.W2[col >> 6], row, col & 63, wn);
-                if (cta_real && row < de) {
-                    const size_t off = (size_t)row * he + HC * me + col;
-                    if (last) {
-#pragma unroll
-                        for (int j = 0; j < 16; j += 4) {
-                            *reinterpret_cast<float4*>(a.W2_final + head + off + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
-                            *reinterpret_cast<float4*>(a.M2_final + head + off + j) =
-                                make_float4(M2[16 * b + j], M2[16 * b + j + 1], M2[16 * b + j + 2], M2[16 * b + j + 3]);
-                        }
+                    for (int j = 0; j < 16; ++j) {
+                        wn[j] = fmaf(cm, M1[16 * b + j], __uint_as_float(wa[j]));
+                        st[j] = __float_as_uint(NORM ? wn[j] : cwn * wn[j]);
+                        if (NORM) ss1 = fmaf(wn[j], wn[j], ss1);
                     }
-                    if (a.ckpt) {
-                        float* ck = a.ckpt + (size_t)seq * a.ckpt_seq_stride + (size_t)(r + 1) * 4 * dh;
+                    tmem_st16(lane_addr + T_W1 + col, st);
+                    if (!NORM) {
+                        st_slab16(s.W1[col >> 6], row, col & 63, wn);
+                        if (real1 && col < de) {
+                            if (last) {
 #pragma unroll
-                        for (int j = 0; j < 16; j += 4) {
-                            *reinterpret_cast<float4*>(ck + dh + off + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
-                            *reinterpret_cast<float4*>(ck + 3 * dh + off + j) =
-                                make_float4(M2[16 * b + j], M2[16 * b + j + 1], M2[16 * b + j + 2], M2[16 * b + j + 3]);
+                                for (int j = 0; j < 16; j += 4)
+                                    *reinterpret_cast<float4*>(a.W1_final + head + off0 + col + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
+                            } else if (save_ck) {
+#pragma unroll
+                                for (int j = 0; j < 16; j += 4)
+                                    *reinterpret_cast<float4*>(ckn + off0 + col + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
+                            }
                         }
                     }
                 }
+                if (NORM) {
+                    // row sums of squares: the four column-group warps of a row meet in shared memory (the kW pz tile is dead)
+                    float* rs = reinterpret_cast<float*>(s.PzW[0]);  // [NG][128]
+                    rs[g * 128 + row] = ss1;
+                    tmem_wait_st();
+                    named_sync(BAR_EPI, NEPI);
+                    float tot = 0.0f;
+#pragma unroll
+                    for (int gg = 0; gg < NG; ++gg) tot += rs[gg * 128 + row];
+                    // padded hidden units have target 0 and norm 0: keep them at exactly 0 whatever norm_eps is
+                    const float f = cta_real ? tgt1 / (sqrtf(tot) + a.norm_eps) : 0.0f;
+#pragma unroll
+                    for (int b = 0; b < NB; ++b) {
+                        const int col = c0 + 16 * b;
+                        uint32_t wa[16], st[16];
+                        float wn[16];
+                        tmem_ld16(lane_addr + T_W1 + col, wa);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            wn[j] = __uint_as_float(wa[j]) * f;
+                            st[j] = __float_as_uint(cwn * wn[j]);
+                        }
+                        tmem_st16(lane_addr + T_W1 + col, st);
+                        st_slab16(s.W1[col >> 6], row, col & 63, wn);
+                        if (real1 && col < de) {
+                            if (last) {
+#pragma unroll
+                                for (int j = 0; j < 16; j += 4)
+                                    *reinterpret_cast<float4*>(a.W1_final + head + off0 + col + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
+                            }
+                            if (save_ck) {
+#pragma unroll
+                                for (int j = 0; j < 16; j += 4)
+                                    *reinterpret_cast<float4*>(ckn + off0 + col + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
+                            }
+                        }
+                    }
+                    if (a.ckpt && g == 0 && cta_real)  // row norm before the normalisation, for the reverse pass
+                        a.rown[(size_t)seq * a.ckpt_seq_stride + ((size_t)r * 3 + 0) * (size_t)max(de, he) + HC * me + row] = sqrtf(tot);
+                }
+                // momentum half of W1: M1 = cb M1 + aggregate (R0)
+                PROF(19);
+                mbar_wait(&s.bar_am1, ph, wc, 100 + 39);
+                PROF(20);
+                tc_fence_after_sync();
+#pragma unroll
+                for (int b = 0; b < NB; ++b) {
+                    const int col = c0 + 16 * b;
+                    uint32_t ma[16];
+                    tmem_ld16(lane_addr + T_R0 + col, ma);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) M1[16 * b + j] = fmaf(cb, M1[16 * b + j], __uint_as_float(ma[j]));
+                    if (real1 && col < de) {
+                        if (last) {
+#pragma unroll
+                            for (int j = 0; j < 16; j += 4)
+                                *reinterpret_cast<float4*>(a.M1_final + head + off0 + col + j) =
+                                    make_float4(M1[16 * b + j], M1[16 * b + j + 1], M1[16 * b + j + 2], M1[16 * b + j + 3]);
+                        }
+                        if (save_ck) {
+#pragma unroll
+                            for (int j = 0; j < 16; j += 4)
+                                *reinterpret_cast<float4*>(ckn + 2 * dh + off0 + col + j) =
+                                    make_float4(M1[16 * b + j], M1[16 * b + j + 1], M1[16 * b + j + 2], M1[16 * b + j + 3]);
+                        }
+                    }
+                }
+                tmem_wait_st();
+                warp_release(&s.bar_w1);  // bf16 W1 complete, master rescaled, R0 free: the next chunk's G1 may run
             }
-            if (a.ckpt && g == 0 && me == 0 && row < de)
-                a.rown[(size_t)seq * a.ckpt_seq_stride + ((size_t)r * 3 + 1) * (size_t)max(de, he) + row] = sqrtf(tot);
+            PROF(10);
+
+            // W2 half
+            mbar_wait(&s.bar_am2, ph, wc, 100 + 40);
+            tc_fence_after_sync();
+            PROF(11);
+            {
+                const bool real2 = cta_real && row < de;
+                const size_t off0 = (size_t)row * he + HC * me;
+                float ss2 = 0.0f;
+#pragma unroll
+                for (int b = 0; b < NB; ++b) {
+                    const int col = c0 + 16 * b;
+                    uint32_t wa[16], ma[16], st[16];
+                    float wn[16];
+                    tmem_ld16(lane_addr + T_W2 + col, wa);
+                    tmem_ld16(lane_addr + T_R1 + col, ma);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const float m0 = M2[16 * b + j];
+                        wn[j] = fmaf(cm, m0, __uint_as_float(wa[j]));
+                        M2[16 * b + j] = fmaf(cb, m0, __uint_as_float(ma[j]));
+                        st[j] = __float_as_uint(NORM ? wn[j] : cwn * wn[j]);
+                        if (NORM) ss2 = fmaf(wn[j], wn[j], ss2);
+                    }
+                    tmem_st16(lane_addr + T_W2 + col, st);
+                    if (real2) {
+                        if (last) {
+#pragma unroll
+                            for (int j = 0; j < 16; j += 4)
+                                *reinterpret_cast<float4*>(a.M2_final + head + off0 + col + j) =
+                                    make_float4(M2[16 * b + j], M2[16 * b + j + 1], M2[16 * b + j + 2], M2[16 * b + j + 3]);
+                        }
+                        if (save_ck) {
+#pragma unroll
+                            for (int j = 0; j < 16; j += 4)
+                                *reinterpret_cast<float4*>(ckn + 3 * dh + off0 + col + j) =
+                                    make_float4(M2[16 * b + j], M2[16 * b + j + 1], M2[16 * b + j + 2], M2[16 * b + j + 3]);
+                        }
+                    }
+                    if (!NORM) {
+                        st_slab16(s.W2[col >> 6], row, col & 63, wn);
+                        if (real2) {
+                            if (last) {
+#pragma unroll
+                                for (int j = 0; j < 16; j += 4)
+                                    *reinterpret_cast<float4*>(a.W2_final + head + off0 + col + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
+                            } else if (save_ck) {
+#pragma unroll
+                                for (int j = 0; j < 16; j += 4)
+                                    *reinterpret_cast<float4*>(ckn + dh + off0 + col + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
+                            }
+                        }
+                    }
+                }
+                if (NORM) {
+                    // A row of W2 spans the cluster: the CTA's own sum of squares (over its four column-group warps) goes to
+                    // every CTA, each adds the four pieces in CTA order (the same number everywhere).  The kW a tile is dead.
+                    float* rs = reinterpret_cast<float*>(s.AkW[0]);          // [NG][128] this CTA's pieces
+                    float* got = reinterpret_cast<float*>(s.AkW[0]) + 1024;  // [NC][128] one row-sum vector per CTA
+                    rs[g * 128 + row] = ss2;
+                    tmem_wait_st();
+                    named_sync(BAR_EPI, NEPI);
+                    if (warp == 0) {  // 32 lanes x 4 rows
+                        // a peer's receive area overlays an operand tile of its W2 aggregations: it is free once that peer
+                        // has seen them finish, which is what its credit of this chunk says
+                        mbar_wait<true>(&s.bar_credit, ph, wc, 100 + 41);
+                        float4 v;
+                        float* pv = reinterpret_cast<float*>(&v);
+#pragma unroll
+                        for (int x = 0; x < 4; ++x) {
+                            float t = 0.0f;
+#pragma unroll
+                            for (int gg = 0; gg < NG; ++gg) t += rs[gg * 128 + 4 * lane + x];
+                            pv[x] = t;
+                        }
+                        const uint32_t local = smem_u32(got + me * 128 + 4 * lane);
+                        *reinterpret_cast<float4*>(got + me * 128 + 4 * lane) = v;
+#pragma unroll
+                        for (uint32_t dst = 0; dst < NC; ++dst)
+                            if (dst != me)
+                                st_async_v4(map_to_cta(local, dst), __float_as_uint(v.x), __float_as_uint(v.y), __float_as_uint(v.z),
+                                            __float_as_uint(v.w), map_to_cta(smem_u32(&s.bar_rs), dst));
+                    }
+                    named_sync(BAR_EPI, NEPI);  // the CTA's own vector is in place
+                    mbar_wait<true>(&s.bar_rs, ph, wc, 100 + 42);
+                    float tot = 0.0f;
+#pragma unroll
+                    for (uint32_t c = 0; c < NC; ++c) tot += got[c * 128 + row];
+                    // padded rows have target 0 and norm 0: keep them at exactly 0 whatever norm_eps is
+                    const float f = row < de ? tgt2 / (sqrtf(tot) + a.norm_eps) : 0.0f;
+#pragma unroll
+                    for (int b = 0; b < NB; ++b) {
+                        const int col = c0 + 16 * b;
+                        uint32_t wa[16], st[16];
+                        float wn[16];
+                        tmem_ld16(lane_addr + T_W2 + col, wa);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            wn[j] = __uint_as_float(wa[j]) * f;
+                            st[j] = __float_as_uint(cwn * wn[j]);
+                        }
+                        tmem_st16(lane_addr + T_W2 + col, st);
+                        st_slab16(s.W2[col >> 6], row, col & 63, wn);
+                        if (real2) {
+                            if (last) {
+#pragma unroll
+                                for (int j = 0; j < 16; j += 4)
+                                    *reinterpret_cast<float4*>(a.W2_final + head + off0 + col + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
+                            }
+                            if (save_ck) {
+#pragma unroll
+                                for (int j = 0; j < 16; j += 4)
+                                    *reinterpret_cast<float4*>(ckn + dh + off0 + col + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
+                            }
+                        }
+                    }
+                    if (a.ckpt && g == 0 && me == 0 && row < de)
+                        a.rown[(size_t)seq * a.ckpt_seq_stride + ((size_t)r * 3 + 1) * (size_t)max(de, he) + row] = sqrtf(tot);
+                }
+                tmem_wait_st();
+                warp_release(&s.bar_w2);  // bf16 W2 complete, master rescaled, R1 free: the next chunk's G2 may run
+            }
+            PROF(12);
         }
-        tmem_wait_st();
-        fence_proxy_async_smem();
-        tc_fence_before_sync();
-        __syncthreads();
-        tc_fence_after_sync();
-        PROF(13);
     }
 
     // no CTA leaves while a peer may still write into its shared memory or arrive on its barriers
     tc_fence_before_sync();
+    __syncwarp();
     cluster_sync();
     if (warp == 0) tmem_dealloc(tb, 512);
 }

@@ -3,10 +3,6 @@
 #include <cuda_bf16.h>
 #include <stddef.h>
 
-#ifndef TC_NG
-#define TC_NG 4  // column groups per tensor-memory lane quadrant: the kernel runs 128 * TC_NG threads
-#endif
-
 namespace e2ttt {
 
 struct TcFwdArgs {
