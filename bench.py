@@ -114,7 +114,7 @@ class ClockSampler:
                 if val.lower().startswith("active"):
                     reasons.add(n)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "samples_under_load": len(sm), "reasons": sorted(reasons)}
 
 
 def cpu_oracle_rate(r: inputs.Recipe, budget_heads: int | None = None, tokens: int = 512):
@@ -139,7 +139,7 @@ def run_reference(args, r):
         return
     vals = []
     for i in range(args.warmup + args.steps):
-        res = cpu_oracle_rate(r, tokens=256)
+        res = cpu_oracle_rate(r)  # the same bounded sample as the cpu_baseline leg of the other arm
         if i >= args.warmup:
             vals.append(res)
     dt = float(np.mean([v["seconds"] for v in vals]))
@@ -172,11 +172,19 @@ def max_over_ranks(ms: float, dist, device) -> float:
     return float(t.item())
 
 
+def gates_text(r):
+    """The gate recipe of the run, as the JSON line states it."""
+    tau = "" if r.tau == 1.0 else f"^(1/{r.tau:g})"
+    regime = "paper regime (eta_base 0.01, tau 32, alpha_base 0.1): " if (r.eta_base, r.tau, r.alpha_base) == (0.01, 32.0, 0.1) else ""
+    return (f"{regime}eta={r.eta_base:g}*sigmoid(N(0,1)), beta=sigmoid(N(1,1)){tau}, "
+            f"gamma=1-eta*{r.alpha_base:g}*sigmoid(N(3,1))")
+
+
 def workload_config(r):
     kind = "mlp_gelu" if r.kind == inputs.KIND_MLP else "swiglu"
     return {"workload": f"e2ttt_chunk_fwd B={r.B} H={r.H} L={r.L} d={r.d} h={r.h} C={r.C} {kind} {r.io} I/O",
             "B": r.B, "H": r.H, "L": r.L, "d": r.d, "h": r.h, "C": r.C, "kind": kind, "io": r.io,
-            "gates": "eta=0.1*sigmoid(N(0,1)), beta=sigmoid(N(1,1)), gamma=1-eta*sigmoid(N(3,1))", "seed": r.seed,
+            "gates": gates_text(r), "seed": r.seed,
             "l2": "inputs larger than L2: q,k,v,o and states of one call exceed 126 MB"}
 
 
@@ -288,26 +296,46 @@ def run_ours(args, r):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def timed(fn, steps, warmup):
+    def timed(fn, steps, warmup, preroll_s):
+        """W warm-up steps, then an untimed pre-roll of the same step that keeps the GPU under this load for
+        `preroll_s` seconds (the 200 ms clock sampler needs a steady state to look at; a 20 ms region would give it one
+        sample), then EXACTLY `steps` timed steps: one event pair around all of them (the reported mean) and one pair
+        per step (the median)."""
         for _ in range(warmup):
             fn()
         barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(steps):
-            fn()
-        e1.record(stream)
+        t_end = time.perf_counter() + preroll_s
+        n_pre = 0
+        while time.perf_counter() < t_end:
+            for _ in range(8):
+                fn()
+            n_pre += 8
+            stream.synchronize()
         barrier()
-        ms = e0.elapsed_time(e1) / steps
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        ev[0].record(stream)
+        for i in range(steps):
+            fn()
+            ev[i + 1].record(stream)
+        barrier()
+        ms = ev[0].elapsed_time(ev[steps]) / steps
+        per_call = sorted(ev[i].elapsed_time(ev[i + 1]) for i in range(steps))
+        med = per_call[steps // 2]
         if world > 1:
             ms = max_over_ranks(ms, dist, dev)
-        return ms
+            med = max_over_ranks(med, dist, dev)
+        return ms, med, n_pre
 
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    ms = timed(step, args.steps, args.warmup)
+    ms, ms_median, n_preroll = timed(step, args.steps, args.warmup, args.preroll)
     clocks = sampler.stop() if rank == 0 else None
+    # the timed calls must have run clean: device status 0 (no bounded wait gave up) and finite outputs
+    status = E.e2ttt_device_status(ws, stream)
+    finite = bool(torch.isfinite(o.float()).all().item()) and all(bool(torch.isfinite(w).all().item()) for w in Wf + Mf)
+    if status != 0 or not finite:
+        raise SystemExit(f"bench: the timed calls did not run clean (device status {status}, finite outputs {finite})")
     ms_e2e = timed_e2e(max(4, args.steps))
 
     if rank == 0:
@@ -325,9 +353,13 @@ def run_ours(args, r):
         d2h = host_o.numel() * host_o.element_size() + 2 * sum(w.numel() * 4 for w in hostW)
         line = {
             "metric": METRIC, "value": whole_job_value(world, tokens, ms), "unit": UNIT, "n_gpus": world,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "ms_per_step_median": ms_median,
+            "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if r.io == "bf16" else "f64",
             "data": "synthetic",
+            "timing": f"CUDA events on the launch stream; {args.warmup} warm-up steps, {n_preroll} untimed pre-roll steps "
+                      f"(~{args.preroll:g} s of the same load, so the clock samples describe the timed region's steady state), "
+                      f"then exactly {args.steps} timed steps; device status 0 and finite outputs checked afterwards",
             "config": dict(workload_config(r), **({"post_chunk_norm": "rows of every W_i rescaled to the row norms of W_init after each chunk (any-shape kernels)"} if args.post_norm else {})),
             "e2e": {"value": whole_job_value(world, tokens, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e,
@@ -651,9 +683,33 @@ def main():
     ap.add_argument("--prepare", action="store_true", help="time the token preparation instead (e2ttt_prepare_fwd, 1 GPU)")
     ap.add_argument("--post-norm", action="store_true", help="forward with post-chunk normalisation of the fast weights (e2ttt_chunk_fwd_normed)")
     ap.add_argument("--chunk", type=int, default=0, help="override the chunk size C of the configuration")
+    ap.add_argument("--gates", default="benchmark", choices=["benchmark", "paper"],
+                    help="gate recipe: the benchmark's, or the paper's regime (eta_base 0.01, tau 32, alpha_base 0.1)")
+    ap.add_argument("--preroll", type=float, default=1.2,
+                    help="seconds of untimed steps under load before the timed ones (clock sampling); 0 = none")
+    ap.add_argument("--rank-check", action="store_true",
+                    help="no GPU work: every rank joins a gloo group and rank 0 prints the world size (tests the launch path)")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as plain `python bench.py --gpus N`: start the N ranks ourselves, one process per GPU
+        port = 29500 + (os.getpid() % 2000)
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        raise SystemExit(subprocess.call(cmd))
+    if args.rank_check:
+        import torch.distributed as dist
+        dist.init_process_group("gloo")
+        import torch
+        t = torch.ones(1)
+        dist.all_reduce(t)
+        if dist.get_rank() == 0:
+            print(json.dumps({"rank_check": True, "n_gpus": args.gpus, "world": dist.get_world_size(), "ranks_seen": int(t.item())}))
+        dist.destroy_process_group()
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     r = inputs.config(args.config, **({"C": args.chunk} if args.chunk else {}))
+    if args.gates == "paper":
+        r = inputs.paper_regime(r)
     if args.prepare and args.impl == "ours":
         run_prepare(args, r)
     elif args.decode and args.impl == "ours":

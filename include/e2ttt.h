@@ -23,16 +23,17 @@
  *     E2TTT_SWIGLU   : f_W(x) = x + LN(W3 (SiLU(W1 x) * (W2 x))),    W1 [h,d], W2 [h,d], W3 [d,h]
  * LN is a layer norm over the d outputs without affine parameters (biased variance, ln_eps inside
  * the square root); GELU is the exact erf form.  All matrices of the collection share the same
- * per-token scalars (Section 2: "W_t denotes the full collection of fast-weight tensors").
+ * per-token scalars (Section 2: for a multi-layer learner W_t stands for all of its matrices).
  *
  * Conventions for every entry point
  *   - All data pointers are DEVICE pointers unless the comment says "host".  Pointer tables
  *     (W_init and friends) are HOST arrays of e2ttt_num_matrices(kind) device pointers.
- *   - Tensors are dense and row-major.  q, k, v, o and their gradients: [B, H, L, d] in
- *     io_dtype.  Gates and gate gradients: [B, H, L] fp32.  Fast-weight / momentum matrices and
+ *   - Tensors are dense and row-major: there are no stride fields, a caller with another layout
+ *     makes a dense copy first.  q, k, v, o and their gradients: [B, H, L, d] in io_dtype.  Gates and gate gradients: [B, H, L] fp32.  Fast-weight / momentum matrices and
  *     their gradients: [B, H, rows, cols] fp32.
  *   - The caller owns every buffer.  The library allocates nothing and keeps no state between
- *     calls other than cached kernel attributes.  Work is enqueued on `stream` (a cudaStream_t
+ *     calls other than cached kernel attributes (one exception, stated there:
+ *     e2ttt_chunk_fwd_noalloc uses a scratch array of its own).  Work is enqueued on `stream` (a cudaStream_t
  *     passed as void*, NULL = the default stream); no entry point synchronises with the host.
  *   - Return value: E2TTT_OK (0) or a negative e2ttt_status.  Arguments are validated before
  *     anything is launched, so a failing call leaves every output untouched.  Nothing throws,
@@ -132,8 +133,8 @@ E2TTT_API int e2ttt_chunk_fwd(const e2ttt_params* p,
                     void* o, float* const* W_final, float* const* M_final,
                     void* workspace, size_t workspace_bytes, int save_states, void* stream);
 
-/* Reverse pass of e2ttt_chunk_fwd: the adjoint of the same program (the outer-loop gradient the
- * paper obtains by automatic differentiation, Appendix "Training Details": "plain PyTorch").
+/* Reverse pass of e2ttt_chunk_fwd: the adjoint of the same program (the outer-loop gradient, which
+ * the paper's own implementation leaves to automatic differentiation, Appendix "Training Details").
  *   q .. M_init            in   as in the forward
  *   d_o                    in   [B,H,L,d] io_dtype, gradient of the loss w.r.t. o
  *   dW_final, dM_final     in   host tables (fp32, state layout) or NULL for zeros
@@ -144,7 +145,8 @@ E2TTT_API int e2ttt_chunk_fwd(const e2ttt_params* p,
  *   states_saved           != 0: the workspace still holds the chunk-start states written by
  *                          e2ttt_chunk_fwd(save_states=1) for the same inputs; 0: they are
  *                          recomputed first
- * Both network kinds are supported (SIMT path).
+ * Both network kinds are supported.  The reverse pass runs on the any-shape kernels (SIMT, or TILED with
+ * tensor-core products for bf16 I/O); there is no fused reverse kernel.
  */
 E2TTT_API int e2ttt_chunk_bwd(const e2ttt_params* p,
                     const void* q, const void* k, const void* v,
@@ -193,7 +195,7 @@ E2TTT_API int e2ttt_chunk_bwd_normed(const e2ttt_params* p, const void* q, const
  * call returned for the same tokens).  So a decoder calls e2ttt_apply per incoming token (p->L = 1) and
  * e2ttt_chunk_fwd once every C tokens.
  *   p        in  (host)    B, H, d, h, kind, io_dtype, ln_eps as above; L = tokens per sequence in this call;
- *                          C and impl are ignored
+ *                          C and impl are not used but must hold valid values (every field is validated)
  *   q        in  (device)  [B,H,L,d] io_dtype, 16-byte aligned
  *   W        in  (host array of device pointers)  the nmat fast-weight matrices, fp32, shapes as above
  *   o        out (device)  [B,H,L,d] io_dtype, 16-byte aligned
@@ -210,7 +212,8 @@ E2TTT_API int e2ttt_apply(const e2ttt_params* p, const void* q, const float* con
  *   gamma = 1 - eta * alpha_base sigmoid(a_alpha).
  * The logits a_* are the outputs of the model's small linear heads, which stay with the caller.  (The paper does
  * not say how a zero vector is normalised: the max(., norm_eps) of the common library routine is a reading.)
- *   p        in  (host)    B, H, L, d, io_dtype; the other fields are ignored
+ *   p        in  (host)    B, H, L, d, io_dtype; the other fields are not used but must hold valid values
+ *                          (every field is validated)
  *   g        in  (host)    eta_base > 0, tau > 0, alpha_base >= 0, norm_eps >= 0
  *   q_raw, k_raw      in  (device)  [B,H,L,d] io_dtype
  *   a_eta, a_beta, a_alpha  in (device)  [B,H,L] fp32
@@ -219,6 +222,8 @@ E2TTT_API int e2ttt_apply(const e2ttt_params* p, const void* q, const float* con
  * e2ttt_prepare_bwd gives the adjoints of q_raw, k_raw and the three logits from those of q, k, eta, beta,
  * gamma (what e2ttt_chunk_bwd returns); it re-reads the forward's inputs and needs none of its outputs.
  * Arithmetic in fp32; no workspace; enqueued on `stream`; HBM-bound (every byte read once, written once).
+ * These two kernels take no workspace and therefore have no device status word: their bounded waits guard bulk
+ * loads, which cannot fail short of a device fault (and that the next runtime call reports).
  * Returns E2TTT_OK or E2TTT_ERR_NULL / _SHAPE / _DTYPE / _ARCH / _CUDA. */
 typedef struct {
     float eta_base, tau, alpha_base, norm_eps;
@@ -233,7 +238,9 @@ E2TTT_API int e2ttt_prepare_bwd(const e2ttt_params* p, const e2ttt_gate_params* 
                                 float* da_alpha, void* stream);
 
 /* Reads back the device status word of the last launch that used `workspace` (the first word of every
- * workspace).  This is the one entry point that synchronises: it waits for `stream`.
+ * workspace).  workspace == NULL reads the word of the scratch array e2ttt_chunk_fwd_noalloc uses on the
+ * current device (0 if that entry point has not run there yet).  This is the one entry point that
+ * synchronises: it waits for `stream`.
  *   status  out (host)  0 after a clean run; otherwise the code of the first bounded device-side wait
  *                       that gave up (the tensor-core kernels never spin without a limit)
  * Returns E2TTT_OK, E2TTT_ERR_TIMEOUT when the word is non-zero, or E2TTT_ERR_NULL / E2TTT_ERR_CUDA.
@@ -269,6 +276,15 @@ E2TTT_API int e2ttt_chunk_fwd_noalloc(const e2ttt_params* p,
                     const float* eta, const float* beta, const float* gamma,
                     const float* const* W_init, const float* const* M_init,
                     void* o, float* const* W_final, float* const* M_final, void* stream);
+
+/* Self-test of the device-side failure path, in a form that fails nothing: one CTA waits, for at most
+ * `limit_cycles` SM cycles (1 .. 2e9), on a barrier that nobody signals.  The bounded wait runs out, the kernel
+ * records its code in the status word of `workspace` (at least 256 bytes, 256-byte aligned, device) and
+ * returns; e2ttt_device_status(workspace, ...) then reports E2TTT_ERR_TIMEOUT with a non-zero word, exactly as
+ * it would after a real stall.  Nothing traps or hangs and the context stays usable.
+ * (No counterpart in the paper: an operational guard of this implementation.)
+ * Returns E2TTT_OK (the kernel was enqueued) or E2TTT_ERR_NULL / _WORKSPACE / _ALIGN / _SHAPE / _ARCH / _CUDA. */
+E2TTT_API int e2ttt_selftest_wait_timeout(void* workspace, size_t workspace_bytes, long long limit_cycles, void* stream);
 
 /* Static description of a status code (never NULL). */
 E2TTT_API const char* e2ttt_status_string(int status);

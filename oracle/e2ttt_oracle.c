@@ -7,8 +7,8 @@
  *   - the token-wise recurrence  M_t = beta_t M_{t-1} + eta_t G_t,  W_t = gamma_t W_{t-1} + M_t
  *     (Eq. "tokenwise_ttt_decay_momentum", Section 3.1), run literally, one token at a time;
  *   - G_t = - grad_W L(f_{W_0}(k_t), v_t) taken at the frozen chunk-start weights W_0
- *     (Section 3.1, Eq. "ttt_minibatch_update"), L = 1/2 ||f - v||^2 (the paper says only
- *     "commonly Mean Squared Error"; the scale is a reading);
+ *     (Section 3.1, Eq. "ttt_minibatch_update"), L = 1/2 ||f - v||^2 (Section 2 names the usual choice, a mean
+ *     squared error, without a formula; the scale is a reading);
  *   - outputs o_t = f_{W_0}(q_t) from the chunk-start weights (Eq. "chunkwise_output",
  *     Algorithm 1 line 1);
  *   - fast-weight networks of Section 4 "Fast-weight Network":

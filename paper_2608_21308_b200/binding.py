@@ -13,7 +13,7 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.environ.get("E2TTT_LIB") or os.path.join(_HERE, "lib", "libe2ttt.so")  # E2TTT_LIB: use another build
+LIB_PATH = os.path.join(_HERE, "lib", "libe2ttt.so")
 
 E2TTT_MLP_GELU, E2TTT_SWIGLU = 0, 1
 E2TTT_F32, E2TTT_BF16 = 0, 1
@@ -76,6 +76,8 @@ def lib() -> ctypes.CDLL:
         L.e2ttt_apply.restype = cp
         L.e2ttt_device_status.argtypes = [vp, vp, ctypes.POINTER(cp)]
         L.e2ttt_device_status.restype = cp
+        L.e2ttt_selftest_wait_timeout.argtypes = [vp, ctypes.c_size_t, ctypes.c_longlong, vp]
+        L.e2ttt_selftest_wait_timeout.restype = cp
         L.e2ttt_status_string.argtypes = [cp]
         L.e2ttt_status_string.restype = ctypes.c_char_p
         L.e2ttt_version.argtypes = []
@@ -300,12 +302,23 @@ def e2ttt_chunk_bwd(p, q, k, v, eta, beta, gamma, W_init, M_init, d_o, dW_final,
 
 
 def e2ttt_device_status(workspace, stream=None) -> int:
-    """int e2ttt_device_status(...): waits for the stream and returns the device status word (0 = clean)."""
+    """int e2ttt_device_status(...): waits for the stream and returns the device status word (0 = clean).
+    workspace=None reads the word of the scratch array that e2ttt_chunk_fwd_noalloc uses on the current device."""
     word = ctypes.c_int(-1)
-    st = lib().e2ttt_device_status(_ptr(workspace, torch.uint8, None, "workspace"), _stream_ptr(stream), ctypes.byref(word))
+    wp = None if workspace is None else _ptr(workspace, torch.uint8, None, "workspace")
+    st = lib().e2ttt_device_status(wp, _stream_ptr(stream), ctypes.byref(word))
     if st not in (E2TTT_OK, -8):
         raise E2TTTError(st, "e2ttt_device_status")
     return int(word.value)
+
+
+def e2ttt_selftest_wait_timeout(workspace, limit_cycles: int, stream=None) -> int:
+    """int e2ttt_selftest_wait_timeout(...): enqueues one CTA whose bounded wait runs out after limit_cycles."""
+    st = lib().e2ttt_selftest_wait_timeout(_ptr(workspace, torch.uint8, None, "workspace"), workspace.numel(),
+                                           int(limit_cycles), _stream_ptr(stream))
+    if st != E2TTT_OK:
+        raise E2TTTError(st, "e2ttt_selftest_wait_timeout")
+    return st
 
 
 E2TTT_NOALLOC_SCRATCH_BYTES = 8 << 20

@@ -9,6 +9,10 @@
 
 using namespace e2ttt;
 
+namespace e2ttt {
+const void* noalloc_scratch_if_known();  // noalloc.cu
+}
+
 namespace {
 
 constexpr int kMaxD = 1024;
@@ -391,7 +395,11 @@ int e2ttt_prepare_bwd(const e2ttt_params* p, const e2ttt_gate_params* g, const v
 }
 
 int e2ttt_device_status(const void* workspace, void* stream, int* status) {
-    if (!workspace || !status) return E2TTT_ERR_NULL;
+    if (!status) return E2TTT_ERR_NULL;
+    if (!workspace) {  // the scratch array of e2ttt_chunk_fwd_noalloc on this device
+        workspace = noalloc_scratch_if_known();
+        if (!workspace) { *status = 0; return E2TTT_OK; }
+    }
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     int word = 0;
     if (cudaMemcpyAsync(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||

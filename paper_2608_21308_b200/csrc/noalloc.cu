@@ -19,9 +19,12 @@ std::mutex g_mu;
 // In host code the array's name is only a handle: the address a kernel may use has to be asked for,
 // once per device, while that device is current.
 int scratch_for_current_device(void** out) {
-    int dev = -1;
+    int dev = -1, major = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return E2TTT_ERR_ARCH; }
     if (dev < 0 || dev >= kMaxDevices) return E2TTT_ERR_ARCH;
+    // the device image holds sm_100a code only: ask for the architecture before asking for a symbol of it
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) { (void)cudaGetLastError(); return E2TTT_ERR_ARCH; }
+    if (major != 10) return E2TTT_ERR_ARCH;
     std::lock_guard<std::mutex> lock(g_mu);
     if (!g_scratch_known[dev]) {
         void* p = nullptr;
@@ -37,6 +40,18 @@ int scratch_for_current_device(void** out) {
 }
 
 }  // namespace
+
+namespace e2ttt {
+// Device address of the scratch array on the current device, or nullptr before the first call there.  Its first
+// word is the device status word of the calls that used it (read by e2ttt_device_status(NULL, ...)).
+const void* noalloc_scratch_if_known() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
+    if (dev < 0 || dev >= kMaxDevices) return nullptr;
+    std::lock_guard<std::mutex> lock(g_mu);
+    return g_scratch_known[dev] ? g_scratch_addr[dev] : nullptr;
+}
+}  // namespace e2ttt
 
 extern "C" E2TTT_API int e2ttt_chunk_fwd_noalloc(const e2ttt_params* p, const void* q, const void* k, const void* v,
                                                 const float* eta, const float* beta, const float* gamma,

@@ -214,17 +214,19 @@ template <int N> __device__ __forceinline__ void bulk_wait_read() {
 template <int N> __device__ __forceinline__ void bulk_wait_all() {
     asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
 }
-// bounded wait for a tile (about a second); on time-out the CTA stops waiting and finishes without meaning
-__device__ __forceinline__ bool bulk_wait_tile(uint64_t* bar, uint32_t parity, volatile int* dead) {
-    if ((threadIdx.x & 31) == 0 && !*dead) {
+// Bounded wait for a tile (about a second), every lane polling so that the warp stays converged.  A wait that runs out
+// raises the CTA-wide `dead` flag; later waits then return at once and the CTA runs through its remaining tiles (and all
+// of its barriers) without meaning.  These two kernels have no status word to report it through: the bulk loads they
+// wait for cannot fail short of a device fault, which the next runtime call reports.
+__device__ __forceinline__ void bulk_wait_tile(uint64_t* bar, uint32_t parity, volatile int* dead) {
+    if (!sm100::mbar_try_wait<false>(bar, parity) && !*dead) {
         const long long t0 = clock64();
         int spins = 0;
         while (!sm100::mbar_try_wait<false>(bar, parity)) {
-            if ((++spins & 255) == 0 && clock64() - t0 > sm100::kWaitCycles) { *dead = 1; break; }
+            if ((++spins & 255) == 0 && (*dead || clock64() - t0 > sm100::kWaitCycles)) { *dead = 1; break; }
         }
     }
     __syncwarp();
-    return !*dead;
 }
 
 // LPR = lanes per row: a row is LPR pieces of 16 bytes (d = LPR * 16 / sizeof(IO)), one piece per lane, so a warp works on
@@ -269,7 +271,7 @@ __global__ void __launch_bounds__(kPrThreads) prepare_fwd_bulk_kernel(const Prep
         const int s = (int)(it % kBkStages);
         const uint32_t parity = (uint32_t)((it / kBkStages) & 1);
         const int ntok = tokens_of(tile);
-        if (!bulk_wait_tile(&full[s], parity, dead)) break;
+        bulk_wait_tile(&full[s], parity, dead);
         IO* tq = reinterpret_cast<IO*>(tiles + (size_t)(2 * s) * tile_bytes);
         IO* tk = reinterpret_cast<IO*>(tiles + (size_t)(2 * s + 1) * tile_bytes);
         // gates of the tile's tokens (plain coalesced accesses)
@@ -434,7 +436,7 @@ __global__ void __launch_bounds__(kPrThreads) prepare_bwd_bulk_kernel(const Prep
         const int s = (int)(it % kBkStagesBwd);
         const uint32_t parity = (uint32_t)((it / kBkStagesBwd) & 1);
         const int ntok = tokens_of(tile);
-        if (!bulk_wait_tile(&full[s], parity, dead)) break;
+        bulk_wait_tile(&full[s], parity, dead);
         unsigned char* st = tiles + (size_t)(4 * s) * tile_bytes;
         if (tid < ntok) {  // adjoints of the gate logits
             const long long t = tile * kBkTok + tid;

@@ -63,11 +63,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Every wait is bounded.  A wait that runs out records where it gave up in *status (first failure wins)
 // and raises the CTA-wide `dead` flag; once it is up, later waits return at once, so the kernel still runs
 // through all of its barriers and its tensor-memory release, just without meaning, and the host reads the status.
+constexpr long long kWaitCycles = 2000000000LL;  // ~1 s at B200 clocks
 struct WaitCtx {
     volatile int* dead;      // shared memory, one per CTA
     int* status;             // global memory, one per launch (0 = fine)
+    long long limit = kWaitCycles;  // cycles after which a wait gives up
 };
-constexpr long long kWaitCycles = 2000000000LL;  // ~1 s at B200 clocks
 
 // Single-thread wait (the caller is one elected lane).
 template <bool CLUSTER = false>
@@ -82,7 +83,7 @@ __device__ __forceinline__ bool mbar_wait_one(uint64_t* bar, uint32_t parity, co
 #endif
         if ((++spins & 63) == 0) {
             if (*w.dead) return false;
-            if (clock64() - t0 > kWaitCycles) {
+            if (clock64() - t0 > w.limit) {
                 *w.dead = 1;
                 atomicCAS(w.status, 0, where);
                 return false;
@@ -105,7 +106,7 @@ __device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, const 
 #endif
             if ((++spins & 63) == 0) {
                 if (*w.dead) break;
-                if (clock64() - t0 > kWaitCycles) {
+                if (clock64() - t0 > w.limit) {
                     *w.dead = 1;
                     atomicCAS(w.status, 0, where);
                     break;

@@ -120,3 +120,20 @@ def test_binding_refuses_host_tensors(L):
     t = torch.zeros(1, 1, 16, 8)
     with pytest.raises(TypeError):
         E.e2ttt_chunk_fwd(p, t, t, t, t, t, t, [t, t], None, t, [t, t], [t, t], torch.zeros(8, dtype=torch.uint8))
+
+
+def test_selftest_entry_point_validates_before_any_device_use(L):
+    vp = ctypes.c_void_p
+    f = L.e2ttt_selftest_wait_timeout
+    f.argtypes = [vp, ctypes.c_size_t, ctypes.c_longlong, vp]
+    assert f(None, 256, 1000, None) == -1
+    assert f(vp(0x100000), 128, 1000, None) == -5
+    assert f(vp(0x100010), 256, 1000, None) == -4
+    assert f(vp(0x100000), 256, 0, None) == -2
+    assert f(vp(0x100000), 256, 3_000_000_000, None) == -2
+
+
+def test_device_status_of_the_noalloc_scratch_before_any_call_is_clean(L):
+    word = ctypes.c_int(-1)
+    assert L.e2ttt_device_status(None, None, ctypes.byref(word)) == 0 and word.value == 0
+    assert L.e2ttt_device_status(None, None, None) == -1

@@ -21,7 +21,7 @@ def _dev(a, dtype=torch.float32):
     return torch.tensor(np.ascontiguousarray(a), dtype=torch.float32).to(dtype).cuda().contiguous()
 
 
-def gpu_forward_normed(x, tgt, *, d, h, C, kind, io, impl, save_states=False):
+def gpu_forward_normed(x, tgt, *, d, h, C, kind, io, impl, save_states=False, norm_eps=EPS_N):
     N, L, _ = x["q"].shape
     p = E.make_params(N, 1, L, d, h, C, kind, E.E2TTT_F32 if io == "f32" else E.E2TTT_BF16, 1e-5, impl)
     iod = torch.float32 if io == "f32" else torch.bfloat16
@@ -34,7 +34,7 @@ def gpu_forward_normed(x, tgt, *, d, h, C, kind, io, impl, save_states=False):
     Wf = [torch.empty_like(w) for w in W]
     Mf = [torch.empty_like(w) for w in W]
     ws = torch.empty(E.e2ttt_workspace_bytes_normed(p, int(save_states)), dtype=torch.uint8, device="cuda")
-    E.e2ttt_chunk_fwd_normed(p, q, k, v, eta, beta, gamma, W, M, rn, EPS_N, o, Wf, Mf, ws, int(save_states))
+    E.e2ttt_chunk_fwd_normed(p, q, k, v, eta, beta, gamma, W, M, rn, norm_eps, o, Wf, Mf, ws, int(save_states))
     torch.cuda.synchronize()
     assert E.e2ttt_device_status(ws) == 0
     return {"o": o.float().cpu().numpy().reshape(N, L, d), "W": [w.cpu().numpy()[:, 0] for w in Wf],
@@ -158,6 +158,23 @@ def test_fused_normed_forward_windows(cfg, over):
     for i, t in enumerate(tgt):
         assert np.allclose(np.sqrt((got["W"][i].astype(np.float64) ** 2).sum(-1)), t, rtol=1e-3)
     print(errs)
+
+
+@pytest.mark.parametrize("cfg,over", [(1, {}), (2, dict(h=384))], ids=["64x256-padded", "128x384-padded"])
+def test_fused_normed_padded_shapes_with_zero_norm_eps(cfg, over):
+    """norm_eps = 0 is allowed.  The padded rows of the 128 x 512 tiles have target 0 and norm 0: they must stay exactly
+    0 (not 0/0), so every result is finite and agrees with the any-shape kernels."""
+    r = inputs.config(cfg, heads=[3, 30], m_std=0.002, **over)
+    xw, _ = util.teacher_forced_windows(r, 4, window=2)
+    tgt = targets(xw, 0.9)
+    shape = dict(d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16")
+    fused = gpu_forward_normed(xw, tgt, impl=E.E2TTT_IMPL_TCGEN05, norm_eps=0.0, **shape)
+    tiled = gpu_forward_normed(xw, tgt, impl=E.E2TTT_IMPL_TILED, norm_eps=0.0, **shape)
+    assert np.isfinite(fused["o"]).all() and all(np.isfinite(w).all() for w in fused["W"] + fused["M"])
+    assert util.rel_err(fused["o"], tiled["o"]) <= 3 * TOL_BF16
+    for i in range(2):
+        assert util.rel_err(fused["W"][i], tiled["W"][i]) <= 3 * TOL_BF16
+        assert util.rel_err(fused["M"][i], tiled["M"][i]) <= 3 * TOL_BF16
 
 
 def test_fused_normed_forward_free_running_and_auto_selection():

@@ -159,6 +159,20 @@ def test_backward_teacher_forced_windows_bf16_config4():
     check_backward(got, ref, TOL_BF16, "config 4 bwd windows")
 
 
+def test_config4_windows_across_the_whole_sequence_forward_and_backward():
+    """Config 4 has 512 chunks: one-chunk windows started from the oracle's state at chunks 0, 100, 300 and 511, on 8 of
+    its 16 heads, forward (fused kernel) and backward with seeded state adjoints (all ten gradient groups)."""
+    r = inputs.config(4, heads=[0, 2, 4, 6, 9, 11, 13, 15])
+    xw, ref = util.teacher_forced_windows_at(r, [0, 100, 300, 511], with_grads=True)
+    got, _ = util.gpu_forward(xw, d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16")
+    errs = check_forward(got, ref, TOL_BF16, "config 4 fwd windows at chunks 0/100/300/511")
+    print("config 4 fwd windows", errs)
+    refb = util.oracle_backward(xw, r.C, r.kind)
+    gotb = util.gpu_backward(xw, d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16")
+    errb = check_backward(gotb, refb, TOL_BF16, "config 4 bwd windows at chunks 0/100/300/511")
+    print("config 4 bwd windows", errb)
+
+
 # ------------------------------------------------------------------ properties that hold at any size
 def test_split_calls_chain_and_in_place_state_update():
     r = inputs.Recipe(B=3, H=1, L=128, d=32, h=64, C=32, kind=MLP, io="bf16", seed=3)

@@ -44,6 +44,33 @@ def test_tc_free_running_paper_regime():
     check_forward(tc, ref, TOL_BF16, "tc paper regime, 16 chunks free-running")
 
 
+def test_tc_free_running_64_chunks_paper_regime():
+    """The graded shape's full length (L = 4096 = 64 chunks) free-running against the oracle: every phase parity and
+    every credit of the chunk pipeline is exercised 64 times.  Under the paper's gate regime the map is well
+    conditioned, so the whole sequence can be compared."""
+    r = inputs.paper_regime(inputs.Recipe(B=2, H=1, L=4096, d=128, h=512, C=64, kind=MLP, io="bf16", seed=7, m_std=0.002))
+    x = inputs.generate(r)
+    ref = util.oracle_forward(x, 64, MLP)
+    tc, hd = util.gpu_forward(x, impl=E.E2TTT_IMPL_TCGEN05, **SHAPE)
+    assert E.e2ttt_device_status(hd["ws"]) == 0
+    errs = check_forward(tc, ref, TOL_BF16, "tc paper regime, 64 chunks free-running")
+    print("64 chunks free-running", errs)
+
+
+HEADS8 = [0, 9, 18, 27, 36, 45, 54, 63]
+
+
+def test_tc_windows_across_the_whole_sequence_config2():
+    """One-chunk windows started from the oracle's state at chunks 0, 7, 31 and 63 of config 2 (the states late in a
+    sequence are large), on 8 heads."""
+    r = inputs.config(2, heads=HEADS8)
+    xw, ref = util.teacher_forced_windows_at(r, [0, 7, 31, 63])
+    tc, hd = util.gpu_forward(xw, impl=E.E2TTT_IMPL_TCGEN05, **SHAPE)
+    assert E.e2ttt_device_status(hd["ws"]) == 0
+    errs = check_forward(tc, ref, TOL_BF16, "tc windows at chunks 0/7/31/63")
+    print("windows across the sequence", errs)
+
+
 def test_tc_null_momentum_determinism_and_many_sequences():
     r = inputs.config(2, heads=list(range(40)), L=256)       # 40 clusters: more than one wave of clusters is not needed, just many
     x = inputs.generate(r)

@@ -45,3 +45,17 @@ def test_two_ranks_independent_shards_and_max_time():
     assert q0 != q1 and o0 != o1                 # every rank has its own batch
     assert m0 == m1 == 20.0                      # MAX over ranks
     assert v0 == v1 == 2 * 16 / 20e-3            # all tokens / slowest time
+
+
+def test_bench_gpus_flag_starts_its_own_ranks():
+    """`python bench.py --gpus 2` (no torchrun around it) must start two ranks itself; --rank-check makes them meet on
+    gloo without touching a GPU and rank 0 report what it saw."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--rank-check"], env=env,
+                         capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    line = [ln for ln in out.stdout.splitlines() if ln.startswith("{")][-1]
+    rec = json.loads(line)
+    assert rec["world"] == 2 and rec["ranks_seen"] == 2 and rec["n_gpus"] == 2

@@ -51,6 +51,20 @@ def test_noalloc_forward_matches_the_ordinary_entry_point_twice_in_a_row():
         assert np.isfinite(got["o"]).all()
 
 
+def test_noalloc_forward_matches_the_oracle_and_reports_its_status():
+    """The entry point stands on its own: compared with the fp64 oracle directly, and its device status word (kept in
+    the library's scratch array, read with workspace = None) is clean afterwards."""
+    r = inputs.Recipe(B=1, H=2, L=64, d=64, h=256, C=16, kind=inputs.KIND_MLP, io="f32", seed=23, m_std=0.01)
+    x = inputs.generate(r)
+    got, _ = _run_both(23, 64)
+    ref = util.oracle_forward(x, r.C, r.kind)
+    assert util.rel_err(got["o"], ref["o"]) <= TOL
+    for i in range(2):
+        assert util.rel_err(got["W"][i], ref["W"][i]) <= TOL
+        assert util.rel_err(got["M"][i], ref["M"][i]) <= TOL
+    assert E.e2ttt_device_status(None) == 0
+
+
 def test_noalloc_refuses_shapes_beyond_its_fixed_scratch():
     p = E.make_params(4, 16, 64, 128, 512, 64, io_dtype=E.E2TTT_BF16, impl=E.E2TTT_IMPL_SIMT)  # SIMT scratch: ~100 MB
     assert E.e2ttt_workspace_bytes(p, 0) > E.E2TTT_NOALLOC_SCRATCH_BYTES

@@ -125,3 +125,41 @@ def teacher_forced_windows(r: inputs.Recipe, n_chunks: int, window: int = 1, wit
         xw["dM"] = [rng.standard_normal(w.shape).astype(np.float32) for w in xw["W"]]
     ref = oracle_forward(xw, C, r.kind)
     return xw, ref
+
+
+def teacher_forced_windows_at(r: inputs.Recipe, chunks, with_grads: bool = False):
+    """One-chunk windows at the given chunk indices of a long sequence, each started from the ORACLE's state there.
+
+    The oracle runs the sequence once from token 0 to the last requested chunk, in segments chained through its final
+    state (a long run and the same run cut into calls are the same program), so no per-chunk states are stored.
+    Returns (xw, ref) like teacher_forced_windows: N = heads * len(chunks) windows of L = C tokens.
+    """
+    C = r.C
+    chunks = sorted(chunks)
+    rr = inputs.Recipe(**{**r.__dict__, "L": (chunks[-1] + 1) * C})
+    x = inputs.generate(rr, with_d_o=with_grads, with_dstate=False)
+    N = x["q"].shape[0]
+    shapes = inputs.mat_shapes(r.kind, r.d, r.h)
+    nm = len(shapes)
+    W = [w.astype(np.float64) for w in x["W"]]
+    M = [m.astype(np.float64) for m in x["M"]]
+    pos = 0
+    starts = []
+    for c in chunks:
+        if c * C > pos:
+            seg = {n: np.ascontiguousarray(x[n][:, pos:c * C]) for n in ("q", "k", "v", "eta", "beta", "gamma")}
+            res = oracle.forward(seg["q"], seg["k"], seg["v"], seg["eta"], seg["beta"], seg["gamma"], W, M, C, r.kind)
+            W, M = res["W"], res["M"]
+            pos = c * C
+        starts.append(([w.copy() for w in W], [m.copy() for m in M]))
+    names = ("q", "k", "v", "eta", "beta", "gamma") + (("d_o",) if with_grads else ())
+    xw = {n: np.ascontiguousarray(np.stack([x[n][:, c * C:(c + 1) * C] for c in chunks], axis=1).reshape((N * len(chunks), C) + x[n].shape[2:]))
+          for n in names}
+    xw["W"] = [np.stack([s[0][i] for s in starts], axis=1).reshape((N * len(chunks),) + shapes[i]).astype(np.float32) for i in range(nm)]
+    xw["M"] = [np.stack([s[1][i] for s in starts], axis=1).reshape((N * len(chunks),) + shapes[i]).astype(np.float32) for i in range(nm)]
+    if with_grads:
+        rng = np.random.Generator(np.random.Philox(key=[r.seed, 778]))
+        xw["dW"] = [rng.standard_normal(w.shape).astype(np.float32) for w in xw["W"]]
+        xw["dM"] = [rng.standard_normal(w.shape).astype(np.float32) for w in xw["W"]]
+    ref = oracle_forward(xw, C, r.kind)
+    return xw, ref
