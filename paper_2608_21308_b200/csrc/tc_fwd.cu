@@ -547,23 +547,24 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             tc_fence_after_sync();
             PROF(1);
             {
-                {
-                    uint32_t z[NB][16];
 #pragma unroll
-                    for (int b = 0; b < NB; ++b) tmem_ld16(lane_addr + T_R0 + c0 + 16 * b, z[b]);
+                for (int b = 0; b < NB; ++b) {
+                    uint32_t z[16];
+                    tmem_ld16(lane_addr + T_R0 + c0 + 16 * b, z);
                     tmem_wait_ld();
+                    uint32_t p[8];
 #pragma unroll
-                    for (int b = 0; b < NB; ++b) {
-                        uint32_t p[8], ph16[8];
+                    for (int i = 0; i < 8; ++i) {
+                        const float a0 = gelu_only(__uint_as_float(z[2 * i])), a1 = gelu_only(__uint_as_float(z[2 * i + 1]));
+                        p[i] = pack_bf16(a0, a1);
+                        z[i] = pack_f16(a0, a1);  // fp16 keeps 3 more bits: no visible second rounding in kW a, kM a
+                    }
+                    const int col = c0 + 16 * b;
+                    st_slab16p(s.A[col >> 6], row, col & 63, p);
+                    if (q < 2) {
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            const float a0 = gelu_only(__uint_as_float(z[b][2 * i])), a1 = gelu_only(__uint_as_float(z[b][2 * i + 1]));
-                            p[i] = pack_bf16(a0, a1);
-                            ph16[i] = pack_f16(a0, a1);  // fp16 keeps 3 more bits: no visible second rounding in kW a, kM a
-                        }
-                        const int col = c0 + 16 * b;
-                        st_slab16p(s.A[col >> 6], row, col & 63, p);
-                        if (q < 2) st_slab16p(s.AkW[col >> 6], row, col & 63, ph16);
+                        for (int i = 0; i < 8; ++i) p[i] = z[i];
+                        st_slab16p(s.AkW[col >> 6], row, col & 63, p);
                     }
                 }
                 warp_release(&s.bar_a);
@@ -626,17 +627,16 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                     dst_base = map_to_cta(smem_u32(p), owner);
                     dst_bar = map_to_cta(smem_u32(&s.bar_partK), owner);
                 }
-                uint32_t u[NB][16];
-#pragma unroll
-                for (int b = 0; b < NB; ++b) tmem_ld16(lane_addr + T_R1 + c0 + 16 * b, u[b]);
-                tmem_wait_ld();
 #pragma unroll
                 for (int b = 0; b < NB; ++b) {
+                    uint32_t u[16];
+                    tmem_ld16(lane_addr + T_R1 + c0 + 16 * b, u);
+                    tmem_wait_ld();
 #pragma unroll
                     for (int j = 0; j < 16; j += 4) {
                         const uint32_t dst = dst_base + stage_offset((uint32_t)((c0 + 16 * b + j) >> 2), srow);
-                        if (mine) st_cluster_v4_b32(dst, u[b][j], u[b][j + 1], u[b][j + 2], u[b][j + 3]);
-                        else st_async_v4(dst, u[b][j], u[b][j + 1], u[b][j + 2], u[b][j + 3], dst_bar);
+                        if (mine) st_cluster_v4_b32(dst, u[j], u[j + 1], u[j + 2], u[j + 3]);
+                        else st_async_v4(dst, u[j], u[j + 1], u[j + 2], u[j + 3], dst_bar);
                     }
                 }
                 // R1 may be overwritten by G3 once every warp has taken its rows
@@ -646,32 +646,27 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             };
             auto send_q = [&]() {
                 const bool mine = owner == me;
-                uint32_t u[NB][16];
+                const uint32_t own_base = smem_u32(s.A[1]) + 8192u;
+                const uint32_t dst_base = map_to_cta(smem_u32(s.Stage2) + slot * 4096u, owner);
+                const uint32_t dst_bar = map_to_cta(smem_u32(&s.bar_partQ), owner);
 #pragma unroll
-                for (int b = 0; b < NB; ++b) tmem_ld16(lane_addr + T_R1 + c0 + 16 * b, u[b]);
-                tmem_wait_ld();
-                if (mine) {
-                    const uint32_t dst_base = smem_u32(s.A[1]) + 8192u;
-#pragma unroll
-                    for (int b = 0; b < NB; ++b)
+                for (int b = 0; b < NB; ++b) {
+                    uint32_t u[16];
+                    tmem_ld16(lane_addr + T_R1 + c0 + 16 * b, u);
+                    tmem_wait_ld();
+                    if (mine) {
 #pragma unroll
                         for (int j = 0; j < 16; j += 4)
-                            st_cluster_v4_b32(dst_base + stage_offset((uint32_t)((c0 + 16 * b + j) >> 2), srow), u[b][j], u[b][j + 1],
-                                              u[b][j + 2], u[b][j + 3]);
-                } else {
-                    const uint32_t dst_base = map_to_cta(smem_u32(s.Stage2) + slot * 4096u, owner);
-                    const uint32_t dst_bar = map_to_cta(smem_u32(&s.bar_partQ), owner);
+                            st_cluster_v4_b32(own_base + stage_offset((uint32_t)((c0 + 16 * b + j) >> 2), srow), u[j], u[j + 1], u[j + 2], u[j + 3]);
+                    } else {
 #pragma unroll
-                    for (int b = 0; b < NB; ++b)
-#pragma unroll
-                        for (int j = 0; j < 16; j += 8) {
-                            const uint32_t c8 = (uint32_t)((c0 + 16 * b + j) >> 3);
-                            st_async_v4(dst_base + stage_offset_q(c8, srow),
-                                        pack_bf16(__uint_as_float(u[b][j]), __uint_as_float(u[b][j + 1])),
-                                        pack_bf16(__uint_as_float(u[b][j + 2]), __uint_as_float(u[b][j + 3])),
-                                        pack_bf16(__uint_as_float(u[b][j + 4]), __uint_as_float(u[b][j + 5])),
-                                        pack_bf16(__uint_as_float(u[b][j + 6]), __uint_as_float(u[b][j + 7])), dst_bar);
-                        }
+                        for (int j = 0; j < 16; j += 8)
+                            st_async_v4(dst_base + stage_offset_q((uint32_t)((c0 + 16 * b + j) >> 3), srow),
+                                        pack_bf16(__uint_as_float(u[j]), __uint_as_float(u[j + 1])),
+                                        pack_bf16(__uint_as_float(u[j + 2]), __uint_as_float(u[j + 3])),
+                                        pack_bf16(__uint_as_float(u[j + 4]), __uint_as_float(u[j + 5])),
+                                        pack_bf16(__uint_as_float(u[j + 6]), __uint_as_float(u[j + 7])), dst_bar);
+                    }
                 }
                 tc_fence_before_sync();
                 __syncwarp();
@@ -817,25 +812,22 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 PROF(7);
                 {
                     const float kw = sc.kW[row], km = sc.kM[row];
-                    uint32_t pa[NB][16], dg[NB][16];
 #pragma unroll
                     for (int b = 0; b < NB; ++b) {
-                        tmem_ld16(lane_addr + T_R1 + c0 + 16 * b, pa[b]);
-                        tmem_ld16(lane_addr + T_R0 + c0 + 16 * b, dg[b]);
-                    }
-                    tmem_wait_ld();
+                        uint32_t pa[16], dg[16];
+                        tmem_ld16(lane_addr + T_R1 + c0 + 16 * b, pa);
+                        tmem_ld16(lane_addr + T_R0 + c0 + 16 * b, dg);
+                        tmem_wait_ld();
+                        uint32_t p[8];
 #pragma unroll
-                    for (int b = 0; b < NB; ++b) {
-                        float pw[16], pm[16];
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const float pz = __uint_as_float(pa[b][j]) * __uint_as_float(dg[b][j]);
-                            pw[j] = kw * pz;
-                            pm[j] = km * pz;
-                        }
+                        for (int j = 0; j < 16; ++j) pa[j] = __float_as_uint(__uint_as_float(pa[j]) * __uint_as_float(dg[j]));  // pz
                         const int col = c0 + 16 * b;
-                        st_slab16(s.PzW[col >> 6], row, col & 63, pw);
-                        st_slab16(s.PzM[col >> 6], row, col & 63, pm);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) p[i] = pack_bf16(kw * __uint_as_float(pa[2 * i]), kw * __uint_as_float(pa[2 * i + 1]));
+                        st_slab16p(s.PzW[col >> 6], row, col & 63, p);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) p[i] = pack_bf16(km * __uint_as_float(pa[2 * i]), km * __uint_as_float(pa[2 * i + 1]));
+                        st_slab16p(s.PzM[col >> 6], row, col & 63, p);
                     }
                 }
                 warp_release(&s.bar_pz);
@@ -871,31 +863,30 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 #pragma unroll
                 for (int b = 0; b < NB; ++b) {
                     const int col = c0 + 16 * b;
-                    uint32_t wa[16], st[16];
-                    float wn[16];
+                    uint32_t wa[16];  // the new weights, in place: unscaled first, then pre-scaled for the next chunk
                     tmem_ld16(lane_addr + T_W1 + col, wa);
                     tmem_wait_ld();
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
-                        wn[j] = fmaf(cm, M1[16 * b + j], __uint_as_float(wa[j]));
-                        st[j] = __float_as_uint(NORM ? wn[j] : cwn * wn[j]);
-                        if (NORM) ss1 = fmaf(wn[j], wn[j], ss1);
+                        const float wn = fmaf(cm, M1[16 * b + j], __uint_as_float(wa[j]));
+                        wa[j] = __float_as_uint(wn);
+                        if (NORM) ss1 = fmaf(wn, wn, ss1);
                     }
-                    tmem_st16(lane_addr + T_W1 + col, st);
                     if (!NORM) {
-                        st_slab16(s.W1[col >> 6], row, col & 63, wn);
-                        if (real1 && col < de) {
-                            if (last) {
+                        uint32_t p[8];
 #pragma unroll
-                                for (int j = 0; j < 16; j += 4)
-                                    *reinterpret_cast<float4*>(a.W1_final + head + off0 + col + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
-                            } else if (save_ck) {
+                        for (int i = 0; i < 8; ++i) p[i] = pack_bf16(__uint_as_float(wa[2 * i]), __uint_as_float(wa[2 * i + 1]));
+                        st_slab16p(s.W1[col >> 6], row, col & 63, p);
+                        if (real1 && col < de && (last || save_ck)) {
+                            float* dst = (last ? a.W1_final + head : ckn) + off0 + col;
 #pragma unroll
-                                for (int j = 0; j < 16; j += 4)
-                                    *reinterpret_cast<float4*>(ckn + off0 + col + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
-                            }
+                            for (int j = 0; j < 16; j += 4)
+                                *reinterpret_cast<uint4*>(dst + j) = make_uint4(wa[j], wa[j + 1], wa[j + 2], wa[j + 3]);
                         }
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) wa[j] = __float_as_uint(cwn * __uint_as_float(wa[j]));
                     }
+                    tmem_st16(lane_addr + T_W1 + col, wa);
                 }
                 if (NORM) {
                     // row sums of squares: the four column-group warps of a row meet in shared memory (the kW pz tile is dead)
@@ -982,20 +973,39 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 #pragma unroll
                 for (int b = 0; b < NB; ++b) {
                     const int col = c0 + 16 * b;
-                    uint32_t wa[16], ma[16], st[16];
-                    float wn[16];
-                    tmem_ld16(lane_addr + T_W2 + col, wa);
-                    tmem_ld16(lane_addr + T_R1 + col, ma);
-                    tmem_wait_ld();
+                    {
+                        uint32_t wa[16];  // the new weights, in place: unscaled first, then pre-scaled for the next chunk
+                        tmem_ld16(lane_addr + T_W2 + col, wa);
+                        tmem_wait_ld();
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const float m0 = M2[16 * b + j];
-                        wn[j] = fmaf(cm, m0, __uint_as_float(wa[j]));
-                        M2[16 * b + j] = fmaf(cb, m0, __uint_as_float(ma[j]));
-                        st[j] = __float_as_uint(NORM ? wn[j] : cwn * wn[j]);
-                        if (NORM) ss2 = fmaf(wn[j], wn[j], ss2);
+                        for (int j = 0; j < 16; ++j) {
+                            const float wn = fmaf(cm, M2[16 * b + j], __uint_as_float(wa[j]));
+                            wa[j] = __float_as_uint(wn);
+                            if (NORM) ss2 = fmaf(wn, wn, ss2);
+                        }
+                        if (!NORM) {
+                            uint32_t p[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) p[i] = pack_bf16(__uint_as_float(wa[2 * i]), __uint_as_float(wa[2 * i + 1]));
+                            st_slab16p(s.W2[col >> 6], row, col & 63, p);
+                            if (real2 && (last || save_ck)) {
+                                float* dst = (last ? a.W2_final + head : ckn + dh) + off0 + col;
+#pragma unroll
+                                for (int j = 0; j < 16; j += 4)
+                                    *reinterpret_cast<uint4*>(dst + j) = make_uint4(wa[j], wa[j + 1], wa[j + 2], wa[j + 3]);
+                            }
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) wa[j] = __float_as_uint(cwn * __uint_as_float(wa[j]));
+                        }
+                        tmem_st16(lane_addr + T_W2 + col, wa);
                     }
-                    tmem_st16(lane_addr + T_W2 + col, st);
+                    {
+                        uint32_t ma[16];
+                        tmem_ld16(lane_addr + T_R1 + col, ma);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) M2[16 * b + j] = fmaf(cb, M2[16 * b + j], __uint_as_float(ma[j]));
+                    }
                     if (real2) {
                         if (last) {
 #pragma unroll
@@ -1008,20 +1018,6 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                             for (int j = 0; j < 16; j += 4)
                                 *reinterpret_cast<float4*>(ckn + 3 * dh + off0 + col + j) =
                                     make_float4(M2[16 * b + j], M2[16 * b + j + 1], M2[16 * b + j + 2], M2[16 * b + j + 3]);
-                        }
-                    }
-                    if (!NORM) {
-                        st_slab16(s.W2[col >> 6], row, col & 63, wn);
-                        if (real2) {
-                            if (last) {
-#pragma unroll
-                                for (int j = 0; j < 16; j += 4)
-                                    *reinterpret_cast<float4*>(a.W2_final + head + off0 + col + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
-                            } else if (save_ck) {
-#pragma unroll
-                                for (int j = 0; j < 16; j += 4)
-                                    *reinterpret_cast<float4*>(ckn + dh + off0 + col + j) = make_float4(wn[j], wn[j + 1], wn[j + 2], wn[j + 3]);
-                            }
                         }
                     }
                 }

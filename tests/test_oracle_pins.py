@@ -512,3 +512,72 @@ def test_prepare_oracle_matches_library_ops_and_autograd():
     # ranges the method relies on: 0 < eta < eta_base, 0 < beta < 1, 1 - eta_base alpha_base < gamma < 1
     assert (eta > 0).all() and (eta < eb).all() and (beta > 0).all() and (beta < 1).all()
     assert (gamma < 1).all() and (gamma > 1 - eb * ab).all()
+
+
+# ------------------------------------------------------------------ matrix form of the chunk (oracle/chunk_form.py)
+def test_chunk_matrix_form_equals_the_sequential_oracle():
+    """Algorithm 1 in matrix form (one inner forward/backward at the chunk-start weights, scalar kernels, Proposition 1)
+    against the token-by-token program, four chunks free-running: a pin of both (different language, different
+    formulation, same numbers)."""
+    from oracle import chunk_form
+    r = inputs.Recipe(B=1, H=2, L=28, d=8, h=16, C=8, kind=inputs.KIND_MLP, io="f32", seed=11, m_std=0.05, w_std=0.3)   # ragged last chunk
+    x = inputs.generate(r)
+    ref = oracle.forward(x["q"], x["k"], x["v"], x["eta"], x["beta"], x["gamma"], x["W"], x["M"], r.C, r.kind)
+    for n in range(2):
+        o, (W1, W2, M1, M2) = chunk_form.forward_mlp(x["q"][n], x["k"][n], x["v"][n], x["eta"][n], x["beta"][n], x["gamma"][n],
+                                                     x["W"][0][n], x["W"][1][n], x["M"][0][n], x["M"][1][n], r.C)
+        assert np.max(np.abs(o - ref["o"][n])) < 1e-10
+        for got, want in ((W1, ref["W"][0][n]), (W2, ref["W"][1][n]), (M1, ref["M"][0][n]), (M2, ref["M"][1][n])):
+            assert np.max(np.abs(got - want)) < 1e-10 * max(1.0, np.max(np.abs(want)))
+
+
+def test_closed_form_in_fp32_tracks_the_sequential_recurrence_in_fp32():
+    """The paper's numerical-equivalence experiment (Section 3.2; Appendix "Exactness"): closed form and token-wise
+    recurrence, both in fp32, over many chunks of 512 tokens under the paper's gate regime, stay at a relative l2
+    deviation of order 1e-6 in W_C and M_C (the paper reports < 2e-6 over 128 chunks).  Synthetic inputs, 16 chunks,
+    small d.  Two readings are checked: every chunk from the same start state (the two evaluations of one chunk), and
+    two free-running fp32 chains (where the map's own sensitivity adds to the rounding)."""
+    from oracle import chunk_form
+    r = inputs.paper_regime(inputs.Recipe(B=1, H=1, L=16 * 512, d=16, h=32, C=512, kind=inputs.KIND_MLP, io="f32", seed=5, m_std=0.002))
+    x = inputs.generate(r)
+    f32 = np.float32
+    q, k, v, eta, beta, gamma = (x[n][0] for n in ("q", "k", "v", "eta", "beta", "gamma"))
+    a = tuple(m[0].astype(f32) for m in (x["W"][0], x["W"][1], x["M"][0], x["M"][1]))   # closed-form chain
+    b = a                                                                                 # sequential chain
+
+    def rel(x_, y_):
+        return float(np.linalg.norm(x_.astype(np.float64) - y_.astype(np.float64)) / np.linalg.norm(y_.astype(np.float64)))
+
+    def sequential_chunk(state, sl):
+        _, _, pc = chunk_form.chunk_mlp(k[sl], q[sl], v[sl], eta[sl], beta[sl], gamma[sl], *state, dtype=f32)
+        G2 = [-np.outer(pc["Pu"][t], pc["A"][t]) for t in range(r.C)]
+        G1 = [-np.outer(pc["Pz"][t], k[sl][t].astype(f32)) for t in range(r.C)]
+        W1s, M1s = chunk_form.sequential_from_grads(state[0], state[2], G1, eta[sl], beta[sl], gamma[sl], f32)
+        W2s, M2s = chunk_form.sequential_from_grads(state[1], state[3], G2, eta[sl], beta[sl], gamma[sl], f32)
+        return (W1s, W2s, M1s, M2s)
+
+    worst_chunk = 0.0
+    for s in range(0, r.L, r.C):
+        sl = slice(s, s + r.C)
+        same_start = sequential_chunk(a, sl)
+        _, a, _ = chunk_form.chunk_mlp(k[sl], q[sl], v[sl], eta[sl], beta[sl], gamma[sl], *a, dtype=f32)
+        worst_chunk = max(worst_chunk, max(rel(x_, y_) for x_, y_ in zip(a, same_start)))
+        b = sequential_chunk(b, sl)
+    free = max(rel(x_, y_) for x_, y_ in zip(a, b))
+    print(f"fp32 closed form vs fp32 sequential, 16 chunks of 512: worst single chunk {worst_chunk:.2e}, free-running chains {free:.2e}")
+    assert worst_chunk < 3e-6
+    assert free < 5e-5
+
+
+def test_rounding_hooks_move_the_result_by_a_bf16_amount_and_nothing_else():
+    """Hooked mode = the same fp64 program with bf16 roundings at the declared points: it must stay within a few bf16
+    ulps of the unhooked result (and must differ from it)."""
+    from oracle import chunk_form
+    r = inputs.Recipe(B=1, H=1, L=64, d=32, h=64, C=64, kind=inputs.KIND_MLP, io="bf16", seed=2, m_std=0.002)
+    x = inputs.generate(r)
+    args = [x[n][0] for n in ("q", "k", "v", "eta", "beta", "gamma")] + [x["W"][0][0], x["W"][1][0], x["M"][0][0], x["M"][1][0], r.C]
+    o0, s0 = chunk_form.forward_mlp(*args)
+    o1, s1 = chunk_form.forward_mlp(*args, hooks=chunk_form.Hooks(gelu="erf"))
+    for got, want in [(o1, o0)] + list(zip(s1, s0)):
+        e = np.max(np.abs(got - want)) / np.max(np.abs(want))
+        assert 1e-5 < e < 2e-2, e
