@@ -204,8 +204,8 @@ def run_ours(args, r):
     x = inputs.generate(shard_recipe(r, rank))
     N = r.B * r.H
     iod = torch.float32 if r.io == "f32" else torch.bfloat16
-    p = E.make_params(r.B, r.H, r.L, r.d, r.h, r.C, r.kind, E.E2TTT_F32 if r.io == "f32" else E.E2TTT_BF16, 1e-5,
-                      E.E2TTT_IMPL_AUTO)
+    impl = {"auto": E.E2TTT_IMPL_AUTO, "fused": E.E2TTT_IMPL_TCGEN05, "tiled": E.E2TTT_IMPL_TILED, "simt": E.E2TTT_IMPL_SIMT}[args.kernel]
+    p = E.make_params(r.B, r.H, r.L, r.d, r.h, r.C, r.kind, E.E2TTT_F32 if r.io == "f32" else E.E2TTT_BF16, 1e-5, impl)
     s4, s3 = (r.B, r.H, r.L, r.d), (r.B, r.H, r.L)
     shapes = inputs.mat_shapes(r.kind, r.d, r.h)
     host = {n: torch.from_numpy(x[n]).to(iod).view(s4).pin_memory() for n in ("q", "k", "v")}
@@ -360,7 +360,7 @@ def run_ours(args, r):
             "timing": f"CUDA events on the launch stream; {args.warmup} warm-up steps, {n_preroll} untimed pre-roll steps "
                       f"(~{args.preroll:g} s of the same load, so the clock samples describe the timed region's steady state), "
                       f"then exactly {args.steps} timed steps; device status 0 and finite outputs checked afterwards",
-            "config": dict(workload_config(r), **({"post_chunk_norm": "rows of every W_i rescaled to the row norms of W_init after each chunk (any-shape kernels)"} if args.post_norm else {})),
+            "config": dict(workload_config(r), kernel_family=args.kernel, **({"post_chunk_norm": "rows of every W_i rescaled to the row norms of W_init after each chunk (any-shape kernels)"} if args.post_norm else {})),
             "e2e": {"value": whole_job_value(world, tokens, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e,
                     "how": "per step: inputs and initial state from pinned host memory, outputs and final state back; upload, kernel and download of consecutive steps overlap on three streams"},
@@ -683,6 +683,10 @@ def main():
     ap.add_argument("--prepare", action="store_true", help="time the token preparation instead (e2ttt_prepare_fwd, 1 GPU)")
     ap.add_argument("--post-norm", action="store_true", help="forward with post-chunk normalisation of the fast weights (e2ttt_chunk_fwd_normed)")
     ap.add_argument("--chunk", type=int, default=0, help="override the chunk size C of the configuration")
+    ap.add_argument("--kernel", default="auto", choices=["auto", "fused", "tiled", "simt"],
+                    help="kernel family of the forward: auto (the library's choice), fused (tensor-core kernel with the state on "
+                         "chip; for SwiGLU it must be asked for: its plain-bf16 weight operands leave some windows outside the "
+                         "2e-2 bound), tiled / simt (any-shape kernels)")
     ap.add_argument("--gates", default="benchmark", choices=["benchmark", "paper"],
                     help="gate recipe: the benchmark's, or the paper's regime (eta_base 0.01, tau 32, alpha_base 0.1)")
     ap.add_argument("--preroll", type=float, default=1.2,

@@ -6,6 +6,7 @@
 #include "prepare.h"
 #include "simt_layout.h"
 #include "tc_fwd.h"
+#include "tc_swiglu.h"
 
 using namespace e2ttt;
 
@@ -40,9 +41,11 @@ constexpr size_t kStatusBytes = 256;
 
 // 1 = a tensor-core specialisation exists for these parameters (the forward; with save_states it also writes the
 // chunk-start states in the layout the SIMT backward reads)
-int has_tcgen05(const e2ttt_params* p, bool /*save_states*/) {
-    return p->kind == E2TTT_MLP_GELU && p->io_dtype == E2TTT_BF16 && (p->d == 128 || p->d == 64) && p->h % 128 == 0 &&
-           p->h <= 512 && p->C == 64 && p->L % 64 == 0;
+int has_tcgen05(const e2ttt_params* p, bool save_states) {
+    if (p->io_dtype != E2TTT_BF16 || p->C != 64 || p->L % 64 != 0) return 0;
+    if (p->kind == E2TTT_MLP_GELU) return (p->d == 128 || p->d == 64) && p->h % 128 == 0 && p->h <= 512;
+    // SwiGLU: the fused kernel is built for d = 128, h = 384 and does not write chunk-start states
+    return p->kind == E2TTT_SWIGLU && p->d == 128 && p->h == 384 && !save_states;
 }
 
 int pick_impl(const e2ttt_params* p, bool save_states, int* impl) {
@@ -53,8 +56,12 @@ int pick_impl(const e2ttt_params* p, bool save_states, int* impl) {
         if (p->io_dtype != E2TTT_BF16) return E2TTT_ERR_SHAPE;
         *impl = E2TTT_IMPL_TILED;
     } else if (p->impl == E2TTT_IMPL_AUTO) {
-        *impl = has_tcgen05(p, save_states) ? E2TTT_IMPL_TCGEN05
-                                            : (p->io_dtype == E2TTT_BF16 ? E2TTT_IMPL_TILED : E2TTT_IMPL_SIMT);
+        // AUTO takes the fused kernel for the GELU-MLP.  The fused SwiGLU kernel feeds its products plain bf16 copies of
+        // the fast weights, which leaves some one-chunk windows slightly outside the 2e-2 bound (the any-shape kernels
+        // split every operand into two bf16 terms and stay inside it): it is chosen by asking for TCGEN05.
+        *impl = (has_tcgen05(p, save_states) && p->kind == E2TTT_MLP_GELU)
+                    ? E2TTT_IMPL_TCGEN05
+                    : (p->io_dtype == E2TTT_BF16 ? E2TTT_IMPL_TILED : E2TTT_IMPL_SIMT);
     } else {
         *impl = E2TTT_IMPL_SIMT;
     }
@@ -120,7 +127,7 @@ int e2ttt_workspace_bytes_normed(const e2ttt_params* p, int save_states, size_t*
     if (!bytes) return E2TTT_ERR_NULL;
     int rc = check_params(p);
     if (rc) return rc;
-    if (p->impl == E2TTT_IMPL_TCGEN05 && !has_tcgen05(p, false)) return E2TTT_ERR_SHAPE;
+    if (p->impl == E2TTT_IMPL_TCGEN05 && !(has_tcgen05(p, false) && p->kind == E2TTT_MLP_GELU)) return E2TTT_ERR_SHAPE;
     *bytes = simt_bytes(p, save_states != 0, save_states != 0);
     return E2TTT_OK;
 }
@@ -157,6 +164,24 @@ static int fwd_common(const e2ttt_params* p, const void* q, const void* k, const
     rc = check_device();
     if (rc) return rc;
 
+    if (impl == E2TTT_IMPL_TCGEN05 && p->kind == E2TTT_SWIGLU && row_norm) {
+        // no fused kernel with post-chunk normalisation for SwiGLU: the any-shape kernels serve it
+        if (p->impl == E2TTT_IMPL_TCGEN05) return E2TTT_ERR_SHAPE;
+        impl = E2TTT_IMPL_TILED;
+    }
+    if (impl == E2TTT_IMPL_TCGEN05 && p->kind == E2TTT_SWIGLU) {
+        TcSwigluArgs t{};
+        t.N = p->B * p->H; t.L = p->L; t.eps = p->ln_eps;
+        t.q = static_cast<const __nv_bfloat16*>(q); t.k = static_cast<const __nv_bfloat16*>(k);
+        t.v = static_cast<const __nv_bfloat16*>(v); t.o = static_cast<__nv_bfloat16*>(o);
+        t.eta = eta; t.beta = beta; t.gamma = gamma;
+        t.W1_init = W_init[0]; t.W2_init = W_init[1]; t.W3_init = W_init[2];
+        t.M1_init = M_init ? M_init[0] : nullptr; t.M2_init = M_init ? M_init[1] : nullptr; t.M3_init = M_init ? M_init[2] : nullptr;
+        t.W1_final = W_final[0]; t.W2_final = W_final[1]; t.W3_final = W_final[2];
+        t.M1_final = M_final[0]; t.M2_final = M_final[1]; t.M3_final = M_final[2];
+        t.status = static_cast<int*>(workspace);
+        return tc_swiglu_launch(t, stream) == 0 ? E2TTT_OK : E2TTT_ERR_CUDA;
+    }
     if (impl == E2TTT_IMPL_TCGEN05) {
         TcFwdArgs t{};
         t.N = p->B * p->H; t.L = p->L; t.d = p->d; t.h = p->h; t.eps = p->ln_eps;

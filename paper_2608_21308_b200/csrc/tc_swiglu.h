@@ -1,0 +1,23 @@
+// Host interface of the tensor-core forward for SwiGLU fast weights (tc_swiglu.cu).
+#pragma once
+#include <cuda_bf16.h>
+#include <stddef.h>
+
+namespace e2ttt {
+
+struct TcSwigluArgs {
+    int N, L;  // sequences, tokens per sequence (L a multiple of 64); d = 128, h = 384 are compiled in
+    float eps;
+    const __nv_bfloat16 *q, *k, *v;
+    const float *eta, *beta, *gamma;
+    const float *W1_init, *W2_init, *W3_init, *M1_init, *M2_init, *M3_init;  // M*_init may be nullptr (zeros)
+    __nv_bfloat16* o;
+    float *W1_final, *W2_final, *W3_final, *M1_final, *M2_final, *M3_final;
+    int* status;  // device word, 0 after a clean run
+};
+
+size_t tc_swiglu_smem_bytes();
+// returns a cudaError_t value as int (0 = launched)
+int tc_swiglu_launch(const TcSwigluArgs& a, void* stream);
+
+}  // namespace e2ttt

@@ -1,0 +1,91 @@
+"""Fused tensor-core forward for SwiGLU fast weights (d = 128, h = 384, C = 64, bf16; asked for with impl = TCGEN05)."""
+import numpy as np
+import pytest
+
+from paper_2608_21308_b200 import binding as E
+from paper_2608_21308_b200 import inputs
+from tests import util
+from tests.test_gpu_parity import TOL_BF16, check_forward
+
+pytestmark = pytest.mark.gpu
+SW = inputs.KIND_SWIGLU
+SHAPE = dict(d=128, h=384, C=64, kind=SW, io="bf16")
+NAMES = ["o", "W1", "W2", "W3", "M1", "M2", "M3"]
+
+
+def per_window_errors(got, ref):
+    """rows = windows, columns = NAMES: max|x - ref| / max|ref| of every tensor of every window."""
+    n = got["o"].shape[0]
+    out = np.zeros((n, len(NAMES)))
+    for w in range(n):
+        vals = [(got["o"][w], ref["o"][w])] + [(got["W"][i][w], ref["W"][i][w]) for i in range(3)] + \
+               [(got["M"][i][w], ref["M"][i][w]) for i in range(3)]
+        out[w] = [util.rel_err(a, b) for a, b in vals]
+    return out
+
+
+def test_fused_swiglu_windows_across_the_sequence_and_the_split_operand_kernels_beside_it():
+    """One-chunk windows started from the oracle's state at chunks 0, 1, 2, 3, 7, 15, 31, 63 of config 3, four heads.
+    The fused kernel rounds the fast-weight operands to plain bf16; SwiGLU is the badly conditioned network (a chunk
+    whose pre-norm outputs have a variance below the layer-norm epsilon amplifies every rounding), so its worst windows
+    are outside the 2e-2 bound (measured: 63 % of the windows inside, median 1.1e-2, worst 0.24) while the any-shape
+    kernels with two-term bf16 operands pass the bound on every window.  Both facts are asserted, and the distribution
+    is printed; this is why AUTO does not select the fused SwiGLU kernel."""
+    r = inputs.config(3, heads=[3, 21, 40, 62])
+    xw, ref = util.teacher_forced_windows_at(r, [0, 1, 2, 3, 7, 15, 31, 63])
+    fused, hd = util.gpu_forward(xw, impl=E.E2TTT_IMPL_TCGEN05, **SHAPE)
+    assert E.e2ttt_device_status(hd["ws"]) == 0 and hd["ws"].numel() == 256      # fused path: status block only
+    e = per_window_errors(fused, ref)
+    worst = e.max(axis=1)
+    print("fused SwiGLU, per tensor: median", dict(zip(NAMES, np.round(np.median(e, axis=0), 4))),
+          "worst", dict(zip(NAMES, np.round(e.max(axis=0), 4))))
+    print(f"fused SwiGLU: {np.mean(worst <= TOL_BF16):.2f} of the windows within {TOL_BF16}, median of the worst tensor "
+          f"{np.median(worst):.4f}, worst window {worst.max():.4f}")
+    chunks = [0, 1, 2, 3, 7, 15, 31, 63]
+    print("fused SwiGLU, worst tensor per start chunk (max over the 4 heads):",
+          {c: round(float(worst.reshape(4, len(chunks))[:, i].max()), 4) for i, c in enumerate(chunks)})
+    assert np.isfinite(e).all()
+    assert np.median(worst) <= TOL_BF16 and np.mean(worst <= TOL_BF16) >= 0.6 and worst.max() <= 0.5
+    tiled, _ = util.gpu_forward(xw, impl=E.E2TTT_IMPL_TILED, **SHAPE)
+    check_forward(tiled, ref, TOL_BF16, "any-shape kernels (two-term bf16 operands) on the same windows")
+
+
+def test_fused_swiglu_free_running_paper_regime_split_calls_and_repeatability():
+    """16 chunks free-running under the paper's gate regime (well conditioned) against the oracle; two calls of half the
+    length chain bitwise to the same result; a second run gives the same bits; AUTO keeps the any-shape kernels."""
+    r = inputs.paper_regime(inputs.Recipe(B=3, H=1, L=1024, d=128, h=384, C=64, kind=SW, io="bf16", seed=4, m_std=0.002))
+    x = inputs.generate(r)
+    ref = util.oracle_forward(x, 64, SW)
+    got, hd = util.gpu_forward(x, impl=E.E2TTT_IMPL_TCGEN05, **SHAPE)
+    assert E.e2ttt_device_status(hd["ws"]) == 0
+    errs = check_forward(got, ref, TOL_BF16, "fused SwiGLU, paper regime, 16 chunks free-running")
+    print("fused SwiGLU free-running", errs)
+    again, _ = util.gpu_forward(x, impl=E.E2TTT_IMPL_TCGEN05, **SHAPE)
+    assert np.array_equal(again["o"], got["o"]) and all(np.array_equal(a, b) for a, b in zip(again["W"] + again["M"], got["W"] + got["M"]))
+    half = r.L // 2
+    first = {n: (np.ascontiguousarray(v[:, :half]) if not isinstance(v, list) else v) for n, v in x.items()}
+    a, _ = util.gpu_forward(first, impl=E.E2TTT_IMPL_TCGEN05, **SHAPE)
+    rest = {n: (np.ascontiguousarray(v[:, half:]) if not isinstance(v, list) else v) for n, v in x.items()}
+    rest["W"], rest["M"] = a["W"], a["M"]
+    b, _ = util.gpu_forward(rest, impl=E.E2TTT_IMPL_TCGEN05, **SHAPE)
+    assert np.array_equal(np.concatenate([a["o"], b["o"]], 1), got["o"])
+    for i in range(3):
+        assert np.array_equal(b["W"][i], got["W"][i]) and np.array_equal(b["M"][i], got["M"][i])
+    _, hauto = util.gpu_forward(first, impl=E.E2TTT_IMPL_AUTO, **SHAPE)
+    assert hauto["ws"].numel() > 256                                             # AUTO: the any-shape kernels' workspace
+
+
+def test_fused_swiglu_null_momentum_many_sequences_and_other_shapes_are_refused():
+    r = inputs.config(3, heads=list(range(30)), L=128)
+    x = inputs.generate(r)
+    got, hd = util.gpu_forward(x, impl=E.E2TTT_IMPL_TCGEN05, use_M=False, **SHAPE)
+    assert E.e2ttt_device_status(hd["ws"]) == 0
+    first = {n: (np.ascontiguousarray(v[:, :64]) if not isinstance(v, list) else v) for n, v in x.items()}
+    ref = util.oracle_forward(first, 64, SW, use_M=False)
+    assert util.rel_err(got["o"][:, :64], ref["o"]) <= TOL_BF16                  # first chunk of 30 sequences
+    p = E.make_params(1, 1, 128, 128, 512, 64, E.E2TTT_SWIGLU, E.E2TTT_BF16, 1e-5, E.E2TTT_IMPL_TCGEN05)
+    with pytest.raises(E.E2TTTError):
+        E.e2ttt_workspace_bytes(p, 0)                                            # h = 512: no fused SwiGLU kernel
+    p = E.make_params(1, 1, 128, 128, 384, 64, E.E2TTT_SWIGLU, E.E2TTT_BF16, 1e-5, E.E2TTT_IMPL_TCGEN05)
+    with pytest.raises(E.E2TTTError):
+        E.e2ttt_workspace_bytes(p, 1)                                            # it does not save chunk-start states
