@@ -64,7 +64,11 @@ typedef enum { E2TTT_F32 = 0, E2TTT_BF16 = 1 } e2ttt_dtype;
  *   AUTO    : TCGEN05 where it serves (kind, io_dtype, d, h, C); else TILED for bf16 I/O and SIMT for
  *             fp32 I/O.  The backward has no fused kernel: AUTO and TCGEN05 mean TILED there.
  *             TCGEN05 serves today: GELU-MLP, bf16 I/O, C = 64, L a multiple of 64, d in {64, 128},
- *             h in {128, 256, 384, 512} (shapes below 128 x 512 run zero-padded in the same tiles).
+ *             h in {128, 256, 384, 512} (shapes below 128 x 512 run zero-padded in the same tiles); and the
+ *             SwiGLU forward at d = 128, h = 384, C = 64, bf16 I/O, without saved states or normalisation.
+ *             AUTO selects the fused kernel for the GELU-MLP only: the fused SwiGLU kernel gives its products
+ *             plain bf16 copies of the fast weights, which leaves some chunks outside the 2e-2 parity bound
+ *             (the any-shape kernels, with two-term bf16 operands, stay inside it); ask for it with TCGEN05.
  *   SIMT    : plain CUDA-core kernels for any shape.  With fp32 I/O they compute in fp64
  *             internally; with bf16 I/O in fp32.
  *   TCGEN05 : the fused kernel: bf16 operands on the 5th-generation tensor cores, fp32 accumulation
