@@ -88,6 +88,30 @@ def test_tc_free_running_64_chunks_paper_regime():
     print("64 chunks free-running", errs)
 
 
+def test_tc_error_growth_under_the_benchmark_gates_beside_the_fp32_noise_floor():
+    """Free-running under the BENCHMARK gates the chunk-to-chunk map amplifies any rounding (why configs 1-4 are compared
+    in windows).  The curve of the fused kernel's output error per chunk is printed beside the same curve for the
+    oracle's own formulas evaluated in fp32 (no bf16 anywhere): both grow at the map's rate, the kernel's from a
+    bf16-sized start, the fp32 run's from an fp32-sized one - the growth is the map's, not the kernel's."""
+    from oracle import chunk_form
+    n = 24
+    r = inputs.config(2, heads=[3], L=n * 64, m_std=0.002)
+    x = inputs.generate(r)
+    ref = util.oracle_forward(x, 64, MLP)
+    tc, hd = util.gpu_forward(x, impl=E.E2TTT_IMPL_TCGEN05, **SHAPE)
+    assert E.e2ttt_device_status(hd["ws"]) == 0
+    o32, _ = chunk_form.forward_mlp(x["q"][0], x["k"][0], x["v"][0], x["eta"][0], x["beta"][0], x["gamma"][0],
+                                    x["W"][0][0], x["W"][1][0], x["M"][0][0], x["M"][1][0], 64, dtype=np.float32)
+    cut = lambda a, c: a[64 * c:64 * c + 64]
+    gpu = [util.rel_err(cut(tc["o"][0], c), cut(ref["o"][0], c)) for c in range(n)]
+    f32 = [util.rel_err(cut(o32, c), cut(ref["o"][0], c)) for c in range(n)]
+    print("chunk           :", " ".join(f"{c:8d}" for c in range(0, n, 2)))
+    print("fused kernel    :", " ".join(f"{gpu[c]:8.1e}" for c in range(0, n, 2)))
+    print("fp32 formulas   :", " ".join(f"{f32[c]:8.1e}" for c in range(0, n, 2)))
+    assert gpu[0] <= TOL_BF16 and f32[0] <= 1e-5 and np.isfinite(gpu).all()
+    assert f32[n - 1] > 50 * f32[0]     # the map amplifies an fp32-sized perturbation too
+
+
 HEADS8 = [0, 9, 18, 27, 36, 45, 54, 63]
 
 
