@@ -392,7 +392,7 @@ def run_fwd_bwd(args, r):
     N = r.B * r.H
     iod = torch.float32 if r.io == "f32" else torch.bfloat16
     p = E.make_params(r.B, r.H, r.L, r.d, r.h, r.C, r.kind, E.E2TTT_F32 if r.io == "f32" else E.E2TTT_BF16, 1e-5,
-                      E.E2TTT_IMPL_AUTO)
+                      E.E2TTT_IMPL_AUTO, args.ckpt_every)
     s4, s3 = (r.B, r.H, r.L, r.d), (r.B, r.H, r.L)
     shapes = inputs.mat_shapes(r.kind, r.d, r.h)
     host = {n: torch.from_numpy(x[n]).to(iod).view(s4).pin_memory() for n in ("q", "k", "v", "d_o")}
@@ -446,13 +446,16 @@ def run_fwd_bwd(args, r):
     cfg = workload_config(r)
     cfg["workload"] = cfg["workload"].replace("e2ttt_chunk_fwd", "e2ttt_chunk_fwd(save_states) + e2ttt_chunk_bwd")
     cfg["path"] = "fused tensor-core forward writing chunk-start states where it serves the shape, any-shape backward with tcgen05 GEMMs"
+    cfg["ckpt_every"] = args.ckpt_every
+    cfg["workspace_bytes"] = ws.numel()
+    nseg = -(-(r.L // r.C) // args.ckpt_every) if args.ckpt_every >= 2 else 0
     line = {"metric": "e2ttt_layer_fwd_bwd_tokens_per_s", "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if r.io == "bf16" else "f64", "data": "synthetic", "config": cfg,
             "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": sum(v.numel() * v.element_size() for v in host.values()),
                     "d2h_bytes_per_step": sum(v.numel() * v.element_size() for v in hout), "ms_per_step": ms_e2e},
-            "gpu_launches": 2 * args.steps, "clocks": clocks,
+            "gpu_launches": (1 + max(1, 2 * nseg)) * args.steps, "clocks": clocks,
             "roofline": {"bound": "tensor", "achieved": flop / (ms * 1e-3) / 1e12, "peak": pk["bf16_tflops"],
                          "unit": "TFLOP/s", "frac": flop / (ms * 1e-3) / 1e12 / pk["bf16_tflops"], "traffic": None,
                          "peak_source": pk["_source"], "flop_per_step": flop}}
@@ -679,6 +682,9 @@ def main():
     ap.add_argument("--config", type=int, default=2, help="benchmark configuration index (default: the 1.3B-layer shape)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--backward", action="store_true", help="time forward + backward instead (1 GPU, GELU-MLP configs)")
+    ap.add_argument("--ckpt-every", type=int, default=0,
+                    help="with --backward: keep the state of every n-th chunk only and recompute n chunks at a time in the "
+                         "backward (0: every chunk's state is kept)")
     ap.add_argument("--decode", action="store_true", help="time the decode step instead: e2ttt_apply on one token per sequence (1 GPU)")
     ap.add_argument("--prepare", action="store_true", help="time the token preparation instead (e2ttt_prepare_fwd, 1 GPU)")
     ap.add_argument("--post-norm", action="store_true", help="forward with post-chunk normalisation of the fast weights (e2ttt_chunk_fwd_normed)")

@@ -103,6 +103,14 @@ typedef struct {
     int32_t io_dtype; /* e2ttt_dtype of q, k, v, o, d_o, dq, dk, dv */
     float ln_eps;     /* layer-norm epsilon (the paper gives none; 1e-5 is the usual default) */
     int32_t impl;     /* e2ttt_impl */
+    int32_t ckpt_every; /* which chunk-start states a forward with save_states keeps for the backward
+                         (Section 3.2 leaves the training-time memory plan to the implementation):
+                         0 or 1: the state of every chunk (2 * matrices * d * h values per chunk and sequence);
+                         n >= 2: only the states of chunks 0, n, 2n, ..; the backward then recomputes the states
+                         of n chunks at a time from the nearest checkpoint (one more any-shape forward over the
+                         sequence in exchange for ceil(L/C/n) + n + 2 stored states instead of L/C + 1).
+                         The forward and the backward of one training step must be given the same value.
+                         Not with the *_normed calls (E2TTT_ERR_SHAPE for n >= 2 there). */
 } e2ttt_params;
 
 /* Number of fast-weight matrices of a network kind (2 or 3); 0 for an unknown kind. */
@@ -113,8 +121,9 @@ E2TTT_API int e2ttt_num_matrices(int kind);
 E2TTT_API int e2ttt_matrix_shape(int kind, int d, int h, int i, int* rows, int* cols);
 
 /* Bytes of caller-provided device workspace a call with these parameters needs.
- * save_states != 0: the size for a forward that also records the chunk-start states, and for
- * the backward that consumes them.  `bytes` is a host pointer. */
+ * save_states != 0: the size for a forward that also records the chunk-start states (every chunk's, or
+ * the checkpoints p->ckpt_every selects plus room for one recomputed segment), and for the backward
+ * that consumes them.  `bytes` is a host pointer. */
 E2TTT_API int e2ttt_workspace_bytes(const e2ttt_params* p, int save_states, size_t* bytes);
 
 /* Forward over all chunks of all sequences (Algorithm 1 applied chunk after chunk, Section 3.2).

@@ -29,7 +29,8 @@ class e2ttt_gate_params(ctypes.Structure):
 class e2ttt_params(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("L", ctypes.c_int32), ("d", ctypes.c_int32),
                 ("h", ctypes.c_int32), ("C", ctypes.c_int32), ("kind", ctypes.c_int32),
-                ("io_dtype", ctypes.c_int32), ("ln_eps", ctypes.c_float), ("impl", ctypes.c_int32)]
+                ("io_dtype", ctypes.c_int32), ("ln_eps", ctypes.c_float), ("impl", ctypes.c_int32),
+                ("ckpt_every", ctypes.c_int32)]
 
 
 class E2TTTError(RuntimeError):
@@ -124,8 +125,9 @@ def e2ttt_workspace_bytes_normed(p: e2ttt_params, save_states: int) -> int:
     return int(n.value)
 
 
-def make_params(B, H, L, d, h, C, kind=E2TTT_MLP_GELU, io_dtype=E2TTT_F32, ln_eps=1e-5, impl=E2TTT_IMPL_AUTO):
-    return e2ttt_params(B, H, L, d, h, C, kind, io_dtype, ln_eps, impl)
+def make_params(B, H, L, d, h, C, kind=E2TTT_MLP_GELU, io_dtype=E2TTT_F32, ln_eps=1e-5, impl=E2TTT_IMPL_AUTO,
+                ckpt_every=0):
+    return e2ttt_params(B, H, L, d, h, C, kind, io_dtype, ln_eps, impl, ckpt_every)
 
 
 def _io_torch_dtype(p):

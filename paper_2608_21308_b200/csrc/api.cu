@@ -33,8 +33,12 @@ int check_params(const e2ttt_params* p) {
     if (p->C > kMaxChunk || p->d > kMaxD || p->h > kMaxH) return E2TTT_ERR_SHAPE;
     if ((int64_t)p->B * p->H > (int64_t)1 << 24) return E2TTT_ERR_SHAPE;
     if (!(p->ln_eps >= 0.0f)) return E2TTT_ERR_SHAPE;
+    if (p->ckpt_every < 0) return E2TTT_ERR_SHAPE;
     return E2TTT_OK;
 }
+
+// chunks per recomputed segment of the backward; 0 = every chunk's state is kept
+int segment_chunks(const e2ttt_params* p) { return p->ckpt_every >= 2 ? p->ckpt_every : 0; }
 
 // Every workspace starts with a status block: word 0 is the device status of the last launch that used it.
 constexpr size_t kStatusBytes = 256;
@@ -68,9 +72,9 @@ int pick_impl(const e2ttt_params* p, bool save_states, int* impl) {
     return E2TTT_OK;
 }
 
-size_t simt_bytes(const e2ttt_params* p, bool save_states, bool backward) {
+size_t simt_bytes(const e2ttt_params* p, bool save_states, bool backward, bool normed) {
     const int nchunks = (p->L + p->C - 1) / p->C;
-    SimtLayout l = simt_layout(p->d, p->h, p->C, nmat_of(p->kind), nchunks, save_states, backward);
+    SimtLayout l = simt_layout(p->d, p->h, p->C, nmat_of(p->kind), nchunks, save_states, backward, normed ? 0 : segment_chunks(p));
     const size_t elem = (p->io_dtype == E2TTT_F32) ? sizeof(double) : sizeof(float);
     return kStatusBytes + l.per_seq * elem * (size_t)p->B * p->H;
 }
@@ -119,7 +123,7 @@ int e2ttt_workspace_bytes(const e2ttt_params* p, int save_states, size_t* bytes)
     if (rc) return rc;
     // fused tensor-core path: all state lives on chip, only the status block is needed.
     // any-shape kernels: with saved states the same buffer serves the backward, which needs the larger layout.
-    *bytes = (impl == E2TTT_IMPL_TCGEN05 && !save_states) ? kStatusBytes : simt_bytes(p, save_states != 0, save_states != 0);
+    *bytes = (impl == E2TTT_IMPL_TCGEN05 && !save_states) ? kStatusBytes : simt_bytes(p, save_states != 0, save_states != 0, false);
     return E2TTT_OK;
 }
 
@@ -128,7 +132,8 @@ int e2ttt_workspace_bytes_normed(const e2ttt_params* p, int save_states, size_t*
     int rc = check_params(p);
     if (rc) return rc;
     if (p->impl == E2TTT_IMPL_TCGEN05 && !(has_tcgen05(p, false) && p->kind == E2TTT_MLP_GELU)) return E2TTT_ERR_SHAPE;
-    *bytes = simt_bytes(p, save_states != 0, save_states != 0);
+    if (segment_chunks(p)) return E2TTT_ERR_SHAPE;
+    *bytes = simt_bytes(p, save_states != 0, save_states != 0, true);
     return E2TTT_OK;
 }
 
@@ -151,10 +156,10 @@ static int fwd_common(const e2ttt_params* p, const void* q, const void* k, const
     if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(o, 16)) return E2TTT_ERR_ALIGN;
     size_t need = 0;
     if (row_norm) {
-        if (!(norm_eps >= 0.0f)) return E2TTT_ERR_SHAPE;
+        if (!(norm_eps >= 0.0f) || segment_chunks(p)) return E2TTT_ERR_SHAPE;
         for (int i = 0; i < nmat; ++i)
             if (!row_norm[i]) return E2TTT_ERR_NULL;
-        need = simt_bytes(p, save_states != 0, save_states != 0);  // the size e2ttt_workspace_bytes_normed reports
+        need = simt_bytes(p, save_states != 0, save_states != 0, true);  // the size e2ttt_workspace_bytes_normed reports
     } else {
         rc = e2ttt_workspace_bytes(p, save_states, &need);
         if (rc) return rc;
@@ -194,9 +199,11 @@ static int fwd_common(const e2ttt_params* p, const void* q, const void* k, const
         t.status = static_cast<int*>(workspace);
         if (row_norm) { t.norm1 = row_norm[0]; t.norm2 = row_norm[1]; t.norm_eps = norm_eps; }
         if (save_states) {
-            const SimtLayout lay = simt_layout(p->d, p->h, p->C, nmat, p->L / p->C, true, true);
-            t.ckpt = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBytes) + lay.ckpt;
+            const int seg = row_norm ? 0 : segment_chunks(p);
+            const SimtLayout lay = simt_layout(p->d, p->h, p->C, nmat, p->L / p->C, true, true, seg);
+            t.ckpt = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBytes) + (seg ? lay.cck : lay.ckpt);
             t.ckpt_seq_stride = lay.per_seq;
+            t.ckpt_every = seg;
             t.rown = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBytes) + lay.rown;
         }
         return tc_fwd_launch(t, stream) == 0 ? E2TTT_OK : E2TTT_ERR_CUDA;
@@ -212,7 +219,9 @@ static int fwd_common(const e2ttt_params* p, const void* q, const void* k, const
     a.cl = simt_cluster_size(a.N);
     a.tc = impl == E2TTT_IMPL_TILED;
     a.status = static_cast<int*>(workspace);
-    a.save_states = save_states != 0;
+    const int seg = row_norm ? 0 : segment_chunks(p);
+    a.save_states = save_states ? (seg ? 2 : 1) : 0;
+    a.Ls = p->L; a.init_slot = -1;
     a.eps = p->ln_eps;
     a.q = q; a.k = k; a.v = v; a.eta = eta; a.beta = beta; a.gamma = gamma; a.o = o;
     a.ws = static_cast<char*>(workspace) + kStatusBytes;
@@ -224,7 +233,7 @@ static int fwd_common(const e2ttt_params* p, const void* q, const void* k, const
         a.row_norm[i] = row_norm ? row_norm[i] : nullptr;
     }
     a.norm_eps = norm_eps;
-    a.lay = simt_layout(p->d, p->h, p->C, nmat, a.nchunks, a.save_states, a.save_states);
+    a.lay = simt_layout(p->d, p->h, p->C, nmat, a.nchunks, save_states != 0, save_states != 0, seg);
     return simt_fwd_launch(a, p->kind, p->io_dtype, stream) == 0 ? E2TTT_OK : E2TTT_ERR_CUDA;
 }
 
@@ -269,37 +278,44 @@ static int bwd_common(const e2ttt_params* p, const void* q, const void* k, const
     rc = pick_impl(p, true, &impl);
     if (rc) return rc;
     if (row_norm) {
-        if (!(norm_eps >= 0.0f)) return E2TTT_ERR_SHAPE;
+        if (!(norm_eps >= 0.0f) || segment_chunks(p)) return E2TTT_ERR_SHAPE;
         for (int i = 0; i < nmat; ++i)
             if (!row_norm[i]) return E2TTT_ERR_NULL;
     }
     if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(d_o, 16) || !aligned(dq, 16) ||
         !aligned(dk, 16) || !aligned(dv, 16))
         return E2TTT_ERR_ALIGN;
-    size_t need = 0;
-    rc = e2ttt_workspace_bytes(p, 1, &need);
-    if (rc) return rc;
+    const size_t need = simt_bytes(p, true, true, row_norm != nullptr);
     if (!workspace || workspace_bytes < need) return E2TTT_ERR_WORKSPACE;
     if (!aligned(workspace, 256)) return E2TTT_ERR_ALIGN;
     rc = check_device();
     if (rc) return rc;
 
     const int nchunks = (p->L + p->C - 1) / p->C;
-    const SimtLayout lay = simt_layout(p->d, p->h, p->C, nmat, nchunks, true, true);
+    const int seg = row_norm ? 0 : segment_chunks(p);
+    const SimtLayout lay = simt_layout(p->d, p->h, p->C, nmat, nchunks, true, true, seg);
     void* ws_data = static_cast<char*>(workspace) + kStatusBytes;
     if (cudaMemsetAsync(workspace, 0, sizeof(int), reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) {
         (void)cudaGetLastError();
         return E2TTT_ERR_CUDA;
     }
-    if (!states_saved) {
-        // recompute the chunk-start states: a forward whose outputs and final states land in scratch slots
-        // that the reverse sweep overwrites later (the adjoint carries T, S and the accumulators Wb)
+    // A forward that only records chunk-start states: outputs and final states are not written.
+    //   first_chunk, n  : the chunks it covers;  mode 1: every chunk's state -> lay.ckpt, 2: checkpoints -> lay.cck
+    //   init_slot       : -1 = start from W_init / M_init, else from checkpoint init_slot
+    auto recompute = [&](int first_chunk, int n, int mode, int init_slot) -> int {
+        const size_t t0 = (size_t)first_chunk * p->C;
+        const size_t esz = p->io_dtype == E2TTT_F32 ? 4 : 2;
         SimtFwdArgs f{};
-        f.N = p->B * p->H; f.L = p->L; f.d = p->d; f.h = p->h; f.C = p->C; f.nchunks = nchunks;
-        f.save_states = 1; f.eps = p->ln_eps; f.cl = simt_cluster_size(f.N);
+        f.N = p->B * p->H; f.d = p->d; f.h = p->h; f.C = p->C; f.nchunks = n;
+        f.L = (int)((size_t)p->L - t0 < (size_t)n * p->C ? (size_t)p->L - t0 : (size_t)n * p->C);
+        f.Ls = p->L; f.init_slot = init_slot;
+        f.save_states = mode; f.eps = p->ln_eps; f.cl = simt_cluster_size(f.N);
         f.tc = impl != E2TTT_IMPL_SIMT; f.status = static_cast<int*>(workspace);
-        f.q = q; f.k = k; f.v = v; f.eta = eta; f.beta = beta; f.gamma = gamma; f.ws = ws_data; f.lay = lay;
-        f.o = nullptr; // outputs are not needed
+        f.q = static_cast<const char*>(q) + t0 * p->d * esz;
+        f.k = static_cast<const char*>(k) + t0 * p->d * esz;
+        f.v = static_cast<const char*>(v) + t0 * p->d * esz;
+        f.eta = eta + t0; f.beta = beta + t0; f.gamma = gamma + t0; f.ws = ws_data; f.lay = lay;
+        f.o = nullptr;
         for (int i = 0; i < nmat; ++i) {
             f.W_init[i] = W_init[i];
             f.M_init[i] = M_init ? M_init[i] : nullptr;
@@ -308,25 +324,54 @@ static int bwd_common(const e2ttt_params* p, const void* q, const void* k, const
             f.row_norm[i] = row_norm ? row_norm[i] : nullptr;
         }
         f.norm_eps = norm_eps;
-        if (simt_fwd_launch(f, p->kind, p->io_dtype, stream) != 0) return E2TTT_ERR_CUDA;
+        return simt_fwd_launch(f, p->kind, p->io_dtype, stream);
+    };
+    // The reverse sweep over chunks [first_chunk, first_chunk + n), whose start states sit in lay.ckpt slots 0 .. n-1.
+    auto reverse = [&](int first_chunk, int n, bool carry_in, bool carry_out) -> int {
+        const size_t t0 = (size_t)first_chunk * p->C;
+        const size_t esz = p->io_dtype == E2TTT_F32 ? 4 : 2;
+        const size_t tok = t0 * p->d * esz;
+        SimtBwdArgs b{};
+        b.N = p->B * p->H; b.d = p->d; b.h = p->h; b.C = p->C; b.nchunks = n; b.eps = p->ln_eps;
+        b.L = (int)((size_t)p->L - t0 < (size_t)n * p->C ? (size_t)p->L - t0 : (size_t)n * p->C);
+        b.Ls = p->L; b.carry_in = carry_in; b.carry_out = carry_out;
+        b.cl = simt_cluster_size(b.N);
+        b.tc = impl != E2TTT_IMPL_SIMT; b.status = static_cast<int*>(workspace);
+        b.q = static_cast<const char*>(q) + tok; b.k = static_cast<const char*>(k) + tok;
+        b.v = static_cast<const char*>(v) + tok; b.d_o = static_cast<const char*>(d_o) + tok;
+        b.eta = eta + t0; b.beta = beta + t0; b.gamma = gamma + t0;
+        b.dq = static_cast<char*>(dq) + tok; b.dk = static_cast<char*>(dk) + tok; b.dv = static_cast<char*>(dv) + tok;
+        b.d_eta = d_eta + t0; b.d_beta = d_beta + t0; b.d_gamma = d_gamma + t0;
+        b.ws = ws_data; b.lay = lay;
+        for (int i = 0; i < nmat; ++i) {
+            b.dW_final[i] = dW_final ? dW_final[i] : nullptr;
+            b.dM_final[i] = dM_final ? dM_final[i] : nullptr;
+            b.dW_init[i] = dW_init[i];
+            b.dM_init[i] = dM_init[i];
+            b.row_norm[i] = row_norm ? row_norm[i] : nullptr;
+            b.d_row_norm[i] = (row_norm && d_row_norm) ? d_row_norm[i] : nullptr;
+        }
+        b.norm_eps = norm_eps;
+        return simt_bwd_launch(b, p->kind, p->io_dtype, stream);
+    };
+
+    if (seg == 0) {
+        // every chunk's start state is in the workspace, or is recomputed into it by one forward
+        if (!states_saved && recompute(0, nchunks, 1, -1) != 0) return E2TTT_ERR_CUDA;
+        return reverse(0, nchunks, false, false) == 0 ? E2TTT_OK : E2TTT_ERR_CUDA;
     }
-    SimtBwdArgs b{};
-    b.N = p->B * p->H; b.L = p->L; b.d = p->d; b.h = p->h; b.C = p->C; b.nchunks = nchunks; b.eps = p->ln_eps;
-    b.cl = simt_cluster_size(b.N);
-    b.tc = impl != E2TTT_IMPL_SIMT; b.status = static_cast<int*>(workspace);
-    b.q = q; b.k = k; b.v = v; b.d_o = d_o; b.eta = eta; b.beta = beta; b.gamma = gamma;
-    b.dq = dq; b.dk = dk; b.dv = dv; b.d_eta = d_eta; b.d_beta = d_beta; b.d_gamma = d_gamma;
-    b.ws = ws_data; b.lay = lay;
-    for (int i = 0; i < nmat; ++i) {
-        b.dW_final[i] = dW_final ? dW_final[i] : nullptr;
-        b.dM_final[i] = dM_final ? dM_final[i] : nullptr;
-        b.dW_init[i] = dW_init[i];
-        b.dM_init[i] = dM_init[i];
-        b.row_norm[i] = row_norm ? row_norm[i] : nullptr;
-        b.d_row_norm[i] = (row_norm && d_row_norm) ? d_row_norm[i] : nullptr;
+    // checkpoints every seg chunks: the segments are walked from the last to the first; each one gets the start
+    // states of its chunks recomputed from its checkpoint, then its reverse sweep.  The adjoints of the state
+    // (and nothing else) pass from one launch to the next, in the workspace.
+    if (!states_saved && recompute(0, nchunks, 2, -1) != 0) return E2TTT_ERR_CUDA;
+    const int nseg = (nchunks + seg - 1) / seg;
+    for (int sgi = nseg - 1; sgi >= 0; --sgi) {
+        const int first = sgi * seg;
+        const int n = nchunks - first < seg ? nchunks - first : seg;
+        if (recompute(first, n, 1, sgi) != 0) return E2TTT_ERR_CUDA;
+        if (reverse(first, n, sgi != nseg - 1, sgi != 0) != 0) return E2TTT_ERR_CUDA;
     }
-    b.norm_eps = norm_eps;
-    return simt_bwd_launch(b, p->kind, p->io_dtype, stream) == 0 ? E2TTT_OK : E2TTT_ERR_CUDA;
+    return E2TTT_OK;
 }
 
 int e2ttt_chunk_bwd(const e2ttt_params* p, const void* q, const void* k, const void* v, const float* eta,
@@ -451,6 +496,6 @@ const char* e2ttt_status_string(int status) {
     }
 }
 
-int e2ttt_version(void) { return 100; }
+int e2ttt_version(void) { return 101; }
 
 }  // extern "C"

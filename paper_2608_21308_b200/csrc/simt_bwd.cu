@@ -81,19 +81,19 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_ke
     const SimtLayout& lay = a.lay;
     Real* ws = reinterpret_cast<Real*>(a.ws) + (size_t)seq * lay.per_seq;
     G.set_scratch(ws + lay.splitk);
-    const IO* q = reinterpret_cast<const IO*>(a.q) + (size_t)seq * L * d;
-    const IO* k = reinterpret_cast<const IO*>(a.k) + (size_t)seq * L * d;
-    const IO* v = reinterpret_cast<const IO*>(a.v) + (size_t)seq * L * d;
-    const IO* d_o = reinterpret_cast<const IO*>(a.d_o) + (size_t)seq * L * d;
-    IO* dq = reinterpret_cast<IO*>(a.dq) + (size_t)seq * L * d;
-    IO* dk = reinterpret_cast<IO*>(a.dk) + (size_t)seq * L * d;
-    IO* dv = reinterpret_cast<IO*>(a.dv) + (size_t)seq * L * d;
-    const float* eta = a.eta + (size_t)seq * L;
-    const float* beta = a.beta + (size_t)seq * L;
-    const float* gamma = a.gamma + (size_t)seq * L;
-    float* d_eta = a.d_eta + (size_t)seq * L;
-    float* d_beta = a.d_beta + (size_t)seq * L;
-    float* d_gamma = a.d_gamma + (size_t)seq * L;
+    const IO* q = reinterpret_cast<const IO*>(a.q) + (size_t)seq * a.Ls * d;
+    const IO* k = reinterpret_cast<const IO*>(a.k) + (size_t)seq * a.Ls * d;
+    const IO* v = reinterpret_cast<const IO*>(a.v) + (size_t)seq * a.Ls * d;
+    const IO* d_o = reinterpret_cast<const IO*>(a.d_o) + (size_t)seq * a.Ls * d;
+    IO* dq = reinterpret_cast<IO*>(a.dq) + (size_t)seq * a.Ls * d;
+    IO* dk = reinterpret_cast<IO*>(a.dk) + (size_t)seq * a.Ls * d;
+    IO* dv = reinterpret_cast<IO*>(a.dv) + (size_t)seq * a.Ls * d;
+    const float* eta = a.eta + (size_t)seq * a.Ls;
+    const float* beta = a.beta + (size_t)seq * a.Ls;
+    const float* gamma = a.gamma + (size_t)seq * a.Ls;
+    float* d_eta = a.d_eta + (size_t)seq * a.Ls;
+    float* d_beta = a.d_beta + (size_t)seq * a.Ls;
+    float* d_gamma = a.d_gamma + (size_t)seq * a.Ls;
     const Real eps = (Real)a.eps;
 
     Real *T[NMAT], *S[NMAT], *Wb[NMAT];
@@ -102,6 +102,7 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_ke
         T[i] = ws + lay.T[i]; S[i] = ws + lay.S[i]; Wb[i] = ws + lay.Wb[i];
         const float* tf = a.dW_final[i] ? a.dW_final[i] + (size_t)seq * dh : nullptr;
         const float* sf = a.dM_final[i] ? a.dM_final[i] + (size_t)seq * dh : nullptr;
+        if (a.carry_in) continue;  // a later segment's launch left them in place
         for (size_t e = tid + (size_t)rank * NT; e < dh; e += (size_t)NT * CL) {
             T[i][e] = tf ? (Real)tf[e] : (Real)0;
             S[i][e] = sf ? (Real)sf[e] : (Real)0;
@@ -567,6 +568,7 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_bwd_ke
 
 #pragma unroll
     for (int i = 0; i < NMAT; ++i) {
+        if (a.carry_out) break;  // the launch for the segment before this one picks T, S up from the workspace
         float* wf = a.dW_init[i] + (size_t)seq * dh;
         float* mf = a.dM_init[i] + (size_t)seq * dh;
         for (size_t e = tid + (size_t)rank * NT; e < dh; e += (size_t)NT * CL) {

@@ -53,13 +53,13 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_fwd_ke
     const SimtLayout& lay = a.lay;
     Real* ws = reinterpret_cast<Real*>(a.ws) + (size_t)seq * lay.per_seq;
     G.set_scratch(ws + lay.splitk);
-    const IO* q = reinterpret_cast<const IO*>(a.q) + (size_t)seq * L * d;
-    const IO* k = reinterpret_cast<const IO*>(a.k) + (size_t)seq * L * d;
-    const IO* v = reinterpret_cast<const IO*>(a.v) + (size_t)seq * L * d;
-    IO* o = reinterpret_cast<IO*>(a.o) + (size_t)seq * L * d;
-    const float* eta = a.eta + (size_t)seq * L;
-    const float* beta = a.beta + (size_t)seq * L;
-    const float* gamma = a.gamma + (size_t)seq * L;
+    const IO* q = reinterpret_cast<const IO*>(a.q) + (size_t)seq * a.Ls * d;
+    const IO* k = reinterpret_cast<const IO*>(a.k) + (size_t)seq * a.Ls * d;
+    const IO* v = reinterpret_cast<const IO*>(a.v) + (size_t)seq * a.Ls * d;
+    IO* o = reinterpret_cast<IO*>(a.o) + (size_t)seq * a.Ls * d;
+    const float* eta = a.eta + (size_t)seq * a.Ls;
+    const float* beta = a.beta + (size_t)seq * a.Ls;
+    const float* gamma = a.gamma + (size_t)seq * a.Ls;
     const Real eps = (Real)a.eps;
 
     Real* W[NMAT];
@@ -68,12 +68,19 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_fwd_ke
     for (int i = 0; i < NMAT; ++i) {
         W[i] = ws + lay.W[i];
         M[i] = ws + lay.M[i];
-        const float* wi = a.W_init[i] + (size_t)seq * dh;
-        const float* mi = a.M_init[i] ? a.M_init[i] + (size_t)seq * dh : nullptr;
         struct WM { Real w, m; };
-        batched_for<8>(tid + (size_t)rank * NT, dh, (size_t)NT * CL,
-                       [&](size_t e) { return WM{(Real)wi[e], mi ? (Real)mi[e] : (Real)0}; },
-                       [&](size_t e, const WM& x) { W[i][e] = x.w; M[i][e] = x.m; });
+        if (a.init_slot >= 0) {  // a segment of the backward's recomputation: start from a checkpoint
+            const Real* ck = ws + lay.cck + (size_t)a.init_slot * 2 * NMAT * dh;
+            batched_for<8>(tid + (size_t)rank * NT, dh, (size_t)NT * CL,
+                           [&](size_t e) { return WM{ck[(size_t)i * dh + e], ck[(size_t)(NMAT + i) * dh + e]}; },
+                           [&](size_t e, const WM& x) { W[i][e] = x.w; M[i][e] = x.m; });
+        } else {
+            const float* wi = a.W_init[i] + (size_t)seq * dh;
+            const float* mi = a.M_init[i] ? a.M_init[i] + (size_t)seq * dh : nullptr;
+            batched_for<8>(tid + (size_t)rank * NT, dh, (size_t)NT * CL,
+                           [&](size_t e) { return WM{(Real)wi[e], mi ? (Real)mi[e] : (Real)0}; },
+                           [&](size_t e, const WM& x) { W[i][e] = x.w; M[i][e] = x.m; });
+        }
     }
     Real* Z1 = ws + lay.Z1;
     Real* Z2 = ws + lay.Z2;
@@ -94,8 +101,9 @@ __global__ void __launch_bounds__(TC ? kTgThreads : kSimtThreads, 1) simt_fwd_ke
         SPROF(0);
         // Algorithm 1 line 2: scalar kernels and carries
         if (warp == 0) chunk_scalars_warp<Real>(eta + s, beta + s, gamma + s, len, &sc);
-        if (a.save_states) {
-            Real* ck = ws + lay.ckpt + (size_t)c * 2 * NMAT * dh;
+        if (a.save_states == 1 || (a.save_states == 2 && c % lay.seg == 0)) {
+            Real* ck = a.save_states == 1 ? ws + lay.ckpt + (size_t)c * 2 * NMAT * dh
+                                          : ws + lay.cck + (size_t)(c / lay.seg) * 2 * NMAT * dh;
 #pragma unroll
             for (int i = 0; i < NMAT; ++i) {
                 struct WM { Real w, m; };

@@ -20,11 +20,14 @@ struct SimtLayout {
     size_t kWb, kMb;     // adjoints of the scalar kernels, one per token of the chunk
     size_t splitk;       // split-K partial sums of the tensor-core GEMM engine (2 * 8 * 128 * 64 elements)
     size_t rown;         // [nchunks][3][max(d,h)] row norms of the chunk-end weights before their normalisation
-    size_t ckpt;         // [nchunks + 1][2][nmat][d*h] chunk-start (W, M) and, last, the final state; when states are saved
+    size_t ckpt;         // [nchunks + 1][2][nmat][d*h] chunk-start (W, M) and, last, the final state; when states are saved.
+                         // With seg > 0: [seg + 1] slots, the chunk-start states of ONE segment (recomputed by the backward)
+    size_t cck;          // seg > 0: [nseg + 1][2][nmat][d*h] chunk-start states of every seg-th chunk (the checkpoints)
+    int seg;             // chunks per segment (e2ttt_params.ckpt_every >= 2); 0 = the state of every chunk is kept
     size_t per_seq;      // elements per sequence
 };
 
-inline SimtLayout simt_layout(int d, int h, int C, int nmat, int nchunks, bool save_states, bool backward) {
+inline SimtLayout simt_layout(int d, int h, int C, int nmat, int nchunks, bool save_states, bool backward, int seg = 0) {
     SimtLayout l{};
     size_t o = 0;
     const size_t dh = (size_t)d * h;
@@ -49,13 +52,24 @@ inline SimtLayout simt_layout(int d, int h, int C, int nmat, int nchunks, bool s
     }
     l.splitk = take((size_t)2 * 8 * 128 * 64);
     l.rown = take(save_states ? (size_t)nchunks * 3 * (size_t)(d > h ? d : h) : 0);
-    l.ckpt = take(save_states ? (size_t)(nchunks + 1) * 2 * nmat * dh : 0);
+    l.seg = save_states ? seg : 0;
+    if (l.seg > 0) {
+        l.ckpt = take((size_t)(l.seg + 1) * 2 * nmat * dh);
+        l.cck = take((size_t)((nchunks + l.seg - 1) / l.seg + 1) * 2 * nmat * dh);
+    } else {
+        l.ckpt = take(save_states ? (size_t)(nchunks + 1) * 2 * nmat * dh : 0);
+        l.cck = 0;
+    }
     l.per_seq = o;
     return l;
 }
 
 struct SimtFwdArgs {
-    int N, L, d, h, C, nchunks, save_states;
+    int N, L, d, h, C, nchunks;
+    int save_states;  // 0: none; 1: the start state of every chunk -> lay.ckpt; 2: of every lay.seg-th chunk -> lay.cck
+    int Ls;           // tokens between two sequences in q, k, v, o and the gates (L for a whole-sequence call; a segment
+                      // call passes pointers to its first token and the full length here)
+    int init_slot;    // >= 0: start from checkpoint slot init_slot of lay.cck instead of W_init / M_init; -1 otherwise
     int cl;  // CTAs per sequence (cluster size), chosen by the launcher
     int tc;  // GEMMs on the tensor cores with bf16 operands (bf16 I/O only) instead of fp32 FMAs
     int* status;  // device status word of the call (bounded waits report here)
@@ -75,6 +89,10 @@ struct SimtFwdArgs {
 
 struct SimtBwdArgs {
     int N, L, d, h, C, nchunks;
+    int Ls;           // tokens between two sequences in the token tensors (see SimtFwdArgs)
+    int carry_in;     // 1: the adjoints T, S of the chunk-end state are already in the workspace (left there by the launch
+                      // for the next segment); 0: read them from dW_final / dM_final
+    int carry_out;    // 1: leave T, S in the workspace for the previous segment's launch; 0: write dW_init / dM_init
     int cl;  // CTAs per sequence (cluster size), chosen by the launcher
     int tc;  // GEMMs on the tensor cores with bf16 operands (bf16 I/O only) instead of fp32 FMAs
     int* status;  // device status word of the call (bounded waits report here)

@@ -734,8 +734,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             const float cwn = last ? 1.0f : s.sc[(r + 1) & 1].cw;
             const size_t head = (size_t)seq * dh;
             // slot of the state after this chunk in the saved states (the slot after the last chunk is the final state)
-            float* ckn = a.ckpt ? a.ckpt + (size_t)seq * a.ckpt_seq_stride + (size_t)(r + 1) * 4 * dh : nullptr;
-            const bool save_ck = a.ckpt && (NORM || !last);
+            const int ce = NORM ? 1 : max(a.ckpt_every, 1);
+            float* ckn = a.ckpt ? a.ckpt + (size_t)seq * a.ckpt_seq_stride + (size_t)((r + 1) / ce) * 4 * dh : nullptr;
+            const bool save_ck = a.ckpt && (NORM || !last) && (r + 1) % ce == 0;
 
             // W1 half, as soon as the W1 aggregation is in (the momentum aggregate follows right behind it)
             mbar_wait(&s.bar_aw1, ph, wc, 100 + 38);
@@ -1032,6 +1033,7 @@ int tc_fwd_launch(const TcFwdArgs& a, void* stream) {
     const bool native = a.d == D && a.h == NC * HC;
     if (a.norm1 && a.norm2) {
         if (a.ckpt && !a.rown) return (int)cudaErrorInvalidValue;
+        if (a.ckpt_every > 1) return (int)cudaErrorInvalidValue;
         e = native ? cudaLaunchKernelEx(&cfg, tc_fwd_kernel<false, true>, tmK, tmQ, tmV, a)
                    : cudaLaunchKernelEx(&cfg, tc_fwd_kernel<true, true>, tmK, tmQ, tmV, a);
     } else {

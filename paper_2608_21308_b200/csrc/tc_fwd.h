@@ -19,6 +19,7 @@ struct TcFwdArgs {
     // optional: chunk-start states for the backward, fp32, [N][nchunks][W1 | W2 | M1 | M2] (nullptr = do not save)
     float* ckpt;
     size_t ckpt_seq_stride;  // floats between two sequences
+    int ckpt_every;          // >= 2: only the start states of chunks 0, n, 2n, .. are saved, in slots 0, 1, 2, .. (not with norm1)
     // optional post-chunk normalisation: per-row target norms of W1 [N, h] and W2 [N, d] (nullptr = none).  With ckpt
     // the kernel also writes what the normalised reverse pass reads: the final state as one more ckpt slot and the
     // row norms before normalisation, rown[N (stride ckpt_seq_stride)][nchunks][3][max(d, h)]

@@ -74,9 +74,26 @@ def test_workspace_sizes(L):
     assert E.e2ttt_workspace_bytes(pt, 0) > 256
 
 
+def test_checkpoints_every_n_chunks_shrink_the_workspace_and_are_refused_by_the_normed_calls(L):
+    from paper_2608_21308_b200 import binding as E
+    kw = dict(io_dtype=E.E2TTT_BF16)
+    full = E.make_params(4, 16, 32768, 128, 512, 64, **kw)
+    seg = E.make_params(4, 16, 32768, 128, 512, 64, ckpt_every=32, **kw)
+    a, b = E.e2ttt_workspace_bytes(full, 1), E.e2ttt_workspace_bytes(seg, 1)
+    per_state = 64 * 4 * 128 * 512 * 4  # all sequences, (W1, W2, M1, M2), fp32
+    assert a > 513 * per_state
+    assert (16 + 1 + 32 + 1) * per_state < b < (16 + 1 + 32 + 1 + 12) * per_state
+    assert E.e2ttt_workspace_bytes(full, 0) == E.e2ttt_workspace_bytes(seg, 0) == 256  # forward only: unchanged
+    one = E.make_params(4, 16, 32768, 128, 512, 64, ckpt_every=1, **kw)
+    assert E.e2ttt_workspace_bytes(one, 1) == a
+    with pytest.raises(E.E2TTTError) as ei:
+        E.e2ttt_workspace_bytes_normed(seg, 1)
+    assert ei.value.status == -2
+
+
 @pytest.mark.parametrize("field,value,status", [
     ("B", 0, -2), ("L", -1, -2), ("C", 0, -2), ("C", 513, -2), ("d", 0, -2), ("h", 100000, -2),
-    ("kind", 2, -2), ("io_dtype", 5, -3), ("impl", 9, -3), ("impl", 2, -2),
+    ("kind", 2, -2), ("io_dtype", 5, -3), ("impl", 9, -3), ("impl", 2, -2), ("ckpt_every", -1, -2),
 ])
 def test_bad_parameters_are_rejected(L, field, value, status):
     from paper_2608_21308_b200 import binding as E

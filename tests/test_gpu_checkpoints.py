@@ -1,0 +1,78 @@
+"""Training-memory plan (Section 3.2 leaves it to the implementation): with e2ttt_params.ckpt_every = n >= 2 the forward
+keeps the state of every n-th chunk only and the backward recomputes n chunk-start states at a time.  The arithmetic of
+every chunk is unchanged, so the gradients must equal those of the keep-everything plan bit for bit whenever both plans
+read states produced by the same kernel, and agree with the oracle's backward as before."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_21308_b200 import binding as E
+from paper_2608_21308_b200 import inputs
+from tests import util
+from tests.test_gpu_parity import check_backward
+
+pytestmark = pytest.mark.gpu
+
+MLP, SWIGLU = E.E2TTT_MLP_GELU, E.E2TTT_SWIGLU
+TOL_F32, TOL_BF16 = 1e-4, 2e-2
+GRADS = ("dq", "dk", "dv", "deta", "dbeta", "dgamma")
+
+
+def same_bits(a, b, what):
+    for n in GRADS:
+        assert np.array_equal(a[n], b[n]), f"{what}: {n}"
+    for i in range(len(a["dW"])):
+        assert np.array_equal(a["dW"][i], b["dW"][i]), f"{what}: dW{i + 1}"
+        assert np.array_equal(a["dM"][i], b["dM"][i]), f"{what}: dM{i + 1}"
+
+
+@pytest.mark.parametrize("kind", [MLP, SWIGLU])
+@pytest.mark.parametrize("every,L", [(3, 8 * 8 + 3), (2, 8 * 5), (4, 8 * 4), (16, 8 * 6)])
+def test_segmented_backward_fp32_matches_the_oracle_and_the_keep_everything_plan(kind, every, L):
+    """9 chunks with a ragged last one in segments of 3; an odd number of segments of 2; exactly one segment; a segment
+    longer than the sequence."""
+    r = inputs.paper_regime(inputs.Recipe(B=3, H=1, L=L, d=24, h=40, C=8, kind=kind, seed=31, m_std=0.002))
+    x = inputs.generate(r, with_d_o=True, with_dstate=True)
+    shape = dict(d=r.d, h=r.h, C=r.C, kind=kind, io="f32")
+    ref = util.oracle_backward(x, r.C, kind)
+    full = util.gpu_backward(x, **shape)
+    check_backward(full, ref, TOL_F32, "every chunk kept")
+    for saved in (False, True):
+        got = util.gpu_backward(x, ckpt_every=every, via_saved_states=saved, **shape)
+        check_backward(got, ref, TOL_F32, f"checkpoints every {every}, saved={saved}")
+        same_bits(got, full, f"every {every}, saved={saved}")
+
+
+@pytest.mark.parametrize("kind,d,h", [(MLP, 128, 512), (SWIGLU, 128, 384)])
+def test_segmented_backward_bf16_tiled(kind, d, h):
+    """bf16 I/O on the tensor-core any-shape kernels, 20 chunks in segments of 8 (8 + 8 + 4), paper-regime gates."""
+    r = inputs.paper_regime(inputs.Recipe(B=2, H=1, L=64 * 20, d=d, h=h, C=64, kind=kind, io="bf16", seed=33, m_std=0.002))
+    x = inputs.generate(r, with_d_o=True, with_dstate=True)
+    shape = dict(d=d, h=h, C=64, kind=kind, io="bf16", impl=E.E2TTT_IMPL_TILED)
+    full = util.gpu_backward(x, **shape)
+    for saved in (False, True):
+        got = util.gpu_backward(x, ckpt_every=8, via_saved_states=saved, **shape)
+        same_bits(got, full, f"tiled, saved={saved}")
+
+
+def test_fused_forward_writes_the_checkpoints():
+    """Training flow at the benchmark shape: the fused forward keeps every 4th chunk-start state, the backward
+    recomputes the rest with the any-shape kernels.  Against the same flow with every state kept by the fused forward
+    (states from two kernel families, at most 3 chunks apart from a shared checkpoint: close, not equal), and the last
+    segment bit for bit against a backward that is handed the fused kernel's own state after 4 chunks."""
+    r = inputs.config(2, heads=[3, 40])
+    shape = dict(d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16")
+    x2, _ = util.teacher_forced_windows(r, 8, window=8, with_grads=True)   # 8 chunks per call, 2 segments of 4
+    a = util.gpu_backward(x2, via_saved_states=True, ckpt_every=4, fwd_impl=E.E2TTT_IMPL_TCGEN05, **shape)
+    b = util.gpu_backward(x2, via_saved_states=True, fwd_impl=E.E2TTT_IMPL_TCGEN05, **shape)
+    for n in GRADS:
+        assert util.rel_err(a[n], b[n]) <= 3 * TOL_BF16, n
+    # checkpoint slot 1 (start of chunk 4) as written by the fused kernel == the state it reports after 4 chunks
+    N, L = x2["q"].shape[0], 8 * 64
+    x4 = {n: (np.ascontiguousarray(v[:, :4 * 64]) if not isinstance(v, list) else v) for n, v in x2.items()}
+    st4, _ = util.gpu_forward(x4, impl=E.E2TTT_IMPL_TCGEN05, **shape)
+    x_tail = {n: (np.ascontiguousarray(v[:, 4 * 64:]) if not isinstance(v, list) else v) for n, v in x2.items()}
+    x_tail["W"], x_tail["M"] = st4["W"], st4["M"]
+    tail_a = util.gpu_backward(x_tail, via_saved_states=False, use_dstate=True, **shape)
+    for n in GRADS:  # the second segment of `a` started from the fused kernel's checkpoint: same states, same bits
+        assert np.array_equal(a[n][:, 4 * 64:], tail_a[n]), n

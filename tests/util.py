@@ -30,10 +30,10 @@ def _io_dtype(io):
     return torch.float32 if io == "f32" else torch.bfloat16
 
 
-def gpu_forward(x, *, d, h, C, kind, io, impl=E.E2TTT_IMPL_AUTO, eps=1e-5, save_states=False, use_M=True):
+def gpu_forward(x, *, d, h, C, kind, io, impl=E.E2TTT_IMPL_AUTO, eps=1e-5, save_states=False, use_M=True, ckpt_every=0):
     """x: dict from inputs.generate (arrays [N, ...]).  Runs e2ttt_chunk_fwd with B=N, H=1.  Returns numpy + handles."""
     N, L, _ = x["q"].shape
-    p = E.make_params(N, 1, L, d, h, C, kind, E.E2TTT_F32 if io == "f32" else E.E2TTT_BF16, eps, impl)
+    p = E.make_params(N, 1, L, d, h, C, kind, E.E2TTT_F32 if io == "f32" else E.E2TTT_BF16, eps, impl, ckpt_every)
     iod = _io_dtype(io)
     q, k, v = (_dev(x[n], iod).view(N, 1, L, d) for n in ("q", "k", "v"))
     eta, beta, gamma = (_dev(x[n], torch.float32).view(N, 1, L) for n in ("eta", "beta", "gamma"))
@@ -52,9 +52,9 @@ def gpu_forward(x, *, d, h, C, kind, io, impl=E.E2TTT_IMPL_AUTO, eps=1e-5, save_
 
 
 def gpu_backward(x, *, d, h, C, kind, io, impl=E.E2TTT_IMPL_AUTO, eps=1e-5, use_M=True, use_dstate=True,
-                 via_saved_states=False):
+                 via_saved_states=False, ckpt_every=0, fwd_impl=None):
     N, L, _ = x["q"].shape
-    p = E.make_params(N, 1, L, d, h, C, kind, E.E2TTT_F32 if io == "f32" else E.E2TTT_BF16, eps, impl)
+    p = E.make_params(N, 1, L, d, h, C, kind, E.E2TTT_F32 if io == "f32" else E.E2TTT_BF16, eps, impl, ckpt_every)
     iod = _io_dtype(io)
     q, k, v, d_o = (_dev(x[n], iod).view(N, 1, L, d) for n in ("q", "k", "v", "d_o"))
     eta, beta, gamma = (_dev(x[n], torch.float32).view(N, 1, L) for n in ("eta", "beta", "gamma"))
@@ -71,7 +71,11 @@ def gpu_backward(x, *, d, h, C, kind, io, impl=E.E2TTT_IMPL_AUTO, eps=1e-5, use_
         o = torch.empty_like(q)
         Wf = [torch.empty_like(w) for w in W]
         Mf = [torch.empty_like(w) for w in W]
-        E.e2ttt_chunk_fwd(p, q, k, v, eta, beta, gamma, W, M, o, Wf, Mf, ws, 1)
+        pf = p
+        if fwd_impl is not None:  # the forward on another kernel family than the backward (same workspace layout)
+            pf = E.make_params(N, 1, L, d, h, C, kind, p.io_dtype, eps, fwd_impl, ckpt_every)
+            assert E.e2ttt_workspace_bytes(pf, 1) == ws.numel()
+        E.e2ttt_chunk_fwd(pf, q, k, v, eta, beta, gamma, W, M, o, Wf, Mf, ws, 1)
     E.e2ttt_chunk_bwd(p, q, k, v, eta, beta, gamma, W, M, d_o, dWf, dMf, dq, dk, dv, de, db, dg, dW, dM, ws,
                       int(via_saved_states))
     torch.cuda.synchronize()
