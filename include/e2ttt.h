@@ -65,10 +65,9 @@ typedef enum { E2TTT_F32 = 0, E2TTT_BF16 = 1 } e2ttt_dtype;
  *             fp32 I/O.  The backward has no fused kernel: AUTO and TCGEN05 mean TILED there.
  *             TCGEN05 serves today: GELU-MLP, bf16 I/O, C = 64, L a multiple of 64, d in {64, 128},
  *             h in {128, 256, 384, 512} (shapes below 128 x 512 run zero-padded in the same tiles); and the
- *             SwiGLU forward at d = 128, h = 384, C = 64, bf16 I/O, without saved states or normalisation.
- *             AUTO selects the fused kernel for the GELU-MLP only: the fused SwiGLU kernel gives its products
- *             plain bf16 copies of the fast weights, which leaves some chunks outside the 2e-2 parity bound
- *             (the any-shape kernels, with two-term bf16 operands, stay inside it); ask for it with TCGEN05.
+ *             SwiGLU forward at d = 128, h = 384, C = 64, bf16 I/O, without saved states or normalisation
+ *             (its gate / up projection reads the fast weights as two bf16 terms: a plain bf16 copy leaves
+ *             some chunks outside the 2e-2 parity bound, the product z1 z2 multiplies the rounding up).
  *   SIMT    : plain CUDA-core kernels for any shape.  With fp32 I/O they compute in fp64
  *             internally; with bf16 I/O in fp32.
  *   TCGEN05 : the fused kernel: bf16 operands on the 5th-generation tensor cores, fp32 accumulation

@@ -60,10 +60,7 @@ int pick_impl(const e2ttt_params* p, bool save_states, int* impl) {
         if (p->io_dtype != E2TTT_BF16) return E2TTT_ERR_SHAPE;
         *impl = E2TTT_IMPL_TILED;
     } else if (p->impl == E2TTT_IMPL_AUTO) {
-        // AUTO takes the fused kernel for the GELU-MLP.  The fused SwiGLU kernel feeds its products plain bf16 copies of
-        // the fast weights, which leaves some one-chunk windows slightly outside the 2e-2 bound (the any-shape kernels
-        // split every operand into two bf16 terms and stay inside it): it is chosen by asking for TCGEN05.
-        *impl = (has_tcgen05(p, save_states) && p->kind == E2TTT_MLP_GELU)
+        *impl = has_tcgen05(p, save_states)
                     ? E2TTT_IMPL_TCGEN05
                     : (p->io_dtype == E2TTT_BF16 ? E2TTT_IMPL_TILED : E2TTT_IMPL_SIMT);
     } else {

@@ -612,13 +612,16 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 float sum = 0.0f;
 #pragma unroll
                 for (int j = 0; j < CPT; ++j) sum += u[j];
+                if (key_rows) PROF(21);
                 const float mu = row_sum(sum) * inv_d;
+                if (key_rows) PROF(22);
                 float sq = 0.0f;
 #pragma unroll
                 for (int j = 0; j < CPT; ++j) { u[j] = real ? u[j] - mu : 0.0f; sq = fmaf(u[j], u[j], sq); }
                 const float rstd = rsqrtf(row_sum(sq) * inv_d + a.eps);
 #pragma unroll
                 for (int j = 0; j < CPT; ++j) u[j] *= rstd;  // y (zero in the padding)
+                if (key_rows) PROF(23);
                 if (key_rows) {
                     // key rows: e = k + y - v, pu = rstd (e - mean(e) - y mean(e y))
                     mbar_wait(&s.bar_v, ph, wc, 100 + 36);

@@ -26,6 +26,10 @@ using namespace sm100;
 using namespace tc;
 
 namespace {
+// The issuer's MMA loops stay rolled: unrolled, the 76 descriptor words of a chunk are hoisted out of the chunk loop
+// and spilled (the control warps run with 32 registers), and every MMA then waits for reloads (2.28 ms instead of
+// 1.73 ms on the 4 x 16 x 4096 workload).
+constexpr int kIssueUnroll = 1;
 
 constexpr int D = 128, HS = 64, NC = 6;
 constexpr int NG = 4;                    // column groups per TMEM lane quadrant
@@ -44,6 +48,7 @@ __device__ __forceinline__ uint32_t tok_owner(int t) {
 
 struct __align__(1024) Smem {
     uint8_t W12[2][16384];   // bf16 [W1c; W2c]  [128 rows][64 i] per slab                 K-major B of G1
+    uint8_t W12lo[2][16384]; // bf16 of what the first copy leaves of the fp32 master      second K-major B of G1
     uint8_t W3[16384];       // bf16 W3c  [128 i][64 j]                                    K-major B of G2, MN-major B of G3
     uint8_t X[2][16384];     // [128 tokens][64 i] per slab; rows 0..63 keys, 64..127 queries (TMA)
     uint8_t Hd[16384];       // bf16 hd [128 tokens][64 j]                                 K-major A of G2; then the CTA's own partial rows
@@ -52,7 +57,10 @@ struct __align__(1024) Smem {
     uint8_t Pu[2][8192];     // bf16 pu [64 t][64 i] per slab                              K-major A of G3, MN-major A of the W3 aggregations
     uint8_t PzW[2][8192];    // kW_t [pz1 | pz2]  [64 t][64 j] per slab                    MN-major A of the W12 aggregation
     uint8_t PzM[2][8192];    // kM_t [pz1 | pz2]
-    uint8_t StageK[NC - 1][8192];  // the peers' fp32 partial sums of the owned key rows
+    // The peers' fp32 partial sums of the owned key rows, one 8 KB slot per peer: slots 0..3 lie over the four pz tiles
+    // (written after G3, when the layer norm has consumed the slots; a peer sends a chunk's sums only after this CTA's
+    // aggregations of the chunk before have completed: the credits), slot 4 has a place of its own.
+    uint8_t StageK4[8192];
     uint8_t StageQ[NC - 1][4096];  // the peers' bf16 partial sums of the owned query rows
     uint8_t Vrows[4096];     // value rows of the owned key tokens (TMA, 16 rows)
     Scalars sc[2];
@@ -63,6 +71,21 @@ struct __align__(1024) Smem {
     uint32_t tmem_base;
     int dead;
 };
+
+// Two-term bf16 form of 16 fp32 values: hi = bf16(w) and lo = bf16(w - hi) into the same place of two slabs
+// (w - hi is exact in fp32; what hi + lo leaves of w is below 2^-16 |w|).
+__device__ __forceinline__ void st_two_term(uint8_t* hi_slab, uint8_t* lo_slab, int row, int col0, const uint32_t (&w)[16]) {
+    uint32_t ph[8], pl[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float w0 = __uint_as_float(w[2 * i]), w1 = __uint_as_float(w[2 * i + 1]);
+        ph[i] = pack_bf16(w0, w1);
+        // a bf16 is the upper half of the fp32 with the same value
+        pl[i] = pack_bf16(w0 - __uint_as_float(ph[i] << 16), w1 - __uint_as_float(ph[i] & 0xFFFF0000u));
+    }
+    st_slab16p(hi_slab, row, col0, ph);
+    st_slab16p(lo_slab, row, col0, pl);
+}
 
 // sigmoid by the hardware tanh: s(z) = 0.5 + 0.5 tanh(z / 2)
 __device__ __forceinline__ float fast_sigmoid(float z) { return fmaf(0.5f, fast_tanh(0.5f * z), 0.5f); }
@@ -136,7 +159,7 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             // The whole warp runs the loop converged (every lane polls the barriers); the MMA and commit instructions are
             // predicated to lane 0.  The descriptor's address field has 14 bits; a shared::cta address carries more above.
             const uint32_t sb = (smem_u32(smem_raw) >> 4) & 0x3FFFu;
-            constexpr uint32_t oW12 = offsetof(Smem, W12) >> 4, oW3 = offsetof(Smem, W3) >> 4, oX = offsetof(Smem, X) >> 4,
+            constexpr uint32_t oW12 = offsetof(Smem, W12) >> 4, oW12lo = offsetof(Smem, W12lo) >> 4, oW3 = offsetof(Smem, W3) >> 4, oX = offsetof(Smem, X) >> 4,
                                oHd = offsetof(Smem, Hd) >> 4, oHdW = offsetof(Smem, HdW) >> 4, oHdM = offsetof(Smem, HdM) >> 4,
                                oPu = offsetof(Smem, Pu) >> 4, oPzW = offsetof(Smem, PzW) >> 4, oPzM = offsetof(Smem, PzM) >> 4;
             const uint32_t id_kk = make_idesc(128, 128, false, false);
@@ -150,38 +173,41 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 mbar_wait(&s.bar_x, ph, wc, 300 + 1);
                 mbar_wait(&s.bar_w12, ph, wc, 300 + 2);
                 tc_fence_after_sync();
-#pragma unroll
+#pragma unroll kIssueUnroll
                 for (int k = 0; k < 8; ++k) umma_bf16_elect(tb + T_R0, dk(sb + oX, 16384, k), dk(sb + oW12, 16384, k), id_kk, k > 0, el);
+                // second term of the two-term bf16 form of W12: z1 z2 multiplies the rounding of a plain bf16 copy up
+#pragma unroll kIssueUnroll
+                for (int k = 0; k < 8; ++k) umma_bf16_elect(tb + T_R0, dk(sb + oX, 16384, k), dk(sb + oW12lo, 16384, k), id_kk, true, el);
                 umma_commit_elect(&s.bar_g1, el);
                 // G2: Upart = Hd W3c^T -> R1 (contraction over the CTA's 64 hidden units)
                 mbar_wait(&s.bar_a, ph, wc, 300 + 3);
                 mbar_wait(&s.bar_w3, ph, wc, 300 + 4);
                 tc_fence_after_sync();
-#pragma unroll
+#pragma unroll kIssueUnroll
                 for (int k = 0; k < 4; ++k) umma_bf16_elect(tb + T_R1, dk(sb + oHd, 16384, k), dk(sb + oW3, 16384, k), id_kk, k > 0, el);
                 umma_commit_elect(&s.bar_g2, el);
                 // G3: Ph = Pu W3c -> R1 columns 0..63
                 mbar_wait<true>(&s.bar_pu, ph, wc, 300 + 5);
                 mbar_wait(&s.bar_r1, ph, wc, 300 + 6);
                 tc_fence_after_sync();
-#pragma unroll
+#pragma unroll kIssueUnroll
                 for (int k = 0; k < 8; ++k) umma_bf16_elect(tb + T_R1, dk(sb + oPu, 8192, k), dmn(sb + oW3, 16384, k), id_kmn64, k > 0, el);
                 umma_commit_elect(&s.bar_g3, el);
                 // W3 aggregation on top of the master
                 mbar_wait(&s.bar_ak, ph, wc, 300 + 7);
                 tc_fence_after_sync();
-#pragma unroll
+#pragma unroll kIssueUnroll
                 for (int k = 0; k < 4; ++k) umma_bf16_elect(tb + T_W3, dmn(sb + oPu, 8192, k), dmn(sb + oHdW, 8192, k), id_agg64, true, el);
                 // W12 aggregation first (the next chunk's G1 hangs on it), then the two momentum aggregates
                 mbar_wait(&s.bar_pz, ph, wc, 300 + 8);
                 tc_fence_after_sync();
-#pragma unroll
+#pragma unroll kIssueUnroll
                 for (int k = 0; k < 4; ++k) umma_bf16_elect(tb + T_W12, dmn(sb + oPzW, 8192, k), dmn(sb + oX, 16384, k), id_agg, true, el);
                 umma_commit_elect(&s.bar_aw12, el);
-#pragma unroll
+#pragma unroll kIssueUnroll
                 for (int k = 0; k < 4; ++k) umma_bf16_elect(tb + T_R0, dmn(sb + oPzM, 8192, k), dmn(sb + oX, 16384, k), id_agg, k > 0, el);
                 umma_commit_elect(&s.bar_am12, el);
-#pragma unroll
+#pragma unroll kIssueUnroll
                 for (int k = 0; k < 4; ++k) umma_bf16_elect(tb + T_R1, dmn(sb + oPu, 8192, k), dmn(sb + oHdM, 8192, k), id_agg64, k > 0, el);
                 umma_commit_elect(&s.bar_am3, el);
             }
@@ -283,7 +309,10 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 for (int j = 0; j < 16; ++j) { st[j] = __float_as_uint(cw0 * w[j]); M12[16 * b + j] = m12 ? m12[16 * b + j] : 0.0f; }
                 const int col = 32 * g + 16 * b;
                 tmem_st16(lane_addr + T_W12 + col, st);
-                st_slab16(s.W12[col >> 6], row, col & 63, w);
+                uint32_t wu[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) wu[j] = __float_as_uint(w[j]);
+                st_two_term(s.W12[col >> 6], s.W12lo[col >> 6], row, col & 63, wu);
             }
             {
                 const float* w3 = a.W3_init + head + off3;
@@ -405,8 +434,9 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 if (key_rows) {
 #pragma unroll
                     for (int sl = 0; sl < NC - 1; ++sl) {
-                        const float4 x0 = *reinterpret_cast<const float4*>(s.StageK[sl] + stage_offset((uint32_t)(2 * cg), (uint32_t)lrow));
-                        const float4 x1 = *reinterpret_cast<const float4*>(s.StageK[sl] + stage_offset((uint32_t)(2 * cg + 1), (uint32_t)lrow));
+                        const uint8_t* sk = sl < 4 ? s.PzW[0] + sl * 8192 : s.StageK4;
+                        const float4 x0 = *reinterpret_cast<const float4*>(sk + stage_offset((uint32_t)(2 * cg), (uint32_t)lrow));
+                        const float4 x1 = *reinterpret_cast<const float4*>(sk + stage_offset((uint32_t)(2 * cg + 1), (uint32_t)lrow));
                         u[0] += x0.x; u[1] += x0.y; u[2] += x0.z; u[3] += x0.w; u[4] += x1.x; u[5] += x1.y; u[6] += x1.z; u[7] += x1.w;
                     }
                 } else {
@@ -496,7 +526,7 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     if (mine) {
                         dst_base = smem_u32(s.Hd);  // the hd tile is dead once G2 has completed
                     } else {
-                        dst_base = map_to_cta(smem_u32(s.StageK[0]) + slot * 8192u, owner);
+                        dst_base = map_to_cta(slot < 4u ? smem_u32(s.PzW[0]) + slot * 8192u : smem_u32(s.StageK4), owner);
                         dst_bar = map_to_cta(smem_u32(&s.bar_partK), owner);
                     }
 #pragma unroll
@@ -595,10 +625,7 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 tmem_wait_ld();
 #pragma unroll
                 for (int j = 0; j < 16; ++j) wa[j] = __float_as_uint(fmaf(cm, M12[16 * b + j], __uint_as_float(wa[j])));
-                uint32_t p[8];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) p[i] = pack_bf16(__uint_as_float(wa[2 * i]), __uint_as_float(wa[2 * i + 1]));
-                st_slab16p(s.W12[col >> 6], row, col & 63, p);
+                st_two_term(s.W12[col >> 6], s.W12lo[col >> 6], row, col & 63, wa);
                 if (last) {
                     float* dst = (row < 64 ? a.W1_final : a.W2_final) + head + off12 + 16 * b;
 #pragma unroll

@@ -1,4 +1,4 @@
-"""Fused tensor-core forward for SwiGLU fast weights (d = 128, h = 384, C = 64, bf16; asked for with impl = TCGEN05)."""
+"""Fused tensor-core forward for SwiGLU fast weights (d = 128, h = 384, C = 64, bf16)."""
 import numpy as np
 import pytest
 
@@ -26,13 +26,14 @@ def per_window_errors(got, ref):
 
 def test_fused_swiglu_windows_across_the_sequence_and_the_split_operand_kernels_beside_it():
     """One-chunk windows started from the oracle's state at chunks 0, 1, 2, 3, 7, 15, 31, 63 of config 3, four heads.
-    The fused kernel rounds the fast-weight operands to plain bf16; SwiGLU is the badly conditioned network (a chunk
-    whose pre-norm outputs have a variance below the layer-norm epsilon amplifies every rounding), so its worst windows
-    are outside the 2e-2 bound (measured: 63 % of the windows inside, median 1.1e-2, worst 0.24) while the any-shape
-    kernels with two-term bf16 operands pass the bound on every window.  Both facts are asserted, and the distribution
-    is printed; this is why AUTO does not select the fused SwiGLU kernel."""
+    SwiGLU is the badly conditioned network: hd = silu(z1) z2 multiplies the rounding of the gate / up projection up,
+    and a plain bf16 copy of W1, W2 as the operand of that product leaves half of these windows outside the 2e-2 bound
+    (worst 0.24, also in fp64 arithmetic with only that rounding applied).  The fused kernel therefore reads [W1; W2] as
+    two bf16 terms (hi + lo); everything else (W3, activations, pu, scaled tiles) is plain bf16.  Every window must be
+    inside the bound, like on the any-shape kernels beside it; the distribution is printed."""
     r = inputs.config(3, heads=[3, 21, 40, 62])
-    xw, ref = util.teacher_forced_windows_at(r, [0, 1, 2, 3, 7, 15, 31, 63])
+    chunks = [0, 1, 2, 3, 7, 15, 31, 63]
+    xw, ref = util.teacher_forced_windows_at(r, chunks)
     fused, hd = util.gpu_forward(xw, impl=E.E2TTT_IMPL_TCGEN05, **SHAPE)
     assert E.e2ttt_device_status(hd["ws"]) == 0 and hd["ws"].numel() == 256      # fused path: status block only
     e = per_window_errors(fused, ref)
@@ -41,18 +42,18 @@ def test_fused_swiglu_windows_across_the_sequence_and_the_split_operand_kernels_
           "worst", dict(zip(NAMES, np.round(e.max(axis=0), 4))))
     print(f"fused SwiGLU: {np.mean(worst <= TOL_BF16):.2f} of the windows within {TOL_BF16}, median of the worst tensor "
           f"{np.median(worst):.4f}, worst window {worst.max():.4f}")
-    chunks = [0, 1, 2, 3, 7, 15, 31, 63]
     print("fused SwiGLU, worst tensor per start chunk (max over the 4 heads):",
           {c: round(float(worst.reshape(4, len(chunks))[:, i].max()), 4) for i, c in enumerate(chunks)})
     assert np.isfinite(e).all()
-    assert np.median(worst) <= TOL_BF16 and np.mean(worst <= TOL_BF16) >= 0.6 and worst.max() <= 0.5
+    check_forward(fused, ref, TOL_BF16, "fused SwiGLU kernel on windows across the sequence")
+    assert worst.max() <= TOL_BF16
     tiled, _ = util.gpu_forward(xw, impl=E.E2TTT_IMPL_TILED, **SHAPE)
     check_forward(tiled, ref, TOL_BF16, "any-shape kernels (two-term bf16 operands) on the same windows")
 
 
 def test_fused_swiglu_free_running_paper_regime_split_calls_and_repeatability():
     """16 chunks free-running under the paper's gate regime (well conditioned) against the oracle; two calls of half the
-    length chain bitwise to the same result; a second run gives the same bits; AUTO keeps the any-shape kernels."""
+    length chain bitwise to the same result; a second run gives the same bits; AUTO selects the fused kernel."""
     r = inputs.paper_regime(inputs.Recipe(B=3, H=1, L=1024, d=128, h=384, C=64, kind=SW, io="bf16", seed=4, m_std=0.002))
     x = inputs.generate(r)
     ref = util.oracle_forward(x, 64, SW)
@@ -71,8 +72,8 @@ def test_fused_swiglu_free_running_paper_regime_split_calls_and_repeatability():
     assert np.array_equal(np.concatenate([a["o"], b["o"]], 1), got["o"])
     for i in range(3):
         assert np.array_equal(b["W"][i], got["W"][i]) and np.array_equal(b["M"][i], got["M"][i])
-    _, hauto = util.gpu_forward(first, impl=E.E2TTT_IMPL_AUTO, **SHAPE)
-    assert hauto["ws"].numel() > 256                                             # AUTO: the any-shape kernels' workspace
+    auto, hauto = util.gpu_forward(first, impl=E.E2TTT_IMPL_AUTO, **SHAPE)
+    assert hauto["ws"].numel() == 256 and np.array_equal(auto["o"], a["o"])      # AUTO: the fused kernel (status block only)
 
 
 def test_fused_swiglu_null_momentum_many_sequences_and_other_shapes_are_refused():
