@@ -609,43 +609,53 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                     for (int o = TPR / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
                     return v;
                 };
-                float sum = 0.0f;
-#pragma unroll
-                for (int j = 0; j < CPT; ++j) sum += u[j];
-                if (key_rows) PROF(21);
-                const float mu = row_sum(sum) * inv_d;
-                if (key_rows) PROF(22);
-                float sq = 0.0f;
-#pragma unroll
-                for (int j = 0; j < CPT; ++j) { u[j] = real ? u[j] - mu : 0.0f; sq = fmaf(u[j], u[j], sq); }
-                const float rstd = rsqrtf(row_sum(sq) * inv_d + a.eps);
-#pragma unroll
-                for (int j = 0; j < CPT; ++j) u[j] *= rstd;  // y (zero in the padding)
-                if (key_rows) PROF(23);
                 if (key_rows) {
-                    // key rows: e = k + y - v, pu = rstd (e - mean(e) - y mean(e y))
+                    // Key rows (the critical path of the whole cluster): e = k + y - v, pu = rstd (e - mean(e) - y mean(e y)).
+                    // All four row sums the two statistics need are taken in ONE pass of shuffles (the shuffles share the
+                    // shared-memory data path with the cluster traffic, a dependent round costs ~60 cycles here):
+                    //   s1 = sum u, s2 = sum u^2, s3 = sum (k - v), s4 = sum (k - v) u
+                    //   mu = s1/d, var = s2/d - mu^2, mean(e) = s3/d (the mean of y is 0),
+                    //   mean(e y) = rstd (s4 - mu s3)/d + var rstd^2
                     mbar_wait(&s.bar_v, ph, wc, 100 + 36);
                     PROF(16);
                     const uint4 vraw = real ? *reinterpret_cast<const uint4*>(s.A[0] + (col0 >> 6) * 2048 + lrow * 128 + ((c ^ (lrow & 7)) << 4))
                                             : make_uint4(0u, 0u, 0u, 0u);
-                    float e[CPT];
-                    float se = 0.0f, sey = 0.0f;
                     const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&xraw);
                     const __nv_bfloat162* v2 = reinterpret_cast<const __nv_bfloat162*>(&vraw);
+                    float kv[CPT];
 #pragma unroll
                     for (int x = 0; x < 4; ++x) {
                         const float2 kf = __bfloat1622float2(k2[x]), vf = __bfloat1622float2(v2[x]);
-                        e[2 * x] = kf.x + u[2 * x] - vf.x;
-                        e[2 * x + 1] = kf.y + u[2 * x + 1] - vf.y;
+                        kv[2 * x] = kf.x - vf.x;
+                        kv[2 * x + 1] = kf.y - vf.y;
+                    }
+                    float s1 = 0.0f, s2 = 0.0f, s3 = 0.0f, s4 = 0.0f;
+#pragma unroll
+                    for (int j = 0; j < CPT; ++j) {
+                        if (!real) u[j] = 0.0f;
+                        s1 += u[j]; s2 = fmaf(u[j], u[j], s2); s3 += kv[j]; s4 = fmaf(kv[j], u[j], s4);
                     }
 #pragma unroll
-                    for (int j = 0; j < CPT; ++j) { se += e[j]; sey = fmaf(e[j], u[j], sey); }
-                    const float me_ = real ? row_sum(se) * inv_d : (row_sum(se), 0.0f);
-                    const float mey = row_sum(sey) * inv_d;
+                    for (int o = TPR / 2; o > 0; o >>= 1) {
+                        const float t1 = __shfl_xor_sync(0xffffffffu, s1, o), t2 = __shfl_xor_sync(0xffffffffu, s2, o);
+                        const float t3 = __shfl_xor_sync(0xffffffffu, s3, o), t4 = __shfl_xor_sync(0xffffffffu, s4, o);
+                        s1 += t1; s2 += t2; s3 += t3; s4 += t4;
+                    }
+                    const float mu = s1 * inv_d;
+                    const float var = fmaxf(fmaf(-mu, mu, s2 * inv_d), 0.0f);
+                    const float rstd = rsqrtf(var + a.eps);
+                    const float me_ = s3 * inv_d;
+                    const float mey = fmaf(rstd * inv_d, fmaf(-mu, s3, s4), var * rstd * rstd);
+                    float e[CPT];
+#pragma unroll
+                    for (int j = 0; j < CPT; ++j) {
+                        u[j] = real ? (u[j] - mu) * rstd : 0.0f;  // y (zero in the padding)
+                        e[j] = kv[j] + u[j];
+                    }
                     uint32_t pk[CPT / 2];
 #pragma unroll
                     for (int j = 0; j < CPT; j += 2)
-                        pk[j / 2] = pack_bf16(rstd * (e[j] - me_ - u[j] * mey), rstd * (e[j + 1] - me_ - u[j + 1] * mey));  // 0 in the padding
+                        pk[j / 2] = real ? pack_bf16(rstd * (e[j] - me_ - u[j] * mey), rstd * (e[j + 1] - me_ - u[j + 1] * mey)) : 0u;  // 0 in the padding
                     // The bf16 pu rows go into this CTA's own pu tile; one bulk copy per peer and slab (2 KB: the 16 rows of a
                     // slab are contiguous) then carries them to the peers' tiles.  Bulk copies write through the async proxy,
                     // the one the MMAs read through, so the receivers need no proxy fence.
@@ -661,7 +671,17 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                         if (lane == 0) mbar_arrive(&s.bar_pu);  // the own rows are in place
                     }
                 } else {
-                    // query rows: o = q + y
+                    // query rows (not on the critical path): two-pass statistics, o = q + y
+                    float sum = 0.0f;
+#pragma unroll
+                    for (int j = 0; j < CPT; ++j) sum += u[j];
+                    const float mu = row_sum(sum) * inv_d;
+                    float sq = 0.0f;
+#pragma unroll
+                    for (int j = 0; j < CPT; ++j) { u[j] = real ? u[j] - mu : 0.0f; sq = fmaf(u[j], u[j], sq); }
+                    const float rstd = rsqrtf(row_sum(sq) * inv_d + a.eps);
+#pragma unroll
+                    for (int j = 0; j < CPT; ++j) u[j] *= rstd;  // y (zero in the padding)
                     const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&xraw);
                     uint4 ov;
                     uint32_t* o32 = reinterpret_cast<uint32_t*>(&ov);
