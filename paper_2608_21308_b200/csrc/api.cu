@@ -299,9 +299,39 @@ static int bwd_common(const e2ttt_params* p, const void* q, const void* k, const
     // A forward that only records chunk-start states: outputs and final states are not written.
     //   first_chunk, n  : the chunks it covers;  mode 1: every chunk's state -> lay.ckpt, 2: checkpoints -> lay.cck
     //   init_slot       : -1 = start from W_init / M_init, else from checkpoint init_slot
+    // The fused tensor-core forward serves the recomputation where it serves the shape (bit-identical to the states a
+    // fused forward with save_states wrote, since it is the same kernel restarted from its own fp32 state).
+    const bool fused_recompute = impl == E2TTT_IMPL_TCGEN05 && p->kind == E2TTT_MLP_GELU && !row_norm;
     auto recompute = [&](int first_chunk, int n, int mode, int init_slot) -> int {
         const size_t t0 = (size_t)first_chunk * p->C;
         const size_t esz = p->io_dtype == E2TTT_F32 ? 4 : 2;
+        if (fused_recompute) {
+            const size_t dh = (size_t)p->d * p->h;
+            float* wsf = static_cast<float*>(ws_data);
+            TcFwdArgs t{};
+            t.N = p->B * p->H; t.L = n * p->C; t.Ls = p->L; t.d = p->d; t.h = p->h; t.eps = p->ln_eps;
+            t.q = static_cast<const __nv_bfloat16*>(q) + t0 * p->d; t.k = static_cast<const __nv_bfloat16*>(k) + t0 * p->d;
+            t.v = static_cast<const __nv_bfloat16*>(v) + t0 * p->d; t.o = nullptr;
+            t.eta = eta + t0; t.beta = beta + t0; t.gamma = gamma + t0;
+            if (init_slot >= 0) {
+                const float* ck = wsf + lay.cck + (size_t)init_slot * 4 * dh;
+                t.W1_init = ck; t.W2_init = ck + dh; t.M1_init = ck + 2 * dh; t.M2_init = ck + 3 * dh;
+                t.init_seq_stride = lay.per_seq;
+            } else {
+                t.W1_init = W_init[0]; t.W2_init = W_init[1];
+                t.M1_init = M_init ? M_init[0] : nullptr; t.M2_init = M_init ? M_init[1] : nullptr;
+            }
+            // the state after the call is not wanted: it lands in the slot behind the last one the reverse sweep reads
+            // (mode 1: slot n of the per-chunk states; mode 2: the slot behind the last checkpoint)
+            float* fin = wsf + (mode == 1 ? lay.ckpt + (size_t)n * 4 * dh : lay.cck + (size_t)((n + seg - 1) / seg) * 4 * dh);
+            t.W1_final = fin; t.W2_final = fin + dh; t.M1_final = fin + 2 * dh; t.M2_final = fin + 3 * dh;
+            t.final_seq_stride = lay.per_seq;
+            t.status = static_cast<int*>(workspace); t.keep_status = 1;
+            t.ckpt = wsf + (mode == 1 ? lay.ckpt : lay.cck);
+            t.ckpt_seq_stride = lay.per_seq;
+            t.ckpt_every = mode == 1 ? 0 : seg;
+            return tc_fwd_launch(t, stream);
+        }
         SimtFwdArgs f{};
         f.N = p->B * p->H; f.d = p->d; f.h = p->h; f.C = p->C; f.nchunks = n;
         f.L = (int)((size_t)p->L - t0 < (size_t)n * p->C ? (size_t)p->L - t0 : (size_t)n * p->C);

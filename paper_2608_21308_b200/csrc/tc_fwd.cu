@@ -135,14 +135,15 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     const uint32_t me = cluster_ctarank();
     const int seq = blockIdx.x / NC;
     const int L = a.L, nchunks = L / C;
+    const int Ls = a.Ls;  // sequence stride in tokens
     WaitCtx wc{&s.dead, a.status};
 
     // Real shape: de x he.  Columns >= de of every token tile and hidden units >= he are zero padding: they stay
     // exactly zero through every product, so only the layer norm (divisor, masks) and the global I/O know about them.
     const int de = PAD ? a.d : D, he = PAD ? a.h : NC * HC;
-    const float* eta = a.eta + (size_t)seq * L;
-    const float* beta = a.beta + (size_t)seq * L;
-    const float* gamma = a.gamma + (size_t)seq * L;
+    const float* eta = a.eta + (size_t)seq * Ls;
+    const float* beta = a.beta + (size_t)seq * Ls;
+    const float* gamma = a.gamma + (size_t)seq * Ls;
 
     if (tid == 0) {
         s.dead = 0;
@@ -264,7 +265,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 if (r == 0) {
                     if (lane == 0) {
                         mbar_expect_tx(&s.bar_x, de == 128 ? 32768u : 16384u);
-                        const int y = seq * L;
+                        const int y = seq * Ls;
                         tma_load_2d(s.X[0], &tmK, 0, y, &s.bar_x);
                         tma_load_2d(s.X[0] + 8192, &tmQ, 0, y, &s.bar_x);
                         if (de == 128) {
@@ -283,7 +284,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                     if (NORM) mbar_expect_tx(&s.bar_rs, 3 * 512);
                     if (r + 1 < nchunks) {
                         // the next chunk's tokens: into L2 now, so that the loads issued at the end of this chunk are short
-                        const int y = seq * L + tok0 + C;
+                        const int y = seq * Ls + tok0 + C;
                         tma_prefetch_l2_2d(&tmK, 0, y);
                         tma_prefetch_l2_2d(&tmQ, 0, y);
                         tma_prefetch_l2_2d(&tmV, 0, y + 16 * (int)me);
@@ -305,7 +306,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 mbar_wait(&s.bar_g2, ph, wc, 100 + 21);
                 if (lane == 0) {
                     mbar_expect_tx(&s.bar_v, de == 128 ? 4096u : 2048u);
-                    const int y = seq * L + tok0 + 16 * (int)me;
+                    const int y = seq * Ls + tok0 + 16 * (int)me;
                     tma_load_2d(s.A[0], &tmV, 0, y, &s.bar_v);
                     if (de == 128) tma_load_2d(s.A[0] + 2048, &tmV, 64, y, &s.bar_v);
                 }
@@ -314,7 +315,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                     mbar_wait(&s.bar_am1, ph, wc, 100 + 22);
                     if (lane == 0) {
                         mbar_expect_tx(&s.bar_x, de == 128 ? 32768u : 16384u);
-                        const int y2 = seq * L + tok0 + C;
+                        const int y2 = seq * Ls + tok0 + C;
                         tma_load_2d(s.X[0], &tmK, 0, y2, &s.bar_x);
                         tma_load_2d(s.X[0] + 8192, &tmQ, 0, y2, &s.bar_x);
                         if (de == 128) {
@@ -358,13 +359,13 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         // normalisation targets of this thread's rows: hidden unit 128 me + row of W1, output row `row` of W2
         const float tgt1 = (NORM && cta_real) ? a.norm1[(size_t)seq * he + HC * me + row] : 0.0f;
         const float tgt2 = (NORM && row < de) ? a.norm2[(size_t)seq * de + row] : 0.0f;
-        __nv_bfloat16* go = a.o + (size_t)seq * L * de;
+        __nv_bfloat16* go = a.o ? a.o + (size_t)seq * Ls * de : nullptr;
 
         // ---- load the state: fp32 master of W -> TMEM (pre-scaled by the first decay carry) and bf16 -> shared; M -> registers
         float M1[CW], M2[CW];
         {
             const float cw0 = s.sc[0].cw;
-            const size_t head = (size_t)seq * dh;
+            const size_t head = (size_t)seq * a.init_seq_stride;
             // W1c[j][i]: global W1 [h][d], row 128 me + j
             const float* w1 = a.W1_init + head + ((size_t)(HC * me) + row) * de + c0;
             const float* m1 = a.M1_init ? a.M1_init + head + ((size_t)(HC * me) + row) * de + c0 : nullptr;
@@ -690,7 +691,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                         const float2 qf = __bfloat1622float2(q2[x]);
                         o32[x] = pack_bf16(qf.x + u[2 * x], qf.y + u[2 * x + 1]);
                     }
-                    if (real) *reinterpret_cast<uint4*>(go + off) = ov;
+                    if (real && go) *reinterpret_cast<uint4*>(go + off) = ov;
                 }
             };
 
@@ -755,7 +756,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             PROF(18);
             const float cm = sc.cm, cb = sc.cb;
             const float cwn = last ? 1.0f : s.sc[(r + 1) & 1].cw;
-            const size_t head = (size_t)seq * dh;
+            const size_t head = (size_t)seq * a.final_seq_stride;
             // slot of the state after this chunk in the saved states (the slot after the last chunk is the final state)
             const int ce = NORM ? 1 : max(a.ckpt_every, 1);
             float* ckn = a.ckpt ? a.ckpt + (size_t)seq * a.ckpt_seq_stride + (size_t)((r + 1) / ce) * 4 * dh : nullptr;
@@ -1020,10 +1021,16 @@ extern "C" __attribute__((visibility("default"))) int e2ttt_debug_read_profile(l
 }
 #endif
 
-int tc_fwd_launch(const TcFwdArgs& a, void* stream) {
+int tc_fwd_launch(const TcFwdArgs& a_in, void* stream) {
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    TcFwdArgs a = a_in;
+    if (a.Ls == 0) a.Ls = a.L;
+    if (a.init_seq_stride == 0) a.init_seq_stride = (size_t)a.d * a.h;
+    if (a.final_seq_stride == 0) a.final_seq_stride = (size_t)a.d * a.h;
+    if (a.Ls < a.L) return (int)cudaErrorInvalidValue;
     CUtensorMap tmK, tmQ, tmV;
-    const size_t rows = (size_t)a.N * a.L;
+    // token rows the maps cover: up to the end of the last sequence's range
+    const size_t rows = (size_t)(a.N - 1) * a.Ls + a.L;
     if (!make_token_map(&tmK, a.k, rows, 64, a.d) || !make_token_map(&tmQ, a.q, rows, 64, a.d) ||
         !make_token_map(&tmV, a.v, rows, 16, a.d))
         return (int)cudaErrorInvalidValue;
@@ -1039,7 +1046,7 @@ int tc_fwd_launch(const TcFwdArgs& a, void* stream) {
         if (e != cudaSuccess) return (int)e;
         if (dev >= 0 && dev < 64) attr_done[dev] = true;
     }
-    cudaError_t e = cudaMemsetAsync(a.status, 0, sizeof(int), st);
+    cudaError_t e = a.keep_status ? cudaSuccess : cudaMemsetAsync(a.status, 0, sizeof(int), st);
     if (e != cudaSuccess) return (int)e;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)(a.N * NC));

@@ -7,13 +7,17 @@ namespace e2ttt {
 
 struct TcFwdArgs {
     int N, L;  // sequences, tokens per sequence (L a multiple of 64)
+    int Ls;    // tokens between two sequences in q, k, v, o and the gates; 0 = L.  A call on a token sub-range of longer
+               // sequences (the backward's recomputation) passes pointers to its first token and the full length here
+    size_t init_seq_stride, final_seq_stride;  // floats between two sequences in *_init / *_final; 0 = d * h
+    int keep_status;  // 1: one launch of several that share the status word: do not clear it
     int d, h;  // head dimension (64 or 128) and hidden width (a multiple of 128, at most 512): smaller shapes run
                // zero-padded inside the 128 x 512 tiles the kernel is built for
     float eps;
     const __nv_bfloat16 *q, *k, *v;
     const float *eta, *beta, *gamma;
     const float *W1_init, *W2_init, *M1_init, *M2_init;  // M*_init may be nullptr (zeros)
-    __nv_bfloat16* o;
+    __nv_bfloat16* o;  // nullptr: the outputs are not wanted
     float *W1_final, *W2_final, *M1_final, *M2_final;
     int* status;  // device word, 0 after a clean run
     // optional: chunk-start states for the backward, fp32, [N][nchunks][W1 | W2 | M1 | M2] (nullptr = do not save)

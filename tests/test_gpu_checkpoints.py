@@ -55,24 +55,29 @@ def test_segmented_backward_bf16_tiled(kind, d, h):
         same_bits(got, full, f"tiled, saved={saved}")
 
 
-def test_fused_forward_writes_the_checkpoints():
-    """Training flow at the benchmark shape: the fused forward keeps every 4th chunk-start state, the backward
-    recomputes the rest with the any-shape kernels.  Against the same flow with every state kept by the fused forward
-    (states from two kernel families, at most 3 chunks apart from a shared checkpoint: close, not equal), and the last
-    segment bit for bit against a backward that is handed the fused kernel's own state after 4 chunks."""
+def test_fused_forward_writes_the_checkpoints_and_recomputes_the_segments():
+    """Training flow at the benchmark shape: the fused forward keeps every 4th chunk-start state and the backward has the
+    same fused kernel recompute the others, restarted from its own fp32 checkpoint: bit for bit the gradients of the flow
+    in which the fused forward kept every state, of the flow in which nothing was saved (everything recomputed), and, on
+    the last segment, of a backward that is handed the fused kernel's own state after 4 chunks as its initial state."""
     r = inputs.config(2, heads=[3, 40])
     shape = dict(d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16")
     x2, _ = util.teacher_forced_windows(r, 8, window=8, with_grads=True)   # 8 chunks per call, 2 segments of 4
-    a = util.gpu_backward(x2, via_saved_states=True, ckpt_every=4, fwd_impl=E.E2TTT_IMPL_TCGEN05, **shape)
-    b = util.gpu_backward(x2, via_saved_states=True, fwd_impl=E.E2TTT_IMPL_TCGEN05, **shape)
-    for n in GRADS:
-        assert util.rel_err(a[n], b[n]) <= 3 * TOL_BF16, n
-    # checkpoint slot 1 (start of chunk 4) as written by the fused kernel == the state it reports after 4 chunks
-    N, L = x2["q"].shape[0], 8 * 64
+    a = util.gpu_backward(x2, via_saved_states=True, ckpt_every=4, **shape)
+    b = util.gpu_backward(x2, via_saved_states=True, **shape)
+    c = util.gpu_backward(x2, via_saved_states=False, ckpt_every=4, **shape)
+    d = util.gpu_backward(x2, via_saved_states=False, **shape)
+    same_bits(a, b, "checkpoints every 4 vs every state kept")
+    same_bits(a, c, "saved checkpoints vs recomputed checkpoints")
+    same_bits(a, d, "vs everything recomputed in one go")
     x4 = {n: (np.ascontiguousarray(v[:, :4 * 64]) if not isinstance(v, list) else v) for n, v in x2.items()}
     st4, _ = util.gpu_forward(x4, impl=E.E2TTT_IMPL_TCGEN05, **shape)
     x_tail = {n: (np.ascontiguousarray(v[:, 4 * 64:]) if not isinstance(v, list) else v) for n, v in x2.items()}
     x_tail["W"], x_tail["M"] = st4["W"], st4["M"]
-    tail_a = util.gpu_backward(x_tail, via_saved_states=False, use_dstate=True, **shape)
-    for n in GRADS:  # the second segment of `a` started from the fused kernel's checkpoint: same states, same bits
-        assert np.array_equal(a[n][:, 4 * 64:], tail_a[n]), n
+    tail = util.gpu_backward(x_tail, via_saved_states=False, **shape)
+    for n in GRADS:
+        assert np.array_equal(a[n][:, 4 * 64:], tail[n]), n
+    # the any-shape kernels on the same flow (two-term bf16 operands): close to the fused states' gradients, not equal
+    t = util.gpu_backward(x2, via_saved_states=False, ckpt_every=4, impl=E.E2TTT_IMPL_TILED, **shape)
+    for n in GRADS:
+        assert util.rel_err(a[n], t[n]) <= 0.15, n   # 8 chunks free-running under the benchmark gates (a chaotic map)
