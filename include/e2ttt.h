@@ -155,10 +155,11 @@ E2TTT_API int e2ttt_chunk_fwd(const e2ttt_params* p,
  *   dW_init, dM_init       out  host tables, state layout, fp32; may alias dW_final / dM_final
  *   workspace              sized by e2ttt_workspace_bytes(p, 1)
  *   states_saved           != 0: the workspace still holds the chunk-start states written by
- *                          e2ttt_chunk_fwd(save_states=1) for the same inputs; 0: they are
- *                          recomputed first
+ *                          e2ttt_chunk_fwd(save_states=1) for the same inputs (same p->ckpt_every); 0: they
+ *                          are recomputed first, by the fused forward where it serves the shape
  * Both network kinds are supported.  The reverse pass runs on the any-shape kernels (SIMT, or TILED with
- * tensor-core products for bf16 I/O); there is no fused reverse kernel.
+ * tensor-core products for bf16 I/O); there is no fused reverse kernel.  With p->ckpt_every >= 2 the call is a
+ * sequence of launches on `stream` (per segment: one forward that recomputes its states, one reverse sweep).
  */
 E2TTT_API int e2ttt_chunk_bwd(const e2ttt_params* p,
                     const void* q, const void* k, const void* v,
