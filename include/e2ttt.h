@@ -63,9 +63,10 @@ typedef enum { E2TTT_F32 = 0, E2TTT_BF16 = 1 } e2ttt_dtype;
 /* Which kernel family serves the call.
  *   AUTO    : TCGEN05 where it serves (kind, io_dtype, d, h, C); else TILED for bf16 I/O and SIMT for
  *             fp32 I/O.  The backward has no fused kernel: AUTO and TCGEN05 mean TILED there.
- *             TCGEN05 serves today: GELU-MLP, bf16 I/O, C = 64, L a multiple of 64, d in {64, 128},
- *             h in {128, 256, 384, 512} (shapes below 128 x 512 run zero-padded in the same tiles); and the
- *             SwiGLU forward at d = 128, h = 384, C = 64, bf16 I/O, without saved states or normalisation
+ *             TCGEN05 serves today: GELU-MLP, bf16 I/O, C in {16, 32, 64}, L a multiple of C, d in {64, 128},
+ *             h in {128, 256, 384, 512} (shapes below 128 x 512 and chunks below 64 tokens run zero-padded in
+ *             the same tiles); and the SwiGLU forward at d = 128, h = 384, C in {16, 32, 64}, bf16 I/O, without
+ *             saved states or normalisation
  *             (its gate / up projection reads the fast weights as two bf16 terms: a plain bf16 copy leaves
  *             some chunks outside the 2e-2 parity bound, the product z1 z2 multiplies the rounding up).
  *   SIMT    : plain CUDA-core kernels for any shape.  With fp32 I/O they compute in fp64
@@ -96,7 +97,7 @@ typedef struct {
     int32_t L;        /* tokens per sequence */
     int32_t d;        /* head dimension (input and output width of the fast-weight network) */
     int32_t h;        /* hidden width of the fast-weight network */
-    int32_t C;        /* chunk size, 1..512 (the paper trains with 512); the tensor-core path serves C = 64.
+    int32_t C;        /* chunk size, 1..512 (the paper trains with 512); the fused kernels serve C = 16, 32, 64.
                          The SIMT path accepts a shorter last chunk. */
     int32_t kind;     /* e2ttt_kind */
     int32_t io_dtype; /* e2ttt_dtype of q, k, v, o, d_o, dq, dk, dv */

@@ -46,7 +46,8 @@ constexpr size_t kStatusBytes = 256;
 // 1 = a tensor-core specialisation exists for these parameters (the forward; with save_states it also writes the
 // chunk-start states in the layout the SIMT backward reads)
 int has_tcgen05(const e2ttt_params* p, bool save_states) {
-    if (p->io_dtype != E2TTT_BF16 || p->C != 64 || p->L % 64 != 0) return 0;
+    // chunks of 32 or 16 tokens run in the same 64-row tiles (unused rows zero): half / a quarter of the tile's work is useful
+    if (p->io_dtype != E2TTT_BF16 || (p->C != 64 && p->C != 32 && p->C != 16) || p->L % p->C != 0) return 0;
     if (p->kind == E2TTT_MLP_GELU) return (p->d == 128 || p->d == 64) && p->h % 128 == 0 && p->h <= 512;
     // SwiGLU: the fused kernel is built for d = 128, h = 384 and does not write chunk-start states
     return p->kind == E2TTT_SWIGLU && p->d == 128 && p->h == 384 && !save_states;
@@ -173,7 +174,7 @@ static int fwd_common(const e2ttt_params* p, const void* q, const void* k, const
     }
     if (impl == E2TTT_IMPL_TCGEN05 && p->kind == E2TTT_SWIGLU) {
         TcSwigluArgs t{};
-        t.N = p->B * p->H; t.L = p->L; t.eps = p->ln_eps;
+        t.N = p->B * p->H; t.L = p->L; t.C = p->C; t.eps = p->ln_eps;
         t.q = static_cast<const __nv_bfloat16*>(q); t.k = static_cast<const __nv_bfloat16*>(k);
         t.v = static_cast<const __nv_bfloat16*>(v); t.o = static_cast<__nv_bfloat16*>(o);
         t.eta = eta; t.beta = beta; t.gamma = gamma;
@@ -186,7 +187,7 @@ static int fwd_common(const e2ttt_params* p, const void* q, const void* k, const
     }
     if (impl == E2TTT_IMPL_TCGEN05) {
         TcFwdArgs t{};
-        t.N = p->B * p->H; t.L = p->L; t.d = p->d; t.h = p->h; t.eps = p->ln_eps;
+        t.N = p->B * p->H; t.L = p->L; t.C = p->C; t.d = p->d; t.h = p->h; t.eps = p->ln_eps;
         t.q = static_cast<const __nv_bfloat16*>(q); t.k = static_cast<const __nv_bfloat16*>(k);
         t.v = static_cast<const __nv_bfloat16*>(v); t.o = static_cast<__nv_bfloat16*>(o);
         t.eta = eta; t.beta = beta; t.gamma = gamma;
@@ -309,7 +310,7 @@ static int bwd_common(const e2ttt_params* p, const void* q, const void* k, const
             const size_t dh = (size_t)p->d * p->h;
             float* wsf = static_cast<float*>(ws_data);
             TcFwdArgs t{};
-            t.N = p->B * p->H; t.L = n * p->C; t.Ls = p->L; t.d = p->d; t.h = p->h; t.eps = p->ln_eps;
+            t.N = p->B * p->H; t.L = n * p->C; t.C = p->C; t.Ls = p->L; t.d = p->d; t.h = p->h; t.eps = p->ln_eps;
             t.q = static_cast<const __nv_bfloat16*>(q) + t0 * p->d; t.k = static_cast<const __nv_bfloat16*>(k) + t0 * p->d;
             t.v = static_cast<const __nv_bfloat16*>(v) + t0 * p->d; t.o = nullptr;
             t.eta = eta + t0; t.beta = beta + t0; t.gamma = gamma + t0;

@@ -38,16 +38,29 @@ __device__ __forceinline__ void named_arrive(int id, int nthreads) { asm volatil
 // barrier ids (0 is __syncthreads)
 constexpr int BAR_EPI = 1, BAR_STAGE = 3, BAR_KOWN = 4, BAR_QOWN = 5;
 
-// Suffix scans of one 64-token chunk by one warp (two tokens per lane), same recurrences as the SIMT path:
+// Suffix scans of one chunk of len <= 64 tokens by one warp (two tokens per lane), same recurrences as the SIMT path:
 // a step is the map (bt, gt, S) -> (beta bt, gamma gt, beta S + gamma gt); suffix composites by warp shuffles.
-static __device__ void tc_chunk_scalars(const float* eta, const float* beta, const float* gamma, Scalars* out) {
+// Positions at and beyond len (the unused rows of a 64-row tile) are the identity map with a zero learning rate: their
+// kW, kM come out as 0 and the carries are those of the len real tokens.
+// The composition of two scan maps with the rounding pinned (one fused multiply-add), so that the scalars do not depend
+// on how the compiler contracts the expression at a given call site.
+__device__ __forceinline__ ScanMap<float> compose_pinned(const ScanMap<float>& outer, const ScanMap<float>& inner) {
+    ScanMap<float> r;
+    r.B = outer.B * inner.B;
+    r.G = outer.G * inner.G;
+    r.X = __fmaf_rn(outer.B, inner.X, __fmul_rn(outer.X, inner.G));
+    return r;
+}
+static __device__ void tc_chunk_scalars(const float* eta, const float* beta, const float* gamma, Scalars* out, int len = 64) {
     const int lane = threadIdx.x & 31;
     ScanMap<float> e0, e1, id;
     id.B = 1.0f; id.G = 1.0f; id.X = 0.0f;
-    e0.B = beta[2 * lane]; e0.G = gamma[2 * lane]; e0.X = e0.G;
-    e1.B = beta[2 * lane + 1]; e1.G = gamma[2 * lane + 1]; e1.X = e1.G;
+    const bool in0 = 2 * lane < len, in1 = 2 * lane + 1 < len;
+    e0 = id; e1 = id;
+    if (in0) { e0.B = beta[2 * lane]; e0.G = gamma[2 * lane]; e0.X = e0.G; }
+    if (in1) { e1.B = beta[2 * lane + 1]; e1.G = gamma[2 * lane + 1]; e1.X = e1.G; }
     const ScanMap<float> loc1 = e1;                 // tokens 2l+1 .. of this lane
-    const ScanMap<float> loc0 = compose(e0, loc1);  // tokens 2l ..   of this lane
+    const ScanMap<float> loc0 = compose_pinned(e0, loc1);  // tokens 2l ..   of this lane
     ScanMap<float> incl = loc0;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
@@ -55,7 +68,7 @@ static __device__ void tc_chunk_scalars(const float* eta, const float* beta, con
         o.B = __shfl_down_sync(0xffffffffu, incl.B, off);
         o.G = __shfl_down_sync(0xffffffffu, incl.G, off);
         o.X = __shfl_down_sync(0xffffffffu, incl.X, off);
-        if (lane + off < 32) incl = compose(incl, o);
+        if (lane + off < 32) incl = compose_pinned(incl, o);
     }
     ScanMap<float> excl;
     excl.B = __shfl_down_sync(0xffffffffu, incl.B, 1);
@@ -63,17 +76,17 @@ static __device__ void tc_chunk_scalars(const float* eta, const float* beta, con
     excl.X = __shfl_down_sync(0xffffffffu, incl.X, 1);
     if (lane == 31) excl = id;
     // token index 2l sees the state after tokens 2l+1.., token 2l+1 the state after the later lanes' tokens
-    const ScanMap<float> f1 = compose(loc1, excl);
-    const float et0 = eta[2 * lane], et1 = eta[2 * lane + 1];
-    out->kW[2 * lane] = et0 * (f1.B + f1.X);
+    const ScanMap<float> f1 = compose_pinned(loc1, excl);
+    const float et0 = in0 ? eta[2 * lane] : 0.0f, et1 = in1 ? eta[2 * lane + 1] : 0.0f;
+    out->kW[2 * lane] = __fmul_rn(et0, __fadd_rn(f1.B, f1.X));
     out->kM[2 * lane] = et0 * f1.B;
-    out->kW[2 * lane + 1] = et1 * (excl.B + excl.X);
+    out->kW[2 * lane + 1] = __fmul_rn(et1, __fadd_rn(excl.B, excl.X));
     out->kM[2 * lane + 1] = et1 * excl.B;
     if (lane == 0) {
-        const ScanMap<float> f0 = compose(loc0, excl);
+        const ScanMap<float> f0 = compose_pinned(loc0, excl);
         out->cw = f0.G;
         out->cb = f0.B;
-        out->cm = e0.B * (f1.B + f1.X);  // beta_1 S_1
+        out->cm = __fmul_rn(e0.B, __fadd_rn(f1.B, f1.X));  // beta_1 S_1
     }
 }
 

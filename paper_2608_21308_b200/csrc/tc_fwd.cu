@@ -134,7 +134,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t me = cluster_ctarank();
     const int seq = blockIdx.x / NC;
-    const int L = a.L, nchunks = L / C;
+    const int Cr = a.C;  // tokens per chunk (<= C = 64, the tile's rows)
+    const int L = a.L, nchunks = L / Cr;
     const int Ls = a.Ls;  // sequence stride in tokens
     WaitCtx wc{&s.dead, a.status};
 
@@ -175,9 +176,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         tma_prefetch_desc(&tmV);
     }
     if (warp == 0) { tmem_alloc(&s.tmem_base, 512); tmem_relinquish(); }
-    if (warp == 1) tc_chunk_scalars(eta, beta, gamma, &s.sc[0]);
+    if (warp == 1) tc_chunk_scalars(eta, beta, gamma, &s.sc[0], Cr);
     if (de < 128)  // the padded half of the token tile is never loaded: zero it once
         for (int i = tid; i < 16384 / 16; i += NTHREADS) reinterpret_cast<uint4*>(s.X[1])[i] = make_uint4(0u, 0u, 0u, 0u);
+    if (Cr < C)    // short chunks: the key and query rows past the chunk are never loaded either (128-byte rows, 8 pieces each)
+        for (int i = tid; i < 32768 / 16; i += NTHREADS)
+            if (((i >> 3) & 63) >= Cr) reinterpret_cast<uint4*>(s.X[0])[i] = make_uint4(0u, 0u, 0u, 0u);
     fence_proxy_async_smem();
     tc_fence_before_sync();
     __syncthreads();
@@ -261,10 +265,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             // ------------------------------------------------------------------- token loads and gate scans
             for (int r = 0; r < nchunks; ++r) {
                 const uint32_t ph = (uint32_t)(r & 1);
-                const int tok0 = r * C;
+                const int tok0 = r * Cr;
                 if (r == 0) {
                     if (lane == 0) {
-                        mbar_expect_tx(&s.bar_x, de == 128 ? 32768u : 16384u);
+                        mbar_expect_tx(&s.bar_x, (uint32_t)Cr * (de == 128 ? 512u : 256u));
                         const int y = seq * Ls;
                         tma_load_2d(s.X[0], &tmK, 0, y, &s.bar_x);
                         tma_load_2d(s.X[0] + 8192, &tmQ, 0, y, &s.bar_x);
@@ -284,7 +288,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                     if (NORM) mbar_expect_tx(&s.bar_rs, 3 * 512);
                     if (r + 1 < nchunks) {
                         // the next chunk's tokens: into L2 now, so that the loads issued at the end of this chunk are short
-                        const int y = seq * Ls + tok0 + C;
+                        const int y = seq * Ls + tok0 + Cr;
                         tma_prefetch_l2_2d(&tmK, 0, y);
                         tma_prefetch_l2_2d(&tmQ, 0, y);
                         tma_prefetch_l2_2d(&tmV, 0, y + 16 * (int)me);
@@ -298,7 +302,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 __syncwarp();
                 if (r + 1 < nchunks) {
                     // scalars of the next chunk (suffix scans over its gates)
-                    tc_chunk_scalars(eta + tok0 + C, beta + tok0 + C, gamma + tok0 + C, &s.sc[(r + 1) & 1]);
+                    tc_chunk_scalars(eta + tok0 + Cr, beta + tok0 + Cr, gamma + tok0 + Cr, &s.sc[(r + 1) & 1], Cr);
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&s.bar_sc);
                 }
@@ -314,8 +318,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                     // the W1 / M1 aggregations were the last readers of the key tile: the next chunk's tokens may land in X
                     mbar_wait(&s.bar_am1, ph, wc, 100 + 22);
                     if (lane == 0) {
-                        mbar_expect_tx(&s.bar_x, de == 128 ? 32768u : 16384u);
-                        const int y2 = seq * Ls + tok0 + C;
+                        mbar_expect_tx(&s.bar_x, (uint32_t)Cr * (de == 128 ? 512u : 256u));
+                        const int y2 = seq * Ls + tok0 + Cr;
                         tma_load_2d(s.X[0], &tmK, 0, y2, &s.bar_x);
                         tma_load_2d(s.X[0] + 8192, &tmQ, 0, y2, &s.bar_x);
                         if (de == 128) {
@@ -424,7 +428,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         for (int r = 0; r < nchunks; ++r) {
             const uint32_t ph = (uint32_t)(r & 1);
             const Scalars& sc = s.sc[r & 1];
-            const int tok0 = r * C;
+            const int tok0 = r * Cr;
             const bool last = (r + 1 == nchunks);
             PROF(0);
             // ---------------- G1 epilogue: a = gelu(z) -> A (bf16), all that G2 needs.  The key rows' a also goes, unscaled,
@@ -691,7 +695,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                         const float2 qf = __bfloat1622float2(q2[x]);
                         o32[x] = pack_bf16(qf.x + u[2 * x], qf.y + u[2 * x + 1]);
                     }
-                    if (real && go) *reinterpret_cast<uint4*>(go + off) = ov;
+                    if (real && go && t < Cr) *reinterpret_cast<uint4*>(go + off) = ov;
                 }
             };
 
@@ -1025,13 +1029,15 @@ int tc_fwd_launch(const TcFwdArgs& a_in, void* stream) {
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     TcFwdArgs a = a_in;
     if (a.Ls == 0) a.Ls = a.L;
+    if (a.C == 0) a.C = C;
+    if ((a.C != 64 && a.C != 32 && a.C != 16) || a.L % a.C != 0) return (int)cudaErrorInvalidValue;
     if (a.init_seq_stride == 0) a.init_seq_stride = (size_t)a.d * a.h;
     if (a.final_seq_stride == 0) a.final_seq_stride = (size_t)a.d * a.h;
     if (a.Ls < a.L) return (int)cudaErrorInvalidValue;
     CUtensorMap tmK, tmQ, tmV;
     // token rows the maps cover: up to the end of the last sequence's range
     const size_t rows = (size_t)(a.N - 1) * a.Ls + a.L;
-    if (!make_token_map(&tmK, a.k, rows, 64, a.d) || !make_token_map(&tmQ, a.q, rows, 64, a.d) ||
+    if (!make_token_map(&tmK, a.k, rows, (unsigned)a.C, a.d) || !make_token_map(&tmQ, a.q, rows, (unsigned)a.C, a.d) ||
         !make_token_map(&tmV, a.v, rows, 16, a.d))
         return (int)cudaErrorInvalidValue;
     static bool attr_done[64];

@@ -6,7 +6,9 @@
 namespace e2ttt {
 
 struct TcFwdArgs {
-    int N, L;  // sequences, tokens per sequence (L a multiple of 64)
+    int N, L;  // sequences, tokens per sequence (L a multiple of the chunk size)
+    int C;     // chunk size: 64, or 32 / 16 (a short chunk runs in the 64-row tiles with the unused rows zero and their
+               // scalar kernels zero); 0 = 64
     int Ls;    // tokens between two sequences in q, k, v, o and the gates; 0 = L.  A call on a token sub-range of longer
                // sequences (the backward's recomputation) passes pointers to its first token and the full length here
     size_t init_seq_stride, final_seq_stride;  // floats between two sequences in *_init / *_final; 0 = d * h

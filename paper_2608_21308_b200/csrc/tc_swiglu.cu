@@ -103,7 +103,8 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t me = cluster_ctarank();
     const int seq = blockIdx.x / NC;
-    const int L = a.L, nchunks = L / C;
+    const int Cr = a.C;  // tokens per chunk (<= C = 64, the tile's rows)
+    const int L = a.L, nchunks = L / Cr;
     const int h = NC * HS;
     WaitCtx wc{&s.dead, a.status};
     const int t0 = tok_begin((int)me), nown = tok_begin((int)me + 1) - t0;   // the key / query tokens this CTA normalises
@@ -140,7 +141,10 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         tma_prefetch_desc(&tmV);
     }
     if (warp == 0) { tmem_alloc(&s.tmem_base, 512); tmem_relinquish(); }
-    if (warp == 1) tc_chunk_scalars(eta, beta, gamma, &s.sc[0]);
+    if (warp == 1) tc_chunk_scalars(eta, beta, gamma, &s.sc[0], Cr);
+    if (Cr < C)    // short chunks: the key and query rows past the chunk are never loaded (128-byte rows, 8 pieces each)
+        for (int i = tid; i < 32768 / 16; i += NTHREADS)
+            if (((i >> 3) & 63) >= Cr) reinterpret_cast<uint4*>(s.X[0])[i] = make_uint4(0u, 0u, 0u, 0u);
     fence_proxy_async_smem();
     tc_fence_before_sync();
     __syncthreads();
@@ -214,7 +218,7 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         } else if (warp == NEW + 3) {
             // ------------------------------------------------------------------- token loads, gate scans, credits
             auto load_tokens = [&](int y) {
-                mbar_expect_tx(&s.bar_x, 32768u);
+                mbar_expect_tx(&s.bar_x, (uint32_t)Cr * 512u);
                 tma_load_2d(s.X[0], &tmK, 0, y, &s.bar_x);
                 tma_load_2d(s.X[0] + 8192, &tmQ, 0, y, &s.bar_x);
                 tma_load_2d(s.X[1], &tmK, 64, y, &s.bar_x);
@@ -222,7 +226,7 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             };
             for (int r = 0; r < nchunks; ++r) {
                 const uint32_t ph = (uint32_t)(r & 1);
-                const int tok0 = r * C;
+                const int tok0 = r * Cr;
                 if (r == 0) {
                     if (lane == 0) load_tokens(seq * L);
                 } else {
@@ -233,7 +237,7 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     mbar_expect_tx(&s.bar_partQ, (uint32_t)((NC - 1) * nown * 256));
                     mbar_expect_tx(&s.bar_pu, (uint32_t)((C - nown) * 256));
                     if (r + 1 < nchunks) {
-                        const int y = seq * L + tok0 + C;
+                        const int y = seq * L + tok0 + Cr;
                         tma_prefetch_l2_2d(&tmK, 0, y);
                         tma_prefetch_l2_2d(&tmQ, 0, y);
                         tma_prefetch_l2_2d(&tmK, 64, y);
@@ -244,7 +248,7 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 }
                 __syncwarp();
                 if (r + 1 < nchunks) {
-                    tc_chunk_scalars(eta + tok0 + C, beta + tok0 + C, gamma + tok0 + C, &s.sc[(r + 1) & 1]);
+                    tc_chunk_scalars(eta + tok0 + Cr, beta + tok0 + Cr, gamma + tok0 + Cr, &s.sc[(r + 1) & 1], Cr);
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&s.bar_sc);
                 }
@@ -258,7 +262,7 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 if (r + 1 < nchunks) {
                     // the W12 / M12 aggregations were the last readers of the key tile: the next chunk's tokens may land in X
                     mbar_wait(&s.bar_am12, ph, wc, 300 + 22);
-                    if (lane == 0) load_tokens(seq * L + tok0 + C);
+                    if (lane == 0) load_tokens(seq * L + tok0 + Cr);
                     // every reader of this chunk's staging / pu / scaled tiles is done once the aggregations have completed and
                     // every epilogue warp has left its layer norm (it has then released W12): credits to and from the peers
                     mbar_wait(&s.bar_am3, ph, wc, 300 + 23);
@@ -337,7 +341,7 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         for (int r = 0; r < nchunks; ++r) {
             const uint32_t ph = (uint32_t)(r & 1);
             const Scalars& sc = s.sc[r & 1];
-            const int tok0 = r * C;
+            const int tok0 = r * Cr;
             const bool last = (r + 1 == nchunks);
             // ---------------- G1 epilogue: hd = silu(z1) z2 -> Hd (bf16), all that G2 needs.  The key rows' hd also goes, as
             // fp16, into the kW hd tile: the query-row warps turn it into bf16 kW hd and kM hd while G2 runs.
@@ -506,7 +510,7 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         }
                         if (lane == 0) mbar_arrive(&s.bar_pu);  // the own rows are in place
                     }
-                } else if (act) {
+                } else if (act && t < Cr) {
                     // query rows: o = q + y
                     uint4 ov;
                     const float2 q0 = __bfloat1622float2(x2[0]), q1 = __bfloat1622float2(x2[1]), q2 = __bfloat1622float2(x2[2]),
@@ -702,11 +706,15 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
 size_t tc_swiglu_smem_bytes() { return sizeof(Smem); }
 
-int tc_swiglu_launch(const TcSwigluArgs& a, void* stream) {
+int tc_swiglu_launch(const TcSwigluArgs& a_in, void* stream) {
+    TcSwigluArgs a = a_in;
+    if (a.C == 0) a.C = C;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     CUtensorMap tmK, tmQ, tmV;
     const size_t rows = (size_t)a.N * a.L;
-    if (!make_token_map(&tmK, a.k, rows, 64, D) || !make_token_map(&tmQ, a.q, rows, 64, D) || !make_token_map(&tmV, a.v, rows, 16, D))
+    const int Cc = a.C;
+    if ((Cc != 64 && Cc != 32 && Cc != 16) || a.L % Cc != 0) return (int)cudaErrorInvalidValue;
+    if (!make_token_map(&tmK, a.k, rows, (unsigned)Cc, D) || !make_token_map(&tmQ, a.q, rows, (unsigned)Cc, D) || !make_token_map(&tmV, a.v, rows, 16, D))
         return (int)cudaErrorInvalidValue;
     static bool attr_done[64];
     int dev = 0;

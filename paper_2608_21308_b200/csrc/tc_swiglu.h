@@ -6,7 +6,8 @@
 namespace e2ttt {
 
 struct TcSwigluArgs {
-    int N, L;  // sequences, tokens per sequence (L a multiple of 64); d = 128, h = 384 are compiled in
+    int N, L;  // sequences, tokens per sequence (L a multiple of the chunk size); d = 128, h = 384 are compiled in
+    int C;     // chunk size: 64, or 32 / 16 (short chunks run in the 64-row tiles, unused rows zero); 0 = 64
     float eps;
     const __nv_bfloat16 *q, *k, *v;
     const float *eta, *beta, *gamma;

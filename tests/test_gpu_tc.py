@@ -245,3 +245,42 @@ def test_tc_boundary_gates():
         check_forward(got, ref, TOL_BF16, f"boundary gates, impl {impl}")
     # eta = 0 for a whole chunk: the gradients do not enter; W_C = cw W_0 + cm M_0, M_C = cb M_0 exactly in the oracle
     assert util.rel_err(ref["M"][0][4], np.prod(x["beta"][4].astype(np.float64)) * x["M"][0][4]) <= 1e-12
+
+
+# ---- chunks of 16 and 32 tokens run in the same 64-row tiles (unused rows zero, their scalar kernels zero)
+
+@pytest.mark.parametrize("C", [16, 32])
+def test_tc_short_chunks_windows_free_running_and_auto_selection(C):
+    r = inputs.config(2, heads=[5, 33], C=C, m_std=0.002)
+    shape = dict(d=128, h=512, C=C, kind=MLP, io="bf16")
+    xw, ref = util.teacher_forced_windows(r, 6, window=1)
+    tc, hd = util.gpu_forward(xw, impl=E.E2TTT_IMPL_TCGEN05, **shape)
+    assert hd["ws"].numel() == 256 and E.e2ttt_device_status(hd["ws"]) == 0
+    print(C, check_forward(tc, ref, TOL_BF16, f"fused kernel, C = {C}, one-chunk windows"))
+    x2, ref2 = util.teacher_forced_windows(r, 6, window=3)   # three chunks per call: the state pass between short chunks
+    tc2, _ = util.gpu_forward(x2, **shape)                   # impl left to the library
+    check_forward(tc2, ref2, 3 * TOL_BF16, f"fused kernel, C = {C}, three-chunk windows")
+    tiled, _ = util.gpu_forward(x2, impl=E.E2TTT_IMPL_TILED, **shape)
+    assert util.rel_err(tc2["o"], tiled["o"]) <= 3 * TOL_BF16
+    # free-running under the paper's gates, 1024 tokens (64 / 32 chunks), against the oracle
+    rp = inputs.paper_regime(inputs.Recipe(B=2, H=1, L=1024, d=128, h=512, C=C, kind=MLP, io="bf16", seed=8, m_std=0.002))
+    x = inputs.generate(rp)
+    refp = util.oracle_forward(x, C, MLP)
+    got, hd = util.gpu_forward(x, **shape)
+    assert hd["ws"].numel() == 256 and E.e2ttt_device_status(hd["ws"]) == 0
+    check_forward(got, refp, TOL_BF16, f"fused kernel, C = {C}, paper regime free-running")
+
+
+def test_tc_short_chunks_saved_states_feed_the_backward():
+    from tests.test_gpu_parity import check_backward
+    r = inputs.config(2, heads=[9], C=32, m_std=0.002)
+    shape = dict(d=128, h=512, C=32, kind=MLP, io="bf16")
+    x1, _ = util.teacher_forced_windows(r, 3, window=1, with_grads=True)
+    ref = util.oracle_backward(x1, 32, MLP)
+    got = util.gpu_backward(x1, via_saved_states=True, **shape)
+    check_backward(got, ref, TOL_BF16, "C = 32: backward from the fused kernel's saved states")
+    x3, _ = util.teacher_forced_windows(r, 6, window=6, with_grads=True)
+    a = util.gpu_backward(x3, via_saved_states=True, ckpt_every=2, **shape)
+    b = util.gpu_backward(x3, via_saved_states=False, **shape)
+    for n in ("dq", "dk", "dv", "deta", "dbeta", "dgamma"):
+        assert np.array_equal(a[n], b[n]), n

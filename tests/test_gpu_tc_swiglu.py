@@ -90,3 +90,21 @@ def test_fused_swiglu_null_momentum_many_sequences_and_other_shapes_are_refused(
     p = E.make_params(1, 1, 128, 128, 384, 64, E.E2TTT_SWIGLU, E.E2TTT_BF16, 1e-5, E.E2TTT_IMPL_TCGEN05)
     with pytest.raises(E.E2TTTError):
         E.e2ttt_workspace_bytes(p, 1)                                            # it does not save chunk-start states
+
+
+@pytest.mark.parametrize("C", [16, 32])
+def test_fused_swiglu_short_chunks(C):
+    """Chunks of 16 and 32 tokens in the 64-row tiles: windows from the oracle's state, and a free-running run."""
+    r = inputs.config(3, heads=[3, 40], C=C)
+    shape = dict(d=128, h=384, C=C, kind=SW, io="bf16")
+    xw, ref = util.teacher_forced_windows_at(r, [0, 1, 5, 20])
+    got, hd = util.gpu_forward(xw, **shape)                                      # impl left to the library
+    assert hd["ws"].numel() == 256 and E.e2ttt_device_status(hd["ws"]) == 0
+    print(C, check_forward(got, ref, TOL_BF16, f"fused SwiGLU, C = {C}, windows"))
+    # 16 chunks free-running, like the C = 64 run above (a longer free-running run compounds the per-chunk rounding)
+    rp = inputs.paper_regime(inputs.Recipe(B=2, H=1, L=16 * C, d=128, h=384, C=C, kind=SW, io="bf16", seed=5, m_std=0.002))
+    x = inputs.generate(rp)
+    refp = util.oracle_forward(x, C, SW)
+    gp, hd = util.gpu_forward(x, **shape)
+    assert E.e2ttt_device_status(hd["ws"]) == 0
+    check_forward(gp, refp, TOL_BF16, f"fused SwiGLU, C = {C}, paper regime free-running")

@@ -64,7 +64,7 @@ def test_tiled_backward_odd_shape_free_running(kind, L, tol):
 
 
 def test_tiled_is_the_default_for_bf16_shapes_without_a_fused_kernel_and_is_repeatable():
-    r = inputs.config(3, heads=[1, 2, 3], L=256, C=32)                   # the fused SwiGLU kernel serves C = 64 only
+    r = inputs.config(3, heads=[1, 2, 3], L=256, C=128)                  # the fused kernels serve C = 16, 32, 64
     x = inputs.generate(r)
     a, hd = util.gpu_forward(x, **_shape(r))                              # AUTO
     b, _ = util.gpu_forward(x, impl=E.E2TTT_IMPL_TILED, **_shape(r))
