@@ -64,8 +64,10 @@ def test_workspace_sizes(L):
     assert b - a >= 16 * 2 * 2 * 64 * 256 * 8
     p2 = E.make_params(2, 3, 256, 64, 256, 16)
     assert E.e2ttt_workspace_bytes(p2, 0) - 256 == 6 * (a - 256)   # 256-byte status block + per-sequence scratch
-    pb = E.make_params(1, 1, 256, 64, 256, 16, io_dtype=E.E2TTT_BF16)
+    pb = E.make_params(1, 1, 256, 64, 256, 16, io_dtype=E.E2TTT_BF16, impl=E.E2TTT_IMPL_SIMT)
     assert (E.e2ttt_workspace_bytes(pb, 0) - 256) * 2 == a - 256
+    pb.impl = E.E2TTT_IMPL_AUTO            # bf16, d = 64, h = 256, C = 16: the fused kernel serves it
+    assert E.e2ttt_workspace_bytes(pb, 0) == 256
     # the tensor-core forward keeps all state on chip: only the status block
     pt = E.make_params(4, 16, 4096, 128, 512, 64, io_dtype=E.E2TTT_BF16)
     assert E.e2ttt_workspace_bytes(pt, 0) == 256
