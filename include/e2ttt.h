@@ -66,7 +66,7 @@ typedef enum { E2TTT_F32 = 0, E2TTT_BF16 = 1 } e2ttt_dtype;
  *             TCGEN05 serves today: GELU-MLP, bf16 I/O, C in {16, 32, 64}, L a multiple of C, d in {64, 128},
  *             h in {128, 256, 384, 512} (shapes below 128 x 512 and chunks below 64 tokens run zero-padded in
  *             the same tiles); and the SwiGLU forward at d = 128, h = 384, C in {16, 32, 64}, bf16 I/O, without
- *             saved states or normalisation
+ *             post-chunk normalisation
  *             (its gate / up projection reads the fast weights as two bf16 terms: a plain bf16 copy leaves
  *             some chunks outside the 2e-2 parity bound, the product z1 z2 multiplies the rounding up).
  *   SIMT    : plain CUDA-core kernels for any shape.  With fp32 I/O they compute in fp64

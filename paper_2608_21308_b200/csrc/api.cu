@@ -49,8 +49,9 @@ int has_tcgen05(const e2ttt_params* p, bool save_states) {
     // chunks of 32 or 16 tokens run in the same 64-row tiles (unused rows zero): half / a quarter of the tile's work is useful
     if (p->io_dtype != E2TTT_BF16 || (p->C != 64 && p->C != 32 && p->C != 16) || p->L % p->C != 0) return 0;
     if (p->kind == E2TTT_MLP_GELU) return (p->d == 128 || p->d == 64) && p->h % 128 == 0 && p->h <= 512;
-    // SwiGLU: the fused kernel is built for d = 128, h = 384 and does not write chunk-start states
-    return p->kind == E2TTT_SWIGLU && p->d == 128 && p->h == 384 && !save_states;
+    // SwiGLU: the fused kernel is built for d = 128, h = 384
+    (void)save_states;
+    return p->kind == E2TTT_SWIGLU && p->d == 128 && p->h == 384;
 }
 
 int pick_impl(const e2ttt_params* p, bool save_states, int* impl) {
@@ -183,6 +184,13 @@ static int fwd_common(const e2ttt_params* p, const void* q, const void* k, const
         t.W1_final = W_final[0]; t.W2_final = W_final[1]; t.W3_final = W_final[2];
         t.M1_final = M_final[0]; t.M2_final = M_final[1]; t.M3_final = M_final[2];
         t.status = static_cast<int*>(workspace);
+        if (save_states) {
+            const int seg = segment_chunks(p);
+            const SimtLayout lay = simt_layout(p->d, p->h, p->C, nmat, p->L / p->C, true, true, seg);
+            t.ckpt = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBytes) + (seg ? lay.cck : lay.ckpt);
+            t.ckpt_seq_stride = lay.per_seq;
+            t.ckpt_every = seg;
+        }
         return tc_swiglu_launch(t, stream) == 0 ? E2TTT_OK : E2TTT_ERR_CUDA;
     }
     if (impl == E2TTT_IMPL_TCGEN05) {
@@ -302,10 +310,38 @@ static int bwd_common(const e2ttt_params* p, const void* q, const void* k, const
     //   init_slot       : -1 = start from W_init / M_init, else from checkpoint init_slot
     // The fused tensor-core forward serves the recomputation where it serves the shape (bit-identical to the states a
     // fused forward with save_states wrote, since it is the same kernel restarted from its own fp32 state).
-    const bool fused_recompute = impl == E2TTT_IMPL_TCGEN05 && p->kind == E2TTT_MLP_GELU && !row_norm;
+    const bool fused_recompute = impl == E2TTT_IMPL_TCGEN05 && !row_norm;
     auto recompute = [&](int first_chunk, int n, int mode, int init_slot) -> int {
         const size_t t0 = (size_t)first_chunk * p->C;
         const size_t esz = p->io_dtype == E2TTT_F32 ? 4 : 2;
+        if (fused_recompute && p->kind == E2TTT_SWIGLU) {
+            const size_t dh = (size_t)p->d * p->h;
+            float* wsf = static_cast<float*>(ws_data);
+            TcSwigluArgs t{};
+            t.N = p->B * p->H; t.L = n * p->C; t.C = p->C; t.Ls = p->L; t.eps = p->ln_eps;
+            t.q = static_cast<const __nv_bfloat16*>(q) + t0 * p->d; t.k = static_cast<const __nv_bfloat16*>(k) + t0 * p->d;
+            t.v = static_cast<const __nv_bfloat16*>(v) + t0 * p->d; t.o = nullptr;
+            t.eta = eta + t0; t.beta = beta + t0; t.gamma = gamma + t0;
+            if (init_slot >= 0) {
+                const float* ck = wsf + lay.cck + (size_t)init_slot * 6 * dh;
+                t.W1_init = ck; t.W2_init = ck + dh; t.W3_init = ck + 2 * dh;
+                t.M1_init = ck + 3 * dh; t.M2_init = ck + 4 * dh; t.M3_init = ck + 5 * dh;
+                t.init_seq_stride = lay.per_seq;
+            } else {
+                t.W1_init = W_init[0]; t.W2_init = W_init[1]; t.W3_init = W_init[2];
+                t.M1_init = M_init ? M_init[0] : nullptr; t.M2_init = M_init ? M_init[1] : nullptr;
+                t.M3_init = M_init ? M_init[2] : nullptr;
+            }
+            float* fin = wsf + (mode == 1 ? lay.ckpt + (size_t)n * 6 * dh : lay.cck + (size_t)((n + seg - 1) / seg) * 6 * dh);
+            t.W1_final = fin; t.W2_final = fin + dh; t.W3_final = fin + 2 * dh;
+            t.M1_final = fin + 3 * dh; t.M2_final = fin + 4 * dh; t.M3_final = fin + 5 * dh;
+            t.final_seq_stride = lay.per_seq;
+            t.status = static_cast<int*>(workspace); t.keep_status = 1;
+            t.ckpt = wsf + (mode == 1 ? lay.ckpt : lay.cck);
+            t.ckpt_seq_stride = lay.per_seq;
+            t.ckpt_every = mode == 1 ? 0 : seg;
+            return tc_swiglu_launch(t, stream);
+        }
         if (fused_recompute) {
             const size_t dh = (size_t)p->d * p->h;
             float* wsf = static_cast<float*>(ws_data);

@@ -105,12 +105,13 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const int seq = blockIdx.x / NC;
     const int Cr = a.C;  // tokens per chunk (<= C = 64, the tile's rows)
     const int L = a.L, nchunks = L / Cr;
+    const int Ls = a.Ls;  // sequence stride in tokens
     const int h = NC * HS;
     WaitCtx wc{&s.dead, a.status};
     const int t0 = tok_begin((int)me), nown = tok_begin((int)me + 1) - t0;   // the key / query tokens this CTA normalises
-    const float* eta = a.eta + (size_t)seq * L;
-    const float* beta = a.beta + (size_t)seq * L;
-    const float* gamma = a.gamma + (size_t)seq * L;
+    const float* eta = a.eta + (size_t)seq * Ls;
+    const float* beta = a.beta + (size_t)seq * Ls;
+    const float* gamma = a.gamma + (size_t)seq * Ls;
 
     if (tid == 0) {
         s.dead = 0;
@@ -228,7 +229,7 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 const uint32_t ph = (uint32_t)(r & 1);
                 const int tok0 = r * Cr;
                 if (r == 0) {
-                    if (lane == 0) load_tokens(seq * L);
+                    if (lane == 0) load_tokens(seq * Ls);
                 } else {
                     mbar_wait(&s.bar_w3, ph, wc, 300 + 20);  // the previous chunk is over in this CTA
                 }
@@ -237,7 +238,7 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     mbar_expect_tx(&s.bar_partQ, (uint32_t)((NC - 1) * nown * 256));
                     mbar_expect_tx(&s.bar_pu, (uint32_t)((C - nown) * 256));
                     if (r + 1 < nchunks) {
-                        const int y = seq * L + tok0 + Cr;
+                        const int y = seq * Ls + tok0 + Cr;
                         tma_prefetch_l2_2d(&tmK, 0, y);
                         tma_prefetch_l2_2d(&tmQ, 0, y);
                         tma_prefetch_l2_2d(&tmK, 64, y);
@@ -255,14 +256,14 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 if (lane == 0) {
                     // the value rows of the owned key tokens (a box of 16 rows: the rows past the owned ones are not read)
                     mbar_expect_tx(&s.bar_v, 4096u);
-                    const int y = seq * L + tok0 + t0;
+                    const int y = seq * Ls + tok0 + t0;
                     tma_load_2d(s.Vrows, &tmV, 0, y, &s.bar_v);
                     tma_load_2d(s.Vrows + 2048, &tmV, 64, y, &s.bar_v);
                 }
                 if (r + 1 < nchunks) {
                     // the W12 / M12 aggregations were the last readers of the key tile: the next chunk's tokens may land in X
                     mbar_wait(&s.bar_am12, ph, wc, 300 + 22);
-                    if (lane == 0) load_tokens(seq * L + tok0 + Cr);
+                    if (lane == 0) load_tokens(seq * Ls + tok0 + Cr);
                     // every reader of this chunk's staging / pu / scaled tiles is done once the aggregations have completed and
                     // every epilogue warp has left its layer norm (it has then released W12): credits to and from the peers
                     mbar_wait(&s.bar_am3, ph, wc, 300 + 23);
@@ -286,8 +287,9 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         const uint32_t lane_addr = tb + ((uint32_t)(32 * q) << 16);
         const size_t dh = (size_t)D * h;
         const float inv_d = 1.0f / (float)D;
-        __nv_bfloat16* go = a.o + (size_t)seq * L * D;
-        const size_t head = (size_t)seq * dh;
+        __nv_bfloat16* go = a.o ? a.o + (size_t)seq * Ls * D : nullptr;
+        const size_t head = (size_t)seq * a.final_seq_stride, head0 = (size_t)seq * a.init_seq_stride;
+        float* const ck0 = a.ckpt ? a.ckpt + (size_t)seq * a.ckpt_seq_stride : nullptr;  // slot 0: the initial state
         // W12 row `row`: W1 (row < 64) or W2 row of hidden unit 64 me + (row & 63); this thread's columns 32 g ..
         const size_t off12 = ((size_t)(HS * me) + (row & 63)) * D + 32 * g;
         // W3c[i = row][j]: global W3 [d][h], this thread's columns 64 me + 16 g ..
@@ -297,9 +299,9 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         float M12[32], M3[16];
         {
             const float cw0 = s.sc[0].cw;
-            const float* w12 = (row < 64 ? a.W1_init : a.W2_init) + head + off12;
+            const float* w12 = (row < 64 ? a.W1_init : a.W2_init) + head0 + off12;
             const float* m12p = row < 64 ? a.M1_init : a.M2_init;
-            const float* m12 = m12p ? m12p + head + off12 : nullptr;
+            const float* m12 = m12p ? m12p + head0 + off12 : nullptr;
 #pragma unroll
             for (int b = 0; b < 2; ++b) {
                 float w[16];
@@ -317,10 +319,19 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 #pragma unroll
                 for (int j = 0; j < 16; ++j) wu[j] = __float_as_uint(w[j]);
                 st_two_term(s.W12[col >> 6], s.W12lo[col >> 6], row, col & 63, wu);
+                if (ck0) {
+                    float* cw = ck0 + (row < 64 ? 0 : dh) + off12 + 16 * b;       // W1 | W2
+                    float* cm_ = ck0 + (row < 64 ? 3 : 4) * dh + off12 + 16 * b;   // M1 | M2
+#pragma unroll
+                    for (int j = 0; j < 16; j += 4) {
+                        *reinterpret_cast<float4*>(cw + j) = make_float4(w[j], w[j + 1], w[j + 2], w[j + 3]);
+                        *reinterpret_cast<float4*>(cm_ + j) = make_float4(M12[16 * b + j], M12[16 * b + j + 1], M12[16 * b + j + 2], M12[16 * b + j + 3]);
+                    }
+                }
             }
             {
-                const float* w3 = a.W3_init + head + off3;
-                const float* m3 = a.M3_init ? a.M3_init + head + off3 : nullptr;
+                const float* w3 = a.W3_init + head0 + off3;
+                const float* m3 = a.M3_init ? a.M3_init + head0 + off3 : nullptr;
                 float w[16];
                 uint32_t st[16];
 #pragma unroll
@@ -332,6 +343,13 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 for (int j = 0; j < 16; ++j) { st[j] = __float_as_uint(cw0 * w[j]); M3[j] = m3 ? m3[j] : 0.0f; }
                 tmem_st16(lane_addr + T_W3 + 16 * g, st);
                 st_slab16(s.W3, row, 16 * g, w);
+                if (ck0) {
+#pragma unroll
+                    for (int j = 0; j < 16; j += 4) {
+                        *reinterpret_cast<float4*>(ck0 + 2 * dh + off3 + j) = make_float4(w[j], w[j + 1], w[j + 2], w[j + 3]);
+                        *reinterpret_cast<float4*>(ck0 + 5 * dh + off3 + j) = make_float4(M3[j], M3[j + 1], M3[j + 2], M3[j + 3]);
+                    }
+                }
             }
             tmem_wait_st();
             warp_release(&s.bar_w12);
@@ -510,7 +528,7 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         }
                         if (lane == 0) mbar_arrive(&s.bar_pu);  // the own rows are in place
                     }
-                } else if (act && t < Cr) {
+                } else if (act && t < Cr && go) {
                     // query rows: o = q + y
                     uint4 ov;
                     const float2 q0 = __bfloat1622float2(x2[0]), q1 = __bfloat1622float2(x2[1]), q2 = __bfloat1622float2(x2[2]),
@@ -618,6 +636,10 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             if (!last) mbar_wait(&s.bar_sc, ph, wc, 300 + 37);  // the next chunk's scalars (its decay carry pre-scales the masters)
             const float cm = sc.cm, cb = sc.cb;
             const float cwn = last ? 1.0f : s.sc[(r + 1) & 1].cw;
+            // slot of the state after this chunk in the saved states (every chunk's, or every ckpt_every-th)
+            const int ce = max(a.ckpt_every, 1);
+            float* const ckn = ck0 ? ck0 + (size_t)((r + 1) / ce) * 6 * dh : nullptr;
+            const bool save_ck = ck0 && !last && (r + 1) % ce == 0;
             // W12 half, as soon as its aggregation is in (the momentum aggregate follows right behind it)
             mbar_wait(&s.bar_aw12, ph, wc, 300 + 38);
             tc_fence_after_sync();
@@ -630,8 +652,8 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 #pragma unroll
                 for (int j = 0; j < 16; ++j) wa[j] = __float_as_uint(fmaf(cm, M12[16 * b + j], __uint_as_float(wa[j])));
                 st_two_term(s.W12[col >> 6], s.W12lo[col >> 6], row, col & 63, wa);
-                if (last) {
-                    float* dst = (row < 64 ? a.W1_final : a.W2_final) + head + off12 + 16 * b;
+                if (last || save_ck) {
+                    float* dst = (last ? (row < 64 ? a.W1_final : a.W2_final) + head : ckn + (row < 64 ? 0 : dh)) + off12 + 16 * b;
 #pragma unroll
                     for (int j = 0; j < 16; j += 4) *reinterpret_cast<uint4*>(dst + j) = make_uint4(wa[j], wa[j + 1], wa[j + 2], wa[j + 3]);
                 }
@@ -648,8 +670,8 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 tmem_wait_ld();
 #pragma unroll
                 for (int j = 0; j < 16; ++j) M12[16 * b + j] = fmaf(cb, M12[16 * b + j], __uint_as_float(ma[j]));
-                if (last) {
-                    float* dst = (row < 64 ? a.M1_final : a.M2_final) + head + off12 + 16 * b;
+                if (last || save_ck) {
+                    float* dst = (last ? (row < 64 ? a.M1_final : a.M2_final) + head : ckn + (row < 64 ? 3 : 4) * dh) + off12 + 16 * b;
 #pragma unroll
                     for (int j = 0; j < 16; j += 4)
                         *reinterpret_cast<float4*>(dst + j) = make_float4(M12[16 * b + j], M12[16 * b + j + 1], M12[16 * b + j + 2], M12[16 * b + j + 3]);
@@ -671,8 +693,8 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 #pragma unroll
                 for (int i = 0; i < 8; ++i) p[i] = pack_bf16(__uint_as_float(wa[2 * i]), __uint_as_float(wa[2 * i + 1]));
                 st_slab16p(s.W3, row, 16 * g, p);
-                if (last) {
-                    float* dst = a.W3_final + head + off3;
+                if (last || save_ck) {
+                    float* dst = (last ? a.W3_final + head : ckn + 2 * dh) + off3;
 #pragma unroll
                     for (int j = 0; j < 16; j += 4) *reinterpret_cast<uint4*>(dst + j) = make_uint4(wa[j], wa[j + 1], wa[j + 2], wa[j + 3]);
                 }
@@ -684,8 +706,8 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 tmem_wait_ld();
 #pragma unroll
                 for (int j = 0; j < 16; ++j) M3[j] = fmaf(cb, M3[j], __uint_as_float(ma[j]));
-                if (last) {
-                    float* dst = a.M3_final + head + off3;
+                if (last || save_ck) {
+                    float* dst = (last ? a.M3_final + head : ckn + 5 * dh) + off3;
 #pragma unroll
                     for (int j = 0; j < 16; j += 4) *reinterpret_cast<float4*>(dst + j) = make_float4(M3[j], M3[j + 1], M3[j + 2], M3[j + 3]);
                 }
@@ -709,9 +731,13 @@ size_t tc_swiglu_smem_bytes() { return sizeof(Smem); }
 int tc_swiglu_launch(const TcSwigluArgs& a_in, void* stream) {
     TcSwigluArgs a = a_in;
     if (a.C == 0) a.C = C;
+    if (a.Ls == 0) a.Ls = a.L;
+    if (a.init_seq_stride == 0) a.init_seq_stride = (size_t)D * NC * HS;
+    if (a.final_seq_stride == 0) a.final_seq_stride = (size_t)D * NC * HS;
+    if (a.Ls < a.L) return (int)cudaErrorInvalidValue;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     CUtensorMap tmK, tmQ, tmV;
-    const size_t rows = (size_t)a.N * a.L;
+    const size_t rows = (size_t)(a.N - 1) * a.Ls + a.L;  // token rows the maps cover: up to the end of the last sequence's range
     const int Cc = a.C;
     if ((Cc != 64 && Cc != 32 && Cc != 16) || a.L % Cc != 0) return (int)cudaErrorInvalidValue;
     if (!make_token_map(&tmK, a.k, rows, (unsigned)Cc, D) || !make_token_map(&tmQ, a.q, rows, (unsigned)Cc, D) || !make_token_map(&tmV, a.v, rows, 16, D))
@@ -725,7 +751,7 @@ int tc_swiglu_launch(const TcSwigluArgs& a_in, void* stream) {
         if (e != cudaSuccess) return (int)e;
         if (dev >= 0 && dev < 64) attr_done[dev] = true;
     }
-    cudaError_t e = cudaMemsetAsync(a.status, 0, sizeof(int), st);
+    cudaError_t e = a.keep_status ? cudaSuccess : cudaMemsetAsync(a.status, 0, sizeof(int), st);
     if (e != cudaSuccess) return (int)e;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)(a.N * NC));

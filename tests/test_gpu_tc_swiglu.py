@@ -88,8 +88,35 @@ def test_fused_swiglu_null_momentum_many_sequences_and_other_shapes_are_refused(
     with pytest.raises(E.E2TTTError):
         E.e2ttt_workspace_bytes(p, 0)                                            # h = 512: no fused SwiGLU kernel
     p = E.make_params(1, 1, 128, 128, 384, 64, E.E2TTT_SWIGLU, E.E2TTT_BF16, 1e-5, E.E2TTT_IMPL_TCGEN05)
+    assert E.e2ttt_workspace_bytes(p, 1) > 256                                   # with saved states: the backward's workspace
     with pytest.raises(E.E2TTTError):
-        E.e2ttt_workspace_bytes(p, 1)                                            # it does not save chunk-start states
+        E.e2ttt_workspace_bytes_normed(p, 0)                                     # no fused SwiGLU kernel with normalisation
+
+
+def test_fused_swiglu_saves_states_checkpoints_and_recomputes_for_the_backward():
+    """Training flow: the fused forward writes the chunk-start states (all of them, or every 2nd with the others
+    recomputed by the same kernel in the backward): gradients against the oracle on one-chunk windows, and bit for bit
+    among the memory plans on four-chunk windows."""
+    from tests.test_gpu_parity import check_backward
+    r = inputs.config(3, heads=[7, 50])
+    x1, _ = util.teacher_forced_windows(r, 3, window=1, with_grads=True)
+    ref = util.oracle_backward(x1, 64, SW)
+    got = util.gpu_backward(x1, via_saved_states=True, **SHAPE)
+    check_backward(got, ref, TOL_BF16, "SwiGLU backward from the fused kernel's saved states")
+    x4, _ = util.teacher_forced_windows(r, 4, window=4, with_grads=True)
+    a = util.gpu_backward(x4, via_saved_states=True, **SHAPE)
+    b = util.gpu_backward(x4, via_saved_states=True, ckpt_every=2, **SHAPE)
+    c = util.gpu_backward(x4, via_saved_states=False, ckpt_every=2, **SHAPE)
+    d = util.gpu_backward(x4, via_saved_states=False, **SHAPE)
+    for other, what in ((b, "checkpoints every 2"), (c, "checkpoints recomputed"), (d, "everything recomputed")):
+        for n in ("dq", "dk", "dv", "deta", "dbeta", "dgamma"):
+            assert np.array_equal(a[n], other[n]), (what, n)
+        for i in range(3):
+            assert np.array_equal(a["dW"][i], other["dW"][i]) and np.array_equal(a["dM"][i], other["dM"][i]), (what, i)
+    # the forward's own results do not depend on whether it also writes the states
+    plain, _ = util.gpu_forward(x4, **SHAPE)
+    saving, _ = util.gpu_forward(x4, save_states=True, **SHAPE)
+    assert np.array_equal(plain["o"], saving["o"]) and all(np.array_equal(p_, q_) for p_, q_ in zip(plain["W"] + plain["M"], saving["W"] + saving["M"]))
 
 
 @pytest.mark.parametrize("C", [16, 32])
