@@ -63,7 +63,7 @@ typedef enum { E2TTT_F32 = 0, E2TTT_BF16 = 1 } e2ttt_dtype;
 /* Which kernel family serves the call.
  *   AUTO    : TCGEN05 where it serves (kind, io_dtype, d, h, C); else TILED for bf16 I/O and SIMT for
  *             fp32 I/O.  The backward has no fused kernel: AUTO and TCGEN05 mean TILED there.
- *             TCGEN05 serves today: GELU-MLP, bf16 I/O, C in {16, 32, 64}, L a multiple of C, d in {64, 128},
+ *             TCGEN05 serves today: GELU-MLP, bf16 I/O, C in {16, 32, 64}, any L (a shorter last chunk), d in {64, 128},
  *             h in {128, 256, 384, 512} (shapes below 128 x 512 and chunks below 64 tokens run zero-padded in
  *             the same tiles); and the SwiGLU forward at d = 128, h = 384, C in {16, 32, 64}, bf16 I/O, without
  *             post-chunk normalisation
@@ -98,7 +98,7 @@ typedef struct {
     int32_t d;        /* head dimension (input and output width of the fast-weight network) */
     int32_t h;        /* hidden width of the fast-weight network */
     int32_t C;        /* chunk size, 1..512 (the paper trains with 512); the fused kernels serve C = 16, 32, 64.
-                         The SIMT path accepts a shorter last chunk. */
+                         Every path accepts a shorter last chunk (L need not be a multiple of C). */
     int32_t kind;     /* e2ttt_kind */
     int32_t io_dtype; /* e2ttt_dtype of q, k, v, o, d_o, dq, dk, dv */
     float ln_eps;     /* layer-norm epsilon (the paper gives none; 1e-5 is the usual default) */

@@ -47,7 +47,7 @@ constexpr size_t kStatusBytes = 256;
 // chunk-start states in the layout the SIMT backward reads)
 int has_tcgen05(const e2ttt_params* p, bool save_states) {
     // chunks of 32 or 16 tokens run in the same 64-row tiles (unused rows zero): half / a quarter of the tile's work is useful
-    if (p->io_dtype != E2TTT_BF16 || (p->C != 64 && p->C != 32 && p->C != 16) || p->L % p->C != 0) return 0;
+    if (p->io_dtype != E2TTT_BF16 || (p->C != 64 && p->C != 32 && p->C != 16)) return 0;
     if (p->kind == E2TTT_MLP_GELU) return (p->d == 128 || p->d == 64) && p->h % 128 == 0 && p->h <= 512;
     // SwiGLU: the fused kernel is built for d = 128, h = 384
     (void)save_states;
@@ -186,7 +186,7 @@ static int fwd_common(const e2ttt_params* p, const void* q, const void* k, const
         t.status = static_cast<int*>(workspace);
         if (save_states) {
             const int seg = segment_chunks(p);
-            const SimtLayout lay = simt_layout(p->d, p->h, p->C, nmat, p->L / p->C, true, true, seg);
+            const SimtLayout lay = simt_layout(p->d, p->h, p->C, nmat, (p->L + p->C - 1) / p->C, true, true, seg);
             t.ckpt = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBytes) + (seg ? lay.cck : lay.ckpt);
             t.ckpt_seq_stride = lay.per_seq;
             t.ckpt_every = seg;
@@ -206,7 +206,7 @@ static int fwd_common(const e2ttt_params* p, const void* q, const void* k, const
         if (row_norm) { t.norm1 = row_norm[0]; t.norm2 = row_norm[1]; t.norm_eps = norm_eps; }
         if (save_states) {
             const int seg = row_norm ? 0 : segment_chunks(p);
-            const SimtLayout lay = simt_layout(p->d, p->h, p->C, nmat, p->L / p->C, true, true, seg);
+            const SimtLayout lay = simt_layout(p->d, p->h, p->C, nmat, (p->L + p->C - 1) / p->C, true, true, seg);
             t.ckpt = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBytes) + (seg ? lay.cck : lay.ckpt);
             t.ckpt_seq_stride = lay.per_seq;
             t.ckpt_every = seg;
@@ -318,7 +318,7 @@ static int bwd_common(const e2ttt_params* p, const void* q, const void* k, const
             const size_t dh = (size_t)p->d * p->h;
             float* wsf = static_cast<float*>(ws_data);
             TcSwigluArgs t{};
-            t.N = p->B * p->H; t.L = n * p->C; t.C = p->C; t.Ls = p->L; t.eps = p->ln_eps;
+            t.N = p->B * p->H; t.L = (int)((size_t)p->L - t0 < (size_t)n * p->C ? (size_t)p->L - t0 : (size_t)n * p->C); t.C = p->C; t.Ls = p->L; t.eps = p->ln_eps;
             t.q = static_cast<const __nv_bfloat16*>(q) + t0 * p->d; t.k = static_cast<const __nv_bfloat16*>(k) + t0 * p->d;
             t.v = static_cast<const __nv_bfloat16*>(v) + t0 * p->d; t.o = nullptr;
             t.eta = eta + t0; t.beta = beta + t0; t.gamma = gamma + t0;
@@ -346,7 +346,7 @@ static int bwd_common(const e2ttt_params* p, const void* q, const void* k, const
             const size_t dh = (size_t)p->d * p->h;
             float* wsf = static_cast<float*>(ws_data);
             TcFwdArgs t{};
-            t.N = p->B * p->H; t.L = n * p->C; t.C = p->C; t.Ls = p->L; t.d = p->d; t.h = p->h; t.eps = p->ln_eps;
+            t.N = p->B * p->H; t.L = (int)((size_t)p->L - t0 < (size_t)n * p->C ? (size_t)p->L - t0 : (size_t)n * p->C); t.C = p->C; t.Ls = p->L; t.d = p->d; t.h = p->h; t.eps = p->ln_eps;
             t.q = static_cast<const __nv_bfloat16*>(q) + t0 * p->d; t.k = static_cast<const __nv_bfloat16*>(k) + t0 * p->d;
             t.v = static_cast<const __nv_bfloat16*>(v) + t0 * p->d; t.o = nullptr;
             t.eta = eta + t0; t.beta = beta + t0; t.gamma = gamma + t0;

@@ -135,7 +135,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     const uint32_t me = cluster_ctarank();
     const int seq = blockIdx.x / NC;
     const int Cr = a.C;  // tokens per chunk (<= C = 64, the tile's rows)
-    const int L = a.L, nchunks = L / Cr;
+    const int L = a.L, nchunks = (L + Cr - 1) / Cr;  // the last chunk may be shorter: its unused rows get zero scalar kernels
     const int Ls = a.Ls;  // sequence stride in tokens
     WaitCtx wc{&s.dead, a.status};
 
@@ -176,7 +176,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         tma_prefetch_desc(&tmV);
     }
     if (warp == 0) { tmem_alloc(&s.tmem_base, 512); tmem_relinquish(); }
-    if (warp == 1) tc_chunk_scalars(eta, beta, gamma, &s.sc[0], Cr);
+    if (warp == 1) tc_chunk_scalars(eta, beta, gamma, &s.sc[0], min(Cr, L));
     if (de < 128)  // the padded half of the token tile is never loaded: zero it once
         for (int i = tid; i < 16384 / 16; i += NTHREADS) reinterpret_cast<uint4*>(s.X[1])[i] = make_uint4(0u, 0u, 0u, 0u);
     if (Cr < C)    // short chunks: the key and query rows past the chunk are never loaded either (128-byte rows, 8 pieces each)
@@ -302,7 +302,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 __syncwarp();
                 if (r + 1 < nchunks) {
                     // scalars of the next chunk (suffix scans over its gates)
-                    tc_chunk_scalars(eta + tok0 + Cr, beta + tok0 + Cr, gamma + tok0 + Cr, &s.sc[(r + 1) & 1], Cr);
+                    tc_chunk_scalars(eta + tok0 + Cr, beta + tok0 + Cr, gamma + tok0 + Cr, &s.sc[(r + 1) & 1], min(Cr, L - tok0 - Cr));
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&s.bar_sc);
                 }
@@ -695,7 +695,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                         const float2 qf = __bfloat1622float2(q2[x]);
                         o32[x] = pack_bf16(qf.x + u[2 * x], qf.y + u[2 * x + 1]);
                     }
-                    if (real && go && t < Cr) *reinterpret_cast<uint4*>(go + off) = ov;
+                    if (real && go && t < min(Cr, L - tok0)) *reinterpret_cast<uint4*>(go + off) = ov;
                 }
             };
 
@@ -1030,7 +1030,7 @@ int tc_fwd_launch(const TcFwdArgs& a_in, void* stream) {
     TcFwdArgs a = a_in;
     if (a.Ls == 0) a.Ls = a.L;
     if (a.C == 0) a.C = C;
-    if ((a.C != 64 && a.C != 32 && a.C != 16) || a.L % a.C != 0) return (int)cudaErrorInvalidValue;
+    if ((a.C != 64 && a.C != 32 && a.C != 16) || a.L <= 0) return (int)cudaErrorInvalidValue;
     if (a.init_seq_stride == 0) a.init_seq_stride = (size_t)a.d * a.h;
     if (a.final_seq_stride == 0) a.final_seq_stride = (size_t)a.d * a.h;
     if (a.Ls < a.L) return (int)cudaErrorInvalidValue;

@@ -104,7 +104,7 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const uint32_t me = cluster_ctarank();
     const int seq = blockIdx.x / NC;
     const int Cr = a.C;  // tokens per chunk (<= C = 64, the tile's rows)
-    const int L = a.L, nchunks = L / Cr;
+    const int L = a.L, nchunks = (L + Cr - 1) / Cr;  // the last chunk may be shorter: its unused rows get zero scalar kernels
     const int Ls = a.Ls;  // sequence stride in tokens
     const int h = NC * HS;
     WaitCtx wc{&s.dead, a.status};
@@ -142,7 +142,7 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         tma_prefetch_desc(&tmV);
     }
     if (warp == 0) { tmem_alloc(&s.tmem_base, 512); tmem_relinquish(); }
-    if (warp == 1) tc_chunk_scalars(eta, beta, gamma, &s.sc[0], Cr);
+    if (warp == 1) tc_chunk_scalars(eta, beta, gamma, &s.sc[0], min(Cr, L));
     if (Cr < C)    // short chunks: the key and query rows past the chunk are never loaded (128-byte rows, 8 pieces each)
         for (int i = tid; i < 32768 / 16; i += NTHREADS)
             if (((i >> 3) & 63) >= Cr) reinterpret_cast<uint4*>(s.X[0])[i] = make_uint4(0u, 0u, 0u, 0u);
@@ -249,7 +249,7 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 }
                 __syncwarp();
                 if (r + 1 < nchunks) {
-                    tc_chunk_scalars(eta + tok0 + Cr, beta + tok0 + Cr, gamma + tok0 + Cr, &s.sc[(r + 1) & 1], Cr);
+                    tc_chunk_scalars(eta + tok0 + Cr, beta + tok0 + Cr, gamma + tok0 + Cr, &s.sc[(r + 1) & 1], min(Cr, L - tok0 - Cr));
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&s.bar_sc);
                 }
@@ -528,7 +528,7 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         }
                         if (lane == 0) mbar_arrive(&s.bar_pu);  // the own rows are in place
                     }
-                } else if (act && t < Cr && go) {
+                } else if (act && t < min(Cr, L - tok0) && go) {
                     // query rows: o = q + y
                     uint4 ov;
                     const float2 q0 = __bfloat1622float2(x2[0]), q1 = __bfloat1622float2(x2[1]), q2 = __bfloat1622float2(x2[2]),
@@ -739,7 +739,7 @@ int tc_swiglu_launch(const TcSwigluArgs& a_in, void* stream) {
     CUtensorMap tmK, tmQ, tmV;
     const size_t rows = (size_t)(a.N - 1) * a.Ls + a.L;  // token rows the maps cover: up to the end of the last sequence's range
     const int Cc = a.C;
-    if ((Cc != 64 && Cc != 32 && Cc != 16) || a.L % Cc != 0) return (int)cudaErrorInvalidValue;
+    if ((Cc != 64 && Cc != 32 && Cc != 16) || a.L <= 0) return (int)cudaErrorInvalidValue;
     if (!make_token_map(&tmK, a.k, rows, (unsigned)Cc, D) || !make_token_map(&tmQ, a.q, rows, (unsigned)Cc, D) || !make_token_map(&tmV, a.v, rows, 16, D))
         return (int)cudaErrorInvalidValue;
     static bool attr_done[64];

@@ -284,3 +284,30 @@ def test_tc_short_chunks_saved_states_feed_the_backward():
     b = util.gpu_backward(x3, via_saved_states=False, **shape)
     for n in ("dq", "dk", "dv", "deta", "dbeta", "dgamma"):
         assert np.array_equal(a[n], b[n]), n
+
+
+@pytest.mark.parametrize("kind,h", [(MLP, 512), (E.E2TTT_SWIGLU, 384)])
+def test_fused_kernels_take_a_shorter_last_chunk(kind, h):
+    """L = 3 chunks + 23 tokens (and a call shorter than one chunk) on both fused kernels against the oracle under the
+    paper's gates; three sequences, so the tiles of a ragged chunk also hold the next sequence's first tokens."""
+    shape = dict(d=128, h=h, C=64, kind=kind, io="bf16")
+    for L in (3 * 64 + 23, 17):
+        r = inputs.paper_regime(inputs.Recipe(B=3, H=1, L=L, d=128, h=h, C=64, kind=kind, io="bf16", seed=21, m_std=0.002))
+        x = inputs.generate(r, with_d_o=True, with_dstate=True)
+        ref = util.oracle_forward(x, 64, kind)
+        got, hd = util.gpu_forward(x, **shape)
+        assert hd["ws"].numel() == 256 and E.e2ttt_device_status(hd["ws"]) == 0      # the fused kernel ran
+        check_forward(got, ref, TOL_BF16, f"fused kernel, ragged L = {L}")
+        tiled, _ = util.gpu_forward(x, impl=E.E2TTT_IMPL_TILED, **shape)
+        assert util.rel_err(got["o"], tiled["o"]) <= TOL_BF16
+    # training flow over the ragged sequence: saved states, checkpoints every 2 chunks, nothing saved: the same bits
+    r = inputs.paper_regime(inputs.Recipe(B=2, H=1, L=3 * 64 + 23, d=128, h=h, C=64, kind=kind, io="bf16", seed=22, m_std=0.002))
+    x = inputs.generate(r, with_d_o=True, with_dstate=True)
+    a = util.gpu_backward(x, via_saved_states=True, **shape)
+    b = util.gpu_backward(x, via_saved_states=True, ckpt_every=2, **shape)
+    c = util.gpu_backward(x, via_saved_states=False, **shape)
+    refb = util.oracle_backward(x, 64, kind)
+    for n in ("dq", "dk", "dv", "deta", "dbeta", "dgamma"):
+        assert np.array_equal(a[n], b[n]) and np.array_equal(a[n], c[n]), n
+    from tests.test_gpu_parity import check_backward
+    check_backward(a, refb, 3 * TOL_BF16, "backward over a ragged sequence from the fused kernel's states")
