@@ -81,3 +81,23 @@ def test_fused_forward_writes_the_checkpoints_and_recomputes_the_segments():
     t = util.gpu_backward(x2, via_saved_states=False, ckpt_every=4, impl=E.E2TTT_IMPL_TILED, **shape)
     for n in GRADS:
         assert util.rel_err(a[n], t[n]) <= 0.15, n   # 8 chunks free-running under the benchmark gates (a chaotic map)
+
+
+def test_padded_shape_short_chunks_ragged_tail_and_checkpoints_together():
+    """Config 1's shape (d = 64, h = 256: the fused kernel's zero-padded instantiation) with chunks of 32 tokens, a
+    ragged last chunk and checkpoints every 2 chunks: forward against the oracle, and the three memory plans of the
+    backward bit for bit."""
+    r = inputs.paper_regime(inputs.Recipe(B=3, H=1, L=5 * 32 + 9, d=64, h=256, C=32, kind=MLP, io="bf16", seed=41, m_std=0.002))
+    x = inputs.generate(r, with_d_o=True, with_dstate=True)
+    shape = dict(d=64, h=256, C=32, kind=MLP, io="bf16")
+    ref = util.oracle_forward(x, 32, MLP)
+    got, hd = util.gpu_forward(x, **shape)
+    assert hd["ws"].numel() == 256 and E.e2ttt_device_status(hd["ws"]) == 0
+    from tests.test_gpu_parity import check_forward
+    check_forward(got, ref, TOL_BF16, "padded shape, C = 32, ragged")
+    a = util.gpu_backward(x, via_saved_states=True, **shape)
+    b = util.gpu_backward(x, via_saved_states=True, ckpt_every=2, **shape)
+    c = util.gpu_backward(x, via_saved_states=False, ckpt_every=4, **shape)
+    same_bits(a, b, "padded: every state vs checkpoints every 2")
+    same_bits(a, c, "padded: every state vs recomputed checkpoints every 4")
+    check_backward(a, util.oracle_backward(x, 32, MLP), 3 * TOL_BF16, "padded shape backward, 6 chunks free-running")
