@@ -101,3 +101,17 @@ def test_padded_shape_short_chunks_ragged_tail_and_checkpoints_together():
     same_bits(a, b, "padded: every state vs checkpoints every 2")
     same_bits(a, c, "padded: every state vs recomputed checkpoints every 4")
     check_backward(a, util.oracle_backward(x, 32, MLP), 3 * TOL_BF16, "padded shape backward, 6 chunks free-running")
+
+
+def test_full_size_training_flow_memory_plans_agree_config2():
+    """The launch configuration bench.py --backward times (B=4, H=16, L=4096, 64 chunks): forward with saved states +
+    backward, with every state kept and with checkpoints every 8 chunks (8 segments, each recomputed by the fused
+    forward): device status clean, gradients finite and the same bits."""
+    r = inputs.config(2)
+    x = inputs.generate(r, with_d_o=True, with_dstate=True)
+    shape = dict(d=r.d, h=r.h, C=r.C, kind=r.kind, io="bf16")
+    a = util.gpu_backward(x, via_saved_states=True, **shape)
+    b = util.gpu_backward(x, via_saved_states=True, ckpt_every=8, **shape)
+    for n in GRADS:
+        assert np.isfinite(a[n]).all(), n
+    same_bits(a, b, "full size: every state kept vs checkpoints every 8")
