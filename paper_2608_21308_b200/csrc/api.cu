@@ -46,9 +46,13 @@ constexpr size_t kStatusBytes = 256;
 // 1 = a tensor-core specialisation exists for these parameters (the forward; with save_states it also writes the
 // chunk-start states in the layout the SIMT backward reads)
 int has_tcgen05(const e2ttt_params* p, bool save_states) {
-    // chunks of 32 or 16 tokens run in the same 64-row tiles (unused rows zero): half / a quarter of the tile's work is useful
-    if (p->io_dtype != E2TTT_BF16 || (p->C != 64 && p->C != 32 && p->C != 16)) return 0;
-    if (p->kind == E2TTT_MLP_GELU) return (p->d == 128 || p->d == 64) && p->h % 128 == 0 && p->h <= 512;
+    // chunks of 32 or 16 tokens run in the same 64-row tiles (unused rows zero): half / a quarter of the tile's work is useful;
+    // the GELU-MLP kernel also runs chunks of 128, 256 or 512 tokens as 2, 4 or 8 blocks of 64
+    if (p->io_dtype != E2TTT_BF16) return 0;
+    const bool small = p->C == 64 || p->C == 32 || p->C == 16;
+    const bool large = p->C == 128 || p->C == 256 || p->C == 512;
+    if (p->kind == E2TTT_MLP_GELU) return (small || large) && (p->d == 128 || p->d == 64) && p->h % 128 == 0 && p->h <= 512;
+    if (!small) return 0;
     // SwiGLU: the fused kernel is built for d = 128, h = 384
     (void)save_states;
     return p->kind == E2TTT_SWIGLU && p->d == 128 && p->h == 384;
@@ -62,7 +66,10 @@ int pick_impl(const e2ttt_params* p, bool save_states, int* impl) {
         if (p->io_dtype != E2TTT_BF16) return E2TTT_ERR_SHAPE;
         *impl = E2TTT_IMPL_TILED;
     } else if (p->impl == E2TTT_IMPL_AUTO) {
-        *impl = has_tcgen05(p, save_states)
+        // Chunks above 64 tokens run on the fused GELU-MLP kernel when asked for (TCGEN05), not by default: its plain bf16
+        // kM pz tile leaves the W1 momentum of long chunks outside the 2e-2 bound when the chunk's gradients cancel
+        // (measured 3-4e-2 at C = 512 under the paper's gates; the any-shape kernels' two-term operands do not).
+        *impl = (has_tcgen05(p, save_states) && p->C <= 64)
                     ? E2TTT_IMPL_TCGEN05
                     : (p->io_dtype == E2TTT_BF16 ? E2TTT_IMPL_TILED : E2TTT_IMPL_SIMT);
     } else {
@@ -130,7 +137,7 @@ int e2ttt_workspace_bytes_normed(const e2ttt_params* p, int save_states, size_t*
     if (!bytes) return E2TTT_ERR_NULL;
     int rc = check_params(p);
     if (rc) return rc;
-    if (p->impl == E2TTT_IMPL_TCGEN05 && !(has_tcgen05(p, false) && p->kind == E2TTT_MLP_GELU)) return E2TTT_ERR_SHAPE;
+    if (p->impl == E2TTT_IMPL_TCGEN05 && !(has_tcgen05(p, false) && p->kind == E2TTT_MLP_GELU && p->C <= 64)) return E2TTT_ERR_SHAPE;
     if (segment_chunks(p)) return E2TTT_ERR_SHAPE;
     *bytes = simt_bytes(p, save_states != 0, save_states != 0, true);
     return E2TTT_OK;
@@ -168,8 +175,8 @@ static int fwd_common(const e2ttt_params* p, const void* q, const void* k, const
     rc = check_device();
     if (rc) return rc;
 
-    if (impl == E2TTT_IMPL_TCGEN05 && p->kind == E2TTT_SWIGLU && row_norm) {
-        // no fused kernel with post-chunk normalisation for SwiGLU: the any-shape kernels serve it
+    if (impl == E2TTT_IMPL_TCGEN05 && row_norm && (p->kind == E2TTT_SWIGLU || p->C > 64)) {
+        // no fused kernel with post-chunk normalisation for SwiGLU or for chunks of several blocks: the any-shape kernels serve it
         if (p->impl == E2TTT_IMPL_TCGEN05) return E2TTT_ERR_SHAPE;
         impl = E2TTT_IMPL_TILED;
     }

@@ -51,7 +51,10 @@ __device__ __forceinline__ ScanMap<float> compose_pinned(const ScanMap<float>& o
     r.X = __fmaf_rn(outer.B, inner.X, __fmul_rn(outer.X, inner.G));
     return r;
 }
-static __device__ void tc_chunk_scalars(const float* eta, const float* beta, const float* gamma, Scalars* out, int len = 64) {
+// `tail` (optional): the composite map of the chunk's tokens behind this block, for chunks of several 64-token blocks;
+// the scalars and, for the chunk's first block, the carries are then those of the whole chunk.
+static __device__ void tc_chunk_scalars(const float* eta, const float* beta, const float* gamma, Scalars* out, int len = 64,
+                                        const ScanMap<float>* tail = nullptr) {
     const int lane = threadIdx.x & 31;
     ScanMap<float> e0, e1, id;
     id.B = 1.0f; id.G = 1.0f; id.X = 0.0f;
@@ -75,6 +78,7 @@ static __device__ void tc_chunk_scalars(const float* eta, const float* beta, con
     excl.G = __shfl_down_sync(0xffffffffu, incl.G, 1);
     excl.X = __shfl_down_sync(0xffffffffu, incl.X, 1);
     if (lane == 31) excl = id;
+    if (tail) excl = compose_pinned(excl, *tail);
     // token index 2l sees the state after tokens 2l+1.., token 2l+1 the state after the later lanes' tokens
     const ScanMap<float> f1 = compose_pinned(loc1, excl);
     const float et0 = in0 ? eta[2 * lane] : 0.0f, et1 = in1 ? eta[2 * lane + 1] : 0.0f;
@@ -88,6 +92,44 @@ static __device__ void tc_chunk_scalars(const float* eta, const float* beta, con
         out->cb = f0.B;
         out->cm = __fmul_rn(e0.B, __fadd_rn(f1.B, f1.X));  // beta_1 S_1
     }
+}
+
+// Composite map of a block of len <= 64 tokens (all of them, first token outermost), the same in every lane.
+static __device__ ScanMap<float> tc_block_composite(const float* beta, const float* gamma, int len) {
+    const int lane = threadIdx.x & 31;
+    ScanMap<float> e0, e1, id;
+    id.B = 1.0f; id.G = 1.0f; id.X = 0.0f;
+    e0 = id; e1 = id;
+    if (2 * lane < len) { e0.B = beta[2 * lane]; e0.G = gamma[2 * lane]; e0.X = e0.G; }
+    if (2 * lane + 1 < len) { e1.B = beta[2 * lane + 1]; e1.G = gamma[2 * lane + 1]; e1.X = e1.G; }
+    ScanMap<float> incl = compose_pinned(e0, e1);
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        ScanMap<float> o;
+        o.B = __shfl_down_sync(0xffffffffu, incl.B, off);
+        o.G = __shfl_down_sync(0xffffffffu, incl.G, off);
+        o.X = __shfl_down_sync(0xffffffffu, incl.X, off);
+        if (lane + off < 32) incl = compose_pinned(incl, o);
+    }
+    ScanMap<float> r;
+    r.B = __shfl_sync(0xffffffffu, incl.B, 0);
+    r.G = __shfl_sync(0xffffffffu, incl.G, 0);
+    r.X = __shfl_sync(0xffffffffu, incl.X, 0);
+    return r;
+}
+// Tails of the blocks of one chunk: tails[j] = composite of the blocks behind block j (identity for the last one).
+// tokens: the chunk's real tokens (<= 64 * nblk).  Called by one converged warp.
+static __device__ void tc_chunk_tails(const float* beta, const float* gamma, int tokens, int nblk, ScanMap<float>* tails) {
+    ScanMap<float> tail;
+    tail.B = 1.0f; tail.G = 1.0f; tail.X = 0.0f;
+    for (int j = nblk - 1; j >= 0; --j) {
+        if ((threadIdx.x & 31) == 0) tails[j] = tail;
+        if (j > 0) {
+            const ScanMap<float> comp = tc_block_composite(beta + 64 * j, gamma + 64 * j, min(64, tokens - 64 * j));
+            tail = compose_pinned(comp, tail);
+        }
+    }
+    __syncwarp();
 }
 
 __device__ __forceinline__ float fast_tanh(float x) {

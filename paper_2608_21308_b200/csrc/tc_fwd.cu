@@ -76,6 +76,7 @@ struct __align__(1024) Smem {
     uint8_t PzM[2][8192];  // kM_t pz                                                 staging slot 1
     uint8_t Stage2[16384]; // staging slot 2
     Scalars sc[2];
+    ScanMap<float> tails[8];  // chunks of several blocks: composite gate map of the chunk's tokens behind each block
     // TMA / loader
     uint64_t bar_x, bar_v, bar_sc;
     // MMA completions (tcgen05.commit)
@@ -120,7 +121,9 @@ __device__ __forceinline__ float gelu_d1_fast(float z) {
 // NORM = true: post-chunk normalisation - after the state transition every row of W1 and of W2 is rescaled to its
 // target norm.  A row of W1c lives in one CTA (its 128 columns spread over the 4 column-group warps); a row of W2
 // spans the 4 CTAs, so its sum of squares crosses the cluster once per chunk.
-template <bool PAD, bool NORM>
+// MULTI: chunks of several 64-token blocks (128, 256, 512 tokens); a compile-time switch, so that the single-block
+// instantiations are exactly the code they were without it
+template <bool PAD, bool NORM, bool MULTI = false>
 __global__ void __launch_bounds__(NTHREADS, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
               const __grid_constant__ CUtensorMap tmV, const TcFwdArgs a) {
@@ -134,8 +137,13 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t me = cluster_ctarank();
     const int seq = blockIdx.x / NC;
-    const int Cr = a.C;  // tokens per chunk (<= C = 64, the tile's rows)
-    const int L = a.L, nchunks = (L + Cr - 1) / Cr;  // the last chunk may be shorter: its unused rows get zero scalar kernels
+    const int Cc = a.C;                     // chunk size
+    const int Cr = min(Cc, C);              // tokens per block (<= C = 64, the tile's rows)
+    const int m = MULTI ? Cc / C : 1;       // 64-token blocks per chunk
+    constexpr bool multi = MULTI;
+    // `nchunks` counts the blocks (= chunks unless a chunk has several); the last one may be shorter: its unused rows
+    // get zero scalar kernels
+    const int L = a.L, nchunks = (L + Cr - 1) / Cr;
     const int Ls = a.Ls;  // sequence stride in tokens
     WaitCtx wc{&s.dead, a.status};
 
@@ -176,7 +184,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         tma_prefetch_desc(&tmV);
     }
     if (warp == 0) { tmem_alloc(&s.tmem_base, 512); tmem_relinquish(); }
-    if (warp == 1) tc_chunk_scalars(eta, beta, gamma, &s.sc[0], min(Cr, L));
+    if (warp == 1) {
+        if (multi) tc_chunk_tails(beta, gamma, min(Cc, L), min(m, nchunks), s.tails);
+        tc_chunk_scalars(eta, beta, gamma, &s.sc[0], min(Cr, L), multi ? &s.tails[0] : nullptr);
+    }
     if (de < 128)  // the padded half of the token tile is never loaded: zero it once
         for (int i = tid; i < 16384 / 16; i += NTHREADS) reinterpret_cast<uint4*>(s.X[1])[i] = make_uint4(0u, 0u, 0u, 0u);
     if (Cr < C)    // short chunks: the key and query rows past the chunk are never loaded either (128-byte rows, 8 pieces each)
@@ -250,12 +261,19 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 mbar_wait(&s.bar_pz, ph, wc, 100 + 8);
                 tc_fence_after_sync();
                 PROF(6);
+                if (multi) {  // several blocks per chunk: the momentum aggregate is read out after every block, the weights' is not
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) umma_bf16_elect(tb + T_R0, dmn(sb + oPzM, 8192, k), dmn(sb + oX, 16384, k), id_agg, k > 0, el);
+                    umma_commit_elect(&s.bar_am1, el);
+                }
 #pragma unroll
                 for (int k = 0; k < 4; ++k) umma_bf16_elect(tb + T_W1, dmn(sb + oPzW, 8192, k), dmn(sb + oX, 16384, k), id_agg, true, el);
                 umma_commit_elect(&s.bar_aw1, el);
+                if (!multi) {
 #pragma unroll
-                for (int k = 0; k < 4; ++k) umma_bf16_elect(tb + T_R0, dmn(sb + oPzM, 8192, k), dmn(sb + oX, 16384, k), id_agg, k > 0, el);
-                umma_commit_elect(&s.bar_am1, el);
+                    for (int k = 0; k < 4; ++k) umma_bf16_elect(tb + T_R0, dmn(sb + oPzM, 8192, k), dmn(sb + oX, 16384, k), id_agg, k > 0, el);
+                    umma_commit_elect(&s.bar_am1, el);
+                }
 #pragma unroll
                 for (int k = 0; k < 4; ++k) umma_bf16_elect(tb + T_R1, dmn(sb + oPu, 8192, k), dmn(sb + oAkM, 8192, k), id_agg, k > 0, el);
                 umma_commit_elect(&s.bar_am2, el);
@@ -302,7 +320,14 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 __syncwarp();
                 if (r + 1 < nchunks) {
                     // scalars of the next chunk (suffix scans over its gates)
-                    tc_chunk_scalars(eta + tok0 + Cr, beta + tok0 + Cr, gamma + tok0 + Cr, &s.sc[(r + 1) & 1], min(Cr, L - tok0 - Cr));
+                    const int tokn = tok0 + Cr;
+                    const ScanMap<float>* tl = nullptr;
+                    if (multi) {
+                        const int bn = (r + 1) % m;  // a chunk's first block: the tails of all its blocks first
+                        if (bn == 0) tc_chunk_tails(beta + tokn, gamma + tokn, min(Cc, L - tokn), min(m, nchunks - r - 1), s.tails);
+                        tl = &s.tails[bn];
+                    }
+                    tc_chunk_scalars(eta + tokn, beta + tokn, gamma + tokn, &s.sc[(r + 1) & 1], min(Cr, L - tokn), tl);
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&s.bar_sc);
                 }
@@ -316,7 +341,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 }
                 if (r + 1 < nchunks) {
                     // the W1 / M1 aggregations were the last readers of the key tile: the next chunk's tokens may land in X
-                    mbar_wait(&s.bar_am1, ph, wc, 100 + 22);
+                    mbar_wait(multi ? &s.bar_aw1 : &s.bar_am1, ph, wc, 100 + 22);  // whichever was issued last
                     if (lane == 0) {
                         mbar_expect_tx(&s.bar_x, (uint32_t)Cr * (de == 128 ? 512u : 256u));
                         const int y2 = seq * Ls + tok0 + Cr;
@@ -368,7 +393,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         // ---- load the state: fp32 master of W -> TMEM (pre-scaled by the first decay carry) and bf16 -> shared; M -> registers
         float M1[CW], M2[CW];
         {
-            const float cw0 = s.sc[0].cw;
+            const float cw0 = s.sc[0].cw, cm0 = s.sc[0].cm;
             const size_t head = (size_t)seq * a.init_seq_stride;
             // W1c[j][i]: global W1 [h][d], row 128 me + j
             const float* w1 = a.W1_init + head + ((size_t)(HC * me) + row) * de + c0;
@@ -388,7 +413,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                     w[j] = x.x; w[j + 1] = x.y; w[j + 2] = x.z; w[j + 3] = x.w;
                 }
 #pragma unroll
-                for (int j = 0; j < 16; ++j) { st[j] = __float_as_uint(cw0 * w[j]); M1[16 * b + j] = (m1 && real1) ? m1[16 * b + j] : 0.0f; }
+                for (int j = 0; j < 16; ++j) {
+                    M1[16 * b + j] = (m1 && real1) ? m1[16 * b + j] : 0.0f;
+                    st[j] = __float_as_uint(multi ? fmaf(cm0, M1[16 * b + j], cw0 * w[j]) : cw0 * w[j]);
+                }
                 tmem_st16(lane_addr + T_W1 + c0 + 16 * b, st);
                 st_slab16(s.W1[(c0 + 16 * b) >> 6], row, (c0 + 16 * b) & 63, w);
                 float* ck = a.ckpt ? a.ckpt + (size_t)seq * a.ckpt_seq_stride : nullptr;  // chunk-start state of chunk 0
@@ -407,7 +435,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                     w[j] = x.x; w[j + 1] = x.y; w[j + 2] = x.z; w[j + 3] = x.w;
                 }
 #pragma unroll
-                for (int j = 0; j < 16; ++j) { st[j] = __float_as_uint(cw0 * w[j]); M2[16 * b + j] = (m2 && real2) ? m2[16 * b + j] : 0.0f; }
+                for (int j = 0; j < 16; ++j) {
+                    M2[16 * b + j] = (m2 && real2) ? m2[16 * b + j] : 0.0f;
+                    st[j] = __float_as_uint(multi ? fmaf(cm0, M2[16 * b + j], cw0 * w[j]) : cw0 * w[j]);
+                }
                 tmem_st16(lane_addr + T_W2 + c0 + 16 * b, st);
                 st_slab16(s.W2[(c0 + 16 * b) >> 6], row, (c0 + 16 * b) & 63, w);
                 if (ck && real2) {
@@ -766,6 +797,108 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             float* ckn = a.ckpt ? a.ckpt + (size_t)seq * a.ckpt_seq_stride + (size_t)((r + 1) / ce) * 4 * dh : nullptr;
             const bool save_ck = a.ckpt && (NORM || !last) && (r + 1) % ce == 0;
 
+            if constexpr (!NORM && MULTI) {
+                // ---- chunks of several 64-token blocks.  Every block's products read the chunk-start weights: the bf16
+                // copies and the pre-scaling of the masters are refreshed after the chunk's last block only.  The master
+                // already holds cw W_0 + cm M_0 (the momentum term was added when it was pre-scaled), so the momentum
+                // registers can follow the blocks: M = cb M_0 + aggregate on the first block, M += aggregate afterwards.
+                const int bidx = r % m;
+                const bool final_block = bidx == m - 1 || last;
+                const float cbk = bidx == 0 ? cb : 1.0f;
+                const float cwn2 = last ? 1.0f : s.sc[(r + 1) & 1].cw, cmn2 = last ? 0.0f : s.sc[(r + 1) & 1].cm;
+                const int cdone = r / m + 1;  // chunks completed after this block (if it is a final one)
+                const bool save2 = a.ckpt && final_block && !last && cdone % ce == 0;
+                float* ck2 = a.ckpt ? a.ckpt + (size_t)seq * a.ckpt_seq_stride + (size_t)(cdone / ce) * 4 * dh : nullptr;
+                const bool wr = final_block && (last || save2);
+                {
+                    const bool real1 = cta_real;
+                    const size_t off0 = ((size_t)(HC * me) + row) * de;
+                    mbar_wait(&s.bar_am1, ph, wc, 100 + 39);
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int b = 0; b < NB; ++b) {
+                        const int col = c0 + 16 * b;
+                        uint32_t ma[16];
+                        tmem_ld16(lane_addr + T_R0 + col, ma);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) M1[16 * b + j] = fmaf(cbk, M1[16 * b + j], __uint_as_float(ma[j]));
+                        if (wr && real1 && col < de) {
+                            float* dst = (last ? a.M1_final + head : ck2 + 2 * dh) + off0 + col;
+#pragma unroll
+                            for (int j = 0; j < 16; j += 4)
+                                *reinterpret_cast<float4*>(dst + j) = make_float4(M1[16 * b + j], M1[16 * b + j + 1], M1[16 * b + j + 2], M1[16 * b + j + 3]);
+                        }
+                    }
+                    if (final_block) {
+                        mbar_wait(&s.bar_aw1, ph, wc, 100 + 38);
+                        tc_fence_after_sync();
+#pragma unroll
+                        for (int b = 0; b < NB; ++b) {
+                            const int col = c0 + 16 * b;
+                            uint32_t wa[16];
+                            tmem_ld16(lane_addr + T_W1 + col, wa);
+                            tmem_wait_ld();
+                            uint32_t p[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) p[i] = pack_bf16(__uint_as_float(wa[2 * i]), __uint_as_float(wa[2 * i + 1]));
+                            st_slab16p(s.W1[col >> 6], row, col & 63, p);
+                            if (wr && real1 && col < de) {
+                                float* dst = (last ? a.W1_final + head : ck2) + off0 + col;
+#pragma unroll
+                                for (int j = 0; j < 16; j += 4)
+                                    *reinterpret_cast<uint4*>(dst + j) = make_uint4(wa[j], wa[j + 1], wa[j + 2], wa[j + 3]);
+                            }
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) wa[j] = __float_as_uint(fmaf(cmn2, M1[16 * b + j], cwn2 * __uint_as_float(wa[j])));
+                            tmem_st16(lane_addr + T_W1 + col, wa);
+                        }
+                    }
+                    tmem_wait_st();
+                    warp_release(&s.bar_w1);  // R0 free (and, after a final block, W1 refreshed): the next block's G1 may run
+                }
+                {
+                    const bool real2 = cta_real && row < de;
+                    const size_t off0 = (size_t)row * he + HC * me;
+                    mbar_wait(&s.bar_am2, ph, wc, 100 + 40);
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int b = 0; b < NB; ++b) {
+                        const int col = c0 + 16 * b;
+                        uint32_t ma[16];
+                        tmem_ld16(lane_addr + T_R1 + col, ma);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) M2[16 * b + j] = fmaf(cbk, M2[16 * b + j], __uint_as_float(ma[j]));
+                        if (wr && real2) {
+                            float* dst = (last ? a.M2_final + head : ck2 + 3 * dh) + off0 + col;
+#pragma unroll
+                            for (int j = 0; j < 16; j += 4)
+                                *reinterpret_cast<float4*>(dst + j) = make_float4(M2[16 * b + j], M2[16 * b + j + 1], M2[16 * b + j + 2], M2[16 * b + j + 3]);
+                        }
+                        if (final_block) {
+                            uint32_t wa[16];
+                            tmem_ld16(lane_addr + T_W2 + col, wa);
+                            tmem_wait_ld();
+                            uint32_t p[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) p[i] = pack_bf16(__uint_as_float(wa[2 * i]), __uint_as_float(wa[2 * i + 1]));
+                            st_slab16p(s.W2[col >> 6], row, col & 63, p);
+                            if (wr && real2) {
+                                float* dst = (last ? a.W2_final + head : ck2 + dh) + off0 + col;
+#pragma unroll
+                                for (int j = 0; j < 16; j += 4)
+                                    *reinterpret_cast<uint4*>(dst + j) = make_uint4(wa[j], wa[j + 1], wa[j + 2], wa[j + 3]);
+                            }
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) wa[j] = __float_as_uint(fmaf(cmn2, M2[16 * b + j], cwn2 * __uint_as_float(wa[j])));
+                            tmem_st16(lane_addr + T_W2 + col, wa);
+                        }
+                    }
+                    tmem_wait_st();
+                    warp_release(&s.bar_w2);  // R1 free (and, after a final block, W2 refreshed)
+                }
+            } else {
             // W1 half, as soon as the W1 aggregation is in (the momentum aggregate follows right behind it)
             mbar_wait(&s.bar_aw1, ph, wc, 100 + 38);
             tc_fence_after_sync();
@@ -1004,6 +1137,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 tmem_wait_st();
                 warp_release(&s.bar_w2);  // bf16 W2 complete, master rescaled, R1 free: the next chunk's G2 may run
             }
+            }  // single-block chunks
             PROF(12);
         }
     }
@@ -1030,14 +1164,16 @@ int tc_fwd_launch(const TcFwdArgs& a_in, void* stream) {
     TcFwdArgs a = a_in;
     if (a.Ls == 0) a.Ls = a.L;
     if (a.C == 0) a.C = C;
-    if ((a.C != 64 && a.C != 32 && a.C != 16) || a.L <= 0) return (int)cudaErrorInvalidValue;
+    if ((a.C != 512 && a.C != 256 && a.C != 128 && a.C != 64 && a.C != 32 && a.C != 16) || a.L <= 0) return (int)cudaErrorInvalidValue;
+    if (a.C > 64 && a.norm1) return (int)cudaErrorInvalidValue;
     if (a.init_seq_stride == 0) a.init_seq_stride = (size_t)a.d * a.h;
     if (a.final_seq_stride == 0) a.final_seq_stride = (size_t)a.d * a.h;
     if (a.Ls < a.L) return (int)cudaErrorInvalidValue;
     CUtensorMap tmK, tmQ, tmV;
     // token rows the maps cover: up to the end of the last sequence's range
     const size_t rows = (size_t)(a.N - 1) * a.Ls + a.L;
-    if (!make_token_map(&tmK, a.k, rows, (unsigned)a.C, a.d) || !make_token_map(&tmQ, a.q, rows, (unsigned)a.C, a.d) ||
+    const unsigned box_rows = (unsigned)(a.C < 64 ? a.C : 64);
+    if (!make_token_map(&tmK, a.k, rows, box_rows, a.d) || !make_token_map(&tmQ, a.q, rows, box_rows, a.d) ||
         !make_token_map(&tmV, a.v, rows, 16, a.d))
         return (int)cudaErrorInvalidValue;
     static bool attr_done[64];
@@ -1049,6 +1185,8 @@ int tc_fwd_launch(const TcFwdArgs& a_in, void* stream) {
         if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_fwd_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_fwd_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_fwd_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_fwd_kernel<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_fwd_kernel<true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return (int)e;
         if (dev >= 0 && dev < 64) attr_done[dev] = true;
     }
@@ -1073,8 +1211,12 @@ int tc_fwd_launch(const TcFwdArgs& a_in, void* stream) {
         e = native ? cudaLaunchKernelEx(&cfg, tc_fwd_kernel<false, true>, tmK, tmQ, tmV, a)
                    : cudaLaunchKernelEx(&cfg, tc_fwd_kernel<true, true>, tmK, tmQ, tmV, a);
     } else {
-        e = native ? cudaLaunchKernelEx(&cfg, tc_fwd_kernel<false, false>, tmK, tmQ, tmV, a)
-                   : cudaLaunchKernelEx(&cfg, tc_fwd_kernel<true, false>, tmK, tmQ, tmV, a);
+        if (a.C > 64)
+            e = native ? cudaLaunchKernelEx(&cfg, tc_fwd_kernel<false, false, true>, tmK, tmQ, tmV, a)
+                       : cudaLaunchKernelEx(&cfg, tc_fwd_kernel<true, false, true>, tmK, tmQ, tmV, a);
+        else
+            e = native ? cudaLaunchKernelEx(&cfg, tc_fwd_kernel<false, false>, tmK, tmQ, tmV, a)
+                       : cudaLaunchKernelEx(&cfg, tc_fwd_kernel<true, false>, tmK, tmQ, tmV, a);
     }
     if (e != cudaSuccess) return (int)e;
     return (int)cudaGetLastError();
