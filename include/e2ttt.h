@@ -68,7 +68,7 @@ typedef enum { E2TTT_F32 = 0, E2TTT_BF16 = 1 } e2ttt_dtype;
  *             the same tiles); and the SwiGLU forward at d = 128, h = 384, C in {16, 32, 64}, bf16 I/O, without
  *             post-chunk normalisation.  Asked for with TCGEN05 (not chosen by AUTO), the GELU-MLP kernel also
  *             runs chunks of 128, 256 and 512 tokens (the paper's chunk size) as 2, 4, 8 blocks of 64 at the
- *             chunk-start weights; its plain bf16 operand tiles then leave the W1 momentum outside the 2e-2
+ *             chunk-start weights; its plain bf16 operands then leave the W1 momentum outside the 2e-2
  *             bound when the gradients of a long chunk cancel (3-4e-2 measured at C = 512)
  *             (its gate / up projection reads the fast weights as two bf16 terms: a plain bf16 copy leaves
  *             some chunks outside the 2e-2 parity bound, the product z1 z2 multiplies the rounding up).

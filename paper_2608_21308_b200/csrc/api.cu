@@ -67,7 +67,7 @@ int pick_impl(const e2ttt_params* p, bool save_states, int* impl) {
         *impl = E2TTT_IMPL_TILED;
     } else if (p->impl == E2TTT_IMPL_AUTO) {
         // Chunks above 64 tokens run on the fused GELU-MLP kernel when asked for (TCGEN05), not by default: its plain bf16
-        // kM pz tile leaves the W1 momentum of long chunks outside the 2e-2 bound when the chunk's gradients cancel
+        // operands leave the W1 momentum of long chunks outside the 2e-2 bound when the chunk's gradients cancel
         // (measured 3-4e-2 at C = 512 under the paper's gates; the any-shape kernels' two-term operands do not).
         *impl = (has_tcgen05(p, save_states) && p->C <= 64)
                     ? E2TTT_IMPL_TCGEN05

@@ -321,8 +321,8 @@ def test_tc_large_chunks_against_the_oracle(C):
     oracle's state under the benchmark gates, a free-running run under the paper's gate regime with a ragged tail (the
     last chunk has fewer blocks, the last block fewer tokens), split calls chain bitwise at a chunk boundary, and the
     any-shape kernels beside it.  Everything is held to 2e-2 except the W1 momentum of the free-running run at C = 512:
-    under these gates the momentum shrinks to ~5e-4 while the per-token terms of its sum do not, and the plain bf16
-    kM pz tile leaves an absolute error of ~1.5e-5 (2.9e-2 of max|M1|; the any-shape kernels, with two-term operands,
+    under these gates the momentum shrinks to ~5e-4 while the per-token terms of its sum do not, and their bf16-sized
+    errors leave an absolute error of ~1.5e-5 (2.9e-2 of max|M1|; the any-shape kernels, with two-term operands,
     show none).  That is why AUTO does not select the fused kernel for these chunk sizes."""
     shape = dict(d=128, h=512, C=C, kind=MLP, io="bf16")
     r = inputs.config(2, heads=[5, 33], C=C, m_std=0.002)
