@@ -371,3 +371,15 @@ def test_tc_large_chunks_training_flow():
     for n in ("dq", "dk", "dv", "deta", "dbeta", "dgamma"):
         assert np.array_equal(a[n], b[n]) and np.array_equal(a[n], c[n]), n
     check_backward(a, util.oracle_backward(x, C, MLP), 3 * TOL_BF16, "C = 128 backward from the fused kernel's states, 6 chunks")
+
+
+@pytest.mark.parametrize("C,L", [(512, 100), (512, 192), (256, 17), (128, 129), (512, 513)])
+def test_tc_large_chunks_sequences_shorter_than_a_chunk_or_just_past_one(C, L):
+    """Fewer blocks than a chunk has, a single short block, one token past a block and one token past a chunk."""
+    shape = dict(d=128, h=512, C=C, kind=MLP, io="bf16")
+    rp = inputs.paper_regime(inputs.Recipe(B=2, H=1, L=L, d=128, h=512, C=C, kind=MLP, io="bf16", seed=3, m_std=0.002))
+    x = inputs.generate(rp)
+    ref = util.oracle_forward(x, C, MLP)
+    got, hd = util.gpu_forward(x, impl=E.E2TTT_IMPL_TCGEN05, **shape)
+    assert hd["ws"].numel() == 256 and E.e2ttt_device_status(hd["ws"]) == 0
+    check_forward(got, ref, TOL_BF16, f"fused kernel, C = {C}, L = {L}")
