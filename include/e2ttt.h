@@ -66,9 +66,9 @@ typedef enum { E2TTT_F32 = 0, E2TTT_BF16 = 1 } e2ttt_dtype;
  *             TCGEN05 serves today: GELU-MLP, bf16 I/O, C in {16, 32, 64}, any L (a shorter last chunk), d in {64, 128},
  *             h in {128, 256, 384, 512} (shapes below 128 x 512 and chunks below 64 tokens run zero-padded in
  *             the same tiles); and the SwiGLU forward at d = 128, h = 384, C in {16, 32, 64}, bf16 I/O, without
- *             post-chunk normalisation.  Asked for with TCGEN05 (not chosen by AUTO), the GELU-MLP kernel also
- *             runs chunks of 128, 256 and 512 tokens (the paper's chunk size) as 2, 4, 8 blocks of 64 at the
- *             chunk-start weights; its plain bf16 operands then leave the W1 momentum outside the 2e-2
+ *             post-chunk normalisation.  Asked for with TCGEN05 (not chosen by AUTO), both kernels also
+ *             run chunks of 128, 256 and 512 tokens (the paper's chunk size) as 2, 4, 8 blocks of 64 at the
+ *             chunk-start weights; the GELU-MLP kernel's plain bf16 operands then leave the W1 momentum outside the 2e-2
  *             bound when the gradients of a long chunk cancel (3-4e-2 measured at C = 512)
  *             (its gate / up projection reads the fast weights as two bf16 terms: a plain bf16 copy leaves
  *             some chunks outside the 2e-2 parity bound, the product z1 z2 multiplies the rounding up).
@@ -101,7 +101,7 @@ typedef struct {
     int32_t d;        /* head dimension (input and output width of the fast-weight network) */
     int32_t h;        /* hidden width of the fast-weight network */
     int32_t C;        /* chunk size, 1..512 (the paper trains with 512); the fused kernels serve C = 16, 32, 64
-                         (and 128, 256, 512 for the GELU-MLP on request).
+                         (and 128, 256, 512 on request).
                          Every path accepts a shorter last chunk (L need not be a multiple of C). */
     int32_t kind;     /* e2ttt_kind */
     int32_t io_dtype; /* e2ttt_dtype of q, k, v, o, d_o, dq, dk, dv */

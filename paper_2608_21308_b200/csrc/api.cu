@@ -47,15 +47,14 @@ constexpr size_t kStatusBytes = 256;
 // chunk-start states in the layout the SIMT backward reads)
 int has_tcgen05(const e2ttt_params* p, bool save_states) {
     // chunks of 32 or 16 tokens run in the same 64-row tiles (unused rows zero): half / a quarter of the tile's work is useful;
-    // the GELU-MLP kernel also runs chunks of 128, 256 or 512 tokens as 2, 4 or 8 blocks of 64
+    // both kernels also run chunks of 128, 256 or 512 tokens as 2, 4 or 8 blocks of 64 (on request, see pick_impl)
     if (p->io_dtype != E2TTT_BF16) return 0;
     const bool small = p->C == 64 || p->C == 32 || p->C == 16;
     const bool large = p->C == 128 || p->C == 256 || p->C == 512;
     if (p->kind == E2TTT_MLP_GELU) return (small || large) && (p->d == 128 || p->d == 64) && p->h % 128 == 0 && p->h <= 512;
-    if (!small) return 0;
     // SwiGLU: the fused kernel is built for d = 128, h = 384
     (void)save_states;
-    return p->kind == E2TTT_SWIGLU && p->d == 128 && p->h == 384;
+    return (small || large) && p->kind == E2TTT_SWIGLU && p->d == 128 && p->h == 384;
 }
 
 int pick_impl(const e2ttt_params* p, bool save_states, int* impl) {
@@ -66,7 +65,7 @@ int pick_impl(const e2ttt_params* p, bool save_states, int* impl) {
         if (p->io_dtype != E2TTT_BF16) return E2TTT_ERR_SHAPE;
         *impl = E2TTT_IMPL_TILED;
     } else if (p->impl == E2TTT_IMPL_AUTO) {
-        // Chunks above 64 tokens run on the fused GELU-MLP kernel when asked for (TCGEN05), not by default: its plain bf16
+        // Chunks above 64 tokens run on the fused kernels when asked for (TCGEN05), not by default: their plain bf16
         // operands leave the W1 momentum of long chunks outside the 2e-2 bound when the chunk's gradients cancel
         // (measured 3-4e-2 at C = 512 under the paper's gates; the any-shape kernels' two-term operands do not).
         *impl = (has_tcgen05(p, save_states) && p->C <= 64)

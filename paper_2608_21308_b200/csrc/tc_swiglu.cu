@@ -64,6 +64,7 @@ struct __align__(1024) Smem {
     uint8_t StageQ[NC - 1][4096];  // the peers' bf16 partial sums of the owned query rows
     uint8_t Vrows[4096];     // value rows of the owned key tokens (TMA, 16 rows)
     Scalars sc[2];
+    ScanMap<float> tails[8];  // chunks of several blocks: composite gate map of the chunk's tokens behind each block
     uint64_t bar_x, bar_v, bar_sc;
     uint64_t bar_g1, bar_g2, bar_g3, bar_aw12, bar_am12, bar_am3;
     uint64_t bar_a, bar_ak, bar_pz, bar_r1, bar_w12, bar_w3;
@@ -90,6 +91,8 @@ __device__ __forceinline__ void st_two_term(uint8_t* hi_slab, uint8_t* lo_slab, 
 // sigmoid by the hardware tanh: s(z) = 0.5 + 0.5 tanh(z / 2)
 __device__ __forceinline__ float fast_sigmoid(float z) { return fmaf(0.5f, fast_tanh(0.5f * z), 0.5f); }
 
+// MULTI: chunks of several 64-token blocks (128, 256, 512 tokens), a compile-time switch
+template <bool MULTI>
 __global__ void __launch_bounds__(NTHREADS, 1)
 tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
                  const __grid_constant__ CUtensorMap tmV, const TcSwigluArgs a) {
@@ -103,8 +106,12 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t me = cluster_ctarank();
     const int seq = blockIdx.x / NC;
-    const int Cr = a.C;  // tokens per chunk (<= C = 64, the tile's rows)
-    const int L = a.L, nchunks = (L + Cr - 1) / Cr;  // the last chunk may be shorter: its unused rows get zero scalar kernels
+    const int Cc = a.C;                     // chunk size
+    const int Cr = min(Cc, C);              // tokens per block (<= C = 64, the tile's rows)
+    const int m = MULTI ? Cc / C : 1;       // 64-token blocks per chunk
+    constexpr bool multi = MULTI;
+    // `nchunks` counts the blocks (= chunks unless a chunk has several); the last one may be shorter
+    const int L = a.L, nchunks = (L + Cr - 1) / Cr;
     const int Ls = a.Ls;  // sequence stride in tokens
     const int h = NC * HS;
     WaitCtx wc{&s.dead, a.status};
@@ -142,7 +149,10 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         tma_prefetch_desc(&tmV);
     }
     if (warp == 0) { tmem_alloc(&s.tmem_base, 512); tmem_relinquish(); }
-    if (warp == 1) tc_chunk_scalars(eta, beta, gamma, &s.sc[0], min(Cr, L));
+    if (warp == 1) {
+        if (multi) tc_chunk_tails(beta, gamma, min(Cc, L), min(m, nchunks), s.tails);
+        tc_chunk_scalars(eta, beta, gamma, &s.sc[0], min(Cr, L), multi ? &s.tails[0] : nullptr);
+    }
     if (Cr < C)    // short chunks: the key and query rows past the chunk are never loaded (128-byte rows, 8 pieces each)
         for (int i = tid; i < 32768 / 16; i += NTHREADS)
             if (((i >> 3) & 63) >= Cr) reinterpret_cast<uint4*>(s.X[0])[i] = make_uint4(0u, 0u, 0u, 0u);
@@ -206,12 +216,19 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 // W12 aggregation first (the next chunk's G1 hangs on it), then the two momentum aggregates
                 mbar_wait(&s.bar_pz, ph, wc, 300 + 8);
                 tc_fence_after_sync();
+                if (multi) {  // the momentum aggregate is read out after every block, the weights' only after the chunk's last
+#pragma unroll kIssueUnroll
+                    for (int k = 0; k < 4; ++k) umma_bf16_elect(tb + T_R0, dmn(sb + oPzM, 8192, k), dmn(sb + oX, 16384, k), id_agg, k > 0, el);
+                    umma_commit_elect(&s.bar_am12, el);
+                }
 #pragma unroll kIssueUnroll
                 for (int k = 0; k < 4; ++k) umma_bf16_elect(tb + T_W12, dmn(sb + oPzW, 8192, k), dmn(sb + oX, 16384, k), id_agg, true, el);
                 umma_commit_elect(&s.bar_aw12, el);
+                if (!multi) {
 #pragma unroll kIssueUnroll
-                for (int k = 0; k < 4; ++k) umma_bf16_elect(tb + T_R0, dmn(sb + oPzM, 8192, k), dmn(sb + oX, 16384, k), id_agg, k > 0, el);
-                umma_commit_elect(&s.bar_am12, el);
+                    for (int k = 0; k < 4; ++k) umma_bf16_elect(tb + T_R0, dmn(sb + oPzM, 8192, k), dmn(sb + oX, 16384, k), id_agg, k > 0, el);
+                    umma_commit_elect(&s.bar_am12, el);
+                }
 #pragma unroll kIssueUnroll
                 for (int k = 0; k < 4; ++k) umma_bf16_elect(tb + T_R1, dmn(sb + oPu, 8192, k), dmn(sb + oHdM, 8192, k), id_agg64, k > 0, el);
                 umma_commit_elect(&s.bar_am3, el);
@@ -249,7 +266,14 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 }
                 __syncwarp();
                 if (r + 1 < nchunks) {
-                    tc_chunk_scalars(eta + tok0 + Cr, beta + tok0 + Cr, gamma + tok0 + Cr, &s.sc[(r + 1) & 1], min(Cr, L - tok0 - Cr));
+                    const int tokn = tok0 + Cr;
+                    const ScanMap<float>* tl = nullptr;
+                    if (multi) {
+                        const int bn = (r + 1) % m;  // a chunk's first block: the tails of all its blocks first
+                        if (bn == 0) tc_chunk_tails(beta + tokn, gamma + tokn, min(Cc, L - tokn), min(m, nchunks - r - 1), s.tails);
+                        tl = &s.tails[bn];
+                    }
+                    tc_chunk_scalars(eta + tokn, beta + tokn, gamma + tokn, &s.sc[(r + 1) & 1], min(Cr, L - tokn), tl);
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&s.bar_sc);
                 }
@@ -262,7 +286,7 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 }
                 if (r + 1 < nchunks) {
                     // the W12 / M12 aggregations were the last readers of the key tile: the next chunk's tokens may land in X
-                    mbar_wait(&s.bar_am12, ph, wc, 300 + 22);
+                    mbar_wait(multi ? &s.bar_aw12 : &s.bar_am12, ph, wc, 300 + 22);  // whichever was issued last
                     if (lane == 0) load_tokens(seq * Ls + tok0 + Cr);
                     // every reader of this chunk's staging / pu / scaled tiles is done once the aggregations have completed and
                     // every epilogue warp has left its layer norm (it has then released W12): credits to and from the peers
@@ -298,7 +322,7 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         // ---- load the state: fp32 masters -> TMEM (pre-scaled by the first decay carry), bf16 copies -> shared, M -> registers
         float M12[32], M3[16];
         {
-            const float cw0 = s.sc[0].cw;
+            const float cw0 = s.sc[0].cw, cm0 = s.sc[0].cm;
             const float* w12 = (row < 64 ? a.W1_init : a.W2_init) + head0 + off12;
             const float* m12p = row < 64 ? a.M1_init : a.M2_init;
             const float* m12 = m12p ? m12p + head0 + off12 : nullptr;
@@ -312,7 +336,10 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     w[j] = x.x; w[j + 1] = x.y; w[j + 2] = x.z; w[j + 3] = x.w;
                 }
 #pragma unroll
-                for (int j = 0; j < 16; ++j) { st[j] = __float_as_uint(cw0 * w[j]); M12[16 * b + j] = m12 ? m12[16 * b + j] : 0.0f; }
+                for (int j = 0; j < 16; ++j) {
+                    M12[16 * b + j] = m12 ? m12[16 * b + j] : 0.0f;
+                    st[j] = __float_as_uint(multi ? fmaf(cm0, M12[16 * b + j], cw0 * w[j]) : cw0 * w[j]);
+                }
                 const int col = 32 * g + 16 * b;
                 tmem_st16(lane_addr + T_W12 + col, st);
                 uint32_t wu[16];
@@ -340,7 +367,10 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     w[j] = x.x; w[j + 1] = x.y; w[j + 2] = x.z; w[j + 3] = x.w;
                 }
 #pragma unroll
-                for (int j = 0; j < 16; ++j) { st[j] = __float_as_uint(cw0 * w[j]); M3[j] = m3 ? m3[j] : 0.0f; }
+                for (int j = 0; j < 16; ++j) {
+                    M3[j] = m3 ? m3[j] : 0.0f;
+                    st[j] = __float_as_uint(multi ? fmaf(cm0, M3[j], cw0 * w[j]) : cw0 * w[j]);
+                }
                 tmem_st16(lane_addr + T_W3 + 16 * g, st);
                 st_slab16(s.W3, row, 16 * g, w);
                 if (ck0) {
@@ -640,6 +670,90 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             const int ce = max(a.ckpt_every, 1);
             float* const ckn = ck0 ? ck0 + (size_t)((r + 1) / ce) * 6 * dh : nullptr;
             const bool save_ck = ck0 && !last && (r + 1) % ce == 0;
+            if constexpr (MULTI) {
+                // ---- chunks of several 64-token blocks (see the GELU-MLP kernel): the bf16 copies and the masters' pre-scaling
+                // are refreshed after the chunk's last block only; the master carries cw W_0 + cm M_0, so the momentum
+                // registers follow the blocks (M = cb M_0 + aggregate on the first block, M += aggregate afterwards).
+                const int bidx = r % m;
+                const bool final_block = bidx == m - 1 || last;
+                const float cbk = bidx == 0 ? cb : 1.0f;
+                const float cwn2 = last ? 1.0f : s.sc[(r + 1) & 1].cw, cmn2 = last ? 0.0f : s.sc[(r + 1) & 1].cm;
+                const int cdone = r / m + 1;
+                const bool save2 = ck0 && final_block && !last && cdone % ce == 0;
+                float* const ck2 = ck0 ? ck0 + (size_t)(cdone / ce) * 6 * dh : nullptr;
+                const bool wr = final_block && (last || save2);
+                mbar_wait(&s.bar_am12, ph, wc, 300 + 39);
+                tc_fence_after_sync();
+#pragma unroll
+                for (int b = 0; b < 2; ++b) {
+                    uint32_t ma[16];
+                    tmem_ld16(lane_addr + T_R0 + 32 * g + 16 * b, ma);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) M12[16 * b + j] = fmaf(cbk, M12[16 * b + j], __uint_as_float(ma[j]));
+                    if (wr) {
+                        float* dst = (last ? (row < 64 ? a.M1_final : a.M2_final) + head : ck2 + (row < 64 ? 3 : 4) * dh) + off12 + 16 * b;
+#pragma unroll
+                        for (int j = 0; j < 16; j += 4)
+                            *reinterpret_cast<float4*>(dst + j) = make_float4(M12[16 * b + j], M12[16 * b + j + 1], M12[16 * b + j + 2], M12[16 * b + j + 3]);
+                    }
+                }
+                if (final_block) {
+                    mbar_wait(&s.bar_aw12, ph, wc, 300 + 38);
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int b = 0; b < 2; ++b) {
+                        const int col = 32 * g + 16 * b;
+                        uint32_t wa[16];
+                        tmem_ld16(lane_addr + T_W12 + col, wa);
+                        tmem_wait_ld();
+                        st_two_term(s.W12[col >> 6], s.W12lo[col >> 6], row, col & 63, wa);
+                        if (wr) {
+                            float* dst = (last ? (row < 64 ? a.W1_final : a.W2_final) + head : ck2 + (row < 64 ? 0 : dh)) + off12 + 16 * b;
+#pragma unroll
+                            for (int j = 0; j < 16; j += 4) *reinterpret_cast<uint4*>(dst + j) = make_uint4(wa[j], wa[j + 1], wa[j + 2], wa[j + 3]);
+                        }
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) wa[j] = __float_as_uint(fmaf(cmn2, M12[16 * b + j], cwn2 * __uint_as_float(wa[j])));
+                        tmem_st16(lane_addr + T_W12 + col, wa);
+                    }
+                }
+                tmem_wait_st();
+                warp_release(&s.bar_w12);  // R0 free (and, after a final block, W12 refreshed)
+                mbar_wait(&s.bar_am3, ph, wc, 300 + 40);
+                tc_fence_after_sync();
+                {
+                    uint32_t ma[16];
+                    tmem_ld16(lane_addr + T_R1 + 16 * g, ma);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) M3[j] = fmaf(cbk, M3[j], __uint_as_float(ma[j]));
+                    if (wr) {
+                        float* dst = (last ? a.M3_final + head : ck2 + 5 * dh) + off3;
+#pragma unroll
+                        for (int j = 0; j < 16; j += 4) *reinterpret_cast<float4*>(dst + j) = make_float4(M3[j], M3[j + 1], M3[j + 2], M3[j + 3]);
+                    }
+                    if (final_block) {
+                        uint32_t wa[16];
+                        tmem_ld16(lane_addr + T_W3 + 16 * g, wa);
+                        tmem_wait_ld();
+                        uint32_t p[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) p[i] = pack_bf16(__uint_as_float(wa[2 * i]), __uint_as_float(wa[2 * i + 1]));
+                        st_slab16p(s.W3, row, 16 * g, p);
+                        if (wr) {
+                            float* dst = (last ? a.W3_final + head : ck2 + 2 * dh) + off3;
+#pragma unroll
+                            for (int j = 0; j < 16; j += 4) *reinterpret_cast<uint4*>(dst + j) = make_uint4(wa[j], wa[j + 1], wa[j + 2], wa[j + 3]);
+                        }
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) wa[j] = __float_as_uint(fmaf(cmn2, M3[j], cwn2 * __uint_as_float(wa[j])));
+                        tmem_st16(lane_addr + T_W3 + 16 * g, wa);
+                    }
+                }
+                tmem_wait_st();
+                warp_release(&s.bar_w3);  // R1 free (and, after a final block, W3 refreshed)
+            } else {
             // W12 half, as soon as its aggregation is in (the momentum aggregate follows right behind it)
             mbar_wait(&s.bar_aw12, ph, wc, 300 + 38);
             tc_fence_after_sync();
@@ -714,6 +828,7 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             }
             tmem_wait_st();
             warp_release(&s.bar_w3);  // bf16 W3 complete, master rescaled, R1 free: the next chunk's G2 may run
+            }  // single-block chunks
         }
     }
 
@@ -739,15 +854,17 @@ int tc_swiglu_launch(const TcSwigluArgs& a_in, void* stream) {
     CUtensorMap tmK, tmQ, tmV;
     const size_t rows = (size_t)(a.N - 1) * a.Ls + a.L;  // token rows the maps cover: up to the end of the last sequence's range
     const int Cc = a.C;
-    if ((Cc != 64 && Cc != 32 && Cc != 16) || a.L <= 0) return (int)cudaErrorInvalidValue;
-    if (!make_token_map(&tmK, a.k, rows, (unsigned)Cc, D) || !make_token_map(&tmQ, a.q, rows, (unsigned)Cc, D) || !make_token_map(&tmV, a.v, rows, 16, D))
+    if ((Cc != 512 && Cc != 256 && Cc != 128 && Cc != 64 && Cc != 32 && Cc != 16) || a.L <= 0) return (int)cudaErrorInvalidValue;
+    const unsigned box_rows = (unsigned)(Cc < 64 ? Cc : 64);
+    if (!make_token_map(&tmK, a.k, rows, box_rows, D) || !make_token_map(&tmQ, a.q, rows, box_rows, D) || !make_token_map(&tmV, a.v, rows, 16, D))
         return (int)cudaErrorInvalidValue;
     static bool attr_done[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return (int)cudaGetLastError();
     const int smem = (int)tc_swiglu_smem_bytes();
     if (dev < 0 || dev >= 64 || !attr_done[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(tc_swiglu_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        cudaError_t e = cudaFuncSetAttribute(tc_swiglu_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_swiglu_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return (int)e;
         if (dev >= 0 && dev < 64) attr_done[dev] = true;
     }
@@ -765,7 +882,8 @@ int tc_swiglu_launch(const TcSwigluArgs& a_in, void* stream) {
     at[0].val.clusterDim.z = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    e = cudaLaunchKernelEx(&cfg, tc_swiglu_kernel, tmK, tmQ, tmV, a);
+    e = a.C > 64 ? cudaLaunchKernelEx(&cfg, tc_swiglu_kernel<true>, tmK, tmQ, tmV, a)
+                 : cudaLaunchKernelEx(&cfg, tc_swiglu_kernel<false>, tmK, tmQ, tmV, a);
     if (e != cudaSuccess) return (int)e;
     return (int)cudaGetLastError();
 }

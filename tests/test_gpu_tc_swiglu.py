@@ -135,3 +135,44 @@ def test_fused_swiglu_short_chunks(C):
     gp, hd = util.gpu_forward(x, **shape)
     assert E.e2ttt_device_status(hd["ws"]) == 0
     check_forward(gp, refp, TOL_BF16, f"fused SwiGLU, C = {C}, paper regime free-running")
+
+
+@pytest.mark.parametrize("C", [128, 512])
+def test_fused_swiglu_large_chunks(C):
+    """Chunks of 128 and 512 tokens as blocks of 64 at the chunk-start weights (asked for with impl = TCGEN05; AUTO keeps
+    the any-shape kernels above 64 tokens): one-chunk windows from the oracle's state, a free-running run under the
+    paper's gates with a ragged tail, split calls chain bitwise at a chunk boundary, and the training flow's memory
+    plans bit for bit.  Bounds: 2e-2 on the windows; the free-running run's momenta get 3x that (the sums of a long chunk
+    cancel while the bf16-sized errors of their terms do not; printed)."""
+    shape = dict(d=128, h=384, C=C, kind=SW, io="bf16")
+    r = inputs.config(3, heads=[3, 40], C=C)
+    xw, ref = util.teacher_forced_windows(r, 2, window=1)
+    got, hd = util.gpu_forward(xw, impl=E.E2TTT_IMPL_TCGEN05, **shape)
+    assert hd["ws"].numel() == 256 and E.e2ttt_device_status(hd["ws"]) == 0
+    print(C, "windows", check_forward(got, ref, TOL_BF16, f"fused SwiGLU, C = {C}, windows"))
+    L = 2 * C + 64 + 29
+    rp = inputs.paper_regime(inputs.Recipe(B=2, H=1, L=L, d=128, h=384, C=C, kind=SW, io="bf16", seed=6, m_std=0.002))
+    x = inputs.generate(rp, with_d_o=True, with_dstate=True)
+    refp = util.oracle_forward(x, C, SW)
+    gp, hd = util.gpu_forward(x, impl=E.E2TTT_IMPL_TCGEN05, **shape)
+    assert E.e2ttt_device_status(hd["ws"]) == 0
+    errs = {"o": util.rel_err(gp["o"], refp["o"])}
+    for i in range(3):
+        errs[f"W{i + 1}"] = util.rel_err(gp["W"][i], refp["W"][i])
+        errs[f"M{i + 1}"] = util.rel_err(gp["M"][i], refp["M"][i])
+    print(C, "free-running", errs)
+    assert all(v <= (3 * TOL_BF16 if n.startswith("M") else TOL_BF16) for n, v in errs.items()), errs
+    _, hauto = util.gpu_forward(x, **shape)
+    assert hauto["ws"].numel() > 256                                             # AUTO: the any-shape kernels
+    first = {n: (np.ascontiguousarray(v[:, :C]) if not isinstance(v, list) else v) for n, v in x.items()}
+    a, _ = util.gpu_forward(first, impl=E.E2TTT_IMPL_TCGEN05, **shape)
+    rest = {n: (np.ascontiguousarray(v[:, C:]) if not isinstance(v, list) else v) for n, v in x.items()}
+    rest["W"], rest["M"] = a["W"], a["M"]
+    b, _ = util.gpu_forward(rest, impl=E.E2TTT_IMPL_TCGEN05, **shape)
+    assert np.array_equal(np.concatenate([a["o"], b["o"]], 1), gp["o"])
+    for i in range(3):
+        assert np.array_equal(b["W"][i], gp["W"][i]) and np.array_equal(b["M"][i], gp["M"][i])
+    g1 = util.gpu_backward(x, via_saved_states=True, impl=E.E2TTT_IMPL_TCGEN05, **shape)
+    g2 = util.gpu_backward(x, via_saved_states=False, ckpt_every=2, impl=E.E2TTT_IMPL_TCGEN05, **shape)
+    for n in ("dq", "dk", "dv", "deta", "dbeta", "dgamma"):
+        assert np.array_equal(g1[n], g2[n]), n
