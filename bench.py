@@ -691,7 +691,8 @@ def main():
     ap.add_argument("--chunk", type=int, default=0, help="override the chunk size C of the configuration")
     ap.add_argument("--kernel", default="auto", choices=["auto", "fused", "tiled", "simt"],
                     help="kernel family of the forward: auto (the library's choice), fused (tensor-core kernel with the state on "
-                         "chip; the library's choice wherever it serves the shape), tiled / simt (any-shape kernels)")
+                         "chip; the library's choice wherever it serves the shape at up to 64 tokens per chunk; chunks of 128, 256, 512 "
+                         "tokens must ask for it), tiled / simt (any-shape kernels)")
     ap.add_argument("--gates", default="benchmark", choices=["benchmark", "paper"],
                     help="gate recipe: the benchmark's, or the paper's regime (eta_base 0.01, tau 32, alpha_base 0.1)")
     ap.add_argument("--preroll", type=float, default=1.2,
