@@ -241,7 +241,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 umma_commit_elect(&s.bar_g2, el);
                 PROF(3);
                 // G3: Pa = Pu W2c -> R1.  Needs every CTA's pu rows (bulk copies: async proxy, no proxy fence needed here) and
-                // the partial sums read out of R1 by all warps.
+                // the partial sums read out of R1 by all warps.  The instruction is M = 128 although pu has 64 token rows: an
+                // M = 64 instruction costs the same, so rows 64..127 of the A descriptor run on into whatever lies behind the
+                // pu slab, and lanes 64..127 of R1 receive values that nobody reads (the next writer of R1 starts afresh).
                 mbar_wait<true>(&s.bar_pu, ph, wc, 100 + 5);
                 PROF(13);
                 mbar_wait(&s.bar_r1, ph, wc, 100 + 6);

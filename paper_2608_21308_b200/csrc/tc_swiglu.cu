@@ -201,7 +201,7 @@ tc_swiglu_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 #pragma unroll kIssueUnroll
                 for (int k = 0; k < 4; ++k) umma_bf16_elect(tb + T_R1, dk(sb + oHd, 16384, k), dk(sb + oW3, 16384, k), id_kk, k > 0, el);
                 umma_commit_elect(&s.bar_g2, el);
-                // G3: Ph = Pu W3c -> R1 columns 0..63
+                // G3: Ph = Pu W3c -> R1 columns 0..63 (M = 128 costs what M = 64 costs: lanes 64..127 get values nobody reads)
                 mbar_wait<true>(&s.bar_pu, ph, wc, 300 + 5);
                 mbar_wait(&s.bar_r1, ph, wc, 300 + 6);
                 tc_fence_after_sync();
